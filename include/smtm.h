@@ -1,0 +1,194 @@
+/*
+ * smtm.h — C ABI of the SMTM semantic-memory hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, on one GPU, the per-exit-layer procedure of
+ * "Boosting Mobile CNN Inference through Semantic Memory" (arxiv 2112.02644):
+ *
+ *   Sec. 4.1        semantic vector = global average pooling of a feature map
+ *   Sec. 4.2 Eq. 1  cosine similarity against the semantic centres in fast memory
+ *   Sec. 4.2 Eq. 2  single-layer separability
+ *   Sec. 5   Eq. 3  cross-layer cumulative similarity, weights 2^(l-1)
+ *   Sec. 5   Eq. 4  accumulated confidence; exit when it exceeds the threshold
+ *   Sec. 6.1        frequency table and time-stamp table
+ *   Sec. 6.1 Eq. 5  replacement score, top-k members of the fast memory
+ *   Sec. 6.2 Eq. 6  adaptive fast-memory size at a confidence level
+ *   Sec. 6.3 Eq. 7  running-mean update of the semantic centres
+ *
+ * Conventions
+ *   d_*  device pointer on the current CUDA device, owned by the caller.
+ *   h_*  host pointer; read or written during the call, never retained.
+ *   stream  a cudaStream_t passed as void* (NULL = the default stream).
+ *   Calls that take a stream only enqueue work on it and return without
+ *   synchronising; their results are valid once the caller has synchronised
+ *   that stream.  Calls without a stream argument synchronise the device.
+ *   `layer` is 0-based in this interface; the paper's l is layer + 1, so the
+ *   weight of Eq. 3 is 2^layer.
+ *   Every function returns an smtm_status_t.  Arguments are checked on the host
+ *   before anything is launched; on an error nothing has been enqueued and no
+ *   output argument has been written.  The library never aborts, throws, or
+ *   traps on the device; a device-side bounded wait that gives up records
+ *   SMTM_ERR_TIMEOUT in a sticky status word read by smtm_cache_status.
+ *   A cache object is not thread-safe; distinct caches are independent.
+ */
+#ifndef SMTM_H
+#define SMTM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct smtm_cache smtm_cache_t; /* opaque; owns centres, tables, fast memories, scratch */
+
+typedef enum {
+    SMTM_OK = 0,
+    SMTM_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, value out of range */
+    SMTM_ERR_SHAPE = 2,       /* feature-map shape does not match the cache's layer */
+    SMTM_ERR_DTYPE = 3,       /* unknown dtype or layout code */
+    SMTM_ERR_ALIGN = 4,       /* a device buffer is not aligned as documented */
+    SMTM_ERR_ALLOC = 5,       /* device or host allocation failed */
+    SMTM_ERR_CUDA = 6,        /* a CUDA runtime call failed */
+    SMTM_ERR_STATE = 7,       /* call not valid in the cache's current state */
+    SMTM_ERR_TIMEOUT = 8      /* a bounded device-side wait gave up */
+} smtm_status_t;
+
+enum { SMTM_F32 = 0, SMTM_F16 = 1, SMTM_BF16 = 2 }; /* feature-map element types */
+enum { SMTM_NCHW = 0, SMTM_NHWC = 1 };              /* feature-map layouts */
+enum { SMTM_MAX_LAYERS = 16 };
+enum { SMTM_MAX_CLASSES = 8192 };
+
+/* Counter slots returned by smtm_cache_get_counters. */
+enum {
+    SMTM_CTR_EXITS = 0,                           /* [0, MAX_LAYERS): exits taken at each layer */
+    SMTM_CTR_NEAR = SMTM_MAX_LAYERS,              /* lookups with |AC - tau| <= 1e-4 */
+    SMTM_CTR_LOOKUPS = SMTM_MAX_LAYERS + 1,       /* frames scored (not yet exited) over all layers */
+    SMTM_CTR_COUNT = SMTM_MAX_LAYERS + 2
+};
+
+typedef struct {
+    int32_t n_classes;      /* n: classes in global memory (Sec. 6), 1..SMTM_MAX_CLASSES */
+    int32_t n_layers;       /* L: candidate exit layers (Sec. 4.2), 1..SMTM_MAX_LAYERS */
+    const int32_t* dims;    /* h_ [L] C_l = length of the semantic vector at layer l (Sec. 4.1) */
+    const float* tau;       /* h_ [L] exit thresholds; the paper's single tau = all equal (Sec. 5) */
+    int32_t n_streams;      /* S: independent fast memories (1 = the paper's single video stream) */
+    int32_t k_init;         /* initial fast-memory size, k_min <= k_init <= k_max */
+    int32_t k_min, k_max;   /* bounds of the adaptive size, 1 <= k_min <= k_max <= n (Sec. 6.2) */
+    int32_t window_W;       /* W of Eq. 5, >= 1 */
+    int32_t cl_num, cl_den; /* confidence level of Eq. 6 as a fraction, e.g. 19/20 */
+    int32_t max_batch;      /* largest B any call will pass; sizes the library's scratch */
+    uint32_t flags;         /* reserved, must be 0 */
+} smtm_config_t;
+
+/* A batch of feature maps at one exit layer: dense, frame stride C*H*W elements,
+ * d_data aligned to 16 bytes.  NCHW: [B][C][H][W];  NHWC: [B][H][W][C]. */
+typedef struct {
+    const void* d_data;
+    int32_t dtype;  /* SMTM_F32 / SMTM_F16 / SMTM_BF16 */
+    int32_t layout; /* SMTM_NCHW / SMTM_NHWC */
+    int32_t B, C, H, W;
+} smtm_fmap_t;
+
+/* Per-batch carry across the exit layers of one inference; every array is a
+ * caller-owned device array.  Before the first layer of a batch the caller
+ * zeroes d_sa, d_done and d_exit_layer and sets d_pred to -1. */
+typedef struct {
+    int32_t B;
+    const int32_t* d_stream_id; /* [B] fast memory each frame looks up; NULL = all stream 0 */
+    float* d_sa;                /* [B][k_max] cumulative similarity per fast-memory slot (Eq. 3) */
+    uint8_t* d_done;            /* [B] 1 once a frame has exited; later lookups skip it, reading none of its map */
+    int32_t* d_exit_layer;      /* [B] 0 = not exited, else the paper's l in 1..L */
+    int32_t* d_pred;            /* [B] class of SA_H at the exit layer */
+    float* d_ac;                /* [B][L] accumulated confidence (Eq. 4) per evaluated layer; may be NULL */
+    float* d_sep;               /* [B][L] separability (Eq. 2) per evaluated layer; may be NULL */
+    int32_t* d_top;             /* [B][2] classes of SA_H, SA_SH at the last evaluated layer (-1 = none); may be NULL */
+    float* d_sv[SMTM_MAX_LAYERS]; /* [l] -> [B][C_l] semantic vectors, kept for Eq. 7; 16-byte aligned */
+} smtm_batch_t;
+
+/* Creates a cache on the current device.  h_centers[l] -> [n][C_l] fp32 initial
+ * semantic centres (the paper warms them up on training data, Sec. 5);
+ * h_counts[l] -> [n] their update counts m (Eq. 7), NULL = all 1;
+ * h_init_members -> [S][k_init] class ids initially in each fast memory,
+ * NULL = 0..k_init-1 for every stream.  Frequency and time-stamp tables start
+ * at zero (Sec. 6.1).  On success *out receives the cache. */
+smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_centers,
+                                const uint32_t* const* h_counts, const int32_t* h_init_members,
+                                smtm_cache_t** out);
+
+/* Frees the cache and everything it owns (synchronises the device). */
+smtm_status_t smtm_cache_destroy(smtm_cache_t* cache);
+
+/* Prepares the carry for a new batch of frames: d_sa = 0, d_done = 0,
+ * d_exit_layer = 0, d_pred = -1 (one kernel; d_ac/d_sep/d_top/d_sv untouched). */
+smtm_status_t smtm_batch_reset(smtm_cache_t* cache, const smtm_batch_t* batch, void* stream);
+
+/* Sec. 4.1.  d_sv[b][c] = mean over H x W of frame b, channel c, accumulated in
+ * fp32, for every frame with d_skip[b] == 0 (d_skip NULL = all frames); rows of
+ * skipped frames are not written and none of their map is read.
+ * d_sv_norm2 (may be NULL) receives the squared length of each written row.
+ * fmap->C must equal dims[layer]. */
+smtm_status_t smtm_encode(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t* fmap,
+                          const uint8_t* d_skip, float* d_sv, float* d_sv_norm2, void* stream);
+
+/* Sec. 5, one candidate exit layer, for every frame with d_done[b] == 0:
+ * encode (as smtm_encode, into batch->d_sv[layer]); Eq. 1 against the k members
+ * of the frame's fast memory; Eq. 3 into d_sa; top-1/top-2 (ties: lower class
+ * id first; NaN ranks last); Eq. 4 and Eq. 2 into d_ac/d_sep[b][layer]; exit
+ * when  SA_H > 0  and  SA_H - SA_SH > tau * max(SA_SH, 0)  (Eq. 4's AC > tau,
+ * division-free, evaluated in fp32), which sets d_done, d_exit_layer = layer+1
+ * and d_pred.  Fewer than two members never exit.  A zero-length vector has
+ * similarity 0 to everything. */
+smtm_status_t smtm_lookup_exit(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t* fmap,
+                               const smtm_batch_t* batch, void* stream);
+
+/* Sec. 6.1 tables and Eq. 7 centres for a finished batch.  The label of frame b
+ * is d_pred[b] if it exited, else d_fallback_label[b] (the full network's
+ * answer; -1 or a NULL array = no label); its stop layer is d_exit_layer[b] if it
+ * exited, else L.  Per stream, frames are applied in ascending b: FT[label] + 1
+ * (saturating at 2^20), TS[label] = 0, TS of every other class + 1.  For every
+ * class j and layer l0 the frames with label j and stop layer >= l0 are folded
+ * into the centre in ascending b:  SC = (SC m + sum SV) / (m + q), m += q. */
+smtm_status_t smtm_cache_update(smtm_cache_t* cache, const smtm_batch_t* batch,
+                                const int32_t* d_fallback_label, void* stream);
+
+/* Eq. 5 and Eq. 6 for every stream: Score_i = FT_i 0.25^floor(TS_i / W) (exact,
+ * floor clamped at 12); classes ranked by (score descending, id ascending); the
+ * new size is the smallest k in [k_min, k_max] whose k best scores sum to more
+ * than cl_num/cl_den of all scores (k_max if none); the fast memory becomes the
+ * first k of the ranking.  A stream whose scores are all zero is left as is. */
+smtm_status_t smtm_cache_resize(smtm_cache_t* cache, void* stream);
+
+/* One whole step from host memory: copies the L feature maps (h_maps[l], host,
+ * dtype/layout/shape as in fmaps[l] whose d_data is ignored) to the device,
+ * runs smtm_lookup_exit for layers 0..L-1, smtm_cache_update and, if
+ * do_resize, smtm_cache_resize, then copies the decisions back.  Synchronises
+ * `stream` before returning.  h_stream_id / h_fallback_label may be NULL as in
+ * the device calls; h_done [B], h_exit_layer [B], h_pred [B] receive the results.
+ * B <= max_batch.  Pinned host buffers make the copies asynchronous. */
+smtm_status_t smtm_step_host(smtm_cache_t* cache, const smtm_fmap_t* fmaps, const void* const* h_maps,
+                             const int32_t* h_stream_id, const int32_t* h_fallback_label,
+                             int32_t do_resize, uint8_t* h_done, int32_t* h_exit_layer,
+                             int32_t* h_pred, void* stream);
+
+/* State read-back (each synchronises the device). */
+smtm_status_t smtm_cache_get_members(smtm_cache_t* cache, int32_t* h_members /*[S][k_max]*/,
+                                     int32_t* h_k /*[S]*/);
+smtm_status_t smtm_cache_get_centers(smtm_cache_t* cache, int32_t layer, float* h_centers /*[n][C_l]*/,
+                                     uint32_t* h_counts /*[n], may be NULL*/);
+smtm_status_t smtm_cache_get_tables(smtm_cache_t* cache, int32_t* h_ft /*[S][n]*/,
+                                    int32_t* h_ts /*[S][n]*/);
+smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMTM_CTR_COUNT]*/);
+
+/* Number of kernels the library has launched on behalf of this cache so far. */
+smtm_status_t smtm_cache_get_launches(smtm_cache_t* cache, int64_t* h_out);
+
+/* Reads the sticky device status word (synchronises the device): SMTM_OK or
+ * the first device-side error recorded since creation. */
+smtm_status_t smtm_cache_status(smtm_cache_t* cache);
+
+const char* smtm_status_string(smtm_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SMTM_H */

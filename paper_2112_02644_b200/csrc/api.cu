@@ -1,0 +1,471 @@
+// C ABI of the SMTM library: argument checking, state ownership and launch planning.
+// Every step of the path runs in the kernels of encode.cu, lookup.cu and memory.cu.
+#include <new>
+#include <vector>
+
+#include "internal.h"
+
+using namespace smtm;
+
+struct smtm_cache {
+    int n, L, S, k_init, k_min, k_max, W, cl_num, cl_den, max_batch;
+    int dims[SMTM_MAX_LAYERS];
+    float tau[SMTM_MAX_LAYERS];
+    float* d_centers[SMTM_MAX_LAYERS];
+    float* d_cnorm[SMTM_MAX_LAYERS];
+    uint32_t* d_m[SMTM_MAX_LAYERS];
+    int32_t* d_ft;
+    int32_t* d_ts;
+    int32_t* d_members;
+    int32_t* d_k;
+    unsigned long long* d_counters;
+    int* d_status;
+    int device, sm_count;
+    int64_t launches;
+    // device-side carry and staging used only by smtm_step_host (allocated on first use)
+    bool host_ready;
+    smtm_batch_t hb;
+    int32_t* d_stream_id;
+    int32_t* d_fallback;
+    void* d_stage[SMTM_MAX_LAYERS];
+    size_t stage_bytes[SMTM_MAX_LAYERS];
+};
+
+namespace {
+
+#define SMTM_CUDA(call)                          \
+    do {                                         \
+        if ((call) != cudaSuccess) {             \
+            (void)cudaGetLastError();            \
+            return SMTM_ERR_CUDA;                \
+        }                                        \
+    } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <class T>
+cudaError_t dev_alloc(T** p, size_t count) {
+    return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
+}
+
+void free_all(smtm_cache* c) {
+    for (int l = 0; l < SMTM_MAX_LAYERS; ++l) {
+        cudaFree(c->d_centers[l]);
+        cudaFree(c->d_cnorm[l]);
+        cudaFree(c->d_m[l]);
+        cudaFree(c->d_stage[l]);
+        cudaFree(c->hb.d_sv[l]);
+    }
+    cudaFree(c->d_ft);
+    cudaFree(c->d_ts);
+    cudaFree(c->d_members);
+    cudaFree(c->d_k);
+    cudaFree(c->d_counters);
+    cudaFree(c->d_status);
+    cudaFree(c->hb.d_sa);
+    cudaFree(c->hb.d_done);
+    cudaFree(c->hb.d_exit_layer);
+    cudaFree(c->hb.d_pred);
+    cudaFree(c->d_stream_id);
+    cudaFree(c->d_fallback);
+    delete c;
+}
+
+smtm_status_t check_fmap(const smtm_cache* c, int32_t layer, const smtm_fmap_t* f) {
+    if (!c || !f) return SMTM_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= c->L) return SMTM_ERR_INVALID_ARG;
+    if (f->dtype < SMTM_F32 || f->dtype > SMTM_BF16 || f->layout < SMTM_NCHW || f->layout > SMTM_NHWC)
+        return SMTM_ERR_DTYPE;
+    if (f->B < 1 || f->B > c->max_batch || f->H < 1 || f->W < 1) return SMTM_ERR_SHAPE;
+    if (f->C != c->dims[layer]) return SMTM_ERR_SHAPE;
+    if ((long long)f->H * f->W > (1 << 24)) return SMTM_ERR_SHAPE;
+    return SMTM_OK;
+}
+
+smtm_status_t check_batch(const smtm_cache* c, const smtm_batch_t* b) {
+    if (!b) return SMTM_ERR_INVALID_ARG;
+    if (b->B < 1 || b->B > c->max_batch) return SMTM_ERR_SHAPE;
+    if (!b->d_sa || !b->d_done || !b->d_exit_layer || !b->d_pred) return SMTM_ERR_INVALID_ARG;
+    return SMTM_OK;
+}
+
+EncodeArgs encode_args(const smtm_cache* c, const smtm_fmap_t* f, const uint8_t* skip, float* sv) {
+    EncodeArgs e{};
+    e.x = f->d_data;
+    e.dtype = f->dtype;
+    e.layout = f->layout;
+    e.B = f->B;
+    e.C = f->C;
+    e.H = f->H;
+    e.W = f->W;
+    e.skip = skip;
+    e.sv = sv;
+    e.status = c->d_status;
+    return e;
+}
+
+smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b,
+                          cudaStream_t st) {
+    SMTM_CUDA(launch_encode(encode_args(c, f, b->d_done, b->d_sv[layer]), c->sm_count, st, &c->launches));
+    LookupArgs a{};
+    a.layer = layer;
+    a.L = c->L;
+    a.B = f->B;
+    a.D = f->C;
+    a.n = c->n;
+    a.k_max = c->k_max;
+    a.tau = c->tau[layer];
+    a.sv = b->d_sv[layer];
+    a.centers = c->d_centers[layer];
+    a.cnorm = c->d_cnorm[layer];
+    a.stream_id = b->d_stream_id;
+    a.members = c->d_members;
+    a.k = c->d_k;
+    a.sa = b->d_sa;
+    a.done = b->d_done;
+    a.exit_layer = b->d_exit_layer;
+    a.pred = b->d_pred;
+    a.ac = b->d_ac;
+    a.sep = b->d_sep;
+    a.top = b->d_top;
+    a.counters = c->d_counters;
+    SMTM_CUDA(launch_score_exit(a, st, &c->launches));
+    return SMTM_OK;
+}
+
+smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d_fallback, cudaStream_t st) {
+    UpdateArgs a{};
+    a.B = b->B;
+    a.S = c->S;
+    a.n = c->n;
+    a.L = c->L;
+    a.stream_id = b->d_stream_id;
+    a.done = b->d_done;
+    a.exit_layer = b->d_exit_layer;
+    a.pred = b->d_pred;
+    a.fallback = d_fallback;
+    a.ft = c->d_ft;
+    a.ts = c->d_ts;
+    for (int l = 0; l < c->L; ++l) {
+        a.dims[l] = c->dims[l];
+        a.sv[l] = b->d_sv[l];
+        a.centers[l] = c->d_centers[l];
+        a.cnorm[l] = c->d_cnorm[l];
+        a.m[l] = c->d_m[l];
+    }
+    SMTM_CUDA(launch_update(a, st, &c->launches));
+    return SMTM_OK;
+}
+
+smtm_status_t resize_impl(smtm_cache* c, cudaStream_t st) {
+    ResizeArgs a{};
+    a.S = c->S;
+    a.n = c->n;
+    a.W = c->W;
+    a.k_min = c->k_min;
+    a.k_max = c->k_max;
+    a.cl_num = c->cl_num;
+    a.cl_den = c->cl_den;
+    a.ft = c->d_ft;
+    a.ts = c->d_ts;
+    a.members = c->d_members;
+    a.k = c->d_k;
+    SMTM_CUDA(launch_resize(a, st, &c->launches));
+    return SMTM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_centers,
+                                const uint32_t* const* h_counts, const int32_t* h_init_members,
+                                smtm_cache_t** out) {
+    if (!cfg || !h_centers || !out || !cfg->dims || !cfg->tau) return SMTM_ERR_INVALID_ARG;
+    if (cfg->n_classes < 1 || cfg->n_classes > SMTM_MAX_CLASSES) return SMTM_ERR_INVALID_ARG;
+    if (cfg->n_layers < 1 || cfg->n_layers > SMTM_MAX_LAYERS) return SMTM_ERR_INVALID_ARG;
+    if (cfg->n_streams < 1 || cfg->max_batch < 1 || cfg->flags != 0) return SMTM_ERR_INVALID_ARG;
+    if (cfg->k_min < 1 || cfg->k_min > cfg->k_init || cfg->k_init > cfg->k_max || cfg->k_max > cfg->n_classes)
+        return SMTM_ERR_INVALID_ARG;
+    if (cfg->window_W < 1 || cfg->cl_den < 1 || cfg->cl_num < 0 || cfg->cl_num > cfg->cl_den ||
+        cfg->cl_den > 1024)
+        return SMTM_ERR_INVALID_ARG;
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        if (cfg->dims[l] < 1 || cfg->dims[l] > (1 << 20) || !h_centers[l]) return SMTM_ERR_INVALID_ARG;
+        if (cfg->tau[l] != cfg->tau[l]) return SMTM_ERR_INVALID_ARG;  // NaN
+    }
+    const int n = cfg->n_classes, S = cfg->n_streams;
+    if (h_init_members)
+        for (long long i = 0; i < (long long)S * cfg->k_init; ++i)
+            if (h_init_members[i] < 0 || h_init_members[i] >= n) return SMTM_ERR_INVALID_ARG;
+
+    smtm_cache* c = new (std::nothrow) smtm_cache();
+    if (!c) return SMTM_ERR_ALLOC;
+    c->n = n;
+    c->L = cfg->n_layers;
+    c->S = S;
+    c->k_init = cfg->k_init;
+    c->k_min = cfg->k_min;
+    c->k_max = cfg->k_max;
+    c->W = cfg->window_W;
+    c->cl_num = cfg->cl_num;
+    c->cl_den = cfg->cl_den;
+    c->max_batch = cfg->max_batch;
+    for (int l = 0; l < c->L; ++l) {
+        c->dims[l] = cfg->dims[l];
+        c->tau[l] = cfg->tau[l];
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&c->device) != cudaSuccess || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete c;
+        return SMTM_ERR_CUDA;
+    }
+    c->sm_count = prop.multiProcessorCount;
+    if (prop.major < 10) {  // the kernels are built for sm_100a only
+        delete c;
+        return SMTM_ERR_CUDA;
+    }
+
+    bool ok = encode_setup() == cudaSuccess;
+    for (int l = 0; ok && l < c->L; ++l) {
+        const size_t nd = size_t(n) * c->dims[l];
+        ok = ok && dev_alloc(&c->d_centers[l], nd) == cudaSuccess;
+        ok = ok && dev_alloc(&c->d_cnorm[l], n) == cudaSuccess;
+        ok = ok && dev_alloc(&c->d_m[l], n) == cudaSuccess;
+    }
+    ok = ok && dev_alloc(&c->d_ft, size_t(S) * n) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_ts, size_t(S) * n) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_members, size_t(S) * c->k_max) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_k, S) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_counters, SMTM_CTR_COUNT) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_status, 1) == cudaSuccess;
+    if (!ok) {
+        (void)cudaGetLastError();
+        free_all(c);
+        return SMTM_ERR_ALLOC;
+    }
+
+    std::vector<int32_t> members(size_t(S) * c->k_max, 0), ks(S, c->k_init);
+    std::vector<uint32_t> ones(n, 1u);
+    for (int s = 0; s < S; ++s)
+        for (int j = 0; j < c->k_max; ++j) {
+            int32_t v = j % n;
+            if (j < c->k_init && h_init_members) v = h_init_members[size_t(s) * c->k_init + j];
+            members[size_t(s) * c->k_max + j] = v;
+        }
+    cudaError_t e = cudaSuccess;
+    for (int l = 0; e == cudaSuccess && l < c->L; ++l) {
+        const size_t nd = size_t(n) * c->dims[l];
+        e = cudaMemcpy(c->d_centers[l], h_centers[l], nd * sizeof(float), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(c->d_m[l], (h_counts && h_counts[l]) ? h_counts[l] : ones.data(), n * sizeof(uint32_t),
+                           cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = launch_center_norms(c->d_centers[l], n, c->dims[l], c->d_cnorm[l], 0, &c->launches);
+    }
+    if (e == cudaSuccess) e = cudaMemset(c->d_ft, 0, size_t(S) * n * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(c->d_ts, 0, size_t(S) * n * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(c->d_counters, 0, SMTM_CTR_COUNT * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
+    if (e == cudaSuccess)
+        e = cudaMemcpy(c->d_members, members.data(), members.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(c->d_k, ks.data(), ks.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        free_all(c);
+        return SMTM_ERR_CUDA;
+    }
+    *out = c;
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_destroy(smtm_cache_t* c) {
+    if (!c) return SMTM_ERR_INVALID_ARG;
+    (void)cudaDeviceSynchronize();
+    free_all(c);
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_batch_reset(smtm_cache_t* c, const smtm_batch_t* b, void* stream) {
+    if (!c) return SMTM_ERR_INVALID_ARG;
+    smtm_status_t s = check_batch(c, b);
+    if (s != SMTM_OK) return s;
+    SMTM_CUDA(launch_batch_reset(b->d_sa, b->d_done, b->d_exit_layer, b->d_pred, b->B, c->k_max,
+                                 static_cast<cudaStream_t>(stream), &c->launches));
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_encode(smtm_cache_t* c, int32_t layer, const smtm_fmap_t* f, const uint8_t* d_skip, float* d_sv,
+                          float* d_sv_norm2, void* stream) {
+    smtm_status_t s = check_fmap(c, layer, f);
+    if (s != SMTM_OK) return s;
+    if (!f->d_data || !d_sv) return SMTM_ERR_INVALID_ARG;
+    if (!aligned16(f->d_data) || !aligned16(d_sv)) return SMTM_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SMTM_CUDA(launch_encode(encode_args(c, f, d_skip, d_sv), c->sm_count, st, &c->launches));
+    if (d_sv_norm2) SMTM_CUDA(launch_row_norm2(d_sv, d_skip, f->B, f->C, d_sv_norm2, st, &c->launches));
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_lookup_exit(smtm_cache_t* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b,
+                               void* stream) {
+    smtm_status_t s = check_fmap(c, layer, f);
+    if (s != SMTM_OK) return s;
+    if ((s = check_batch(c, b)) != SMTM_OK) return s;
+    if (b->B != f->B) return SMTM_ERR_SHAPE;
+    if (!f->d_data || !b->d_sv[layer]) return SMTM_ERR_INVALID_ARG;
+    if (!aligned16(f->d_data) || !aligned16(b->d_sv[layer])) return SMTM_ERR_ALIGN;
+    return lookup_impl(c, layer, f, b, static_cast<cudaStream_t>(stream));
+}
+
+smtm_status_t smtm_cache_update(smtm_cache_t* c, const smtm_batch_t* b, const int32_t* d_fallback_label,
+                                void* stream) {
+    if (!c) return SMTM_ERR_INVALID_ARG;
+    smtm_status_t s = check_batch(c, b);
+    if (s != SMTM_OK) return s;
+    for (int l = 0; l < c->L; ++l)
+        if (!b->d_sv[l]) return SMTM_ERR_INVALID_ARG;
+    return update_impl(c, b, d_fallback_label, static_cast<cudaStream_t>(stream));
+}
+
+smtm_status_t smtm_cache_resize(smtm_cache_t* c, void* stream) {
+    if (!c) return SMTM_ERR_INVALID_ARG;
+    return resize_impl(c, static_cast<cudaStream_t>(stream));
+}
+
+smtm_status_t smtm_step_host(smtm_cache_t* c, const smtm_fmap_t* fmaps, const void* const* h_maps,
+                             const int32_t* h_stream_id, const int32_t* h_fallback_label, int32_t do_resize,
+                             uint8_t* h_done, int32_t* h_exit_layer, int32_t* h_pred, void* stream) {
+    if (!c || !fmaps || !h_maps || !h_done || !h_exit_layer || !h_pred) return SMTM_ERR_INVALID_ARG;
+    const int B = fmaps[0].B;
+    for (int l = 0; l < c->L; ++l) {
+        smtm_status_t s = check_fmap(c, l, &fmaps[l]);
+        if (s != SMTM_OK) return s;
+        if (fmaps[l].B != B) return SMTM_ERR_SHAPE;
+        if (!h_maps[l]) return SMTM_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t mb = size_t(c->max_batch);
+    if (!c->host_ready) {  // first use: allocate the device-side carry
+        bool ok = dev_alloc(&c->hb.d_sa, mb * c->k_max) == cudaSuccess;
+        ok = ok && dev_alloc(&c->hb.d_done, mb) == cudaSuccess;
+        ok = ok && dev_alloc(&c->hb.d_exit_layer, mb) == cudaSuccess;
+        ok = ok && dev_alloc(&c->hb.d_pred, mb) == cudaSuccess;
+        ok = ok && dev_alloc(&c->d_stream_id, mb) == cudaSuccess;
+        ok = ok && dev_alloc(&c->d_fallback, mb) == cudaSuccess;
+        for (int l = 0; ok && l < c->L; ++l) ok = dev_alloc(&c->hb.d_sv[l], mb * c->dims[l]) == cudaSuccess;
+        if (!ok) {
+            (void)cudaGetLastError();
+            return SMTM_ERR_ALLOC;
+        }
+        c->host_ready = true;
+    }
+    for (int l = 0; l < c->L; ++l) {
+        const size_t need = size_t(B) * fmaps[l].C * fmaps[l].H * fmaps[l].W * (fmaps[l].dtype == SMTM_F32 ? 4 : 2);
+        if (need > c->stage_bytes[l]) {
+            (void)cudaStreamSynchronize(st);
+            cudaFree(c->d_stage[l]);
+            c->d_stage[l] = nullptr;
+            c->stage_bytes[l] = 0;
+            if (cudaMalloc(&c->d_stage[l], need) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return SMTM_ERR_ALLOC;
+            }
+            c->stage_bytes[l] = need;
+        }
+    }
+    smtm_batch_t b = c->hb;
+    b.B = B;
+    b.d_stream_id = nullptr;
+    b.d_ac = nullptr;
+    b.d_sep = nullptr;
+    b.d_top = nullptr;
+    SMTM_CUDA(launch_batch_reset(b.d_sa, b.d_done, b.d_exit_layer, b.d_pred, B, c->k_max, st, &c->launches));
+    if (h_stream_id) {
+        SMTM_CUDA(cudaMemcpyAsync(c->d_stream_id, h_stream_id, size_t(B) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+        b.d_stream_id = c->d_stream_id;
+    }
+    if (h_fallback_label)
+        SMTM_CUDA(cudaMemcpyAsync(c->d_fallback, h_fallback_label, size_t(B) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    for (int l = 0; l < c->L; ++l) {
+        smtm_fmap_t f = fmaps[l];
+        const size_t bytes = size_t(B) * f.C * f.H * f.W * (f.dtype == SMTM_F32 ? 4 : 2);
+        SMTM_CUDA(cudaMemcpyAsync(c->d_stage[l], h_maps[l], bytes, cudaMemcpyHostToDevice, st));
+        f.d_data = c->d_stage[l];
+        smtm_status_t s = lookup_impl(c, l, &f, &b, st);
+        if (s != SMTM_OK) return s;
+    }
+    smtm_status_t s = update_impl(c, &b, h_fallback_label ? c->d_fallback : nullptr, st);
+    if (s != SMTM_OK) return s;
+    if (do_resize && (s = resize_impl(c, st)) != SMTM_OK) return s;
+    SMTM_CUDA(cudaMemcpyAsync(h_done, b.d_done, size_t(B), cudaMemcpyDeviceToHost, st));
+    SMTM_CUDA(cudaMemcpyAsync(h_exit_layer, b.d_exit_layer, size_t(B) * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    SMTM_CUDA(cudaMemcpyAsync(h_pred, b.d_pred, size_t(B) * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    SMTM_CUDA(cudaStreamSynchronize(st));
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_get_members(smtm_cache_t* c, int32_t* h_members, int32_t* h_k) {
+    if (!c || !h_members || !h_k) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    SMTM_CUDA(cudaMemcpy(h_members, c->d_members, size_t(c->S) * c->k_max * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    SMTM_CUDA(cudaMemcpy(h_k, c->d_k, size_t(c->S) * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_get_centers(smtm_cache_t* c, int32_t layer, float* h_centers, uint32_t* h_counts) {
+    if (!c || !h_centers || layer < 0 || layer >= c->L) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    SMTM_CUDA(cudaMemcpy(h_centers, c->d_centers[layer], size_t(c->n) * c->dims[layer] * sizeof(float),
+                         cudaMemcpyDeviceToHost));
+    if (h_counts)
+        SMTM_CUDA(cudaMemcpy(h_counts, c->d_m[layer], size_t(c->n) * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_get_tables(smtm_cache_t* c, int32_t* h_ft, int32_t* h_ts) {
+    if (!c || !h_ft || !h_ts) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    SMTM_CUDA(cudaMemcpy(h_ft, c->d_ft, size_t(c->S) * c->n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    SMTM_CUDA(cudaMemcpy(h_ts, c->d_ts, size_t(c->S) * c->n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_get_counters(smtm_cache_t* c, int64_t* h_out) {
+    if (!c || !h_out) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    SMTM_CUDA(cudaMemcpy(h_out, c->d_counters, SMTM_CTR_COUNT * sizeof(int64_t), cudaMemcpyDeviceToHost));
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_get_launches(smtm_cache_t* c, int64_t* h_out) {
+    if (!c || !h_out) return SMTM_ERR_INVALID_ARG;
+    *h_out = c->launches;
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_status(smtm_cache_t* c) {
+    if (!c) return SMTM_ERR_INVALID_ARG;
+    int v = 0;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    SMTM_CUDA(cudaMemcpy(&v, c->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+    return static_cast<smtm_status_t>(v);
+}
+
+const char* smtm_status_string(smtm_status_t s) {
+    switch (s) {
+        case SMTM_OK: return "ok";
+        case SMTM_ERR_INVALID_ARG: return "invalid argument";
+        case SMTM_ERR_SHAPE: return "shape mismatch";
+        case SMTM_ERR_DTYPE: return "unknown dtype or layout";
+        case SMTM_ERR_ALIGN: return "misaligned device buffer";
+        case SMTM_ERR_ALLOC: return "allocation failed";
+        case SMTM_ERR_CUDA: return "CUDA runtime error";
+        case SMTM_ERR_STATE: return "invalid state";
+        case SMTM_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,80 @@
+// Host-side declarations shared by the translation units of the SMTM library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/smtm.h"
+
+namespace smtm {
+
+// ---- encode (Sec. 4.1) ------------------------------------------------------------------
+struct EncodeArgs {
+    const void* x;        // device, 16-byte aligned
+    int dtype, layout;
+    int B, C, H, W;
+    const uint8_t* skip;  // device [B] or nullptr
+    float* sv;            // device [B][C]
+    int* status;          // device sticky status word
+};
+// Enqueues the pooling of every non-skipped frame.  *launches is incremented per kernel launched.
+cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches);
+// Opt-in to large dynamic shared memory for the kernels that need it (once per device).
+cudaError_t encode_setup();
+cudaError_t launch_row_norm2(const float* sv, const uint8_t* skip, int B, int D, float* out, cudaStream_t st,
+                             int64_t* launches);
+
+// ---- lookup (Sec. 4.2, Sec. 5) -------------------------------------------------------------
+struct LookupArgs {
+    int layer, L, B, D, n, k_max;
+    float tau;
+    const float* sv;          // [B][D]
+    const float* centers;     // [n][D]
+    const float* cnorm;       // [n] lengths of the centres
+    const int32_t* stream_id; // [B] or nullptr
+    const int32_t* members;   // [S][k_max]
+    const int32_t* k;         // [S]
+    float* sa;                // [B][k_max]
+    uint8_t* done;
+    int32_t* exit_layer;
+    int32_t* pred;
+    float* ac;                // [B][L] or nullptr
+    float* sep;               // [B][L] or nullptr
+    int32_t* top;             // [B][2] or nullptr
+    unsigned long long* counters;
+};
+cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches);
+cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,
+                               cudaStream_t st, int64_t* launches);
+
+// ---- memory maintenance (Sec. 6) -------------------------------------------------------------
+cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm, cudaStream_t st,
+                                int64_t* launches);
+
+struct UpdateArgs {
+    int B, S, n, L;
+    const int32_t* stream_id;  // [B] or nullptr
+    const uint8_t* done;
+    const int32_t* exit_layer;
+    const int32_t* pred;
+    const int32_t* fallback;   // [B] or nullptr
+    int32_t* ft;               // [S][n]
+    int32_t* ts;               // [S][n]
+    int dims[SMTM_MAX_LAYERS];
+    const float* sv[SMTM_MAX_LAYERS];
+    float* centers[SMTM_MAX_LAYERS];
+    float* cnorm[SMTM_MAX_LAYERS];
+    uint32_t* m[SMTM_MAX_LAYERS];
+};
+cudaError_t launch_update(const UpdateArgs& a, cudaStream_t st, int64_t* launches);
+
+struct ResizeArgs {
+    int S, n, W, k_min, k_max, cl_num, cl_den;
+    const int32_t* ft;
+    const int32_t* ts;
+    int32_t* members;  // [S][k_max]
+    int32_t* k;        // [S]
+};
+cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches);
+
+}  // namespace smtm

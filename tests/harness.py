@@ -1,0 +1,164 @@
+"""Runs a synthetic workload through the CUDA library and the CPU oracle side by side.
+
+Both sides see the same bytes: the feature maps are generated once (on the GPU),
+handed to the library by device pointer and copied to the host for the oracle.
+Decisions are compared layer by layer; a frame whose decision differs must lie in
+the near-threshold band (|AC - tau| <= 1e-4), is counted, and the oracle is re-run
+for that layer with the library's decision imposed so that the states stay comparable.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+import oracle
+import paper_2112_02644_b200 as smtm
+import smtm_inputs as si
+
+SV_RTOL = 1e-5       # semantic vectors, relative to the channel's mean |x|
+SCORE_ATOL = 1e-5    # cosines live in [-1, 1]
+CENTER_RTOL = 2e-5
+
+
+@dataclass
+class Report:
+    frames: int = 0
+    lookups: int = 0
+    exits: list = field(default_factory=list)
+    band_mismatches: int = 0
+    near_oracle: int = 0
+    max_sv_err: float = 0.0
+    max_sa_err: float = 0.0
+    max_center_err: float = 0.0
+
+
+def make_pair(w: si.Workload, max_batch=None):
+    cents, counts = si.initial_centers(w)
+    tau = [w.tau] * w.L
+    mem = oracle.OracleMemory(w.n, w.dims, tau, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W)
+    cache = smtm.smtm_cache_create(w.n, w.dims, tau, cents, counts, n_streams=w.S, k_init=w.k_init, k_min=w.k_min,
+                                   k_max=w.k_max, window_W=w.window_W, max_batch=max_batch or w.B)
+    return cache, mem
+
+
+def abs_mean_scale(x: torch.Tensor, w: si.Workload, layer: int) -> np.ndarray:
+    """Mean |x| per (frame, channel): the scale the fp32 summation error is relative to."""
+    axes = (2, 3) if w.layout == si.NCHW else (1, 2)
+    return x.float().abs().mean(dim=axes).cpu().numpy().astype(np.float64)
+
+
+def compare_layer(w, layer, x, gb, ob, todo, rep: Report):
+    """Element-wise comparison of everything one lookup produced for the frames in ``todo``."""
+    sv_g = gb.sv[layer].cpu().numpy().astype(np.float64)
+    sv_o = ob["sv"][layer]
+    scale = np.maximum(abs_mean_scale(x, w, layer), 1e-30)
+    err = np.abs(sv_g - sv_o)[todo] / scale[todo]
+    rep.max_sv_err = max(rep.max_sv_err, float(err.max(initial=0.0)))
+    assert err.max(initial=0.0) <= SV_RTOL, f"semantic vectors off by {err.max():.3g} (relative) at layer {layer}"
+    # cumulative similarity: weights add up to 2^(layer+1) - 1, each cosine within SCORE_ATOL
+    sa_g = gb.sa.cpu().numpy().astype(np.float64)
+    sa_err = np.abs(sa_g - ob["sa"])[todo]
+    rep.max_sa_err = max(rep.max_sa_err, float(sa_err.max(initial=0.0)))
+    assert sa_err.max(initial=0.0) <= SCORE_ATOL * (2 ** (layer + 1) - 1), f"cumulative similarity off by {sa_err.max():.3g}"
+    # accumulated confidence and separability where the ratio is well conditioned
+    ac_g = gb.ac.cpu().numpy().astype(np.float64)[:, layer]
+    ac_o = ob["ac"][:, layer]
+    sep_g = gb.sep.cpu().numpy().astype(np.float64)[:, layer]
+    sep_o = ob["sep"][:, layer]
+    for g, o in ((ac_g, ac_o), (sep_g, sep_o)):
+        fin = todo & np.isfinite(o) & np.isfinite(g) & (np.abs(o) < 5.0)
+        assert np.all(np.abs(g[fin] - o[fin]) <= 2e-3 * (1 + np.abs(o[fin]))), "AC / separability mismatch"
+    # top-1 class wherever the oracle's lead is clear of rounding
+    top_g = gb.top.cpu().numpy()
+    sa_sorted = np.sort(np.where(np.isnan(ob["sa"]), -np.inf, ob["sa"]), axis=1)
+    if sa_sorted.shape[1] >= 2:
+        clear = todo & ((sa_sorted[:, -1] - sa_sorted[:, -2]) > 1e-4)
+        assert np.array_equal(top_g[clear, 0], ob["top"][clear, 0]), "top-1 class differs"
+
+
+def step_pair(w, cache, mem, gb, lab, step, rep: Report, device="cuda", compare_values=True):
+    """One step on both sides, compared layer by layer.  Returns the oracle's batch."""
+    sid = si.stream_ids(w) if w.S > 1 else None
+    ob = mem.new_batch(w.B, sid)
+    smtm.smtm_batch_reset(cache, gb)
+    fb = si.fallback_labels(w, lab)
+    for l in range(w.L):
+        x = si.frames(w, l, lab, step, device=device)
+        B, C, H, W = si.shape4(w, l)
+        todo = ob["done"] == 0
+        smtm.smtm_lookup_exit(cache, l, smtm.Fmap(x, w.dtype, w.layout, B, C, H, W), gb)
+        torch.cuda.synchronize()
+        snap = {k: ob[k].copy() for k in ("sa", "done", "exit_layer", "pred")}
+        xh = x.cpu()
+        mem_exits, mem_near = mem.exits_per_layer.copy(), mem.near_count
+        mem.lookup_exit(l, xh, w.dtype, w.layout, (B, C, H, W), ob)
+        done_g = gb.done.cpu().numpy()
+        diff = np.nonzero(done_g != ob["done"])[0]
+        if diff.size:
+            ac_g = gb.ac.cpu().numpy()[:, l]
+            in_band = (ob["near"][diff, l] == 1) | (np.abs(ac_g[diff] - np.float32(w.tau)) <= 1e-4)
+            assert in_band.all(), f"decision mismatch outside the 1e-4 band at layer {l}: frames {diff[~in_band][:8]}"
+            rep.band_mismatches += int(diff.size)
+            for k, v in snap.items():
+                ob[k][...] = v
+            mem.exits_per_layer[:] = mem_exits
+            mem.near_count = mem_near
+            force = np.full(w.B, -1, np.int8)
+            force[diff] = done_g[diff]
+            mem.lookup_exit(l, xh, w.dtype, w.layout, (B, C, H, W), ob, force=force)
+        assert np.array_equal(done_g, ob["done"])
+        assert np.array_equal(gb.exit_layer.cpu().numpy(), ob["exit_layer"])
+        # predicted labels are bit-exact wherever a frame exited
+        ex = ob["done"] == 1
+        assert np.array_equal(gb.pred.cpu().numpy()[ex], ob["pred"][ex])
+        if compare_values:
+            compare_layer(w, l, x, gb, ob, todo, rep)
+        rep.lookups += int(todo.sum())
+        del x
+    fb_d = torch.from_numpy(fb).to(device)
+    smtm.smtm_cache_update(cache, gb, fb_d)
+    smtm.smtm_cache_resize(cache)
+    mem.update(ob, fb)
+    mem.resize()
+    rep.frames += w.B
+    rep.near_oracle = mem.near_count
+    return ob
+
+
+def compare_state(w, cache, mem, rep: Report):
+    """Tables, counts, fast memories bit-exact; centres within rounding."""
+    ft, ts = smtm.smtm_cache_get_tables(cache)
+    assert np.array_equal(ft, mem.ft), "frequency table differs"
+    assert np.array_equal(ts, mem.ts), "time-stamp table differs"
+    members, k = smtm.smtm_cache_get_members(cache)
+    assert np.array_equal(k, mem.k), "fast-memory sizes differ"
+    assert np.array_equal(members, mem.members), "fast-memory members differ"
+    for l in range(w.L):
+        cen, m = smtm.smtm_cache_get_centers(cache, l)
+        assert np.array_equal(m, mem.m[l]), "update counts differ"
+        scale = np.maximum(np.abs(mem.centers[l]), np.abs(mem.centers[l]).mean(axis=1, keepdims=True))
+        err = np.abs(cen.astype(np.float64) - mem.centers[l]) / np.maximum(scale, 1e-30)
+        rep.max_center_err = max(rep.max_center_err, float(err.max()))
+        assert err.max() <= CENTER_RTOL, f"centres off by {err.max():.3g} at layer {l}"
+    assert smtm.smtm_cache_status(cache) == 0, "device status word set"
+
+
+def run_workload(w: si.Workload, steps=None, device="cuda", compare_values=True, state_every=1) -> Report:
+    cache, mem = make_pair(w)
+    rep = Report()
+    labs = si.labels(w)
+    sid = si.stream_ids(w) if w.S > 1 else None
+    gb = smtm.Batch(cache, w.B, stream_id=sid, device=device)
+    T = w.T if steps is None else steps
+    for t in range(T):
+        step_pair(w, cache, mem, gb, labs[t], t, rep, device, compare_values)
+        if (t + 1) % state_every == 0 or t == T - 1:
+            compare_state(w, cache, mem, rep)
+    ctr = smtm.smtm_cache_get_counters(cache)
+    rep.exits = [int(v) for v in ctr[: w.L]]
+    assert rep.exits == [int(v) for v in mem.exits_per_layer], (rep.exits, mem.exits_per_layer)
+    assert int(ctr[smtm.CTR_LOOKUPS]) == rep.lookups
+    smtm.smtm_cache_destroy(cache)
+    return rep

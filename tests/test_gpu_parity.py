@@ -1,0 +1,202 @@
+"""CUDA library vs CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2112_02644_b200 as smtm
+import smtm_inputs as si
+from harness import run_workload
+
+pytestmark = pytest.mark.gpu
+
+TORCH_DT = {si.F32: torch.float32, si.F16: torch.float16, si.BF16: torch.bfloat16}
+
+
+def dummy_cache(C, n=4, max_batch=4096):
+    cen = [np.ones((n, C), np.float32)]
+    return smtm.smtm_cache_create(n, [C], [0.8], cen, k_init=2, k_min=2, k_max=n, max_batch=max_batch)
+
+
+# ---------------------------------------------------------------------------- encode
+
+ENCODE_SHAPES = [
+    # (dtype, layout, B, C, H, W): the five workloads' stages, ragged channel counts, odd shapes
+    (si.F32, si.NCHW, 8, 64, 56, 56),
+    (si.BF16, si.NCHW, 5, 256, 56, 56), (si.BF16, si.NCHW, 5, 512, 28, 28),
+    (si.BF16, si.NCHW, 7, 1024, 14, 14), (si.BF16, si.NCHW, 9, 2048, 7, 7),
+    (si.BF16, si.NCHW, 3, 2048 + 8 * 5, 7, 7),      # ragged last chunk, unit-per-lane
+    (si.BF16, si.NCHW, 3, 70, 14, 14), (si.F16, si.NCHW, 3, 24, 7, 7), (si.F32, si.NCHW, 3, 36, 7, 7),
+    (si.F16, si.NCHW, 2, 33, 28, 28),               # ragged, team-per-channel
+    (si.F32, si.NCHW, 2, 5, 2, 2), (si.F32, si.NCHW, 2, 3, 112, 112),  # 16-byte channels; channel > one stage
+    (si.BF16, si.NCHW, 2, 7, 5, 3), (si.F16, si.NCHW, 1, 1, 1, 1),     # nothing aligned: plain path
+    (si.F16, si.NHWC, 6, 24, 56, 56), (si.F16, si.NHWC, 6, 32, 28, 28),
+    (si.F16, si.NHWC, 6, 96, 14, 14), (si.F16, si.NHWC, 6, 320, 7, 7),
+    (si.BF16, si.NHWC, 2, 4096, 3, 3), (si.F32, si.NHWC, 3, 20, 9, 5), (si.F16, si.NHWC, 3, 12, 4, 4),
+    (si.F32, si.NHWC, 2, 7, 3, 3),
+]
+
+
+@pytest.mark.parametrize("dt,layout,B,C,H,W", ENCODE_SHAPES)
+def test_encode_matches_oracle(dt, layout, B, C, H, W):
+    g = torch.Generator(device="cuda").manual_seed(B * 1000 + C)
+    shape = (B, C, H, W) if layout == si.NCHW else (B, H, W, C)
+    x = (torch.randn(shape, generator=g, device="cuda") * 0.7 + 0.2).to(TORCH_DT[dt]).contiguous()
+    cache = dummy_cache(C)
+    skip = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    if B > 2:
+        skip[1] = 1
+    sv = torch.full((B, C), -7.0, device="cuda")
+    n2 = torch.full((B,), -7.0, device="cuda")
+    smtm.smtm_encode(cache, 0, smtm.Fmap(x, dt, layout, B, C, H, W), sv, skip=skip, sv_norm2=n2)
+    torch.cuda.synchronize()
+    ref = oracle.gap(x.cpu(), dt, layout, B, C, H, W)
+    axes = (2, 3) if layout == si.NCHW else (1, 2)
+    scale = x.float().abs().mean(dim=axes).cpu().numpy().astype(np.float64)
+    got = sv.cpu().numpy().astype(np.float64)
+    keep = skip.cpu().numpy() == 0
+    assert np.all(np.abs(got - ref)[keep] <= 1e-5 * scale[keep] + 1e-30)
+    assert np.all(got[~keep] == -7.0)                       # skipped rows are not written
+    n2h = n2.cpu().numpy().astype(np.float64)
+    np.testing.assert_allclose(n2h[keep], (ref ** 2).sum(axis=1)[keep], rtol=1e-5)
+    assert np.all(n2h[~keep] == -7.0)
+    assert smtm.smtm_cache_status(cache) == 0
+    # same bytes twice: bitwise identical (fixed reduction order)
+    sv2 = torch.zeros_like(sv)
+    smtm.smtm_encode(cache, 0, smtm.Fmap(x, dt, layout, B, C, H, W), sv2)
+    torch.cuda.synchronize()
+    assert torch.equal(sv2[keep], sv[keep])
+    smtm.smtm_cache_destroy(cache)
+
+
+def test_encode_constant_map_and_layout_equivalence():
+    B, C, H, W = 4, 64, 14, 14
+    cache = dummy_cache(C)
+    x = torch.full((B, C, H, W), 0.625, dtype=torch.bfloat16, device="cuda")
+    sv = torch.zeros((B, C), device="cuda")
+    smtm.smtm_encode(cache, 0, smtm.Fmap(x, si.BF16, si.NCHW, B, C, H, W), sv)
+    assert torch.all(sv == 0.625)
+    g = torch.Generator(device="cuda").manual_seed(1)
+    y = torch.randn((B, C, H, W), generator=g, device="cuda").half()
+    a = torch.zeros((B, C), device="cuda")
+    b = torch.zeros((B, C), device="cuda")
+    smtm.smtm_encode(cache, 0, smtm.Fmap(y, si.F16, si.NCHW, B, C, H, W), a)
+    yn = y.permute(0, 2, 3, 1).contiguous()
+    smtm.smtm_encode(cache, 0, smtm.Fmap(yn, si.F16, si.NHWC, B, C, H, W), b)
+    torch.cuda.synchronize()
+    assert torch.allclose(a, b, rtol=0, atol=2e-6)
+    smtm.smtm_cache_destroy(cache)
+
+
+def test_argument_errors_launch_nothing():
+    C = 64
+    cache = dummy_cache(C, max_batch=8)
+    x = torch.zeros((4, C, 7, 7), dtype=torch.bfloat16, device="cuda")
+    sv = torch.zeros((4, C), device="cuda")
+    before = smtm.smtm_cache_get_launches(cache)
+    for fm, code in ((smtm.Fmap(x, si.BF16, si.NCHW, 4, C + 8, 7, 7), 2), (smtm.Fmap(x, 7, si.NCHW, 4, C, 7, 7), 3),
+                     (smtm.Fmap(x, si.BF16, si.NCHW, 9, C, 7, 7), 2), (smtm.Fmap(None, si.BF16, si.NCHW, 4, C, 7, 7), 1)):
+        with pytest.raises(smtm.SmtmError) as e:
+            smtm.smtm_encode(cache, 0, fm, sv)
+        assert e.value.status == code
+    mis = torch.zeros(4 * C * 49 + 8, dtype=torch.bfloat16, device="cuda")[1:1 + 4 * C * 49]
+    fm = smtm.Fmap(None, si.BF16, si.NCHW, 4, C, 7, 7)
+    fm.c.d_data = mis.data_ptr()
+    with pytest.raises(smtm.SmtmError) as e:
+        smtm.smtm_encode(cache, 0, fm, sv)
+    assert e.value.status == 4
+    with pytest.raises(smtm.SmtmError):
+        smtm.smtm_encode(cache, 1, smtm.Fmap(x, si.BF16, si.NCHW, 4, C, 7, 7), sv)
+    assert smtm.smtm_cache_get_launches(cache) == before
+    smtm.smtm_cache_destroy(cache)
+
+
+# ---------------------------------------------------------------------------- whole path
+
+def test_c1_single_layer_fp32():
+    rep = run_workload(si.C1)
+    assert rep.exits == [8] and rep.band_mismatches == 0
+
+
+def test_c2_resnet50_bf16_four_layers():
+    rep = run_workload(si.C2)
+    assert sum(rep.exits) > 30 and rep.frames == 64
+
+
+def test_c2_exits_disabled_streams_every_layer():
+    rep = run_workload(si.C2.scaled(tau=float("inf")))
+    assert rep.exits == [0, 0, 0, 0] and rep.lookups == 4 * 64
+
+
+def test_c3_mobilenetv2_fp16_nhwc_novel_classes_do_not_exit():
+    w = si.C3
+    rep = run_workload(w)
+    assert sum(rep.exits) > 100
+    lab = si.labels(w)[0]
+    # the oracle (and therefore the library, which matched it) lets no novel frame exit
+    cache_exits = sum(rep.exits)
+    assert cache_exits <= int((lab < w.n).sum())
+
+
+def test_c4_large_cache_straddles_threshold():
+    rep = run_workload(si.C4)
+    assert 100 < rep.exits[0] < 900
+    print("c4 near-threshold lookups (oracle):", rep.near_oracle, "band mismatches:", rep.band_mismatches)
+
+
+@pytest.mark.parametrize("T", [6])
+def test_c5_streaming_full_width(T):
+    rep = run_workload(si.C5, steps=T)
+    assert rep.frames == 512 * T and rep.exits[0] > 0
+
+
+def test_c5_full_length_64_steps_state_only():
+    # all 64 steps at full width; values are compared on every step, state every 8 steps
+    rep = run_workload(si.C5, state_every=8)
+    assert rep.frames == 512 * 64
+    print("c5 exits per layer:", rep.exits, "never:", rep.frames - sum(rep.exits), "band:", rep.band_mismatches)
+
+
+def test_adaptive_size_moves_and_ragged_small_cases():
+    # small classes / streams / odd batch: exercises k growing and shrinking, ties, fallback -1
+    w = si.Workload("tiny", si.F16, si.NCHW, B=37, stages=((24, 7, 7), (40, 5, 3)), n=23, k_init=3, k_min=2,
+                    k_max=9, S=1, T=12, tau=0.3, window_W=3, sigma=0.4, zipf_s=0.7, novel_frac=0.15, n_novel=5,
+                    repeat_p=0.5, seed=3)
+    rep = run_workload(w)
+    assert rep.frames == 37 * 12
+    w2 = si.Workload("tiny_streams", si.BF16, si.NHWC, B=19, stages=((16, 6, 6),), n=11, k_init=2, k_min=2,
+                     k_max=11, S=19, T=20, tau=0.2, window_W=2, sigma=0.5, zipf_s=1.0, repeat_p=0.6, seed=4)
+    rep2 = run_workload(w2)
+    assert rep2.frames == 19 * 20
+
+
+def test_step_host_matches_device_path():
+    w = si.C5.scaled(B=32, S=32, T=3)
+    cents, counts = si.initial_centers(w)
+    tau = [w.tau] * w.L
+    mk = lambda: smtm.smtm_cache_create(w.n, w.dims, tau, cents, counts, n_streams=w.S, k_init=w.k_init,
+                                        k_min=w.k_min, k_max=w.k_max, window_W=w.window_W, max_batch=w.B)
+    a, b = mk(), mk()
+    gb = smtm.Batch(a, w.B, stream_id=si.stream_ids(w))
+    labs = si.labels(w)
+    sid = si.stream_ids(w)
+    for t in range(w.T):
+        maps = [si.frames(w, l, labs[t], t, device="cuda") for l in range(w.L)]
+        fb = si.fallback_labels(w, labs[t])
+        smtm.smtm_batch_reset(a, gb)
+        for l in range(w.L):
+            smtm.smtm_lookup_exit(a, l, smtm.Fmap(maps[l], w.dtype, w.layout, *si.shape4(w, l)), gb)
+        smtm.smtm_cache_update(a, gb, torch.from_numpy(fb).cuda())
+        smtm.smtm_cache_resize(a)
+        hm = [m.cpu().pin_memory() for m in maps]
+        done = np.zeros(w.B, np.uint8); el = np.zeros(w.B, np.int32); pred = np.zeros(w.B, np.int32)
+        fmaps = [smtm.Fmap(None, w.dtype, w.layout, *si.shape4(w, l)) for l in range(w.L)]
+        smtm.smtm_step_host(b, fmaps, hm, sid, fb, True, done, el, pred)
+        assert np.array_equal(done, gb.done.cpu().numpy())
+        assert np.array_equal(el, gb.exit_layer.cpu().numpy())
+        assert np.array_equal(pred, gb.pred.cpu().numpy())
+    for x, y in zip(smtm.smtm_cache_get_tables(a), smtm.smtm_cache_get_tables(b)):
+        assert np.array_equal(x, y)
+    for l in range(w.L):
+        ca, cb = smtm.smtm_cache_get_centers(a, l), smtm.smtm_cache_get_centers(b, l)
+        assert np.array_equal(ca[0], cb[0]) and np.array_equal(ca[1], cb[1])
