@@ -141,6 +141,33 @@ smtm_status_t smtm_encode(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t*
 smtm_status_t smtm_lookup_exit(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t* fmap,
                                const smtm_batch_t* batch, void* stream);
 
+/* (No counterpart in the paper: a packaging of smtm_lookup_exit for callers that
+ * must not allocate.)  Some callers cannot call cudaMalloc or anything that may:
+ * a plug-in running inside another engine's enqueue step that is handed only its
+ * inputs and outputs, a real-time thread that must not take the allocator's
+ * locks, a process whose memory budget is frozen after start-up.  This entry
+ * point does one self-contained lookup at `layer` (the cumulative similarity
+ * starts from zero, so the decision is that layer's alone) and keeps its working
+ * memory (semantic vectors [B][C], similarities [B][k_max], exit layers [B]) in a
+ * fixed array of SMTM_STATIC_SCRATCH_BYTES compiled into the library; every GPU
+ * that loads the library holds that array until the process exits.  It calls no
+ * cudaMalloc / cudaFree and no allocating library routine.
+ *   fmap, d_stream_id   as in smtm_lookup_exit.
+ *   d_exit [B]          1 where the frame exits at this layer, else 0.
+ *   d_pred [B]          class of the best match where it exits, else -1.
+ *   d_ac   [B][L]       column `layer` receives Eq. 4's value; may be NULL.
+ * A batch whose working memory would exceed the array (roughly
+ * 4 B (C + k_max + 1) bytes > SMTM_STATIC_SCRATCH_BYTES) is refused with
+ * SMTM_ERR_SHAPE before anything is launched.  The first call on a device looks
+ * up the array's device address; make that first call outside any stream
+ * capture.  All calls on a device share the one array, which keeps the previous
+ * call's contents (the call clears what it accumulates into): two calls whose
+ * GPU work overlaps, e.g. on different streams, race on it. */
+enum { SMTM_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024 };
+smtm_status_t smtm_lookup_exit_static(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t* fmap,
+                                      const int32_t* d_stream_id, uint8_t* d_exit, int32_t* d_pred,
+                                      float* d_ac, void* stream);
+
 /* Sec. 6.1 tables and Eq. 7 centres for a finished batch.  The label of frame b
  * is d_pred[b] if it exited, else d_fallback_label[b] (the full network's
  * answer; -1 or a NULL array = no label); its stop layer is d_exit_layer[b] if it

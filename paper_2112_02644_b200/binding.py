@@ -78,6 +78,7 @@ def load_library():
     lib.smtm_batch_reset.argtypes = [vp, ctypes.POINTER(_Batch), vp]
     lib.smtm_encode.argtypes = [vp, i32, ctypes.POINTER(_Fmap), vp, vp, vp, vp]
     lib.smtm_lookup_exit.argtypes = [vp, i32, ctypes.POINTER(_Fmap), ctypes.POINTER(_Batch), vp]
+    lib.smtm_lookup_exit_static.argtypes = [vp, i32, ctypes.POINTER(_Fmap), vp, vp, vp, vp, vp]
     lib.smtm_cache_update.argtypes = [vp, ctypes.POINTER(_Batch), vp, vp]
     lib.smtm_cache_resize.argtypes = [vp, vp]
     lib.smtm_step_host.argtypes = [vp, ctypes.POINTER(_Fmap), ctypes.POINTER(vp), vp, vp, i32, vp, vp, vp, vp]
@@ -219,6 +220,14 @@ def smtm_encode(cache: Cache, layer: int, fmap: Fmap, sv, skip=None, sv_norm2=No
 def smtm_lookup_exit(cache: Cache, layer: int, fmap: Fmap, batch: Batch, stream=None) -> None:
     _check(load_library().smtm_lookup_exit(cache.handle, layer, ctypes.byref(fmap.c), ctypes.byref(batch.c),
                                            _stream(stream)), "smtm_lookup_exit")
+
+
+def smtm_lookup_exit_static(cache: Cache, layer: int, fmap: Fmap, stream_id, exit_flags, pred, ac=None,
+                            stream=None) -> None:
+    """Single-layer lookup whose working memory is a fixed array inside the library (allocates nothing)."""
+    _check(load_library().smtm_lookup_exit_static(cache.handle, layer, ctypes.byref(fmap.c), _dptr(stream_id),
+                                                  _dptr(exit_flags), _dptr(pred), _dptr(ac), _stream(stream)),
+           "smtm_lookup_exit_static")
 
 
 def smtm_cache_update(cache: Cache, batch: Batch, fallback_label=None, stream=None) -> None:

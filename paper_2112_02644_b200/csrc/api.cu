@@ -31,9 +31,14 @@ struct smtm_cache {
     size_t stage_bytes[SMTM_MAX_LAYERS];
 };
 
+void smtm::cache_shape(const smtm_cache_t* cache, int* n_layers, int* k_max) {
+    *n_layers = cache->L;
+    *k_max = cache->k_max;
+}
+
 namespace {
 
-#define SMTM_CUDA(call)                          \
+#define SMTM_CUDA(call)                         \
     do {                                         \
         if ((call) != cudaSuccess) {             \
             (void)cudaGetLastError();            \

@@ -8,6 +8,9 @@
 
 namespace smtm {
 
+// Number of exit layers and the fast-memory capacity of a cache.
+void cache_shape(const smtm_cache_t* cache, int* n_layers, int* k_max);
+
 // ---- encode (Sec. 4.1) ------------------------------------------------------------------
 struct EncodeArgs {
     const void* x;        // device, 16-byte aligned
