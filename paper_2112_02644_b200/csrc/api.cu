@@ -20,6 +20,8 @@ struct smtm_cache {
     int32_t* d_k;
     unsigned long long* d_counters;
     int* d_status;
+    float* d_partials;  // scratch of the fused lookup: partial dot products per (frame, part)
+    int* d_frame_ctr;   // scratch of the fused lookup: parts delivered per frame (zero between launches)
     int device, sm_count;
     int64_t launches;
     // device-side carry and staging used only by smtm_step_host (allocated on first use)
@@ -67,6 +69,8 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_k);
     cudaFree(c->d_counters);
     cudaFree(c->d_status);
+    cudaFree(c->d_partials);
+    cudaFree(c->d_frame_ctr);
     cudaFree(c->hb.d_sa);
     cudaFree(c->hb.d_done);
     cudaFree(c->hb.d_exit_layer);
@@ -111,7 +115,6 @@ EncodeArgs encode_args(const smtm_cache* c, const smtm_fmap_t* f, const uint8_t*
 
 smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b,
                           cudaStream_t st) {
-    SMTM_CUDA(launch_encode(encode_args(c, f, b->d_done, b->d_sv[layer]), c->sm_count, st, &c->launches));
     LookupArgs a{};
     a.layer = layer;
     a.L = c->L;
@@ -134,6 +137,11 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     a.sep = b->d_sep;
     a.top = b->d_top;
     a.counters = c->d_counters;
+    const EncodeArgs e = encode_args(c, f, b->d_done, b->d_sv[layer]);
+    bool fused = false;
+    SMTM_CUDA(launch_lookup_fused(e, a, c->d_partials, c->d_frame_ctr, c->sm_count, st, &c->launches, &fused));
+    if (fused) return SMTM_OK;
+    SMTM_CUDA(launch_encode(e, c->sm_count, st, &c->launches));
     SMTM_CUDA(launch_score_exit(a, st, &c->launches));
     return SMTM_OK;
 }
@@ -245,6 +253,8 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     ok = ok && dev_alloc(&c->d_k, S) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_counters, SMTM_CTR_COUNT) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_status, 1) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_partials, fused_partials_floats(c->max_batch, c->k_max)) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_frame_ctr, size_t(c->max_batch)) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();
         free_all(c);
@@ -272,6 +282,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     if (e == cudaSuccess) e = cudaMemset(c->d_ts, 0, size_t(S) * n * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(c->d_counters, 0, SMTM_CTR_COUNT * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(c->d_frame_ctr, 0, size_t(c->max_batch) * sizeof(int));
     if (e == cudaSuccess)
         e = cudaMemcpy(c->d_members, members.data(), members.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(c->d_k, ks.data(), ks.size() * sizeof(int32_t), cudaMemcpyHostToDevice);

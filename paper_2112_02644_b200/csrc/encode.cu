@@ -22,8 +22,7 @@
 // Any other shape falls back to a plain thread-per-(frame, channel) loop.
 #include <algorithm>
 
-#include "common.cuh"
-#include "internal.h"
+#include "lookup_common.cuh"
 
 namespace smtm {
 
@@ -61,8 +60,8 @@ struct UnitPerLane {
     static constexpr int G = 16 / gcd16(kUnitBytesRaw);
     static constexpr int UW = G * kUnitBytesRaw / 16;
 
-    static __device__ __forceinline__ void run(const uint8_t* stage, int nch, int lane, float* out, float inv_hw,
-                                               const NchwParams&) {
+    static __device__ __forceinline__ void run(const uint8_t* stage, int nch, int lane, float* out, float* out_s,
+                                               float inv_hw, const NchwParams&) {
         const int units = nch / G;
         if (lane >= units) return;
         const uint4* u = reinterpret_cast<const uint4*>(stage) + lane * UW;
@@ -85,14 +84,24 @@ struct UnitPerLane {
             for (int g = 0; g + 3 < G; g += 4)
                 *reinterpret_cast<float4*>(o + g) = make_float4(acc[g], acc[g + 1], acc[g + 2], acc[g + 3]);
         }
+        if (out_s) {
+            float* os = out_s + lane * G;
+            if (G == 2) {
+                *reinterpret_cast<float2*>(os) = make_float2(acc[0], acc[1]);
+            } else {
+#pragma unroll
+                for (int g = 0; g + 3 < G; g += 4)
+                    *reinterpret_cast<float4*>(os + g) = make_float4(acc[g], acc[g + 1], acc[g + 2], acc[g + 3]);
+            }
+        }
     }
 };
 
 // T lanes per channel; channel bytes are a multiple of 16.
 template <class E>
 struct TeamPerChannel {
-    static __device__ __forceinline__ void run(const uint8_t* stage, int nch, int lane, float* out, float inv_hw,
-                                               const NchwParams& p) {
+    static __device__ __forceinline__ void run(const uint8_t* stage, int nch, int lane, float* out, float* out_s,
+                                               float inv_hw, const NchwParams& p) {
         const int T = p.team, uw = p.vec_per_channel;
         const int per_pass = kWarp / T;
         const int team = lane / T, r = lane - team * T;
@@ -114,7 +123,10 @@ struct TeamPerChannel {
             }
             float s = (a0 + a1) + (a2 + a3);
             for (int o = T >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(kFull, s, o);
-            if (c < nch && r == 0) out[c] = s * inv_hw;
+            if (c < nch && r == 0) {
+                out[c] = s * inv_hw;
+                if (out_s) out_s[c] = s * inv_hw;
+            }
         }
     }
 };
@@ -165,7 +177,7 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
                     failed = true;
                     break;
                 }
-                R::run(stages + size_t(stage) * kStageCap, nch, lane, p.sv + (long long)b * p.C + c0, p.inv_hw, p);
+                R::run(stages + size_t(stage) * kStageCap, nch, lane, p.sv + (long long)b * p.C + c0, nullptr, p.inv_hw, p);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[stage]);
             }
@@ -178,6 +190,244 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
     if (any_failed && producer && lane == 0) {
         for (int s = 0; s < kStages && s < it; ++s) {
             const uint32_t last_use = uint32_t((it - 1 - s) / kStages);
+            mbar_wait_bounded(&full[s], last_use & 1, p.status);
+        }
+    }
+}
+
+// ---- fused lookup: encode + score + exit in one persistent kernel ----------------------------
+//
+// Work is cut into units: (frame, part), a part being a run of chunks_per_unit chunks, i.e. a
+// slice of the frame's channels.  Every CTA first compacts the frames that are still active
+// and takes the units u = blockIdx.x, blockIdx.x + gridDim.x, ... of that list, so exited
+// frames cost nothing and the load is even.  Per unit the reducer warps leave the slice of
+// the semantic vector in shared memory (double-buffered) as well as in the SV stash; four
+// scorer warps take it from there: partial dot products against the slice of each member's
+// centre and the partial squared length.  With one part per frame the frame is decided on
+// the spot; otherwise the partials go to global scratch and the CTA that delivers a frame's
+// last part adds them up in part order and decides.  No floating-point atomics anywhere:
+// the evaluation order of every sum is fixed.
+constexpr int kScorers = 4;
+constexpr int kThreadsFused = (kConsumers + 1 + kScorers) * kWarp;
+constexpr int kFusedMaxK = 64;      // fast-memory capacity the fused kernel supports
+constexpr int kMaxUnits = 1024;     // units per CTA
+constexpr int kMaxSlice = 2048;     // floats of a semantic-vector slice held in shared memory
+constexpr int kMaxParts = 16;
+
+struct FusedParams {
+    NchwParams e;
+    LookupArgs a;
+    int parts;            // P: parts per frame (divides chunks_per_frame)
+    int chunks_per_unit;  // chunks_per_frame / P
+    int slice_cap;        // channels of a full slice = chunks_per_unit * chunk_channels
+    float* partials;      // [B][P][k_max + 1], used when P > 1
+    int* frame_ctr;       // [B] parts delivered so far (returns to zero)
+};
+
+constexpr size_t fused_smem(int slice_cap) {
+    return size_t(kStages) * kStageCap + 2 * size_t(slice_cap) * 4 + 2 * (kFusedMaxK + 1) * 4 + 2 * kFusedMaxK * 4 +
+           kMaxUnits * 4 + (2 * kStages + 5) * 8 + 40 * 4 + 192;
+}
+
+template <class R>
+__global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedParams f) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    uint8_t* stages = base;
+    float* sv_s = reinterpret_cast<float*>(base + size_t(kStages) * kStageCap);  // [2][slice_cap]
+    float* s_dot = sv_s + 2 * f.slice_cap;                                       // [2][kFusedMaxK + 1]
+    float* s_cur = s_dot + 2 * (kFusedMaxK + 1);                                 // [kFusedMaxK]
+    float* s_acc = s_cur + kFusedMaxK;                                           // [kFusedMaxK]
+    int* my_units = reinterpret_cast<int*>(s_acc + kFusedMaxK);                  // [kMaxUnits]
+    int* s_scan = my_units + kMaxUnits;                                          // [40]
+    uint64_t* full = reinterpret_cast<uint64_t*>(
+        (reinterpret_cast<uintptr_t>(s_scan + 40) + 7) & ~uintptr_t(7));         // [kStages]
+    uint64_t* empty = full + kStages;                                            // [kStages]
+    uint64_t* sv_full = empty + kStages;                                         // [2]
+    uint64_t* sv_empty = sv_full + 2;                                            // [2]
+    uint64_t* sc_bar = sv_empty + 2;                                             // [1]
+
+    const NchwParams& p = f.e;
+    const LookupArgs& a = f.a;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int P = f.parts, cpu = f.chunks_per_unit;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&sv_full[s], cpu);
+            mbar_init(&sv_empty[s], kScorers);
+        }
+        mbar_init(sc_bar, kScorers);
+        mbar_init_fence();
+    }
+
+    // ---- the active frames and this CTA's share of their units -----------------------------
+    // A frame counts as active if it had not exited before this layer; one that this very
+    // launch has already decided (another CTA may be ahead) still counts, so that every CTA
+    // derives the same list.
+    int n_active = 0;
+    for (int t0 = 0; t0 < a.B; t0 += kThreadsFused) {
+        const int b = t0 + threadIdx.x;
+        int act = 0;
+        if (b < a.B) act = (!a.done[b] || *(volatile const int32_t*)(a.exit_layer + b) == a.layer + 1) ? 1 : 0;
+        int cnt;
+        const int pos = block_exclusive_scan(act, s_scan, &cnt);
+        if (act) {
+            for (int part = 0; part < P; ++part) {
+                const int u = (n_active + pos) * P + part;
+                if (u % int(gridDim.x) == int(blockIdx.x)) {
+                    const int idx = u / int(gridDim.x);
+                    if (idx < kMaxUnits) my_units[idx] = b * kMaxParts + part;
+                }
+            }
+        }
+        n_active += cnt;
+    }
+    const int total_units = n_active * P;
+    int nu = total_units > int(blockIdx.x) ? (total_units - int(blockIdx.x) + int(gridDim.x) - 1) / int(gridDim.x) : 0;
+    nu = min(nu, kMaxUnits);
+    __syncthreads();
+
+    const int n_chunks = nu * cpu;
+    bool failed = false;
+    int issued = 0;
+    if (warp < kConsumers) {
+        // ---- reducers: warp w owns stage w and the chunks it, it + kConsumers, ... ------------
+        for (int it = warp; it < n_chunks; it += kConsumers) {
+            const int i = it / cpu, c = it - i * cpu;
+            const int unit = my_units[i], b = unit / kMaxParts, part = unit % kMaxParts;
+            const int c0 = (part * cpu + c) * p.chunk_channels;
+            const int nch = min(p.chunk_channels, p.C - c0);
+            const int buf = i & 1;
+            if (i >= 2 && !mbar_wait_bounded(&sv_empty[buf], ((i >> 1) - 1) & 1, p.status)) { failed = true; break; }
+            if (!mbar_wait_bounded(&full[warp], (it / kStages) & 1, p.status)) { failed = true; break; }
+            R::run(stages + size_t(warp) * kStageCap, nch, lane, p.sv + (long long)b * p.C + c0,
+                   sv_s + buf * f.slice_cap + c * p.chunk_channels, p.inv_hw, p);
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&empty[warp]);
+                mbar_arrive(&sv_full[buf]);
+            }
+        }
+    } else if (warp == kConsumers) {
+        // ---- producer -------------------------------------------------------------------------
+        if (lane == 0) {
+            for (int it = 0; it < n_chunks; ++it) {
+                const int i = it / cpu, c = it - i * cpu;
+                const int unit = my_units[i], b = unit / kMaxParts, part = unit % kMaxParts;
+                const int c0 = (part * cpu + c) * p.chunk_channels;
+                const int nch = min(p.chunk_channels, p.C - c0);
+                const int stage = it % kStages;
+                const uint32_t use = uint32_t(it / kStages);
+                if (use > 0 && !mbar_wait_bounded(&empty[stage], (use - 1) & 1, p.status)) { failed = true; break; }
+                const uint32_t bytes = uint32_t(nch) * uint32_t(p.ch_bytes);
+                mbar_expect_tx(&full[stage], bytes);
+                bulk_load(stages + size_t(stage) * kStageCap,
+                          p.x + (long long)b * p.frame_bytes + (long long)c0 * p.ch_bytes, bytes, &full[stage]);
+                issued = it + 1;
+            }
+        }
+    } else {
+        // ---- scorers ----------------------------------------------------------------------------
+        const int sw = warp - kConsumers - 1;
+        const float weight = float(1u << a.layer);  // 2^(l-1) with l = layer + 1
+        uint32_t sc_phase = 0;
+        for (int i = 0; i < nu; ++i) {
+            const int unit = my_units[i], b = unit / kMaxParts, part = unit % kMaxParts;
+            const int buf = i & 1;
+            const int sb = part * f.slice_cap;                 // first channel of the slice
+            const int Dp = min(f.slice_cap, p.C - sb);         // channels in it
+            const int sid = a.stream_id ? a.stream_id[b] : 0;
+            const int k = min(a.k[sid], kFusedMaxK);
+            const int32_t* mem = a.members + (size_t)sid * a.k_max;
+            const float* v = sv_s + buf * f.slice_cap;
+            if (!mbar_wait_bounded(&sv_full[buf], (i >> 1) & 1, p.status)) { failed = true; break; }
+            const bool vec = ((p.C | sb | Dp) & 3) == 0;
+            const int n4 = vec ? Dp >> 2 : 0;
+            const float4* v4 = reinterpret_cast<const float4*>(v);
+            float* out = P == 1 ? s_dot + buf * (kFusedMaxK + 1)
+                                : f.partials + ((size_t)b * P + part) * (a.k_max + 1);
+            const int norm_slot = P == 1 ? kFusedMaxK : a.k_max;
+            if (sw == 0) {  // partial squared length of the semantic vector
+                float n0 = 0.f, n1 = 0.f, n2 = 0.f, n3 = 0.f;
+                for (int q = lane; q < n4; q += kWarp) {
+                    const float4 x = v4[q];
+                    n0 = fmaf(x.x, x.x, n0); n1 = fmaf(x.y, x.y, n1); n2 = fmaf(x.z, x.z, n2); n3 = fmaf(x.w, x.w, n3);
+                }
+                for (int q = (n4 << 2) + lane; q < Dp; q += kWarp) n0 = fmaf(v[q], v[q], n0);
+                float nn = (n0 + n1) + (n2 + n3);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(kFull, nn, o);
+                if (lane == 0) out[norm_slot] = nn;
+            }
+            for (int j = sw; j < k; j += kScorers) {  // partial dot products, Eq. 1's numerator
+                const float* crow = a.centers + (size_t)mem[j] * p.C + sb;
+                const float4* c4 = reinterpret_cast<const float4*>(crow);
+                float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+                for (int q = lane; q < n4; q += kWarp) {
+                    const float4 cc = __ldg(c4 + q);
+                    const float4 x = v4[q];
+                    d0 = fmaf(cc.x, x.x, d0); d1 = fmaf(cc.y, x.y, d1); d2 = fmaf(cc.z, x.z, d2); d3 = fmaf(cc.w, x.w, d3);
+                }
+                for (int q = (n4 << 2) + lane; q < Dp; q += kWarp) d0 = fmaf(crow[q], v[q], d0);
+                float dot = (d0 + d1) + (d2 + d3);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(kFull, dot, o);
+                if (lane == 0) out[j] = dot;
+            }
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&sv_empty[buf]);  // done reading the slice
+                mbar_arrive(sc_bar);
+            }
+            if (!mbar_wait_bounded(sc_bar, sc_phase, p.status)) { failed = true; break; }
+            sc_phase ^= 1;
+            if (sw != 0) continue;
+
+            // scorer warp 0: is the frame complete?  (with P > 1: did we deliver its last part?)
+            int last = 1;
+            if (P > 1) {
+                if (lane == 0) {
+                    __threadfence();
+                    last = atomicAdd(&f.frame_ctr[b], 1) == P - 1 ? 1 : 0;
+                    if (last) f.frame_ctr[b] = 0;
+                    __threadfence();
+                }
+                last = __shfl_sync(kFull, last, 0);
+            }
+            if (!last) continue;
+            float nrm = 0.f;
+            if (P == 1) {
+                nrm = out[norm_slot];
+            } else {
+                for (int q = 0; q < P; ++q) nrm += __ldcg(f.partials + ((size_t)b * P + q) * (a.k_max + 1) + a.k_max);
+            }
+            for (int j = lane; j < k; j += kWarp) {
+                float dot = 0.f;
+                if (P == 1) {
+                    dot = out[j];
+                } else {
+                    for (int q = 0; q < P; ++q) dot += __ldcg(f.partials + ((size_t)b * P + q) * (a.k_max + 1) + j);
+                }
+                const float s = cosine_from(dot, nrm, a.cnorm[mem[j]]);                    // Eq. 1
+                const float acc = __fmaf_rn(s, weight, a.sa[(size_t)b * a.k_max + j]);     // Eq. 3
+                a.sa[(size_t)b * a.k_max + j] = acc;
+                s_cur[j] = s;
+                s_acc[j] = acc;
+            }
+            __syncwarp();
+            decide_frame(a, b, s_cur, s_acc, mem, k, lane);
+            __syncwarp();
+        }
+    }
+    // No thread leaves before every copy that was issued has landed.
+    const int any_failed = __syncthreads_or(failed ? 1 : 0);
+    if (any_failed && warp == kConsumers && lane == 0) {
+        for (int s = 0; s < kStages && s < issued; ++s) {
+            const uint32_t last_use = uint32_t((issued - 1 - s) / kStages);
             mbar_wait_bounded(&full[s], last_use & 1, p.status);
         }
     }
@@ -312,79 +562,142 @@ int pow2_floor(int v) {
     return p;
 }
 
+
+
+// Which reducer a shape is served by, and the chunking that goes with it.
+enum Reducer { kNone, kUnitBf16x49, kUnitBf16x196, kUnitF16x49, kUnitF16x196, kUnitF32x49, kTeamF32, kTeamF16, kTeamBf16 };
+
+Reducer plan_nchw(const EncodeArgs& a, NchwParams* p) {
+    const int HW = a.H * a.W;
+    const int es = a.dtype == SMTM_F32 ? 4 : 2;
+    *p = NchwParams{};
+    p->x = static_cast<const uint8_t*>(a.x);
+    p->skip = a.skip;
+    p->sv = a.sv;
+    p->status = a.status;
+    p->C = a.C;
+    p->ch_bytes = HW * es;
+    p->frame_bytes = (long long)a.C * p->ch_bytes;
+    p->inv_hw = 1.0f / float(HW);
+    // unit-per-lane shapes (compile-time H*W)
+    int G = 0;
+    if ((HW == 49 || HW == 196) && es == 2) G = HW == 49 ? 8 : 2;
+    if (HW == 49 && es == 4) G = 4;
+    if (G && a.C % G == 0) {
+        p->chunk_channels = 32 * G;
+        p->chunks_per_frame = (a.C + p->chunk_channels - 1) / p->chunk_channels;
+        p->total_chunks = (long long)a.B * p->chunks_per_frame;
+        if (es == 4) return kUnitF32x49;
+        if (a.dtype == SMTM_BF16) return HW == 49 ? kUnitBf16x49 : kUnitBf16x196;
+        return HW == 49 ? kUnitF16x49 : kUnitF16x196;
+    }
+    // team-per-channel: channel bytes a multiple of 16 and at most one stage
+    if (p->ch_bytes % 16 == 0 && p->ch_bytes <= kStageCap) {
+        p->vec_per_channel = p->ch_bytes / 16;
+        p->team = std::min(32, pow2_floor(std::max(1, p->vec_per_channel / 4)));
+        const int per_pass = 32 / p->team;
+        int cc = kStageCap / p->ch_bytes;
+        if (cc > per_pass) cc -= cc % per_pass;
+        p->chunk_channels = std::min(cc, a.C);
+        p->chunks_per_frame = (a.C + p->chunk_channels - 1) / p->chunk_channels;
+        p->total_chunks = (long long)a.B * p->chunks_per_frame;
+        return a.dtype == SMTM_F32 ? kTeamF32 : a.dtype == SMTM_F16 ? kTeamF16 : kTeamBf16;
+    }
+    return kNone;
+}
+
+#define SMTM_FOR_REDUCER(r, CALL)                                   \
+    switch (r) {                                                    \
+        case kUnitBf16x49: CALL(UnitPerLane<BF16, 49>); break;      \
+        case kUnitBf16x196: CALL(UnitPerLane<BF16, 196>); break;    \
+        case kUnitF16x49: CALL(UnitPerLane<F16, 49>); break;        \
+        case kUnitF16x196: CALL(UnitPerLane<F16, 196>); break;      \
+        case kUnitF32x49: CALL(UnitPerLane<F32, 49>); break;        \
+        case kTeamF32: CALL(TeamPerChannel<F32>); break;            \
+        case kTeamF16: CALL(TeamPerChannel<F16>); break;            \
+        case kTeamBf16: CALL(TeamPerChannel<BF16>); break;          \
+        default: break;                                             \
+    }
+
+template <class R>
+cudaError_t opt_in_fused() {
+    return cudaFuncSetAttribute(k_lookup_nchw<R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                int(fused_smem(kMaxSlice)));
+}
+
 }  // namespace
 
 cudaError_t encode_setup() {
-    cudaError_t e;
-    if ((e = opt_in<UnitPerLane<BF16, 49>>()) != cudaSuccess) return e;
-    if ((e = opt_in<UnitPerLane<BF16, 196>>()) != cudaSuccess) return e;
-    if ((e = opt_in<UnitPerLane<F16, 49>>()) != cudaSuccess) return e;
-    if ((e = opt_in<UnitPerLane<F16, 196>>()) != cudaSuccess) return e;
-    if ((e = opt_in<UnitPerLane<F32, 49>>()) != cudaSuccess) return e;
-    if ((e = opt_in<TeamPerChannel<BF16>>()) != cudaSuccess) return e;
-    if ((e = opt_in<TeamPerChannel<F16>>()) != cudaSuccess) return e;
-    if ((e = opt_in<TeamPerChannel<F32>>()) != cudaSuccess) return e;
-    return cudaSuccess;
+    cudaError_t e = cudaSuccess;
+#define SMTM_OPT_IN(...)                                        \
+    if (e == cudaSuccess) e = opt_in<__VA_ARGS__>();            \
+    if (e == cudaSuccess) e = opt_in_fused<__VA_ARGS__>();
+    for (int r = kUnitBf16x49; r <= kTeamBf16; ++r) SMTM_FOR_REDUCER(r, SMTM_OPT_IN)
+#undef SMTM_OPT_IN
+    return e;
 }
 
 cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
-    const int HW = a.H * a.W;
-    const int es = a.dtype == SMTM_F32 ? 4 : 2;
-    const float inv_hw = 1.0f / float(HW);
     ++*launches;
-
     if (a.layout == SMTM_NHWC) {
-        const int V = 16 / es;
+        const int V = a.dtype == SMTM_F32 ? 4 : 8;
         if (a.C % V == 0) {
             if (a.dtype == SMTM_F32) return launch_nhwc<F32>(a, st);
             if (a.dtype == SMTM_F16) return launch_nhwc<F16>(a, st);
             return launch_nhwc<BF16>(a, st);
         }
     } else {
-        NchwParams p{};
-        p.x = static_cast<const uint8_t*>(a.x);
-        p.skip = a.skip;
-        p.sv = a.sv;
-        p.status = a.status;
-        p.C = a.C;
-        p.ch_bytes = HW * es;
-        p.frame_bytes = (long long)a.C * p.ch_bytes;
-        p.inv_hw = inv_hw;
-        const int grid = sm_count;
-        // unit-per-lane shapes (compile-time H*W)
-        int G = 0;
-        if ((HW == 49 || HW == 196) && es == 2) G = HW == 49 ? 8 : 2;
-        if (HW == 49 && es == 4) G = 4;
-        if (G && a.C % G == 0) {
-            p.chunk_channels = 32 * G;
-            p.chunks_per_frame = (a.C + p.chunk_channels - 1) / p.chunk_channels;
-            p.total_chunks = (long long)a.B * p.chunks_per_frame;
-            if (es == 4) return launch_nchw<UnitPerLane<F32, 49>>(p, grid, st);
-            if (a.dtype == SMTM_BF16)
-                return HW == 49 ? launch_nchw<UnitPerLane<BF16, 49>>(p, grid, st)
-                                : launch_nchw<UnitPerLane<BF16, 196>>(p, grid, st);
-            return HW == 49 ? launch_nchw<UnitPerLane<F16, 49>>(p, grid, st)
-                            : launch_nchw<UnitPerLane<F16, 196>>(p, grid, st);
-        }
-        // team-per-channel: channel bytes a multiple of 16 and at most one stage
-        if (p.ch_bytes % 16 == 0 && p.ch_bytes <= kStageCap) {
-            p.vec_per_channel = p.ch_bytes / 16;
-            p.team = std::min(32, pow2_floor(std::max(1, p.vec_per_channel / 4)));
-            const int per_pass = 32 / p.team;
-            int cc = kStageCap / p.ch_bytes;
-            if (cc > per_pass) cc -= cc % per_pass;
-            p.chunk_channels = std::min(cc, a.C);
-            p.chunks_per_frame = (a.C + p.chunk_channels - 1) / p.chunk_channels;
-            p.total_chunks = (long long)a.B * p.chunks_per_frame;
-            if (a.dtype == SMTM_F32) return launch_nchw<TeamPerChannel<F32>>(p, grid, st);
-            if (a.dtype == SMTM_F16) return launch_nchw<TeamPerChannel<F16>>(p, grid, st);
-            return launch_nchw<TeamPerChannel<BF16>>(p, grid, st);
+        NchwParams p;
+        const Reducer r = plan_nchw(a, &p);
+        if (r != kNone) {
+            cudaError_t e = cudaSuccess;
+#define SMTM_LAUNCH(...) e = launch_nchw<__VA_ARGS__>(p, sm_count, st)
+            SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
+#undef SMTM_LAUNCH
+            return e;
         }
     }
     if (a.dtype == SMTM_F32) return launch_generic<F32>(a, st);
     if (a.dtype == SMTM_F16) return launch_generic<F16>(a, st);
     return launch_generic<BF16>(a, st);
+}
+
+size_t fused_partials_floats(int max_batch, int k_max) {
+    return size_t(max_batch) * kMaxParts * (size_t(std::min(k_max, kFusedMaxK)) + 1);
+}
+
+cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float* partials, int* frame_ctr,
+                                int sm_count, cudaStream_t st, int64_t* launches, bool* handled) {
+    *handled = false;
+    if (e.B <= 0 || e.layout != SMTM_NCHW || a.k_max > kFusedMaxK || !partials || !frame_ctr) return cudaSuccess;
+    FusedParams f{};
+    const Reducer r = plan_nchw(e, &f.e);
+    if (r == kNone) return cudaSuccess;
+    // parts per frame: as many as leave at least four chunks per unit; more if a slice would
+    // not fit its shared-memory buffer
+    const int cpf = f.e.chunks_per_frame;
+    int P = 1;
+    for (int d = 1; d <= std::min(cpf, kMaxParts); ++d)
+        if (cpf % d == 0 && cpf / d >= 4) P = d;
+    while (P < cpf && (cpf % P != 0 || (cpf / P) * f.e.chunk_channels > kMaxSlice)) ++P;
+    if (cpf % P != 0 || P > kMaxParts || (cpf / P) * f.e.chunk_channels > kMaxSlice) return cudaSuccess;
+    if (((long long)e.B * P + sm_count - 1) / sm_count > kMaxUnits) return cudaSuccess;
+    f.a = a;
+    f.parts = P;
+    f.chunks_per_unit = cpf / P;
+    f.slice_cap = f.chunks_per_unit * f.e.chunk_channels;
+    f.partials = partials;
+    f.frame_ctr = frame_ctr;
+    const size_t smem = fused_smem(f.slice_cap);
+    cudaError_t err = cudaSuccess;
+#define SMTM_LAUNCH(...) k_lookup_nchw<__VA_ARGS__><<<sm_count, kThreadsFused, smem, st>>>(f)
+    SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
+#undef SMTM_LAUNCH
+    err = cudaGetLastError();
+    ++*launches;
+    *handled = true;
+    return err;
 }
 
 cudaError_t launch_row_norm2(const float* sv, const uint8_t* skip, int B, int D, float* out, cudaStream_t st,

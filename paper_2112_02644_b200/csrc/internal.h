@@ -47,6 +47,12 @@ struct LookupArgs {
     unsigned long long* counters;
 };
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches);
+// Encode + score + exit in one kernel (NCHW shapes the streaming pipeline serves, fast
+// memories of at most 64 entries).  *handled is false when the shape is not served, in which
+// case nothing was launched.  partials: fused_partials_floats() floats; frame_ctr: [max_batch] zeros.
+size_t fused_partials_floats(int max_batch, int k_max);
+cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float* partials, int* frame_ctr,
+                                int sm_count, cudaStream_t st, int64_t* launches, bool* handled);
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,
                                cudaStream_t st, int64_t* launches);
 

@@ -1,0 +1,94 @@
+// Decision logic shared by the lookup kernels: ranking, top-1 / top-2, the margin ratio of
+// Eq. 2 / Eq. 4 and the exit rule (Sec. 4.2, Sec. 5).
+#pragma once
+
+#include <math.h>
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace smtm {
+
+// Ranking used for top-1 / top-2: NaN ranks last, larger value first, ties -> lower class id.
+__device__ __forceinline__ bool ranks_before(float va, int ida, float vb, int idb) {
+    const bool na = isnan(va), nb = isnan(vb);
+    if (na != nb) return nb;
+    if (!na && va != vb) return va > vb;
+    return ida < idb;
+}
+
+struct Top2 {
+    float v1, v2;
+    int id1, id2;  // class ids, -1 = absent
+};
+
+__device__ __forceinline__ void top2_push(Top2& t, float v, int id) {
+    if (t.id1 < 0 || ranks_before(v, id, t.v1, t.id1)) {
+        t.v2 = t.v1; t.id2 = t.id1;
+        t.v1 = v; t.id1 = id;
+    } else if (t.id2 < 0 || ranks_before(v, id, t.v2, t.id2)) {
+        t.v2 = v; t.id2 = id;
+    }
+}
+
+// Best two of the values v[0..k) with class ids ids[0..k); executed by one full warp.
+__device__ __forceinline__ Top2 warp_top2(const float* v, const int32_t* ids, int k, int lane) {
+    Top2 t{0.f, 0.f, -1, -1};
+    for (int j = lane; j < k; j += kWarp) top2_push(t, v[j], ids[j]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov1 = __shfl_xor_sync(kFull, t.v1, o), ov2 = __shfl_xor_sync(kFull, t.v2, o);
+        const int oi1 = __shfl_xor_sync(kFull, t.id1, o), oi2 = __shfl_xor_sync(kFull, t.id2, o);
+        if (oi1 >= 0) top2_push(t, ov1, oi1);
+        if (oi2 >= 0) top2_push(t, ov2, oi2);
+    }
+    return t;
+}
+
+// (top - second) / second with the sign cases: top <= 0 -> 0; second <= 0 < top -> +inf.
+__device__ __forceinline__ float ratio_margin(float top, float second) {
+    if (!(top > 0.f)) return 0.f;
+    if (!(second > 0.f)) return INFINITY;
+    return __fdiv_rn(__fsub_rn(top, second), second);
+}
+
+// Executed by one full warp once the similarities of frame b are known: s_cur[j] (this
+// layer, Eq. 1) and s_acc[j] (cumulative, Eq. 3) for the k slots whose classes are mem[j].
+// Selects the two best of each, evaluates Eq. 4 / Eq. 2 and the exit rule in fp32, and
+// writes the frame's outputs and the counters.
+__device__ __forceinline__ void decide_frame(const LookupArgs& a, int b, const float* s_cur, const float* s_acc,
+                                             const int32_t* mem, int k, int lane) {
+    const Top2 ta = warp_top2(s_acc, mem, k, lane);
+    const Top2 ts = warp_top2(s_cur, mem, k, lane);
+    if (lane != 0) return;
+    float ac = 0.f, sep = 0.f;
+    bool leave = false;
+    if (ta.id2 >= 0) {
+        ac = ratio_margin(ta.v1, ta.v2);   // Eq. 4
+        sep = ratio_margin(ts.v1, ts.v2);  // Eq. 2
+        leave = (ta.v1 > 0.f) && (__fsub_rn(ta.v1, ta.v2) > __fmul_rn(a.tau, fmaxf(ta.v2, 0.f)));
+    }
+    if (a.ac) a.ac[(size_t)b * a.L + a.layer] = ac;
+    if (a.sep) a.sep[(size_t)b * a.L + a.layer] = sep;
+    if (a.top) {
+        a.top[2 * b] = ta.id1;
+        a.top[2 * b + 1] = ta.id2;
+    }
+    atomicAdd(&a.counters[SMTM_CTR_LOOKUPS], 1ull);
+    if (isfinite(ac) && fabsf(ac - a.tau) <= 1e-4f) atomicAdd(&a.counters[SMTM_CTR_NEAR], 1ull);
+    if (leave) {
+        a.exit_layer[b] = a.layer + 1;
+        a.pred[b] = ta.id1;
+        __threadfence();  // whoever sees the flag also sees the layer it was set at
+        a.done[b] = 1;
+        atomicAdd(&a.counters[SMTM_CTR_EXITS + a.layer], 1ull);
+    }
+}
+
+// Eq. 1 from a dot product and the two lengths; a zero-length vector is similar to nothing.
+__device__ __forceinline__ float cosine_from(float dot, float sv_norm2, float center_len) {
+    return (sv_norm2 == 0.f || center_len == 0.f) ? 0.f
+                                                  : __fdiv_rn(dot, __fmul_rn(__fsqrt_rn(sv_norm2), center_len));
+}
+
+}  // namespace smtm

@@ -22,33 +22,41 @@ __device__ __forceinline__ int final_label(const UpdateArgs& a, int b) {
 __device__ __forceinline__ int stop_layer(const UpdateArgs& a, int b) { return a.done[b] ? a.exit_layer[b] : a.L; }
 
 constexpr int kUpdThreads = 256;
-constexpr int kTile = 1024;  // frames staged per pass by a table CTA
+constexpr int kSliceCols = kUpdThreads * 4;  // columns of a centre handled by one CTA (one float4 per thread)
 
-// blockIdx.x <  S          : frequency / time-stamp tables of stream blockIdx.x
-// blockIdx.x >= S          : centre of (class, layer) = divmod(blockIdx.x - S, L)
+// Compacts, in ascending frame index, the frames of [t0, t0 + kUpdThreads) for which `hit`
+// is set into list[0..cnt); returns cnt (the same in every thread).
+__device__ __forceinline__ int compact_tile(int hit, int value, int* list, int* s_scan) {
+    int cnt;
+    const int pos = block_exclusive_scan(hit, s_scan, &cnt);
+    if (cnt) {
+        __syncthreads();  // the previous tile's readers are done with list
+        if (hit) list[pos] = value;
+        __syncthreads();
+    }
+    return cnt;
+}
+
+// blockIdx.x <  S : frequency / time-stamp tables of stream blockIdx.x
+// blockIdx.x >= S : centre of (class, layer) = divmod(blockIdx.x - S, L)
 __global__ void __launch_bounds__(kUpdThreads) k_update(const UpdateArgs a) {
-    __shared__ int s_sid[kTile];
-    __shared__ int s_lab[kTile];
+    __shared__ int s_list[kUpdThreads];
     __shared__ int s_scan[33];
     __shared__ float s_red[32];
     const int tid = threadIdx.x;
 
     if (int(blockIdx.x) < a.S) {
-        // ---- Sec. 6.1: each thread replays the batch for its own classes -------------------
+        // ---- Sec. 6.1: the stream's frames, in ascending index, replayed per class ----------
         const int s = blockIdx.x;
-        for (int t0 = 0; t0 < a.B; t0 += kTile) {
-            const int nt = min(kTile, a.B - t0);
-            __syncthreads();
-            for (int i = tid; i < nt; i += kUpdThreads) {
-                s_sid[i] = a.stream_id ? a.stream_id[t0 + i] : 0;
-                s_lab[i] = final_label(a, t0 + i);
-            }
-            __syncthreads();
+        for (int t0 = 0; t0 < a.B; t0 += kUpdThreads) {
+            const int b = t0 + tid;
+            const int hit = (b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
+            const int cnt = compact_tile(hit, hit ? final_label(a, b) : -1, s_list, s_scan);
+            if (cnt == 0) continue;
             for (int c = tid; c < a.n; c += kUpdThreads) {
                 int f = a.ft[(size_t)s * a.n + c], t = a.ts[(size_t)s * a.n + c];
-                for (int i = 0; i < nt; ++i) {
-                    if (s_sid[i] != s) continue;
-                    if (s_lab[i] == c) {
+                for (int i = 0; i < cnt; ++i) {
+                    if (s_list[i] == c) {
                         f = min(f + 1, kFtMax);
                         t = 0;
                     } else if (t < INT32_MAX) {
@@ -66,54 +74,47 @@ __global__ void __launch_bounds__(kUpdThreads) k_update(const UpdateArgs a) {
     const int job = blockIdx.x - a.S;
     const int cls = job / a.L, l0 = job - cls * a.L;  // l0 is 0-based here; the paper's l0 is l0 + 1
     const int D = a.dims[l0];
+    const bool vec = (D & 3) == 0;  // rows are 16-byte aligned
     const float* sv = a.sv[l0];
     float* cen = a.centers[l0] + (size_t)cls * D;
-    int* list = s_sid;  // matching frames of the current tile, ascending
-
-    constexpr int kCols = 8;  // columns per thread per sweep
+    const float m = float(a.m[l0][cls]);
     float nrm = 0.f;
-    int q_total = 0;
-    for (int d0 = 0; d0 < D; d0 += kUpdThreads * kCols) {
-        float acc[kCols];
-#pragma unroll
-        for (int j = 0; j < kCols; ++j) acc[j] = 0.f;
-        int q = 0;
+    int q = 0;
+    for (int d0 = 0; d0 < D; d0 += kSliceCols) {  // a slice of columns per sweep, four per thread
+        const int d = d0 + tid * 4;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        q = 0;
         for (int t0 = 0; t0 < a.B; t0 += kUpdThreads) {
             const int b = t0 + tid;
             const int hit = (b < a.B && final_label(a, b) == cls && stop_layer(a, b) >= l0 + 1) ? 1 : 0;
-            int cnt;
-            const int pos = block_exclusive_scan(hit, s_scan, &cnt);
-            if (cnt == 0) continue;  // uniform: cnt is the same in every thread
-            __syncthreads();
-            if (hit) list[pos] = b;
-            __syncthreads();
-            for (int i = 0; i < cnt; ++i) {
-                const float* row = sv + (size_t)list[i] * D + d0;
-#pragma unroll
-                for (int j = 0; j < kCols; ++j) {
-                    const int d = d0 + j * kUpdThreads + tid;
-                    if (d < D) acc[j] += row[j * kUpdThreads + tid];
-                }
-            }
+            const int cnt = compact_tile(hit, b, s_list, s_scan);
+            if (cnt == 0) continue;
             q += cnt;
+            if (d >= D) continue;
+            if (vec) {
+#pragma unroll 4
+                for (int i = 0; i < cnt; ++i) {
+                    const float4 r = __ldg(reinterpret_cast<const float4*>(sv + (size_t)s_list[i] * D + d));
+                    acc[0] += r.x; acc[1] += r.y; acc[2] += r.z; acc[3] += r.w;
+                }
+            } else {
+                for (int i = 0; i < cnt; ++i)
+                    for (int j = 0; j < 4; ++j)
+                        if (d + j < D) acc[j] += sv[(size_t)s_list[i] * D + d + j];
+            }
         }
         if (q == 0) return;  // class not seen at this layer in this batch: nothing changes
-        q_total = q;
-        const float m = float(a.m[l0][cls]);
-#pragma unroll
-        for (int j = 0; j < kCols; ++j) {
-            const int d = d0 + j * kUpdThreads + tid;
-            if (d < D) {
-                const float v = __fdiv_rn(__fmaf_rn(cen[d], m, acc[j]), m + float(q));
-                cen[d] = v;
+        for (int j = 0; j < 4; ++j)
+            if (d + j < D) {
+                const float v = __fdiv_rn(__fmaf_rn(cen[d + j], m, acc[j]), m + float(q));
+                cen[d + j] = v;
                 nrm = fmaf(v, v, nrm);
             }
-        }
     }
     nrm = block_sum(nrm, s_red);
     if (tid == 0) {
         a.cnorm[l0][cls] = __fsqrt_rn(nrm);
-        a.m[l0][cls] += (uint32_t)q_total;
+        a.m[l0][cls] += (uint32_t)q;
     }
 }
 
