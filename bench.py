@@ -57,7 +57,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except OSError:
@@ -132,8 +132,7 @@ def run_ours(args):
         smtm.smtm_batch_reset(cache, gb, sh)
         for l in range(w.L):
             smtm.smtm_lookup_exit(cache, l, fmaps[t % T][l], gb, sh)
-        smtm.smtm_cache_update(cache, gb, fbs[t % T], sh)
-        smtm.smtm_cache_resize(cache, sh)
+        smtm.smtm_cache_update_resize(cache, gb, fbs[t % T], sh)
 
     # warm-up on a scratch cache (kernels, clocks), then a fresh cache for the timed steps
     scratch = make_cache(smtm, w, cents, counts)
@@ -162,8 +161,7 @@ def run_ours(args):
         ev1[t].record(stream)
         for l in range(1, w.L):
             smtm.smtm_lookup_exit(cache, l, fmaps[t % T][l], gb, sh)
-        smtm.smtm_cache_update(cache, gb, fbs[t % T], sh)
-        smtm.smtm_cache_resize(cache, sh)
+        smtm.smtm_cache_update_resize(cache, gb, fbs[t % T], sh)
     stop.record(stream)
     torch.cuda.synchronize()
     if world > 1:
@@ -310,7 +308,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--steps", type=int, default=640)
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()

@@ -178,6 +178,13 @@ smtm_status_t smtm_lookup_exit_static(smtm_cache_t* cache, int32_t layer, const 
 smtm_status_t smtm_cache_update(smtm_cache_t* cache, const smtm_batch_t* batch,
                                 const int32_t* d_fallback_label, void* stream);
 
+/* smtm_cache_update followed by smtm_cache_resize restricted to the streams that
+ * had at least one frame in the batch, in one pass (the tables of the other
+ * streams did not change, so neither would their fast memories if they were
+ * refreshed after their own last update). */
+smtm_status_t smtm_cache_update_resize(smtm_cache_t* cache, const smtm_batch_t* batch,
+                                       const int32_t* d_fallback_label, void* stream);
+
 /* Eq. 5 and Eq. 6 for every stream: Score_i = FT_i 0.25^floor(TS_i / W) (exact,
  * floor clamped at 12); classes ranked by (score descending, id ascending); the
  * new size is the smallest k in [k_min, k_max] whose k best scores sum to more
@@ -187,8 +194,8 @@ smtm_status_t smtm_cache_resize(smtm_cache_t* cache, void* stream);
 
 /* One whole step from host memory: copies the L feature maps (h_maps[l], host,
  * dtype/layout/shape as in fmaps[l] whose d_data is ignored) to the device,
- * runs smtm_lookup_exit for layers 0..L-1, smtm_cache_update and, if
- * do_resize, smtm_cache_resize, then copies the decisions back.  Synchronises
+ * runs smtm_lookup_exit for layers 0..L-1, then smtm_cache_update_resize if
+ * do_resize else smtm_cache_update, then copies the decisions back.  Synchronises
  * `stream` before returning.  h_stream_id / h_fallback_label may be NULL as in
  * the device calls; h_done [B], h_exit_layer [B], h_pred [B] receive the results.
  * B <= max_batch.  Pinned host buffers make the copies asynchronous. */

@@ -81,6 +81,7 @@ def load_library():
     lib.smtm_lookup_exit_static.argtypes = [vp, i32, ctypes.POINTER(_Fmap), vp, vp, vp, vp, vp]
     lib.smtm_cache_update.argtypes = [vp, ctypes.POINTER(_Batch), vp, vp]
     lib.smtm_cache_resize.argtypes = [vp, vp]
+    lib.smtm_cache_update_resize.argtypes = [vp, ctypes.POINTER(_Batch), vp, vp]
     lib.smtm_step_host.argtypes = [vp, ctypes.POINTER(_Fmap), ctypes.POINTER(vp), vp, vp, i32, vp, vp, vp, vp]
     lib.smtm_cache_get_members.argtypes = [vp, vp, vp]
     lib.smtm_cache_get_centers.argtypes = [vp, i32, vp, vp]
@@ -233,6 +234,11 @@ def smtm_lookup_exit_static(cache: Cache, layer: int, fmap: Fmap, stream_id, exi
 def smtm_cache_update(cache: Cache, batch: Batch, fallback_label=None, stream=None) -> None:
     _check(load_library().smtm_cache_update(cache.handle, ctypes.byref(batch.c), _dptr(fallback_label),
                                             _stream(stream)), "smtm_cache_update")
+
+
+def smtm_cache_update_resize(cache: Cache, batch: Batch, fallback_label=None, stream=None) -> None:
+    _check(load_library().smtm_cache_update_resize(cache.handle, ctypes.byref(batch.c), _dptr(fallback_label),
+                                                   _stream(stream)), "smtm_cache_update_resize")
 
 
 def smtm_cache_resize(cache: Cache, stream=None) -> None:

@@ -22,6 +22,7 @@ struct smtm_cache {
     int* d_status;
     float* d_partials;  // scratch of the fused lookup: partial dot products per (frame, part)
     int* d_frame_ctr;   // scratch of the fused lookup: parts delivered per frame (zero between launches)
+    int32_t* d_plan;    // scratch of the update: 4 x [max_batch] + [2], see UpdatePlan
     int device, sm_count;
     int64_t launches;
     // device-side carry and staging used only by smtm_step_host (allocated on first use)
@@ -71,6 +72,7 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_status);
     cudaFree(c->d_partials);
     cudaFree(c->d_frame_ctr);
+    cudaFree(c->d_plan);
     cudaFree(c->hb.d_sa);
     cudaFree(c->hb.d_done);
     cudaFree(c->hb.d_exit_layer);
@@ -146,12 +148,35 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     return SMTM_OK;
 }
 
-smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d_fallback, cudaStream_t st) {
+ResizeArgs resize_args(const smtm_cache* c) {
+    ResizeArgs a{};
+    a.S = c->S;
+    a.n = c->n;
+    a.W = c->W;
+    a.k_min = c->k_min;
+    a.k_max = c->k_max;
+    a.cl_num = c->cl_num;
+    a.cl_den = c->cl_den;
+    a.ft = c->d_ft;
+    a.ts = c->d_ts;
+    a.members = c->d_members;
+    a.k = c->d_k;
+    return a;
+}
+
+smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d_fallback, bool with_resize,
+                          cudaStream_t st) {
     UpdateArgs a{};
     a.B = b->B;
     a.S = c->S;
     a.n = c->n;
     a.L = c->L;
+    const size_t mb = size_t(c->max_batch);
+    a.plan.final_label = c->d_plan;
+    a.plan.stop_layer = c->d_plan + mb;
+    a.plan.first_of_class = c->d_plan + 2 * mb;
+    a.plan.first_of_stream = c->d_plan + 3 * mb;
+    a.plan.counts = c->d_plan + 4 * mb;
     a.stream_id = b->d_stream_id;
     a.done = b->d_done;
     a.exit_layer = b->d_exit_layer;
@@ -166,24 +191,22 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
         a.cnorm[l] = c->d_cnorm[l];
         a.m[l] = c->d_m[l];
     }
-    SMTM_CUDA(launch_update(a, st, &c->launches));
+    const ResizeArgs rz = resize_args(c);
+    SMTM_CUDA(launch_update(a, with_resize ? &rz : nullptr, st, &c->launches));
     return SMTM_OK;
 }
 
 smtm_status_t resize_impl(smtm_cache* c, cudaStream_t st) {
-    ResizeArgs a{};
-    a.S = c->S;
-    a.n = c->n;
-    a.W = c->W;
-    a.k_min = c->k_min;
-    a.k_max = c->k_max;
-    a.cl_num = c->cl_num;
-    a.cl_den = c->cl_den;
-    a.ft = c->d_ft;
-    a.ts = c->d_ts;
-    a.members = c->d_members;
-    a.k = c->d_k;
-    SMTM_CUDA(launch_resize(a, st, &c->launches));
+    SMTM_CUDA(launch_resize(resize_args(c), st, &c->launches));
+    return SMTM_OK;
+}
+
+smtm_status_t check_update(const smtm_cache* c, const smtm_batch_t* b) {
+    if (!c) return SMTM_ERR_INVALID_ARG;
+    const smtm_status_t s = check_batch(c, b);
+    if (s != SMTM_OK) return s;
+    for (int l = 0; l < c->L; ++l)
+        if (!b->d_sv[l]) return SMTM_ERR_INVALID_ARG;
     return SMTM_OK;
 }
 
@@ -255,6 +278,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     ok = ok && dev_alloc(&c->d_status, 1) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_partials, fused_partials_floats(c->max_batch, c->k_max)) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_frame_ctr, size_t(c->max_batch)) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_plan, 4 * size_t(c->max_batch) + 2) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();
         free_all(c);
@@ -337,12 +361,16 @@ smtm_status_t smtm_lookup_exit(smtm_cache_t* c, int32_t layer, const smtm_fmap_t
 
 smtm_status_t smtm_cache_update(smtm_cache_t* c, const smtm_batch_t* b, const int32_t* d_fallback_label,
                                 void* stream) {
-    if (!c) return SMTM_ERR_INVALID_ARG;
-    smtm_status_t s = check_batch(c, b);
+    const smtm_status_t s = check_update(c, b);
     if (s != SMTM_OK) return s;
-    for (int l = 0; l < c->L; ++l)
-        if (!b->d_sv[l]) return SMTM_ERR_INVALID_ARG;
-    return update_impl(c, b, d_fallback_label, static_cast<cudaStream_t>(stream));
+    return update_impl(c, b, d_fallback_label, false, static_cast<cudaStream_t>(stream));
+}
+
+smtm_status_t smtm_cache_update_resize(smtm_cache_t* c, const smtm_batch_t* b, const int32_t* d_fallback_label,
+                                       void* stream) {
+    const smtm_status_t s = check_update(c, b);
+    if (s != SMTM_OK) return s;
+    return update_impl(c, b, d_fallback_label, true, static_cast<cudaStream_t>(stream));
 }
 
 smtm_status_t smtm_cache_resize(smtm_cache_t* c, void* stream) {
@@ -412,9 +440,8 @@ smtm_status_t smtm_step_host(smtm_cache_t* c, const smtm_fmap_t* fmaps, const vo
         smtm_status_t s = lookup_impl(c, l, &f, &b, st);
         if (s != SMTM_OK) return s;
     }
-    smtm_status_t s = update_impl(c, &b, h_fallback_label ? c->d_fallback : nullptr, st);
+    smtm_status_t s = update_impl(c, &b, h_fallback_label ? c->d_fallback : nullptr, do_resize != 0, st);
     if (s != SMTM_OK) return s;
-    if (do_resize && (s = resize_impl(c, st)) != SMTM_OK) return s;
     SMTM_CUDA(cudaMemcpyAsync(h_done, b.d_done, size_t(B), cudaMemcpyDeviceToHost, st));
     SMTM_CUDA(cudaMemcpyAsync(h_exit_layer, b.d_exit_layer, size_t(B) * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     SMTM_CUDA(cudaMemcpyAsync(h_pred, b.d_pred, size_t(B) * sizeof(int32_t), cudaMemcpyDeviceToHost, st));

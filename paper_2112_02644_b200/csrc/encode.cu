@@ -21,6 +21,8 @@
 // directly and the phases are combined through shared memory in ascending order.
 // Any other shape falls back to a plain thread-per-(frame, channel) loop.
 #include <algorithm>
+#include <cmath>
+#include <cstdlib>
 
 #include "lookup_common.cuh"
 
@@ -48,6 +50,7 @@ struct NchwParams {
     float inv_hw;
     int team;                // team-per-channel: lanes per channel (power of two)
     int vec_per_channel;     // team-per-channel: 16-byte vectors per channel
+    int max_in_flight;       // copies the producer keeps outstanding (<= kStages)
 };
 
 // ---- reducers --------------------------------------------------------------------------
@@ -168,6 +171,13 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
                     failed = true;
                     break;
                 }
+                if (it >= p.max_in_flight) {  // bound the bytes in flight: wait for an older copy to land
+                    const int old = it - p.max_in_flight;
+                    if (!mbar_wait_bounded(&full[old % kStages], (old / kStages) & 1, p.status)) {
+                        failed = true;
+                        break;
+                    }
+                }
                 const uint32_t bytes = uint32_t(nch) * uint32_t(p.ch_bytes);
                 mbar_expect_tx(&full[stage], bytes);
                 bulk_load(stages + size_t(stage) * kStageCap,
@@ -207,26 +217,38 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
 // the spot; otherwise the partials go to global scratch and the CTA that delivers a frame's
 // last part adds them up in part order and decides.  No floating-point atomics anywhere:
 // the evaluation order of every sum is fixed.
-constexpr int kScorers = 4;
-constexpr int kThreadsFused = (kConsumers + 1 + kScorers) * kWarp;
-constexpr int kFusedMaxK = 64;      // fast-memory capacity the fused kernel supports
+constexpr int kReducersF = 4;       // reducer warps of the fused kernel; stage s belongs to warp s % kReducersF
+constexpr int kDotWarps = 8;        // warps that share the dot products of a unit, slot j going to warp j % 8
+constexpr int kFinalizers = 2;      // warps that complete units alternately (partials, Eq. 1-4, decision)
+constexpr int kSvBufs = 4;          // shared-memory slices; unit u passes through buffer u % kSvBufs
+constexpr int kThreadsFused = (kReducersF + 1 + kDotWarps + kFinalizers) * kWarp;
+constexpr int kFusedMaxK = 64;      // fast-memory capacity the fused kernel supports (two slots per lane)
 constexpr int kMaxUnits = 1024;     // units per CTA
-constexpr int kMaxSlice = 2048;     // floats of a semantic-vector slice held in shared memory
+constexpr int kMaxSlice = 1024;     // floats of a semantic-vector slice (eight 16-byte vectors per lane)
 constexpr int kMaxParts = 16;
+static_assert(kStages % kReducersF == 0, "stage ownership must be periodic");
 
 struct FusedParams {
     NchwParams e;
     LookupArgs a;
     int parts;            // P: parts per frame (divides chunks_per_frame)
     int chunks_per_unit;  // chunks_per_frame / P
-    int slice_cap;        // channels of a full slice = chunks_per_unit * chunk_channels
+    int slice_cap;        // channels of a full slice = chunks_per_unit * chunk_channels (multiple of 4)
     float* partials;      // [B][P][k_max + 1], used when P > 1
     int* frame_ctr;       // [B] parts delivered so far (returns to zero)
 };
 
 constexpr size_t fused_smem(int slice_cap) {
-    return size_t(kStages) * kStageCap + 2 * size_t(slice_cap) * 4 + 2 * (kFusedMaxK + 1) * 4 + 2 * kFusedMaxK * 4 +
-           kMaxUnits * 4 + (2 * kStages + 5) * 8 + 40 * 4 + 192;
+    return size_t(kStages) * kStageCap + size_t(kSvBufs) * size_t(slice_cap) * 4 + kMaxUnits * 4 +
+           kFinalizers * (kFusedMaxK + 1) * 4 + (2 * kStages + 2 * kSvBufs + 2 * kFinalizers) * 8 + 40 * 4 + 192;
+}
+
+// acq_rel so that the partials written before it (by this warp) are visible to whoever
+// observes the count, and the partials of the parts counted before are visible to us.
+__device__ __forceinline__ int atomic_add_acq_rel(int* addr, int v) {
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
+    return old;
 }
 
 template <class R>
@@ -234,18 +256,17 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     uint8_t* stages = base;
-    float* sv_s = reinterpret_cast<float*>(base + size_t(kStages) * kStageCap);  // [2][slice_cap]
-    float* s_dot = sv_s + 2 * f.slice_cap;                                       // [2][kFusedMaxK + 1]
-    float* s_cur = s_dot + 2 * (kFusedMaxK + 1);                                 // [kFusedMaxK]
-    float* s_acc = s_cur + kFusedMaxK;                                           // [kFusedMaxK]
-    int* my_units = reinterpret_cast<int*>(s_acc + kFusedMaxK);                  // [kMaxUnits]
+    float* sv_s = reinterpret_cast<float*>(base + size_t(kStages) * kStageCap);  // [kSvBufs][slice_cap]
+    float* s_dot = sv_s + kSvBufs * f.slice_cap;                                 // [kFinalizers][kFusedMaxK + 1]
+    int* my_units = reinterpret_cast<int*>(s_dot + kFinalizers * (kFusedMaxK + 1));  // [kMaxUnits]
     int* s_scan = my_units + kMaxUnits;                                          // [40]
     uint64_t* full = reinterpret_cast<uint64_t*>(
         (reinterpret_cast<uintptr_t>(s_scan + 40) + 7) & ~uintptr_t(7));         // [kStages]
     uint64_t* empty = full + kStages;                                            // [kStages]
-    uint64_t* sv_full = empty + kStages;                                         // [2]
-    uint64_t* sv_empty = sv_full + 2;                                            // [2]
-    uint64_t* sc_bar = sv_empty + 2;                                             // [1]
+    uint64_t* sv_full = empty + kStages;                                         // [kSvBufs]  slice written
+    uint64_t* sv_empty = sv_full + kSvBufs;                                      // [kSvBufs]  slice read by all dot warps
+    uint64_t* dot_full = sv_empty + kSvBufs;                                     // [kFinalizers] dot products written
+    uint64_t* dot_empty = dot_full + kFinalizers;                                // [kFinalizers] ... and taken
 
     const NchwParams& p = f.e;
     const LookupArgs& a = f.a;
@@ -256,11 +277,14 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < kSvBufs; ++s) {
             mbar_init(&sv_full[s], cpu);
-            mbar_init(&sv_empty[s], kScorers);
+            mbar_init(&sv_empty[s], kDotWarps);
         }
-        mbar_init(sc_bar, kScorers);
+        for (int s = 0; s < kFinalizers; ++s) {
+            mbar_init(&dot_full[s], kDotWarps);
+            mbar_init(&dot_empty[s], 1);
+        }
         mbar_init_fence();
     }
 
@@ -294,25 +318,26 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
     const int n_chunks = nu * cpu;
     bool failed = false;
     int issued = 0;
-    if (warp < kConsumers) {
-        // ---- reducers: warp w owns stage w and the chunks it, it + kConsumers, ... ------------
-        for (int it = warp; it < n_chunks; it += kConsumers) {
+    if (warp < kReducersF) {
+        // ---- reducers: warp w owns the stages w, w + kReducersF, ... -----------------------------
+        for (int it = warp; it < n_chunks; it += kReducersF) {
             const int i = it / cpu, c = it - i * cpu;
             const int unit = my_units[i], b = unit / kMaxParts, part = unit % kMaxParts;
             const int c0 = (part * cpu + c) * p.chunk_channels;
             const int nch = min(p.chunk_channels, p.C - c0);
-            const int buf = i & 1;
-            if (i >= 2 && !mbar_wait_bounded(&sv_empty[buf], ((i >> 1) - 1) & 1, p.status)) { failed = true; break; }
-            if (!mbar_wait_bounded(&full[warp], (it / kStages) & 1, p.status)) { failed = true; break; }
-            R::run(stages + size_t(warp) * kStageCap, nch, lane, p.sv + (long long)b * p.C + c0,
+            const int stage = it % kStages;
+            const int buf = i % kSvBufs, round = i / kSvBufs;
+            if (round > 0 && !mbar_wait_bounded(&sv_empty[buf], (round - 1) & 1, p.status)) { failed = true; break; }
+            if (!mbar_wait_bounded(&full[stage], (it / kStages) & 1, p.status)) { failed = true; break; }
+            R::run(stages + size_t(stage) * kStageCap, nch, lane, p.sv + (long long)b * p.C + c0,
                    sv_s + buf * f.slice_cap + c * p.chunk_channels, p.inv_hw, p);
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&empty[warp]);
+                mbar_arrive(&empty[stage]);
                 mbar_arrive(&sv_full[buf]);
             }
         }
-    } else if (warp == kConsumers) {
+    } else if (warp == kReducersF) {
         // ---- producer -------------------------------------------------------------------------
         if (lane == 0) {
             for (int it = 0; it < n_chunks; ++it) {
@@ -323,6 +348,10 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
                 const int stage = it % kStages;
                 const uint32_t use = uint32_t(it / kStages);
                 if (use > 0 && !mbar_wait_bounded(&empty[stage], (use - 1) & 1, p.status)) { failed = true; break; }
+                if (it >= p.max_in_flight) {  // bound the bytes in flight: wait for an older copy to land
+                    const int old = it - p.max_in_flight;
+                    if (!mbar_wait_bounded(&full[old % kStages], (old / kStages) & 1, p.status)) { failed = true; break; }
+                }
                 const uint32_t bytes = uint32_t(nch) * uint32_t(p.ch_bytes);
                 mbar_expect_tx(&full[stage], bytes);
                 bulk_load(stages + size_t(stage) * kStageCap,
@@ -330,102 +359,157 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
                 issued = it + 1;
             }
         }
-    } else {
-        // ---- scorers ----------------------------------------------------------------------------
-        const int sw = warp - kConsumers - 1;
-        const float weight = float(1u << a.layer);  // 2^(l-1) with l = layer + 1
-        uint32_t sc_phase = 0;
-        for (int i = 0; i < nu; ++i) {
-            const int unit = my_units[i], b = unit / kMaxParts, part = unit % kMaxParts;
-            const int buf = i & 1;
-            const int sb = part * f.slice_cap;                 // first channel of the slice
-            const int Dp = min(f.slice_cap, p.C - sb);         // channels in it
+    } else if (warp < kReducersF + 1 + kDotWarps) {
+        // ---- dot warps: all of them work on unit u together, slot j on warp j % kDotWarps --------
+        const int dw = warp - kReducersF - 1;
+        // fast memory of the unit in hand, fetched one unit ahead
+        int nx_k = 0, nx_ids[2] = {0, 0};
+        if (nu > 0) {
+            const int b = my_units[0] / kMaxParts;
             const int sid = a.stream_id ? a.stream_id[b] : 0;
-            const int k = min(a.k[sid], kFusedMaxK);
+            nx_k = min(a.k[sid], kFusedMaxK);
             const int32_t* mem = a.members + (size_t)sid * a.k_max;
-            const float* v = sv_s + buf * f.slice_cap;
-            if (!mbar_wait_bounded(&sv_full[buf], (i >> 1) & 1, p.status)) { failed = true; break; }
-            const bool vec = ((p.C | sb | Dp) & 3) == 0;
-            const int n4 = vec ? Dp >> 2 : 0;
-            const float4* v4 = reinterpret_cast<const float4*>(v);
-            float* out = P == 1 ? s_dot + buf * (kFusedMaxK + 1)
-                                : f.partials + ((size_t)b * P + part) * (a.k_max + 1);
-            const int norm_slot = P == 1 ? kFusedMaxK : a.k_max;
-            if (sw == 0) {  // partial squared length of the semantic vector
-                float n0 = 0.f, n1 = 0.f, n2 = 0.f, n3 = 0.f;
+            nx_ids[0] = lane < nx_k ? mem[lane] : 0;
+            nx_ids[1] = lane + kWarp < nx_k ? mem[lane + kWarp] : 0;
+        }
+        for (int u = 0; u < nu; ++u) {
+            const int unit = my_units[u], part = unit % kMaxParts;
+            const int sb = part * f.slice_cap;          // first channel of the slice
+            const int Dp = min(f.slice_cap, p.C - sb);  // channels in it (a multiple of 4)
+            const int n4 = Dp >> 2;
+            const int k = nx_k;
+            const int ids[2] = {nx_ids[0], nx_ids[1]};  // lane l knows the classes of slots l and l + 32
+            const int buf = u % kSvBufs, db = u % kFinalizers;
+            int nb_sid = 0;
+            if (u + 1 < nu) {
+                const int nb = my_units[u + 1] / kMaxParts;
+                nb_sid = a.stream_id ? a.stream_id[nb] : 0;  // in flight while this unit is scored
+            }
+            if (!mbar_wait_bounded(&sv_full[buf], (u / kSvBufs) & 1, p.status)) { failed = true; break; }
+            if (u >= kFinalizers &&
+                !mbar_wait_bounded(&dot_empty[db], (u / kFinalizers - 1) & 1, p.status)) { failed = true; break; }
+            const float4* v4 = reinterpret_cast<const float4*>(sv_s + buf * f.slice_cap);
+            float* out = s_dot + db * (kFusedMaxK + 1);
+            if (dw == kDotWarps - 1) {  // partial squared length of the semantic vector
+                float nn = 0.f;
                 for (int q = lane; q < n4; q += kWarp) {
                     const float4 x = v4[q];
-                    n0 = fmaf(x.x, x.x, n0); n1 = fmaf(x.y, x.y, n1); n2 = fmaf(x.z, x.z, n2); n3 = fmaf(x.w, x.w, n3);
+                    nn = fmaf(x.x, x.x, nn); nn = fmaf(x.y, x.y, nn); nn = fmaf(x.z, x.z, nn); nn = fmaf(x.w, x.w, nn);
                 }
-                for (int q = (n4 << 2) + lane; q < Dp; q += kWarp) n0 = fmaf(v[q], v[q], n0);
-                float nn = (n0 + n1) + (n2 + n3);
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(kFull, nn, o);
-                if (lane == 0) out[norm_slot] = nn;
+                if (lane == 0) out[kFusedMaxK] = nn;
             }
-            for (int j = sw; j < k; j += kScorers) {  // partial dot products, Eq. 1's numerator
-                const float* crow = a.centers + (size_t)mem[j] * p.C + sb;
-                const float4* c4 = reinterpret_cast<const float4*>(crow);
-                float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
-                for (int q = lane; q < n4; q += kWarp) {
-                    const float4 cc = __ldg(c4 + q);
-                    const float4 x = v4[q];
-                    d0 = fmaf(cc.x, x.x, d0); d1 = fmaf(cc.y, x.y, d1); d2 = fmaf(cc.z, x.z, d2); d3 = fmaf(cc.w, x.w, d3);
-                }
-                for (int q = (n4 << 2) + lane; q < Dp; q += kWarp) d0 = fmaf(crow[q], v[q], d0);
-                float dot = (d0 + d1) + (d2 + d3);
+            for (int j = dw; j < k; j += kDotWarps) {  // partial dot product of slot j (Eq. 1's numerator)
+                const int cls = __shfl_sync(kFull, (j & 32) ? ids[1] : ids[0], j & 31);
+                const float4* crow = reinterpret_cast<const float4*>(a.centers + (size_t)cls * p.C + sb);
+                float4 cc[kMaxSlice / 4 / kWarp];  // every load of the slot in flight at once
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(kFull, dot, o);
-                if (lane == 0) out[j] = dot;
+                for (int r = 0; r < kMaxSlice / 4 / kWarp; ++r) {
+                    const int q = lane + r * kWarp;
+                    cc[r] = q < n4 ? __ldg(crow + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                float d = 0.f;
+#pragma unroll
+                for (int r = 0; r < kMaxSlice / 4 / kWarp; ++r) {
+                    const int q = lane + r * kWarp;
+                    if (q < n4) {
+                        const float4 x = v4[q];
+                        d = fmaf(cc[r].x, x.x, d); d = fmaf(cc[r].y, x.y, d);
+                        d = fmaf(cc[r].z, x.z, d); d = fmaf(cc[r].w, x.w, d);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(kFull, d, o);
+                if (lane == 0) out[j] = d;
             }
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&sv_empty[buf]);  // done reading the slice
-                mbar_arrive(sc_bar);
+                mbar_arrive(&sv_empty[buf]);
+                mbar_arrive(&dot_full[db]);
             }
-            if (!mbar_wait_bounded(sc_bar, sc_phase, p.status)) { failed = true; break; }
-            sc_phase ^= 1;
-            if (sw != 0) continue;
+            if (u + 1 < nu) {  // fast memory of the next unit (its stream id has arrived by now)
+                nx_k = min(a.k[nb_sid], kFusedMaxK);
+                const int32_t* mem = a.members + (size_t)nb_sid * a.k_max;
+                nx_ids[0] = lane < nx_k ? mem[lane] : 0;
+                nx_ids[1] = lane + kWarp < nx_k ? mem[lane + kWarp] : 0;
+            }
+        }
+    } else {
+        // ---- finalizers: warp fw completes the units fw, fw + kFinalizers, ... ---------------------
+        const int fw = warp - kReducersF - 1 - kDotWarps;
+        const float weight = float(1u << a.layer);  // 2^(l-1) with l = layer + 1
+        const float* in = s_dot + fw * (kFusedMaxK + 1);
+        for (int u = fw; u < nu; u += kFinalizers) {
+            const int unit = my_units[u], b = unit / kMaxParts, part = unit % kMaxParts;
+            // everything that does not depend on the dot products is fetched while they are computed
+            const int sid = a.stream_id ? a.stream_id[b] : 0;
+            const int k = min(a.k[sid], kFusedMaxK);
+            const int32_t* mem = a.members + (size_t)sid * a.k_max;
+            int ids[2];
+            float clen[2], sa_old[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = lane + h * kWarp;
+                ids[h] = j < k ? mem[j] : 0;
+                clen[h] = j < k ? a.cnorm[ids[h]] : 0.f;
+                sa_old[h] = j < k ? a.sa[(size_t)b * a.k_max + j] : 0.f;
+            }
+            if (!mbar_wait_bounded(&dot_full[fw], (u / kFinalizers) & 1, p.status)) { failed = true; break; }
+            float dots[2], nn = in[kFusedMaxK];
+            dots[0] = lane < k ? in[lane] : 0.f;
+            dots[1] = lane + kWarp < k ? in[lane + kWarp] : 0.f;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&dot_empty[fw]);
 
-            // scorer warp 0: is the frame complete?  (with P > 1: did we deliver its last part?)
-            int last = 1;
+            // is the frame complete?  (with P > 1: did we deliver its last part?)
             if (P > 1) {
+                float* out = f.partials + ((size_t)b * P + part) * (a.k_max + 1);
+                if (lane < k) out[lane] = dots[0];
+                if (lane + kWarp < k) out[lane + kWarp] = dots[1];
+                if (lane == 0) out[a.k_max] = nn;
+                __syncwarp();
+                int last = 0;
                 if (lane == 0) {
-                    __threadfence();
-                    last = atomicAdd(&f.frame_ctr[b], 1) == P - 1 ? 1 : 0;
+                    last = atomic_add_acq_rel(&f.frame_ctr[b], 1) == P - 1 ? 1 : 0;
                     if (last) f.frame_ctr[b] = 0;
-                    __threadfence();
                 }
                 last = __shfl_sync(kFull, last, 0);
-            }
-            if (!last) continue;
-            float nrm = 0.f;
-            if (P == 1) {
-                nrm = out[norm_slot];
-            } else {
-                for (int q = 0; q < P; ++q) nrm += __ldcg(f.partials + ((size_t)b * P + q) * (a.k_max + 1) + a.k_max);
-            }
-            for (int j = lane; j < k; j += kWarp) {
-                float dot = 0.f;
-                if (P == 1) {
-                    dot = out[j];
-                } else {
-                    for (int q = 0; q < P; ++q) dot += __ldcg(f.partials + ((size_t)b * P + q) * (a.k_max + 1) + j);
+                if (!last) continue;
+                // add the parts up in part order
+                float pn[kMaxParts], p0[kMaxParts], p1[kMaxParts];
+#pragma unroll
+                for (int q = 0; q < kMaxParts; ++q) {
+                    const float* src = f.partials + ((size_t)b * P + q) * (a.k_max + 1);
+                    pn[q] = q < P ? __ldcg(src + a.k_max) : 0.f;
+                    p0[q] = (q < P && lane < k) ? __ldcg(src + lane) : 0.f;
+                    p1[q] = (q < P && lane + kWarp < k) ? __ldcg(src + lane + kWarp) : 0.f;
                 }
-                const float s = cosine_from(dot, nrm, a.cnorm[mem[j]]);                    // Eq. 1
-                const float acc = __fmaf_rn(s, weight, a.sa[(size_t)b * a.k_max + j]);     // Eq. 3
-                a.sa[(size_t)b * a.k_max + j] = acc;
-                s_cur[j] = s;
-                s_acc[j] = acc;
+                nn = 0.f; dots[0] = 0.f; dots[1] = 0.f;
+#pragma unroll
+                for (int q = 0; q < kMaxParts; ++q) {
+                    if (q < P) { nn += pn[q]; dots[0] += p0[q]; dots[1] += p1[q]; }
+                }
             }
-            __syncwarp();
-            decide_frame(a, b, s_cur, s_acc, mem, k, lane);
+            float s_cur[2] = {0.f, 0.f}, s_acc[2] = {0.f, 0.f};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = lane + h * kWarp;
+                if (j < k) {
+                    s_cur[h] = cosine_from(dots[h], nn, clen[h]);        // Eq. 1
+                    s_acc[h] = __fmaf_rn(s_cur[h], weight, sa_old[h]);   // Eq. 3
+                    a.sa[(size_t)b * a.k_max + j] = s_acc[h];
+                }
+            }
+            const Top2 ta = warp_top2_regs(s_acc, ids, k, lane);
+            const Top2 ts = warp_top2_regs(s_cur, ids, k, lane);
+            if (lane == 0) decide_from_top2(a, b, ta, ts);
             __syncwarp();
         }
     }
     // No thread leaves before every copy that was issued has landed.
     const int any_failed = __syncthreads_or(failed ? 1 : 0);
-    if (any_failed && warp == kConsumers && lane == 0) {
+    if (any_failed && warp == kReducersF && lane == 0) {
         for (int s = 0; s < kStages && s < issued; ++s) {
             const uint32_t last_use = uint32_t((issued - 1 - s) / kStages);
             mbar_wait_bounded(&full[s], last_use & 1, p.status);
@@ -564,6 +648,15 @@ int pow2_floor(int v) {
 
 
 
+int in_flight_limit() {
+    static int v = [] {
+        const char* e = getenv("SMTM_INFLIGHT");
+        const int n = e ? atoi(e) : kStages;
+        return std::max(1, std::min(n, kStages));
+    }();
+    return v;
+}
+
 // Which reducer a shape is served by, and the chunking that goes with it.
 enum Reducer { kNone, kUnitBf16x49, kUnitBf16x196, kUnitF16x49, kUnitF16x196, kUnitF32x49, kTeamF32, kTeamF16, kTeamBf16 };
 
@@ -579,6 +672,7 @@ Reducer plan_nchw(const EncodeArgs& a, NchwParams* p) {
     p->ch_bytes = HW * es;
     p->frame_bytes = (long long)a.C * p->ch_bytes;
     p->inv_hw = 1.0f / float(HW);
+    p->max_in_flight = in_flight_limit();
     // unit-per-lane shapes (compile-time H*W)
     int G = 0;
     if ((HW == 49 || HW == 196) && es == 2) G = HW == 49 ? 8 : 2;
@@ -674,15 +768,30 @@ cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float*
     FusedParams f{};
     const Reducer r = plan_nchw(e, &f.e);
     if (r == kNone) return cudaSuccess;
-    // parts per frame: as many as leave at least four chunks per unit; more if a slice would
-    // not fit its shared-memory buffer
+    // Parts per frame.  A unit must fit the scorers' registers (slice <= kMaxSlice channels, a
+    // multiple of 4); among the divisors of the chunk count take the smallest that fills the
+    // last round of units to 95 % (else the best filled), preferring units of >= 4 chunks.
     const int cpf = f.e.chunks_per_frame;
-    int P = 1;
-    for (int d = 1; d <= std::min(cpf, kMaxParts); ++d)
-        if (cpf % d == 0 && cpf / d >= 4) P = d;
-    while (P < cpf && (cpf % P != 0 || (cpf / P) * f.e.chunk_channels > kMaxSlice)) ++P;
-    if (cpf % P != 0 || P > kMaxParts || (cpf / P) * f.e.chunk_channels > kMaxSlice) return cudaSuccess;
-    if (((long long)e.B * P + sm_count - 1) / sm_count > kMaxUnits) return cudaSuccess;
+    if ((e.C & 3) || (f.e.chunk_channels & 3)) return cudaSuccess;
+    const auto pick = [&](int min_chunks) {
+        int best_d = 0;
+        double best_eff = -1.0;
+        for (int d = 1; d <= std::min(cpf, kMaxParts); ++d) {
+            if (cpf % d || cpf / d < min_chunks || (cpf / d) * f.e.chunk_channels > kMaxSlice) continue;
+            if (((long long)e.B * d + sm_count - 1) / sm_count > kMaxUnits) continue;
+            const double rounds = double(e.B) * d / sm_count;
+            const double eff = rounds / std::ceil(rounds);
+            if (eff >= 0.95) return d;
+            if (eff > best_eff + 1e-9) {
+                best_eff = eff;
+                best_d = d;
+            }
+        }
+        return (best_eff >= 0.8 || min_chunks <= 1) ? best_d : 0;
+    };
+    int P = pick(4);
+    if (P == 0) P = pick(1);
+    if (P <= 0) return cudaSuccess;
     f.a = a;
     f.parts = P;
     f.chunks_per_unit = cpf / P;

@@ -60,8 +60,18 @@ cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, in
 cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm, cudaStream_t st,
                                 int64_t* launches);
 
+// Scratch written by the planning kernel of an update (all device, sized for max_batch).
+struct UpdatePlan {
+    int32_t* final_label;      // [B] label each frame ends up with (-1 = none)
+    int32_t* stop_layer;       // [B] the paper's l at which its inference stopped
+    int32_t* first_of_class;   // first frame of every class present in the batch, ascending
+    int32_t* first_of_stream;  // first frame of every stream present in the batch, ascending
+    int32_t* counts;           // [2] how many of each
+};
+
 struct UpdateArgs {
     int B, S, n, L;
+    UpdatePlan plan;
     const int32_t* stream_id;  // [B] or nullptr
     const uint8_t* done;
     const int32_t* exit_layer;
@@ -75,7 +85,7 @@ struct UpdateArgs {
     float* cnorm[SMTM_MAX_LAYERS];
     uint32_t* m[SMTM_MAX_LAYERS];
 };
-cudaError_t launch_update(const UpdateArgs& a, cudaStream_t st, int64_t* launches);
+
 
 struct ResizeArgs {
     int S, n, W, k_min, k_max, cl_num, cl_den;
@@ -85,5 +95,8 @@ struct ResizeArgs {
     int32_t* k;        // [S]
 };
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches);
+// Tables and centres; with rz != nullptr also the Eq. 5 / Eq. 6 refresh of every stream that
+// had a frame in the batch.
+cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, cudaStream_t st, int64_t* launches);
 
 }  // namespace smtm

@@ -52,6 +52,23 @@ __device__ __forceinline__ float ratio_margin(float top, float second) {
     return __fdiv_rn(__fsub_rn(top, second), second);
 }
 
+__device__ __forceinline__ void decide_from_top2(const LookupArgs& a, int b, const Top2& ta, const Top2& ts);
+
+// Best two of values held in registers: lane l holds slots l and l + 32 (v[0], v[1]) of k.
+__device__ __forceinline__ Top2 warp_top2_regs(const float (&v)[2], const int (&ids)[2], int k, int lane) {
+    Top2 t{0.f, 0.f, -1, -1};
+    if (lane < k) top2_push(t, v[0], ids[0]);
+    if (lane + kWarp < k) top2_push(t, v[1], ids[1]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov1 = __shfl_xor_sync(kFull, t.v1, o), ov2 = __shfl_xor_sync(kFull, t.v2, o);
+        const int oi1 = __shfl_xor_sync(kFull, t.id1, o), oi2 = __shfl_xor_sync(kFull, t.id2, o);
+        if (oi1 >= 0) top2_push(t, ov1, oi1);
+        if (oi2 >= 0) top2_push(t, ov2, oi2);
+    }
+    return t;
+}
+
 // Executed by one full warp once the similarities of frame b are known: s_cur[j] (this
 // layer, Eq. 1) and s_acc[j] (cumulative, Eq. 3) for the k slots whose classes are mem[j].
 // Selects the two best of each, evaluates Eq. 4 / Eq. 2 and the exit rule in fp32, and
@@ -61,6 +78,12 @@ __device__ __forceinline__ void decide_frame(const LookupArgs& a, int b, const f
     const Top2 ta = warp_top2(s_acc, mem, k, lane);
     const Top2 ts = warp_top2(s_cur, mem, k, lane);
     if (lane != 0) return;
+    decide_from_top2(a, b, ta, ts);
+}
+
+// Lane-0 part of the decision: Eq. 4 / Eq. 2 from the two best cumulative (ta) and
+// single-layer (ts) similarities, the exit rule in fp32, outputs and counters.
+__device__ __forceinline__ void decide_from_top2(const LookupArgs& a, int b, const Top2& ta, const Top2& ts) {
     float ac = 0.f, sep = 0.f;
     bool leave = false;
     if (ta.id2 >= 0) {

@@ -118,8 +118,11 @@ def step_pair(w, cache, mem, gb, lab, step, rep: Report, device="cuda", compare_
         rep.lookups += int(todo.sum())
         del x
     fb_d = torch.from_numpy(fb).to(device)
-    smtm.smtm_cache_update(cache, gb, fb_d)
-    smtm.smtm_cache_resize(cache)
+    if step % 2 == 0:       # both forms of the after-inference update are exercised
+        smtm.smtm_cache_update(cache, gb, fb_d)
+        smtm.smtm_cache_resize(cache)
+    else:
+        smtm.smtm_cache_update_resize(cache, gb, fb_d)
     mem.update(ob, fb)
     mem.resize()
     rep.frames += w.B
