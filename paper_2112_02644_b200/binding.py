@@ -88,6 +88,8 @@ def load_library():
     lib.smtm_cache_get_tables.argtypes = [vp, vp, vp]
     lib.smtm_cache_get_counters.argtypes = [vp, vp]
     lib.smtm_cache_get_launches.argtypes = [vp, vp]
+    lib.smtm_cache_profile.argtypes = [vp, i32]
+    lib.smtm_cache_get_profile.argtypes = [vp, i32, vp, vp]
     lib.smtm_cache_status.argtypes = [vp]
     lib.smtm_status_string.argtypes = [i32]
     lib.smtm_status_string.restype = ctypes.c_char_p
@@ -292,6 +294,19 @@ def smtm_cache_get_launches(cache: Cache) -> int:
     out = np.zeros(1, np.int64)
     _check(load_library().smtm_cache_get_launches(cache.handle, out.ctypes.data), "smtm_cache_get_launches")
     return int(out[0])
+
+
+def smtm_cache_profile(cache: Cache, max_lookups: int) -> None:
+    _check(load_library().smtm_cache_profile(cache.handle, int(max_lookups)), "smtm_cache_profile")
+
+
+def smtm_cache_get_profile(cache: Cache, layer: int):
+    """(total milliseconds, launches) of the streaming kernel at ``layer`` since profiling was switched on."""
+    total = ctypes.c_double(0.0)
+    count = ctypes.c_int64(0)
+    _check(load_library().smtm_cache_get_profile(cache.handle, layer, ctypes.byref(total), ctypes.byref(count)),
+           "smtm_cache_get_profile")
+    return total.value, count.value
 
 
 def smtm_cache_status(cache: Cache) -> int:

@@ -21,8 +21,13 @@ struct smtm_cache {
     unsigned long long* d_counters;
     int* d_status;
     float* d_partials;  // scratch of the fused lookup: partial dot products per (frame, part)
-    int* d_frame_ctr;   // scratch of the fused lookup: parts delivered per frame (zero between launches)
-    int32_t* d_plan;    // scratch of the update: 4 x [max_batch] + [2], see UpdatePlan
+    int32_t* d_plan;    // scratch of the update: final label and stop layer, 2 x [max_batch]
+    unsigned long long* d_tags;  // scratch of the update: election tags, [n] + [S]
+    unsigned long long epoch;    // update calls so far
+    // optional timing of the streaming kernel of every lookup (smtm_cache_profile)
+    std::vector<cudaEvent_t>* prof_events;  // pairs, in launch order
+    std::vector<int>* prof_layer;           // layer of each pair
+    size_t prof_used;                       // pairs recorded so far
     int device, sm_count;
     int64_t launches;
     // device-side carry and staging used only by smtm_step_host (allocated on first use)
@@ -56,7 +61,19 @@ cudaError_t dev_alloc(T** p, size_t count) {
     return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
 }
 
+void drop_profile(smtm_cache* c) {
+    if (c->prof_events) {
+        for (cudaEvent_t e : *c->prof_events) cudaEventDestroy(e);
+        delete c->prof_events;
+        delete c->prof_layer;
+        c->prof_events = nullptr;
+        c->prof_layer = nullptr;
+    }
+    c->prof_used = 0;
+}
+
 void free_all(smtm_cache* c) {
+    drop_profile(c);
     for (int l = 0; l < SMTM_MAX_LAYERS; ++l) {
         cudaFree(c->d_centers[l]);
         cudaFree(c->d_cnorm[l]);
@@ -71,8 +88,8 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_counters);
     cudaFree(c->d_status);
     cudaFree(c->d_partials);
-    cudaFree(c->d_frame_ctr);
     cudaFree(c->d_plan);
+    cudaFree(c->d_tags);
     cudaFree(c->hb.d_sa);
     cudaFree(c->hb.d_done);
     cudaFree(c->hb.d_exit_layer);
@@ -141,9 +158,16 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     a.counters = c->d_counters;
     const EncodeArgs e = encode_args(c, f, b->d_done, b->d_sv[layer]);
     bool fused = false;
-    SMTM_CUDA(launch_lookup_fused(e, a, c->d_partials, c->d_frame_ctr, c->sm_count, st, &c->launches, &fused));
+    const cudaEvent_t* timing = nullptr;
+    if (c->prof_events && 2 * (c->prof_used + 1) <= c->prof_events->size()) {
+        timing = c->prof_events->data() + 2 * c->prof_used;
+        (*c->prof_layer)[c->prof_used++] = layer;
+    }
+    SMTM_CUDA(launch_lookup_fused(e, a, c->d_partials, c->sm_count, st, &c->launches, &fused, timing));
     if (fused) return SMTM_OK;
+    if (timing) SMTM_CUDA(cudaEventRecord(timing[0], st));
     SMTM_CUDA(launch_encode(e, c->sm_count, st, &c->launches));
+    if (timing) SMTM_CUDA(cudaEventRecord(timing[1], st));
     SMTM_CUDA(launch_score_exit(a, st, &c->launches));
     return SMTM_OK;
 }
@@ -174,9 +198,9 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     const size_t mb = size_t(c->max_batch);
     a.plan.final_label = c->d_plan;
     a.plan.stop_layer = c->d_plan + mb;
-    a.plan.first_of_class = c->d_plan + 2 * mb;
-    a.plan.first_of_stream = c->d_plan + 3 * mb;
-    a.plan.counts = c->d_plan + 4 * mb;
+    a.plan.class_tag = c->d_tags;
+    a.plan.stream_tag = c->d_tags + c->n;
+    a.plan.epoch = ++c->epoch;
     a.stream_id = b->d_stream_id;
     a.done = b->d_done;
     a.exit_layer = b->d_exit_layer;
@@ -277,8 +301,8 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     ok = ok && dev_alloc(&c->d_counters, SMTM_CTR_COUNT) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_status, 1) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_partials, fused_partials_floats(c->max_batch, c->k_max)) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_frame_ctr, size_t(c->max_batch)) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_plan, 4 * size_t(c->max_batch) + 2) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_plan, 2 * size_t(c->max_batch)) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_tags, size_t(n) + size_t(S)) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();
         free_all(c);
@@ -306,7 +330,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     if (e == cudaSuccess) e = cudaMemset(c->d_ts, 0, size_t(S) * n * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(c->d_counters, 0, SMTM_CTR_COUNT * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
-    if (e == cudaSuccess) e = cudaMemset(c->d_frame_ctr, 0, size_t(c->max_batch) * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(c->d_tags, 0, (size_t(n) + size_t(S)) * sizeof(unsigned long long));
     if (e == cudaSuccess)
         e = cudaMemcpy(c->d_members, members.data(), members.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(c->d_k, ks.data(), ks.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
@@ -479,6 +503,44 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* c, int64_t* h_out) {
     if (!c || !h_out) return SMTM_ERR_INVALID_ARG;
     SMTM_CUDA(cudaDeviceSynchronize());
     SMTM_CUDA(cudaMemcpy(h_out, c->d_counters, SMTM_CTR_COUNT * sizeof(int64_t), cudaMemcpyDeviceToHost));
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_profile(smtm_cache_t* c, int32_t max_lookups) {
+    if (!c || max_lookups < 0 || max_lookups > (1 << 20)) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    drop_profile(c);
+    if (max_lookups == 0) return SMTM_OK;
+    c->prof_events = new (std::nothrow) std::vector<cudaEvent_t>();
+    c->prof_layer = new (std::nothrow) std::vector<int>(size_t(max_lookups), 0);
+    if (!c->prof_events || !c->prof_layer) return SMTM_ERR_ALLOC;
+    c->prof_events->reserve(2 * size_t(max_lookups));
+    for (int i = 0; i < 2 * max_lookups; ++i) {
+        cudaEvent_t ev;
+        if (cudaEventCreate(&ev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            drop_profile(c);
+            return SMTM_ERR_ALLOC;
+        }
+        c->prof_events->push_back(ev);
+    }
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_get_profile(smtm_cache_t* c, int32_t layer, double* h_total_ms, int64_t* h_count) {
+    if (!c || !h_total_ms || !h_count || layer < 0 || layer >= c->L) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    double total = 0.0;
+    int64_t count = 0;
+    for (size_t i = 0; c->prof_events && i < c->prof_used; ++i) {
+        if ((*c->prof_layer)[i] != layer) continue;
+        float ms = 0.f;
+        SMTM_CUDA(cudaEventElapsedTime(&ms, (*c->prof_events)[2 * i], (*c->prof_events)[2 * i + 1]));
+        total += ms;
+        ++count;
+    }
+    *h_total_ms = total;
+    *h_count = count;
     return SMTM_OK;
 }
 

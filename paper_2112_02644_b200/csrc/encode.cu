@@ -205,27 +205,24 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
     }
 }
 
-// ---- fused lookup: encode + score + exit in one persistent kernel ----------------------------
+// ---- fused lookup: encode + similarity scoring in one persistent kernel -----------------------
 //
 // Work is cut into units: (frame, part), a part being a run of chunks_per_unit chunks, i.e. a
 // slice of the frame's channels.  Every CTA first compacts the frames that are still active
 // and takes the units u = blockIdx.x, blockIdx.x + gridDim.x, ... of that list, so exited
 // frames cost nothing and the load is even.  Per unit the reducer warps leave the slice of
-// the semantic vector in shared memory (double-buffered) as well as in the SV stash; four
-// scorer warps take it from there: partial dot products against the slice of each member's
-// centre and the partial squared length.  With one part per frame the frame is decided on
-// the spot; otherwise the partials go to global scratch and the CTA that delivers a frame's
-// last part adds them up in part order and decides.  No floating-point atomics anywhere:
+// the semantic vector in shared memory (four buffers) as well as in the SV stash; eight dot
+// warps then share the unit's dot products, slot j on warp j % 8: each lane has every load of
+// its slot's centre slice in flight at once, so a unit costs one trip to L2.  The partial dot
+// products and the partial squared length go to global scratch [frame][part][slot]; the small
+// finishing kernel in lookup.cu adds the parts up in part order and decides.  No atomics:
 // the evaluation order of every sum is fixed.
 constexpr int kReducersF = 4;       // reducer warps of the fused kernel; stage s belongs to warp s % kReducersF
-constexpr int kDotWarps = 8;        // warps that share the dot products of a unit, slot j going to warp j % 8
-constexpr int kFinalizers = 2;      // warps that complete units alternately (partials, Eq. 1-4, decision)
+constexpr int kDotWarps = 8;        // warps that share the dot products of a unit
 constexpr int kSvBufs = 4;          // shared-memory slices; unit u passes through buffer u % kSvBufs
-constexpr int kThreadsFused = (kReducersF + 1 + kDotWarps + kFinalizers) * kWarp;
-constexpr int kFusedMaxK = 64;      // fast-memory capacity the fused kernel supports (two slots per lane)
+constexpr int kThreadsFused = (kReducersF + 1 + kDotWarps) * kWarp;
 constexpr int kMaxUnits = 1024;     // units per CTA
 constexpr int kMaxSlice = 1024;     // floats of a semantic-vector slice (eight 16-byte vectors per lane)
-constexpr int kMaxParts = 16;
 static_assert(kStages % kReducersF == 0, "stage ownership must be periodic");
 
 struct FusedParams {
@@ -234,21 +231,12 @@ struct FusedParams {
     int parts;            // P: parts per frame (divides chunks_per_frame)
     int chunks_per_unit;  // chunks_per_frame / P
     int slice_cap;        // channels of a full slice = chunks_per_unit * chunk_channels (multiple of 4)
-    float* partials;      // [B][P][k_max + 1], used when P > 1
-    int* frame_ctr;       // [B] parts delivered so far (returns to zero)
+    float* partials;      // [B][P][k_max + 1]: partial dot products per slot, then the partial squared length
 };
 
 constexpr size_t fused_smem(int slice_cap) {
     return size_t(kStages) * kStageCap + size_t(kSvBufs) * size_t(slice_cap) * 4 + kMaxUnits * 4 +
-           kFinalizers * (kFusedMaxK + 1) * 4 + (2 * kStages + 2 * kSvBufs + 2 * kFinalizers) * 8 + 40 * 4 + 192;
-}
-
-// acq_rel so that the partials written before it (by this warp) are visible to whoever
-// observes the count, and the partials of the parts counted before are visible to us.
-__device__ __forceinline__ int atomic_add_acq_rel(int* addr, int v) {
-    int old;
-    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
-    return old;
+           (2 * kStages + 2 * kSvBufs) * 8 + 40 * 4 + 192;
 }
 
 template <class R>
@@ -257,16 +245,13 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     uint8_t* stages = base;
     float* sv_s = reinterpret_cast<float*>(base + size_t(kStages) * kStageCap);  // [kSvBufs][slice_cap]
-    float* s_dot = sv_s + kSvBufs * f.slice_cap;                                 // [kFinalizers][kFusedMaxK + 1]
-    int* my_units = reinterpret_cast<int*>(s_dot + kFinalizers * (kFusedMaxK + 1));  // [kMaxUnits]
+    int* my_units = reinterpret_cast<int*>(sv_s + kSvBufs * f.slice_cap);        // [kMaxUnits]
     int* s_scan = my_units + kMaxUnits;                                          // [40]
     uint64_t* full = reinterpret_cast<uint64_t*>(
         (reinterpret_cast<uintptr_t>(s_scan + 40) + 7) & ~uintptr_t(7));         // [kStages]
     uint64_t* empty = full + kStages;                                            // [kStages]
     uint64_t* sv_full = empty + kStages;                                         // [kSvBufs]  slice written
     uint64_t* sv_empty = sv_full + kSvBufs;                                      // [kSvBufs]  slice read by all dot warps
-    uint64_t* dot_full = sv_empty + kSvBufs;                                     // [kFinalizers] dot products written
-    uint64_t* dot_empty = dot_full + kFinalizers;                                // [kFinalizers] ... and taken
 
     const NchwParams& p = f.e;
     const LookupArgs& a = f.a;
@@ -281,22 +266,14 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
             mbar_init(&sv_full[s], cpu);
             mbar_init(&sv_empty[s], kDotWarps);
         }
-        for (int s = 0; s < kFinalizers; ++s) {
-            mbar_init(&dot_full[s], kDotWarps);
-            mbar_init(&dot_empty[s], 1);
-        }
         mbar_init_fence();
     }
 
     // ---- the active frames and this CTA's share of their units -----------------------------
-    // A frame counts as active if it had not exited before this layer; one that this very
-    // launch has already decided (another CTA may be ahead) still counts, so that every CTA
-    // derives the same list.
     int n_active = 0;
     for (int t0 = 0; t0 < a.B; t0 += kThreadsFused) {
         const int b = t0 + threadIdx.x;
-        int act = 0;
-        if (b < a.B) act = (!a.done[b] || *(volatile const int32_t*)(a.exit_layer + b) == a.layer + 1) ? 1 : 0;
+        const int act = (b < a.B && !a.done[b]) ? 1 : 0;
         int cnt;
         const int pos = block_exclusive_scan(act, s_scan, &cnt);
         if (act) {
@@ -359,7 +336,7 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
                 issued = it + 1;
             }
         }
-    } else if (warp < kReducersF + 1 + kDotWarps) {
+    } else {
         // ---- dot warps: all of them work on unit u together, slot j on warp j % kDotWarps --------
         const int dw = warp - kReducersF - 1;
         // fast memory of the unit in hand, fetched one unit ahead
@@ -373,23 +350,21 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
             nx_ids[1] = lane + kWarp < nx_k ? mem[lane + kWarp] : 0;
         }
         for (int u = 0; u < nu; ++u) {
-            const int unit = my_units[u], part = unit % kMaxParts;
+            const int unit = my_units[u], b = unit / kMaxParts, part = unit % kMaxParts;
             const int sb = part * f.slice_cap;          // first channel of the slice
             const int Dp = min(f.slice_cap, p.C - sb);  // channels in it (a multiple of 4)
             const int n4 = Dp >> 2;
             const int k = nx_k;
             const int ids[2] = {nx_ids[0], nx_ids[1]};  // lane l knows the classes of slots l and l + 32
-            const int buf = u % kSvBufs, db = u % kFinalizers;
+            const int buf = u % kSvBufs;
             int nb_sid = 0;
             if (u + 1 < nu) {
                 const int nb = my_units[u + 1] / kMaxParts;
                 nb_sid = a.stream_id ? a.stream_id[nb] : 0;  // in flight while this unit is scored
             }
+            float* out = f.partials + ((size_t)b * P + part) * (a.k_max + 1);
             if (!mbar_wait_bounded(&sv_full[buf], (u / kSvBufs) & 1, p.status)) { failed = true; break; }
-            if (u >= kFinalizers &&
-                !mbar_wait_bounded(&dot_empty[db], (u / kFinalizers - 1) & 1, p.status)) { failed = true; break; }
             const float4* v4 = reinterpret_cast<const float4*>(sv_s + buf * f.slice_cap);
-            float* out = s_dot + db * (kFusedMaxK + 1);
             if (dw == kDotWarps - 1) {  // partial squared length of the semantic vector
                 float nn = 0.f;
                 for (int q = lane; q < n4; q += kWarp) {
@@ -398,7 +373,7 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
                 }
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(kFull, nn, o);
-                if (lane == 0) out[kFusedMaxK] = nn;
+                if (lane == 0) out[a.k_max] = nn;
             }
             for (int j = dw; j < k; j += kDotWarps) {  // partial dot product of slot j (Eq. 1's numerator)
                 const int cls = __shfl_sync(kFull, (j & 32) ? ids[1] : ids[0], j & 31);
@@ -424,87 +399,13 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
                 if (lane == 0) out[j] = d;
             }
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(&sv_empty[buf]);
-                mbar_arrive(&dot_full[db]);
-            }
+            if (lane == 0) mbar_arrive(&sv_empty[buf]);
             if (u + 1 < nu) {  // fast memory of the next unit (its stream id has arrived by now)
                 nx_k = min(a.k[nb_sid], kFusedMaxK);
                 const int32_t* mem = a.members + (size_t)nb_sid * a.k_max;
                 nx_ids[0] = lane < nx_k ? mem[lane] : 0;
                 nx_ids[1] = lane + kWarp < nx_k ? mem[lane + kWarp] : 0;
             }
-        }
-    } else {
-        // ---- finalizers: warp fw completes the units fw, fw + kFinalizers, ... ---------------------
-        const int fw = warp - kReducersF - 1 - kDotWarps;
-        const float weight = float(1u << a.layer);  // 2^(l-1) with l = layer + 1
-        const float* in = s_dot + fw * (kFusedMaxK + 1);
-        for (int u = fw; u < nu; u += kFinalizers) {
-            const int unit = my_units[u], b = unit / kMaxParts, part = unit % kMaxParts;
-            // everything that does not depend on the dot products is fetched while they are computed
-            const int sid = a.stream_id ? a.stream_id[b] : 0;
-            const int k = min(a.k[sid], kFusedMaxK);
-            const int32_t* mem = a.members + (size_t)sid * a.k_max;
-            int ids[2];
-            float clen[2], sa_old[2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int j = lane + h * kWarp;
-                ids[h] = j < k ? mem[j] : 0;
-                clen[h] = j < k ? a.cnorm[ids[h]] : 0.f;
-                sa_old[h] = j < k ? a.sa[(size_t)b * a.k_max + j] : 0.f;
-            }
-            if (!mbar_wait_bounded(&dot_full[fw], (u / kFinalizers) & 1, p.status)) { failed = true; break; }
-            float dots[2], nn = in[kFusedMaxK];
-            dots[0] = lane < k ? in[lane] : 0.f;
-            dots[1] = lane + kWarp < k ? in[lane + kWarp] : 0.f;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&dot_empty[fw]);
-
-            // is the frame complete?  (with P > 1: did we deliver its last part?)
-            if (P > 1) {
-                float* out = f.partials + ((size_t)b * P + part) * (a.k_max + 1);
-                if (lane < k) out[lane] = dots[0];
-                if (lane + kWarp < k) out[lane + kWarp] = dots[1];
-                if (lane == 0) out[a.k_max] = nn;
-                __syncwarp();
-                int last = 0;
-                if (lane == 0) {
-                    last = atomic_add_acq_rel(&f.frame_ctr[b], 1) == P - 1 ? 1 : 0;
-                    if (last) f.frame_ctr[b] = 0;
-                }
-                last = __shfl_sync(kFull, last, 0);
-                if (!last) continue;
-                // add the parts up in part order
-                float pn[kMaxParts], p0[kMaxParts], p1[kMaxParts];
-#pragma unroll
-                for (int q = 0; q < kMaxParts; ++q) {
-                    const float* src = f.partials + ((size_t)b * P + q) * (a.k_max + 1);
-                    pn[q] = q < P ? __ldcg(src + a.k_max) : 0.f;
-                    p0[q] = (q < P && lane < k) ? __ldcg(src + lane) : 0.f;
-                    p1[q] = (q < P && lane + kWarp < k) ? __ldcg(src + lane + kWarp) : 0.f;
-                }
-                nn = 0.f; dots[0] = 0.f; dots[1] = 0.f;
-#pragma unroll
-                for (int q = 0; q < kMaxParts; ++q) {
-                    if (q < P) { nn += pn[q]; dots[0] += p0[q]; dots[1] += p1[q]; }
-                }
-            }
-            float s_cur[2] = {0.f, 0.f}, s_acc[2] = {0.f, 0.f};
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int j = lane + h * kWarp;
-                if (j < k) {
-                    s_cur[h] = cosine_from(dots[h], nn, clen[h]);        // Eq. 1
-                    s_acc[h] = __fmaf_rn(s_cur[h], weight, sa_old[h]);   // Eq. 3
-                    a.sa[(size_t)b * a.k_max + j] = s_acc[h];
-                }
-            }
-            const Top2 ta = warp_top2_regs(s_acc, ids, k, lane);
-            const Top2 ts = warp_top2_regs(s_cur, ids, k, lane);
-            if (lane == 0) decide_from_top2(a, b, ta, ts);
-            __syncwarp();
         }
     }
     // No thread leaves before every copy that was issued has landed.
@@ -761,10 +662,10 @@ size_t fused_partials_floats(int max_batch, int k_max) {
     return size_t(max_batch) * kMaxParts * (size_t(std::min(k_max, kFusedMaxK)) + 1);
 }
 
-cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float* partials, int* frame_ctr,
-                                int sm_count, cudaStream_t st, int64_t* launches, bool* handled) {
+cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float* partials, int sm_count,
+                                cudaStream_t st, int64_t* launches, bool* handled, const cudaEvent_t* timing) {
     *handled = false;
-    if (e.B <= 0 || e.layout != SMTM_NCHW || a.k_max > kFusedMaxK || !partials || !frame_ctr) return cudaSuccess;
+    if (e.B <= 0 || e.layout != SMTM_NCHW || a.k_max > kFusedMaxK || !partials) return cudaSuccess;
     FusedParams f{};
     const Reducer r = plan_nchw(e, &f.e);
     if (r == kNone) return cudaSuccess;
@@ -797,16 +698,18 @@ cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float*
     f.chunks_per_unit = cpf / P;
     f.slice_cap = f.chunks_per_unit * f.e.chunk_channels;
     f.partials = partials;
-    f.frame_ctr = frame_ctr;
     const size_t smem = fused_smem(f.slice_cap);
     cudaError_t err = cudaSuccess;
+    if (timing) cudaEventRecord(timing[0], st);
 #define SMTM_LAUNCH(...) k_lookup_nchw<__VA_ARGS__><<<sm_count, kThreadsFused, smem, st>>>(f)
     SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
 #undef SMTM_LAUNCH
     err = cudaGetLastError();
+    if (timing) cudaEventRecord(timing[1], st);
     ++*launches;
     *handled = true;
-    return err;
+    if (err != cudaSuccess) return err;
+    return launch_finish_partials(a, partials, P, st, launches);
 }
 
 cudaError_t launch_row_norm2(const float* sv, const uint8_t* skip, int B, int D, float* out, cudaStream_t st,

@@ -49,10 +49,17 @@ struct LookupArgs {
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches);
 // Encode + score + exit in one kernel (NCHW shapes the streaming pipeline serves, fast
 // memories of at most 64 entries).  *handled is false when the shape is not served, in which
-// case nothing was launched.  partials: fused_partials_floats() floats; frame_ctr: [max_batch] zeros.
+// case nothing was launched.  partials: fused_partials_floats() floats of scratch.
+constexpr int kFusedMaxK = 64;  // fast-memory capacity the fused path supports (two slots per lane)
+constexpr int kMaxParts = 16;   // most parts a frame is cut into
 size_t fused_partials_floats(int max_batch, int k_max);
-cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float* partials, int* frame_ctr,
-                                int sm_count, cudaStream_t st, int64_t* launches, bool* handled);
+// timing: nullptr, or two events recorded on `st` right before and after the streaming kernel.
+cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float* partials, int sm_count,
+                                cudaStream_t st, int64_t* launches, bool* handled, const cudaEvent_t* timing);
+// Second half of the fused lookup: adds up the parts of every active frame in part order,
+// then Eq. 1, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule.  partials: [B][parts][k_max + 1].
+cudaError_t launch_finish_partials(const LookupArgs& a, const float* partials, int parts, cudaStream_t st,
+                                   int64_t* launches);
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,
                                cudaStream_t st, int64_t* launches);
 
@@ -60,13 +67,13 @@ cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, in
 cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm, cudaStream_t st,
                                 int64_t* launches);
 
-// Scratch written by the planning kernel of an update (all device, sized for max_batch).
+// Scratch of an update (all device).
 struct UpdatePlan {
-    int32_t* final_label;      // [B] label each frame ends up with (-1 = none)
-    int32_t* stop_layer;       // [B] the paper's l at which its inference stopped
-    int32_t* first_of_class;   // first frame of every class present in the batch, ascending
-    int32_t* first_of_stream;  // first frame of every stream present in the batch, ascending
-    int32_t* counts;           // [2] how many of each
+    int32_t* final_label;            // [max_batch] label each frame ends up with (-1 = none)
+    int32_t* stop_layer;             // [max_batch] the paper's l at which its inference stopped
+    unsigned long long* class_tag;   // [n] election of the first frame of each class, see memory.cu
+    unsigned long long* stream_tag;  // [S] election of the first frame of each stream
+    unsigned long long epoch;        // sequence number of this update call (>= 1)
 };
 
 struct UpdateArgs {

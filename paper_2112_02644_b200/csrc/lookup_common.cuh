@@ -100,10 +100,9 @@ __device__ __forceinline__ void decide_from_top2(const LookupArgs& a, int b, con
     atomicAdd(&a.counters[SMTM_CTR_LOOKUPS], 1ull);
     if (isfinite(ac) && fabsf(ac - a.tau) <= 1e-4f) atomicAdd(&a.counters[SMTM_CTR_NEAR], 1ull);
     if (leave) {
+        a.done[b] = 1;
         a.exit_layer[b] = a.layer + 1;
         a.pred[b] = ta.id1;
-        __threadfence();  // whoever sees the flag also sees the layer it was set at
-        a.done[b] = 1;
         atomicAdd(&a.counters[SMTM_CTR_EXITS + a.layer], 1ull);
     }
 }

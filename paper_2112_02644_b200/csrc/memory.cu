@@ -1,15 +1,17 @@
 // Adaptive priming memory (Sec. 6): frequency / time-stamp tables, running-mean centres
 // (Eq. 7), replacement score and top-k (Eq. 5), adaptive fast-memory size (Eq. 6).
 //
-// All reductions are segmented and atomics-free: a CTA owns a stream's tables, or one
-// (class, layer) centre, and walks the batch in ascending frame index, so the result is
-// the one a frame-by-frame replay would give and does not depend on scheduling.
+// All floating-point reductions are segmented and atomics-free: one owner walks the batch in
+// ascending frame index, so the result is the one a frame-by-frame replay would give and does
+// not depend on scheduling.
 //
-// An update is two launches.  k_update_plan (one CTA) writes every frame's final label and
-// stop layer and lists the first frame of every class and of every stream present in the
-// batch.  k_update_apply then starts one CTA per listed stream (tables, optionally followed
-// by that stream's Eq. 5 / Eq. 6 refresh) and one per (listed class, layer) (Eq. 7); classes
-// and streams the batch does not touch cost nothing.
+// An update is two launches.  k_update_plan writes every frame's final label and stop layer
+// and elects, per class and per stream present in the batch, its first frame (an integer
+// atomicMax on a tag that carries the call's sequence number, so the election tables never
+// need clearing).  In k_update_apply every frame's warp (tables, optionally followed by its
+// stream's Eq. 5 / Eq. 6 refresh) and every (frame, layer) CTA (Eq. 7) first checks whether
+// its frame was elected and leaves at once if not; classes and streams the batch does not
+// touch cost nothing.
 #include <algorithm>
 
 #include "common.cuh"
@@ -22,54 +24,32 @@ namespace {
 constexpr int kFtMax = 1 << 20;  // frequency counts saturate here so that Eq. 6's sums fit 64 bits
 constexpr int kEMax = 12;        // floor(TS / W) is clamped here: 0.25^12 of a count is below one
 
-constexpr int kPlanThreads = 1024;
 constexpr int kUpdThreads = 256;
+constexpr int kUpdWarps = kUpdThreads / kWarp;
 constexpr int kSliceCols = kUpdThreads * 4;  // columns of a centre handled per sweep (one float4 per thread)
+constexpr int kWarpTablesMaxN = 1024;        // classes a warp can keep in registers (32 per lane)
+constexpr int kTagBits = 24;                 // frames per batch < 2^24
+
+// Election tag of frame b in call number `epoch`: larger epoch wins over anything older,
+// within a call the smallest frame index wins.
+__device__ __forceinline__ unsigned long long tag_of(unsigned long long epoch, int b) {
+    return (epoch << kTagBits) | (unsigned long long)((1 << kTagBits) - 1 - b);
+}
 
 // ---- plan -----------------------------------------------------------------------------------
 
 // Label and stop layer of a finished frame: the prediction and exit layer if it exited,
 // else the fallback label (the full network's answer, -1 = none) and L.
-__global__ void __launch_bounds__(kPlanThreads) k_update_plan(const UpdateArgs a) {
-    extern __shared__ int s_keys[];  // [B] labels, [B] stream ids
-    int* s_lab = s_keys;
-    int* s_sid = s_keys + a.B;
-    __shared__ int s_scan[33];
-    const int tid = threadIdx.x;
-    for (int b = tid; b < a.B; b += kPlanThreads) {
-        const bool ex = a.done[b] != 0;
-        const int lab = ex ? a.pred[b] : (a.fallback ? a.fallback[b] : -1);
-        s_lab[b] = lab;
-        s_sid[b] = a.stream_id ? a.stream_id[b] : 0;
-        a.plan.final_label[b] = lab;
-        a.plan.stop_layer[b] = ex ? a.exit_layer[b] : a.L;
-    }
-    __syncthreads();
-    int n_cls = 0, n_str = 0;
-    for (int b0 = 0; b0 < a.B; b0 += kPlanThreads) {
-        const int b = b0 + tid;
-        int first_c = 0, first_s = 0;
-        if (b < a.B) {
-            const int lab = s_lab[b], sid = s_sid[b];
-            first_c = lab >= 0;
-            first_s = 1;
-            for (int j = b - 1; j >= 0 && (first_c | first_s); --j) {
-                if (s_lab[j] == lab) first_c = 0;
-                if (s_sid[j] == sid) first_s = 0;
-            }
-        }
-        int cnt;
-        int pos = block_exclusive_scan(first_c, s_scan, &cnt);
-        if (first_c) a.plan.first_of_class[n_cls + pos] = b;
-        n_cls += cnt;
-        pos = block_exclusive_scan(first_s, s_scan, &cnt);
-        if (first_s) a.plan.first_of_stream[n_str + pos] = b;
-        n_str += cnt;
-    }
-    if (tid == 0) {
-        a.plan.counts[0] = n_cls;
-        a.plan.counts[1] = n_str;
-    }
+__global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a) {
+    const int b = blockIdx.x * kUpdThreads + threadIdx.x;
+    if (b >= a.B) return;
+    const bool ex = a.done[b] != 0;
+    const int lab = ex ? a.pred[b] : (a.fallback ? a.fallback[b] : -1);
+    a.plan.final_label[b] = lab;
+    a.plan.stop_layer[b] = ex ? a.exit_layer[b] : a.L;
+    const unsigned long long tag = tag_of(a.plan.epoch, b);
+    if (lab >= 0) atomicMax(a.plan.class_tag + lab, tag);
+    atomicMax(a.plan.stream_tag + (a.stream_id ? a.stream_id[b] : 0), tag);
 }
 
 // ---- Eq. 5 / Eq. 6 ------------------------------------------------------------------------
@@ -81,7 +61,7 @@ __device__ __forceinline__ unsigned long long score_of(int ft, int ts, int W) {
     return f << (2 * (kEMax - e));  // FT * 4^(12 - e) = 4^12 * FT * 0.25^e
 }
 
-constexpr size_t resize_smem(int n, int k_max) { return size_t(n) * 8 + size_t(n + (n & 1)) * 4 + size_t(k_max) * 8; }
+__host__ __device__ constexpr size_t resize_smem(int n, int k_max) { return size_t(n) * 8 + size_t(n + (n & 1)) * 4 + size_t(k_max) * 8; }
 
 // Refresh of one stream's fast memory by a CTA of kUpdThreads threads.  Classes with a
 // non-zero score are compacted in ascending id and ranked among themselves by counting;
@@ -186,25 +166,161 @@ __device__ __forceinline__ int compact_tile(int hit, int value, int* list, int* 
     return cnt;
 }
 
-// blockIdx.x <  table_ctas : tables (and, if asked, the refresh) of the stream of the
-//                            blockIdx.x-th listed frame
-// blockIdx.x >= table_ctas : centre of (class of the g-th listed frame, layer), g, layer =
-//                            divmod(blockIdx.x - table_ctas, L)
+// Sec. 6.1 for the stream whose first frame in the batch is g, by one warp with the stream's
+// tables in registers (class c lives in lane c % 32, register c / 32), then, if asked, that
+// stream's Eq. 5 / Eq. 6 refresh.  `smem` is this warp's resize_smem(n, k_max) bytes.
+__device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g, int s, int do_resize,
+                               unsigned char* smem) {
+    constexpr int NC = kWarpTablesMaxN / kWarp;
+    const int lane = threadIdx.x & 31;
+    const unsigned lt = (1u << lane) - 1u;
+    int32_t* ftp = a.ft + (size_t)s * a.n;
+    int32_t* tsp = a.ts + (size_t)s * a.n;
+    int ft[NC], ts[NC];
+#pragma unroll
+    for (int i = 0; i < NC; ++i) {
+        const int c = lane + i * kWarp;
+        ft[i] = c < a.n ? ftp[c] : 0;
+        ts[i] = c < a.n ? tsp[c] : 0;
+    }
+    // the stream's frames in ascending index (none precedes g)
+    for (int b0 = g - g % kWarp; b0 < a.B; b0 += kWarp) {
+        const int b = b0 + lane;
+        const bool hit = b >= g && b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s;
+        const int lab = hit ? a.plan.final_label[b] : -1;
+        unsigned mask = __ballot_sync(kFull, hit);
+        while (mask) {
+            const int src = __ffs(mask) - 1;
+            mask &= mask - 1;
+            const int l = __shfl_sync(kFull, lab, src);
+#pragma unroll
+            for (int i = 0; i < NC; ++i) {
+                if (lane + i * kWarp == l) {
+                    ft[i] = min(ft[i] + 1, kFtMax);
+                    ts[i] = 0;
+                } else if (ts[i] < INT32_MAX) {
+                    ++ts[i];
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < NC; ++i) {
+        const int c = lane + i * kWarp;
+        if (c < a.n) {
+            ftp[c] = ft[i];
+            tsp[c] = ts[i];
+        }
+    }
+    if (!do_resize) return;
+
+    // Eq. 5 scores; non-zero ones compacted in ascending class id
+    unsigned long long* s_score = reinterpret_cast<unsigned long long*>(smem);  // [n]
+    int* s_id = reinterpret_cast<int*>(s_score + a.n);                          // [n]
+    unsigned long long* s_top = reinterpret_cast<unsigned long long*>(s_id + a.n + (a.n & 1));  // [k_max]
+    int32_t* mem = rz.members + (size_t)s * rz.k_max;
+    unsigned long long total = 0;
+    int nz = 0;
+#pragma unroll
+    for (int i = 0; i < NC; ++i) {
+        const int c = lane + i * kWarp;
+        const unsigned long long sc = c < a.n ? score_of(ft[i], ts[i], rz.W) : 0ull;
+        const unsigned m = __ballot_sync(kFull, sc != 0);
+        if (sc != 0) {
+            const int pos = nz + __popc(m & lt);
+            s_score[pos] = sc;
+            s_id[pos] = c;
+        }
+        nz += __popc(m);
+        total += sc;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(kFull, total, o);
+    if (total == 0) return;  // nothing seen yet: keep size and members
+    __syncwarp();
+    // rank the non-zero classes by counting; rank r < k_max goes to slot r
+    for (int i = lane; i < nz; i += kWarp) {
+        const unsigned long long sc = s_score[i];
+        int r = 0;
+        for (int j = 0; j < nz; ++j) {
+            const unsigned long long o = s_score[j];
+            r += (o > sc || (o == sc && j < i)) ? 1 : 0;  // compacted order is ascending id
+        }
+        if (r < rz.k_max) {
+            mem[r] = s_id[i];
+            s_top[r] = sc;
+        }
+    }
+    // zero-score classes fill the remaining slots in ascending id
+    int filled = nz;
+#pragma unroll
+    for (int i = 0; i < NC; ++i) {
+        const int c = lane + i * kWarp;
+        const bool z = filled < rz.k_max && c < a.n && score_of(ft[i], ts[i], rz.W) == 0;
+        const unsigned m = __ballot_sync(kFull, z);
+        if (z) {
+            const int pos = filled + __popc(m & lt);
+            if (pos < rz.k_max) {
+                mem[pos] = c;
+                s_top[pos] = 0;
+            }
+        }
+        filled += __popc(m);
+    }
+    __syncwarp();
+    // Eq. 6: smallest k in [k_min, k_max] with cl_den * prefix(k) > cl_num * total
+    unsigned long long carry = 0;
+    int chosen = rz.k_max;
+    for (int base = 0; base < rz.k_max; base += kWarp) {
+        const int idx = base + lane;
+        unsigned long long v = idx < rz.k_max ? s_top[idx] : 0ull;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long t = __shfl_up_sync(kFull, v, o);
+            if (lane >= o) v += t;
+        }
+        const unsigned long long prefix = carry + v;
+        const bool ok = idx < rz.k_max && idx + 1 >= rz.k_min &&
+                        (unsigned long long)rz.cl_den * prefix > (unsigned long long)rz.cl_num * total;
+        const unsigned m = __ballot_sync(kFull, ok);
+        if (m) {
+            chosen = base + __ffs(m);
+            break;
+        }
+        carry += __shfl_sync(kFull, v, 31);
+    }
+    if (lane == 0) rz.k[s] = chosen;
+}
+
+// blockIdx.x <  table_ctas : tables (and, if asked, the refresh) of the streams whose first
+//                            frames are among this CTA's frames: a warp per frame, or, when
+//                            the classes do not fit a warp's registers, the whole CTA for one
+// blockIdx.x >= table_ctas : centre of (class of frame g, layer), g, layer = divmod(blockIdx.x
+//                            - table_ctas, L), if g is the first frame of its class
 __global__ void __launch_bounds__(kUpdThreads) k_update_apply(const UpdateArgs a, const ResizeArgs rz, int table_ctas,
-                                                              int do_resize) {
+                                                              int do_resize, int warp_tables) {
     extern __shared__ unsigned long long s_dyn[];
     __shared__ int s_list[kUpdThreads];
     __shared__ int s_scan[33];
     __shared__ float s_red[32];
-    __shared__ unsigned long long s_part[kUpdThreads / 32];
+    __shared__ unsigned long long s_part[kUpdWarps];
     const int tid = threadIdx.x;
 
     if (int(blockIdx.x) < table_ctas) {
-        // ---- Sec. 6.1: the stream's frames, in ascending index, replayed per class ----------
-        if (int(blockIdx.x) >= a.plan.counts[1]) return;
-        const int bf = a.plan.first_of_stream[blockIdx.x];
-        const int s = a.stream_id ? a.stream_id[bf] : 0;
-        for (int t0 = bf - bf % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
+        if (warp_tables) {
+            const int g = blockIdx.x * kUpdWarps + (tid >> 5);
+            if (g >= a.B) return;
+            const int s = a.stream_id ? a.stream_id[g] : 0;
+            if (a.plan.stream_tag[s] != tag_of(a.plan.epoch, g)) return;  // not the stream's first frame
+            tables_by_warp(a, rz, g, s, do_resize,
+                           reinterpret_cast<unsigned char*>(s_dyn) + size_t(tid >> 5) * resize_smem(a.n, rz.k_max));
+            return;
+        }
+        // ---- Sec. 6.1 by a whole CTA: the stream's frames, ascending, replayed per class -------
+        const int g = blockIdx.x;
+        const int s = a.stream_id ? a.stream_id[g] : 0;
+        if (a.plan.stream_tag[s] != tag_of(a.plan.epoch, g)) return;
+        for (int t0 = g - g % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
             const int b = t0 + tid;
             const int hit = (b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
             const int cnt = compact_tile(hit, hit ? a.plan.final_label[b] : -1, s_list, s_scan);
@@ -233,9 +349,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_apply(const UpdateArgs a
     // ---- Eq. 7 for one (class, layer): fold the matching frames in ascending index --------
     const int job = blockIdx.x - table_ctas;
     const int g = job / a.L, l0 = job - g * a.L;  // l0 is 0-based here; the paper's l0 is l0 + 1
-    if (g >= a.plan.counts[0]) return;
-    const int bf = a.plan.first_of_class[g];
-    const int cls = a.plan.final_label[bf];
+    const int cls = a.plan.final_label[g];
+    if (cls < 0 || a.plan.class_tag[cls] != tag_of(a.plan.epoch, g)) return;  // not the class's first frame
     const int D = a.dims[l0];
     const bool vec = (D & 3) == 0;  // rows are 16-byte aligned
     const float* sv = a.sv[l0];
@@ -247,7 +362,7 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_apply(const UpdateArgs a
         const int d = d0 + tid * 4;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         q = 0;
-        for (int t0 = bf - bf % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
+        for (int t0 = g - g % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
             const int b = t0 + tid;
             const int hit = (b < a.B && a.plan.final_label[b] == cls && a.plan.stop_layer[b] >= l0 + 1) ? 1 : 0;
             const int cnt = compact_tile(hit, b, s_list, s_scan);
@@ -255,16 +370,16 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_apply(const UpdateArgs a
             q += cnt;
             if (d >= D) continue;
             if (vec) {
-                // eight rows in flight per thread; the additions stay in ascending frame order
-                for (int i0 = 0; i0 < cnt; i0 += 8) {
-                    float4 r[8];
+                // sixteen rows in flight per thread; the additions stay in ascending frame order
+                for (int i0 = 0; i0 < cnt; i0 += 16) {
+                    float4 r[16];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u)
+                    for (int u = 0; u < 16; ++u)
                         r[u] = i0 + u < cnt
                                    ? __ldg(reinterpret_cast<const float4*>(sv + (size_t)s_list[i0 + u] * D + d))
                                    : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
+                    for (int u = 0; u < 16; ++u) {
                         if (i0 + u < cnt) {
                             acc[0] += r[u].x; acc[1] += r[u].y; acc[2] += r[u].z; acc[3] += r[u].w;
                         }
@@ -321,21 +436,21 @@ cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm
 
 cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, cudaStream_t st, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
-    static size_t opted_plan = 48 * 1024, opted_apply = 48 * 1024;
-    const size_t plan_smem = size_t(a.B) * 2 * sizeof(int);
-    cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_plan), plan_smem, &opted_plan);
-    if (e != cudaSuccess) return e;
-    const size_t apply_smem = rz ? resize_smem(a.n, rz->k_max) : 0;
-    e = opt_in_smem(reinterpret_cast<const void*>(k_update_apply), apply_smem, &opted_apply);
+    if (a.B >= (1 << kTagBits)) return cudaErrorInvalidValue;
+    static size_t opted = 48 * 1024;
+    const size_t per_stream = rz ? resize_smem(a.n, rz->k_max) : 0;
+    // a warp per frame when the classes fit its registers and eight refresh buffers fit a CTA
+    const bool warp_tables = a.n <= kWarpTablesMaxN && per_stream * kUpdWarps <= 96 * 1024;
+    const size_t smem = warp_tables ? per_stream * kUpdWarps : per_stream;
+    cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_apply), smem, &opted);
     if (e != cudaSuccess) return e;
     *launches += 2;
-    k_update_plan<<<1, kPlanThreads, plan_smem, st>>>(a);
+    k_update_plan<<<(a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st>>>(a);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const int table_ctas = std::min(a.B, a.S);
-    const int centre_ctas = std::min(a.B, a.n) * a.L;
-    k_update_apply<<<table_ctas + centre_ctas, kUpdThreads, apply_smem, st>>>(a, rz ? *rz : ResizeArgs{}, table_ctas,
-                                                                              rz ? 1 : 0);
+    const int table_ctas = warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
+    k_update_apply<<<table_ctas + a.B * a.L, kUpdThreads, smem, st>>>(a, rz ? *rz : ResizeArgs{}, table_ctas,
+                                                                     rz ? 1 : 0, warp_tables ? 1 : 0);
     return cudaGetLastError();
 }
 
