@@ -22,7 +22,6 @@
 // Any other shape falls back to a plain thread-per-(frame, channel) loop.
 #include <algorithm>
 #include <cmath>
-#include <cstdlib>
 
 #include "lookup_common.cuh"
 
@@ -549,14 +548,10 @@ int pow2_floor(int v) {
 
 
 
-int in_flight_limit() {
-    static int v = [] {
-        const char* e = getenv("SMTM_INFLIGHT");
-        const int n = e ? atoi(e) : kStages;
-        return std::max(1, std::min(n, kStages));
-    }();
-    return v;
-}
+// Copies the producer keeps outstanding.  Four 25 KB copies per SM (15 MB over the chip) cover
+// the bandwidth-delay product of HBM with margin; more only lengthens the queues that the
+// centre loads of the dot warps wait in.
+constexpr int kMaxInFlight = 4;
 
 // Which reducer a shape is served by, and the chunking that goes with it.
 enum Reducer { kNone, kUnitBf16x49, kUnitBf16x196, kUnitF16x49, kUnitF16x196, kUnitF32x49, kTeamF32, kTeamF16, kTeamBf16 };
@@ -573,7 +568,7 @@ Reducer plan_nchw(const EncodeArgs& a, NchwParams* p) {
     p->ch_bytes = HW * es;
     p->frame_bytes = (long long)a.C * p->ch_bytes;
     p->inv_hw = 1.0f / float(HW);
-    p->max_in_flight = in_flight_limit();
+    p->max_in_flight = kMaxInFlight;
     // unit-per-lane shapes (compile-time H*W)
     int G = 0;
     if ((HW == 49 || HW == 196) && es == 2) G = HW == 49 ? 8 : 2;
