@@ -21,6 +21,8 @@ struct smtm_cache {
     unsigned long long* d_counters;
     int* d_status;
     float* d_partials;  // scratch of the fused lookup: partial dot products per (frame, part)
+    void* d_dense;      // scratch of the tensor-core scorer (fast memories above 64 entries), else NULL
+    int d_max;          // largest C_l
     int32_t* d_plan;    // scratch of the update: final label and stop layer, 2 x [max_batch]
     unsigned long long* d_tags;  // scratch of the update: election tags, [n] + [S]
     unsigned long long epoch;    // update calls so far
@@ -89,6 +91,7 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_status);
     cudaFree(c->d_partials);
     cudaFree(c->d_plan);
+    cudaFree(c->d_dense);
     cudaFree(c->d_tags);
     cudaFree(c->hb.d_sa);
     cudaFree(c->hb.d_done);
@@ -168,6 +171,13 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     if (timing) SMTM_CUDA(cudaEventRecord(timing[0], st));
     SMTM_CUDA(launch_encode(e, c->sm_count, st, &c->launches));
     if (timing) SMTM_CUDA(cudaEventRecord(timing[1], st));
+    if (c->d_dense && dense_scoring_supported(a.D, a.n)) {  // large fast memory: tensor cores
+        float* dots = nullptr;
+        SMTM_CUDA(launch_dense_dots(a.sv, a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max, &dots,
+                                    c->d_status, st, &c->launches));
+        SMTM_CUDA(launch_finish_dense(a, dots, st, &c->launches));
+        return SMTM_OK;
+    }
     SMTM_CUDA(launch_score_exit(a, st, &c->launches));
     return SMTM_OK;
 }
@@ -302,6 +312,10 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     ok = ok && dev_alloc(&c->d_status, 1) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_partials, fused_partials_floats(c->max_batch, c->k_max)) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_plan, 2 * size_t(c->max_batch)) == cudaSuccess;
+    for (int l = 0; l < c->L; ++l) c->d_max = c->dims[l] > c->d_max ? c->dims[l] : c->d_max;
+    c->d_max = (c->d_max + 7) / 8 * 8;  // keeps the bf16 operand arrays of the tensor-core scorer 16-byte aligned
+    if (ok && c->k_max > kFusedMaxK)
+        ok = cudaMalloc(&c->d_dense, dense_scratch_bytes(c->max_batch, n, c->d_max)) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_tags, size_t(n) + size_t(S)) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();

@@ -60,6 +60,15 @@ cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float*
 // then Eq. 1, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule.  partials: [B][parts][k_max + 1].
 cudaError_t launch_finish_partials(const LookupArgs& a, const float* partials, int parts, cudaStream_t st,
                                    int64_t* launches);
+// ---- large fast memories: dot products against every class on the tensor cores ---------------
+bool dense_scoring_supported(int D, int n);
+size_t dense_scratch_bytes(int max_batch, int n, int d_max);
+// DOT[b][c] = <sv[b], centers[c]> for b < B, c < n into scratch; *dots_out = the [B][n] result.
+cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
+                              void* scratch, int max_batch, int d_max, float** dots_out, int* status,
+                              cudaStream_t st, int64_t* launches);
+// Eq. 1 from the dot products, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule; dots: [B][n].
+cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, cudaStream_t st, int64_t* launches);
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,
                                cudaStream_t st, int64_t* launches);
 

@@ -72,6 +72,36 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
     decide_frame(a, b, s_cur, s_acc, mem, k, lane);
 }
 
+// Finishing kernel of the tensor-core path: one CTA per frame turns the frame's row of dot
+// products into similarities of its fast-memory slots and decides.
+__global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, const float* __restrict__ dots) {
+    extern __shared__ float smem[];
+    float* s_cur = smem;             // [k_max]
+    float* s_acc = smem + a.k_max;   // [k_max]
+    __shared__ float scratch[32];
+    const int b = blockIdx.x;
+    if (a.done[b]) return;
+    const int tid = threadIdx.x;
+    const int sid = a.stream_id ? a.stream_id[b] : 0;
+    const int k = a.k[sid];
+    const int32_t* mem = a.members + (size_t)sid * a.k_max;
+    const float* row = a.sv + (size_t)b * a.D;
+    float nrm = 0.f;
+    for (int d = tid; d < a.D; d += kThreads) nrm = fmaf(row[d], row[d], nrm);
+    nrm = block_sum(nrm, scratch);
+    const float weight = float(1u << a.layer);
+    for (int j = tid; j < k; j += kThreads) {
+        const int cls = mem[j];
+        const float s = cosine_from(dots[(size_t)b * a.n + cls], nrm, a.cnorm[cls]);   // Eq. 1
+        const float acc = __fmaf_rn(s, weight, a.sa[(size_t)b * a.k_max + j]);         // Eq. 3
+        a.sa[(size_t)b * a.k_max + j] = acc;
+        s_cur[j] = s;
+        s_acc[j] = acc;
+    }
+    __syncthreads();
+    if (tid < kWarp) decide_frame(a, b, s_cur, s_acc, mem, k, tid);
+}
+
 // Finishing kernel of the fused lookup: a warp per frame.  Lane l looks after slots l and
 // l + 32; the parts of each sum are added in part order.
 __global__ void __launch_bounds__(kThreads) k_finish_partials(const LookupArgs a, const float* __restrict__ partials,
@@ -154,6 +184,20 @@ cudaError_t launch_finish_partials(const LookupArgs& a, const float* partials, i
     ++*launches;
     const int per_cta = kThreads / kWarp;
     k_finish_partials<<<(a.B + per_cta - 1) / per_cta, kThreads, 0, st>>>(a, partials, parts);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, cudaStream_t st, int64_t* launches) {
+    if (a.B <= 0) return cudaSuccess;
+    const size_t smem = 2 * size_t(a.k_max) * sizeof(float);
+    static size_t opted = 48 * 1024;
+    if (smem > opted) {
+        cudaError_t e = cudaFuncSetAttribute(k_finish_dense, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
+        opted = smem;
+    }
+    ++*launches;
+    k_finish_dense<<<a.B, kThreads, smem, st>>>(a, dots);
     return cudaGetLastError();
 }
 

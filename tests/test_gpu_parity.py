@@ -170,6 +170,19 @@ def test_adaptive_size_moves_and_ragged_small_cases():
     assert rep2.frames == 19 * 20
 
 
+def test_large_fast_memory_over_several_layers_uses_tensor_cores():
+    # fast memories above 64 entries take the tensor-core scorer; ragged batch, class count that is not a
+    # multiple of the tile, two exit layers (cumulative similarity over all slots), two streams, updates
+    w = si.Workload("dense", si.BF16, si.NCHW, B=70, stages=((256, 14, 14), (512, 7, 7)), n=196, k_init=100,
+                    k_min=70, k_max=196, S=1, T=4, tau=0.8, window_W=2, sigma=0.6, zipf_s=0.9, repeat_p=0.3, seed=6)
+    rep = run_workload(w)
+    assert rep.frames == 70 * 4 and rep.lookups > 70
+    w3 = si.Workload("dense_nhwc", si.F16, si.NHWC, B=33, stages=((320, 7, 7),), n=72, k_init=72, k_min=72, k_max=72,
+                     S=1, T=2, tau=0.8, sigma=1.0, zipf_s=1.0, seed=8)
+    rep3 = run_workload(w3)
+    assert rep3.frames == 66
+
+
 def test_step_host_matches_device_path():
     w = si.C5.scaled(B=32, S=32, T=3)
     cents, counts = si.initial_centers(w)
