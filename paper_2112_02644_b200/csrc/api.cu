@@ -22,6 +22,8 @@ struct smtm_cache {
     int* d_status;
     float* d_partials;  // scratch of the fused lookup: partial dot products per (frame, part)
     void* d_dense;      // scratch of the tensor-core scorer (fast memories above 64 entries), else NULL
+    void* d_cen_split[SMTM_MAX_LAYERS];   // bf16 heads and tails of the centres, per layer (same condition)
+    bool cen_split_current[SMTM_MAX_LAYERS];  // false after creation and after every update
     int d_max;          // largest C_l
     int32_t* d_plan;    // scratch of the update: final label and stop layer, 2 x [max_batch]
     unsigned long long* d_tags;  // scratch of the update: election tags, [n] + [S]
@@ -81,6 +83,7 @@ void free_all(smtm_cache* c) {
         cudaFree(c->d_cnorm[l]);
         cudaFree(c->d_m[l]);
         cudaFree(c->d_stage[l]);
+        cudaFree(c->d_cen_split[l]);
         cudaFree(c->hb.d_sv[l]);
     }
     cudaFree(c->d_ft);
@@ -168,13 +171,19 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     }
     SMTM_CUDA(launch_lookup_fused(e, a, c->d_partials, c->sm_count, st, &c->launches, &fused, timing));
     if (fused) return SMTM_OK;
+    const bool dense = c->d_dense && dense_scoring_supported(a.D, a.n);  // large fast memory: tensor cores
+    EncodeArgs e2 = e;
+    if (dense) dense_sv_split(c->d_dense, c->max_batch, c->d_max, &e2.sv_hi, &e2.sv_lo);
+    bool sv_split = false;
     if (timing) SMTM_CUDA(cudaEventRecord(timing[0], st));
-    SMTM_CUDA(launch_encode(e, c->sm_count, st, &c->launches));
+    SMTM_CUDA(launch_encode(e2, c->sm_count, st, &c->launches, &sv_split));
     if (timing) SMTM_CUDA(cudaEventRecord(timing[1], st));
-    if (c->d_dense && dense_scoring_supported(a.D, a.n)) {  // large fast memory: tensor cores
+    if (dense) {
         float* dots = nullptr;
-        SMTM_CUDA(launch_dense_dots(a.sv, a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max, &dots,
-                                    c->d_status, st, &c->launches));
+        SMTM_CUDA(launch_dense_dots(a.sv, a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max,
+                                    sv_split, c->d_cen_split[layer], c->cen_split_current[layer], &dots, c->d_status,
+                                    st, &c->launches));
+        c->cen_split_current[layer] = true;
         SMTM_CUDA(launch_finish_dense(a, dots, st, &c->launches));
         return SMTM_OK;
     }
@@ -226,6 +235,7 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
         a.m[l] = c->d_m[l];
     }
     const ResizeArgs rz = resize_args(c);
+    for (int l = 0; l < c->L; ++l) c->cen_split_current[l] = false;  // Eq. 7 is about to move centres
     SMTM_CUDA(launch_update(a, with_resize ? &rz : nullptr, st, &c->launches));
     return SMTM_OK;
 }
@@ -314,8 +324,11 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     ok = ok && dev_alloc(&c->d_plan, 2 * size_t(c->max_batch)) == cudaSuccess;
     for (int l = 0; l < c->L; ++l) c->d_max = c->dims[l] > c->d_max ? c->dims[l] : c->d_max;
     c->d_max = (c->d_max + 7) / 8 * 8;  // keeps the bf16 operand arrays of the tensor-core scorer 16-byte aligned
-    if (ok && c->k_max > kFusedMaxK)
+    if (ok && c->k_max > kFusedMaxK) {
         ok = cudaMalloc(&c->d_dense, dense_scratch_bytes(c->max_batch, n, c->d_max)) == cudaSuccess;
+        for (int l = 0; ok && l < c->L; ++l)
+            ok = cudaMalloc(&c->d_cen_split[l], dense_centers_split_bytes(n, c->dims[l])) == cudaSuccess;
+    }
     ok = ok && dev_alloc(&c->d_tags, size_t(n) + size_t(S)) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();
@@ -448,6 +461,7 @@ smtm_status_t smtm_step_host(smtm_cache_t* c, const smtm_fmap_t* fmaps, const vo
         if (need > c->stage_bytes[l]) {
             (void)cudaStreamSynchronize(st);
             cudaFree(c->d_stage[l]);
+        cudaFree(c->d_cen_split[l]);
             c->d_stage[l] = nullptr;
             c->stage_bytes[l] = 0;
             if (cudaMalloc(&c->d_stage[l], need) != cudaSuccess) {

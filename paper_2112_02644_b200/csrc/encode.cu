@@ -39,6 +39,8 @@ struct NchwParams {
     const uint8_t* x;
     const uint8_t* skip;
     float* sv;
+    __nv_bfloat16* sv_hi;    // optional bf16 head and tail of sv (sv = hi + lo), same indexing; may be null
+    __nv_bfloat16* sv_lo;
     int* status;
     long long total_chunks;  // B * chunks per frame
     int C;
@@ -52,6 +54,19 @@ struct NchwParams {
     int max_in_flight;       // copies the producer keeps outstanding (<= kStages)
 };
 
+// Writes the bf16 head and tail of n consecutive values (n a multiple of 2, dst 4-byte aligned).
+template <int N>
+__device__ __forceinline__ void store_split(const float (&v)[N], __nv_bfloat16* hi, __nv_bfloat16* lo) {
+#pragma unroll
+    for (int g = 0; g < N; g += 2) {
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(v[g]), h1 = __float2bfloat16_rn(v[g + 1]);
+        const __nv_bfloat16 l0 = __float2bfloat16_rn(v[g] - __bfloat162float(h0));
+        const __nv_bfloat16 l1 = __float2bfloat16_rn(v[g + 1] - __bfloat162float(h1));
+        *reinterpret_cast<__nv_bfloat162*>(hi + g) = __nv_bfloat162(h0, h1);
+        *reinterpret_cast<__nv_bfloat162*>(lo + g) = __nv_bfloat162(l0, l1);
+    }
+}
+
 // ---- reducers --------------------------------------------------------------------------
 
 // Lane i reduces unit i: G channels of HW elements stored as UW consecutive 16-byte vectors.
@@ -63,7 +78,7 @@ struct UnitPerLane {
     static constexpr int UW = G * kUnitBytesRaw / 16;
 
     static __device__ __forceinline__ void run(const uint8_t* stage, int nch, int lane, float* out, float* out_s,
-                                               float inv_hw, const NchwParams&) {
+                                               float inv_hw, const NchwParams& p) {
         const int units = nch / G;
         if (lane >= units) return;
         const uint4* u = reinterpret_cast<const uint4*>(stage) + lane * UW;
@@ -85,6 +100,10 @@ struct UnitPerLane {
 #pragma unroll
             for (int g = 0; g + 3 < G; g += 4)
                 *reinterpret_cast<float4*>(o + g) = make_float4(acc[g], acc[g + 1], acc[g + 2], acc[g + 3]);
+        }
+        if (p.sv_hi) {
+            const ptrdiff_t at = (o - p.sv);
+            store_split<G>(acc, p.sv_hi + at, p.sv_lo + at);
         }
         if (out_s) {
             float* os = out_s + lane * G;
@@ -126,8 +145,15 @@ struct TeamPerChannel {
             float s = (a0 + a1) + (a2 + a3);
             for (int o = T >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(kFull, s, o);
             if (c < nch && r == 0) {
-                out[c] = s * inv_hw;
-                if (out_s) out_s[c] = s * inv_hw;
+                const float v = s * inv_hw;
+                out[c] = v;
+                if (out_s) out_s[c] = v;
+                if (p.sv_hi) {
+                    const ptrdiff_t at = (out + c) - p.sv;
+                    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+                    p.sv_hi[at] = h;
+                    p.sv_lo[at] = __float2bfloat16_rn(v - __bfloat162float(h));
+                }
             }
         }
     }
@@ -563,6 +589,8 @@ Reducer plan_nchw(const EncodeArgs& a, NchwParams* p) {
     p->x = static_cast<const uint8_t*>(a.x);
     p->skip = a.skip;
     p->sv = a.sv;
+    p->sv_hi = static_cast<__nv_bfloat16*>(a.sv_hi);
+    p->sv_lo = static_cast<__nv_bfloat16*>(a.sv_lo);
     p->status = a.status;
     p->C = a.C;
     p->ch_bytes = HW * es;
@@ -627,7 +655,8 @@ cudaError_t encode_setup() {
     return e;
 }
 
-cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches) {
+cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches, bool* wrote_split) {
+    if (wrote_split) *wrote_split = false;
     if (a.B <= 0) return cudaSuccess;
     ++*launches;
     if (a.layout == SMTM_NHWC) {
@@ -642,6 +671,7 @@ cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, in
         const Reducer r = plan_nchw(a, &p);
         if (r != kNone) {
             cudaError_t e = cudaSuccess;
+            if (wrote_split) *wrote_split = p.sv_hi != nullptr;
 #define SMTM_LAUNCH(...) e = launch_nchw<__VA_ARGS__>(p, sm_count, st)
             SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
 #undef SMTM_LAUNCH

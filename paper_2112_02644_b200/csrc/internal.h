@@ -18,10 +18,14 @@ struct EncodeArgs {
     int B, C, H, W;
     const uint8_t* skip;  // device [B] or nullptr
     float* sv;            // device [B][C]
+    void* sv_hi;          // optional: bf16 head and tail of sv for the tensor-core scorer (same indexing)
+    void* sv_lo;
     int* status;          // device sticky status word
 };
 // Enqueues the pooling of every non-skipped frame.  *launches is incremented per kernel launched.
-cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches);
+// *wrote_split (may be null) tells whether sv_hi / sv_lo were filled by the kernel that ran.
+cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches,
+                          bool* wrote_split = nullptr);
 // Opt-in to large dynamic shared memory for the kernels that need it (once per device).
 cudaError_t encode_setup();
 cudaError_t launch_row_norm2(const float* sv, const uint8_t* skip, int B, int D, float* out, cudaStream_t st,
@@ -64,9 +68,14 @@ cudaError_t launch_finish_partials(const LookupArgs& a, const float* partials, i
 bool dense_scoring_supported(int D, int n);
 size_t dense_scratch_bytes(int max_batch, int n, int d_max);
 // DOT[b][c] = <sv[b], centers[c]> for b < B, c < n into scratch; *dots_out = the [B][n] result.
+// The bf16 heads and tails of the semantic vectors sit at the start of scratch (see
+// dense_sv_split); sv_split_done / centers_split_done say whether they are already current.
+void dense_sv_split(void* scratch, int max_batch, int d_max, void** hi, void** lo);
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
-                              void* scratch, int max_batch, int d_max, float** dots_out, int* status,
-                              cudaStream_t st, int64_t* launches);
+                              void* scratch, int max_batch, int d_max, bool sv_split_done, void* centers_split,
+                              bool centers_split_done, float** dots_out, int* status, cudaStream_t st,
+                              int64_t* launches);
+size_t dense_centers_split_bytes(int n, int D);
 // Eq. 1 from the dot products, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule; dots: [B][n].
 cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, cudaStream_t st, int64_t* launches);
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,

@@ -73,33 +73,72 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
 }
 
 // Finishing kernel of the tensor-core path: one CTA per frame turns the frame's row of dot
-// products into similarities of its fast-memory slots and decides.
+// products into similarities of its fast-memory slots and decides.  Every thread keeps the
+// two best of its own slots; warps merge by shuffles, the CTA through shared memory.
 __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, const float* __restrict__ dots) {
-    extern __shared__ float smem[];
-    float* s_cur = smem;             // [k_max]
-    float* s_acc = smem + a.k_max;   // [k_max]
     __shared__ float scratch[32];
+    __shared__ Top2 s_top[2][kThreads / kWarp];
     const int b = blockIdx.x;
     if (a.done[b]) return;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sid = a.stream_id ? a.stream_id[b] : 0;
     const int k = a.k[sid];
     const int32_t* mem = a.members + (size_t)sid * a.k_max;
     const float* row = a.sv + (size_t)b * a.D;
-    float nrm = 0.f;
-    for (int d = tid; d < a.D; d += kThreads) nrm = fmaf(row[d], row[d], nrm);
-    nrm = block_sum(nrm, scratch);
     const float weight = float(1u << a.layer);
-    for (int j = tid; j < k; j += kThreads) {
-        const int cls = mem[j];
-        const float s = cosine_from(dots[(size_t)b * a.n + cls], nrm, a.cnorm[cls]);   // Eq. 1
-        const float acc = __fmaf_rn(s, weight, a.sa[(size_t)b * a.k_max + j]);         // Eq. 3
-        a.sa[(size_t)b * a.k_max + j] = acc;
-        s_cur[j] = s;
-        s_acc[j] = acc;
+    const float* __restrict__ drow = dots + (size_t)b * a.n;
+    const float* __restrict__ clen = a.cnorm;
+    float* sa_row = a.sa + (size_t)b * a.k_max;
+    Top2 ta{0.f, 0.f, -1, -1}, ts{0.f, 0.f, -1, -1};
+    float nrm = 0.f;
+    for (int j0 = 0; j0 < k; j0 += 4 * kThreads) {  // four slots per thread, every load issued before any store
+        int cls[4];
+        float dot[4], cl[4], old[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + u * kThreads + tid;
+            cls[u] = j < k ? mem[j] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + u * kThreads + tid;
+            dot[u] = j < k ? drow[cls[u]] : 0.f;
+            cl[u] = j < k ? clen[cls[u]] : 0.f;
+            old[u] = j < k ? sa_row[j] : 0.f;
+        }
+        if (j0 == 0) {  // the squared length of the semantic vector, while the loads above are in flight
+            for (int d = tid; d < a.D; d += kThreads) nrm = fmaf(row[d], row[d], nrm);
+            nrm = block_sum(nrm, scratch);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + u * kThreads + tid;
+            if (j < k) {
+                const float s = cosine_from(dot[u], nrm, cl[u]);   // Eq. 1
+                const float acc = __fmaf_rn(s, weight, old[u]);    // Eq. 3
+                sa_row[j] = acc;
+                top2_push(ts, s, cls[u]);
+                top2_push(ta, acc, cls[u]);
+            }
+        }
+    }
+    ta = warp_top2_merge(ta);
+    ts = warp_top2_merge(ts);
+    if (lane == 0) {
+        s_top[0][warp] = ta;
+        s_top[1][warp] = ts;
     }
     __syncthreads();
-    if (tid < kWarp) decide_frame(a, b, s_cur, s_acc, mem, k, tid);
+    if (tid == 0) {
+        for (int w = 1; w < kThreads / kWarp; ++w) {
+            const Top2 oa = s_top[0][w], os = s_top[1][w];
+            if (oa.id1 >= 0) top2_push(ta, oa.v1, oa.id1);
+            if (oa.id2 >= 0) top2_push(ta, oa.v2, oa.id2);
+            if (os.id1 >= 0) top2_push(ts, os.v1, os.id1);
+            if (os.id2 >= 0) top2_push(ts, os.v2, os.id2);
+        }
+        decide_from_top2(a, b, ta, ts);
+    }
 }
 
 // Finishing kernel of the fused lookup: a warp per frame.  Lane l looks after slots l and
@@ -189,15 +228,8 @@ cudaError_t launch_finish_partials(const LookupArgs& a, const float* partials, i
 
 cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, cudaStream_t st, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
-    const size_t smem = 2 * size_t(a.k_max) * sizeof(float);
-    static size_t opted = 48 * 1024;
-    if (smem > opted) {
-        cudaError_t e = cudaFuncSetAttribute(k_finish_dense, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-        if (e != cudaSuccess) return e;
-        opted = smem;
-    }
     ++*launches;
-    k_finish_dense<<<a.B, kThreads, smem, st>>>(a, dots);
+    k_finish_dense<<<a.B, kThreads, 0, st>>>(a, dots);
     return cudaGetLastError();
 }
 

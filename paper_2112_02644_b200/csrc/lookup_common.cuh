@@ -54,6 +54,18 @@ __device__ __forceinline__ float ratio_margin(float top, float second) {
 
 __device__ __forceinline__ void decide_from_top2(const LookupArgs& a, int b, const Top2& ta, const Top2& ts);
 
+// Butterfly merge of per-lane pairs: every lane ends up with the warp's best two.
+__device__ __forceinline__ Top2 warp_top2_merge(Top2 t) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov1 = __shfl_xor_sync(kFull, t.v1, o), ov2 = __shfl_xor_sync(kFull, t.v2, o);
+        const int oi1 = __shfl_xor_sync(kFull, t.id1, o), oi2 = __shfl_xor_sync(kFull, t.id2, o);
+        if (oi1 >= 0) top2_push(t, ov1, oi1);
+        if (oi2 >= 0) top2_push(t, ov2, oi2);
+    }
+    return t;
+}
+
 // Best two of values held in registers: lane l holds slots l and l + 32 (v[0], v[1]) of k.
 __device__ __forceinline__ Top2 warp_top2_regs(const float (&v)[2], const int (&ids)[2], int k, int lane) {
     Top2 t{0.f, 0.f, -1, -1};

@@ -292,19 +292,28 @@ bool dense_scoring_supported(int D, int n) {
 }
 
 size_t dense_scratch_bytes(int max_batch, int n, int d_max) {
-    // bf16 heads and tails of the semantic vectors and of the centres, then the dot products
-    return (size_t(max_batch) + size_t(n)) * d_max * 2 * 2 + size_t(max_batch) * n * sizeof(float) + 1024;
+    // bf16 heads and tails of the semantic vectors, then the dot products
+    return size_t(max_batch) * d_max * 2 * 2 + size_t(max_batch) * n * sizeof(float) + 1024;
+}
+
+size_t dense_centers_split_bytes(int n, int D) { return size_t(n) * D * 2 * 2; }
+
+void dense_sv_split(void* scratch, int max_batch, int d_max, void** hi, void** lo) {
+    __nv_bfloat16* a_hi = reinterpret_cast<__nv_bfloat16*>(scratch);
+    *hi = a_hi;
+    *lo = a_hi + size_t(max_batch) * d_max;
 }
 
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
-                              void* scratch, int max_batch, int d_max, float** dots_out, int* status,
-                              cudaStream_t st, int64_t* launches) {
+                              void* scratch, int max_batch, int d_max, bool sv_split_done, void* centers_split,
+                              bool centers_split_done, float** dots_out, int* status, cudaStream_t st,
+                              int64_t* launches) {
     __nv_bfloat16* a_hi = reinterpret_cast<__nv_bfloat16*>(scratch);
     __nv_bfloat16* a_lo = a_hi + size_t(max_batch) * d_max;
-    __nv_bfloat16* b_hi = a_lo + size_t(max_batch) * d_max;
-    __nv_bfloat16* b_lo = b_hi + size_t(n) * d_max;
+    __nv_bfloat16* b_hi = reinterpret_cast<__nv_bfloat16*>(centers_split);
+    __nv_bfloat16* b_lo = b_hi + size_t(n) * D;
     float* dots = reinterpret_cast<float*>(
-        (reinterpret_cast<uintptr_t>(b_lo + size_t(n) * d_max) + 255) & ~uintptr_t(255));
+        (reinterpret_cast<uintptr_t>(a_lo + size_t(max_batch) * d_max) + 255) & ~uintptr_t(255));
     *dots_out = dots;
 
     CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo;
@@ -318,11 +327,17 @@ cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const
         if (e != cudaSuccess) return e;
         opted = true;
     }
-    *launches += 3;
-    const int grid_a = int(std::min<long long>(((long long)B * D / 4 + 255) / 256, 148 * 8));
-    k_split_bf16<<<grid_a, 256, 0, st>>>(sv, skip, B, D, a_hi, a_lo);
-    const int grid_b = int(std::min<long long>(((long long)n * D / 4 + 255) / 256, 148 * 8));
-    k_split_bf16<<<grid_b, 256, 0, st>>>(centers, nullptr, n, D, b_hi, b_lo);
+    if (!sv_split_done) {
+        ++*launches;
+        const int grid_a = int(std::min<long long>(((long long)B * D / 4 + 255) / 256, 148 * 8));
+        k_split_bf16<<<grid_a, 256, 0, st>>>(sv, skip, B, D, a_hi, a_lo);
+    }
+    if (!centers_split_done) {
+        ++*launches;
+        const int grid_b = int(std::min<long long>(((long long)n * D / 4 + 255) / 256, 148 * 8));
+        k_split_bf16<<<grid_b, 256, 0, st>>>(centers, nullptr, n, D, b_hi, b_lo);
+    }
+    ++*launches;
     TcParams p{};
     p.M = B;
     p.N = n;
