@@ -28,7 +28,7 @@ sys.path.insert(0, ROOT)
 
 import smtm_inputs as si  # noqa: E402
 
-WORKLOAD = si.C5
+WORKLOAD = si.C5   # the default and the benchmark line of record; --workload picks another for profiling
 METRIC = "frames/sec through encode+lookup+exit per exit layer (whole path incl. update+resize)"
 
 
@@ -112,7 +112,8 @@ def run_ours(args):
 
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     # every rank serves its own 512 streams (weak scaling by stream); no data-path collective
-    w = WORKLOAD.scaled(seed=WORKLOAD.seed + rank)
+    base = si.WORKLOADS[[k for k in si.WORKLOADS if k.startswith(args.workload)][0]]
+    w = base.scaled(seed=base.seed + rank, T=max(base.T, 8))
     K, W = args.steps, args.warmup
     T = min(w.T, max(K, W))
     labs = si.labels(w)
@@ -177,16 +178,17 @@ def run_ours(args):
     # roofline of the dominant launch (stage-3 lookup: every frame active)
     dom_total_ms, dom_n = smtm.smtm_cache_get_profile(cache, 0)
     dom_ms = dom_total_ms / max(dom_n, 1)
-    l1_total_ms, l1_n = smtm.smtm_cache_get_profile(cache, 1)
+    l1_total_ms, l1_n = smtm.smtm_cache_get_profile(cache, 1) if w.L > 1 else (0.0, 0)
     C0 = w.stages[0][0]
     dom_bytes = w.B * (w.frame_bytes(0) + 4 * C0)
     peak, peak_src = measured_peaks()
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     exits = [int(v) for v in ctr[: w.L]]
+    sid = sid if w.S > 1 else None
 
     e2e = None
     if rank == 0 or world > 1:
-        e2e = run_e2e(smtm, w, cents, counts, labs, maps, sid, min(K, 16), world, sh)
+        e2e = run_e2e(smtm, w, cents, counts, labs, maps, sid if w.S > 1 else None, min(K, 16), world, sh)
     out = None
     if rank == 0:
         out = {
@@ -194,23 +196,25 @@ def run_ours(args):
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "streams_per_gpu": w.S, "frames_per_step_per_gpu": w.B,
-                       "exit_layers": [list(s) for s in w.stages], "map_dtype": "bf16", "layout": "NCHW",
+                       "exit_layers": [list(s) for s in w.stages],
+                       "map_dtype": {si.F32: "f32", si.F16: "f16", si.BF16: "bf16"}[w.dtype],
+                       "layout": "NCHW" if w.layout == si.NCHW else "NHWC",
                        "classes": w.n, "fast_memory": [w.k_min, w.k_max], "tau": w.tau, "window_W": w.window_W,
-                       "distinct_steps_resident": T, "l2_policy": "inputs larger than L2: 308 MB of distinct maps per step",
+                       "distinct_steps_resident": T, "l2_policy": "distinct maps per step, %.0f MB per step (L2 is 126 MB)" % (sum(w.B * w.frame_bytes(l) for l in range(w.L)) / 1e6),
                        "sharding": "streams across GPUs, no collective"},
             "e2e": e2e,
             "gpu_launches": int(launches),
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "k_lookup_nchw at stage 3 (fused encode + similarity scoring, 512 frames per launch)", "achieved": achieved,
+            "roofline": {"bound": "hbm", "kernel": "streaming kernel of the first exit layer (fused encode + similarity scoring where the fast memory has <= 64 entries), %d frames per launch" % w.B, "achieved": achieved,
                          "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                          "traffic": None, "bytes_per_launch": dom_bytes, "us_per_launch": dom_ms * 1e3,
                          "frac_of_nominal_8TBs": achieved / 8000.0, "launches_timed": int(dom_n),
                          "stage4_kernel_us_per_launch": l1_total_ms / max(l1_n, 1) * 1e3},
-            "exit_histogram": {"stage3": exits[0], "stage4": exits[1], "none": K * w.B - sum(exits)},
+            "exit_histogram": {"per_layer": exits, "none": K * w.B - sum(exits)},
             "near_threshold_lookups": int(ctr[smtm.CTR_NEAR]),
             "device_status": status,
         }
-        if world == 1:
+        if world == 1 and not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline(w, budget_s=12.0)
     smtm.smtm_cache_destroy(cache)
     if world > 1:
@@ -310,6 +314,8 @@ def main():
     ap.add_argument("--steps", type=int, default=640)
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c5", help="c1..c5 (prefix of a workload name); c5 is the benchmark of record")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     out = run_reference(args) if args.impl == "reference" else run_ours(args)

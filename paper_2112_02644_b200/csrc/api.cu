@@ -461,7 +461,6 @@ smtm_status_t smtm_step_host(smtm_cache_t* c, const smtm_fmap_t* fmaps, const vo
         if (need > c->stage_bytes[l]) {
             (void)cudaStreamSynchronize(st);
             cudaFree(c->d_stage[l]);
-        cudaFree(c->d_cen_split[l]);
             c->d_stage[l] = nullptr;
             c->stage_bytes[l] = 0;
             if (cudaMalloc(&c->d_stage[l], need) != cudaSuccess) {
