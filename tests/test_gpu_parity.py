@@ -141,6 +141,7 @@ def test_c3_mobilenetv2_fp16_nhwc_novel_classes_do_not_exit():
 def test_c4_large_cache_straddles_threshold():
     rep = run_workload(si.C4)
     assert 100 < rep.exits[0] < 900
+    print("c4 max |SA error|:", rep.max_sa_err, "max SV error:", rep.max_sv_err)
     print("c4 near-threshold lookups (oracle):", rep.near_oracle, "band mismatches:", rep.band_mismatches)
 
 
