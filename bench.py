@@ -126,8 +126,10 @@ def run_ours(args):
         fmaps.append([smtm.Fmap(m[l], w.dtype, w.layout, *si.shape4(w, l)) for l in range(w.L)])
         fbs.append(torch.from_numpy(si.fallback_labels(w, labs[t])).cuda())
     torch.cuda.synchronize()
-    stream = torch.cuda.current_stream()
-    sh = stream.cuda_stream or None
+    # All launches go to one side stream so that every step can be captured into a CUDA graph.
+    stream = torch.cuda.Stream()
+    sh = stream.cuda_stream
+    PROFILE_EVERY = 8   # steps whose streaming kernels carry timing events (the events cost a few us each)
 
     def step(cache, gb, t):
         smtm.smtm_batch_reset(cache, gb, sh)
@@ -135,38 +137,45 @@ def run_ours(args):
             smtm.smtm_lookup_exit(cache, l, fmaps[t % T][l], gb, sh)
         smtm.smtm_cache_update_resize(cache, gb, fbs[t % T], sh)
 
-    # warm-up on a scratch cache (kernels, clocks), then a fresh cache for the timed steps
-    scratch = make_cache(smtm, w, cents, counts)
-    gb = smtm.Batch(scratch, w.B, stream_id=sid, with_diagnostics=False)
-    for t in range(W):
-        step(scratch, gb, t)
-    torch.cuda.synchronize()
-    smtm.smtm_cache_destroy(scratch)
-
     cache = make_cache(smtm, w, cents, counts)
     gb = smtm.Batch(cache, w.B, stream_id=sid, with_diagnostics=False)
-    smtm.smtm_cache_profile(cache, K * w.L)   # CUDA events around the streaming kernel of every lookup
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local_rank)
-    launches0 = smtm.smtm_cache_get_launches(cache)
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    start.record(stream)
-    for t in range(K):
-        smtm.smtm_batch_reset(cache, gb, sh)
-        for l in range(w.L):
-            smtm.smtm_lookup_exit(cache, l, fmaps[t % T][l], gb, sh)
-        smtm.smtm_cache_update_resize(cache, gb, fbs[t % T], sh)
-    stop.record(stream)
-    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        for t in range(W):          # eager warm-up: kernels, clocks, one-time function attributes
+            step(cache, gb, t)
+        stream.synchronize()
+        # one graph per resident step (its feature maps are baked in); the cache state lives in
+        # device memory the graphs point to, so replaying them in order advances it as eager calls would
+        smtm.smtm_cache_profile(cache, (T // PROFILE_EVERY + 1) * w.L, PROFILE_EVERY)
+        launches0 = smtm.smtm_cache_get_launches(cache)
+        graphs = []
+        for t in range(T):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                step(cache, gb, t)
+            graphs.append(g)
+        launches_per_cycle = smtm.smtm_cache_get_launches(cache) - launches0
+        for t in range(W, W + min(3, T)):   # graph warm-up (uploads), continuing the step sequence
+            graphs[t % T].replay()
+        first = W + min(3, T)
+        stream.synchronize()
+        ctr0 = smtm.smtm_cache_get_counters(cache)
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler = ClockSampler(local_rank)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        start.record(stream)
+        for t in range(first, first + K):
+            graphs[t % T].replay()
+        stop.record(stream)
+        torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     clocks = sampler.stop()
     ms = start.elapsed_time(stop)
-    launches = smtm.smtm_cache_get_launches(cache) - launches0
-    ctr = smtm.smtm_cache_get_counters(cache)
+    launches = launches_per_cycle * K // T
+    ctr = smtm.smtm_cache_get_counters(cache) - ctr0
     status = smtm.smtm_cache_status(cache)
     if world > 1:
         tms = torch.tensor([ms], device="cuda", dtype=torch.float64)
@@ -201,7 +210,8 @@ def run_ours(args):
                        "layout": "NCHW" if w.layout == si.NCHW else "NHWC",
                        "classes": w.n, "fast_memory": [w.k_min, w.k_max], "tau": w.tau, "window_W": w.window_W,
                        "distinct_steps_resident": T, "l2_policy": "distinct maps per step, %.0f MB per step (L2 is 126 MB)" % (sum(w.B * w.frame_bytes(l) for l in range(w.L)) / 1e6),
-                       "sharding": "streams across GPUs, no collective"},
+                       "sharding": "streams across GPUs, no collective",
+                       "launch": "one CUDA graph per step (reset, %d lookups, update+refresh)" % w.L},
             "e2e": e2e,
             "gpu_launches": int(launches),
             "clocks": clocks,

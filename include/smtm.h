@@ -213,12 +213,15 @@ smtm_status_t smtm_cache_get_tables(smtm_cache_t* cache, int32_t* h_ft /*[S][n]*
                                     int32_t* h_ts /*[S][n]*/);
 smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMTM_CTR_COUNT]*/);
 
-/* Timing of the streaming kernel (the one that reads the feature maps) of each
- * lookup: with max_lookups > 0 the next max_lookups calls of smtm_lookup_exit
- * record a pair of CUDA events on the caller's stream right around that kernel;
- * 0 switches it off and frees the events.  smtm_cache_get_profile adds up the
- * elapsed times of the recorded lookups of one layer.  Both synchronise the device. */
-smtm_status_t smtm_cache_profile(smtm_cache_t* cache, int32_t max_lookups);
+/* Timing of the streaming kernel (the one that reads the feature maps) of
+ * lookups: with max_lookups > 0, every `every`-th step's calls of
+ * smtm_lookup_exit (a step = L consecutive calls) record a pair of CUDA events on
+ * the caller's stream right around that kernel, up to max_lookups pairs; 0
+ * switches it off and frees the events.  Inside a stream capture the events
+ * become graph nodes that are re-recorded at every replay.
+ * smtm_cache_get_profile adds up the elapsed times of the recorded lookups of
+ * one layer.  Both synchronise the device. */
+smtm_status_t smtm_cache_profile(smtm_cache_t* cache, int32_t max_lookups, int32_t every);
 smtm_status_t smtm_cache_get_profile(smtm_cache_t* cache, int32_t layer, double* h_total_ms, int64_t* h_count);
 
 /* Number of kernels the library has launched on behalf of this cache so far. */

@@ -88,7 +88,7 @@ def load_library():
     lib.smtm_cache_get_tables.argtypes = [vp, vp, vp]
     lib.smtm_cache_get_counters.argtypes = [vp, vp]
     lib.smtm_cache_get_launches.argtypes = [vp, vp]
-    lib.smtm_cache_profile.argtypes = [vp, i32]
+    lib.smtm_cache_profile.argtypes = [vp, i32, i32]
     lib.smtm_cache_get_profile.argtypes = [vp, i32, vp, vp]
     lib.smtm_cache_status.argtypes = [vp]
     lib.smtm_status_string.argtypes = [i32]
@@ -296,8 +296,8 @@ def smtm_cache_get_launches(cache: Cache) -> int:
     return int(out[0])
 
 
-def smtm_cache_profile(cache: Cache, max_lookups: int) -> None:
-    _check(load_library().smtm_cache_profile(cache.handle, int(max_lookups)), "smtm_cache_profile")
+def smtm_cache_profile(cache: Cache, max_lookups: int, every: int = 1) -> None:
+    _check(load_library().smtm_cache_profile(cache.handle, int(max_lookups), int(every)), "smtm_cache_profile")
 
 
 def smtm_cache_get_profile(cache: Cache, layer: int):

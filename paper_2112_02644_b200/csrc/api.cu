@@ -32,6 +32,8 @@ struct smtm_cache {
     std::vector<cudaEvent_t>* prof_events;  // pairs, in launch order
     std::vector<int>* prof_layer;           // layer of each pair
     size_t prof_used;                       // pairs recorded so far
+    int prof_every;                         // a pair is recorded for every prof_every-th lookup call
+    long long prof_seq;                     // lookup calls since profiling was switched on
     int device, sm_count;
     int64_t launches;
     // device-side carry and staging used only by smtm_step_host (allocated on first use)
@@ -165,7 +167,8 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     const EncodeArgs e = encode_args(c, f, b->d_done, b->d_sv[layer]);
     bool fused = false;
     const cudaEvent_t* timing = nullptr;
-    if (c->prof_events && 2 * (c->prof_used + 1) <= c->prof_events->size()) {
+    if (c->prof_events && (c->prof_seq++ / c->L) % c->prof_every == 0 &&
+        2 * (c->prof_used + 1) <= c->prof_events->size()) {
         timing = c->prof_events->data() + 2 * c->prof_used;
         (*c->prof_layer)[c->prof_used++] = layer;
     }
@@ -175,9 +178,9 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     EncodeArgs e2 = e;
     if (dense) dense_sv_split(c->d_dense, c->max_batch, c->d_max, &e2.sv_hi, &e2.sv_lo);
     bool sv_split = false;
-    if (timing) SMTM_CUDA(cudaEventRecord(timing[0], st));
+    if (timing) SMTM_CUDA(record_timing(timing[0], st));
     SMTM_CUDA(launch_encode(e2, c->sm_count, st, &c->launches, &sv_split));
-    if (timing) SMTM_CUDA(cudaEventRecord(timing[1], st));
+    if (timing) SMTM_CUDA(record_timing(timing[1], st));
     if (dense) {
         float* dots = nullptr;
         SMTM_CUDA(launch_dense_dots(a.sv, a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max,
@@ -533,10 +536,12 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* c, int64_t* h_out) {
     return SMTM_OK;
 }
 
-smtm_status_t smtm_cache_profile(smtm_cache_t* c, int32_t max_lookups) {
-    if (!c || max_lookups < 0 || max_lookups > (1 << 20)) return SMTM_ERR_INVALID_ARG;
+smtm_status_t smtm_cache_profile(smtm_cache_t* c, int32_t max_lookups, int32_t every) {
+    if (!c || max_lookups < 0 || max_lookups > (1 << 20) || every < 1) return SMTM_ERR_INVALID_ARG;
     SMTM_CUDA(cudaDeviceSynchronize());
     drop_profile(c);
+    c->prof_every = every;
+    c->prof_seq = 0;
     if (max_lookups == 0) return SMTM_OK;
     c->prof_events = new (std::nothrow) std::vector<cudaEvent_t>();
     c->prof_layer = new (std::nothrow) std::vector<int>(size_t(max_lookups), 0);

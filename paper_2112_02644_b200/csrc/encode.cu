@@ -725,12 +725,12 @@ cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float*
     f.partials = partials;
     const size_t smem = fused_smem(f.slice_cap);
     cudaError_t err = cudaSuccess;
-    if (timing) cudaEventRecord(timing[0], st);
+    if (timing) record_timing(timing[0], st);
 #define SMTM_LAUNCH(...) k_lookup_nchw<__VA_ARGS__><<<sm_count, kThreadsFused, smem, st>>>(f)
     SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
 #undef SMTM_LAUNCH
     err = cudaGetLastError();
-    if (timing) cudaEventRecord(timing[1], st);
+    if (timing) record_timing(timing[1], st);
     ++*launches;
     *handled = true;
     if (err != cudaSuccess) return err;

@@ -8,6 +8,15 @@
 
 namespace smtm {
 
+// Records a timing event on `st`; inside a stream capture it becomes an event-record node that
+// is re-recorded at every replay of the graph.
+inline cudaError_t record_timing(cudaEvent_t ev, cudaStream_t st) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) return cudaGetLastError();
+    return cudaEventRecordWithFlags(ev, st, cap == cudaStreamCaptureStatusActive ? cudaEventRecordExternal
+                                                                                : cudaEventRecordDefault);
+}
+
 // Number of exit layers and the fast-memory capacity of a cache.
 void cache_shape(const smtm_cache_t* cache, int* n_layers, int* k_max);
 
