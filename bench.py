@@ -95,6 +95,25 @@ def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
 
+# --------------------------------------------------------------------------- sharding across ranks
+
+def shard_for_rank(base, rank: int):
+    """Every rank serves its own streams: the same workload recipe under a rank-specific seed."""
+    return base.scaled(seed=base.seed + rank, T=max(base.T, 8))
+
+
+def job_throughput(frames_per_rank: int, ms_local: float, world: int, device="cuda"):
+    """Whole-job frames/s: all ranks' frames over the slowest rank's time (max over ranks)."""
+    ms = ms_local
+    if world > 1:
+        import torch.distributed as dist
+
+        t = torch.tensor([ms_local], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return frames_per_rank * world / (ms * 1e-3), ms
+
+
 # --------------------------------------------------------------------------- the CUDA arm
 
 def make_cache(smtm, w, cents, counts):
@@ -113,7 +132,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     # every rank serves its own 512 streams (weak scaling by stream); no data-path collective
     base = si.WORKLOADS[[k for k in si.WORKLOADS if k.startswith(args.workload)][0]]
-    w = base.scaled(seed=base.seed + rank, T=max(base.T, 8))
+    w = shard_for_rank(base, rank)
     K, W = args.steps, args.warmup
     T = min(w.T, max(K, W))
     labs = si.labels(w)
@@ -177,12 +196,7 @@ def run_ours(args):
     launches = launches_per_cycle * K // T
     ctr = smtm.smtm_cache_get_counters(cache) - ctr0
     status = smtm.smtm_cache_status(cache)
-    if world > 1:
-        tms = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-        ms = float(tms.item())
-    frames = K * w.B * world
-    value = frames / (ms * 1e-3)
+    value, ms = job_throughput(K * w.B, ms, world)
 
     # roofline of the dominant launch (stage-3 lookup: every frame active)
     dom_total_ms, dom_n = smtm.smtm_cache_get_profile(cache, 0)
