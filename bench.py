@@ -118,7 +118,8 @@ def job_throughput(frames_per_rank: int, ms_local: float, world: int, device="cu
 
 def make_cache(smtm, w, cents, counts):
     return smtm.smtm_cache_create(w.n, w.dims, [w.tau] * w.L, cents, counts, n_streams=w.S, k_init=w.k_init,
-                                  k_min=w.k_min, k_max=w.k_max, window_W=w.window_W, max_batch=w.B)
+                                  k_min=w.k_min, k_max=w.k_max, window_W=w.window_W, max_batch=w.B,
+                                  flags=smtm.FLAG_FORGET_FT if w.forgetting else 0)
 
 
 def run_ours(args):
@@ -285,7 +286,8 @@ def oracle_steps(w, n_steps, budget_s=None, device="cpu"):
 
     labs = si.labels(w)
     cents, counts = si.initial_centers(w)
-    mem = oracle.OracleMemory(w.n, w.dims, [w.tau] * w.L, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W)
+    mem = oracle.OracleMemory(w.n, w.dims, [w.tau] * w.L, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W,
+                              forgetting=w.forgetting)
     sid = si.stream_ids(w)
     spent, frames = 0.0, 0
     for t in range(n_steps):

@@ -66,6 +66,14 @@ enum {
     SMTM_CTR_COUNT = SMTM_MAX_LAYERS + 2
 };
 
+/* Config flag.  SMTM_FLAG_FORGET_FT: the variant the paper uses for rapidly changing scenes
+ * (Sec. 7.1, "decay the historical memory in the frequency table" by the forgetting mechanism
+ * of Sec. 6.1): the 0.25-per-window decay of Eq. 5 is applied to the frequency table itself.
+ * FT is then fixed point with 10 fractional bits (smtm_cache_get_tables returns it raw): an
+ * appearance adds 1024, each further W consecutive unseen frames multiply it by 0.25 rounding
+ * down, and Eq. 5's score is FT itself. */
+enum { SMTM_FLAG_FORGET_FT = 1 };
+
 typedef struct {
     int32_t n_classes;      /* n: classes in global memory (Sec. 6), 1..SMTM_MAX_CLASSES */
     int32_t n_layers;       /* L: candidate exit layers (Sec. 4.2), 1..SMTM_MAX_LAYERS */
@@ -77,7 +85,7 @@ typedef struct {
     int32_t window_W;       /* W of Eq. 5, >= 1 */
     int32_t cl_num, cl_den; /* confidence level of Eq. 6 as a fraction, e.g. 19/20 */
     int32_t max_batch;      /* largest B any call will pass; sizes the library's scratch */
-    uint32_t flags;         /* reserved, must be 0 */
+    uint32_t flags;         /* 0 or SMTM_FLAG_FORGET_FT */
 } smtm_config_t;
 
 /* A batch of feature maps at one exit layer: dense, frame stride C*H*W elements,
@@ -184,6 +192,15 @@ smtm_status_t smtm_cache_update(smtm_cache_t* cache, const smtm_batch_t* batch,
  * refreshed after their own last update). */
 smtm_status_t smtm_cache_update_resize(smtm_cache_t* cache, const smtm_batch_t* batch,
                                        const int32_t* d_fallback_label, void* stream);
+
+/* Centre warm-up (Sec. 5: the centres are "initialized with a grouping center (the
+ * average of semantic vectors) on the training dataset"; Sec. 6.3): encodes a batch
+ * of labelled frames at `layer` and folds each into the centre of its class
+ * d_labels[b] (-1 = skip) by Eq. 7 in ascending frame order; a centre created with
+ * count 0 thereby becomes the class mean.  Tables and fast memories are not touched.
+ * The first call allocates [max_batch][max C_l] floats of scratch. */
+smtm_status_t smtm_cache_warmup(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t* fmap,
+                                const int32_t* d_labels, void* stream);
 
 /* Eq. 5 and Eq. 6 for every stream: Score_i = FT_i 0.25^floor(TS_i / W) (exact,
  * floor clamped at 12); classes ranked by (score descending, id ascending); the

@@ -121,14 +121,24 @@ def lookup_layer(layer: int, sv, centers, stream_id, members, k, tau: float, sa,
     return ac, sep, top, near
 
 
-def tables_update(stream_id, final_label, ft, ts) -> None:
-    """Sec. 6.1 frequency / time-stamp tables, frames applied in ascending index."""
+FT_FRAC = 10   # fractional bits of FT in the forgetting variant
+
+
+def tables_update(stream_id, final_label, ft, ts, forgetting_W: int = 0) -> None:
+    """Sec. 6.1 frequency / time-stamp tables, frames applied in ascending index.
+
+    forgetting_W > 0: the variant of Sec. 7.1 that decays FT itself every W unseen frames."""
     S, n = ft.shape
     for a in (stream_id, final_label, ft, ts):
         assert a.dtype == np.int32 and a.flags.c_contiguous
-    rc = _load().orc_tables_update(len(final_label), _p(stream_id, ctypes.c_int32),
-                                   _p(final_label, ctypes.c_int32), S, n,
-                                   _p(ft, ctypes.c_int32), _p(ts, ctypes.c_int32))
+    if forgetting_W:
+        rc = _load().orc_tables_update_forgetting(len(final_label), _p(stream_id, ctypes.c_int32),
+                                                  _p(final_label, ctypes.c_int32), S, n, int(forgetting_W),
+                                                  _p(ft, ctypes.c_int32), _p(ts, ctypes.c_int32))
+    else:
+        rc = _load().orc_tables_update(len(final_label), _p(stream_id, ctypes.c_int32),
+                                       _p(final_label, ctypes.c_int32), S, n,
+                                       _p(ft, ctypes.c_int32), _p(ts, ctypes.c_int32))
     assert rc == 0, rc
 
 
@@ -146,14 +156,15 @@ def centers_update(l0: int, sv, final_label, stop_layer, centers, m) -> None:
     assert rc == 0, rc
 
 
-def resize(ft, ts, W: int, k_min: int, k_max: int, cl_num: int, cl_den: int, members, k) -> None:
+def resize(ft, ts, W: int, k_min: int, k_max: int, cl_num: int, cl_den: int, members, k,
+           forgetting: bool = False) -> None:
     """Eq. 5 ranking + Eq. 6 adaptive size, per stream; members/k updated in place."""
     S, n = ft.shape
     assert members.shape == (S, k_max) and k.shape == (S,)
     for a in (ft, ts, members, k):
         assert a.dtype == np.int32 and a.flags.c_contiguous
     rc = _load().orc_resize(S, n, _p(ft, ctypes.c_int32), _p(ts, ctypes.c_int32), int(W), int(k_min),
-                            int(k_max), int(cl_num), int(cl_den), _p(members, ctypes.c_int32),
+                            int(k_max), int(cl_num), int(cl_den), int(bool(forgetting)), _p(members, ctypes.c_int32),
                             _p(k, ctypes.c_int32))
     assert rc == 0, rc
 
@@ -171,7 +182,8 @@ class OracleMemory:
     def __init__(self, n_classes: int, dims: Sequence[int], tau: Sequence[float], centers,
                  counts=None, n_streams: int = 1, k_init: int = 5, k_min: int = 2,
                  k_max: int = 5, window_W: int = 16, cl_num: int = 19, cl_den: int = 20,
-                 init_members=None):
+                 init_members=None, forgetting: bool = False):
+        self.forgetting = bool(forgetting)
         self.n, self.L, self.S = int(n_classes), len(dims), int(n_streams)
         self.dims = [int(d) for d in dims]
         self.tau = [float(np.float32(t)) for t in tau]
@@ -222,17 +234,28 @@ class OracleMemory:
         self.exits_per_layer[layer] += int(np.count_nonzero(todo & (batch["done"] == 1)))
         self.near_count += int(near[todo].sum())
 
+    def warmup(self, layer: int, fmap, dtype: int, layout: int, shape, labels) -> None:
+        """Centre warm-up (Sec. 5, Sec. 6.3): labelled frames folded into their classes' centres
+        at one layer (0-based) by Eq. 7, in ascending frame order."""
+        B, C, H, W = shape
+        sv = gap(fmap, dtype, layout, B, C, H, W)
+        lab = np.ascontiguousarray(labels, np.int32)
+        lab = np.where(lab >= self.n, -1, lab).astype(np.int32)
+        stop = np.full(B, self.L, np.int32)
+        centers_update(layer + 1, sv, lab, stop, self.centers[layer], self.m[layer])
+
     def update(self, batch: dict, fallback_label=None) -> None:
         """After-inference updates for the whole batch (Sec. 6.1 tables, Eq. 7 centres)."""
         B = batch["B"]
         fb = np.full(B, -1, np.int32) if fallback_label is None else np.asarray(fallback_label, np.int32)
+        fb = np.where(fb >= self.n, -1, fb)    # a label outside the memory counts as no label
         exited = batch["done"] == 1
         final = np.ascontiguousarray(np.where(exited, batch["pred"], fb), np.int32)
         stop = np.ascontiguousarray(np.where(exited, batch["exit_layer"], self.L), np.int32)
-        tables_update(batch["stream_id"], final, self.ft, self.ts)
+        tables_update(batch["stream_id"], final, self.ft, self.ts, self.W if self.forgetting else 0)
         for l0 in range(1, self.L + 1):
             centers_update(l0, batch["sv"][l0 - 1], final, stop, self.centers[l0 - 1], self.m[l0 - 1])
 
     def resize(self) -> None:
         resize(self.ft, self.ts, self.W, self.k_min, self.k_max, self.cl_num, self.cl_den,
-               self.members, self.k)
+               self.members, self.k, forgetting=self.forgetting)

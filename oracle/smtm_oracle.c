@@ -256,6 +256,41 @@ int orc_tables_update(int B, const int32_t* stream_id, const int32_t* final_labe
     return 0;
 }
 
+/* The variant of Sec. 7.1 ("decay the historical memory in the frequency table
+ * based on the forgetting mechanism" of Sec. 6.1): the decay of Eq. 5 is applied
+ * to the table itself.  FT is held in fixed point with ORC_FT_FRAC fractional
+ * bits: an appearance adds one unit, and each time a class has gone another W
+ * consecutive frames unseen (TS reaches a multiple of W) its FT is multiplied
+ * by 0.25, rounding down.  Until the class reappears this keeps FT equal to
+ * Eq. 5's score of the plain tables (up to that rounding), but the history
+ * stays forgotten when it does reappear. */
+#define ORC_FT_FRAC 10
+
+int orc_tables_update_forgetting(int B, const int32_t* stream_id, const int32_t* final_label, int S, int n,
+                                 int W, int32_t* ft, int32_t* ts) {
+    int b, i;
+    if (W < 1) return 1;
+    for (b = 0; b < B; ++b) {
+        int sid = stream_id ? stream_id[b] : 0;
+        int lab = final_label[b];
+        int32_t* f = ft + (size_t)sid * n;
+        int32_t* t = ts + (size_t)sid * n;
+        if (sid < 0 || sid >= S || lab >= n) return 3;
+        for (i = 0; i < n; ++i) {
+            if (i == lab) {
+                int64_t v = (int64_t)f[i] + (1 << ORC_FT_FRAC);
+                int64_t cap = (int64_t)ORC_FT_MAX << ORC_FT_FRAC;
+                f[i] = (int32_t)(v > cap ? cap : v);
+                t[i] = 0;
+            } else if (t[i] < INT32_MAX) {
+                t[i] += 1;
+                if (t[i] % W == 0) f[i] >>= 2;
+            }
+        }
+    }
+    return 0;
+}
+
 /* ---- Sec. 6.3, Eq. 7: adaptive semantic centres --------------------------- */
 
 /* For one layer l0 (1-based): every frame, in ascending index, whose final
@@ -296,9 +331,10 @@ uint64_t orc_score(int32_t ft, int32_t ts, int W) {
  *     sum of the k best scores / sum of all scores  >  cl_num / cl_den
  * (k_max when none does), and the fast memory the first k of the ranking
  * (members holds the first k_max of it).  A stream whose scores are all zero
- * keeps its size and members. */
+ * keeps its size and members.  forgetting != 0: the tables are those of
+ * orc_tables_update_forgetting. */
 int orc_resize(int S, int n, const int32_t* ft, const int32_t* ts, int W, int k_min, int k_max,
-               int cl_num, int cl_den, int32_t* members, int32_t* k) {
+               int cl_num, int cl_den, int forgetting, int32_t* members, int32_t* k) {
     int s, i, j;
     uint64_t* score;
     int32_t* order;
@@ -314,7 +350,9 @@ int orc_resize(int S, int n, const int32_t* ft, const int32_t* ts, int W, int k_
         uint64_t total = 0, prefix = 0;
         int chosen = k_max;
         for (i = 0; i < n; ++i) {
-            score[i] = orc_score(ft[(size_t)s * n + i], ts[(size_t)s * n + i], W);
+            /* with the forgetting tables the decay already sits in FT: the score is FT itself */
+            score[i] = forgetting ? (uint64_t)(ft[(size_t)s * n + i] < 0 ? 0 : ft[(size_t)s * n + i])
+                                  : orc_score(ft[(size_t)s * n + i], ts[(size_t)s * n + i], W);
             total += score[i];
         }
         if (total == 0) continue;

@@ -18,6 +18,7 @@ import numpy as np
 F32, F16, BF16 = 0, 1, 2
 NCHW, NHWC = 0, 1
 MAX_LAYERS = 16
+FLAG_FORGET_FT = 1   # the frequency table itself forgets (fixed point, 10 fractional bits)
 CTR_EXITS, CTR_NEAR, CTR_LOOKUPS, CTR_COUNT = 0, MAX_LAYERS, MAX_LAYERS + 1, MAX_LAYERS + 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -67,6 +68,14 @@ def load_library():
     global _lib
     if _lib is not None:
         return _lib
+    from . import build as _build
+    if _build.stale():
+        import shutil
+        if shutil.which("nvcc"):
+            _build.build()
+        elif os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} was built from other sources than the ones present and nvcc is not "
+                              "on PATH to rebuild it")
     if not os.path.exists(_LIB_PATH):
         raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2112_02644_b200.build` "
                           "(there is no CPU fallback)")
@@ -81,6 +90,7 @@ def load_library():
     lib.smtm_lookup_exit_static.argtypes = [vp, i32, ctypes.POINTER(_Fmap), vp, vp, vp, vp, vp]
     lib.smtm_cache_update.argtypes = [vp, ctypes.POINTER(_Batch), vp, vp]
     lib.smtm_cache_resize.argtypes = [vp, vp]
+    lib.smtm_cache_warmup.argtypes = [vp, i32, ctypes.POINTER(_Fmap), vp, vp]
     lib.smtm_cache_update_resize.argtypes = [vp, ctypes.POINTER(_Batch), vp, vp]
     lib.smtm_step_host.argtypes = [vp, ctypes.POINTER(_Fmap), ctypes.POINTER(vp), vp, vp, i32, vp, vp, vp, vp]
     lib.smtm_cache_get_members.argtypes = [vp, vp, vp]
@@ -241,6 +251,12 @@ def smtm_cache_update(cache: Cache, batch: Batch, fallback_label=None, stream=No
 def smtm_cache_update_resize(cache: Cache, batch: Batch, fallback_label=None, stream=None) -> None:
     _check(load_library().smtm_cache_update_resize(cache.handle, ctypes.byref(batch.c), _dptr(fallback_label),
                                                    _stream(stream)), "smtm_cache_update_resize")
+
+
+def smtm_cache_warmup(cache: Cache, layer: int, fmap: Fmap, labels, stream=None) -> None:
+    """Folds labelled frames into the centres of their classes at one layer (centre warm-up)."""
+    _check(load_library().smtm_cache_warmup(cache.handle, layer, ctypes.byref(fmap.c), _dptr(labels),
+                                            _stream(stream)), "smtm_cache_warmup")
 
 
 def smtm_cache_resize(cache: Cache, stream=None) -> None:

@@ -9,6 +9,7 @@ using namespace smtm;
 
 struct smtm_cache {
     int n, L, S, k_init, k_min, k_max, W, cl_num, cl_den, max_batch;
+    bool forgetting;    // SMTM_FLAG_FORGET_FT
     int dims[SMTM_MAX_LAYERS];
     float tau[SMTM_MAX_LAYERS];
     float* d_centers[SMTM_MAX_LAYERS];
@@ -21,6 +22,7 @@ struct smtm_cache {
     unsigned long long* d_counters;
     int* d_status;
     float* d_partials;  // scratch of the fused lookup: partial dot products per (frame, part)
+    float* d_warm_sv;   // scratch of smtm_cache_warmup: [max_batch][C_max] semantic vectors (allocated on first use)
     void* d_dense;      // scratch of the tensor-core scorer (fast memories above 64 entries), else NULL
     void* d_cen_split[SMTM_MAX_LAYERS];   // bf16 heads and tails of the centres, per layer (same condition)
     bool cen_split_current[SMTM_MAX_LAYERS];  // false after creation and after every update
@@ -96,6 +98,7 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_status);
     cudaFree(c->d_partials);
     cudaFree(c->d_plan);
+    cudaFree(c->d_warm_sv);
     cudaFree(c->d_dense);
     cudaFree(c->d_tags);
     cudaFree(c->hb.d_sa);
@@ -203,6 +206,7 @@ ResizeArgs resize_args(const smtm_cache* c) {
     a.k_max = c->k_max;
     a.cl_num = c->cl_num;
     a.cl_den = c->cl_den;
+    a.forgetting = c->forgetting ? 1 : 0;
     a.ft = c->d_ft;
     a.ts = c->d_ts;
     a.members = c->d_members;
@@ -217,6 +221,8 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     a.S = c->S;
     a.n = c->n;
     a.L = c->L;
+    a.forget_W = c->forgetting ? c->W : 0;
+    a.warm_layer = -1;
     const size_t mb = size_t(c->max_batch);
     a.plan.final_label = c->d_plan;
     a.plan.stop_layer = c->d_plan + mb;
@@ -267,7 +273,8 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     if (!cfg || !h_centers || !out || !cfg->dims || !cfg->tau) return SMTM_ERR_INVALID_ARG;
     if (cfg->n_classes < 1 || cfg->n_classes > SMTM_MAX_CLASSES) return SMTM_ERR_INVALID_ARG;
     if (cfg->n_layers < 1 || cfg->n_layers > SMTM_MAX_LAYERS) return SMTM_ERR_INVALID_ARG;
-    if (cfg->n_streams < 1 || cfg->max_batch < 1 || cfg->flags != 0) return SMTM_ERR_INVALID_ARG;
+    if (cfg->n_streams < 1 || cfg->max_batch < 1 || (cfg->flags & ~uint32_t(SMTM_FLAG_FORGET_FT)) != 0)
+        return SMTM_ERR_INVALID_ARG;
     if (cfg->k_min < 1 || cfg->k_min > cfg->k_init || cfg->k_init > cfg->k_max || cfg->k_max > cfg->n_classes)
         return SMTM_ERR_INVALID_ARG;
     if (cfg->window_W < 1 || cfg->cl_den < 1 || cfg->cl_num < 0 || cfg->cl_num > cfg->cl_den ||
@@ -294,6 +301,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     c->cl_num = cfg->cl_num;
     c->cl_den = cfg->cl_den;
     c->max_batch = cfg->max_batch;
+    c->forgetting = (cfg->flags & SMTM_FLAG_FORGET_FT) != 0;
     for (int l = 0; l < c->L; ++l) {
         c->dims[l] = cfg->dims[l];
         c->tau[l] = cfg->tau[l];
@@ -425,6 +433,45 @@ smtm_status_t smtm_cache_update_resize(smtm_cache_t* c, const smtm_batch_t* b, c
     const smtm_status_t s = check_update(c, b);
     if (s != SMTM_OK) return s;
     return update_impl(c, b, d_fallback_label, true, static_cast<cudaStream_t>(stream));
+}
+
+smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_t* f, const int32_t* d_labels,
+                                void* stream) {
+    smtm_status_t s = check_fmap(c, layer, f);
+    if (s != SMTM_OK) return s;
+    if (!f->d_data || !d_labels) return SMTM_ERR_INVALID_ARG;
+    if (!aligned16(f->d_data)) return SMTM_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!c->d_warm_sv && dev_alloc(&c->d_warm_sv, size_t(c->max_batch) * c->d_max) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SMTM_ERR_ALLOC;
+    }
+    SMTM_CUDA(launch_encode(encode_args(c, f, nullptr, c->d_warm_sv), c->sm_count, st, &c->launches));
+    UpdateArgs a{};
+    a.B = f->B;
+    a.S = c->S;
+    a.n = c->n;
+    a.L = c->L;
+    a.warm_layer = layer;
+    const size_t mb = size_t(c->max_batch);
+    a.plan.final_label = c->d_plan;
+    a.plan.stop_layer = c->d_plan + mb;
+    a.plan.class_tag = c->d_tags;
+    a.plan.stream_tag = c->d_tags + c->n;
+    a.plan.epoch = ++c->epoch;
+    a.fallback = d_labels;
+    a.ft = c->d_ft;
+    a.ts = c->d_ts;
+    for (int l = 0; l < c->L; ++l) {
+        a.dims[l] = c->dims[l];
+        a.sv[l] = c->d_warm_sv;
+        a.centers[l] = c->d_centers[l];
+        a.cnorm[l] = c->d_cnorm[l];
+        a.m[l] = c->d_m[l];
+    }
+    c->cen_split_current[layer] = false;
+    SMTM_CUDA(launch_update(a, nullptr, st, &c->launches));
+    return SMTM_OK;
 }
 
 smtm_status_t smtm_cache_resize(smtm_cache_t* c, void* stream) {

@@ -105,6 +105,8 @@ struct UpdatePlan {
 
 struct UpdateArgs {
     int B, S, n, L;
+    int forget_W;              // 0, or W when the frequency table itself forgets (SMTM_FLAG_FORGET_FT)
+    int warm_layer;            // -1, or the one layer a warm-up batch folds into (no tables; done == nullptr)
     UpdatePlan plan;
     const int32_t* stream_id;  // [B] or nullptr
     const uint8_t* done;
@@ -123,6 +125,7 @@ struct UpdateArgs {
 
 struct ResizeArgs {
     int S, n, W, k_min, k_max, cl_num, cl_den;
+    int forgetting;    // the tables are the forgetting variant: the score is FT itself
     const int32_t* ft;
     const int32_t* ts;
     int32_t* members;  // [S][k_max]

@@ -23,6 +23,20 @@ namespace {
 
 constexpr int kFtMax = 1 << 20;  // frequency counts saturate here so that Eq. 6's sums fit 64 bits
 constexpr int kEMax = 12;        // floor(TS / W) is clamped here: 0.25^12 of a count is below one
+constexpr int kFtFrac = 10;      // fractional bits of FT when the table itself forgets (SMTM_FLAG_FORGET_FT)
+
+// One frame of a stream applied to one class's table entry (Sec. 6.1).  forget_W > 0 is the
+// variant of Sec. 7.1: FT is fixed point, an appearance adds one unit, and every W-th
+// consecutive unseen frame multiplies it by 0.25 (rounding down).
+__device__ __forceinline__ void table_step(int& ft, int& ts, bool appears, int forget_W) {
+    if (appears) {
+        ft = forget_W ? int(min((long long)ft + (1 << kFtFrac), (long long)kFtMax << kFtFrac)) : min(ft + 1, kFtMax);
+        ts = 0;
+    } else if (ts < INT32_MAX) {
+        ++ts;
+        if (forget_W && ts % forget_W == 0) ft >>= 2;
+    }
+}
 
 constexpr int kUpdThreads = 256;
 constexpr int kUpdWarps = kUpdThreads / kWarp;
@@ -43,8 +57,9 @@ __device__ __forceinline__ unsigned long long tag_of(unsigned long long epoch, i
 __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a) {
     const int b = blockIdx.x * kUpdThreads + threadIdx.x;
     if (b >= a.B) return;
-    const bool ex = a.done[b] != 0;
-    const int lab = ex ? a.pred[b] : (a.fallback ? a.fallback[b] : -1);
+    const bool ex = a.done && a.done[b] != 0;  // no carry at all: a warm-up batch of labelled frames
+    int lab = ex ? a.pred[b] : (a.fallback ? a.fallback[b] : -1);
+    if (lab >= a.n) lab = -1;  // a label outside the memory counts as no label
     a.plan.final_label[b] = lab;
     a.plan.stop_layer[b] = ex ? a.exit_layer[b] : a.L;
     const unsigned long long tag = tag_of(a.plan.epoch, b);
@@ -54,7 +69,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a)
 
 // ---- Eq. 5 / Eq. 6 ------------------------------------------------------------------------
 
-__device__ __forceinline__ unsigned long long score_of(int ft, int ts, int W) {
+__device__ __forceinline__ unsigned long long score_of(int ft, int ts, int W, int forgetting = 0) {
+    if (forgetting) return (unsigned long long)max(ft, 0);  // the decay already sits in the table
     int e = ts / W;
     if (e > kEMax) e = kEMax;
     const unsigned long long f = (unsigned long long)min(max(ft, 0), kFtMax);
@@ -81,7 +97,7 @@ __device__ void resize_stream(const ResizeArgs& a, int s, unsigned char* smem, i
     unsigned long long local = 0;
     for (int c0 = 0; c0 < a.n; c0 += kUpdThreads) {
         const int c = c0 + tid;
-        const unsigned long long sc = c < a.n ? score_of(ft[c], ts[c], a.W) : 0ull;
+        const unsigned long long sc = c < a.n ? score_of(ft[c], ts[c], a.W, a.forgetting) : 0ull;
         int cnt;
         const int pos = block_exclusive_scan(sc != 0 ? 1 : 0, s_scan, &cnt);
         if (sc != 0) {
@@ -118,7 +134,7 @@ __device__ void resize_stream(const ResizeArgs& a, int s, unsigned char* smem, i
         int filled = nz;
         for (int c0 = 0; c0 < a.n && filled < a.k_max; c0 += kUpdThreads) {
             const int c = c0 + tid;
-            const int z = (c < a.n && score_of(ft[c], ts[c], a.W) == 0) ? 1 : 0;
+            const int z = (c < a.n && score_of(ft[c], ts[c], a.W, a.forgetting) == 0) ? 1 : 0;
             int cnt;
             const int pos = block_exclusive_scan(z, s_scan, &cnt);
             if (z && filled + pos < a.k_max) {
@@ -195,12 +211,7 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
             const int l = __shfl_sync(kFull, lab, src);
 #pragma unroll
             for (int i = 0; i < NC; ++i) {
-                if (lane + i * kWarp == l) {
-                    ft[i] = min(ft[i] + 1, kFtMax);
-                    ts[i] = 0;
-                } else if (ts[i] < INT32_MAX) {
-                    ++ts[i];
-                }
+                table_step(ft[i], ts[i], lane + i * kWarp == l, a.forget_W);
             }
         }
     }
@@ -224,7 +235,7 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
 #pragma unroll
     for (int i = 0; i < NC; ++i) {
         const int c = lane + i * kWarp;
-        const unsigned long long sc = c < a.n ? score_of(ft[i], ts[i], rz.W) : 0ull;
+        const unsigned long long sc = c < a.n ? score_of(ft[i], ts[i], rz.W, rz.forgetting) : 0ull;
         const unsigned m = __ballot_sync(kFull, sc != 0);
         if (sc != 0) {
             const int pos = nz + __popc(m & lt);
@@ -256,7 +267,7 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
 #pragma unroll
     for (int i = 0; i < NC; ++i) {
         const int c = lane + i * kWarp;
-        const bool z = filled < rz.k_max && c < a.n && score_of(ft[i], ts[i], rz.W) == 0;
+        const bool z = filled < rz.k_max && c < a.n && score_of(ft[i], ts[i], rz.W, rz.forgetting) == 0;
         const unsigned m = __ballot_sync(kFull, z);
         if (z) {
             const int pos = filled + __popc(m & lt);
@@ -327,14 +338,7 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_apply(const UpdateArgs a
             if (cnt == 0) continue;
             for (int c = tid; c < a.n; c += kUpdThreads) {
                 int f = a.ft[(size_t)s * a.n + c], t = a.ts[(size_t)s * a.n + c];
-                for (int i = 0; i < cnt; ++i) {
-                    if (s_list[i] == c) {
-                        f = min(f + 1, kFtMax);
-                        t = 0;
-                    } else if (t < INT32_MAX) {
-                        ++t;
-                    }
-                }
+                for (int i = 0; i < cnt; ++i) table_step(f, t, s_list[i] == c, a.forget_W);
                 a.ft[(size_t)s * a.n + c] = f;
                 a.ts[(size_t)s * a.n + c] = t;
             }
@@ -348,7 +352,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_apply(const UpdateArgs a
 
     // ---- Eq. 7 for one (class, layer): fold the matching frames in ascending index --------
     const int job = blockIdx.x - table_ctas;
-    const int g = job / a.L, l0 = job - g * a.L;  // l0 is 0-based here; the paper's l0 is l0 + 1
+    const int nl = a.warm_layer >= 0 ? 1 : a.L;  // a warm-up touches one layer only
+    const int g = job / nl, l0 = a.warm_layer >= 0 ? a.warm_layer : job - g * nl;  // l0 is 0-based; the paper's is l0 + 1
     const int cls = a.plan.final_label[g];
     if (cls < 0 || a.plan.class_tag[cls] != tag_of(a.plan.epoch, g)) return;  // not the class's first frame
     const int D = a.dims[l0];
@@ -448,8 +453,8 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, cudaStream_
     k_update_plan<<<(a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st>>>(a);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const int table_ctas = warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
-    k_update_apply<<<table_ctas + a.B * a.L, kUpdThreads, smem, st>>>(a, rz ? *rz : ResizeArgs{}, table_ctas,
+    const int table_ctas = a.warm_layer >= 0 ? 0 : warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
+    k_update_apply<<<table_ctas + a.B * (a.warm_layer >= 0 ? 1 : a.L), kUpdThreads, smem, st>>>(a, rz ? *rz : ResizeArgs{}, table_ctas,
                                                                      rz ? 1 : 0, warp_tables ? 1 : 0);
     return cudaGetLastError();
 }

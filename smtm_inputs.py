@@ -49,6 +49,7 @@ class Workload:
     repeat_p: float = 0.0                   # per-stream probability of repeating the last label
     unit_centroids: bool = False            # centroids L2-normalised and used as centres (m = 1)
     warm_m: int = 32                        # update count attached to the initial centres
+    forgetting: bool = False                # frequency table itself decays (the paper's rapidly-changing-scene setting)
     seed: int = 0
 
     @property
@@ -80,7 +81,13 @@ C4 = Workload("c4_large_cache_bf16", BF16, NCHW, 1024, ((2048, 7, 7),), n=1000, 
               k_min=1000, k_max=1000, sigma=1.0, zipf_s=1.0)
 C5 = Workload("c5_streaming_bf16", BF16, NCHW, 512, (RESNET50[2], RESNET50[3]), n=500, k_init=8,
               k_min=8, k_max=64, S=512, T=64, sigma=0.5, zipf_s=1.1, repeat_p=0.85)
-WORKLOADS = {w.name: w for w in (C1, C2, C3, C4, C5)}
+# VGG16 on 32x32 inputs (the paper's long-tail CIFAR-100 setting): 13 shallow exits with tiny
+# maps, 100 classes, rapidly changing scenes, frequency table with forgetting.
+VGG16_CIFAR = ((64, 32, 32), (64, 32, 32), (128, 16, 16), (128, 16, 16), (256, 8, 8), (256, 8, 8), (256, 8, 8),
+               (512, 4, 4), (512, 4, 4), (512, 4, 4), (512, 2, 2), (512, 2, 2), (512, 2, 2))
+C6 = Workload("c6_vgg16_cifar_fp16", F16, NCHW, 128, VGG16_CIFAR, n=100, k_init=5, k_min=5, k_max=20, S=128, T=8,
+              window_W=4, sigma=0.5, zipf_s=1.0, repeat_p=0.2, forgetting=True)
+WORKLOADS = {w.name: w for w in (C1, C2, C3, C4, C5, C6)}
 
 
 def _rng(w: Workload, *salt: int) -> np.random.Generator:

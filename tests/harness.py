@@ -37,9 +37,11 @@ class Report:
 def make_pair(w: si.Workload, max_batch=None):
     cents, counts = si.initial_centers(w)
     tau = [w.tau] * w.L
-    mem = oracle.OracleMemory(w.n, w.dims, tau, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W)
+    mem = oracle.OracleMemory(w.n, w.dims, tau, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W,
+                              forgetting=w.forgetting)
     cache = smtm.smtm_cache_create(w.n, w.dims, tau, cents, counts, n_streams=w.S, k_init=w.k_init, k_min=w.k_min,
-                                   k_max=w.k_max, window_W=w.window_W, max_batch=max_batch or w.B)
+                                   k_max=w.k_max, window_W=w.window_W, max_batch=max_batch or w.B,
+                                   flags=smtm.FLAG_FORGET_FT if w.forgetting else 0)
     return cache, mem
 
 

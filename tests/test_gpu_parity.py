@@ -184,6 +184,62 @@ def test_large_fast_memory_over_several_layers_uses_tensor_cores():
     assert rep3.frames == 66
 
 
+def test_forgetting_frequency_table_rapid_scene_change():
+    # the paper's long-tail / rapid-change setting: FT itself decays every W unseen frames
+    w = si.Workload("forget", si.BF16, si.NCHW, B=24, stages=((64, 7, 7), (128, 7, 7)), n=30, k_init=4, k_min=2,
+                    k_max=12, S=24, T=30, tau=0.4, window_W=3, sigma=0.5, zipf_s=0.8, repeat_p=0.3, forgetting=True,
+                    seed=12)
+    rep = run_workload(w)
+    assert rep.frames == 24 * 30
+    w1 = w.scaled(name="forget_one_stream", S=1, B=50, T=8, window_W=5)   # many frames of one stream per step
+    rep1 = run_workload(w1)
+    assert rep1.frames == 400
+
+
+def test_centre_warm_up_on_the_gpu_matches_oracle_and_feeds_lookups():
+    # Sec. 5: centres = per-class mean semantic vector of labelled frames, built on the GPU from count 0,
+    # in two batches, then used by a normal step
+    w = si.Workload("warm", si.BF16, si.NCHW, B=96, stages=((256, 14, 14), (512, 7, 7)), n=12, k_init=12, k_min=12,
+                    k_max=12, S=1, T=3, tau=0.5, sigma=0.5, zipf_s=0.5, seed=14)
+    zeros = [np.zeros((w.n, d), np.float32) for d in w.dims]
+    m0 = [np.zeros(w.n, np.uint32) for _ in w.dims]
+    tau = [w.tau] * w.L
+    cache = smtm.smtm_cache_create(w.n, w.dims, tau, zeros, m0, k_init=w.k_init, k_min=w.k_min, k_max=w.k_max,
+                                   max_batch=w.B)
+    mem = oracle.OracleMemory(w.n, w.dims, tau, zeros, m0, 1, w.k_init, w.k_min, w.k_max, w.window_W)
+    labs = si.labels(w)
+    for t in range(2):
+        lab = labs[t].copy()
+        lab[::7] = -1                      # unlabelled frames
+        lab[3::11] = w.n + 2               # labels outside the memory
+        for l in range(w.L):
+            x = si.frames(w, l, labs[t], 100 + t, device="cuda")
+            smtm.smtm_cache_warmup(cache, l, smtm.Fmap(x, w.dtype, w.layout, *si.shape4(w, l)),
+                                   torch.from_numpy(lab).cuda())
+            mem.warmup(l, x.cpu(), w.dtype, w.layout, si.shape4(w, l), lab)
+    for l in range(w.L):
+        cen, m = smtm.smtm_cache_get_centers(cache, l)
+        assert np.array_equal(m, mem.m[l]) and m.sum() > 100
+        np.testing.assert_allclose(cen, mem.centers[l], rtol=2e-5, atol=1e-6)
+    ft, ts = smtm.smtm_cache_get_tables(cache)
+    assert not ft.any() and not ts.any()
+    # a normal step on the warmed-up memory: most frames find their class
+    from harness import Report, step_pair, compare_state
+    gb = smtm.Batch(cache, w.B)
+    rep = Report()
+    step_pair(w, cache, mem, gb, labs[2], 2, rep)
+    compare_state(w, cache, mem, rep)
+    assert int(gb.done.sum()) > w.B // 2
+    smtm.smtm_cache_destroy(cache)
+
+
+def test_c6_vgg16_shaped_thirteen_shallow_exits():
+    # many layers, tiny maps (down to 2x2, which no 16-byte grouping serves), forgetting tables
+    rep = run_workload(si.C6, steps=4)
+    assert rep.frames == 128 * 4 and len(rep.exits) == 13
+    print("c6 exits per layer:", rep.exits)
+
+
 def test_step_host_matches_device_path():
     w = si.C5.scaled(B=32, S=32, T=3)
     cents, counts = si.initial_centers(w)

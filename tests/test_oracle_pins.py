@@ -392,3 +392,38 @@ def test_centre_update_closed_form_and_fixed_point():
     c = np.array([[2.0, 4.0]]); m = np.array([1], np.uint32)
     oracle.centers_update(1, np.array([[4.0, 0.0]]), np.zeros(1, np.int32), np.ones(1, np.int32), c, m)
     assert np.array_equal(c, [[3.0, 2.0]]) and m[0] == 2
+
+
+# --------------------------------------------------------------------------- forgetting variant (Sec. 6.1 / 7.1)
+
+def test_forgetting_tables_equal_eq5_score_until_a_class_reappears_and_forget_afterwards():
+    W, n = 4, 3
+    unit = 1 << oracle.FT_FRAC
+    # class 0 seen five times, then class 1 for 9 frames: class 0 has TS = 9 -> two windows elapsed
+    seq = np.array([0] * 5 + [1] * 9, np.int32)
+    sid = np.zeros(len(seq), np.int32)
+    ft = np.zeros((1, n), np.int32); ts = np.zeros((1, n), np.int32)
+    oracle.tables_update(sid, seq, ft, ts, forgetting_W=W)
+    plain_ft = np.zeros((1, n), np.int32); plain_ts = np.zeros((1, n), np.int32)
+    oracle.tables_update(sid, seq, plain_ft, plain_ts)
+    assert np.array_equal(ts, plain_ts)
+    for i in range(n):   # FT of the forgetting table = Eq. 5's score of the plain tables (exact here: no rounding)
+        want = Fraction(int(plain_ft[0, i])) * Fraction(1, 4) ** (int(plain_ts[0, i]) // W)
+        assert Fraction(int(ft[0, i]), unit) == want
+    assert ft[0, 0] == 5 * unit // 16 and ft[0, 1] == 9 * unit and ft[0, 2] == 0
+    # class 0 reappears once: the plain count is 6, the forgetting table only remembers 5/16 + 1
+    more = np.array([0], np.int32)
+    oracle.tables_update(np.zeros(1, np.int32), more, ft, ts, forgetting_W=W)
+    oracle.tables_update(np.zeros(1, np.int32), more, plain_ft, plain_ts)
+    assert plain_ft[0, 0] == 6 and ft[0, 0] == 5 * unit // 16 + unit and ts[0, 0] == 0
+    # ranking with forgetting uses FT as the score: class 1 (9) > class 0 (21/16) > class 2
+    members = np.zeros((1, 3), np.int32); k = np.zeros(1, np.int32)
+    oracle.resize(ft, ts, W, 1, 3, 19, 20, members, k, forgetting=True)
+    assert list(members[0]) == [1, 0, 2] and k[0] == 2   # 9 / (9 + 21/16) = 0.873 < 0.95 -> two entries
+    # decay rounds down in fixed point: one appearance survives five windows (1024 >> 10 = 1), not six
+    ft = np.zeros((1, 2), np.int32); ts = np.zeros((1, 2), np.int32)
+    seq = np.array([0] + [1] * (5 * W), np.int32)
+    oracle.tables_update(np.zeros(len(seq), np.int32), seq, ft, ts, forgetting_W=W)
+    assert ft[0, 0] == 1
+    oracle.tables_update(np.zeros(W, np.int32), np.ones(W, np.int32), ft, ts, forgetting_W=W)
+    assert ft[0, 0] == 0

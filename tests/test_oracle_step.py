@@ -176,3 +176,24 @@ def test_workload_recipes_have_the_stated_statistics():
     assert x.shape == (8, 64, 56, 56) and x.dtype == torch.float32 and x.min() < 0
     c1 = si.initial_centers(si.C1)[0][0]
     np.testing.assert_allclose(np.linalg.norm(c1, axis=1), 1.0, rtol=1e-6)
+
+
+def test_centre_warm_up_from_zero_is_the_class_mean():
+    # Sec. 5: centres start as the average semantic vector per class over labelled frames.
+    n, C, H, W, B = 5, 12, 3, 4, 40
+    rng = np.random.default_rng(21)
+    x = torch.from_numpy(rng.standard_normal((B, C, H, W)).astype(np.float32))
+    lab = rng.integers(-1, n + 2, B).astype(np.int32)          # -1 and labels >= n are skipped
+    mem = oracle.OracleMemory(n, [C], [0.8], [np.zeros((n, C), np.float32)], [np.zeros(n, np.uint32)], k_init=2,
+                              k_min=2, k_max=3)
+    mem.warmup(0, x[:25], oracle.F32, oracle.NCHW, (25, C, H, W), lab[:25])
+    mem.warmup(0, x[25:], oracle.F32, oracle.NCHW, (15, C, H, W), lab[25:])   # in two batches: same mean
+    sv = x.double().numpy().mean(axis=(2, 3))
+    for j in range(n):
+        rows = sv[lab == j]
+        assert mem.m[0][j] == len(rows)
+        if len(rows):
+            np.testing.assert_allclose(mem.centers[0][j], rows.mean(axis=0), rtol=1e-12, atol=1e-14)
+        else:
+            assert not mem.centers[0][j].any()
+    assert not mem.ft.any() and not mem.ts.any()               # tables untouched
