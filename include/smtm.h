@@ -149,6 +149,15 @@ smtm_status_t smtm_encode(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t*
 smtm_status_t smtm_lookup_exit(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t* fmap,
                                const smtm_batch_t* batch, void* stream);
 
+/* Sec. 5: the first lookup of a batch, where every frame starts with SA = 0 and
+ * nothing has exited.  Same result as smtm_batch_reset followed by
+ * smtm_lookup_exit, without the pass over the carry: whatever d_sa, d_done,
+ * d_exit_layer and d_pred held is ignored and overwritten for all B frames (all
+ * k_max slots of d_sa).  `layer` is normally 0 but may be any layer at which the
+ * caller starts looking up.  Same arguments and errors as smtm_lookup_exit. */
+smtm_status_t smtm_lookup_exit_begin(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t* fmap,
+                                     const smtm_batch_t* batch, void* stream);
+
 /* (No counterpart in the paper: a packaging of smtm_lookup_exit for callers that
  * must not allocate.)  Some callers cannot call cudaMalloc or anything that may:
  * a plug-in running inside another engine's enqueue step that is handed only its

@@ -87,6 +87,7 @@ def load_library():
     lib.smtm_batch_reset.argtypes = [vp, ctypes.POINTER(_Batch), vp]
     lib.smtm_encode.argtypes = [vp, i32, ctypes.POINTER(_Fmap), vp, vp, vp, vp]
     lib.smtm_lookup_exit.argtypes = [vp, i32, ctypes.POINTER(_Fmap), ctypes.POINTER(_Batch), vp]
+    lib.smtm_lookup_exit_begin.argtypes = [vp, i32, ctypes.POINTER(_Fmap), ctypes.POINTER(_Batch), vp]
     lib.smtm_lookup_exit_static.argtypes = [vp, i32, ctypes.POINTER(_Fmap), vp, vp, vp, vp, vp]
     lib.smtm_cache_update.argtypes = [vp, ctypes.POINTER(_Batch), vp, vp]
     lib.smtm_cache_resize.argtypes = [vp, vp]
@@ -233,6 +234,11 @@ def smtm_encode(cache: Cache, layer: int, fmap: Fmap, sv, skip=None, sv_norm2=No
 def smtm_lookup_exit(cache: Cache, layer: int, fmap: Fmap, batch: Batch, stream=None) -> None:
     _check(load_library().smtm_lookup_exit(cache.handle, layer, ctypes.byref(fmap.c), ctypes.byref(batch.c),
                                            _stream(stream)), "smtm_lookup_exit")
+
+
+def smtm_lookup_exit_begin(cache: Cache, layer: int, fmap: Fmap, batch: Batch, stream=None) -> None:
+    _check(load_library().smtm_lookup_exit_begin(cache.handle, layer, ctypes.byref(fmap.c), ctypes.byref(batch.c),
+                                                 _stream(stream)), "smtm_lookup_exit_begin")
 
 
 def smtm_lookup_exit_static(cache: Cache, layer: int, fmap: Fmap, stream_id, exit_flags, pred, ac=None,

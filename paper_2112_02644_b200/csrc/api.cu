@@ -144,8 +144,9 @@ EncodeArgs encode_args(const smtm_cache* c, const smtm_fmap_t* f, const uint8_t*
 }
 
 smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b,
-                          cudaStream_t st) {
+                          cudaStream_t st, bool begin) {
     LookupArgs a{};
+    a.fresh = begin ? 1 : 0;
     a.layer = layer;
     a.L = c->L;
     a.B = f->B;
@@ -177,6 +178,10 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     }
     SMTM_CUDA(launch_lookup_fused(e, a, c->d_partials, c->sm_count, st, &c->launches, &fused, timing));
     if (fused) return SMTM_OK;
+    if (begin) {  // the other routes read the carry: put it into its reset state with a kernel of its own
+        SMTM_CUDA(launch_batch_reset(b->d_sa, b->d_done, b->d_exit_layer, b->d_pred, b->B, c->k_max, st, &c->launches));
+        a.fresh = 0;
+    }
     const bool dense = c->d_dense && dense_scoring_supported(a.D, a.n);  // large fast memory: tensor cores
     EncodeArgs e2 = e;
     if (dense) dense_sv_split(c->d_dense, c->max_batch, c->d_max, &e2.sv_hi, &e2.sv_lo);
@@ -418,7 +423,18 @@ smtm_status_t smtm_lookup_exit(smtm_cache_t* c, int32_t layer, const smtm_fmap_t
     if (b->B != f->B) return SMTM_ERR_SHAPE;
     if (!f->d_data || !b->d_sv[layer]) return SMTM_ERR_INVALID_ARG;
     if (!aligned16(f->d_data) || !aligned16(b->d_sv[layer])) return SMTM_ERR_ALIGN;
-    return lookup_impl(c, layer, f, b, static_cast<cudaStream_t>(stream));
+    return lookup_impl(c, layer, f, b, static_cast<cudaStream_t>(stream), false);
+}
+
+smtm_status_t smtm_lookup_exit_begin(smtm_cache_t* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b,
+                                     void* stream) {
+    smtm_status_t s = check_fmap(c, layer, f);
+    if (s != SMTM_OK) return s;
+    if ((s = check_batch(c, b)) != SMTM_OK) return s;
+    if (b->B != f->B) return SMTM_ERR_SHAPE;
+    if (!f->d_data || !b->d_sv[layer]) return SMTM_ERR_INVALID_ARG;
+    if (!aligned16(f->d_data) || !aligned16(b->d_sv[layer])) return SMTM_ERR_ALIGN;
+    return lookup_impl(c, layer, f, b, static_cast<cudaStream_t>(stream), true);
 }
 
 smtm_status_t smtm_cache_update(smtm_cache_t* c, const smtm_batch_t* b, const int32_t* d_fallback_label,
@@ -526,7 +542,6 @@ smtm_status_t smtm_step_host(smtm_cache_t* c, const smtm_fmap_t* fmaps, const vo
     b.d_ac = nullptr;
     b.d_sep = nullptr;
     b.d_top = nullptr;
-    SMTM_CUDA(launch_batch_reset(b.d_sa, b.d_done, b.d_exit_layer, b.d_pred, B, c->k_max, st, &c->launches));
     if (h_stream_id) {
         SMTM_CUDA(cudaMemcpyAsync(c->d_stream_id, h_stream_id, size_t(B) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
         b.d_stream_id = c->d_stream_id;
@@ -538,7 +553,7 @@ smtm_status_t smtm_step_host(smtm_cache_t* c, const smtm_fmap_t* fmaps, const vo
         const size_t bytes = size_t(B) * f.C * f.H * f.W * (f.dtype == SMTM_F32 ? 4 : 2);
         SMTM_CUDA(cudaMemcpyAsync(c->d_stage[l], h_maps[l], bytes, cudaMemcpyHostToDevice, st));
         f.d_data = c->d_stage[l];
-        smtm_status_t s = lookup_impl(c, l, &f, &b, st);
+        smtm_status_t s = lookup_impl(c, l, &f, &b, st, l == 0);
         if (s != SMTM_OK) return s;
     }
     smtm_status_t s = update_impl(c, &b, h_fallback_label ? c->d_fallback : nullptr, do_resize != 0, st);

@@ -295,8 +295,12 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
     }
 
     // ---- the active frames and this CTA's share of their units -----------------------------
-    int n_active = 0;
-    for (int t0 = 0; t0 < a.B; t0 += kThreadsFused) {
+    int n_active = a.fresh ? a.B : 0;  // a batch that starts here has every frame active: no flags to read
+    for (int idx = threadIdx.x; a.fresh && idx < kMaxUnits; idx += kThreadsFused) {
+        const long long u = (long long)blockIdx.x + (long long)idx * gridDim.x;
+        if (u < (long long)a.B * P) my_units[idx] = int(u / P) * kMaxParts + int(u % P);
+    }
+    for (int t0 = 0; !a.fresh && t0 < a.B; t0 += kThreadsFused) {
         const int b = t0 + threadIdx.x;
         const int act = (b < a.B && !a.done[b]) ? 1 : 0;
         int cnt;

@@ -43,6 +43,7 @@ cudaError_t launch_row_norm2(const float* sv, const uint8_t* skip, int B, int D,
 // ---- lookup (Sec. 4.2, Sec. 5) -------------------------------------------------------------
 struct LookupArgs {
     int layer, L, B, D, n, k_max;
+    int fresh;                // the batch starts here: the carry is taken as SA = 0, nobody done, and is overwritten
     float tau;
     const float* sv;          // [B][D]
     const float* centers;     // [n][D]

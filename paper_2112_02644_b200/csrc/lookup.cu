@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(kThreads) k_finish_partials(const LookupArgs a
                                                               int P) {
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * (kThreads / kWarp) + (threadIdx.x >> 5);
-    if (b >= a.B || a.done[b]) return;
+    if (b >= a.B || (!a.fresh && a.done[b])) return;
     const int sid = a.stream_id ? a.stream_id[b] : 0;
     const int k = min(a.k[sid], kFusedMaxK);
     const int32_t* mem = a.members + (size_t)sid * a.k_max;
@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(kThreads) k_finish_partials(const LookupArgs a
         const int j = lane + h * kWarp;
         ids[h] = j < k ? mem[j] : 0;
         clen[h] = j < k ? a.cnorm[ids[h]] : 0.f;
-        sa_old[h] = j < k ? a.sa[(size_t)b * a.k_max + j] : 0.f;
+        sa_old[h] = (j < k && !a.fresh) ? a.sa[(size_t)b * a.k_max + j] : 0.f;
     }
     float pn[kMaxParts], p0[kMaxParts], p1[kMaxParts];
 #pragma unroll
@@ -186,6 +186,8 @@ __global__ void __launch_bounds__(kThreads) k_finish_partials(const LookupArgs a
             s_cur[h] = cosine_from(dots[h], nn, clen[h]);        // Eq. 1
             s_acc[h] = __fmaf_rn(s_cur[h], weight, sa_old[h]);   // Eq. 3
             a.sa[(size_t)b * a.k_max + j] = s_acc[h];
+        } else if (a.fresh && j < a.k_max) {
+            a.sa[(size_t)b * a.k_max + j] = 0.f;                 // unused slots start from zero too
         }
     }
     const Top2 ta = warp_top2_regs(s_acc, ids, k, lane);

@@ -116,6 +116,10 @@ __device__ __forceinline__ void decide_from_top2(const LookupArgs& a, int b, con
         a.exit_layer[b] = a.layer + 1;
         a.pred[b] = ta.id1;
         atomicAdd(&a.counters[SMTM_CTR_EXITS + a.layer], 1ull);
+    } else if (a.fresh) {  // the reset state of a frame that stays in
+        a.done[b] = 0;
+        a.exit_layer[b] = 0;
+        a.pred[b] = -1;
     }
 }
 

@@ -75,8 +75,6 @@ extern "C" smtm_status_t smtm_lookup_exit_static(smtm_cache_t* cache, int32_t la
     b.d_pred = d_pred;
     b.d_ac = d_ac;
     b.d_sv[layer] = reinterpret_cast<float*>(base);
-    // the array keeps whatever the previous call left: clear what the lookup accumulates into
-    smtm_status_t s = smtm_batch_reset(cache, &b, stream);
-    if (s != SMTM_OK) return s;
-    return smtm_lookup_exit(cache, layer, fmap, &b, stream);
+    // the array keeps whatever the previous call left: the lookup starts the carry afresh
+    return smtm_lookup_exit_begin(cache, layer, fmap, &b, stream);
 }
