@@ -18,6 +18,17 @@ __device__ __forceinline__ void set_status(int* status, int code) {
     if (status) atomicCAS(status, 0, code);
 }
 
+// ---- chained launches -----------------------------------------------------------------
+//
+// Every kernel of the library is launched with programmatic stream serialisation: its CTAs may
+// become resident, and run their prologue, while the kernel before it in the stream is still
+// finishing.  chain_release() lets the next kernel's CTAs in as soon as all of this kernel's
+// have started; chain_wait() returns once the previous kernel has completed and its writes
+// are visible.  Nothing that reads or writes global memory comes before chain_wait().
+
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- shared-memory barriers and bulk asynchronous copies -------------------------------
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

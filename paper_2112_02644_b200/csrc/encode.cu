@@ -177,7 +177,9 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
         }
         mbar_init_fence();
     }
+    chain_release();
     __syncthreads();
+    chain_wait();  // the barriers are set up while the previous kernel finishes
 
     const bool producer = warp == kConsumers;  // last warp; lane 0 issues the copies
     int it = 0;                                // chunks of this CTA that are not skipped, so far
@@ -293,6 +295,7 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         }
         mbar_init_fence();
     }
+    chain_release();
 
     // ---- the active frames and this CTA's share of their units -----------------------------
     int n_active = a.fresh ? a.B : 0;  // a batch that starts here has every frame active: no flags to read
@@ -300,6 +303,7 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         const long long u = (long long)blockIdx.x + (long long)idx * gridDim.x;
         if (u < (long long)a.B * P) my_units[idx] = int(u / P) * kMaxParts + int(u % P);
     }
+    chain_wait();  // everything above touched shared memory only and overlaps the previous kernel's tail
     for (int t0 = 0; !a.fresh && t0 < a.B; t0 += kThreadsFused) {
         const int b = t0 + threadIdx.x;
         const int act = (b < a.B && !a.done[b]) ? 1 : 0;
@@ -457,6 +461,8 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_encode_nhwc(const uint8_t* __r
                                                               float* __restrict__ sv, int B, int C, int HW,
                                                               float inv_hw) {
     extern __shared__ float part[];  // [phases][min(C, 256 * kPerVec)]
+    chain_release();
+    chain_wait();
     constexpr int V = E::kPerVec;
     const int CG = C / V;            // 16-byte vectors per pixel
     for (int b = blockIdx.x; b < B; b += gridDim.x) {
@@ -511,6 +517,8 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_encode_nhwc(const uint8_t* __r
 template <class E>
 __global__ void k_encode_generic(const void* __restrict__ x, const uint8_t* __restrict__ skip,
                                  float* __restrict__ sv, int B, int C, int HW, int nhwc, float inv_hw) {
+    chain_release();
+    chain_wait();
     const long long total = (long long)B * C;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -529,6 +537,8 @@ __global__ void k_encode_generic(const void* __restrict__ x, const uint8_t* __re
 __global__ void k_row_norm2(const float* __restrict__ sv, const uint8_t* __restrict__ skip, int B, int D,
                             float* __restrict__ out) {
     __shared__ float scratch[32];
+    chain_release();
+    chain_wait();
     const int b = blockIdx.x;
     if (skip && skip[b]) return;
     float s = 0.f;
@@ -542,8 +552,7 @@ __global__ void k_row_norm2(const float* __restrict__ sv, const uint8_t* __restr
 
 template <class R>
 cudaError_t launch_nchw(const NchwParams& p, int grid, cudaStream_t st) {
-    k_encode_nchw<R><<<grid, kThreadsTma, kSmemTma, st>>>(p);
-    return cudaGetLastError();
+    return launch_chained(k_encode_nchw<R>, grid, kThreadsTma, kSmemTma, st, p);
 }
 
 template <class R>
@@ -555,9 +564,8 @@ template <class E>
 cudaError_t launch_generic(const EncodeArgs& a, cudaStream_t st) {
     const long long total = (long long)a.B * a.C;
     const int grid = int(std::min<long long>((total + 255) / 256, 148 * 16));
-    k_encode_generic<E><<<grid, 256, 0, st>>>(a.x, a.skip, a.sv, a.B, a.C, a.H * a.W, a.layout == SMTM_NHWC,
-                                               1.0f / float(a.H * a.W));
-    return cudaGetLastError();
+    return launch_chained(k_encode_generic<E>, grid, 256, 0, st, a.x, a.skip, a.sv, a.B, a.C, a.H * a.W,
+                          int(a.layout == SMTM_NHWC), 1.0f / float(a.H * a.W));
 }
 
 template <class E>
@@ -565,9 +573,8 @@ cudaError_t launch_nhwc(const EncodeArgs& a, cudaStream_t st) {
     const int CG = a.C / E::kPerVec;
     const int cgs = std::min(CG, kThreadsNhwc);
     const size_t smem = size_t(kThreadsNhwc / cgs) * cgs * E::kPerVec * sizeof(float);
-    k_encode_nhwc<E><<<a.B, kThreadsNhwc, smem, st>>>(static_cast<const uint8_t*>(a.x), a.skip, a.sv, a.B, a.C,
-                                                      a.H * a.W, 1.0f / float(a.H * a.W));
-    return cudaGetLastError();
+    return launch_chained(k_encode_nhwc<E>, a.B, kThreadsNhwc, smem, st, static_cast<const uint8_t*>(a.x), a.skip, a.sv,
+                          a.B, a.C, a.H * a.W, 1.0f / float(a.H * a.W));
 }
 
 int pow2_floor(int v) {
@@ -730,10 +737,9 @@ cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float*
     const size_t smem = fused_smem(f.slice_cap);
     cudaError_t err = cudaSuccess;
     if (timing) record_timing(timing[0], st);
-#define SMTM_LAUNCH(...) k_lookup_nchw<__VA_ARGS__><<<sm_count, kThreadsFused, smem, st>>>(f)
+#define SMTM_LAUNCH(...) err = launch_chained(k_lookup_nchw<__VA_ARGS__>, sm_count, kThreadsFused, smem, st, f)
     SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
 #undef SMTM_LAUNCH
-    err = cudaGetLastError();
     if (timing) record_timing(timing[1], st);
     ++*launches;
     *handled = true;
@@ -745,8 +751,7 @@ cudaError_t launch_row_norm2(const float* sv, const uint8_t* skip, int B, int D,
                              int64_t* launches) {
     if (B <= 0) return cudaSuccess;
     ++*launches;
-    k_row_norm2<<<B, 256, 0, st>>>(sv, skip, B, D, out);
-    return cudaGetLastError();
+    return launch_chained(k_row_norm2, B, 256, 0, st, sv, skip, B, D, out);
 }
 
 }  // namespace smtm

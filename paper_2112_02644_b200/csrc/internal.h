@@ -17,6 +17,25 @@ inline cudaError_t record_timing(cudaEvent_t ev, cudaStream_t st) {
                                                                                 : cudaEventRecordDefault);
 }
 
+// Launches `kernel` so that it may start while the previous kernel of the stream is finishing
+// (programmatic stream serialisation); the kernel itself waits with chain_wait() before it
+// touches global memory.
+template <class... Params, class... Args>
+cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                           Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 // Number of exit layers and the fast-memory capacity of a cache.
 void cache_shape(const smtm_cache_t* cache, int* n_layers, int* k_max);
 

@@ -25,6 +25,8 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
     float* s_acc = s_cur + a.k_max;   // [k_max] cumulative similarities
     __shared__ float scratch[32];
 
+    chain_release();
+    chain_wait();
     const int b = blockIdx.x;
     if (a.done[b]) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -78,6 +80,8 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
 __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, const float* __restrict__ dots) {
     __shared__ float scratch[32];
     __shared__ Top2 s_top[2][kThreads / kWarp];
+    chain_release();
+    chain_wait();
     const int b = blockIdx.x;
     if (a.done[b]) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -145,6 +149,8 @@ __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, c
 // l + 32; the parts of each sum are added in part order.
 __global__ void __launch_bounds__(kThreads) k_finish_partials(const LookupArgs a, const float* __restrict__ partials,
                                                               int P) {
+    chain_release();
+    chain_wait();
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * (kThreads / kWarp) + (threadIdx.x >> 5);
     if (b >= a.B || (!a.fresh && a.done[b])) return;
@@ -197,6 +203,8 @@ __global__ void __launch_bounds__(kThreads) k_finish_partials(const LookupArgs a
 
 __global__ void k_batch_reset(float* __restrict__ sa, uint8_t* __restrict__ done, int32_t* __restrict__ exit_layer,
                               int32_t* __restrict__ pred, int B, long long n_sa) {
+    chain_release();
+    chain_wait();
     const long long i0 = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     const long long step = (long long)gridDim.x * blockDim.x;
     for (long long i = i0; i < n_sa; i += step) sa[i] = 0.f;
@@ -215,8 +223,7 @@ cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, in
     const long long n_sa = (long long)B * k_max;
     const int grid = int(std::min<long long>((n_sa + 255) / 256, 1184));
     ++*launches;
-    k_batch_reset<<<grid, 256, 0, st>>>(sa, done, exit_layer, pred, B, n_sa);
-    return cudaGetLastError();
+    return launch_chained(k_batch_reset, grid, 256, 0, st, sa, done, exit_layer, pred, B, n_sa);
 }
 
 cudaError_t launch_finish_partials(const LookupArgs& a, const float* partials, int parts, cudaStream_t st,
@@ -224,15 +231,13 @@ cudaError_t launch_finish_partials(const LookupArgs& a, const float* partials, i
     if (a.B <= 0) return cudaSuccess;
     ++*launches;
     const int per_cta = kThreads / kWarp;
-    k_finish_partials<<<(a.B + per_cta - 1) / per_cta, kThreads, 0, st>>>(a, partials, parts);
-    return cudaGetLastError();
+    return launch_chained(k_finish_partials, (a.B + per_cta - 1) / per_cta, kThreads, 0, st, a, partials, parts);
 }
 
 cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, cudaStream_t st, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
     ++*launches;
-    k_finish_dense<<<a.B, kThreads, 0, st>>>(a, dots);
-    return cudaGetLastError();
+    return launch_chained(k_finish_dense, a.B, kThreads, 0, st, a, dots);
 }
 
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches) {
@@ -245,8 +250,7 @@ cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* lau
         opted = smem;
     }
     ++*launches;
-    k_score_exit<<<a.B, kThreads, smem, st>>>(a);
-    return cudaGetLastError();
+    return launch_chained(k_score_exit, a.B, kThreads, smem, st, a);
 }
 
 }  // namespace smtm

@@ -55,6 +55,8 @@ __device__ __forceinline__ unsigned long long tag_of(unsigned long long epoch, i
 // Label and stop layer of a finished frame: the prediction and exit layer if it exited,
 // else the fallback label (the full network's answer, -1 = none) and L.
 __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a) {
+    chain_release();
+    chain_wait();
     const int b = blockIdx.x * kUpdThreads + threadIdx.x;
     if (b >= a.B) return;
     const bool ex = a.done && a.done[b] != 0;  // no carry at all: a warm-up batch of labelled frames
@@ -164,6 +166,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_resize(const ResizeArgs a) {
     extern __shared__ unsigned long long s_dyn[];
     __shared__ int s_scan[33];
     __shared__ unsigned long long s_part[kUpdThreads / 32];
+    chain_release();
+    chain_wait();
     resize_stream(a, blockIdx.x, reinterpret_cast<unsigned char*>(s_dyn), s_scan, s_part);
 }
 
@@ -316,6 +320,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_apply(const UpdateArgs a
     __shared__ float s_red[32];
     __shared__ unsigned long long s_part[kUpdWarps];
     const int tid = threadIdx.x;
+    chain_release();
+    chain_wait();
 
     if (int(blockIdx.x) < table_ctas) {
         if (warp_tables) {
@@ -413,6 +419,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_apply(const UpdateArgs a
 
 __global__ void k_center_norms(const float* __restrict__ centers, int n, int D, float* __restrict__ cnorm) {
     __shared__ float s_red[32];
+    chain_release();
+    chain_wait();
     const int c = blockIdx.x;
     float nrm = 0.f;
     for (int d = threadIdx.x; d < D; d += blockDim.x) {
@@ -435,8 +443,7 @@ cudaError_t opt_in_smem(const void* fn, size_t smem, size_t* opted) {
 cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm, cudaStream_t st,
                                 int64_t* launches) {
     ++*launches;
-    k_center_norms<<<n, 256, 0, st>>>(centers, n, D, cnorm);
-    return cudaGetLastError();
+    return launch_chained(k_center_norms, n, 256, 0, st, centers, n, D, cnorm);
 }
 
 cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, cudaStream_t st, int64_t* launches) {
@@ -450,13 +457,11 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, cudaStream_
     cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_apply), smem, &opted);
     if (e != cudaSuccess) return e;
     *launches += 2;
-    k_update_plan<<<(a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st>>>(a);
-    e = cudaGetLastError();
+    e = launch_chained(k_update_plan, (a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st, a);
     if (e != cudaSuccess) return e;
     const int table_ctas = a.warm_layer >= 0 ? 0 : warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
-    k_update_apply<<<table_ctas + a.B * (a.warm_layer >= 0 ? 1 : a.L), kUpdThreads, smem, st>>>(a, rz ? *rz : ResizeArgs{}, table_ctas,
-                                                                     rz ? 1 : 0, warp_tables ? 1 : 0);
-    return cudaGetLastError();
+    return launch_chained(k_update_apply, table_ctas + a.B * (a.warm_layer >= 0 ? 1 : a.L), kUpdThreads, smem, st, a,
+                          rz ? *rz : ResizeArgs{}, table_ctas, rz ? 1 : 0, warp_tables ? 1 : 0);
 }
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
@@ -465,8 +470,7 @@ cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launche
     const cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_resize), smem, &opted);
     if (e != cudaSuccess) return e;
     ++*launches;
-    k_resize<<<a.S, kUpdThreads, smem, st>>>(a);
-    return cudaGetLastError();
+    return launch_chained(k_resize, a.S, kUpdThreads, smem, st, a);
 }
 
 }  // namespace smtm
