@@ -21,7 +21,6 @@ struct smtm_cache {
     int32_t* d_k;
     unsigned long long* d_counters;
     int* d_status;
-    float* d_partials;  // scratch of the fused lookup: partial dot products per (frame, part)
     float* d_warm_sv;   // scratch of smtm_cache_warmup: [max_batch][C_max] semantic vectors (allocated on first use)
     void* d_dense;      // scratch of the tensor-core scorer (fast memories above 64 entries), else NULL
     void* d_cen_split[SMTM_MAX_LAYERS];   // bf16 heads and tails of the centres, per layer (same condition)
@@ -96,7 +95,6 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_k);
     cudaFree(c->d_counters);
     cudaFree(c->d_status);
-    cudaFree(c->d_partials);
     cudaFree(c->d_plan);
     cudaFree(c->d_warm_sv);
     cudaFree(c->d_dense);
@@ -176,7 +174,7 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
         timing = c->prof_events->data() + 2 * c->prof_used;
         (*c->prof_layer)[c->prof_used++] = layer;
     }
-    SMTM_CUDA(launch_lookup_fused(e, a, c->d_partials, c->sm_count, st, &c->launches, &fused, timing));
+    SMTM_CUDA(launch_lookup_fused(e, a, c->sm_count, st, &c->launches, &fused, timing));
     if (fused) return SMTM_OK;
     if (begin) {  // the other routes read the carry: put it into its reset state with a kernel of its own
         SMTM_CUDA(launch_batch_reset(b->d_sa, b->d_done, b->d_exit_layer, b->d_pred, b->B, c->k_max, st, &c->launches));
@@ -336,7 +334,6 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     ok = ok && dev_alloc(&c->d_k, S) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_counters, SMTM_CTR_COUNT) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_status, 1) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_partials, fused_partials_floats(c->max_batch, c->k_max)) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_plan, 2 * size_t(c->max_batch)) == cudaSuccess;
     for (int l = 0; l < c->L; ++l) c->d_max = c->dims[l] > c->d_max ? c->dims[l] : c->d_max;
     c->d_max = (c->d_max + 7) / 8 * 8;  // keeps the bf16 operand arrays of the tensor-core scorer 16-byte aligned

@@ -232,58 +232,126 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
     }
 }
 
-// ---- fused lookup: encode + similarity scoring in one persistent kernel -----------------------
+// ---- fused lookup: encode + similarity scoring + decision in one persistent kernel ------------
 //
-// Work is cut into units: (frame, part), a part being a run of chunks_per_unit chunks, i.e. a
-// slice of the frame's channels.  Every CTA first compacts the frames that are still active
-// and takes the units u = blockIdx.x, blockIdx.x + gridDim.x, ... of that list, so exited
-// frames cost nothing and the load is even.  Per unit the reducer warps leave the slice of
-// the semantic vector in shared memory (four buffers) as well as in the SV stash; eight dot
-// warps then share the unit's dot products, slot j on warp j % 8: each lane has every load of
-// its slot's centre slice in flight at once, so a unit costs one trip to L2.  The partial dot
-// products and the partial squared length go to global scratch [frame][part][slot]; the small
-// finishing kernel in lookup.cu adds the parts up in part order and decides.  No atomics:
+// A frame is cut into P parts (runs of chunks_per_unit chunks, i.e. slices of its channels) and
+// a thread-block cluster of P CTAs takes whole frames: CTA `rank` of the cluster streams and
+// scores part `rank`.  Every CTA first compacts the frames that are still active; cluster c
+// takes the frames c, c + clusters, ... of that list, so exited frames cost nothing and the
+// load is even.  Per frame the reducer warps leave the slice of the semantic vector in shared
+// memory (four buffers) as well as in the SV stash; eight dot warps then share the slice's dot
+// products, slot j on warp j % 8: each lane has every load of its slot's centre slice in
+// flight at once, so a frame costs one trip to L2.  The partial dot products and the partial
+// squared length go, through distributed shared memory, to a receive buffer in the cluster's
+// first CTA, whose finisher warp adds the parts up in rank order and decides: Eq. 1, Eq. 3,
+// top-2, Eq. 4 / Eq. 2 and the exit rule.  No atomics on floating point and no global scratch:
 // the evaluation order of every sum is fixed.
 constexpr int kReducersF = 4;       // reducer warps of the fused kernel; stage s belongs to warp s % kReducersF
-constexpr int kDotWarps = 8;        // warps that share the dot products of a unit
-constexpr int kSvBufs = 4;          // shared-memory slices; unit u passes through buffer u % kSvBufs
-constexpr int kThreadsFused = (kReducersF + 1 + kDotWarps) * kWarp;
-constexpr int kMaxUnits = 1024;     // units per CTA
+constexpr int kDotWarps = 8;        // warps that share the dot products of a slice
+constexpr int kSvBufs = 4;          // shared-memory slices; frame u passes through buffer u % kSvBufs
+constexpr int kRx = 4;              // receive buffers between the dot warps and the finisher
+constexpr int kRxRow = kFusedMaxK + 4;  // words per row of a receive buffer
+// A receive buffer holds P + 2 rows: one per part (the partial dots, then the partial squared length at
+// [kFusedMaxK]) and, from the first CTA's own dot warps, the slots' classes (then k at [kFusedMaxK]) and the
+// lengths of their centres, so that the finisher has nothing to fetch once the parts are in.
+constexpr int kMaxCluster = 8;      // CTAs per cluster = parts per frame
+constexpr int kThreadsFused = (kReducersF + 1 + kDotWarps + 1) * kWarp;  // reducers, producer, dot warps, finisher
+constexpr int kMaxUnits = 1024;     // frames per cluster
 constexpr int kMaxSlice = 1024;     // floats of a semantic-vector slice (eight 16-byte vectors per lane)
+constexpr size_t kSmemLimit = 227 * 1024;
 static_assert(kStages % kReducersF == 0, "stage ownership must be periodic");
 
 struct FusedParams {
     NchwParams e;
     LookupArgs a;
-    int parts;            // P: parts per frame (divides chunks_per_frame)
+    int parts;            // P: CTAs per cluster, one part of every frame each (divides chunks_per_frame)
     int chunks_per_unit;  // chunks_per_frame / P
     int slice_cap;        // channels of a full slice = chunks_per_unit * chunk_channels (multiple of 4)
-    float* partials;      // [B][P][k_max + 1]: partial dot products per slot, then the partial squared length
 };
 
-constexpr size_t fused_smem(int slice_cap) {
-    return size_t(kStages) * kStageCap + size_t(kSvBufs) * size_t(slice_cap) * 4 + kMaxUnits * 4 +
-           (2 * kStages + 2 * kSvBufs) * 8 + 40 * 4 + 192;
+constexpr size_t fused_smem(int slice_cap, int parts) {
+    return size_t(kStages) * kStageCap + size_t(kSvBufs) * size_t(slice_cap) * 4 +
+           size_t(kRx) * size_t(parts + 2) * kRxRow * 4 + kMaxUnits * 4 + 40 * 4 +
+           (2 * kStages + 2 * kSvBufs + 2 * kRx) * 8 + 192;
+}
+
+// ---- cluster primitives ------------------------------------------------------------------------
+
+// Address of the same shared-memory location in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t peer_smem(const void* p, uint32_t rank) {
+    uint32_t out;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(smem_u32(p)), "r"(rank));
+    return out;
+}
+
+__device__ __forceinline__ void peer_store(uint32_t addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
+// Arrival on a barrier of any CTA of the cluster; orders this thread's earlier writes before it.
+__device__ __forceinline__ void peer_arrive(uint32_t bar_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_addr) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// As mbar_wait_bounded, for a barrier that CTAs of the whole cluster arrive on.
+__device__ __forceinline__ bool mbar_wait_cluster_bounded(uint64_t* bar, uint32_t parity, int* status) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (clock64() - t0 > (1ll << 31)) {
+            set_status(status, kDevTimeout);
+            return false;
+        }
+    }
+}
+
+// All threads of all CTAs of the cluster.
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 template <class R>
 __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedParams f) {
     extern __shared__ uint8_t smem_raw[];
+    const NchwParams& p = f.e;
+    const LookupArgs& a = f.a;
+    const int P = f.parts, cpu = f.chunks_per_unit;
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     uint8_t* stages = base;
     float* sv_s = reinterpret_cast<float*>(base + size_t(kStages) * kStageCap);  // [kSvBufs][slice_cap]
-    int* my_units = reinterpret_cast<int*>(sv_s + kSvBufs * f.slice_cap);        // [kMaxUnits]
-    int* s_scan = my_units + kMaxUnits;                                          // [40]
+    float* rx = sv_s + kSvBufs * f.slice_cap;                                    // [kRx][P + 2][kRxRow]
+    int* my_units = reinterpret_cast<int*>(rx + kRx * (P + 2) * kRxRow);               // [kMaxUnits] frames of this cluster
+    int* s_scan = my_units + kMaxUnits;                                          // [36]
+    unsigned int* s_ctr = reinterpret_cast<unsigned int*>(s_scan + 36);          // [4] lookups, near, exits
     uint64_t* full = reinterpret_cast<uint64_t*>(
         (reinterpret_cast<uintptr_t>(s_scan + 40) + 7) & ~uintptr_t(7));         // [kStages]
     uint64_t* empty = full + kStages;                                            // [kStages]
     uint64_t* sv_full = empty + kStages;                                         // [kSvBufs]  slice written
     uint64_t* sv_empty = sv_full + kSvBufs;                                      // [kSvBufs]  slice read by all dot warps
+    uint64_t* rx_full = sv_empty + kSvBufs;                                      // [kRx]  every part has arrived here
+    uint64_t* rx_empty = rx_full + kRx;                                          // [kRx]  every rank: the finisher is done with it
 
-    const NchwParams& p = f.e;
-    const LookupArgs& a = f.a;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int P = f.parts, cpu = f.chunks_per_unit;
+    const int rank = int(blockIdx.x) % P;       // clusters are runs of P consecutive CTAs
+    const int cluster = int(blockIdx.x) / P, n_clusters = int(gridDim.x) / P;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&full[s], 1);
@@ -293,37 +361,44 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
             mbar_init(&sv_full[s], cpu);
             mbar_init(&sv_empty[s], kDotWarps);
         }
+        for (int s = 0; s < kRx; ++s) {
+            mbar_init(&rx_full[s], P * kDotWarps);
+            mbar_init(&rx_empty[s], 1);
+        }
         mbar_init_fence();
+        s_ctr[0] = s_ctr[1] = s_ctr[2] = 0u;
     }
     chain_release();
 
-    // ---- the active frames and this CTA's share of their units -----------------------------
+    // ---- the active frames and this cluster's share of them ---------------------------------
     int n_active = a.fresh ? a.B : 0;  // a batch that starts here has every frame active: no flags to read
     for (int idx = threadIdx.x; a.fresh && idx < kMaxUnits; idx += kThreadsFused) {
-        const long long u = (long long)blockIdx.x + (long long)idx * gridDim.x;
-        if (u < (long long)a.B * P) my_units[idx] = int(u / P) * kMaxParts + int(u % P);
+        const long long u = (long long)cluster + (long long)idx * n_clusters;
+        if (u < a.B) my_units[idx] = int(u);
     }
     chain_wait();  // everything above touched shared memory only and overlaps the previous kernel's tail
     for (int t0 = 0; !a.fresh && t0 < a.B; t0 += kThreadsFused) {
         const int b = t0 + threadIdx.x;
-        const int act = (b < a.B && !a.done[b]) ? 1 : 0;
+        // Active = not exited at an earlier layer.  A finisher of this launch may already have
+        // decided the frame: an exit at this very layer leaves it active, so every CTA gets
+        // the same list whenever it looks.
+        int act = 0;
+        if (b < a.B) {
+            const int el = *reinterpret_cast<const volatile int32_t*>(a.exit_layer + b);
+            act = (el == 0 || el == a.layer + 1) ? 1 : 0;
+        }
         int cnt;
         const int pos = block_exclusive_scan(act, s_scan, &cnt);
         if (act) {
-            for (int part = 0; part < P; ++part) {
-                const int u = (n_active + pos) * P + part;
-                if (u % int(gridDim.x) == int(blockIdx.x)) {
-                    const int idx = u / int(gridDim.x);
-                    if (idx < kMaxUnits) my_units[idx] = b * kMaxParts + part;
-                }
-            }
+            const int u = n_active + pos;
+            if (u % n_clusters == cluster && u / n_clusters < kMaxUnits) my_units[u / n_clusters] = b;
         }
         n_active += cnt;
     }
-    const int total_units = n_active * P;
-    int nu = total_units > int(blockIdx.x) ? (total_units - int(blockIdx.x) + int(gridDim.x) - 1) / int(gridDim.x) : 0;
+    int nu = n_active > cluster ? (n_active - cluster + n_clusters - 1) / n_clusters : 0;
     nu = min(nu, kMaxUnits);
     __syncthreads();
+    if (P > 1) cluster_sync_all();  // every CTA's barriers exist before anyone arrives on them
 
     const int n_chunks = nu * cpu;
     bool failed = false;
@@ -332,8 +407,8 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         // ---- reducers: warp w owns the stages w, w + kReducersF, ... -----------------------------
         for (int it = warp; it < n_chunks; it += kReducersF) {
             const int i = it / cpu, c = it - i * cpu;
-            const int unit = my_units[i], b = unit / kMaxParts, part = unit % kMaxParts;
-            const int c0 = (part * cpu + c) * p.chunk_channels;
+            const int b = my_units[i];
+            const int c0 = (rank * cpu + c) * p.chunk_channels;
             const int nch = min(p.chunk_channels, p.C - c0);
             const int stage = it % kStages;
             const int buf = i % kSvBufs, round = i / kSvBufs;
@@ -352,8 +427,8 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         if (lane == 0) {
             for (int it = 0; it < n_chunks; ++it) {
                 const int i = it / cpu, c = it - i * cpu;
-                const int unit = my_units[i], b = unit / kMaxParts, part = unit % kMaxParts;
-                const int c0 = (part * cpu + c) * p.chunk_channels;
+                const int b = my_units[i];
+                const int c0 = (rank * cpu + c) * p.chunk_channels;
                 const int nch = min(p.chunk_channels, p.C - c0);
                 const int stage = it % kStages;
                 const uint32_t use = uint32_t(it / kStages);
@@ -369,13 +444,16 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
                 issued = it + 1;
             }
         }
-    } else {
-        // ---- dot warps: all of them work on unit u together, slot j on warp j % kDotWarps --------
+    } else if (warp <= kReducersF + kDotWarps) {
+        // ---- dot warps: all of them work on frame u together, slot j on warp j % kDotWarps -------
         const int dw = warp - kReducersF - 1;
-        // fast memory of the unit in hand, fetched one unit ahead
+        const int sb = rank * f.slice_cap;          // first channel of this CTA's slice
+        const int Dp = max(0, min(f.slice_cap, p.C - sb));  // channels in it (a multiple of 4)
+        const int n4 = Dp >> 2;
+        // fast memory of the frame in hand, fetched one frame ahead
         int nx_k = 0, nx_ids[2] = {0, 0};
         if (nu > 0) {
-            const int b = my_units[0] / kMaxParts;
+            const int b = my_units[0];
             const int sid = a.stream_id ? a.stream_id[b] : 0;
             nx_k = min(a.k[sid], kFusedMaxK);
             const int32_t* mem = a.members + (size_t)sid * a.k_max;
@@ -383,72 +461,159 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
             nx_ids[1] = lane + kWarp < nx_k ? mem[lane + kWarp] : 0;
         }
         for (int u = 0; u < nu; ++u) {
-            const int unit = my_units[u], b = unit / kMaxParts, part = unit % kMaxParts;
-            const int sb = part * f.slice_cap;          // first channel of the slice
-            const int Dp = min(f.slice_cap, p.C - sb);  // channels in it (a multiple of 4)
-            const int n4 = Dp >> 2;
             const int k = nx_k;
             const int ids[2] = {nx_ids[0], nx_ids[1]};  // lane l knows the classes of slots l and l + 32
-            const int buf = u % kSvBufs;
+            const int buf = u % kSvBufs, x = u % kRx;
             int nb_sid = 0;
             if (u + 1 < nu) {
-                const int nb = my_units[u + 1] / kMaxParts;
-                nb_sid = a.stream_id ? a.stream_id[nb] : 0;  // in flight while this unit is scored
+                const int nb = my_units[u + 1];
+                nb_sid = a.stream_id ? a.stream_id[nb] : 0;  // in flight while this frame is scored
             }
-            float* out = f.partials + ((size_t)b * P + part) * (a.k_max + 1);
-            if (!mbar_wait_bounded(&sv_full[buf], (u / kSvBufs) & 1, p.status)) { failed = true; break; }
-            const float4* v4 = reinterpret_cast<const float4*>(sv_s + buf * f.slice_cap);
-            if (dw == kDotWarps - 1) {  // partial squared length of the semantic vector
-                float nn = 0.f;
-                for (int q = lane; q < n4; q += kWarp) {
-                    const float4 x = v4[q];
-                    nn = fmaf(x.x, x.x, nn); nn = fmaf(x.y, x.y, nn); nn = fmaf(x.z, x.z, nn); nn = fmaf(x.w, x.w, nn);
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(kFull, nn, o);
-                if (lane == 0) out[a.k_max] = nn;
-            }
-            for (int j = dw; j < k; j += kDotWarps) {  // partial dot product of slot j (Eq. 1's numerator)
-                const int cls = __shfl_sync(kFull, (j & 32) ? ids[1] : ids[0], j & 31);
+            // The CTAs of a cluster take turns at finishing: frame u goes to CTA u % P.  This part's
+            // row of receive buffer x over there:
+            const int fin = u % P;
+            const uint32_t out = peer_smem(rx + (x * (P + 2) + rank) * kRxRow, fin);
+            // the centre slice of this warp's first slot is fetched while the slice of the
+            // semantic vector is still being pooled
+            float4 cc[kMaxSlice / 4 / kWarp];  // every load of a slot in flight at once
+            float clen = 0.f;
+            if (dw < k) {
+                const int cls = __shfl_sync(kFull, ids[0], dw);
                 const float4* crow = reinterpret_cast<const float4*>(a.centers + (size_t)cls * p.C + sb);
-                float4 cc[kMaxSlice / 4 / kWarp];  // every load of the slot in flight at once
+                if (rank == fin && lane == 0) clen = __ldg(a.cnorm + cls);
 #pragma unroll
                 for (int r = 0; r < kMaxSlice / 4 / kWarp; ++r) {
                     const int q = lane + r * kWarp;
                     cc[r] = q < n4 ? __ldg(crow + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+            if (!mbar_wait_bounded(&sv_full[buf], (u / kSvBufs) & 1, p.status)) { failed = true; break; }
+            if (u >= kRx && !mbar_wait_cluster_bounded(&rx_empty[x], (u / kRx - 1) & 1, p.status)) { failed = true; break; }
+            const float4* v4 = reinterpret_cast<const float4*>(sv_s + buf * f.slice_cap);
+            int* meta_ids = reinterpret_cast<int*>(rx + (x * (P + 2) + P) * kRxRow);  // in the finishing CTA only
+            float* meta_len = rx + (x * (P + 2) + P + 1) * kRxRow;
+            if (rank == fin && dw == 0) {  // the slots' classes and k, in the layout the finisher's lanes want
+                meta_ids[lane] = ids[0];
+                meta_ids[lane + kWarp] = ids[1];
+                if (lane == 0) meta_ids[kFusedMaxK] = k;
+            }
+            if (dw == kDotWarps - 1) {  // partial squared length of the semantic vector
+                float nn = 0.f;
+                for (int q = lane; q < n4; q += kWarp) {
+                    const float4 xv = v4[q];
+                    nn = fmaf(xv.x, xv.x, nn); nn = fmaf(xv.y, xv.y, nn); nn = fmaf(xv.z, xv.z, nn); nn = fmaf(xv.w, xv.w, nn);
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(kFull, nn, o);
+                if (lane == 0) peer_store(out + kFusedMaxK * 4, nn);
+            }
+            for (int j = dw; j < k; j += kDotWarps) {  // partial dot product of slot j (Eq. 1's numerator)
+                if (j != dw) {  // the first slot's loads are already under way
+                    const int cls = __shfl_sync(kFull, (j & 32) ? ids[1] : ids[0], j & 31);
+                    const float4* crow = reinterpret_cast<const float4*>(a.centers + (size_t)cls * p.C + sb);
+                    if (rank == fin && lane == 0) clen = __ldg(a.cnorm + cls);  // in flight with the centre
+#pragma unroll
+                    for (int r = 0; r < kMaxSlice / 4 / kWarp; ++r) {
+                        const int q = lane + r * kWarp;
+                        cc[r] = q < n4 ? __ldg(crow + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
                 }
                 float d = 0.f;
 #pragma unroll
                 for (int r = 0; r < kMaxSlice / 4 / kWarp; ++r) {
                     const int q = lane + r * kWarp;
                     if (q < n4) {
-                        const float4 x = v4[q];
-                        d = fmaf(cc[r].x, x.x, d); d = fmaf(cc[r].y, x.y, d);
-                        d = fmaf(cc[r].z, x.z, d); d = fmaf(cc[r].w, x.w, d);
+                        const float4 xv = v4[q];
+                        d = fmaf(cc[r].x, xv.x, d); d = fmaf(cc[r].y, xv.y, d);
+                        d = fmaf(cc[r].z, xv.z, d); d = fmaf(cc[r].w, xv.w, d);
                     }
                 }
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(kFull, d, o);
-                if (lane == 0) out[j] = d;
+                if (lane == 0) {
+                    peer_store(out + j * 4, d);
+                    if (rank == fin) meta_len[j] = clen;
+                }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sv_empty[buf]);
-            if (u + 1 < nu) {  // fast memory of the next unit (its stream id has arrived by now)
+            if (lane == 0) {
+                mbar_arrive(&sv_empty[buf]);
+                peer_arrive(peer_smem(&rx_full[x], fin));  // this warp's share of the part has been delivered
+            }
+            if (u + 1 < nu) {  // fast memory of the next frame (its stream id has arrived by now)
                 nx_k = min(a.k[nb_sid], kFusedMaxK);
                 const int32_t* mem = a.members + (size_t)nb_sid * a.k_max;
                 nx_ids[0] = lane < nx_k ? mem[lane] : 0;
                 nx_ids[1] = lane + kWarp < nx_k ? mem[lane + kWarp] : 0;
             }
         }
+    } else {
+        // ---- finisher warp: every P-th frame of the cluster; lane l looks after slots l and l + 32 ----
+        const float weight = float(1u << a.layer);  // 2^(l-1) with l = layer + 1
+        const int reuse = max(P, kRx);              // frames between two uses of a receive buffer in this CTA
+        for (int u = rank; u < nu; u += P) {
+            const int b = my_units[u], x = u % kRx;
+            float sa_old[2];  // the carry, fetched while the frame is being scored
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = lane + h * kWarp;
+                sa_old[h] = (j < a.k_max && !a.fresh) ? a.sa[(size_t)b * a.k_max + j] : 0.f;
+            }
+            if (!mbar_wait_cluster_bounded(&rx_full[x], (u / reuse) & 1, p.status)) { failed = true; break; }
+            const int* meta_ids = reinterpret_cast<const int*>(rx + (x * (P + 2) + P) * kRxRow);
+            const float* meta_len = rx + (x * (P + 2) + P + 1) * kRxRow;
+            const int k = meta_ids[kFusedMaxK];
+            const int ids[2] = {meta_ids[lane], meta_ids[lane + kWarp]};
+            const float clen[2] = {lane < k ? meta_len[lane] : 0.f, lane + kWarp < k ? meta_len[lane + kWarp] : 0.f};
+            float nn = 0.f, dots[2] = {0.f, 0.f};
+            for (int r = 0; r < P; ++r) {  // the parts in rank order
+                const float* row = rx + (x * (P + 2) + r) * kRxRow;
+                nn += row[kFusedMaxK];
+                if (lane < k) dots[0] += row[lane];
+                if (lane + kWarp < k) dots[1] += row[lane + kWarp];
+            }
+            __syncwarp();
+            // every rank may fill buffer x again; nobody waits for that after the last kRx frames
+            if (lane < P && u + kRx < nu) peer_arrive(peer_smem(&rx_empty[x], lane));
+            float s_cur[2] = {0.f, 0.f}, s_acc[2] = {0.f, 0.f};
+            const float sv_len = __fsqrt_rn(nn);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = lane + h * kWarp;
+                if (j < k) {
+                    s_cur[h] = (nn == 0.f || clen[h] == 0.f) ? 0.f : __fdiv_rn(dots[h], __fmul_rn(sv_len, clen[h]));  // Eq. 1
+                    s_acc[h] = __fmaf_rn(s_cur[h], weight, sa_old[h]);   // Eq. 3
+                    a.sa[(size_t)b * a.k_max + j] = s_acc[h];
+                } else if (a.fresh && j < a.k_max) {
+                    a.sa[(size_t)b * a.k_max + j] = 0.f;                 // unused slots start from zero too
+                }
+            }
+            const Top2 ta = warp_top2_keys(s_acc, ids, k, lane);
+            Top2 ts{0.f, 0.f, -1, -1};
+            if (a.sep) ts = warp_top2_keys(s_cur, ids, k, lane);  // only Eq. 2 (a diagnostic) needs it
+            if (lane == 0) {
+                const int r = decide_core(a, b, ta, ts);
+                s_ctr[0] += 1u;  // only this lane touches the tallies until the CTA is done
+                if (r & 2) s_ctr[1] += 1u;
+                if (r & 1) s_ctr[2] += 1u;
+            }
+        }
     }
-    // No thread leaves before every copy that was issued has landed.
+    // No thread leaves before every copy that was issued has landed, and no CTA before its
+    // peers are done with its shared memory.
     const int any_failed = __syncthreads_or(failed ? 1 : 0);
+    if (threadIdx.x < 3 && s_ctr[threadIdx.x]) {  // this CTA's tallies: lookups, near-threshold, exits
+        const int slot = threadIdx.x == 0 ? SMTM_CTR_LOOKUPS : threadIdx.x == 1 ? SMTM_CTR_NEAR : SMTM_CTR_EXITS + a.layer;
+        atomicAdd(&a.counters[slot], (unsigned long long)s_ctr[threadIdx.x]);
+    }
     if (any_failed && warp == kReducersF && lane == 0) {
         for (int s = 0; s < kStages && s < issued; ++s) {
             const uint32_t last_use = uint32_t((issued - 1 - s) / kStages);
             mbar_wait_bounded(&full[s], last_use & 1, p.status);
         }
     }
+    __syncthreads();
+    if (P > 1) cluster_sync_all();
 }
 
 // ---- NHWC: direct coalesced loads ----------------------------------------------------------
@@ -650,8 +815,24 @@ Reducer plan_nchw(const EncodeArgs& a, NchwParams* p) {
 
 template <class R>
 cudaError_t opt_in_fused() {
-    return cudaFuncSetAttribute(k_lookup_nchw<R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                int(fused_smem(kMaxSlice)));
+    return cudaFuncSetAttribute(k_lookup_nchw<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemLimit));
+}
+
+// Clusters of `parts` CTAs of the fused kernel that the device runs at once (each CTA fills an SM).
+template <class R>
+cudaError_t max_clusters(int parts, size_t smem, int* out) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(parts));
+    cfg.blockDim = dim3(kThreadsFused);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = unsigned(parts);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaOccupancyMaxActiveClusters(out, k_lookup_nchw<R>, &cfg);
 }
 
 }  // namespace
@@ -694,57 +875,67 @@ cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, in
     return launch_generic<BF16>(a, st);
 }
 
-size_t fused_partials_floats(int max_batch, int k_max) {
-    return size_t(max_batch) * kMaxParts * (size_t(std::min(k_max, kFusedMaxK)) + 1);
-}
-
-cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float* partials, int sm_count,
-                                cudaStream_t st, int64_t* launches, bool* handled, const cudaEvent_t* timing) {
+cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm_count, cudaStream_t st,
+                                int64_t* launches, bool* handled, const cudaEvent_t* timing) {
     *handled = false;
-    if (e.B <= 0 || e.layout != SMTM_NCHW || a.k_max > kFusedMaxK || !partials) return cudaSuccess;
+    if (e.B <= 0 || e.layout != SMTM_NCHW || a.k_max > kFusedMaxK) return cudaSuccess;
     FusedParams f{};
     const Reducer r = plan_nchw(e, &f.e);
     if (r == kNone) return cudaSuccess;
-    // Parts per frame.  A unit must fit the scorers' registers (slice <= kMaxSlice channels, a
-    // multiple of 4); among the divisors of the chunk count take the smallest that fills the
-    // last round of units to 95 % (else the best filled), preferring units of >= 4 chunks.
     const int cpf = f.e.chunks_per_frame;
     if ((e.C & 3) || (f.e.chunk_channels & 3)) return cudaSuccess;
-    const auto pick = [&](int min_chunks) {
-        int best_d = 0;
-        double best_eff = -1.0;
-        for (int d = 1; d <= std::min(cpf, kMaxParts); ++d) {
-            if (cpf % d || cpf / d < min_chunks || (cpf / d) * f.e.chunk_channels > kMaxSlice) continue;
-            if (((long long)e.B * d + sm_count - 1) / sm_count > kMaxUnits) continue;
-            const double rounds = double(e.B) * d / sm_count;
-            const double eff = rounds / std::ceil(rounds);
-            if (eff >= 0.95) return d;
-            if (eff > best_eff + 1e-9) {
-                best_eff = eff;
-                best_d = d;
+    // Parts per frame = CTAs per cluster.  A part must fit the scorers' registers (slice <= kMaxSlice
+    // channels, a multiple of 4) and the CTA's shared memory; among 1, 2, 4, 8 take the smallest
+    // that keeps the SMs 95 % busy over the rounds of frames (else the busiest).
+    static int cluster_cap[kTeamBf16 + 1][kMaxCluster + 1];  // clusters the device runs at once, 0 = not asked yet
+    int best_P = 0, best_grid = 0;
+    double best_eff = -1.0;
+    for (int P = 1; P <= kMaxCluster; P *= 2) {
+        if (cpf % P || (cpf / P) * f.e.chunk_channels > kMaxSlice) continue;
+        const size_t smem = fused_smem((cpf / P) * f.e.chunk_channels, P);
+        if (smem > kSmemLimit) continue;
+        int clusters = sm_count;
+        if (P > 1) {
+            int& cap = cluster_cap[r][P];
+            if (cap == 0) {
+                cudaError_t err = cudaSuccess;
+#define SMTM_ASK(...) err = max_clusters<__VA_ARGS__>(P, smem, &cap)
+                SMTM_FOR_REDUCER(r, SMTM_ASK)
+#undef SMTM_ASK
+                if (err != cudaSuccess) {
+                    (void)cudaGetLastError();
+                    cap = -1;
+                }
             }
+            if (cap <= 0) continue;
+            clusters = std::min(cap, sm_count / P);
         }
-        return (best_eff >= 0.8 || min_chunks <= 1) ? best_d : 0;
-    };
-    int P = pick(4);
-    if (P == 0) P = pick(1);
-    if (P <= 0) return cudaSuccess;
+        if (clusters < 1 || ((long long)e.B + clusters - 1) / clusters > kMaxUnits) continue;
+        const double rounds = double(e.B) / clusters;
+        const double eff = rounds / std::ceil(rounds) * double(clusters * P) / sm_count;
+        if (eff > best_eff + 1e-9) {
+            best_eff = eff;
+            best_P = P;
+            best_grid = clusters * P;
+        }
+        if (eff >= 0.95) break;
+    }
+    if (best_P == 0) return cudaSuccess;
+    const int P = best_P;
     f.a = a;
     f.parts = P;
     f.chunks_per_unit = cpf / P;
     f.slice_cap = f.chunks_per_unit * f.e.chunk_channels;
-    f.partials = partials;
-    const size_t smem = fused_smem(f.slice_cap);
+    const size_t smem = fused_smem(f.slice_cap, P);
     cudaError_t err = cudaSuccess;
     if (timing) record_timing(timing[0], st);
-#define SMTM_LAUNCH(...) err = launch_chained(k_lookup_nchw<__VA_ARGS__>, sm_count, kThreadsFused, smem, st, f)
+#define SMTM_LAUNCH(...) err = launch_chained_cluster(k_lookup_nchw<__VA_ARGS__>, best_grid, kThreadsFused, smem, P, st, f)
     SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
 #undef SMTM_LAUNCH
     if (timing) record_timing(timing[1], st);
     ++*launches;
     *handled = true;
-    if (err != cudaSuccess) return err;
-    return launch_finish_partials(a, partials, P, st, launches);
+    return err;
 }
 
 cudaError_t launch_row_norm2(const float* sv, const uint8_t* skip, int B, int D, float* out, cudaStream_t st,

@@ -21,19 +21,29 @@ inline cudaError_t record_timing(cudaEvent_t ev, cudaStream_t st) {
 // (programmatic stream serialisation); the kernel itself waits with chain_wait() before it
 // touches global memory.
 template <class... Params, class... Args>
-cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                           Args&&... args) {
+cudaError_t launch_chained_cluster(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, int cluster_x,
+                                   cudaStream_t st, Args&&... args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;  // thread-block clusters of cluster_x consecutive CTAs
+    attr[1].val.clusterDim.x = unsigned(cluster_x);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = cluster_x > 1 ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
+template <class... Params, class... Args>
+cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                           Args&&... args) {
+    return launch_chained_cluster(kernel, grid, block, smem, 1, st, static_cast<Args&&>(args)...);
 }
 
 // Number of exit layers and the fast-memory capacity of a cache.
@@ -82,17 +92,11 @@ struct LookupArgs {
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches);
 // Encode + score + exit in one kernel (NCHW shapes the streaming pipeline serves, fast
 // memories of at most 64 entries).  *handled is false when the shape is not served, in which
-// case nothing was launched.  partials: fused_partials_floats() floats of scratch.
+// case nothing was launched.
 constexpr int kFusedMaxK = 64;  // fast-memory capacity the fused path supports (two slots per lane)
-constexpr int kMaxParts = 16;   // most parts a frame is cut into
-size_t fused_partials_floats(int max_batch, int k_max);
-// timing: nullptr, or two events recorded on `st` right before and after the streaming kernel.
-cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, float* partials, int sm_count,
-                                cudaStream_t st, int64_t* launches, bool* handled, const cudaEvent_t* timing);
-// Second half of the fused lookup: adds up the parts of every active frame in part order,
-// then Eq. 1, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule.  partials: [B][parts][k_max + 1].
-cudaError_t launch_finish_partials(const LookupArgs& a, const float* partials, int parts, cudaStream_t st,
-                                   int64_t* launches);
+// timing: nullptr, or two events recorded on `st` right before and after the kernel.
+cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm_count, cudaStream_t st,
+                                int64_t* launches, bool* handled, const cudaEvent_t* timing);
 // ---- large fast memories: dot products against every class on the tensor cores ---------------
 bool dense_scoring_supported(int D, int n);
 size_t dense_scratch_bytes(int max_batch, int n, int d_max);

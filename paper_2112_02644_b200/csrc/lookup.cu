@@ -145,62 +145,6 @@ __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, c
     }
 }
 
-// Finishing kernel of the fused lookup: a warp per frame.  Lane l looks after slots l and
-// l + 32; the parts of each sum are added in part order.
-__global__ void __launch_bounds__(kThreads) k_finish_partials(const LookupArgs a, const float* __restrict__ partials,
-                                                              int P) {
-    chain_release();
-    chain_wait();
-    const int lane = threadIdx.x & 31;
-    const int b = blockIdx.x * (kThreads / kWarp) + (threadIdx.x >> 5);
-    if (b >= a.B || (!a.fresh && a.done[b])) return;
-    const int sid = a.stream_id ? a.stream_id[b] : 0;
-    const int k = min(a.k[sid], kFusedMaxK);
-    const int32_t* mem = a.members + (size_t)sid * a.k_max;
-    const float weight = float(1u << a.layer);  // 2^(l-1) with l = layer + 1
-    int ids[2];
-    float clen[2], sa_old[2];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const int j = lane + h * kWarp;
-        ids[h] = j < k ? mem[j] : 0;
-        clen[h] = j < k ? a.cnorm[ids[h]] : 0.f;
-        sa_old[h] = (j < k && !a.fresh) ? a.sa[(size_t)b * a.k_max + j] : 0.f;
-    }
-    float pn[kMaxParts], p0[kMaxParts], p1[kMaxParts];
-#pragma unroll
-    for (int q = 0; q < kMaxParts; ++q) {
-        const float* src = partials + ((size_t)b * P + q) * (a.k_max + 1);
-        pn[q] = q < P ? src[a.k_max] : 0.f;
-        p0[q] = (q < P && lane < k) ? src[lane] : 0.f;
-        p1[q] = (q < P && lane + kWarp < k) ? src[lane + kWarp] : 0.f;
-    }
-    float nn = 0.f, dots[2] = {0.f, 0.f};
-#pragma unroll
-    for (int q = 0; q < kMaxParts; ++q) {
-        if (q < P) {
-            nn += pn[q];
-            dots[0] += p0[q];
-            dots[1] += p1[q];
-        }
-    }
-    float s_cur[2] = {0.f, 0.f}, s_acc[2] = {0.f, 0.f};
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const int j = lane + h * kWarp;
-        if (j < k) {
-            s_cur[h] = cosine_from(dots[h], nn, clen[h]);        // Eq. 1
-            s_acc[h] = __fmaf_rn(s_cur[h], weight, sa_old[h]);   // Eq. 3
-            a.sa[(size_t)b * a.k_max + j] = s_acc[h];
-        } else if (a.fresh && j < a.k_max) {
-            a.sa[(size_t)b * a.k_max + j] = 0.f;                 // unused slots start from zero too
-        }
-    }
-    const Top2 ta = warp_top2_regs(s_acc, ids, k, lane);
-    const Top2 ts = warp_top2_regs(s_cur, ids, k, lane);
-    if (lane == 0) decide_from_top2(a, b, ta, ts);
-}
-
 __global__ void k_batch_reset(float* __restrict__ sa, uint8_t* __restrict__ done, int32_t* __restrict__ exit_layer,
                               int32_t* __restrict__ pred, int B, long long n_sa) {
     chain_release();
@@ -224,14 +168,6 @@ cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, in
     const int grid = int(std::min<long long>((n_sa + 255) / 256, 1184));
     ++*launches;
     return launch_chained(k_batch_reset, grid, 256, 0, st, sa, done, exit_layer, pred, B, n_sa);
-}
-
-cudaError_t launch_finish_partials(const LookupArgs& a, const float* partials, int parts, cudaStream_t st,
-                                   int64_t* launches) {
-    if (a.B <= 0) return cudaSuccess;
-    ++*launches;
-    const int per_cta = kThreads / kWarp;
-    return launch_chained(k_finish_partials, (a.B + per_cta - 1) / per_cta, kThreads, 0, st, a, partials, parts);
 }
 
 cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, cudaStream_t st, int64_t* launches) {
