@@ -14,6 +14,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import subprocess
 import sys
@@ -154,7 +155,9 @@ def run_ours(args):
     base = si.WORKLOADS[[k for k in si.WORKLOADS if k.startswith(args.workload)][0]]
     w = shard_for_rank(base, rank)
     K, W = args.steps, args.warmup
-    T = min(w.T, max(K, W))
+    G = math.gcd(K, 8)          # steps captured into one CUDA graph
+    T = min(w.T, max(K, W, G))
+    T -= T % G                  # resident steps: a whole number of graphs
     labs = si.labels(w)
     cents, counts = si.initial_centers(w)
     sid = si.stream_ids(w)
@@ -182,20 +185,21 @@ def run_ours(args):
         for t in range(W):          # eager warm-up: kernels, clocks, one-time function attributes
             step(cache, gb, t)
         stream.synchronize()
-        # one graph per resident step (its feature maps are baked in); the cache state lives in
-        # device memory the graphs point to, so replaying them in order advances it as eager calls would
+        # One graph per G resident steps (their feature maps are baked in); the cache state lives in
+        # device memory the graphs point to, so replaying them in order advances it as eager calls
+        # would.  Inside a graph the kernels of consecutive steps are chained like those of one step.
         smtm.smtm_cache_profile(cache, (T // PROFILE_EVERY + 1) * w.L, PROFILE_EVERY)
         launches0 = smtm.smtm_cache_get_launches(cache)
         graphs = []
-        for t in range(T):
+        for g0 in range(0, T, G):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=stream):
-                step(cache, gb, t)
+                for t in range(g0, g0 + G):
+                    step(cache, gb, t)
             graphs.append(g)
         launches_per_cycle = smtm.smtm_cache_get_launches(cache) - launches0
-        for t in range(W, W + min(3, T)):   # graph warm-up (uploads), continuing the step sequence
-            graphs[t % T].replay()
-        first = W + min(3, T)
+        for g in graphs:   # every graph once, untimed: its first launch uploads it to the device
+            g.replay()
         stream.synchronize()
         ctr0 = smtm.smtm_cache_get_counters(cache)
         start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -205,8 +209,8 @@ def run_ours(args):
         torch.cuda.synchronize()
         sampler.start()
         start.record(stream)
-        for t in range(first, first + K):
-            graphs[t % T].replay()
+        for i in range(K // G):
+            graphs[i % len(graphs)].replay()
         stop.record(stream)
         torch.cuda.synchronize()
     if world > 1:
@@ -245,7 +249,7 @@ def run_ours(args):
                        "classes": w.n, "fast_memory": [w.k_min, w.k_max], "tau": w.tau, "window_W": w.window_W,
                        "distinct_steps_resident": T, "l2_policy": "distinct maps per step, %.0f MB per step (L2 is 126 MB)" % (sum(w.B * w.frame_bytes(l) for l in range(w.L)) / 1e6),
                        "sharding": "streams across GPUs, no collective",
-                       "launch": "one CUDA graph per step (%d lookups, update+refresh)" % w.L},
+                       "launch": "CUDA graphs of %d steps (per step: %d lookups, update+refresh), chained launches" % (G, w.L)},
             "e2e": e2e,
             "gpu_launches": int(launches),
             "clocks": clocks,

@@ -5,13 +5,14 @@
 // ascending frame index, so the result is the one a frame-by-frame replay would give and does
 // not depend on scheduling.
 //
-// An update is two launches.  k_update_plan writes every frame's final label and stop layer
+// An update is three launches.  k_update_plan writes every frame's final label and stop layer
 // and elects, per class and per stream present in the batch, its first frame (an integer
 // atomicMax on a tag that carries the call's sequence number, so the election tables never
-// need clearing).  In k_update_apply every frame's warp (tables, optionally followed by its
-// stream's Eq. 5 / Eq. 6 refresh) and every (frame, layer) CTA (Eq. 7) first checks whether
-// its frame was elected and leaves at once if not; classes and streams the batch does not
-// touch cost nothing.
+// need clearing).  In k_update_centers every (frame, layer) CTA (Eq. 7) and in k_update_tables
+// every frame's warp (tables, optionally followed by its stream's Eq. 5 / Eq. 6 refresh)
+// first checks whether its frame was elected and leaves at once if not; classes and streams
+// the batch does not touch cost nothing.  The two are separate kernels because the tables
+// live in registers: with few registers the Eq. 7 CTAs are all resident at once.
 #include <algorithm>
 
 #include "common.cuh"
@@ -307,23 +308,19 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
     if (lane == 0) rz.k[s] = chosen;
 }
 
-// blockIdx.x <  table_ctas : tables (and, if asked, the refresh) of the streams whose first
-//                            frames are among this CTA's frames: a warp per frame, or, when
-//                            the classes do not fit a warp's registers, the whole CTA for one
-// blockIdx.x >= table_ctas : centre of (class of frame g, layer), g, layer = divmod(blockIdx.x
-//                            - table_ctas, L), if g is the first frame of its class
-__global__ void __launch_bounds__(kUpdThreads) k_update_apply(const UpdateArgs a, const ResizeArgs rz, int table_ctas,
-                                                              int do_resize, int warp_tables) {
+// Tables (and, if asked, the refresh) of the streams whose first frames are among this CTA's
+// frames: a warp per frame, or, when the classes do not fit a warp's registers, the whole CTA
+// for one frame.
+__global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs a, const ResizeArgs rz, int do_resize,
+                                                               int warp_tables) {
     extern __shared__ unsigned long long s_dyn[];
     __shared__ int s_list[kUpdThreads];
     __shared__ int s_scan[33];
-    __shared__ float s_red[32];
     __shared__ unsigned long long s_part[kUpdWarps];
     const int tid = threadIdx.x;
     chain_release();
     chain_wait();
-
-    if (int(blockIdx.x) < table_ctas) {
+    {
         if (warp_tables) {
             const int g = blockIdx.x * kUpdWarps + (tid >> 5);
             if (g >= a.B) return;
@@ -353,11 +350,19 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_apply(const UpdateArgs a
             __syncthreads();  // this CTA's table writes are visible to all of its threads
             resize_stream(rz, s, reinterpret_cast<unsigned char*>(s_dyn), s_scan, s_part);
         }
-        return;
     }
+}
 
-    // ---- Eq. 7 for one (class, layer): fold the matching frames in ascending index --------
-    const int job = blockIdx.x - table_ctas;
+// Eq. 7 for one (class, layer): CTA (g, layer) folds, if g is the first frame of its class, the
+// matching frames in ascending index.  g, layer = divmod(blockIdx.x, layers touched).
+__global__ void __launch_bounds__(kUpdThreads) k_update_centers(const UpdateArgs a) {
+    __shared__ int s_list[kUpdThreads];
+    __shared__ int s_scan[33];
+    __shared__ float s_red[32];
+    const int tid = threadIdx.x;
+    chain_release();
+    chain_wait();
+    const int job = blockIdx.x;
     const int nl = a.warm_layer >= 0 ? 1 : a.L;  // a warm-up touches one layer only
     const int g = job / nl, l0 = a.warm_layer >= 0 ? a.warm_layer : job - g * nl;  // l0 is 0-based; the paper's is l0 + 1
     const int cls = a.plan.final_label[g];
@@ -454,14 +459,18 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, cudaStream_
     // a warp per frame when the classes fit its registers and eight refresh buffers fit a CTA
     const bool warp_tables = a.n <= kWarpTablesMaxN && per_stream * kUpdWarps <= 96 * 1024;
     const size_t smem = warp_tables ? per_stream * kUpdWarps : per_stream;
-    cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_apply), smem, &opted);
+    cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_tables), smem, &opted);
     if (e != cudaSuccess) return e;
-    *launches += 2;
+    ++*launches;
     e = launch_chained(k_update_plan, (a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st, a);
     if (e != cudaSuccess) return e;
-    const int table_ctas = a.warm_layer >= 0 ? 0 : warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
-    return launch_chained(k_update_apply, table_ctas + a.B * (a.warm_layer >= 0 ? 1 : a.L), kUpdThreads, smem, st, a,
-                          rz ? *rz : ResizeArgs{}, table_ctas, rz ? 1 : 0, warp_tables ? 1 : 0);
+    ++*launches;
+    e = launch_chained(k_update_centers, a.B * (a.warm_layer >= 0 ? 1 : a.L), kUpdThreads, 0, st, a);
+    if (e != cudaSuccess || a.warm_layer >= 0) return e;  // a warm-up batch has no streams
+    const int table_ctas = warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
+    ++*launches;
+    return launch_chained(k_update_tables, table_ctas, kUpdThreads, smem, st, a, rz ? *rz : ResizeArgs{}, rz ? 1 : 0,
+                          warp_tables ? 1 : 0);
 }
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
