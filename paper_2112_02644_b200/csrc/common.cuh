@@ -22,9 +22,12 @@ __device__ __forceinline__ void set_status(int* status, int code) {
 //
 // Every kernel of the library is launched with programmatic stream serialisation: its CTAs may
 // become resident, and run their prologue, while the kernel before it in the stream is still
-// finishing.  chain_release() lets the next kernel's CTAs in as soon as all of this kernel's
-// have started; chain_wait() returns once the previous kernel has completed and its writes
-// are visible.  Nothing that reads or writes global memory comes before chain_wait().
+// running.  chain_wait() returns once the previous kernel has completed and its writes are
+// visible; nothing that reads or writes global memory comes before it.  chain_release() lets
+// the next kernel's CTAs in as soon as all of this kernel's have called it.  Kernels call it
+// right after chain_wait(): a kernel then only ever shares the device with its direct
+// neighbours (released before the wait, a chain of small kernels would let a much later
+// kernel in, whose CTAs take registers and shared memory away from the ones still running).
 
 __device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

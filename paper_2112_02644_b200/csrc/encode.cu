@@ -177,9 +177,9 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
         }
         mbar_init_fence();
     }
-    chain_release();
     __syncthreads();
     chain_wait();  // the barriers are set up while the previous kernel finishes
+    chain_release();
 
     const bool producer = warp == kConsumers;  // last warp; lane 0 issues the copies
     int it = 0;                                // chunks of this CTA that are not skipped, so far
@@ -368,7 +368,6 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         mbar_init_fence();
         s_ctr[0] = s_ctr[1] = s_ctr[2] = 0u;
     }
-    chain_release();
 
     // ---- the active frames and this cluster's share of them ---------------------------------
     int n_active = a.fresh ? a.B : 0;  // a batch that starts here has every frame active: no flags to read
@@ -377,6 +376,7 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         if (u < a.B) my_units[idx] = int(u);
     }
     chain_wait();  // everything above touched shared memory only and overlaps the previous kernel's tail
+    chain_release();
     for (int t0 = 0; !a.fresh && t0 < a.B; t0 += kThreadsFused) {
         const int b = t0 + threadIdx.x;
         // Active = not exited at an earlier layer.  A finisher of this launch may already have
@@ -626,8 +626,8 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_encode_nhwc(const uint8_t* __r
                                                               float* __restrict__ sv, int B, int C, int HW,
                                                               float inv_hw) {
     extern __shared__ float part[];  // [phases][min(C, 256 * kPerVec)]
-    chain_release();
     chain_wait();
+    chain_release();
     constexpr int V = E::kPerVec;
     const int CG = C / V;            // 16-byte vectors per pixel
     for (int b = blockIdx.x; b < B; b += gridDim.x) {
@@ -682,8 +682,8 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_encode_nhwc(const uint8_t* __r
 template <class E>
 __global__ void k_encode_generic(const void* __restrict__ x, const uint8_t* __restrict__ skip,
                                  float* __restrict__ sv, int B, int C, int HW, int nhwc, float inv_hw) {
-    chain_release();
     chain_wait();
+    chain_release();
     const long long total = (long long)B * C;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -702,8 +702,8 @@ __global__ void k_encode_generic(const void* __restrict__ x, const uint8_t* __re
 __global__ void k_row_norm2(const float* __restrict__ sv, const uint8_t* __restrict__ skip, int B, int D,
                             float* __restrict__ out) {
     __shared__ float scratch[32];
-    chain_release();
     chain_wait();
+    chain_release();
     const int b = blockIdx.x;
     if (skip && skip[b]) return;
     float s = 0.f;

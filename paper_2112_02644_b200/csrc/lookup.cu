@@ -25,8 +25,8 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
     float* s_acc = s_cur + a.k_max;   // [k_max] cumulative similarities
     __shared__ float scratch[32];
 
-    chain_release();
     chain_wait();
+    chain_release();
     const int b = blockIdx.x;
     if (a.done[b]) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -80,8 +80,8 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
 __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, const float* __restrict__ dots) {
     __shared__ float scratch[32];
     __shared__ Top2 s_top[2][kThreads / kWarp];
-    chain_release();
     chain_wait();
+    chain_release();
     const int b = blockIdx.x;
     if (a.done[b]) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -147,8 +147,8 @@ __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, c
 
 __global__ void k_batch_reset(float* __restrict__ sa, uint8_t* __restrict__ done, int32_t* __restrict__ exit_layer,
                               int32_t* __restrict__ pred, int B, long long n_sa) {
-    chain_release();
     chain_wait();
+    chain_release();
     const long long i0 = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     const long long step = (long long)gridDim.x * blockDim.x;
     for (long long i = i0; i < n_sa; i += step) sa[i] = 0.f;

@@ -56,8 +56,8 @@ __device__ __forceinline__ unsigned long long tag_of(unsigned long long epoch, i
 // Label and stop layer of a finished frame: the prediction and exit layer if it exited,
 // else the fallback label (the full network's answer, -1 = none) and L.
 __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a) {
-    chain_release();
     chain_wait();
+    chain_release();
     const int b = blockIdx.x * kUpdThreads + threadIdx.x;
     if (b >= a.B) return;
     const bool ex = a.done && a.done[b] != 0;  // no carry at all: a warm-up batch of labelled frames
@@ -167,8 +167,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_resize(const ResizeArgs a) {
     extern __shared__ unsigned long long s_dyn[];
     __shared__ int s_scan[33];
     __shared__ unsigned long long s_part[kUpdThreads / 32];
-    chain_release();
     chain_wait();
+    chain_release();
     resize_stream(a, blockIdx.x, reinterpret_cast<unsigned char*>(s_dyn), s_scan, s_part);
 }
 
@@ -318,8 +318,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
     __shared__ int s_scan[33];
     __shared__ unsigned long long s_part[kUpdWarps];
     const int tid = threadIdx.x;
-    chain_release();
     chain_wait();
+    chain_release();
     {
         if (warp_tables) {
             const int g = blockIdx.x * kUpdWarps + (tid >> 5);
@@ -360,8 +360,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_centers(const UpdateArgs
     __shared__ int s_scan[33];
     __shared__ float s_red[32];
     const int tid = threadIdx.x;
-    chain_release();
     chain_wait();
+    chain_release();
     const int job = blockIdx.x;
     const int nl = a.warm_layer >= 0 ? 1 : a.L;  // a warm-up touches one layer only
     const int g = job / nl, l0 = a.warm_layer >= 0 ? a.warm_layer : job - g * nl;  // l0 is 0-based; the paper's is l0 + 1
@@ -424,8 +424,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_centers(const UpdateArgs
 
 __global__ void k_center_norms(const float* __restrict__ centers, int n, int D, float* __restrict__ cnorm) {
     __shared__ float s_red[32];
-    chain_release();
     chain_wait();
+    chain_release();
     const int c = blockIdx.x;
     float nrm = 0.f;
     for (int d = threadIdx.x; d < D; d += blockDim.x) {
