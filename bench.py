@@ -225,6 +225,8 @@ def run_ours(args):
     # roofline of the dominant launch (stage-3 lookup: every frame active)
     dom_total_ms, dom_n = smtm.smtm_cache_get_profile(cache, 0)
     dom_ms = dom_total_ms / max(dom_n, 1)
+    dev_total_ms, dev_n = smtm.smtm_cache_get_profile_device(cache, 0)
+    dev_ms = dev_total_ms / dev_n if dev_n else None
     l1_total_ms, l1_n = smtm.smtm_cache_get_profile(cache, 1) if w.L > 1 else (0.0, 0)
     C0 = w.stages[0][0]
     dom_bytes = w.B * (w.frame_bytes(0) + 4 * C0)
@@ -257,7 +259,11 @@ def run_ours(args):
                          "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                          "traffic": ncu_traffic(base.name, w.B, base.B), "bytes_per_launch": dom_bytes, "us_per_launch": dom_ms * 1e3,
                          "frac_of_nominal_8TBs": achieved / 8000.0, "launches_timed": int(dom_n),
-                         "stage4_kernel_us_per_launch": l1_total_ms / max(l1_n, 1) * 1e3},
+                         "stage4_kernel_us_per_launch": l1_total_ms / max(l1_n, 1) * 1e3,
+                         "device_clock": None if dev_ms is None else {
+                             "us_per_launch": dev_ms * 1e3, "achieved": dom_bytes / (dev_ms * 1e-3) / 1e9,
+                             "frac": dom_bytes / (dev_ms * 1e-3) / 1e9 / peak, "launches_timed": int(dev_n),
+                             "note": "first CTA's start to last CTA's end by %globaltimer; the CUDA-event figure above also holds the two event nodes around the kernel"}},
             "exit_histogram": {"per_layer": exits, "none": K * w.B - sum(exits)},
             "near_threshold_lookups": int(ctr[smtm.CTR_NEAR]),
             "device_status": status,

@@ -246,9 +246,16 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * switches it off and frees the events.  Inside a stream capture the events
  * become graph nodes that are re-recorded at every replay.
  * smtm_cache_get_profile adds up the elapsed times of the recorded lookups of
- * one layer.  Both synchronise the device. */
+ * one layer.  smtm_cache_get_profile_device does the same from the device's own
+ * clock: the fused lookup kernel notes when each of its CTAs began and ended,
+ * and a launch lasts from the first beginning to the last end (this leaves out
+ * what the events add around the kernel; only the most recent run of each
+ * recorded lookup is kept, and lookups that took another route count zero).
+ * All three synchronise the device. */
 smtm_status_t smtm_cache_profile(smtm_cache_t* cache, int32_t max_lookups, int32_t every);
 smtm_status_t smtm_cache_get_profile(smtm_cache_t* cache, int32_t layer, double* h_total_ms, int64_t* h_count);
+smtm_status_t smtm_cache_get_profile_device(smtm_cache_t* cache, int32_t layer, double* h_total_ms,
+                                            int64_t* h_count);
 
 /* Number of kernels the library has launched on behalf of this cache so far. */
 smtm_status_t smtm_cache_get_launches(smtm_cache_t* cache, int64_t* h_out);

@@ -101,6 +101,7 @@ def load_library():
     lib.smtm_cache_get_launches.argtypes = [vp, vp]
     lib.smtm_cache_profile.argtypes = [vp, i32, i32]
     lib.smtm_cache_get_profile.argtypes = [vp, i32, vp, vp]
+    lib.smtm_cache_get_profile_device.argtypes = [vp, i32, vp, vp]
     lib.smtm_cache_status.argtypes = [vp]
     lib.smtm_status_string.argtypes = [i32]
     lib.smtm_status_string.restype = ctypes.c_char_p
@@ -328,6 +329,15 @@ def smtm_cache_get_profile(cache: Cache, layer: int):
     count = ctypes.c_int64(0)
     _check(load_library().smtm_cache_get_profile(cache.handle, layer, ctypes.byref(total), ctypes.byref(count)),
            "smtm_cache_get_profile")
+    return total.value, count.value
+
+
+def smtm_cache_get_profile_device(cache: Cache, layer: int):
+    """(total milliseconds, launches) of the fused lookup kernel at ``layer`` by the device's own clock."""
+    total = ctypes.c_double(0.0)
+    count = ctypes.c_int64(0)
+    _check(load_library().smtm_cache_get_profile_device(cache.handle, layer, ctypes.byref(total), ctypes.byref(count)),
+           "smtm_cache_get_profile_device")
     return total.value, count.value
 
 

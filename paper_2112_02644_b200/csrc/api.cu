@@ -33,6 +33,7 @@ struct smtm_cache {
     std::vector<cudaEvent_t>* prof_events;  // pairs, in launch order
     std::vector<int>* prof_layer;           // layer of each pair
     size_t prof_used;                       // pairs recorded so far
+    unsigned long long* d_prof_clock;       // [pairs][kClockCtas][2] device-clock stamps of the profiled streaming kernels
     int prof_every;                         // a pair is recorded for every prof_every-th lookup call
     long long prof_seq;                     // lookup calls since profiling was switched on
     int device, sm_count;
@@ -75,6 +76,8 @@ void drop_profile(smtm_cache* c) {
         delete c->prof_layer;
         c->prof_events = nullptr;
         c->prof_layer = nullptr;
+        cudaFree(c->d_prof_clock);
+        c->d_prof_clock = nullptr;
     }
     c->prof_used = 0;
 }
@@ -172,6 +175,7 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     if (c->prof_events && (c->prof_seq++ / c->L) % c->prof_every == 0 &&
         2 * (c->prof_used + 1) <= c->prof_events->size()) {
         timing = c->prof_events->data() + 2 * c->prof_used;
+        a.clock = c->d_prof_clock + c->prof_used * size_t(2 * kClockCtas);
         (*c->prof_layer)[c->prof_used++] = layer;
     }
     SMTM_CUDA(launch_lookup_fused(e, a, c->sm_count, st, &c->launches, &fused, timing));
@@ -606,6 +610,12 @@ smtm_status_t smtm_cache_profile(smtm_cache_t* c, int32_t max_lookups, int32_t e
     c->prof_layer = new (std::nothrow) std::vector<int>(size_t(max_lookups), 0);
     if (!c->prof_events || !c->prof_layer) return SMTM_ERR_ALLOC;
     c->prof_events->reserve(2 * size_t(max_lookups));
+    const size_t clock_bytes = size_t(max_lookups) * 2 * kClockCtas * sizeof(unsigned long long);
+    if (cudaMalloc(&c->d_prof_clock, clock_bytes) != cudaSuccess || cudaMemset(c->d_prof_clock, 0, clock_bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        drop_profile(c);
+        return SMTM_ERR_ALLOC;
+    }
     for (int i = 0; i < 2 * max_lookups; ++i) {
         cudaEvent_t ev;
         if (cudaEventCreate(&ev) != cudaSuccess) {
@@ -628,6 +638,31 @@ smtm_status_t smtm_cache_get_profile(smtm_cache_t* c, int32_t layer, double* h_t
         float ms = 0.f;
         SMTM_CUDA(cudaEventElapsedTime(&ms, (*c->prof_events)[2 * i], (*c->prof_events)[2 * i + 1]));
         total += ms;
+        ++count;
+    }
+    *h_total_ms = total;
+    *h_count = count;
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_get_profile_device(smtm_cache_t* c, int32_t layer, double* h_total_ms, int64_t* h_count) {
+    if (!c || !h_total_ms || !h_count || layer < 0 || layer >= c->L) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    double total = 0.0;
+    int64_t count = 0;
+    std::vector<unsigned long long> stamps(2 * kClockCtas);
+    for (size_t i = 0; c->d_prof_clock && i < c->prof_used; ++i) {
+        if ((*c->prof_layer)[i] != layer) continue;
+        SMTM_CUDA(cudaMemcpy(stamps.data(), c->d_prof_clock + i * size_t(2 * kClockCtas),
+                             stamps.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+        unsigned long long first = ~0ull, last = 0;
+        for (int b = 0; b < kClockCtas; ++b) {
+            if (stamps[2 * b + 1] == 0) continue;  // no such CTA, or the kernel has not run
+            first = stamps[2 * b] < first ? stamps[2 * b] : first;
+            last = stamps[2 * b + 1] > last ? stamps[2 * b + 1] : last;
+        }
+        if (last == 0) continue;
+        total += double(last - first) * 1e-6;
         ++count;
     }
     *h_total_ms = total;

@@ -88,7 +88,9 @@ struct LookupArgs {
     float* sep;               // [B][L] or nullptr
     int32_t* top;             // [B][2] or nullptr
     unsigned long long* counters;
+    unsigned long long* clock;  // nullptr, or [kClockCtas][2]: the device clock (ns) at which each CTA of the streaming kernel began and ended
 };
+constexpr int kClockCtas = 256;  // CTAs whose stamps a profiled lookup keeps
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches);
 // Encode + score + exit in one kernel (NCHW shapes the streaming pipeline serves, fast
 // memories of at most 64 entries).  *handled is false when the shape is not served, in which
