@@ -225,8 +225,12 @@ def run_ours(args):
     # roofline of the dominant launch (stage-3 lookup: every frame active)
     dom_total_ms, dom_n = smtm.smtm_cache_get_profile(cache, 0)
     dom_ms = dom_total_ms / max(dom_n, 1)
-    dev_total_ms, dev_n = smtm.smtm_cache_get_profile_device(cache, 0)
-    dev_ms = dev_total_ms / dev_n if dev_n else None
+    dev_total, dev_cnt = smtm.smtm_cache_get_profile_device(cache)
+    dev_n = int(dev_cnt[0])
+    dev_ms = float(dev_total[0]) / dev_n if dev_n else None
+    dev_names = ["lookup_layer%d" % l for l in range(w.L)] + ["update_plan", "update_centers", "update_tables"]
+    dev_idx = list(range(w.L)) + [smtm.PROF_PLAN, smtm.PROF_CENTERS, smtm.PROF_TABLES]
+    dev_us = {nm: (float(dev_total[i]) / int(dev_cnt[i]) * 1e3 if dev_cnt[i] else None) for nm, i in zip(dev_names, dev_idx)}
     l1_total_ms, l1_n = smtm.smtm_cache_get_profile(cache, 1) if w.L > 1 else (0.0, 0)
     C0 = w.stages[0][0]
     dom_bytes = w.B * (w.frame_bytes(0) + 4 * C0)
@@ -264,6 +268,7 @@ def run_ours(args):
                              "us_per_launch": dev_ms * 1e3, "achieved": dom_bytes / (dev_ms * 1e-3) / 1e9,
                              "frac": dom_bytes / (dev_ms * 1e-3) / 1e9 / peak, "launches_timed": int(dev_n),
                              "note": "first CTA's start to last CTA's end by %globaltimer; the CUDA-event figure above also holds the two event nodes around the kernel"}},
+            "step_kernels_device_clock_us": dev_us,
             "exit_histogram": {"per_layer": exits, "none": K * w.B - sum(exits)},
             "near_threshold_lookups": int(ctr[smtm.CTR_NEAR]),
             "device_status": status,

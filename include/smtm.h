@@ -246,16 +246,20 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * switches it off and frees the events.  Inside a stream capture the events
  * become graph nodes that are re-recorded at every replay.
  * smtm_cache_get_profile adds up the elapsed times of the recorded lookups of
- * one layer.  smtm_cache_get_profile_device does the same from the device's own
- * clock: the fused lookup kernel notes when each of its CTAs began and ended,
- * and a launch lasts from the first beginning to the last end (this leaves out
- * what the events add around the kernel; only the most recent run of each
- * recorded lookup is kept, and lookups that took another route count zero).
- * All three synchronise the device. */
+ * one layer.  smtm_cache_get_profile_device reports, for the same steps, how long
+ * each kernel of the step ran by the device's own clock, from the moment its
+ * first CTA began (after its wait for the previous kernel) to the moment its
+ * last CTA ended: h_total_ms[i] and h_count[i], i < SMTM_PROF_KERNELS, are the
+ * sum over the profiled steps and their number, for the fused lookup kernel of
+ * layer i (i < SMTM_MAX_LAYERS; lookups that took another route count zero)
+ * and for the three update kernels (SMTM_PROF_PLAN, _CENTERS, _TABLES).  This
+ * leaves out what the event nodes add around a kernel.  Only the most recent
+ * run of each profiled step is kept.  All three synchronise the device. */
+enum { SMTM_PROF_PLAN = SMTM_MAX_LAYERS, SMTM_PROF_CENTERS, SMTM_PROF_TABLES, SMTM_PROF_KERNELS };
 smtm_status_t smtm_cache_profile(smtm_cache_t* cache, int32_t max_lookups, int32_t every);
 smtm_status_t smtm_cache_get_profile(smtm_cache_t* cache, int32_t layer, double* h_total_ms, int64_t* h_count);
-smtm_status_t smtm_cache_get_profile_device(smtm_cache_t* cache, int32_t layer, double* h_total_ms,
-                                            int64_t* h_count);
+smtm_status_t smtm_cache_get_profile_device(smtm_cache_t* cache, double* h_total_ms /*[SMTM_PROF_KERNELS]*/,
+                                            int64_t* h_count /*[SMTM_PROF_KERNELS]*/);
 
 /* Number of kernels the library has launched on behalf of this cache so far. */
 smtm_status_t smtm_cache_get_launches(smtm_cache_t* cache, int64_t* h_out);

@@ -101,7 +101,7 @@ def load_library():
     lib.smtm_cache_get_launches.argtypes = [vp, vp]
     lib.smtm_cache_profile.argtypes = [vp, i32, i32]
     lib.smtm_cache_get_profile.argtypes = [vp, i32, vp, vp]
-    lib.smtm_cache_get_profile_device.argtypes = [vp, i32, vp, vp]
+    lib.smtm_cache_get_profile_device.argtypes = [vp, vp, vp]
     lib.smtm_cache_status.argtypes = [vp]
     lib.smtm_status_string.argtypes = [i32]
     lib.smtm_status_string.restype = ctypes.c_char_p
@@ -332,13 +332,17 @@ def smtm_cache_get_profile(cache: Cache, layer: int):
     return total.value, count.value
 
 
-def smtm_cache_get_profile_device(cache: Cache, layer: int):
-    """(total milliseconds, launches) of the fused lookup kernel at ``layer`` by the device's own clock."""
-    total = ctypes.c_double(0.0)
-    count = ctypes.c_int64(0)
-    _check(load_library().smtm_cache_get_profile_device(cache.handle, layer, ctypes.byref(total), ctypes.byref(count)),
+PROF_PLAN, PROF_CENTERS, PROF_TABLES, PROF_KERNELS = MAX_LAYERS, MAX_LAYERS + 1, MAX_LAYERS + 2, MAX_LAYERS + 3
+
+
+def smtm_cache_get_profile_device(cache: Cache):
+    """(total milliseconds [PROF_KERNELS], steps [PROF_KERNELS]) by the device's own clock: index l < MAX_LAYERS is
+    the fused lookup kernel of layer l, then PROF_PLAN, PROF_CENTERS, PROF_TABLES."""
+    total = np.zeros(PROF_KERNELS, np.float64)
+    count = np.zeros(PROF_KERNELS, np.int64)
+    _check(load_library().smtm_cache_get_profile_device(cache.handle, total.ctypes.data, count.ctypes.data),
            "smtm_cache_get_profile_device")
-    return total.value, count.value
+    return total, count
 
 
 def smtm_cache_status(cache: Cache) -> int:

@@ -33,7 +33,9 @@ struct smtm_cache {
     std::vector<cudaEvent_t>* prof_events;  // pairs, in launch order
     std::vector<int>* prof_layer;           // layer of each pair
     size_t prof_used;                       // pairs recorded so far
-    unsigned long long* d_prof_clock;       // [pairs][kClockCtas][2] device-clock stamps of the profiled streaming kernels
+    unsigned long long* d_prof_clock;       // [steps][SMTM_PROF_KERNELS][2] device-clock stamps of the profiled steps
+    size_t prof_steps_cap, prof_steps_used;  // slots of d_prof_clock
+    unsigned long long* prof_step;          // the slot of the step under way, nullptr if it is not profiled
     int prof_every;                         // a pair is recorded for every prof_every-th lookup call
     long long prof_seq;                     // lookup calls since profiling was switched on
     int device, sm_count;
@@ -78,6 +80,8 @@ void drop_profile(smtm_cache* c) {
         c->prof_layer = nullptr;
         cudaFree(c->d_prof_clock);
         c->d_prof_clock = nullptr;
+        c->prof_step = nullptr;
+        c->prof_steps_used = 0;
     }
     c->prof_used = 0;
 }
@@ -172,10 +176,17 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     const EncodeArgs e = encode_args(c, f, b->d_done, b->d_sv[layer]);
     bool fused = false;
     const cudaEvent_t* timing = nullptr;
+    if (c->prof_events && c->prof_seq % c->L == 0) {  // a step begins: does it get a slot for the device-clock stamps?
+        c->prof_step = nullptr;
+        if ((c->prof_seq / c->L) % c->prof_every == 0 && c->prof_steps_used < c->prof_steps_cap) {
+            c->prof_step = c->d_prof_clock + c->prof_steps_used++ * size_t(2 * SMTM_PROF_KERNELS);
+            SMTM_CUDA(cudaMemsetAsync(c->prof_step, 0, 2 * SMTM_PROF_KERNELS * sizeof(unsigned long long), st));
+        }
+    }
+    a.clock = c->prof_events ? c->prof_step : nullptr;
     if (c->prof_events && (c->prof_seq++ / c->L) % c->prof_every == 0 &&
         2 * (c->prof_used + 1) <= c->prof_events->size()) {
         timing = c->prof_events->data() + 2 * c->prof_used;
-        a.clock = c->d_prof_clock + c->prof_used * size_t(2 * kClockCtas);
         (*c->prof_layer)[c->prof_used++] = layer;
     }
     SMTM_CUDA(launch_lookup_fused(e, a, c->sm_count, st, &c->launches, &fused, timing));
@@ -241,6 +252,7 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     a.exit_layer = b->d_exit_layer;
     a.pred = b->d_pred;
     a.fallback = d_fallback;
+    a.clock = c->prof_events ? c->prof_step : nullptr;
     a.ft = c->d_ft;
     a.ts = c->d_ts;
     for (int l = 0; l < c->L; ++l) {
@@ -610,7 +622,8 @@ smtm_status_t smtm_cache_profile(smtm_cache_t* c, int32_t max_lookups, int32_t e
     c->prof_layer = new (std::nothrow) std::vector<int>(size_t(max_lookups), 0);
     if (!c->prof_events || !c->prof_layer) return SMTM_ERR_ALLOC;
     c->prof_events->reserve(2 * size_t(max_lookups));
-    const size_t clock_bytes = size_t(max_lookups) * 2 * kClockCtas * sizeof(unsigned long long);
+    c->prof_steps_cap = size_t(max_lookups) / size_t(c->L) + 1;
+    const size_t clock_bytes = c->prof_steps_cap * 2 * SMTM_PROF_KERNELS * sizeof(unsigned long long);
     if (cudaMalloc(&c->d_prof_clock, clock_bytes) != cudaSuccess || cudaMemset(c->d_prof_clock, 0, clock_bytes) != cudaSuccess) {
         (void)cudaGetLastError();
         drop_profile(c);
@@ -645,28 +658,24 @@ smtm_status_t smtm_cache_get_profile(smtm_cache_t* c, int32_t layer, double* h_t
     return SMTM_OK;
 }
 
-smtm_status_t smtm_cache_get_profile_device(smtm_cache_t* c, int32_t layer, double* h_total_ms, int64_t* h_count) {
-    if (!c || !h_total_ms || !h_count || layer < 0 || layer >= c->L) return SMTM_ERR_INVALID_ARG;
+smtm_status_t smtm_cache_get_profile_device(smtm_cache_t* c, double* h_total_ms, int64_t* h_count) {
+    if (!c || !h_total_ms || !h_count) return SMTM_ERR_INVALID_ARG;
     SMTM_CUDA(cudaDeviceSynchronize());
-    double total = 0.0;
-    int64_t count = 0;
-    std::vector<unsigned long long> stamps(2 * kClockCtas);
-    for (size_t i = 0; c->d_prof_clock && i < c->prof_used; ++i) {
-        if ((*c->prof_layer)[i] != layer) continue;
-        SMTM_CUDA(cudaMemcpy(stamps.data(), c->d_prof_clock + i * size_t(2 * kClockCtas),
-                             stamps.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
-        unsigned long long first = ~0ull, last = 0;
-        for (int b = 0; b < kClockCtas; ++b) {
-            if (stamps[2 * b + 1] == 0) continue;  // no such CTA, or the kernel has not run
-            first = stamps[2 * b] < first ? stamps[2 * b] : first;
-            last = stamps[2 * b + 1] > last ? stamps[2 * b + 1] : last;
-        }
-        if (last == 0) continue;
-        total += double(last - first) * 1e-6;
-        ++count;
+    for (int k = 0; k < SMTM_PROF_KERNELS; ++k) {
+        h_total_ms[k] = 0.0;
+        h_count[k] = 0;
     }
-    *h_total_ms = total;
-    *h_count = count;
+    std::vector<unsigned long long> stamps(2 * SMTM_PROF_KERNELS);
+    for (size_t i = 0; c->d_prof_clock && i < c->prof_steps_used; ++i) {
+        SMTM_CUDA(cudaMemcpy(stamps.data(), c->d_prof_clock + i * stamps.size(), stamps.size() * sizeof(unsigned long long),
+                             cudaMemcpyDeviceToHost));
+        for (int k = 0; k < SMTM_PROF_KERNELS; ++k) {
+            const unsigned long long begin = ~stamps[2 * k], end = stamps[2 * k + 1];
+            if (end == 0 || end < begin) continue;  // the kernel did not run in this step
+            h_total_ms[k] += double(end - begin) * 1e-6;
+            ++h_count[k];
+        }
+    }
     return SMTM_OK;
 }
 

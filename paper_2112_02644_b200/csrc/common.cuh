@@ -32,6 +32,31 @@ __device__ __forceinline__ void set_status(int* status, int code) {
 __device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// ---- profiling by the device's clock ------------------------------------------------------------
+
+__device__ __forceinline__ unsigned long long device_clock_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Notes when the first CTA of a kernel began and the last one ended.  slot: two words that are
+// zero before the kernel runs; [0] ends up as the complement of the earliest begin, [1] as the
+// latest end (two maxima: one memset prepares both).  Thread 0 of every CTA stamps, so the
+// object has to live in a scope that thread 0 leaves last (or see every_warp).  slot == nullptr:
+// nothing happens.
+struct ClockScope {
+    unsigned long long* slot;
+    // every_warp: lane 0 of every warp stamps (kernels whose warps work on their own and leave at different times)
+    __device__ __forceinline__ explicit ClockScope(unsigned long long* s, bool every_warp = false)
+        : slot((every_warp ? (threadIdx.x & 31) == 0 : threadIdx.x == 0) ? s : nullptr) {
+        if (slot) atomicMax(slot, ~device_clock_ns());
+    }
+    __device__ __forceinline__ ~ClockScope() {
+        if (slot) atomicMax(slot + 1, device_clock_ns());
+    }
+};
+
 // ---- shared-memory barriers and bulk asynchronous copies -------------------------------
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

@@ -350,7 +350,6 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
     uint64_t* rx_empty = rx_full + kRx;                                          // [kRx]  every rank: the finisher is done with it
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned long long t_begin = 0;
     const int rank = int(blockIdx.x) % P;       // clusters are runs of P consecutive CTAs
     const int cluster = int(blockIdx.x) / P, n_clusters = int(gridDim.x) / P;
     if (threadIdx.x == 0) {
@@ -378,7 +377,7 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
     }
     chain_wait();  // everything above touched shared memory only and overlaps the previous kernel's tail
     chain_release();
-    if (a.clock && threadIdx.x == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_begin));  // profiling
+    const ClockScope stamps(a.clock ? a.clock + 2 * a.layer : nullptr);  // profiling
     for (int t0 = 0; !a.fresh && t0 < a.B; t0 += kThreadsFused) {
         const int b = t0 + threadIdx.x;
         // Active = not exited at an earlier layer.  A finisher of this launch may already have
@@ -616,12 +615,6 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
     }
     __syncthreads();
     if (P > 1) cluster_sync_all();
-    if (a.clock && threadIdx.x == 0 && blockIdx.x < kClockCtas) {  // profiling: when this CTA began and ended
-        unsigned long long t_end;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_end));
-        a.clock[2 * blockIdx.x] = t_begin;
-        a.clock[2 * blockIdx.x + 1] = t_end;
-    }
 }
 
 // ---- NHWC: direct coalesced loads ----------------------------------------------------------

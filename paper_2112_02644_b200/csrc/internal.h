@@ -88,9 +88,8 @@ struct LookupArgs {
     float* sep;               // [B][L] or nullptr
     int32_t* top;             // [B][2] or nullptr
     unsigned long long* counters;
-    unsigned long long* clock;  // nullptr, or [kClockCtas][2]: the device clock (ns) at which each CTA of the streaming kernel began and ended
+    unsigned long long* clock;  // nullptr, or the profiled step's stamps [SMTM_PROF_KERNELS][2] (see ClockScope)
 };
-constexpr int kClockCtas = 256;  // CTAs whose stamps a profiled lookup keeps
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches);
 // Encode + score + exit in one kernel (NCHW shapes the streaming pipeline serves, fast
 // memories of at most 64 entries).  *handled is false when the shape is not served, in which
@@ -131,6 +130,7 @@ struct UpdatePlan {
 
 struct UpdateArgs {
     int B, S, n, L;
+    unsigned long long* clock;  // nullptr, or the profiled step's stamps [SMTM_PROF_KERNELS][2] (see ClockScope)
     int forget_W;              // 0, or W when the frequency table itself forgets (SMTM_FLAG_FORGET_FT)
     int warm_layer;            // -1, or the one layer a warm-up batch folds into (no tables; done == nullptr)
     UpdatePlan plan;

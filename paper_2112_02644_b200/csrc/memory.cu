@@ -58,6 +58,7 @@ __device__ __forceinline__ unsigned long long tag_of(unsigned long long epoch, i
 __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a) {
     chain_wait();
     chain_release();
+    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_PLAN : nullptr);
     const int b = blockIdx.x * kUpdThreads + threadIdx.x;
     if (b >= a.B) return;
     const bool ex = a.done && a.done[b] != 0;  // no carry at all: a warm-up batch of labelled frames
@@ -320,6 +321,7 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
     const int tid = threadIdx.x;
     chain_wait();
     chain_release();
+    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_TABLES : nullptr, true);
     {
         if (warp_tables) {
             const int g = blockIdx.x * kUpdWarps + (tid >> 5);
@@ -362,6 +364,7 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_centers(const UpdateArgs
     const int tid = threadIdx.x;
     chain_wait();
     chain_release();
+    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_CENTERS : nullptr);
     const int job = blockIdx.x;
     const int nl = a.warm_layer >= 0 ? 1 : a.L;  // a warm-up touches one layer only
     const int g = job / nl, l0 = a.warm_layer >= 0 ? a.warm_layer : job - g * nl;  // l0 is 0-based; the paper's is l0 + 1
