@@ -99,7 +99,10 @@ typedef struct {
 
 /* Per-batch carry across the exit layers of one inference; every array is a
  * caller-owned device array.  Before the first layer of a batch the caller
- * zeroes d_sa, d_done and d_exit_layer and sets d_pred to -1. */
+ * zeroes d_sa, d_done and d_exit_layer and sets d_pred to -1 (smtm_batch_reset, or
+ * smtm_lookup_exit_begin for the first lookup).  The library keeps
+ * d_done[b] == (d_exit_layer[b] != 0); a caller that edits one edits the other.
+ * A layer is looked up at most once per batch. */
 typedef struct {
     int32_t B;
     const int32_t* d_stream_id; /* [B] fast memory each frame looks up; NULL = all stream 0 */
@@ -145,7 +148,9 @@ smtm_status_t smtm_encode(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t*
  * when  SA_H > 0  and  SA_H - SA_SH > tau * max(SA_SH, 0)  (Eq. 4's AC > tau,
  * division-free, evaluated in fp32), which sets d_done, d_exit_layer = layer+1
  * and d_pred.  Fewer than two members never exit.  A zero-length vector has
- * similarity 0 to everything. */
+ * similarity 0 to everything.  The fused route decides inside the streaming
+ * kernel and tells the frames that are still in from d_exit_layer (0, or this
+ * very layer when another CTA of the same launch has just decided the frame). */
 smtm_status_t smtm_lookup_exit(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t* fmap,
                                const smtm_batch_t* batch, void* stream);
 
