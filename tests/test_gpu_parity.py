@@ -270,3 +270,46 @@ def test_step_host_matches_device_path():
     for l in range(w.L):
         ca, cb = smtm.smtm_cache_get_centers(a, l), smtm.smtm_cache_get_centers(b, l)
         assert np.array_equal(ca[0], cb[0]) and np.array_equal(ca[1], cb[1])
+
+
+# ---------------------------------------------------------------------------- the fused kernel's cluster sizes
+
+@pytest.mark.parametrize("B", [5, 37, 148, 151])
+def test_fused_lookup_every_cluster_size(B):
+    # The fused lookup cuts a frame into 1, 2, 4 or 8 parts (CTAs of a cluster) depending on how many frames there
+    # are: 5 frames -> 8 parts, 37 -> 4, 148 -> 1 at the first layer (2 at the second, whose 2048 channels do not
+    # fit one part), 151 -> a ragged last round.  Fast memories of up to 64 entries use both slots of every lane.
+    w = si.Workload(f"clusters_{B}", si.BF16, si.NCHW, B=B, stages=((1024, 14, 14), (2048, 7, 7)), n=90, k_init=40,
+                    k_min=33, k_max=64, S=B if B < 100 else 1, T=2, tau=0.8, window_W=2, sigma=0.5, zipf_s=1.0, repeat_p=0.5,
+                    seed=20 + B)
+    rep = run_workload(w)
+    assert rep.frames == 2 * B and rep.lookups >= 2 * B
+
+
+def test_fused_lookup_exact_ties_go_to_the_lower_class():
+    # two classes with the same centre at every layer: their similarities tie bit for bit, the lower class id
+    # ranks first (top-1 / top-2 are selected through 64-bit keys in the fused kernel) and such a frame never exits
+    from harness import Report, step_pair
+
+    w = si.Workload("ties", si.BF16, si.NCHW, B=40, stages=((256, 14, 14), (512, 7, 7)), n=12, k_init=12, k_min=12,
+                    k_max=12, S=1, T=1, tau=0.5, window_W=4, sigma=0.3, zipf_s=0.5, seed=31)
+    cents, counts = si.initial_centers(w)
+    for l in range(w.L):
+        cents[l][1] = cents[l][0]
+        cents[l][7] = cents[l][0]
+    tau = [w.tau] * w.L
+    mem = oracle.OracleMemory(w.n, w.dims, tau, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W)
+    cache = smtm.smtm_cache_create(w.n, w.dims, tau, cents, counts, n_streams=w.S, k_init=w.k_init, k_min=w.k_min,
+                                   k_max=w.k_max, window_W=w.window_W, max_batch=w.B)
+    gb = smtm.Batch(cache, w.B)
+    lab = si.labels(w)[0]
+    ob = step_pair(w, cache, mem, gb, lab, 0, Report())
+    tied = lab == 0          # frames drawn around class 0: classes 0, 1 and 7 score the same for them
+    assert tied.sum() >= 3
+    top = gb.top.cpu().numpy()
+    assert np.array_equal(top, ob["top"])
+    assert np.all(top[tied, 0] == 0) and np.all(top[tied, 1] == 1)
+    assert not gb.done.cpu().numpy()[tied].any()
+    ac = gb.ac.cpu().numpy()
+    assert np.all(ac[tied] == 0.0)
+    smtm.smtm_cache_destroy(cache)
