@@ -171,7 +171,7 @@ def run_ours(args):
     # All launches go to one side stream so that every step can be captured into a CUDA graph.
     stream = torch.cuda.Stream()
     sh = stream.cuda_stream
-    PROFILE_EVERY = 8   # steps whose streaming kernels carry timing events (the events cost a few us each)
+    PROFILE_EVERY = 16  # every 16th step carries timing events and device-clock stamps (they cost a few us and break the chain of launches)
 
     def step(cache, gb, t):
         smtm.smtm_lookup_exit_begin(cache, 0, fmaps[t % T][0], gb, sh)     # starts the batch: no separate reset

@@ -191,12 +191,13 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     }
     SMTM_CUDA(launch_lookup_fused(e, a, c->sm_count, st, &c->launches, &fused, timing));
     if (fused) return SMTM_OK;
-    if (begin) {  // the other routes read the carry: put it into its reset state with a kernel of its own
+    const bool dense = c->d_dense && dense_scoring_supported(a.D, a.n);  // large fast memory: tensor cores
+    if (begin && !dense) {  // the plain route reads the carry: put it into its reset state with a kernel of its own
         SMTM_CUDA(launch_batch_reset(b->d_sa, b->d_done, b->d_exit_layer, b->d_pred, b->B, c->k_max, st, &c->launches));
         a.fresh = 0;
     }
-    const bool dense = c->d_dense && dense_scoring_supported(a.D, a.n);  // large fast memory: tensor cores
     EncodeArgs e2 = e;
+    if (a.fresh) e2.skip = nullptr;  // a batch that starts here: every frame is in, whatever the flags hold
     if (dense) dense_sv_split(c->d_dense, c->max_batch, c->d_max, &e2.sv_hi, &e2.sv_lo);
     bool sv_split = false;
     if (timing) SMTM_CUDA(record_timing(timing[0], st));
@@ -204,7 +205,7 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     if (timing) SMTM_CUDA(record_timing(timing[1], st));
     if (dense) {
         float* dots = nullptr;
-        SMTM_CUDA(launch_dense_dots(a.sv, a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max,
+        SMTM_CUDA(launch_dense_dots(a.sv, a.fresh ? nullptr : a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max,
                                     sv_split, c->d_cen_split[layer], c->cen_split_current[layer], &dots, c->d_status,
                                     st, &c->launches));
         c->cen_split_current[layer] = true;

@@ -76,15 +76,46 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
 
 // Finishing kernel of the tensor-core path: one CTA per frame turns the frame's row of dot
 // products into similarities of its fast-memory slots and decides.  Every thread keeps the
-// two best of its own slots; warps merge by shuffles, the CTA through shared memory.
+// two best of its own slots as 64-bit ranking keys; warps merge by two warp-wide maxima, the
+// CTA through shared memory.  With a.fresh the carry is taken as SA = 0, nobody done.
+__device__ __forceinline__ void keep_two(unsigned long long e, unsigned long long& b1, unsigned long long& b2) {
+    if (e > b1) {
+        b2 = b1;
+        b1 = e;
+    } else if (e > b2) {
+        b2 = e;
+    }
+}
+
+// The best two keys of the CTA, valid in thread 0.  (b1, b2): this thread's best two; s_keys: [2 * warps].
+__device__ __forceinline__ Top2 block_top2_keys(unsigned long long b1, unsigned long long b2, unsigned long long* s_keys) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned long long k1 = warp_max_u64(b1);
+    const unsigned long long k2 = warp_max_u64(b1 == k1 ? b2 : b1);  // keys are unique: the runner-up sits below the winner or elsewhere
+    if (lane == 0) {
+        s_keys[2 * warp] = k1;
+        s_keys[2 * warp + 1] = k2;
+    }
+    __syncthreads();
+    Top2 t{0.f, 0.f, -1, -1};
+    if (threadIdx.x == 0) {
+        unsigned long long c1 = 0ull, c2 = 0ull;
+        for (int i = 0; i < 2 * (kThreads / kWarp); ++i) keep_two(s_keys[i], c1, c2);
+        rank_key_decode(c1, &t.v1, &t.id1);
+        rank_key_decode(c2, &t.v2, &t.id2);
+    }
+    __syncthreads();
+    return t;
+}
+
 __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, const float* __restrict__ dots) {
     __shared__ float scratch[32];
-    __shared__ Top2 s_top[2][kThreads / kWarp];
+    __shared__ unsigned long long s_keys[2 * (kThreads / kWarp)];
     chain_wait();
     chain_release();
     const int b = blockIdx.x;
-    if (a.done[b]) return;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (!a.fresh && a.done[b]) return;
+    const int tid = threadIdx.x;
     const int sid = a.stream_id ? a.stream_id[b] : 0;
     const int k = a.k[sid];
     const int32_t* mem = a.members + (size_t)sid * a.k_max;
@@ -93,56 +124,46 @@ __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, c
     const float* __restrict__ drow = dots + (size_t)b * a.n;
     const float* __restrict__ clen = a.cnorm;
     float* sa_row = a.sa + (size_t)b * a.k_max;
-    Top2 ta{0.f, 0.f, -1, -1}, ts{0.f, 0.f, -1, -1};
-    float nrm = 0.f;
+    unsigned long long a1 = 0ull, a2 = 0ull, c1 = 0ull, c2 = 0ull;  // best two cumulative / single-layer keys
+    float nrm = 0.f, sv_len = 0.f;
     for (int j0 = 0; j0 < k; j0 += 4 * kThreads) {  // four slots per thread, every load issued before any store
         int cls[4];
         float dot[4], cl[4], old[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int j = j0 + u * kThreads + tid;
-            cls[u] = j < k ? mem[j] : 0;
+            cls[u] = mem[min(j, k - 1)];
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int j = j0 + u * kThreads + tid;
-            dot[u] = j < k ? drow[cls[u]] : 0.f;
-            cl[u] = j < k ? clen[cls[u]] : 0.f;
-            old[u] = j < k ? sa_row[j] : 0.f;
+            dot[u] = drow[cls[u]];
+            cl[u] = clen[cls[u]];
+            old[u] = (j < k && !a.fresh) ? sa_row[j] : 0.f;
         }
         if (j0 == 0) {  // the squared length of the semantic vector, while the loads above are in flight
             for (int d = tid; d < a.D; d += kThreads) nrm = fmaf(row[d], row[d], nrm);
             nrm = block_sum(nrm, scratch);
+            sv_len = __fsqrt_rn(nrm);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int j = j0 + u * kThreads + tid;
             if (j < k) {
-                const float s = cosine_from(dot[u], nrm, cl[u]);   // Eq. 1
+                const float s = (nrm == 0.f || cl[u] == 0.f) ? 0.f : __fdiv_rn(dot[u], __fmul_rn(sv_len, cl[u]));  // Eq. 1
                 const float acc = __fmaf_rn(s, weight, old[u]);    // Eq. 3
                 sa_row[j] = acc;
-                top2_push(ts, s, cls[u]);
-                top2_push(ta, acc, cls[u]);
+                keep_two(rank_key(acc, cls[u]), a1, a2);
+                if (a.sep) keep_two(rank_key(s, cls[u]), c1, c2);  // only Eq. 2 (a diagnostic) needs it
             }
         }
     }
-    ta = warp_top2_merge(ta);
-    ts = warp_top2_merge(ts);
-    if (lane == 0) {
-        s_top[0][warp] = ta;
-        s_top[1][warp] = ts;
-    }
-    __syncthreads();
-    if (tid == 0) {
-        for (int w = 1; w < kThreads / kWarp; ++w) {
-            const Top2 oa = s_top[0][w], os = s_top[1][w];
-            if (oa.id1 >= 0) top2_push(ta, oa.v1, oa.id1);
-            if (oa.id2 >= 0) top2_push(ta, oa.v2, oa.id2);
-            if (os.id1 >= 0) top2_push(ts, os.v1, os.id1);
-            if (os.id2 >= 0) top2_push(ts, os.v2, os.id2);
-        }
-        decide_from_top2(a, b, ta, ts);
-    }
+    if (a.fresh)
+        for (int j = k + tid; j < a.k_max; j += kThreads) sa_row[j] = 0.f;  // unused slots start from zero too
+    const Top2 ta = block_top2_keys(a1, a2, s_keys);
+    Top2 ts{0.f, 0.f, -1, -1};
+    if (a.sep) ts = block_top2_keys(c1, c2, s_keys);
+    if (tid == 0) decide_from_top2(a, b, ta, ts);
 }
 
 __global__ void k_batch_reset(float* __restrict__ sa, uint8_t* __restrict__ done, int32_t* __restrict__ exit_layer,
