@@ -46,6 +46,8 @@ constexpr size_t kTcSmem = size_t(kTcStages) * kStageBytes + 1024 + 256;
 // x = hi + lo with hi = bf16(x) and lo = bf16(x - hi); rows of skipped frames are left alone.
 __global__ void k_split_bf16(const float* __restrict__ src, const uint8_t* __restrict__ skip, int rows, int D,
                              __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+    chain_wait();
+    chain_release();
     const long long total = (long long)rows * D;
     for (long long i = (blockIdx.x * (long long)blockDim.x + threadIdx.x) * 4; i < total;
          i += (long long)gridDim.x * blockDim.x * 4) {
@@ -148,6 +150,8 @@ k_score_tc(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_acc = *tmem_slot;
+    chain_wait();  // barriers and tensor memory are set up while the previous kernel finishes
+    chain_release();
 
     bool failed = false;
     int issued = 0;
@@ -330,12 +334,14 @@ cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const
     if (!sv_split_done) {
         ++*launches;
         const int grid_a = int(std::min<long long>(((long long)B * D / 4 + 255) / 256, 148 * 8));
-        k_split_bf16<<<grid_a, 256, 0, st>>>(sv, skip, B, D, a_hi, a_lo);
+        const cudaError_t e = launch_chained(k_split_bf16, grid_a, 256, 0, st, sv, skip, B, D, a_hi, a_lo);
+        if (e != cudaSuccess) return e;
     }
     if (!centers_split_done) {
         ++*launches;
         const int grid_b = int(std::min<long long>(((long long)n * D / 4 + 255) / 256, 148 * 8));
-        k_split_bf16<<<grid_b, 256, 0, st>>>(centers, nullptr, n, D, b_hi, b_lo);
+        const cudaError_t e = launch_chained(k_split_bf16, grid_b, 256, 0, st, centers, static_cast<const uint8_t*>(nullptr), n, D, b_hi, b_lo);
+        if (e != cudaSuccess) return e;
     }
     ++*launches;
     TcParams p{};
@@ -346,8 +352,7 @@ cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const
     p.out = dots;
     p.status = status;
     const dim3 grid((n + kTileN - 1) / kTileN, (B + kTileM - 1) / kTileM);
-    k_score_tc<<<grid, kTcThreads, kTcSmem, st>>>(ma_hi, ma_lo, mb_hi, mb_lo, p);
-    return cudaGetLastError();
+    return launch_chained(k_score_tc, grid, kTcThreads, kTcSmem, st, ma_hi, ma_lo, mb_hi, mb_lo, p);
 }
 
 }  // namespace smtm
