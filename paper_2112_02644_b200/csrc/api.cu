@@ -204,12 +204,12 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     SMTM_CUDA(launch_encode(e2, c->sm_count, st, &c->launches, &sv_split));
     if (timing) SMTM_CUDA(record_timing(timing[1], st));
     if (dense) {
-        float* dots = nullptr;
+        float *dots = nullptr, *dots2 = nullptr;
         SMTM_CUDA(launch_dense_dots(a.sv, a.fresh ? nullptr : a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max,
-                                    sv_split, c->d_cen_split[layer], c->cen_split_current[layer], &dots, c->d_status,
+                                    sv_split, c->d_cen_split[layer], c->cen_split_current[layer], &dots, &dots2, c->d_status,
                                     st, &c->launches));
         c->cen_split_current[layer] = true;
-        SMTM_CUDA(launch_finish_dense(a, dots, st, &c->launches));
+        SMTM_CUDA(launch_finish_dense(a, dots, dots2, st, &c->launches));
         return SMTM_OK;
     }
     SMTM_CUDA(launch_score_exit(a, st, &c->launches));

@@ -107,11 +107,13 @@ size_t dense_scratch_bytes(int max_batch, int n, int d_max);
 void dense_sv_split(void* scratch, int max_batch, int d_max, void** hi, void** lo);
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
                               void* scratch, int max_batch, int d_max, bool sv_split_done, void* centers_split,
-                              bool centers_split_done, float** dots_out, int* status, cudaStream_t st,
+                              bool centers_split_done, float** dots_out, float** dots2_out, int* status, cudaStream_t st,
                               int64_t* launches);
 size_t dense_centers_split_bytes(int n, int D);
-// Eq. 1 from the dot products, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule; dots: [B][n].
-cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, cudaStream_t st, int64_t* launches);
+// Eq. 1 from the dot products, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule; dots: [B][n], and dots2
+// (nullptr, or [B][n]: the second half of the vector length, added to the first).
+cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, cudaStream_t st,
+                                int64_t* launches);
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,
                                cudaStream_t st, int64_t* launches);
 

@@ -108,7 +108,8 @@ __device__ __forceinline__ Top2 block_top2_keys(unsigned long long b1, unsigned 
     return t;
 }
 
-__global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, const float* __restrict__ dots) {
+__global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, const float* __restrict__ dots,
+                                                           const float* __restrict__ dots2) {
     __shared__ float scratch[32];
     __shared__ unsigned long long s_keys[2 * (kThreads / kWarp)];
     chain_wait();
@@ -122,6 +123,7 @@ __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, c
     const float* row = a.sv + (size_t)b * a.D;
     const float weight = float(1u << a.layer);
     const float* __restrict__ drow = dots + (size_t)b * a.n;
+    const float* __restrict__ drow2 = dots2 ? dots2 + (size_t)b * a.n : nullptr;  // second half of the vector length
     const float* __restrict__ clen = a.cnorm;
     float* sa_row = a.sa + (size_t)b * a.k_max;
     unsigned long long a1 = 0ull, a2 = 0ull, c1 = 0ull, c2 = 0ull;  // best two cumulative / single-layer keys
@@ -138,6 +140,7 @@ __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, c
         for (int u = 0; u < 4; ++u) {
             const int j = j0 + u * kThreads + tid;
             dot[u] = drow[cls[u]];
+            if (drow2) dot[u] += drow2[cls[u]];
             cl[u] = clen[cls[u]];
             old[u] = (j < k && !a.fresh) ? sa_row[j] : 0.f;
         }
@@ -191,10 +194,11 @@ cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, in
     return launch_chained(k_batch_reset, grid, 256, 0, st, sa, done, exit_layer, pred, B, n_sa);
 }
 
-cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, cudaStream_t st, int64_t* launches) {
+cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, cudaStream_t st,
+                                int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
     ++*launches;
-    return launch_chained(k_finish_dense, a.B, kThreads, 0, st, a, dots);
+    return launch_chained(k_finish_dense, a.B, kThreads, 0, st, a, dots, dots2);
 }
 
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches) {

@@ -7,14 +7,19 @@
 // memory; the dropped lo*lo term is 2^-18 relative.  One k-block therefore loads four tiles
 // (A_hi, A_lo, B_hi, B_lo) and issues three groups of MMAs on them.  The tensor core truncates
 // when it adds into its fp32 accumulator, an error that grows with the number of additions, so
-// the long hi*hi sum is cut into four runs of k-blocks with an accumulator each and the two
-// small cross terms share a fifth; the epilogue adds the five in fp32 with rounding.
+// the long hi*hi sum is cut into three runs of k-blocks with an accumulator each and the two
+// small cross terms share a fourth; the epilogue adds the four in fp32 with rounding.
 //
-// Kernel.  One CTA per 128 x 64 tile of DOT (frames x classes).  Warp 0 is the TMA producer
-// (cp.async.bulk.tensor, 128-byte swizzle, four stages of 48 KB), warp 1 allocates tensor
-// memory and issues tcgen05.mma (M = 128, N = 64, K = 16, kind::f16 with bf16 inputs), warps
-// 2..5 read the accumulator back with tcgen05.ld and store it.  Rows and classes beyond the
-// problem are zero-filled by TMA and dropped by the epilogue.  Every mbarrier wait is bounded.
+// Kernel.  One CTA per 128 x 128 tile of DOT (frames x classes) and half of the vector length:
+// with N = 128 an MMA reads as many bytes of shared memory per cycle as it can use (with N = 64
+// the 128 x 16 slice of A was re-read for half the work and the instruction was operand-bound),
+// and cutting the length in two keeps 128 CTAs busy on the 1024 x 1000 problem.  The two halves
+// go to two result arrays that the finishing kernel adds in a fixed order.  Warp 0 is the TMA
+// producer (cp.async.bulk.tensor, 128-byte swizzle, three stages of 64 KB), warp 1 allocates
+// tensor memory (4 x 128 fp32 columns) and issues tcgen05.mma (M = 128, N = 128, K = 16,
+// kind::f16 with bf16 inputs), warps 2..5 read the accumulators back with tcgen05.ld and store
+// them.  Rows and classes beyond the problem are zero-filled by TMA and dropped by the
+// epilogue.  Every mbarrier wait is bounded.
 #include <cuda.h>
 
 #include <algorithm>
@@ -27,16 +32,16 @@ namespace smtm {
 namespace {
 
 constexpr int kTileM = 128;   // frames per tile = MMA M
-constexpr int kTileN = 64;    // classes per tile = MMA N
+constexpr int kTileN = 128;   // classes per tile = MMA N
 constexpr int kTileK = 64;    // bf16 elements per k-block = one 128-byte swizzled row
 constexpr int kMmaK = 16;     // K of one tcgen05.mma with 16-bit inputs
-constexpr int kTcStages = 4;
+constexpr int kTcStages = 3;
 constexpr int kBytesA = kTileM * kTileK * 2;                   // 16 KB
-constexpr int kBytesB = kTileN * kTileK * 2;                   //  8 KB
+constexpr int kBytesB = kTileN * kTileK * 2;                   // 16 KB
 constexpr int kStageBytes = 2 * kBytesA + 2 * kBytesB;         // hi and lo of both operands
 constexpr int kTcThreads = 6 * kWarp;
-constexpr int kHeadRuns = 4;                                   // accumulators the hi*hi sum is spread over
-static_assert(kHeadRuns == 4, "the epilogue adds the head runs as (0 + 1) + (2 + 3)");
+constexpr int kHeadRuns = 3;                                   // accumulators the hi*hi sum is spread over
+constexpr int kSplitK = 2;                                     // CTAs that share the vector length of a tile
 constexpr int kAccs = kHeadRuns + 1;                           // ... plus one for the cross terms
 constexpr int kTmemCols = 512;                                 // power of two >= kAccs * kTileN fp32 columns
 constexpr size_t kTcSmem = size_t(kTcStages) * kStageBytes + 1024 + 256;
@@ -113,7 +118,8 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 struct TcParams {
     int M, N, D;       // frames, classes, vector length
     int ld_out;        // floats between rows of `out`
-    float* out;        // [M][ld_out] dot products
+    float* out;        // [splits][M][ld_out] dot products over each part of the vector length
+    size_t split_stride;  // floats between the result arrays of two parts
     int* status;
 };
 
@@ -130,7 +136,10 @@ k_score_tc(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.y * kTileM, n0 = blockIdx.x * kTileN;
-    const int n_kb = (p.D + kTileK - 1) / kTileK;
+    // this CTA's share of the k-blocks
+    const int n_kb_all = (p.D + kTileK - 1) / kTileK;
+    const int kb0 = int(blockIdx.z) * n_kb_all / int(gridDim.z);
+    const int n_kb = (int(blockIdx.z) + 1) * n_kb_all / int(gridDim.z) - kb0;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kTcStages; ++s) {
@@ -164,10 +173,11 @@ k_score_tc(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__
                 if (use > 0 && !mbar_wait_bounded(&empty[s], (use - 1) & 1, p.status)) { failed = true; break; }
                 uint8_t* st = base + size_t(s) * kStageBytes;
                 mbar_expect_tx(&full[s], kStageBytes);
-                tma_load_2d(st, &map_a_hi, kb * kTileK, m0, &full[s]);
-                tma_load_2d(st + kBytesA, &map_a_lo, kb * kTileK, m0, &full[s]);
-                tma_load_2d(st + 2 * kBytesA, &map_b_hi, kb * kTileK, n0, &full[s]);
-                tma_load_2d(st + 2 * kBytesA + kBytesB, &map_b_lo, kb * kTileK, n0, &full[s]);
+                const int x = (kb0 + kb) * kTileK;  // a multiple of 64 elements = 128 bytes
+                tma_load_2d(st, &map_a_hi, x, m0, &full[s]);
+                tma_load_2d(st + kBytesA, &map_a_lo, x, m0, &full[s]);
+                tma_load_2d(st + 2 * kBytesA, &map_b_hi, x, n0, &full[s]);
+                tma_load_2d(st + 2 * kBytesA + kBytesB, &map_b_lo, x, n0, &full[s]);
                 issued = kb + 1;
             }
         }
@@ -228,16 +238,17 @@ k_score_tc(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__
                 }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (row < p.M) {
-                    float* dst = p.out + (size_t)row * p.ld_out + n0 + c0;
+                    float* dst = p.out + size_t(blockIdx.z) * p.split_stride + (size_t)row * p.ld_out + n0 + c0;
 #pragma unroll
                     for (int j = 0; j < 16; j += 4) {
                         if (n0 + c0 + j < p.N) {  // N and ld_out are multiples of 4
                             float o[4];
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
-                                const float h01 = __uint_as_float(r[0][j + e]) + __uint_as_float(r[1][j + e]);
-                                const float h23 = __uint_as_float(r[2][j + e]) + __uint_as_float(r[3][j + e]);
-                                o[e] = (h01 + h23) + __uint_as_float(r[kHeadRuns][j + e]);
+                                float h = __uint_as_float(r[0][j + e]);
+#pragma unroll
+                                for (int run = 1; run < kHeadRuns; ++run) h += __uint_as_float(r[run][j + e]);
+                                o[e] = h + __uint_as_float(r[kHeadRuns][j + e]);
                             }
                             *reinterpret_cast<float4*>(dst + j) = make_float4(o[0], o[1], o[2], o[3]);
                         }
@@ -292,12 +303,12 @@ bool make_map(CUtensorMap* map, const __nv_bfloat16* ptr, int rows, int D, int b
 }  // namespace
 
 bool dense_scoring_supported(int D, int n) {
-    return D % 8 == 0 && D >= kHeadRuns * kTileK && n % 4 == 0 && encode_tiled_fn() != nullptr;
+    return D % 8 == 0 && D >= 4 * kTileK && n % 4 == 0 && encode_tiled_fn() != nullptr;
 }
 
 size_t dense_scratch_bytes(int max_batch, int n, int d_max) {
     // bf16 heads and tails of the semantic vectors, then the dot products
-    return size_t(max_batch) * d_max * 2 * 2 + size_t(max_batch) * n * sizeof(float) + 1024;
+    return size_t(max_batch) * d_max * 2 * 2 + size_t(kSplitK) * max_batch * n * sizeof(float) + 1024;
 }
 
 size_t dense_centers_split_bytes(int n, int D) { return size_t(n) * D * 2 * 2; }
@@ -310,7 +321,7 @@ void dense_sv_split(void* scratch, int max_batch, int d_max, void** hi, void** l
 
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
                               void* scratch, int max_batch, int d_max, bool sv_split_done, void* centers_split,
-                              bool centers_split_done, float** dots_out, int* status, cudaStream_t st,
+                              bool centers_split_done, float** dots_out, float** dots2_out, int* status, cudaStream_t st,
                               int64_t* launches) {
     __nv_bfloat16* a_hi = reinterpret_cast<__nv_bfloat16*>(scratch);
     __nv_bfloat16* a_lo = a_hi + size_t(max_batch) * d_max;
@@ -318,7 +329,10 @@ cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const
     __nv_bfloat16* b_lo = b_hi + size_t(n) * D;
     float* dots = reinterpret_cast<float*>(
         (reinterpret_cast<uintptr_t>(a_lo + size_t(max_batch) * d_max) + 255) & ~uintptr_t(255));
+    // the vector length is cut in two when each part still has a k-block for every accumulator
+    const int splits = (D + kTileK - 1) / kTileK >= kSplitK * kHeadRuns ? kSplitK : 1;
     *dots_out = dots;
+    *dots2_out = splits > 1 ? dots + size_t(max_batch) * n : nullptr;
 
     CUtensorMap ma_hi, ma_lo, mb_hi, mb_lo;
     if (!make_map(&ma_hi, a_hi, B, D, kTileM) || !make_map(&ma_lo, a_lo, B, D, kTileM) ||
@@ -350,8 +364,9 @@ cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const
     p.D = D;
     p.ld_out = n;
     p.out = dots;
+    p.split_stride = size_t(max_batch) * n;
     p.status = status;
-    const dim3 grid((n + kTileN - 1) / kTileN, (B + kTileM - 1) / kTileM);
+    const dim3 grid((n + kTileN - 1) / kTileN, (B + kTileM - 1) / kTileM, splits);
     return launch_chained(k_score_tc, grid, kTcThreads, kTcSmem, st, ma_hi, ma_lo, mb_hi, mb_lo, p);
 }
 
