@@ -313,3 +313,29 @@ def test_fused_lookup_exact_ties_go_to_the_lower_class():
     ac = gb.ac.cpu().numpy()
     assert np.all(ac[tied] == 0.0)
     smtm.smtm_cache_destroy(cache)
+
+
+def test_device_clock_profile_reports_every_kernel_of_a_step():
+    # every `every`-th step carries stamps of the device's clock: each kernel of the step reports a duration
+    w = si.C5.scaled(B=64, S=64, T=3)
+    cents, counts = si.initial_centers(w)
+    cache = smtm.smtm_cache_create(w.n, w.dims, [w.tau] * w.L, cents, counts, n_streams=w.S, k_init=w.k_init,
+                                   k_min=w.k_min, k_max=w.k_max, window_W=w.window_W, max_batch=w.B)
+    gb = smtm.Batch(cache, w.B, stream_id=si.stream_ids(w))
+    labs = si.labels(w)
+    smtm.smtm_cache_profile(cache, 8, 2)          # steps 0 and 2 are profiled, step 1 is not
+    for t in range(3):
+        for l in range(w.L):
+            x = si.frames(w, l, labs[t], t, device="cuda")
+            (smtm.smtm_lookup_exit_begin if l == 0 else smtm.smtm_lookup_exit)(
+                cache, l, smtm.Fmap(x, w.dtype, w.layout, *si.shape4(w, l)), gb)
+        smtm.smtm_cache_update_resize(cache, gb, torch.from_numpy(si.fallback_labels(w, labs[t])).cuda())
+    total, count = smtm.smtm_cache_get_profile_device(cache)
+    for i in (0, 1, smtm.PROF_PLAN, smtm.PROF_CENTERS, smtm.PROF_TABLES):
+        assert count[i] == 2 and 0.0 < total[i] < 100.0, (i, count[i], total[i])   # milliseconds
+    assert count[2:smtm.MAX_LAYERS].sum() == 0
+    ev_ms, ev_n = smtm.smtm_cache_get_profile(cache, 0)
+    assert ev_n == 2 and ev_ms >= total[0] * 0.5
+    smtm.smtm_cache_profile(cache, 0, 1)
+    assert smtm.smtm_cache_get_profile_device(cache)[1].sum() == 0
+    smtm.smtm_cache_destroy(cache)
