@@ -229,7 +229,10 @@ smtm_status_t smtm_cache_resize(smtm_cache_t* cache, void* stream);
  * do_resize else smtm_cache_update, then copies the decisions back.  Synchronises
  * `stream` before returning.  h_stream_id / h_fallback_label may be NULL as in
  * the device calls; h_done [B], h_exit_layer [B], h_pred [B] receive the results.
- * B <= max_batch.  Pinned host buffers make the copies asynchronous. */
+ * B <= max_batch.  Pinned host buffers make the copies asynchronous.  After the
+ * first layer only the maps of the frames that have not exited are copied (the
+ * call reads the exit flags back between layers), so the bytes moved follow the
+ * exits: sum over layers l of the frames still in at l times the frame's size. */
 smtm_status_t smtm_step_host(smtm_cache_t* cache, const smtm_fmap_t* fmaps, const void* const* h_maps,
                              const int32_t* h_stream_id, const int32_t* h_fallback_label,
                              int32_t do_resize, uint8_t* h_done, int32_t* h_exit_layer,

@@ -45,6 +45,7 @@ struct smtm_cache {
     smtm_batch_t hb;
     int32_t* d_stream_id;
     int32_t* d_fallback;
+    uint8_t* h_flags;   // pinned host copy of the exit flags between two layers of smtm_step_host
     void* d_stage[SMTM_MAX_LAYERS];
     size_t stage_bytes[SMTM_MAX_LAYERS];
 };
@@ -112,6 +113,7 @@ void free_all(smtm_cache* c) {
     cudaFree(c->hb.d_pred);
     cudaFree(c->d_stream_id);
     cudaFree(c->d_fallback);
+    cudaFreeHost(c->h_flags);
     delete c;
 }
 
@@ -529,6 +531,7 @@ smtm_status_t smtm_step_host(smtm_cache_t* c, const smtm_fmap_t* fmaps, const vo
         ok = ok && dev_alloc(&c->hb.d_pred, mb) == cudaSuccess;
         ok = ok && dev_alloc(&c->d_stream_id, mb) == cudaSuccess;
         ok = ok && dev_alloc(&c->d_fallback, mb) == cudaSuccess;
+        ok = ok && cudaMallocHost(reinterpret_cast<void**>(&c->h_flags), mb) == cudaSuccess;
         for (int l = 0; ok && l < c->L; ++l) ok = dev_alloc(&c->hb.d_sv[l], mb * c->dims[l]) == cudaSuccess;
         if (!ok) {
             (void)cudaGetLastError();
@@ -564,8 +567,27 @@ smtm_status_t smtm_step_host(smtm_cache_t* c, const smtm_fmap_t* fmaps, const vo
         SMTM_CUDA(cudaMemcpyAsync(c->d_fallback, h_fallback_label, size_t(B) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     for (int l = 0; l < c->L; ++l) {
         smtm_fmap_t f = fmaps[l];
-        const size_t bytes = size_t(B) * f.C * f.H * f.W * (f.dtype == SMTM_F32 ? 4 : 2);
-        SMTM_CUDA(cudaMemcpyAsync(c->d_stage[l], h_maps[l], bytes, cudaMemcpyHostToDevice, st));
+        const size_t frame_bytes = size_t(f.C) * f.H * f.W * (f.dtype == SMTM_F32 ? 4 : 2);
+        if (l == 0) {
+            SMTM_CUDA(cudaMemcpyAsync(c->d_stage[l], h_maps[l], size_t(B) * frame_bytes, cudaMemcpyHostToDevice, st));
+        } else {
+            // A frame that has exited needs nothing of the later layers: only the maps of the frames
+            // that are still in cross the bus, one copy per run of consecutive frames.
+            SMTM_CUDA(cudaMemcpyAsync(c->h_flags, b.d_done, size_t(B), cudaMemcpyDeviceToHost, st));
+            SMTM_CUDA(cudaStreamSynchronize(st));
+            for (int b0 = 0; b0 < B;) {
+                if (c->h_flags[b0]) {
+                    ++b0;
+                    continue;
+                }
+                int b1 = b0 + 1;
+                while (b1 < B && !c->h_flags[b1]) ++b1;
+                SMTM_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(c->d_stage[l]) + size_t(b0) * frame_bytes,
+                                          static_cast<const uint8_t*>(h_maps[l]) + size_t(b0) * frame_bytes,
+                                          size_t(b1 - b0) * frame_bytes, cudaMemcpyHostToDevice, st));
+                b0 = b1;
+            }
+        }
         f.d_data = c->d_stage[l];
         smtm_status_t s = lookup_impl(c, l, &f, &b, st, l == 0);
         if (s != SMTM_OK) return s;
