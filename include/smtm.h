@@ -72,7 +72,16 @@ enum {
  * FT is then fixed point with 10 fractional bits (smtm_cache_get_tables returns it raw): an
  * appearance adds 1024, each further W consecutive unseen frames multiply it by 0.25 rounding
  * down, and Eq. 5's score is FT itself. */
-enum { SMTM_FLAG_FORGET_FT = 1 };
+enum { SMTM_FLAG_FORGET_FT = 1, SMTM_FLAG_MAPS_READY = 2 };
+/* SMTM_FLAG_MAPS_READY is a promise of the caller that lets smtm_lookup_exit_begin start reading
+ * feature maps while the library's previous kernel on the stream (the end of the previous
+ * step's update) is still running: (1) the maps given to smtm_lookup_exit_begin are complete in
+ * memory when the call is enqueued, i.e. they are not written by earlier work on the same
+ * stream; (2) consecutive batches use different smtm_batch_t carries (two that alternate are
+ * enough), because the call writes its batch's d_sv[layer] while the previous batch's update
+ * may still read its own.  Everything that depends on the memory (members, centres) and every
+ * other output still waits for the previous kernel.  Without the flag nothing is touched
+ * before the previous kernel is complete. */
 
 typedef struct {
     int32_t n_classes;      /* n: classes in global memory (Sec. 6), 1..SMTM_MAX_CLASSES */
@@ -85,7 +94,7 @@ typedef struct {
     int32_t window_W;       /* W of Eq. 5, >= 1 */
     int32_t cl_num, cl_den; /* confidence level of Eq. 6 as a fraction, e.g. 19/20 */
     int32_t max_batch;      /* largest B any call will pass; sizes the library's scratch */
-    uint32_t flags;         /* 0 or SMTM_FLAG_FORGET_FT */
+    uint32_t flags;         /* 0 or an OR of SMTM_FLAG_FORGET_FT, SMTM_FLAG_MAPS_READY */
 } smtm_config_t;
 
 /* A batch of feature maps at one exit layer: dense, frame stride C*H*W elements,

@@ -19,6 +19,7 @@ F32, F16, BF16 = 0, 1, 2
 NCHW, NHWC = 0, 1
 MAX_LAYERS = 16
 FLAG_FORGET_FT = 1   # the frequency table itself forgets (fixed point, 10 fractional bits)
+FLAG_MAPS_READY = 2  # the first lookup of a batch may read its maps while the previous update finishes (see smtm.h)
 CTR_EXITS, CTR_NEAR, CTR_LOOKUPS, CTR_COUNT = 0, MAX_LAYERS, MAX_LAYERS + 1, MAX_LAYERS + 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))

@@ -10,6 +10,7 @@ using namespace smtm;
 struct smtm_cache {
     int n, L, S, k_init, k_min, k_max, W, cl_num, cl_den, max_batch;
     bool forgetting;    // SMTM_FLAG_FORGET_FT
+    bool maps_ready;    // SMTM_FLAG_MAPS_READY
     int dims[SMTM_MAX_LAYERS];
     float tau[SMTM_MAX_LAYERS];
     float* d_centers[SMTM_MAX_LAYERS];
@@ -151,9 +152,10 @@ EncodeArgs encode_args(const smtm_cache* c, const smtm_fmap_t* f, const uint8_t*
 }
 
 smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b,
-                          cudaStream_t st, bool begin) {
+                          cudaStream_t st, bool begin, bool allow_early = true) {
     LookupArgs a{};
     a.fresh = begin ? 1 : 0;
+    a.early = (begin && c->maps_ready && allow_early) ? 1 : 0;
     a.layer = layer;
     a.L = c->L;
     a.B = f->B;
@@ -295,7 +297,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     if (!cfg || !h_centers || !out || !cfg->dims || !cfg->tau) return SMTM_ERR_INVALID_ARG;
     if (cfg->n_classes < 1 || cfg->n_classes > SMTM_MAX_CLASSES) return SMTM_ERR_INVALID_ARG;
     if (cfg->n_layers < 1 || cfg->n_layers > SMTM_MAX_LAYERS) return SMTM_ERR_INVALID_ARG;
-    if (cfg->n_streams < 1 || cfg->max_batch < 1 || (cfg->flags & ~uint32_t(SMTM_FLAG_FORGET_FT)) != 0)
+    if (cfg->n_streams < 1 || cfg->max_batch < 1 || (cfg->flags & ~uint32_t(SMTM_FLAG_FORGET_FT | SMTM_FLAG_MAPS_READY)) != 0)
         return SMTM_ERR_INVALID_ARG;
     if (cfg->k_min < 1 || cfg->k_min > cfg->k_init || cfg->k_init > cfg->k_max || cfg->k_max > cfg->n_classes)
         return SMTM_ERR_INVALID_ARG;
@@ -324,6 +326,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     c->cl_den = cfg->cl_den;
     c->max_batch = cfg->max_batch;
     c->forgetting = (cfg->flags & SMTM_FLAG_FORGET_FT) != 0;
+    c->maps_ready = (cfg->flags & SMTM_FLAG_MAPS_READY) != 0;
     for (int l = 0; l < c->L; ++l) {
         c->dims[l] = cfg->dims[l];
         c->tau[l] = cfg->tau[l];
@@ -589,7 +592,7 @@ smtm_status_t smtm_step_host(smtm_cache_t* c, const smtm_fmap_t* fmaps, const vo
             }
         }
         f.d_data = c->d_stage[l];
-        smtm_status_t s = lookup_impl(c, l, &f, &b, st, l == 0);
+        smtm_status_t s = lookup_impl(c, l, &f, &b, st, l == 0, false);  // one carry, staged maps: no early start
         if (s != SMTM_OK) return s;
     }
     smtm_status_t s = update_impl(c, &b, h_fallback_label ? c->d_fallback : nullptr, do_resize != 0, st);

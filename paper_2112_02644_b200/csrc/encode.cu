@@ -375,8 +375,15 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         const long long u = (long long)cluster + (long long)idx * n_clusters;
         if (u < a.B) my_units[idx] = int(u);
     }
-    chain_wait();  // everything above touched shared memory only and overlaps the previous kernel's tail
-    chain_release();
+    // Everything above touched shared memory only and overlaps the previous kernel's tail.  With
+    // a.early the producer and the reducers go on without waiting (they read the caller's maps and
+    // write this batch's SV stash, which the previous kernel does not touch); the dot warps and
+    // the finisher, which read the memory and write the carry, wait on their own.
+    const bool early = a.fresh && a.early;
+    if (!early) {
+        chain_wait();
+        chain_release();
+    }
     const ClockScope stamps(a.clock ? a.clock + 2 * a.layer : nullptr);  // profiling
     for (int t0 = 0; !a.fresh && t0 < a.B; t0 += kThreadsFused) {
         const int b = t0 + threadIdx.x;
@@ -448,6 +455,10 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
     } else if (warp <= kReducersF + kDotWarps) {
         // ---- dot warps: all of them work on frame u together, slot j on warp j % kDotWarps -------
         const int dw = warp - kReducersF - 1;
+        if (early) {
+            chain_wait();
+            if (dw == 0 && lane == 0) chain_release();
+        }
         const int sb = rank * f.slice_cap;          // first channel of this CTA's slice
         const int Dp = max(0, min(f.slice_cap, p.C - sb));  // channels in it (a multiple of 4)
         const int n4 = Dp >> 2;
@@ -550,6 +561,7 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         }
     } else {
         // ---- finisher warp: every P-th frame of the cluster; lane l looks after slots l and l + 32 ----
+        if (early) chain_wait();
         const float weight = float(1u << a.layer);  // 2^(l-1) with l = layer + 1
         const int reuse = max(P, kRx);              // frames between two uses of a receive buffer in this CTA
         for (int u = rank; u < nu; u += P) {

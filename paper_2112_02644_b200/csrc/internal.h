@@ -72,6 +72,7 @@ cudaError_t launch_row_norm2(const float* sv, const uint8_t* skip, int B, int D,
 // ---- lookup (Sec. 4.2, Sec. 5) -------------------------------------------------------------
 struct LookupArgs {
     int layer, L, B, D, n, k_max;
+    int early;                // (fused route, with fresh) the maps may be read and the SV stash written before the previous kernel is complete
     int fresh;                // the batch starts here: the carry is taken as SA = 0, nobody done, and is overwritten
     float tau;
     const float* sv;          // [B][D]

@@ -467,13 +467,17 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, cudaStream_
     ++*launches;
     e = launch_chained(k_update_plan, (a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st, a);
     if (e != cudaSuccess) return e;
+    // tables before centres: the next step's streaming kernel may overlap the last kernel of the update, and the
+    // centres' is the longer one
+    if (a.warm_layer < 0) {  // a warm-up batch has no streams
+        const int table_ctas = warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
+        ++*launches;
+        e = launch_chained(k_update_tables, table_ctas, kUpdThreads, smem, st, a, rz ? *rz : ResizeArgs{}, rz ? 1 : 0,
+                           warp_tables ? 1 : 0);
+        if (e != cudaSuccess) return e;
+    }
     ++*launches;
-    e = launch_chained(k_update_centers, a.B * (a.warm_layer >= 0 ? 1 : a.L), kUpdThreads, 0, st, a);
-    if (e != cudaSuccess || a.warm_layer >= 0) return e;  // a warm-up batch has no streams
-    const int table_ctas = warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
-    ++*launches;
-    return launch_chained(k_update_tables, table_ctas, kUpdThreads, smem, st, a, rz ? *rz : ResizeArgs{}, rz ? 1 : 0,
-                          warp_tables ? 1 : 0);
+    return launch_chained(k_update_centers, a.B * (a.warm_layer >= 0 ? 1 : a.L), kUpdThreads, 0, st, a);
 }
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {

@@ -37,7 +37,7 @@ def test_null_and_out_of_range_arguments_are_rejected_before_any_device_work():
     cen = np.zeros((4, 8), np.float32)
     cen_p = (ctypes.c_void_p * 1)(cen.ctypes.data)
     bad = [dict(n_classes=0), dict(n_layers=17), dict(k_max=5), dict(k_min=0), dict(k_init=9),
-           dict(window_W=0), dict(cl_num=21), dict(max_batch=0), dict(flags=2), dict(n_streams=0)]
+           dict(window_W=0), dict(cl_num=21), dict(max_batch=0), dict(flags=4), dict(n_streams=0)]
     for kw in bad:
         f = dict(n_classes=4, n_layers=1, dims=dims, tau=tau, n_streams=1, k_init=2, k_min=2, k_max=4,
                  window_W=16, cl_num=19, cl_den=20, max_batch=8, flags=0)

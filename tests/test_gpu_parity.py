@@ -339,3 +339,42 @@ def test_device_clock_profile_reports_every_kernel_of_a_step():
     smtm.smtm_cache_profile(cache, 0, 1)
     assert smtm.smtm_cache_get_profile_device(cache)[1].sum() == 0
     smtm.smtm_cache_destroy(cache)
+
+
+def test_maps_ready_flag_with_alternating_batches():
+    # SMTM_FLAG_MAPS_READY: the first lookup of a step may read its maps and write its batch's SV stash while the
+    # previous step's update is still running; the caller alternates two carries.  Results are those of the oracle.
+    from harness import Report, compare_state, step_pair
+
+    w = si.C5.scaled(B=96, S=96, T=6)
+    cents, counts = si.initial_centers(w)
+    tau = [w.tau] * w.L
+    mem = oracle.OracleMemory(w.n, w.dims, tau, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W)
+    cache = smtm.smtm_cache_create(w.n, w.dims, tau, cents, counts, n_streams=w.S, k_init=w.k_init, k_min=w.k_min,
+                                   k_max=w.k_max, window_W=w.window_W, max_batch=w.B, flags=smtm.FLAG_MAPS_READY)
+    sid = si.stream_ids(w)
+    gbs = [smtm.Batch(cache, w.B, stream_id=sid), smtm.Batch(cache, w.B, stream_id=sid)]
+    labs = si.labels(w)
+    rep = Report()
+    for t in range(w.T):
+        step_pair(w, cache, mem, gbs[t % 2], labs[t], t, rep)
+    compare_state(w, cache, mem, rep)
+    # back to back without the harness's synchronisation in between: steps overlap on the device
+    maps = [[si.frames(w, l, labs[t], t, device="cuda") for l in range(w.L)] for t in range(w.T)]
+    torch.cuda.synchronize()
+    for t in range(w.T):
+        gb = gbs[t % 2]
+        smtm.smtm_lookup_exit_begin(cache, 0, smtm.Fmap(maps[t][0], w.dtype, w.layout, *si.shape4(w, 0)), gb)
+        smtm.smtm_lookup_exit(cache, 1, smtm.Fmap(maps[t][1], w.dtype, w.layout, *si.shape4(w, 1)), gb)
+        smtm.smtm_cache_update_resize(cache, gb, torch.from_numpy(si.fallback_labels(w, labs[t])).cuda())
+    for t in range(w.T):
+        ob = mem.new_batch(w.B, sid)
+        for l in range(w.L):
+            mem.lookup_exit(l, maps[t][l].cpu(), w.dtype, w.layout, si.shape4(w, l), ob)
+        mem.update(ob, si.fallback_labels(w, labs[t]))
+        mem.resize()
+    torch.cuda.synchronize()
+    assert np.array_equal(gbs[(w.T - 1) % 2].done.cpu().numpy(), ob["done"])
+    assert np.array_equal(gbs[(w.T - 1) % 2].pred.cpu().numpy(), ob["pred"])
+    compare_state(w, cache, mem, rep)
+    smtm.smtm_cache_destroy(cache)
