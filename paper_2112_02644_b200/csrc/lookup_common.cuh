@@ -55,33 +55,6 @@ __device__ __forceinline__ float ratio_margin(float top, float second) {
 __device__ __forceinline__ void decide_from_top2(const LookupArgs& a, int b, const Top2& ta, const Top2& ts);
 __device__ __forceinline__ float cosine_from(float dot, float sv_norm2, float center_len);
 
-// Butterfly merge of per-lane pairs: every lane ends up with the warp's best two.
-__device__ __forceinline__ Top2 warp_top2_merge(Top2 t) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float ov1 = __shfl_xor_sync(kFull, t.v1, o), ov2 = __shfl_xor_sync(kFull, t.v2, o);
-        const int oi1 = __shfl_xor_sync(kFull, t.id1, o), oi2 = __shfl_xor_sync(kFull, t.id2, o);
-        if (oi1 >= 0) top2_push(t, ov1, oi1);
-        if (oi2 >= 0) top2_push(t, ov2, oi2);
-    }
-    return t;
-}
-
-// Best two of values held in registers: lane l holds slots l and l + 32 (v[0], v[1]) of k.
-__device__ __forceinline__ Top2 warp_top2_regs(const float (&v)[2], const int (&ids)[2], int k, int lane) {
-    Top2 t{0.f, 0.f, -1, -1};
-    if (lane < k) top2_push(t, v[0], ids[0]);
-    if (lane + kWarp < k) top2_push(t, v[1], ids[1]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float ov1 = __shfl_xor_sync(kFull, t.v1, o), ov2 = __shfl_xor_sync(kFull, t.v2, o);
-        const int oi1 = __shfl_xor_sync(kFull, t.id1, o), oi2 = __shfl_xor_sync(kFull, t.id2, o);
-        if (oi1 >= 0) top2_push(t, ov1, oi1);
-        if (oi2 >= 0) top2_push(t, ov2, oi2);
-    }
-    return t;
-}
-
 // ---- top-2 through one 64-bit key per entry ------------------------------------------------------
 //
 // The ranking (NaN last, larger value first, ties -> lower class id) as an unsigned comparison:
@@ -117,7 +90,8 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 }
 
 // Best two of values held in registers (lane l holds slots l and l + 32 of k), by two warp-wide
-// maxima over the keys: the same result as warp_top2_regs in a fraction of the instructions.
+// maxima over the keys: the same result as pushing every entry through top2_push and merging by
+// shuffles, in a fraction of the instructions.
 __device__ __forceinline__ Top2 warp_top2_keys(const float (&v)[2], const int (&ids)[2], int k, int lane) {
     const unsigned long long e0 = lane < k ? rank_key(v[0], ids[0]) : 0ull;
     const unsigned long long e1 = lane + kWarp < k ? rank_key(v[1], ids[1]) : 0ull;
