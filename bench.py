@@ -155,7 +155,7 @@ def run_ours(args):
     base = si.WORKLOADS[[k for k in si.WORKLOADS if k.startswith(args.workload)][0]]
     w = shard_for_rank(base, rank)
     K, W = args.steps, args.warmup
-    G = math.gcd(K, 8)          # steps captured into one CUDA graph
+    G = math.gcd(K, 32)         # steps captured into one CUDA graph
     m = G if G % 2 == 0 else 2 * G   # resident steps: a whole number of graphs, and even (two carries alternate)
     T = min(w.T, max(K, W, m))
     T = max(m, T - T % m)
