@@ -156,6 +156,8 @@ def run_ours(args):
     w = shard_for_rank(base, rank)
     K, W = args.steps, args.warmup
     G = math.gcd(K, 32)         # steps captured into one CUDA graph
+    while G > 1 and G > w.T:    # not more than the workload has
+        G //= 2
     m = G if G % 2 == 0 else 2 * G   # resident steps: a whole number of graphs, and even (two carries alternate)
     T = min(w.T, max(K, W, m))
     T = max(m, T - T % m)

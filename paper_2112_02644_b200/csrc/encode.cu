@@ -118,7 +118,10 @@ struct UnitPerLane {
     }
 };
 
-// T lanes per channel; channel bytes are a multiple of 16.
+// T lanes per channel; channel bytes are a multiple of 16.  Two passes (channels per team) are
+// folded at a time, one accumulator per element of a vector and two vectors of each in
+// flight: a single warp has to keep up with the copies, so the loop must not be one chain of
+// dependent additions.
 template <class E>
 struct TeamPerChannel {
     static __device__ __forceinline__ void run(const uint8_t* stage, int nch, int lane, float* out, float* out_s,
@@ -127,32 +130,60 @@ struct TeamPerChannel {
         const int per_pass = kWarp / T;
         const int team = lane / T, r = lane - team * T;
         const int passes = (nch + per_pass - 1) / per_pass;
-        for (int ps = 0; ps < passes; ++ps) {
-            const int c = ps * per_pass + team;
-            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-            if (c < nch) {
-                const uint4* u = reinterpret_cast<const uint4*>(stage) + size_t(c) * uw;
-                for (int i = r; i < uw; i += T) {
-                    const uint4 v = u[i];
-                    if (E::kPerVec == 4) {
-                        a0 += E::at(v, 0); a1 += E::at(v, 1); a2 += E::at(v, 2); a3 += E::at(v, 3);
-                    } else {
-                        a0 += E::at(v, 0); a1 += E::at(v, 1); a2 += E::at(v, 2); a3 += E::at(v, 3);
-                        a0 += E::at(v, 4); a1 += E::at(v, 5); a2 += E::at(v, 6); a3 += E::at(v, 7);
-                    }
+        for (int ps = 0; ps < passes; ps += 2) {
+            const int c0 = ps * per_pass + team, c1 = c0 + per_pass;  // this team's channels of the two passes
+            // a channel past the end is read as the chunk's last one and dropped afterwards
+            const uint4* u0 = reinterpret_cast<const uint4*>(stage) + size_t(min(c0, nch - 1)) * uw;
+            const uint4* u1 = reinterpret_cast<const uint4*>(stage) + size_t(min(c1, nch - 1)) * uw;
+            float a[2][E::kPerVec];
+#pragma unroll
+            for (int j = 0; j < E::kPerVec; ++j) a[0][j] = a[1][j] = 0.f;
+            int i = r;
+            for (; i + T < uw; i += 2 * T) {
+                const uint4 v00 = u0[i], v01 = u0[i + T], v10 = u1[i], v11 = u1[i + T];
+#pragma unroll
+                for (int j = 0; j < E::kPerVec; ++j) {
+                    a[0][j] += E::at(v00, j);
+                    a[1][j] += E::at(v10, j);
+                }
+#pragma unroll
+                for (int j = 0; j < E::kPerVec; ++j) {
+                    a[0][j] += E::at(v01, j);
+                    a[1][j] += E::at(v11, j);
                 }
             }
-            float s = (a0 + a1) + (a2 + a3);
-            for (int o = T >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(kFull, s, o);
-            if (c < nch && r == 0) {
-                const float v = s * inv_hw;
-                out[c] = v;
-                if (out_s) out_s[c] = v;
-                if (p.sv_hi) {
-                    const ptrdiff_t at = (out + c) - p.sv;
-                    const __nv_bfloat16 h = __float2bfloat16_rn(v);
-                    p.sv_hi[at] = h;
-                    p.sv_lo[at] = __float2bfloat16_rn(v - __bfloat162float(h));
+            for (; i < uw; i += T) {
+                const uint4 v0 = u0[i], v1 = u1[i];
+#pragma unroll
+                for (int j = 0; j < E::kPerVec; ++j) {
+                    a[0][j] += E::at(v0, j);
+                    a[1][j] += E::at(v1, j);
+                }
+            }
+            float s[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                s[h] = (a[h][0] + a[h][1]) + (a[h][2] + a[h][3]);
+                if (E::kPerVec == 8)
+                    s[h] += (a[h][4 % E::kPerVec] + a[h][5 % E::kPerVec]) + (a[h][6 % E::kPerVec] + a[h][7 % E::kPerVec]);
+            }
+            for (int o = T >> 1; o > 0; o >>= 1) {
+                s[0] += __shfl_xor_sync(kFull, s[0], o);
+                s[1] += __shfl_xor_sync(kFull, s[1], o);
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int c = h ? c1 : c0;
+                if (c < nch && r == 0) {
+                    const float v = s[h] * inv_hw;
+                    out[c] = v;
+                    if (out_s) out_s[c] = v;
+                    if (p.sv_hi) {
+                        const ptrdiff_t at = (out + c) - p.sv;
+                        const __nv_bfloat16 hh = __float2bfloat16_rn(v);
+                        p.sv_hi[at] = hh;
+                        p.sv_lo[at] = __float2bfloat16_rn(v - __bfloat162float(hh));
+                    }
                 }
             }
         }
