@@ -29,7 +29,7 @@ struct smtm_cache {
     int d_max;          // largest C_l
     int32_t* d_plan;    // scratch of the update: final label and stop layer, 2 x [max_batch]
     unsigned long long* d_tags;  // scratch of the update: election tags, [n] + [S]
-    unsigned long long epoch;    // update calls so far
+    unsigned long long* d_epoch; // [2] device: update calls so far, and the plan kernel's ticket
     // optional timing of the streaming kernel of every lookup (smtm_cache_profile)
     std::vector<cudaEvent_t>* prof_events;  // pairs, in launch order
     std::vector<int>* prof_layer;           // layer of each pair
@@ -108,6 +108,7 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_warm_sv);
     cudaFree(c->d_dense);
     cudaFree(c->d_tags);
+    cudaFree(c->d_epoch);
     cudaFree(c->hb.d_sa);
     cudaFree(c->hb.d_done);
     cudaFree(c->hb.d_exit_layer);
@@ -251,7 +252,7 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     a.plan.stop_layer = c->d_plan + mb;
     a.plan.class_tag = c->d_tags;
     a.plan.stream_tag = c->d_tags + c->n;
-    a.plan.epoch = ++c->epoch;
+    a.plan.epoch = c->d_epoch;
     a.stream_id = b->d_stream_id;
     a.done = b->d_done;
     a.exit_layer = b->d_exit_layer;
@@ -365,6 +366,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
             ok = cudaMalloc(&c->d_cen_split[l], dense_centers_split_bytes(n, c->dims[l])) == cudaSuccess;
     }
     ok = ok && dev_alloc(&c->d_tags, size_t(n) + size_t(S)) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_epoch, 2) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();
         free_all(c);
@@ -393,6 +395,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     if (e == cudaSuccess) e = cudaMemset(c->d_counters, 0, SMTM_CTR_COUNT * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->d_tags, 0, (size_t(n) + size_t(S)) * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(c->d_epoch, 0, 2 * sizeof(unsigned long long));
     if (e == cudaSuccess)
         e = cudaMemcpy(c->d_members, members.data(), members.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(c->d_k, ks.data(), ks.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
@@ -493,7 +496,7 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
     a.plan.stop_layer = c->d_plan + mb;
     a.plan.class_tag = c->d_tags;
     a.plan.stream_tag = c->d_tags + c->n;
-    a.plan.epoch = ++c->epoch;
+    a.plan.epoch = c->d_epoch;
     a.fallback = d_labels;
     a.ft = c->d_ft;
     a.ts = c->d_ts;

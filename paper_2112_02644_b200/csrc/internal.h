@@ -128,7 +128,9 @@ struct UpdatePlan {
     int32_t* stop_layer;             // [max_batch] the paper's l at which its inference stopped
     unsigned long long* class_tag;   // [n] election of the first frame of each class, see memory.cu
     unsigned long long* stream_tag;  // [S] election of the first frame of each stream
-    unsigned long long epoch;        // sequence number of this update call (>= 1)
+    unsigned long long* epoch;       // [2] device: [0] number of update calls completed so far, [1] CTAs of the plan
+                                     // kernel that are through (zero between calls).  The number lives on the
+                                     // device so that a replayed CUDA graph counts on like eager calls do.
 };
 
 struct UpdateArgs {

@@ -8,7 +8,8 @@
 // An update is three launches.  k_update_plan writes every frame's final label and stop layer
 // and elects, per class and per stream present in the batch, its first frame (an integer
 // atomicMax on a tag that carries the call's sequence number, so the election tables never
-// need clearing).  In k_update_centers every (frame, layer) CTA (Eq. 7) and in k_update_tables
+// need clearing; the number is kept on the device and moved on by the plan kernel itself, so
+// that a replayed CUDA graph counts on exactly like eager calls).  In k_update_centers every (frame, layer) CTA (Eq. 7) and in k_update_tables
 // every frame's warp (tables, optionally followed by its stream's Eq. 5 / Eq. 6 refresh)
 // first checks whether its frame was elected and leaves at once if not; classes and streams
 // the batch does not touch cost nothing.  The two are separate kernels because the tables
@@ -60,15 +61,23 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a)
     chain_release();
     const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_PLAN : nullptr);
     const int b = blockIdx.x * kUpdThreads + threadIdx.x;
-    if (b >= a.B) return;
-    const bool ex = a.done && a.done[b] != 0;  // no carry at all: a warm-up batch of labelled frames
-    int lab = ex ? a.pred[b] : (a.fallback ? a.fallback[b] : -1);
-    if (lab >= a.n) lab = -1;  // a label outside the memory counts as no label
-    a.plan.final_label[b] = lab;
-    a.plan.stop_layer[b] = ex ? a.exit_layer[b] : a.L;
-    const unsigned long long tag = tag_of(a.plan.epoch, b);
-    if (lab >= 0) atomicMax(a.plan.class_tag + lab, tag);
-    atomicMax(a.plan.stream_tag + (a.stream_id ? a.stream_id[b] : 0), tag);
+    const unsigned long long epoch = *a.plan.epoch + 1;  // this call's number; every CTA reads it before any is through
+    if (b < a.B) {
+        const bool ex = a.done && a.done[b] != 0;  // no carry at all: a warm-up batch of labelled frames
+        int lab = ex ? a.pred[b] : (a.fallback ? a.fallback[b] : -1);
+        if (lab >= a.n) lab = -1;  // a label outside the memory counts as no label
+        a.plan.final_label[b] = lab;
+        a.plan.stop_layer[b] = ex ? a.exit_layer[b] : a.L;
+        const unsigned long long tag = tag_of(epoch, b);
+        if (lab >= 0) atomicMax(a.plan.class_tag + lab, tag);
+        atomicMax(a.plan.stream_tag + (a.stream_id ? a.stream_id[b] : 0), tag);
+    }
+    // the last CTA through makes the number current for the kernels that follow
+    __syncthreads();
+    if (threadIdx.x == 0 && atomicAdd(a.plan.epoch + 1, 1ull) == gridDim.x - 1) {
+        a.plan.epoch[1] = 0;
+        a.plan.epoch[0] = epoch;
+    }
 }
 
 // ---- Eq. 5 / Eq. 6 ------------------------------------------------------------------------
@@ -327,7 +336,7 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
             const int g = blockIdx.x * kUpdWarps + (tid >> 5);
             if (g >= a.B) return;
             const int s = a.stream_id ? a.stream_id[g] : 0;
-            if (a.plan.stream_tag[s] != tag_of(a.plan.epoch, g)) return;  // not the stream's first frame
+            if (a.plan.stream_tag[s] != tag_of(*a.plan.epoch, g)) return;  // not the stream's first frame
             tables_by_warp(a, rz, g, s, do_resize,
                            reinterpret_cast<unsigned char*>(s_dyn) + size_t(tid >> 5) * resize_smem(a.n, rz.k_max));
             return;
@@ -335,7 +344,7 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
         // ---- Sec. 6.1 by a whole CTA: the stream's frames, ascending, replayed per class -------
         const int g = blockIdx.x;
         const int s = a.stream_id ? a.stream_id[g] : 0;
-        if (a.plan.stream_tag[s] != tag_of(a.plan.epoch, g)) return;
+        if (a.plan.stream_tag[s] != tag_of(*a.plan.epoch, g)) return;
         for (int t0 = g - g % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
             const int b = t0 + tid;
             const int hit = (b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
@@ -369,7 +378,7 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_centers(const UpdateArgs
     const int nl = a.warm_layer >= 0 ? 1 : a.L;  // a warm-up touches one layer only
     const int g = job / nl, l0 = a.warm_layer >= 0 ? a.warm_layer : job - g * nl;  // l0 is 0-based; the paper's is l0 + 1
     const int cls = a.plan.final_label[g];
-    if (cls < 0 || a.plan.class_tag[cls] != tag_of(a.plan.epoch, g)) return;  // not the class's first frame
+    if (cls < 0 || a.plan.class_tag[cls] != tag_of(*a.plan.epoch, g)) return;  // not the class's first frame
     const int D = a.dims[l0];
     const bool vec = (D & 3) == 0;  // rows are 16-byte aligned
     const float* sv = a.sv[l0];

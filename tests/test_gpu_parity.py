@@ -378,3 +378,75 @@ def test_maps_ready_flag_with_alternating_batches():
     assert np.array_equal(gbs[(w.T - 1) % 2].pred.cpu().numpy(), ob["pred"])
     compare_state(w, cache, mem, rep)
     smtm.smtm_cache_destroy(cache)
+
+
+def test_bench_launch_configuration_matches_oracle():
+    # The benchmark's own launch configuration at full width: 512 streams, CUDA graphs of several steps, chained
+    # launches, SMTM_FLAG_MAPS_READY with two alternating carries, no diagnostics.  The graphs are replayed twice
+    # over; decisions of every step (read back from copies taken inside the graphs), counters and the final
+    # state must be the oracle's.
+    from harness import Report, compare_state
+
+    w = si.C5.scaled(T=8)
+    G, passes = 4, 2
+    cents, counts = si.initial_centers(w)
+    tau = [w.tau] * w.L
+    mem = oracle.OracleMemory(w.n, w.dims, tau, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W)
+    cache = smtm.smtm_cache_create(w.n, w.dims, tau, cents, counts, n_streams=w.S, k_init=w.k_init, k_min=w.k_min,
+                                   k_max=w.k_max, window_W=w.window_W, max_batch=w.B, flags=smtm.FLAG_MAPS_READY)
+    sid = si.stream_ids(w)
+    gbs = [smtm.Batch(cache, w.B, stream_id=sid, with_diagnostics=False) for _ in range(2)]
+    labs = si.labels(w)
+    maps = [[si.frames(w, l, labs[t], t, device="cuda") for l in range(w.L)] for t in range(w.T)]
+    fbs = [torch.from_numpy(si.fallback_labels(w, labs[t])).cuda() for t in range(w.T)]
+    kept = [dict(done=torch.zeros(w.B, dtype=torch.uint8, device="cuda"),
+                 pred=torch.zeros(w.B, dtype=torch.int32, device="cuda"),
+                 el=torch.zeros(w.B, dtype=torch.int32, device="cuda")) for _ in range(w.T)]
+    stream = torch.cuda.Stream()
+    sh = stream.cuda_stream
+
+    def step(t):
+        gb = gbs[t % 2]
+        smtm.smtm_lookup_exit_begin(cache, 0, smtm.Fmap(maps[t][0], w.dtype, w.layout, *si.shape4(w, 0)), gb, sh)
+        smtm.smtm_lookup_exit(cache, 1, smtm.Fmap(maps[t][1], w.dtype, w.layout, *si.shape4(w, 1)), gb, sh)
+        smtm.smtm_cache_update_resize(cache, gb, fbs[t], sh)
+        kept[t]["done"].copy_(gb.done, non_blocking=True)      # a copy node of the graph
+        kept[t]["pred"].copy_(gb.pred, non_blocking=True)
+        kept[t]["el"].copy_(gb.exit_layer, non_blocking=True)
+
+    with torch.cuda.stream(stream):
+        graphs = []
+        step(0)                      # eager once: one-time attributes are not set inside a capture
+        stream.synchronize()
+        smtm.smtm_cache_destroy(cache)
+        cache = smtm.smtm_cache_create(w.n, w.dims, tau, cents, counts, n_streams=w.S, k_init=w.k_init,
+                                       k_min=w.k_min, k_max=w.k_max, window_W=w.window_W, max_batch=w.B,
+                                       flags=smtm.FLAG_MAPS_READY)
+        gbs[:] = [smtm.Batch(cache, w.B, stream_id=sid, with_diagnostics=False) for _ in range(2)]
+        for g0 in range(0, w.T, G):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for t in range(g0, g0 + G):
+                    step(t)
+            graphs.append(g)
+        rep = Report()
+        for p in range(passes):
+            for gi, g in enumerate(graphs):
+                g.replay()
+                stream.synchronize()
+                for t in range(gi * G, gi * G + G):   # the oracle, step by step, on the same maps
+                    ob = mem.new_batch(w.B, sid)
+                    for l in range(w.L):
+                        mem.lookup_exit(l, maps[t][l].cpu(), w.dtype, w.layout, si.shape4(w, l), ob)
+                    assert mem.near_count == 0, "a decision within 1e-4 of the threshold: pick another seed"
+                    assert np.array_equal(kept[t]["done"].cpu().numpy(), ob["done"]), (p, t)
+                    assert np.array_equal(kept[t]["el"].cpu().numpy(), ob["exit_layer"]), (p, t)
+                    ex = ob["done"] == 1
+                    assert np.array_equal(kept[t]["pred"].cpu().numpy()[ex], ob["pred"][ex]), (p, t)
+                    mem.update(ob, si.fallback_labels(w, labs[t]))
+                    mem.resize()
+                    rep.frames += w.B
+            compare_state(w, cache, mem, rep)
+    ctr = smtm.smtm_cache_get_counters(cache)
+    assert [int(v) for v in ctr[: w.L]] == [int(v) for v in mem.exits_per_layer]
+    smtm.smtm_cache_destroy(cache)
