@@ -126,8 +126,10 @@ cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm
 struct UpdatePlan {
     int32_t* final_label;            // [max_batch] label each frame ends up with (-1 = none)
     int32_t* stop_layer;             // [max_batch] the paper's l at which its inference stopped
-    unsigned long long* class_tag;   // [n] election of the first frame of each class, see memory.cu
+    unsigned long long* class_tag;   // [L][n] number of the last update call that touched (layer, class)
     unsigned long long* stream_tag;  // [S] election of the first frame of each stream
+    int32_t* job_count;              // [2] (layer, class) pairs listed by this call ([number & 1]) and, zeroed, for the next
+    int32_t* jobs;                   // [L][n] the (layer << 16 | class) pairs Eq. 7 touches in this call, in no particular order
     unsigned long long* epoch;       // [2] device: [0] number of update calls completed so far, [1] CTAs of the plan
                                      // kernel that are through (zero between calls).  The number lives on the
                                      // device so that a replayed CUDA graph counts on like eager calls do.
@@ -165,6 +167,6 @@ struct ResizeArgs {
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches);
 // Tables and centres; with rz != nullptr also the Eq. 5 / Eq. 6 refresh of every stream that
 // had a frame in the batch.
-cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, cudaStream_t st, int64_t* launches);
+cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, int64_t* launches);
 
 }  // namespace smtm

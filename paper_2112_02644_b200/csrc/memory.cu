@@ -5,15 +5,16 @@
 // ascending frame index, so the result is the one a frame-by-frame replay would give and does
 // not depend on scheduling.
 //
-// An update is three launches.  k_update_plan writes every frame's final label and stop layer
-// and elects, per class and per stream present in the batch, its first frame (an integer
-// atomicMax on a tag that carries the call's sequence number, so the election tables never
-// need clearing; the number is kept on the device and moved on by the plan kernel itself, so
-// that a replayed CUDA graph counts on exactly like eager calls).  In k_update_centers every (frame, layer) CTA (Eq. 7) and in k_update_tables
-// every frame's warp (tables, optionally followed by its stream's Eq. 5 / Eq. 6 refresh)
-// first checks whether its frame was elected and leaves at once if not; classes and streams
-// the batch does not touch cost nothing.  The two are separate kernels because the tables
-// live in registers: with few registers the Eq. 7 CTAs are all resident at once.
+// An update is three launches.  k_update_plan writes every frame's final label and stop layer,
+// elects the first frame of every stream present in the batch (an integer atomicMax on a tag
+// that carries the call's sequence number, so the table never needs clearing) and lists the
+// (layer, class) pairs Eq. 7 has to touch (the first frame to stamp a pair with the call's
+// number appends it).  The number is kept on the device and moved on by the plan kernel itself,
+// so that a replayed CUDA graph counts on exactly like eager calls.  In k_update_tables a warp
+// per frame first checks whether its frame was elected and leaves at once if not (tables,
+// optionally followed by the stream's Eq. 5 / Eq. 6 refresh); the CTAs of k_update_centers walk
+// the list of (layer, class) jobs.  Classes and streams the batch does not touch cost nothing.
+// The two are separate kernels because the tables live in registers.
 #include <algorithm>
 
 #include "common.cuh"
@@ -42,7 +43,6 @@ __device__ __forceinline__ void table_step(int& ft, int& ts, bool appears, int f
 
 constexpr int kUpdThreads = 256;
 constexpr int kUpdWarps = kUpdThreads / kWarp;
-constexpr int kSliceCols = kUpdThreads * 4;  // columns of a centre handled per sweep (one float4 per thread)
 constexpr int kWarpTablesMaxN = 1024;        // classes a warp can keep in registers (32 per lane)
 constexpr int kTagBits = 24;                 // frames per batch < 2^24
 
@@ -68,10 +68,18 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a)
         if (lab >= a.n) lab = -1;  // a label outside the memory counts as no label
         a.plan.final_label[b] = lab;
         a.plan.stop_layer[b] = ex ? a.exit_layer[b] : a.L;
-        const unsigned long long tag = tag_of(epoch, b);
-        if (lab >= 0) atomicMax(a.plan.class_tag + lab, tag);
-        atomicMax(a.plan.stream_tag + (a.stream_id ? a.stream_id[b] : 0), tag);
+        if (lab >= 0) {
+            // Eq. 7 touches the layers up to the stop layer: the first frame to stamp (layer, class)
+            // with the call's number lists the pair as a job
+            const int l_lo = a.warm_layer >= 0 ? a.warm_layer : 0;
+            const int l_hi = a.warm_layer >= 0 ? a.warm_layer + 1 : (ex ? a.exit_layer[b] : a.L);
+            for (int l = l_lo; l < l_hi; ++l)
+                if (atomicExch(a.plan.class_tag + (size_t)l * a.n + lab, epoch) != epoch)
+                    a.plan.jobs[atomicAdd(a.plan.job_count + (epoch & 1), 1)] = (l << 16) | lab;
+        }
+        atomicMax(a.plan.stream_tag + (a.stream_id ? a.stream_id[b] : 0), tag_of(epoch, b));
     }
+    if (b == 0) a.plan.job_count[(epoch + 1) & 1] = 0;  // the next call's counter (the call before this one is over)
     // the last CTA through makes the number current for the kernels that follow
     __syncthreads();
     if (threadIdx.x == 0 && atomicAdd(a.plan.epoch + 1, 1ull) == gridDim.x - 1) {
@@ -200,35 +208,52 @@ __device__ __forceinline__ int compact_tile(int hit, int value, int* list, int* 
 // Sec. 6.1 for the stream whose first frame in the batch is g, by one warp with the stream's
 // tables in registers (class c lives in lane c % 32, register c / 32), then, if asked, that
 // stream's Eq. 5 / Eq. 6 refresh.  `smem` is this warp's resize_smem(n, k_max) bytes.
+// NC = classes per lane (n <= 32 * NC): the loops over a lane's classes are unrolled, and the kernel is bound by
+// instruction fetch, so the smallest NC that covers n is used.
+template <int NC>
 __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g, int s, int do_resize,
-                               unsigned char* smem) {
-    constexpr int NC = kWarpTablesMaxN / kWarp;
+                               unsigned char* smem, int* s_hits) {
     const int lane = threadIdx.x & 31;
     const unsigned lt = (1u << lane) - 1u;
     int32_t* ftp = a.ft + (size_t)s * a.n;
     int32_t* tsp = a.ts + (size_t)s * a.n;
     int ft[NC], ts[NC];
 #pragma unroll
-    for (int i = 0; i < NC; ++i) {
+    for (int i = 0; i < NC; ++i) {  // unconditional loads (a clamped index), so that all of them are in flight at once
         const int c = lane + i * kWarp;
-        ft[i] = c < a.n ? ftp[c] : 0;
-        ts[i] = c < a.n ? tsp[c] : 0;
+        const int f = ftp[min(c, a.n - 1)], t = tsp[min(c, a.n - 1)];
+        ft[i] = c < a.n ? f : 0;
+        ts[i] = c < a.n ? t : 0;
     }
-    // the stream's frames in ascending index (none precedes g)
-    for (int b0 = g - g % kWarp; b0 < a.B; b0 += kWarp) {
-        const int b = b0 + lane;
-        const bool hit = b >= g && b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s;
-        const int lab = hit ? a.plan.final_label[b] : -1;
-        unsigned mask = __ballot_sync(kFull, hit);
-        while (mask) {
-            const int src = __ffs(mask) - 1;
-            mask &= mask - 1;
-            const int l = __shfl_sync(kFull, lab, src);
+    // The stream's frames in ascending index (none precedes g), eight groups of 32 frames per trip
+    // to memory: their labels are first listed in order (s_hits, this warp's), then replayed by
+    // one loop, so that the code of the replay exists once (the kernel runs once per warp and is
+    // bound by instruction fetch, not by arithmetic).
+    for (int b0 = g - g % kWarp; b0 < a.B; b0 += 8 * kWarp) {
+        int sidv[8], labv[8];
 #pragma unroll
-            for (int i = 0; i < NC; ++i) {
-                table_step(ft[i], ts[i], lane + i * kWarp == l, a.forget_W);
-            }
+        for (int u = 0; u < 8; ++u) {  // unconditional loads (a clamped index), all in flight at once
+            const int bb = min(b0 + u * kWarp + lane, a.B - 1);
+            sidv[u] = a.stream_id ? a.stream_id[bb] : 0;
+            labv[u] = a.plan.final_label[bb];
         }
+        int n_hits = 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int b = b0 + u * kWarp + lane;
+            const bool hit = b >= g && b < a.B && sidv[u] == s;
+            const unsigned mask = __ballot_sync(kFull, hit);
+            if (hit) s_hits[n_hits + __popc(mask & lt)] = labv[u];
+            n_hits += __popc(mask);
+        }
+        __syncwarp();
+#pragma unroll 1
+        for (int h = 0; h < n_hits; ++h) {
+            const int l = s_hits[h];
+#pragma unroll
+            for (int i = 0; i < NC; ++i) table_step(ft[i], ts[i], lane + i * kWarp == l, a.forget_W);
+        }
+        __syncwarp();
     }
 #pragma unroll
     for (int i = 0; i < NC; ++i) {
@@ -327,6 +352,7 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
     __shared__ int s_list[kUpdThreads];
     __shared__ int s_scan[33];
     __shared__ unsigned long long s_part[kUpdWarps];
+    __shared__ int s_hits[kUpdWarps][8 * kWarp];  // labels of a stream's frames among 256 consecutive ones, per warp
     const int tid = threadIdx.x;
     chain_wait();
     chain_release();
@@ -337,8 +363,13 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
             if (g >= a.B) return;
             const int s = a.stream_id ? a.stream_id[g] : 0;
             if (a.plan.stream_tag[s] != tag_of(*a.plan.epoch, g)) return;  // not the stream's first frame
-            tables_by_warp(a, rz, g, s, do_resize,
-                           reinterpret_cast<unsigned char*>(s_dyn) + size_t(tid >> 5) * resize_smem(a.n, rz.k_max));
+            unsigned char* smem = reinterpret_cast<unsigned char*>(s_dyn) + size_t(tid >> 5) * resize_smem(a.n, rz.k_max);
+            if (a.n <= 8 * kWarp)
+                tables_by_warp<8>(a, rz, g, s, do_resize, smem, s_hits[tid >> 5]);
+            else if (a.n <= 16 * kWarp)
+                tables_by_warp<16>(a, rz, g, s, do_resize, smem, s_hits[tid >> 5]);
+            else
+                tables_by_warp<kWarpTablesMaxN / kWarp>(a, rz, g, s, do_resize, smem, s_hits[tid >> 5]);
             return;
         }
         // ---- Sec. 6.1 by a whole CTA: the stream's frames, ascending, replayed per class -------
@@ -364,73 +395,132 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
     }
 }
 
-// Eq. 7 for one (class, layer): CTA (g, layer) folds, if g is the first frame of its class, the
-// matching frames in ascending index.  g, layer = divmod(blockIdx.x, layers touched).
-__global__ void __launch_bounds__(kUpdThreads) k_update_centers(const UpdateArgs a) {
-    __shared__ int s_list[kUpdThreads];
+// Eq. 7 over the jobs (layer, class) listed by the plan kernel, taken round-robin by CTAs of
+// 1024 threads.  The frames' labels and stop layers are staged in shared memory once; per job the
+// matching frames are listed in ascending index (every thread looks at a run of consecutive
+// frames, one block scan), then thread = (four columns, group): group r folds the listed frames
+// r, r + 4, ... with eight rows in flight, the four groups are added in a fixed order, and the
+// centre, its length and its count are rewritten.  Nothing here waits on another CTA.
+constexpr int kCenThreads = 1024;
+constexpr int kCenCols = kCenThreads;        // columns per sweep: 256 threads x 4 columns, four groups
+constexpr int kCenTile = 2 * kCenThreads;    // frames staged and listed at a time
+
+// Lists, in ascending index, the frames of the staged tile whose label is cls and that stopped at
+// layer l0 + 1 or deeper; returns how many.  s_code[i] = label | stop layer << 16, or -1.
+__device__ __forceinline__ int list_frames(const int* s_code, int tile_frames, int cls, int l0, int* s_list, int* s_scan) {
+    const int per = (tile_frames + kCenThreads - 1) / kCenThreads;  // consecutive frames per thread (1 or 2)
+    const int f0 = threadIdx.x * per;
+    int mine = 0;
+    for (int i = 0; i < per; ++i) {
+        const int code = f0 + i < tile_frames ? s_code[f0 + i] : -1;
+        mine += (code >= 0 && (code & 0xffff) == cls && (code >> 16) >= l0 + 1) ? 1 : 0;
+    }
+    int cnt;
+    int pos = block_exclusive_scan(mine, s_scan, &cnt);
+    for (int i = 0; i < per && mine; ++i) {
+        const int code = f0 + i < tile_frames ? s_code[f0 + i] : -1;
+        if (code >= 0 && (code & 0xffff) == cls && (code >> 16) >= l0 + 1) s_list[pos++] = f0 + i;
+    }
+    __syncthreads();
+    return cnt;
+}
+
+__global__ void __launch_bounds__(kCenThreads, 1) k_update_centers(const UpdateArgs a) {
+    __shared__ int s_code[kCenTile];
+    __shared__ int s_list[kCenTile];
+    __shared__ float4 s_acc[3][kCenCols / 4];
     __shared__ int s_scan[33];
     __shared__ float s_red[32];
     const int tid = threadIdx.x;
     chain_wait();
     chain_release();
     const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_CENTERS : nullptr);
-    const int job = blockIdx.x;
-    const int nl = a.warm_layer >= 0 ? 1 : a.L;  // a warm-up touches one layer only
-    const int g = job / nl, l0 = a.warm_layer >= 0 ? a.warm_layer : job - g * nl;  // l0 is 0-based; the paper's is l0 + 1
-    const int cls = a.plan.final_label[g];
-    if (cls < 0 || a.plan.class_tag[cls] != tag_of(*a.plan.epoch, g)) return;  // not the class's first frame
-    const int D = a.dims[l0];
-    const bool vec = (D & 3) == 0;  // rows are 16-byte aligned
-    const float* sv = a.sv[l0];
-    float* cen = a.centers[l0] + (size_t)cls * D;
-    const float m = float(a.m[l0][cls]);
-    float nrm = 0.f;
-    int q = 0;
-    for (int d0 = 0; d0 < D; d0 += kSliceCols) {  // a slice of columns per sweep, four per thread
-        const int d = d0 + tid * 4;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        q = 0;
-        for (int t0 = g - g % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
-            const int b = t0 + tid;
-            const int hit = (b < a.B && a.plan.final_label[b] == cls && a.plan.stop_layer[b] >= l0 + 1) ? 1 : 0;
-            const int cnt = compact_tile(hit, b, s_list, s_scan);
-            if (cnt == 0) continue;
-            q += cnt;
-            if (d >= D) continue;
-            if (vec) {
-                // sixteen rows in flight per thread; the additions stay in ascending frame order
-                for (int i0 = 0; i0 < cnt; i0 += 16) {
-                    float4 r[16];
+    const bool single = a.B <= kCenTile;  // the whole batch fits one tile: staged once, listed once per job
+    const auto stage = [&](int base) {
+        for (int i = tid; i < kCenTile && base + i < a.B; i += kCenThreads) {
+            const int lab = a.plan.final_label[base + i], stop = a.plan.stop_layer[base + i];
+            s_code[i] = lab < 0 ? -1 : (lab | (stop << 16));
+        }
+        __syncthreads();
+    };
+    const int n_jobs = a.plan.job_count[*a.plan.epoch & 1];
+    int next_code = int(blockIdx.x) < n_jobs ? a.plan.jobs[blockIdx.x] : 0;  // in flight while the labels are staged
+    if (single) stage(0);
+    const int cg = tid & (kCenCols / 4 - 1), grp = tid / (kCenCols / 4);
+    for (int job = blockIdx.x; job < n_jobs; job += gridDim.x) {
+        const int cls = next_code & 0xffff, l0 = next_code >> 16;  // l0 is 0-based; the paper's is l0 + 1
+        if (job + int(gridDim.x) < n_jobs) next_code = a.plan.jobs[job + gridDim.x];
+        const int D = a.dims[l0];
+        const bool vec = (D & 3) == 0;  // rows are 16-byte aligned
+        const float* sv = a.sv[l0];
+        float* cen = a.centers[l0] + (size_t)cls * D;
+        int cnt = single ? list_frames(s_code, a.B, cls, l0, s_list, s_scan) : 0;
+        float nrm = 0.f;
+        int q = 0;
+        for (int d0 = 0; d0 < D; d0 += kCenCols) {  // a sweep of columns, four per thread
+            const int d = d0 + cg * 4;
+            float old[4] = {0.f, 0.f, 0.f, 0.f}, m = 0.f;  // the centre and its count as they are, fetched along with the rows
+            if (grp == 0) {
+                m = float(a.m[l0][cls]);
+                for (int j = 0; j < 4; ++j)
+                    if (d + j < D) old[j] = cen[d + j];
+            }
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            q = 0;
+            for (int base = 0; base < a.B; base += kCenTile) {
+                if (!single) {
+                    __syncthreads();  // the previous tile's readers are done with the staged codes and the list
+                    stage(base);
+                    cnt = list_frames(s_code, min(kCenTile, a.B - base), cls, l0, s_list, s_scan);
+                }
+                q += cnt;
+                if (d >= D) continue;
+                if (vec) {
+                    // eight rows in flight per thread; each group adds its rows in ascending frame order
+                    for (int i0 = grp; i0 < cnt; i0 += 32) {
+                        float4 r[8];
 #pragma unroll
-                    for (int u = 0; u < 16; ++u)
-                        r[u] = i0 + u < cnt
-                                   ? __ldg(reinterpret_cast<const float4*>(sv + (size_t)s_list[i0 + u] * D + d))
-                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int u = 0; u < 8; ++u)  // unconditional loads (past the end: the last row again, unused)
+                            r[u] = __ldg(reinterpret_cast<const float4*>(
+                                sv + (size_t)(base + s_list[min(i0 + 4 * u, cnt - 1)]) * D + d));
 #pragma unroll
-                    for (int u = 0; u < 16; ++u) {
-                        if (i0 + u < cnt) {
-                            acc[0] += r[u].x; acc[1] += r[u].y; acc[2] += r[u].z; acc[3] += r[u].w;
+                        for (int u = 0; u < 8; ++u) {
+                            if (i0 + 4 * u < cnt) {
+                                acc[0] += r[u].x; acc[1] += r[u].y; acc[2] += r[u].z; acc[3] += r[u].w;
+                            }
                         }
                     }
+                } else {
+                    for (int i = grp; i < cnt; i += 4)
+                        for (int j = 0; j < 4; ++j)
+                            if (d + j < D) acc[j] += sv[(size_t)(base + s_list[i]) * D + d + j];
                 }
-            } else {
-                for (int i = 0; i < cnt; ++i)
-                    for (int j = 0; j < 4; ++j)
-                        if (d + j < D) acc[j] += sv[(size_t)s_list[i] * D + d + j];
+            }
+            if (q == 0) break;  // cannot happen for a listed job; kept so that nothing divides by the old count alone
+            // the groups' sums in a fixed order: ((g0 + g1) + g2) + g3
+            __syncthreads();
+            if (grp > 0) s_acc[grp - 1][cg] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            __syncthreads();
+            if (grp == 0 && d < D) {
+#pragma unroll
+                for (int g = 0; g < 3; ++g) {
+                    const float4 o = s_acc[g][cg];
+                    acc[0] += o.x; acc[1] += o.y; acc[2] += o.z; acc[3] += o.w;
+                }
+                for (int j = 0; j < 4; ++j)
+                    if (d + j < D) {
+                        const float v = __fdiv_rn(__fmaf_rn(old[j], m, acc[j]), m + float(q));
+                        cen[d + j] = v;
+                        nrm = fmaf(v, v, nrm);
+                    }
             }
         }
-        if (q == 0) return;  // no frame of this class stopped this deep: nothing changes
-        for (int j = 0; j < 4; ++j)
-            if (d + j < D) {
-                const float v = __fdiv_rn(__fmaf_rn(cen[d + j], m, acc[j]), m + float(q));
-                cen[d + j] = v;
-                nrm = fmaf(v, v, nrm);
-            }
-    }
-    nrm = block_sum(nrm, s_red);
-    if (tid == 0) {
-        a.cnorm[l0][cls] = __fsqrt_rn(nrm);
-        a.m[l0][cls] += (uint32_t)q;
+        if (q == 0) continue;
+        nrm = block_sum(nrm, s_red);  // also separates the reads of the count above from its update below
+        if (tid == 0) {
+            a.cnorm[l0][cls] = __fsqrt_rn(nrm);
+            a.m[l0][cls] += (uint32_t)q;
+        }
     }
 }
 
@@ -463,7 +553,7 @@ cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm
     return launch_chained(k_center_norms, n, 256, 0, st, centers, n, D, cnorm);
 }
 
-cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, cudaStream_t st, int64_t* launches) {
+cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
     if (a.B >= (1 << kTagBits)) return cudaErrorInvalidValue;
     static size_t opted = 48 * 1024;
@@ -485,8 +575,10 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, cudaStream_
                            warp_tables ? 1 : 0);
         if (e != cudaSuccess) return e;
     }
+    // Eq. 7: at most min(B, n) classes appear per layer; a CTA of 1024 threads per (layer, class) job, one per SM
+    const int centre_ctas = std::min(std::min(a.B, a.n) * (a.warm_layer >= 0 ? 1 : a.L), sm_count);
     ++*launches;
-    return launch_chained(k_update_centers, a.B * (a.warm_layer >= 0 ? 1 : a.L), kUpdThreads, 0, st, a);
+    return launch_chained(k_update_centers, centre_ctas, kCenThreads, 0, st, a);
 }
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
