@@ -28,7 +28,9 @@ struct smtm_cache {
     bool cen_split_current[SMTM_MAX_LAYERS];  // false after creation and after every update
     int d_max;          // largest C_l
     int32_t* d_plan;    // scratch of the update: final label and stop layer, 2 x [max_batch]
-    unsigned long long* d_tags;  // scratch of the update: stamps of (layer, class) [L][n], election tags of streams [S]
+    unsigned long long* d_tags;  // scratch of the update: stamps of (layer, class), [L][n]
+    cudaStream_t side_stream;    // the update's tables run here, beside plan + centres on the caller's stream
+    cudaEvent_t ev_fork, ev_join;
     int32_t* d_jobs;             // scratch of the update: [2] counters, [L][n] (layer, class) pairs to fold
     unsigned long long* d_epoch; // [2] device: update calls so far, and the plan kernel's ticket
     // optional timing of the streaming kernel of every lookup (smtm_cache_profile)
@@ -110,6 +112,9 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_dense);
     cudaFree(c->d_tags);
     cudaFree(c->d_epoch);
+    if (c->side_stream) cudaStreamDestroy(c->side_stream);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
     cudaFree(c->d_jobs);
     cudaFree(c->hb.d_sa);
     cudaFree(c->hb.d_done);
@@ -253,9 +258,8 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     a.plan.final_label = c->d_plan;
     a.plan.stop_layer = c->d_plan + mb;
     a.plan.class_tag = c->d_tags;
-    a.plan.stream_tag = c->d_tags + size_t(c->L) * c->n;
     a.plan.job_count = c->d_jobs;
-    a.plan.jobs = c->d_jobs + 2;
+    a.plan.jobs = c->d_jobs + 4;
     a.plan.epoch = c->d_epoch;
     a.stream_id = b->d_stream_id;
     a.done = b->d_done;
@@ -274,7 +278,7 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     }
     const ResizeArgs rz = resize_args(c);
     for (int l = 0; l < c->L; ++l) c->cen_split_current[l] = false;  // Eq. 7 is about to move centres
-    SMTM_CUDA(launch_update(a, with_resize ? &rz : nullptr, c->sm_count, st, &c->launches));
+    SMTM_CUDA(launch_update(a, with_resize ? &rz : nullptr, c->sm_count, st, c->side_stream, c->ev_fork, c->ev_join, &c->launches));
     return SMTM_OK;
 }
 
@@ -369,9 +373,12 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
         for (int l = 0; ok && l < c->L; ++l)
             ok = cudaMalloc(&c->d_cen_split[l], dense_centers_split_bytes(n, c->dims[l])) == cudaSuccess;
     }
-    ok = ok && dev_alloc(&c->d_tags, size_t(c->L) * n + size_t(S)) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_jobs, 2 + size_t(c->L) * n) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_tags, size_t(c->L) * n) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_jobs, 4 + size_t(c->L) * n) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_epoch, 2) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();
         free_all(c);
@@ -399,8 +406,8 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     if (e == cudaSuccess) e = cudaMemset(c->d_ts, 0, size_t(S) * n * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(c->d_counters, 0, SMTM_CTR_COUNT * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
-    if (e == cudaSuccess) e = cudaMemset(c->d_tags, 0, (size_t(c->L) * n + size_t(S)) * sizeof(unsigned long long));
-    if (e == cudaSuccess) e = cudaMemset(c->d_jobs, 0, (2 + size_t(c->L) * n) * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(c->d_tags, 0, size_t(c->L) * n * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(c->d_jobs, 0, (4 + size_t(c->L) * n) * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(c->d_epoch, 0, 2 * sizeof(unsigned long long));
     if (e == cudaSuccess)
         e = cudaMemcpy(c->d_members, members.data(), members.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
@@ -501,9 +508,8 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
     a.plan.final_label = c->d_plan;
     a.plan.stop_layer = c->d_plan + mb;
     a.plan.class_tag = c->d_tags;
-    a.plan.stream_tag = c->d_tags + size_t(c->L) * c->n;
     a.plan.job_count = c->d_jobs;
-    a.plan.jobs = c->d_jobs + 2;
+    a.plan.jobs = c->d_jobs + 4;
     a.plan.epoch = c->d_epoch;
     a.fallback = d_labels;
     a.ft = c->d_ft;
@@ -516,7 +522,7 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
         a.m[l] = c->d_m[l];
     }
     c->cen_split_current[layer] = false;
-    SMTM_CUDA(launch_update(a, nullptr, c->sm_count, st, &c->launches));
+    SMTM_CUDA(launch_update(a, nullptr, c->sm_count, st, c->side_stream, c->ev_fork, c->ev_join, &c->launches));
     return SMTM_OK;
 }
 

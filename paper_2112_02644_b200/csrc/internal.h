@@ -127,8 +127,8 @@ struct UpdatePlan {
     int32_t* final_label;            // [max_batch] label each frame ends up with (-1 = none)
     int32_t* stop_layer;             // [max_batch] the paper's l at which its inference stopped
     unsigned long long* class_tag;   // [L][n] number of the last update call that touched (layer, class)
-    unsigned long long* stream_tag;  // [S] election of the first frame of each stream
-    int32_t* job_count;              // [2] (layer, class) pairs listed by this call ([number & 1]) and, zeroed, for the next
+    int32_t* job_count;              // [0], [1]: (layer, class) pairs listed by this call ([number & 1]) and, zeroed, for the
+                                     // next; [2]: this call's count, published by the plan kernel's last CTA
     int32_t* jobs;                   // [L][n] the (layer << 16 | class) pairs Eq. 7 touches in this call, in no particular order
     unsigned long long* epoch;       // [2] device: [0] number of update calls completed so far, [1] CTAs of the plan
                                      // kernel that are through (zero between calls).  The number lives on the
@@ -167,6 +167,9 @@ struct ResizeArgs {
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches);
 // Tables and centres; with rz != nullptr also the Eq. 5 / Eq. 6 refresh of every stream that
 // had a frame in the batch.
-cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, int64_t* launches);
+// side, fork, join: a second stream and two events (no timing) of the caller's, used to run the tables beside
+// the plan and the centres.
+cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, cudaStream_t side,
+                          cudaEvent_t fork, cudaEvent_t join, int64_t* launches);
 
 }  // namespace smtm

@@ -5,16 +5,16 @@
 // ascending frame index, so the result is the one a frame-by-frame replay would give and does
 // not depend on scheduling.
 //
-// An update is three launches.  k_update_plan writes every frame's final label and stop layer,
-// elects the first frame of every stream present in the batch (an integer atomicMax on a tag
-// that carries the call's sequence number, so the table never needs clearing) and lists the
-// (layer, class) pairs Eq. 7 has to touch (the first frame to stamp a pair with the call's
-// number appends it).  The number is kept on the device and moved on by the plan kernel itself,
-// so that a replayed CUDA graph counts on exactly like eager calls.  In k_update_tables a warp
-// per frame first checks whether its frame was elected and leaves at once if not (tables,
-// optionally followed by the stream's Eq. 5 / Eq. 6 refresh); the CTAs of k_update_centers walk
-// the list of (layer, class) jobs.  Classes and streams the batch does not touch cost nothing.
-// The two are separate kernels because the tables live in registers.
+// An update is three launches on two streams.  k_update_plan writes every frame's final label
+// and stop layer and lists the (layer, class) pairs Eq. 7 has to touch (the first frame to stamp
+// a pair with the call's sequence number appends it; the number is kept on the device and moved
+// on by the plan kernel itself, so that a replayed CUDA graph counts on exactly like eager
+// calls); the CTAs of k_update_centers then walk that list.  k_update_tables depends on neither:
+// a warp per frame checks whether an earlier frame of the batch belongs to the same stream and
+// leaves if so, else it replays the stream's frames on the stream's tables (kept in registers)
+// and, when asked, refreshes the stream's fast memory (Eq. 5 / Eq. 6).  It runs on a side
+// stream, forked before the plan and joined after the centres, so the two halves of the update
+// overlap.  Classes and streams the batch does not touch cost nothing.
 #include <algorithm>
 
 #include "common.cuh"
@@ -44,12 +44,12 @@ __device__ __forceinline__ void table_step(int& ft, int& ts, bool appears, int f
 constexpr int kUpdThreads = 256;
 constexpr int kUpdWarps = kUpdThreads / kWarp;
 constexpr int kWarpTablesMaxN = 1024;        // classes a warp can keep in registers (32 per lane)
-constexpr int kTagBits = 24;                 // frames per batch < 2^24
 
-// Election tag of frame b in call number `epoch`: larger epoch wins over anything older,
-// within a call the smallest frame index wins.
-__device__ __forceinline__ unsigned long long tag_of(unsigned long long epoch, int b) {
-    return (epoch << kTagBits) | (unsigned long long)((1 << kTagBits) - 1 - b);
+// The label a finished frame ends up with: the prediction if it exited, else the fallback label
+// (the full network's answer, -1 = none); a label outside the memory counts as no label.
+__device__ __forceinline__ int final_label_of(const UpdateArgs& a, int b) {
+    const int lab = (a.done && a.done[b] != 0) ? a.pred[b] : (a.fallback ? a.fallback[b] : -1);
+    return lab >= a.n ? -1 : lab;
 }
 
 // ---- plan -----------------------------------------------------------------------------------
@@ -77,12 +77,15 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a)
                 if (atomicExch(a.plan.class_tag + (size_t)l * a.n + lab, epoch) != epoch)
                     a.plan.jobs[atomicAdd(a.plan.job_count + (epoch & 1), 1)] = (l << 16) | lab;
         }
-        atomicMax(a.plan.stream_tag + (a.stream_id ? a.stream_id[b] : 0), tag_of(epoch, b));
     }
     if (b == 0) a.plan.job_count[(epoch + 1) & 1] = 0;  // the next call's counter (the call before this one is over)
-    // the last CTA through makes the number current for the kernels that follow
+    // the last CTA through makes the number current for the kernels that follow and publishes the
+    // number of jobs (every CTA's appends are complete and visible before its ticket)
+    __threadfence();
     __syncthreads();
     if (threadIdx.x == 0 && atomicAdd(a.plan.epoch + 1, 1ull) == gridDim.x - 1) {
+        __threadfence();
+        a.plan.job_count[2] = *reinterpret_cast<volatile int32_t*>(a.plan.job_count + (epoch & 1));
         a.plan.epoch[1] = 0;
         a.plan.epoch[0] = epoch;
     }
@@ -235,7 +238,7 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
         for (int u = 0; u < 8; ++u) {  // unconditional loads (a clamped index), all in flight at once
             const int bb = min(b0 + u * kWarp + lane, a.B - 1);
             sidv[u] = a.stream_id ? a.stream_id[bb] : 0;
-            labv[u] = a.plan.final_label[bb];
+            labv[u] = final_label_of(a, bb);
         }
         int n_hits = 0;
 #pragma unroll
@@ -292,11 +295,20 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
     // rank the non-zero classes by counting; rank r < k_max goes to slot r
     for (int i = lane; i < nz; i += kWarp) {
         const unsigned long long sc = s_score[i];
-        int r = 0;
-        for (int j = 0; j < nz; ++j) {
-            const unsigned long long o = s_score[j];
-            r += (o > sc || (o == sc && j < i)) ? 1 : 0;  // compacted order is ascending id
+        int r0 = 0, r1 = 0, r2 = 0, r3 = 0;  // four counters: the loop is a chain of additions otherwise
+        int j = 0;
+        for (; j + 3 < nz; j += 4) {
+            const unsigned long long o0 = s_score[j], o1 = s_score[j + 1], o2 = s_score[j + 2], o3 = s_score[j + 3];
+            r0 += (o0 > sc || (o0 == sc && j < i)) ? 1 : 0;  // compacted order is ascending id
+            r1 += (o1 > sc || (o1 == sc && j + 1 < i)) ? 1 : 0;
+            r2 += (o2 > sc || (o2 == sc && j + 2 < i)) ? 1 : 0;
+            r3 += (o3 > sc || (o3 == sc && j + 3 < i)) ? 1 : 0;
         }
+        for (; j < nz; ++j) {
+            const unsigned long long o = s_score[j];
+            r0 += (o > sc || (o == sc && j < i)) ? 1 : 0;
+        }
+        const int r = (r0 + r1) + (r2 + r3);
         if (r < rz.k_max) {
             mem[r] = s_id[i];
             s_top[r] = sc;
@@ -362,7 +374,18 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
             const int g = blockIdx.x * kUpdWarps + (tid >> 5);
             if (g >= a.B) return;
             const int s = a.stream_id ? a.stream_id[g] : 0;
-            if (a.plan.stream_tag[s] != tag_of(*a.plan.epoch, g)) return;  // not the stream's first frame
+            // not the stream's first frame in the batch: the warp of that frame does the work
+            bool earlier = !a.stream_id && g > 0;
+            for (int b0 = 0; a.stream_id && b0 < g && !earlier; b0 += 8 * kWarp) {
+                bool same = false;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {  // unconditional loads (a clamped index), all in flight at once
+                    const int bb = b0 + u * kWarp + (tid & 31);
+                    same |= a.stream_id[min(bb, g)] == s && bb < g;
+                }
+                earlier = __any_sync(kFull, same);
+            }
+            if (earlier) return;
             unsigned char* smem = reinterpret_cast<unsigned char*>(s_dyn) + size_t(tid >> 5) * resize_smem(a.n, rz.k_max);
             if (a.n <= 8 * kWarp)
                 tables_by_warp<8>(a, rz, g, s, do_resize, smem, s_hits[tid >> 5]);
@@ -375,11 +398,13 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
         // ---- Sec. 6.1 by a whole CTA: the stream's frames, ascending, replayed per class -------
         const int g = blockIdx.x;
         const int s = a.stream_id ? a.stream_id[g] : 0;
-        if (a.plan.stream_tag[s] != tag_of(*a.plan.epoch, g)) return;
+        int earlier = (!a.stream_id && g > 0) ? 1 : 0;  // an earlier frame of the same stream: its CTA does the work
+        for (int b = tid; a.stream_id && b < g; b += kUpdThreads) earlier |= a.stream_id[b] == s ? 1 : 0;
+        if (__syncthreads_or(earlier)) return;
         for (int t0 = g - g % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
             const int b = t0 + tid;
             const int hit = (b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
-            const int cnt = compact_tile(hit, hit ? a.plan.final_label[b] : -1, s_list, s_scan);
+            const int cnt = compact_tile(hit, hit ? final_label_of(a, b) : -1, s_list, s_scan);
             if (cnt == 0) continue;
             for (int c = tid; c < a.n; c += kUpdThreads) {
                 int f = a.ft[(size_t)s * a.n + c], t = a.ts[(size_t)s * a.n + c];
@@ -443,8 +468,8 @@ __global__ void __launch_bounds__(kCenThreads, 1) k_update_centers(const UpdateA
         }
         __syncthreads();
     };
-    const int n_jobs = a.plan.job_count[*a.plan.epoch & 1];
-    int next_code = int(blockIdx.x) < n_jobs ? a.plan.jobs[blockIdx.x] : 0;  // in flight while the labels are staged
+    const int n_jobs = a.plan.job_count[2];
+    int next_code = a.plan.jobs[blockIdx.x];  // (the list has room for every pair) in flight with the count and the labels
     if (single) stage(0);
     const int cg = tid & (kCenCols / 4 - 1), grp = tid / (kCenCols / 4);
     for (int job = blockIdx.x; job < n_jobs; job += gridDim.x) {
@@ -553,9 +578,9 @@ cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm
     return launch_chained(k_center_norms, n, 256, 0, st, centers, n, D, cnorm);
 }
 
-cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, int64_t* launches) {
+cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, cudaStream_t side,
+                          cudaEvent_t fork, cudaEvent_t join, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
-    if (a.B >= (1 << kTagBits)) return cudaErrorInvalidValue;
     static size_t opted = 48 * 1024;
     const size_t per_stream = rz ? resize_smem(a.n, rz->k_max) : 0;
     // a warp per frame when the classes fit its registers and eight refresh buffers fit a CTA
@@ -563,22 +588,28 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
     const size_t smem = warp_tables ? per_stream * kUpdWarps : per_stream;
     cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_tables), smem, &opted);
     if (e != cudaSuccess) return e;
+    const bool tables = a.warm_layer < 0;  // a warm-up batch has no streams
+    if (tables) {
+        // the tables need nothing of the plan: they run beside plan + centres on the side stream
+        // (inside a stream capture the side stream joins the capture through the events)
+        if ((e = cudaEventRecord(fork, st)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(side, fork, 0)) != cudaSuccess) return e;
+        const int table_ctas = warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
+        ++*launches;
+        e = launch_chained(k_update_tables, table_ctas, kUpdThreads, smem, side, a, rz ? *rz : ResizeArgs{}, rz ? 1 : 0,
+                           warp_tables ? 1 : 0);
+        if (e != cudaSuccess) return e;
+        if ((e = cudaEventRecord(join, side)) != cudaSuccess) return e;
+    }
     ++*launches;
     e = launch_chained(k_update_plan, (a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st, a);
     if (e != cudaSuccess) return e;
-    // tables before centres: the next step's streaming kernel may overlap the last kernel of the update, and the
-    // centres' is the longer one
-    if (a.warm_layer < 0) {  // a warm-up batch has no streams
-        const int table_ctas = warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
-        ++*launches;
-        e = launch_chained(k_update_tables, table_ctas, kUpdThreads, smem, st, a, rz ? *rz : ResizeArgs{}, rz ? 1 : 0,
-                           warp_tables ? 1 : 0);
-        if (e != cudaSuccess) return e;
-    }
     // Eq. 7: at most min(B, n) classes appear per layer; a CTA of 1024 threads per (layer, class) job, one per SM
     const int centre_ctas = std::min(std::min(a.B, a.n) * (a.warm_layer >= 0 ? 1 : a.L), sm_count);
     ++*launches;
-    return launch_chained(k_update_centers, centre_ctas, kCenThreads, 0, st, a);
+    e = launch_chained(k_update_centers, centre_ctas, kCenThreads, 0, st, a);
+    if (e != cudaSuccess) return e;
+    return tables ? cudaStreamWaitEvent(st, join, 0) : cudaSuccess;
 }
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
