@@ -43,7 +43,6 @@ __device__ __forceinline__ void table_step(int& ft, int& ts, bool appears, int f
 
 constexpr int kUpdThreads = 256;
 constexpr int kUpdWarps = kUpdThreads / kWarp;
-constexpr int kWarpTablesMaxN = 1024;        // classes a warp can keep in registers (32 per lane)
 
 // The label a finished frame ends up with: the prediction if it exited, else the fallback label
 // (the full network's answer, -1 = none); a label outside the memory counts as no label.
@@ -211,27 +210,26 @@ __device__ __forceinline__ int compact_tile(int hit, int value, int* list, int* 
 // Sec. 6.1 for the stream whose first frame in the batch is g, by one warp with the stream's
 // tables in registers (class c lives in lane c % 32, register c / 32), then, if asked, that
 // stream's Eq. 5 / Eq. 6 refresh.  `smem` is this warp's resize_smem(n, k_max) bytes.
-// NC = classes per lane (n <= 32 * NC): the loops over a lane's classes are unrolled, and the kernel is bound by
-// instruction fetch, so the smallest NC that covers n is used.
-template <int NC>
+// The stream's tables are staged in shared memory (class c belongs to lane c % 32) and every pass
+// over the classes is a rolled loop: the kernel runs once per warp, so its time is the time to
+// fetch its instructions, and unrolled loops over registers were several times slower.
+__host__ __device__ constexpr size_t tables_smem(int n, int k_max) { return resize_smem(n, k_max) + size_t(n + (n & 1)) * 8; }
+
 __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g, int s, int do_resize,
                                unsigned char* smem, int* s_hits) {
     const int lane = threadIdx.x & 31;
     const unsigned lt = (1u << lane) - 1u;
     int32_t* ftp = a.ft + (size_t)s * a.n;
     int32_t* tsp = a.ts + (size_t)s * a.n;
-    int ft[NC], ts[NC];
-#pragma unroll
-    for (int i = 0; i < NC; ++i) {  // unconditional loads (a clamped index), so that all of them are in flight at once
-        const int c = lane + i * kWarp;
-        const int f = ftp[min(c, a.n - 1)], t = tsp[min(c, a.n - 1)];
-        ft[i] = c < a.n ? f : 0;
-        ts[i] = c < a.n ? t : 0;
+    int* s_ft = reinterpret_cast<int*>(smem + resize_smem(a.n, rz.k_max));  // [n]
+    int* s_ts = s_ft + a.n + (a.n & 1);                                     // [n]
+#pragma unroll 4
+    for (int c = lane; c < a.n; c += kWarp) {
+        s_ft[c] = ftp[c];
+        s_ts[c] = tsp[c];
     }
     // The stream's frames in ascending index (none precedes g), eight groups of 32 frames per trip
-    // to memory: their labels are first listed in order (s_hits, this warp's), then replayed by
-    // one loop, so that the code of the replay exists once (the kernel runs once per warp and is
-    // bound by instruction fetch, not by arithmetic).
+    // to memory: their labels are listed in order (s_hits, this warp's), then replayed.
     for (int b0 = g - g % kWarp; b0 < a.B; b0 += 8 * kWarp) {
         int sidv[8], labv[8];
 #pragma unroll
@@ -253,18 +251,15 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
 #pragma unroll 1
         for (int h = 0; h < n_hits; ++h) {
             const int l = s_hits[h];
-#pragma unroll
-            for (int i = 0; i < NC; ++i) table_step(ft[i], ts[i], lane + i * kWarp == l, a.forget_W);
+#pragma unroll 2
+            for (int c = lane; c < a.n; c += kWarp) table_step(s_ft[c], s_ts[c], c == l, a.forget_W);
         }
         __syncwarp();
     }
-#pragma unroll
-    for (int i = 0; i < NC; ++i) {
-        const int c = lane + i * kWarp;
-        if (c < a.n) {
-            ftp[c] = ft[i];
-            tsp[c] = ts[i];
-        }
+#pragma unroll 4
+    for (int c = lane; c < a.n; c += kWarp) {
+        ftp[c] = s_ft[c];
+        tsp[c] = s_ts[c];
     }
     if (!do_resize) return;
 
@@ -275,10 +270,10 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
     int32_t* mem = rz.members + (size_t)s * rz.k_max;
     unsigned long long total = 0;
     int nz = 0;
-#pragma unroll
-    for (int i = 0; i < NC; ++i) {
-        const int c = lane + i * kWarp;
-        const unsigned long long sc = c < a.n ? score_of(ft[i], ts[i], rz.W, rz.forgetting) : 0ull;
+#pragma unroll 1
+    for (int c0 = 0; c0 < a.n; c0 += kWarp) {
+        const int c = c0 + lane;
+        const unsigned long long sc = c < a.n ? score_of(s_ft[c], s_ts[c], rz.W, rz.forgetting) : 0ull;
         const unsigned m = __ballot_sync(kFull, sc != 0);
         if (sc != 0) {
             const int pos = nz + __popc(m & lt);
@@ -316,10 +311,10 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
     }
     // zero-score classes fill the remaining slots in ascending id
     int filled = nz;
-#pragma unroll
-    for (int i = 0; i < NC; ++i) {
-        const int c = lane + i * kWarp;
-        const bool z = filled < rz.k_max && c < a.n && score_of(ft[i], ts[i], rz.W, rz.forgetting) == 0;
+#pragma unroll 1
+    for (int c0 = 0; c0 < a.n && filled < rz.k_max; c0 += kWarp) {
+        const int c = c0 + lane;
+        const bool z = c < a.n && score_of(s_ft[c], s_ts[c], rz.W, rz.forgetting) == 0;
         const unsigned m = __ballot_sync(kFull, z);
         if (z) {
             const int pos = filled + __popc(m & lt);
@@ -386,13 +381,9 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
                 earlier = __any_sync(kFull, same);
             }
             if (earlier) return;
-            unsigned char* smem = reinterpret_cast<unsigned char*>(s_dyn) + size_t(tid >> 5) * resize_smem(a.n, rz.k_max);
-            if (a.n <= 8 * kWarp)
-                tables_by_warp<8>(a, rz, g, s, do_resize, smem, s_hits[tid >> 5]);
-            else if (a.n <= 16 * kWarp)
-                tables_by_warp<16>(a, rz, g, s, do_resize, smem, s_hits[tid >> 5]);
-            else
-                tables_by_warp<kWarpTablesMaxN / kWarp>(a, rz, g, s, do_resize, smem, s_hits[tid >> 5]);
+            tables_by_warp(a, rz, g, s, do_resize,
+                           reinterpret_cast<unsigned char*>(s_dyn) + size_t(tid >> 5) * tables_smem(a.n, rz.k_max),
+                           s_hits[tid >> 5]);
             return;
         }
         // ---- Sec. 6.1 by a whole CTA: the stream's frames, ascending, replayed per class -------
@@ -582,10 +573,10 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
                           cudaEvent_t fork, cudaEvent_t join, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
     static size_t opted = 48 * 1024;
-    const size_t per_stream = rz ? resize_smem(a.n, rz->k_max) : 0;
-    // a warp per frame when the classes fit its registers and eight refresh buffers fit a CTA
-    const bool warp_tables = a.n <= kWarpTablesMaxN && per_stream * kUpdWarps <= 96 * 1024;
-    const size_t smem = warp_tables ? per_stream * kUpdWarps : per_stream;
+    // a warp per frame when eight streams' tables and refresh buffers fit a CTA's shared memory
+    const size_t per_warp = tables_smem(a.n, rz ? rz->k_max : 0);
+    const bool warp_tables = per_warp * kUpdWarps <= 100 * 1024;
+    const size_t smem = warp_tables ? per_warp * kUpdWarps : (rz ? resize_smem(a.n, rz->k_max) : 0);
     cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_tables), smem, &opted);
     if (e != cudaSuccess) return e;
     const bool tables = a.warm_layer < 0;  // a warm-up batch has no streams
