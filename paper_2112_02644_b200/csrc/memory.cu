@@ -228,8 +228,21 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
         s_ft[c] = ftp[c];
         s_ts[c] = tsp[c];
     }
+    // Plain counts have a closed form (see the one-CTA-per-stream variant in k_update_tables): per class
+    // the number of appearances and the position of the last one, gathered in the space the refresh
+    // uses afterwards.  The forgetting table is replayed frame by frame.
+    const bool plain = a.forget_W == 0;
+    int* s_cnt = reinterpret_cast<int*>(smem);  // [n]
+    int* s_last = s_cnt + a.n;                  // [n]
+    if (plain)
+        for (int c = lane; c < a.n; c += kWarp) {
+            s_cnt[c] = 0;
+            s_last[c] = -1;
+        }
+    __syncwarp();
+    int m = 0;  // frames of the stream so far
     // The stream's frames in ascending index (none precedes g), eight groups of 32 frames per trip
-    // to memory: their labels are listed in order (s_hits, this warp's), then replayed.
+    // to memory: their labels are listed in order (s_hits, this warp's), then applied.
     for (int b0 = g - g % kWarp; b0 < a.B; b0 += 8 * kWarp) {
         int sidv[8], labv[8];
 #pragma unroll
@@ -248,14 +261,36 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
             n_hits += __popc(mask);
         }
         __syncwarp();
+        if (plain) {
+            for (int h = lane; h < n_hits; h += kWarp) {
+                const int l = s_hits[h];
+                if (l >= 0) {
+                    atomicAdd(&s_cnt[l], 1);
+                    atomicMax(&s_last[l], m + h);
+                }
+            }
+        } else {
 #pragma unroll 1
-        for (int h = 0; h < n_hits; ++h) {
-            const int l = s_hits[h];
+            for (int h = 0; h < n_hits; ++h) {
+                const int l = s_hits[h];
 #pragma unroll 2
-            for (int c = lane; c < a.n; c += kWarp) table_step(s_ft[c], s_ts[c], c == l, a.forget_W);
+                for (int c = lane; c < a.n; c += kWarp) table_step(s_ft[c], s_ts[c], c == l, a.forget_W);
+            }
         }
+        m += n_hits;
         __syncwarp();
     }
+    if (plain)
+        for (int c = lane; c < a.n; c += kWarp) {
+            const int q = s_cnt[c];
+            if (q > 0) {
+                s_ft[c] = int(min((long long)s_ft[c] + q, (long long)kFtMax));
+                s_ts[c] = m - 1 - s_last[c];
+            } else {
+                s_ts[c] = int(min((long long)s_ts[c] + m, (long long)INT32_MAX));
+            }
+        }
+    __syncwarp();
 #pragma unroll 4
     for (int c = lane; c < a.n; c += kWarp) {
         ftp[c] = s_ft[c];
@@ -392,16 +427,52 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs 
         int earlier = (!a.stream_id && g > 0) ? 1 : 0;  // an earlier frame of the same stream: its CTA does the work
         for (int b = tid; a.stream_id && b < g; b += kUpdThreads) earlier |= a.stream_id[b] == s ? 1 : 0;
         if (__syncthreads_or(earlier)) return;
-        for (int t0 = g - g % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
-            const int b = t0 + tid;
-            const int hit = (b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
-            const int cnt = compact_tile(hit, hit ? final_label_of(a, b) : -1, s_list, s_scan);
-            if (cnt == 0) continue;
+        if (a.forget_W == 0) {
+            // Plain counts: what a frame-by-frame replay leaves behind has a closed form per class.  With
+            // m frames of the stream in the batch, a class that appears q times, last at position p, ends
+            // with FT + q and TS = m - 1 - p; one that does not appear ends with TS + m.  q and p are
+            // gathered by shared-memory atomics on integers (a sum and a maximum: order does not matter).
+            int* s_cnt = reinterpret_cast<int*>(s_dyn);  // [n]; the refresh below reuses the space
+            int* s_last = s_cnt + a.n;                   // [n]
             for (int c = tid; c < a.n; c += kUpdThreads) {
-                int f = a.ft[(size_t)s * a.n + c], t = a.ts[(size_t)s * a.n + c];
-                for (int i = 0; i < cnt; ++i) table_step(f, t, s_list[i] == c, a.forget_W);
-                a.ft[(size_t)s * a.n + c] = f;
-                a.ts[(size_t)s * a.n + c] = t;
+                s_cnt[c] = 0;
+                s_last[c] = -1;
+            }
+            __syncthreads();
+            int m = 0;
+            for (int t0 = g - g % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
+                const int b = t0 + tid;
+                const int hit = (b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
+                const int cnt = compact_tile(hit, hit ? final_label_of(a, b) : -1, s_list, s_scan);
+                if (tid < cnt && s_list[tid] >= 0) {
+                    atomicAdd(&s_cnt[s_list[tid]], 1);
+                    atomicMax(&s_last[s_list[tid]], m + tid);
+                }
+                m += cnt;
+            }
+            __syncthreads();
+            for (int c = tid; c < a.n; c += kUpdThreads) {
+                const size_t at = (size_t)s * a.n + c;
+                const int q = s_cnt[c];
+                if (q > 0) {
+                    a.ft[at] = int(min((long long)a.ft[at] + q, (long long)kFtMax));
+                    a.ts[at] = m - 1 - s_last[c];
+                } else {
+                    a.ts[at] = int(min((long long)a.ts[at] + m, (long long)INT32_MAX));
+                }
+            }
+        } else {
+            for (int t0 = g - g % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
+                const int b = t0 + tid;
+                const int hit = (b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
+                const int cnt = compact_tile(hit, hit ? final_label_of(a, b) : -1, s_list, s_scan);
+                if (cnt == 0) continue;
+                for (int c = tid; c < a.n; c += kUpdThreads) {
+                    int f = a.ft[(size_t)s * a.n + c], t = a.ts[(size_t)s * a.n + c];
+                    for (int i = 0; i < cnt; ++i) table_step(f, t, s_list[i] == c, a.forget_W);
+                    a.ft[(size_t)s * a.n + c] = f;
+                    a.ts[(size_t)s * a.n + c] = t;
+                }
             }
         }
         if (do_resize) {
@@ -576,7 +647,9 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
     // a warp per frame when eight streams' tables and refresh buffers fit a CTA's shared memory
     const size_t per_warp = tables_smem(a.n, rz ? rz->k_max : 0);
     const bool warp_tables = per_warp * kUpdWarps <= 100 * 1024;
-    const size_t smem = warp_tables ? per_warp * kUpdWarps : (rz ? resize_smem(a.n, rz->k_max) : 0);
+    // one CTA per stream: the refresh buffers, and at least the two integer arrays [n] of the closed-form tables
+    const size_t smem = warp_tables ? per_warp * kUpdWarps
+                                    : std::max<size_t>(rz ? resize_smem(a.n, rz->k_max) : 0, size_t(a.n) * 2 * sizeof(int));
     cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_tables), smem, &opted);
     if (e != cudaSuccess) return e;
     const bool tables = a.warm_layer < 0;  // a warm-up batch has no streams
