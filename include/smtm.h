@@ -205,7 +205,14 @@ smtm_status_t smtm_lookup_exit_static(smtm_cache_t* cache, int32_t layer, const 
  * exited, else L.  Per stream, frames are applied in ascending b: FT[label] + 1
  * (saturating at 2^20), TS[label] = 0, TS of every other class + 1.  For every
  * class j and layer l0 the frames with label j and stop layer >= l0 are folded
- * into the centre in ascending b:  SC = (SC m + sum SV) / (m + q), m += q. */
+ * into the centre in ascending b:  SC = (SC m + sum SV) / (m + q), m += q
+ * (summed as four interleaved partial sums added in a fixed order).
+ * The tables are updated on a stream of the cache's own that is forked from
+ * `stream` and joined back to it before the call returns control of the stream,
+ * so that they run beside the centres; to the caller everything is ordered on
+ * `stream` as usual, and inside a stream capture the fork and join become part
+ * of the captured graph.  The call's bookkeeping lives on the device: a captured
+ * update may be replayed any number of times. */
 smtm_status_t smtm_cache_update(smtm_cache_t* cache, const smtm_batch_t* batch,
                                 const int32_t* d_fallback_label, void* stream);
 
