@@ -101,15 +101,25 @@ __device__ __forceinline__ unsigned long long score_of(int ft, int ts, int W, in
 }
 
 __host__ __device__ constexpr size_t resize_smem(int n, int k_max) { return size_t(n) * 8 + size_t(n + (n & 1)) * 4 + size_t(k_max) * 8; }
+// The one-CTA-per-stream refresh sorts: its score and id arrays are padded to a power of two.
+__host__ __device__ constexpr int pow2_at_least(int v) {
+    int p = 2;
+    while (p < v) p *= 2;
+    return p;
+}
+__host__ __device__ constexpr size_t resize_cta_smem(int n, int k_max) {
+    return size_t(pow2_at_least(n)) * 12 + size_t(k_max) * 8;
+}
 
 // Refresh of one stream's fast memory by a CTA of kUpdThreads threads.  Classes with a
 // non-zero score are compacted in ascending id and ranked among themselves by counting;
-// zero-score classes follow in ascending id.  `smem` holds resize_smem(n, k_max) bytes.
+// zero-score classes follow in ascending id.  `smem` holds resize_cta_smem(n, k_max) bytes.
 __device__ void resize_stream(const ResizeArgs& a, int s, unsigned char* smem, int* s_scan,
                               unsigned long long* s_part) {
     unsigned long long* s_score = reinterpret_cast<unsigned long long*>(smem);  // [n] compacted non-zero scores
-    int* s_id = reinterpret_cast<int*>(s_score + a.n);                          // [n] their class ids
-    unsigned long long* s_top = reinterpret_cast<unsigned long long*>(s_id + a.n + (a.n & 1));  // [k_max]
+    const int cap = pow2_at_least(a.n);                                         // both arrays hold `cap` entries
+    int* s_id = reinterpret_cast<int*>(s_score + cap);                          // their class ids
+    unsigned long long* s_top = reinterpret_cast<unsigned long long*>(s_id + cap);  // [k_max]
     const int tid = threadIdx.x;
     const int32_t* ft = a.ft + (size_t)s * a.n;
     const int32_t* ts = a.ts + (size_t)s * a.n;
@@ -139,18 +149,32 @@ __device__ void resize_stream(const ResizeArgs& a, int s, unsigned char* smem, i
     for (int w = 0; w < kUpdThreads / 32; ++w) total += s_part[w];
     if (total == 0) return;  // nothing seen yet: keep size and members
 
-    // pass 2: rank the non-zero classes; rank r < k_max goes to slot r
-    for (int i = tid; i < nz; i += kUpdThreads) {
-        const unsigned long long sc = s_score[i];
-        int r = 0;
-        for (int j = 0; j < nz; ++j) {
-            const unsigned long long o = s_score[j];
-            r += (o > sc || (o == sc && j < i)) ? 1 : 0;  // compacted order is ascending id
+    // pass 2: order the non-zero classes by (score descending, id ascending): a bitonic sort of the
+    // pairs, padded to a power of two with entries that rank last; rank r < k_max goes to slot r
+    const int P = pow2_at_least(nz);
+    for (int i = nz + tid; i < P; i += kUpdThreads) {
+        s_score[i] = 0ull;
+        s_id[i] = INT32_MAX;
+    }
+    __syncthreads();
+    for (int k = 2; k <= P; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = tid; t < P / 2; t += kUpdThreads) {
+                const int i = 2 * j * (t / j) + (t % j), l = i + j;
+                const unsigned long long si = s_score[i], sl = s_score[l];
+                const int ii = s_id[i], il = s_id[l];
+                const bool l_first = sl > si || (sl == si && il < ii);  // the entry at l ranks before the one at i
+                if (((i & k) == 0) ? l_first : !l_first) {             // (ids are distinct: never equal)
+                    s_score[i] = sl; s_score[l] = si;
+                    s_id[i] = il; s_id[l] = ii;
+                }
+            }
+            __syncthreads();
         }
-        if (r < a.k_max) {
-            mem[r] = s_id[i];
-            s_top[r] = sc;
-        }
+    }
+    for (int r = tid; r < nz && r < a.k_max; r += kUpdThreads) {
+        mem[r] = s_id[r];
+        s_top[r] = s_score[r];
     }
     // pass 3: zero-score classes fill the remaining slots in ascending id
     if (nz < a.k_max) {
@@ -169,17 +193,29 @@ __device__ void resize_stream(const ResizeArgs& a, int s, unsigned char* smem, i
     }
     __syncthreads();
     // pass 4: smallest k in [k_min, k_max] with cl_den * prefix(k) > cl_num * total
-    if (tid == 0) {
-        unsigned long long prefix = 0;
+    if (tid < kWarp) {  // warp 0: a scan of 32 entries per step
+        const int lane = tid;
+        unsigned long long carry = 0;
         int chosen = a.k_max;
-        for (int i = 0; i < a.k_max; ++i) {
-            prefix += s_top[i];
-            if (i + 1 >= a.k_min && (unsigned long long)a.cl_den * prefix > (unsigned long long)a.cl_num * total) {
-                chosen = i + 1;
+        for (int base = 0; base < a.k_max; base += kWarp) {
+            const int idx = base + lane;
+            unsigned long long v = idx < a.k_max ? s_top[idx] : 0ull;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long t = __shfl_up_sync(kFull, v, o);
+                if (lane >= o) v += t;
+            }
+            const unsigned long long prefix = carry + v;
+            const bool ok = idx < a.k_max && idx + 1 >= a.k_min &&
+                            (unsigned long long)a.cl_den * prefix > (unsigned long long)a.cl_num * total;
+            const unsigned m = __ballot_sync(kFull, ok);
+            if (m) {
+                chosen = base + __ffs(m);
                 break;
             }
+            carry += __shfl_sync(kFull, v, 31);
         }
-        a.k[s] = chosen;
+        if (lane == 0) a.k[s] = chosen;
     }
 }
 
@@ -649,7 +685,7 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
     const bool warp_tables = per_warp * kUpdWarps <= 100 * 1024;
     // one CTA per stream: the refresh buffers, and at least the two integer arrays [n] of the closed-form tables
     const size_t smem = warp_tables ? per_warp * kUpdWarps
-                                    : std::max<size_t>(rz ? resize_smem(a.n, rz->k_max) : 0, size_t(a.n) * 2 * sizeof(int));
+                                    : std::max<size_t>(rz ? resize_cta_smem(a.n, rz->k_max) : 0, size_t(a.n) * 2 * sizeof(int));
     cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_tables), smem, &opted);
     if (e != cudaSuccess) return e;
     const bool tables = a.warm_layer < 0;  // a warm-up batch has no streams
@@ -678,7 +714,7 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
     static size_t opted = 48 * 1024;
-    const size_t smem = resize_smem(a.n, a.k_max);
+    const size_t smem = resize_cta_smem(a.n, a.k_max);
     const cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_resize), smem, &opted);
     if (e != cudaSuccess) return e;
     ++*launches;
