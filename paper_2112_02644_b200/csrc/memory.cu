@@ -62,16 +62,20 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a)
     const int b = blockIdx.x * kUpdThreads + threadIdx.x;
     const unsigned long long epoch = *a.plan.epoch + 1;  // this call's number; every CTA reads it before any is through
     if (b < a.B) {
-        const bool ex = a.done && a.done[b] != 0;  // no carry at all: a warm-up batch of labelled frames
-        int lab = ex ? a.pred[b] : (a.fallback ? a.fallback[b] : -1);
+        // every load unconditional, so that they make one trip to memory (no carry at all: a warm-up batch
+        // of labelled frames)
+        const int dn = a.done ? a.done[b] : 0, pr = a.done ? a.pred[b] : -1, el = a.done ? a.exit_layer[b] : 0;
+        const int fb = a.fallback ? a.fallback[b] : -1;
+        const bool ex = dn != 0;
+        int lab = ex ? pr : fb;
         if (lab >= a.n) lab = -1;  // a label outside the memory counts as no label
         a.plan.final_label[b] = lab;
-        a.plan.stop_layer[b] = ex ? a.exit_layer[b] : a.L;
+        a.plan.stop_layer[b] = ex ? el : a.L;
         if (lab >= 0) {
             // Eq. 7 touches the layers up to the stop layer: the first frame to stamp (layer, class)
             // with the call's number lists the pair as a job
             const int l_lo = a.warm_layer >= 0 ? a.warm_layer : 0;
-            const int l_hi = a.warm_layer >= 0 ? a.warm_layer + 1 : (ex ? a.exit_layer[b] : a.L);
+            const int l_hi = a.warm_layer >= 0 ? a.warm_layer + 1 : (ex ? el : a.L);
             for (int l = l_lo; l < l_hi; ++l)
                 if (atomicExch(a.plan.class_tag + (size_t)l * a.n + lab, epoch) != epoch)
                     a.plan.jobs[atomicAdd(a.plan.job_count + (epoch & 1), 1)] = (l << 16) | lab;
