@@ -25,7 +25,7 @@ struct smtm_cache {
     float* d_warm_sv;   // scratch of smtm_cache_warmup: [max_batch][C_max] semantic vectors (allocated on first use)
     void* d_dense;      // scratch of the tensor-core scorer (fast memories above 64 entries), else NULL
     void* d_cen_split[SMTM_MAX_LAYERS];   // bf16 heads and tails of the centres, per layer (same condition)
-    bool cen_split_current[SMTM_MAX_LAYERS];  // false after creation and after every update
+    int* d_split_current;  // [L] device flags: the centres' split of a layer is current (same condition as d_dense)
     int d_max;          // largest C_l
     int32_t* d_plan;    // scratch of the update: final label and stop layer, 2 x [max_batch]
     unsigned long long* d_tags;  // scratch of the update: stamps of (layer, class), [L][n]
@@ -110,6 +110,7 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_plan);
     cudaFree(c->d_warm_sv);
     cudaFree(c->d_dense);
+    cudaFree(c->d_split_current);
     cudaFree(c->d_tags);
     cudaFree(c->d_epoch);
     if (c->side_stream) cudaStreamDestroy(c->side_stream);
@@ -218,10 +219,9 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     if (dense) {
         float *dots = nullptr, *dots2 = nullptr;
         SMTM_CUDA(launch_dense_dots(a.sv, a.fresh ? nullptr : a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max,
-                                    sv_split, c->d_cen_split[layer], c->cen_split_current[layer], &dots, &dots2, c->d_status,
+                                    sv_split, c->d_cen_split[layer], c->d_split_current + layer, &dots, &dots2, c->d_status,
                                     st, &c->launches));
-        c->cen_split_current[layer] = true;
-        SMTM_CUDA(launch_finish_dense(a, dots, dots2, st, &c->launches));
+        SMTM_CUDA(launch_finish_dense(a, dots, dots2, c->d_split_current + layer, st, &c->launches));
         return SMTM_OK;
     }
     SMTM_CUDA(launch_score_exit(a, st, &c->launches));
@@ -267,6 +267,7 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     a.pred = b->d_pred;
     a.fallback = d_fallback;
     a.clock = c->prof_events ? c->prof_step : nullptr;
+    a.split_current = c->d_split_current;
     a.ft = c->d_ft;
     a.ts = c->d_ts;
     for (int l = 0; l < c->L; ++l) {
@@ -277,7 +278,6 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
         a.m[l] = c->d_m[l];
     }
     const ResizeArgs rz = resize_args(c);
-    for (int l = 0; l < c->L; ++l) c->cen_split_current[l] = false;  // Eq. 7 is about to move centres
     SMTM_CUDA(launch_update(a, with_resize ? &rz : nullptr, c->sm_count, st, c->side_stream, c->ev_fork, c->ev_join, &c->launches));
     return SMTM_OK;
 }
@@ -370,6 +370,8 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     c->d_max = (c->d_max + 7) / 8 * 8;  // keeps the bf16 operand arrays of the tensor-core scorer 16-byte aligned
     if (ok && c->k_max > kFusedMaxK) {
         ok = cudaMalloc(&c->d_dense, dense_scratch_bytes(c->max_batch, n, c->d_max)) == cudaSuccess;
+        ok = ok && dev_alloc(&c->d_split_current, SMTM_MAX_LAYERS) == cudaSuccess &&
+             cudaMemset(c->d_split_current, 0, SMTM_MAX_LAYERS * sizeof(int)) == cudaSuccess;
         for (int l = 0; ok && l < c->L; ++l)
             ok = cudaMalloc(&c->d_cen_split[l], dense_centers_split_bytes(n, c->dims[l])) == cudaSuccess;
     }
@@ -512,6 +514,7 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
     a.plan.jobs = c->d_jobs + 4;
     a.plan.epoch = c->d_epoch;
     a.fallback = d_labels;
+    a.split_current = c->d_split_current;
     a.ft = c->d_ft;
     a.ts = c->d_ts;
     for (int l = 0; l < c->L; ++l) {
@@ -521,7 +524,6 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
         a.cnorm[l] = c->d_cnorm[l];
         a.m[l] = c->d_m[l];
     }
-    c->cen_split_current[layer] = false;
     SMTM_CUDA(launch_update(a, nullptr, c->sm_count, st, c->side_stream, c->ev_fork, c->ev_join, &c->launches));
     return SMTM_OK;
 }

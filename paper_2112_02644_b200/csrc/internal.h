@@ -104,17 +104,18 @@ bool dense_scoring_supported(int D, int n);
 size_t dense_scratch_bytes(int max_batch, int n, int d_max);
 // DOT[b][c] = <sv[b], centers[c]> for b < B, c < n into scratch; *dots_out = the [B][n] result.
 // The bf16 heads and tails of the semantic vectors sit at the start of scratch (see
-// dense_sv_split); sv_split_done / centers_split_done say whether they are already current.
+// dense_sv_split); sv_split_done says whether they are already current; centers_split_current is a device flag
+// that says the same of the centres' split (set by the finishing kernel, cleared by every update of the layer).
 void dense_sv_split(void* scratch, int max_batch, int d_max, void** hi, void** lo);
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
                               void* scratch, int max_batch, int d_max, bool sv_split_done, void* centers_split,
-                              bool centers_split_done, float** dots_out, float** dots2_out, int* status, cudaStream_t st,
+                              int* centers_split_current, float** dots_out, float** dots2_out, int* status, cudaStream_t st,
                               int64_t* launches);
 size_t dense_centers_split_bytes(int n, int D);
 // Eq. 1 from the dot products, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule; dots: [B][n], and dots2
 // (nullptr, or [B][n]: the second half of the vector length, added to the first).
-cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, cudaStream_t st,
-                                int64_t* launches);
+cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, int* split_current,
+                                cudaStream_t st, int64_t* launches);
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,
                                cudaStream_t st, int64_t* launches);
 
@@ -138,6 +139,7 @@ struct UpdatePlan {
 struct UpdateArgs {
     int B, S, n, L;
     unsigned long long* clock;  // nullptr, or the profiled step's stamps [SMTM_PROF_KERNELS][2] (see ClockScope)
+    int* split_current;         // nullptr, or [L]: the centres' bf16 split of a layer is current (cleared when Eq. 7 moves a centre)
     int forget_W;              // 0, or W when the frequency table itself forgets (SMTM_FLAG_FORGET_FT)
     int warm_layer;            // -1, or the one layer a warm-up batch folds into (no tables; done == nullptr)
     UpdatePlan plan;

@@ -109,12 +109,13 @@ __device__ __forceinline__ Top2 block_top2_keys(unsigned long long b1, unsigned 
 }
 
 __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, const float* __restrict__ dots,
-                                                           const float* __restrict__ dots2) {
+                                                           const float* __restrict__ dots2, int* split_current) {
     __shared__ float scratch[32];
     __shared__ unsigned long long s_keys[2 * (kThreads / kWarp)];
     chain_wait();
     chain_release();
     const int b = blockIdx.x;
+    if (b == 0 && threadIdx.x == 0 && split_current) *split_current = 1;  // the scorer before this kernel used (or made) a current split
     if (!a.fresh && a.done[b]) return;
     const int tid = threadIdx.x;
     const int sid = a.stream_id ? a.stream_id[b] : 0;
@@ -194,11 +195,11 @@ cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, in
     return launch_chained(k_batch_reset, grid, 256, 0, st, sa, done, exit_layer, pred, B, n_sa);
 }
 
-cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, cudaStream_t st,
-                                int64_t* launches) {
+cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, int* split_current,
+                                cudaStream_t st, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
     ++*launches;
-    return launch_chained(k_finish_dense, a.B, kThreads, 0, st, a, dots, dots2);
+    return launch_chained(k_finish_dense, a.B, kThreads, 0, st, a, dots, dots2, split_current);
 }
 
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches) {

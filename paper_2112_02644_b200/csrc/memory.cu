@@ -647,6 +647,7 @@ __global__ void __launch_bounds__(kCenThreads, 1) k_update_centers(const UpdateA
         if (tid == 0) {
             a.cnorm[l0][cls] = __fsqrt_rn(nrm);
             a.m[l0][cls] += (uint32_t)q;
+            if (a.split_current) a.split_current[l0] = 0;  // the tensor-core scorer's copy of this layer's centres is stale
         }
     }
 }

@@ -50,9 +50,11 @@ constexpr size_t kTcSmem = size_t(kTcStages) * kStageBytes + 1024 + 256;
 
 // x = hi + lo with hi = bf16(x) and lo = bf16(x - hi); rows of skipped frames are left alone.
 __global__ void k_split_bf16(const float* __restrict__ src, const uint8_t* __restrict__ skip, int rows, int D,
-                             __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+                             __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                             const int* __restrict__ current) {
     chain_wait();
     chain_release();
+    if (current && *current) return;  // the split on file is that of the source as it stands
     const long long total = (long long)rows * D;
     for (long long i = (blockIdx.x * (long long)blockDim.x + threadIdx.x) * 4; i < total;
          i += (long long)gridDim.x * blockDim.x * 4) {
@@ -321,7 +323,7 @@ void dense_sv_split(void* scratch, int max_batch, int d_max, void** hi, void** l
 
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
                               void* scratch, int max_batch, int d_max, bool sv_split_done, void* centers_split,
-                              bool centers_split_done, float** dots_out, float** dots2_out, int* status, cudaStream_t st,
+                              int* centers_split_current, float** dots_out, float** dots2_out, int* status, cudaStream_t st,
                               int64_t* launches) {
     __nv_bfloat16* a_hi = reinterpret_cast<__nv_bfloat16*>(scratch);
     __nv_bfloat16* a_lo = a_hi + size_t(max_batch) * d_max;
@@ -348,13 +350,16 @@ cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const
     if (!sv_split_done) {
         ++*launches;
         const int grid_a = int(std::min<long long>(((long long)B * D / 4 + 255) / 256, 148 * 8));
-        const cudaError_t e = launch_chained(k_split_bf16, grid_a, 256, 0, st, sv, skip, B, D, a_hi, a_lo);
+        const cudaError_t e = launch_chained(k_split_bf16, grid_a, 256, 0, st, sv, skip, B, D, a_hi, a_lo,
+                                             static_cast<const int*>(nullptr));
         if (e != cudaSuccess) return e;
     }
-    if (!centers_split_done) {
+    {  // always launched: whether the centres' split is current is a flag on the device (a replayed graph must not
+       // rely on what the host knew at capture); the kernel leaves at once when it is
         ++*launches;
         const int grid_b = int(std::min<long long>(((long long)n * D / 4 + 255) / 256, 148 * 8));
-        const cudaError_t e = launch_chained(k_split_bf16, grid_b, 256, 0, st, centers, static_cast<const uint8_t*>(nullptr), n, D, b_hi, b_lo);
+        const cudaError_t e = launch_chained(k_split_bf16, grid_b, 256, 0, st, centers, static_cast<const uint8_t*>(nullptr), n, D, b_hi, b_lo,
+                                             static_cast<const int*>(centers_split_current));
         if (e != cudaSuccess) return e;
     }
     ++*launches;
