@@ -380,14 +380,18 @@ def test_maps_ready_flag_with_alternating_batches():
     smtm.smtm_cache_destroy(cache)
 
 
-def test_bench_launch_configuration_matches_oracle():
+DENSE_GRAPH = si.Workload("dense_graph", si.BF16, si.NCHW, B=70, stages=((256, 14, 14), (512, 7, 7)), n=196, k_init=100,
+                           k_min=70, k_max=196, S=1, T=8, tau=0.8, window_W=2, sigma=0.6, zipf_s=0.9, repeat_p=0.3, seed=6)
+
+
+@pytest.mark.parametrize("w", [si.C5.scaled(T=8), DENSE_GRAPH], ids=["c5_full_width", "tensor_core_route"])
+def test_bench_launch_configuration_matches_oracle(w):
     # The benchmark's own launch configuration at full width: 512 streams, CUDA graphs of several steps, chained
     # launches, SMTM_FLAG_MAPS_READY with two alternating carries, no diagnostics.  The graphs are replayed twice
     # over; decisions of every step (read back from copies taken inside the graphs), counters and the final
     # state must be the oracle's.
     from harness import Report, compare_state
 
-    w = si.C5.scaled(T=8)
     G, passes = 4, 2
     cents, counts = si.initial_centers(w)
     tau = [w.tau] * w.L
