@@ -5,13 +5,15 @@
 // ascending frame index, so the result is the one a frame-by-frame replay would give and does
 // not depend on scheduling.
 //
-// An update is three launches on two streams.  k_update_plan writes every frame's final label
-// and stop layer and lists the (layer, class) pairs Eq. 7 has to touch (the first frame to stamp
-// a pair with the call's sequence number appends it; the number is kept on the device and moved
-// on by the plan kernel itself, so that a replayed CUDA graph counts on exactly like eager
-// calls); the CTAs of k_update_centers then walk that list.  k_update_tables depends on neither:
+// An update is three launches on two streams.  The plan kernel writes every frame's final label
+// and stop layer and lists the (layer, class) pairs Eq. 7 has to touch: up to 4096 frames and
+// 65 536 pairs a single CTA elects the pairs in a shared-memory bitmap (k_update_plan_one); past
+// that k_update_plan does it with many CTAs (the first frame to stamp a pair with the call's
+// sequence number appends it; the number is kept on the device and moved on by the kernel
+// itself, so that a replayed CUDA graph counts on exactly like eager calls).  The CTAs of
+// k_update_centers then walk that list.  k_update_tables depends on neither:
 // a warp per frame checks whether an earlier frame of the batch belongs to the same stream and
-// leaves if so, else it replays the stream's frames on the stream's tables (kept in registers)
+// leaves if so, else it applies the stream's frames to the stream's tables (staged in shared memory)
 // and, when asked, refreshes the stream's fast memory (Eq. 5 / Eq. 6).  It runs on a side
 // stream, forked before the plan and joined after the centres, so the two halves of the update
 // overlap.  Classes and streams the batch does not touch cost nothing.
@@ -43,6 +45,7 @@ __device__ __forceinline__ void table_step(int& ft, int& ts, bool appears, int f
 
 constexpr int kUpdThreads = 256;
 constexpr int kUpdWarps = kUpdThreads / kWarp;
+constexpr int kTblWarps = 16;  // warps (streams) to a CTA of k_update_tables in its warp-per-stream form
 
 // The label a finished frame ends up with: the prediction if it exited, else the fallback label
 // (the full network's answer, -1 = none); a label outside the memory counts as no label.
@@ -92,6 +95,45 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a)
         a.plan.epoch[1] = 0;
         a.plan.epoch[0] = epoch;
     }
+}
+
+// The same plan by a single CTA, for batches and memories small enough that one CTA's trip to
+// memory is all it takes: the pairs are elected in a bitmap in shared memory and counted there, so
+// nothing waits on a ticket or a fence.
+constexpr int kPlanOneThreads = 1024;
+constexpr int kPlanOneMaxB = 4 * kPlanOneThreads;
+constexpr int kPlanOneWords = 2048;  // 65 536 (layer, class) pairs
+
+__global__ void __launch_bounds__(kPlanOneThreads) k_update_plan_one(const UpdateArgs a) {
+    __shared__ unsigned int s_seen[kPlanOneWords];
+    __shared__ int s_jobs;
+    const int tid = threadIdx.x;
+    for (int i = tid; i < (a.L * a.n + 31) / 32; i += kPlanOneThreads) s_seen[i] = 0u;
+    if (tid == 0) s_jobs = 0;
+    chain_wait();
+    chain_release();
+    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_PLAN : nullptr);
+    __syncthreads();
+    for (int b = tid; b < a.B; b += kPlanOneThreads) {
+        const int dn = a.done ? a.done[b] : 0, pr = a.done ? a.pred[b] : -1, el = a.done ? a.exit_layer[b] : 0;
+        const int fb = a.fallback ? a.fallback[b] : -1;
+        const bool ex = dn != 0;
+        int lab = ex ? pr : fb;
+        if (lab >= a.n) lab = -1;
+        a.plan.final_label[b] = lab;
+        a.plan.stop_layer[b] = ex ? el : a.L;
+        if (lab >= 0) {
+            const int l_lo = a.warm_layer >= 0 ? a.warm_layer : 0;
+            const int l_hi = a.warm_layer >= 0 ? a.warm_layer + 1 : (ex ? el : a.L);
+            for (int l = l_lo; l < l_hi; ++l) {
+                const int pair = l * a.n + lab;
+                const unsigned int bit = 1u << (pair & 31);
+                if (!(atomicOr(&s_seen[pair >> 5], bit) & bit)) a.plan.jobs[atomicAdd(&s_jobs, 1)] = (l << 16) | lab;
+            }
+        }
+    }
+    __syncthreads();
+    if (tid == 0) a.plan.job_count[2] = s_jobs;
 }
 
 // ---- Eq. 5 / Eq. 6 ------------------------------------------------------------------------
@@ -428,20 +470,20 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
 // Tables (and, if asked, the refresh) of the streams whose first frames are among this CTA's
 // frames: a warp per frame, or, when the classes do not fit a warp's registers, the whole CTA
 // for one frame.
-__global__ void __launch_bounds__(kUpdThreads) k_update_tables(const UpdateArgs a, const ResizeArgs rz, int do_resize,
+__global__ void __launch_bounds__(kTblWarps * kWarp) k_update_tables(const UpdateArgs a, const ResizeArgs rz, int do_resize,
                                                                int warp_tables) {
     extern __shared__ unsigned long long s_dyn[];
     __shared__ int s_list[kUpdThreads];
     __shared__ int s_scan[33];
     __shared__ unsigned long long s_part[kUpdWarps];
-    __shared__ int s_hits[kUpdWarps][8 * kWarp];  // labels of a stream's frames among 256 consecutive ones, per warp
+    __shared__ int s_hits[kTblWarps][8 * kWarp];  // labels of a stream's frames among 256 consecutive ones, per warp
     const int tid = threadIdx.x;
     chain_wait();
     chain_release();
     const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_TABLES : nullptr, true);
     {
         if (warp_tables) {
-            const int g = blockIdx.x * kUpdWarps + (tid >> 5);
+            const int g = blockIdx.x * (blockDim.x >> 5) + (tid >> 5);  // the launch decides how many warps share a CTA
             if (g >= a.B) return;
             const int s = a.stream_id ? a.stream_id[g] : 0;
             // not the stream's first frame in the batch: the warp of that frame does the work
@@ -684,12 +726,17 @@ cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm
 cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, cudaStream_t side,
                           cudaEvent_t fork, cudaEvent_t join, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
-    static size_t opted = 48 * 1024;
+    // static + dynamic shared memory above 48 KB needs the opt-in; the kernel's static arrays take 18 KB of that
+    static size_t opted = 24 * 1024;
     // a warp per frame when eight streams' tables and refresh buffers fit a CTA's shared memory
     const size_t per_warp = tables_smem(a.n, rz ? rz->k_max : 0);
     const bool warp_tables = per_warp * kUpdWarps <= 100 * 1024;
     // one CTA per stream: the refresh buffers, and at least the two integer arrays [n] of the closed-form tables
-    const size_t smem = warp_tables ? per_warp * kUpdWarps
+    // Sixteen warps to a CTA when their buffers fit: the CTAs of k_update_centers fill an SM's registers, so
+    // every SM a tables CTA sits on is one that Eq. 7 cannot use until the tables are done (512 streams: 32
+    // SMs for the tables, 116 for the centres; with eight warps to a CTA it was 64 and 84)
+    const int warps = !warp_tables ? kUpdWarps : (per_warp * kTblWarps <= 180 * 1024 ? kTblWarps : kUpdWarps);
+    const size_t smem = warp_tables ? per_warp * warps
                                     : std::max<size_t>(rz ? resize_cta_smem(a.n, rz->k_max) : 0, size_t(a.n) * 2 * sizeof(int));
     cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_tables), smem, &opted);
     if (e != cudaSuccess) return e;
@@ -699,15 +746,18 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
         // (inside a stream capture the side stream joins the capture through the events)
         if ((e = cudaEventRecord(fork, st)) != cudaSuccess) return e;
         if ((e = cudaStreamWaitEvent(side, fork, 0)) != cudaSuccess) return e;
-        const int table_ctas = warp_tables ? (a.B + kUpdWarps - 1) / kUpdWarps : a.B;
+        const int table_ctas = warp_tables ? (a.B + warps - 1) / warps : a.B;
         ++*launches;
-        e = launch_chained(k_update_tables, table_ctas, kUpdThreads, smem, side, a, rz ? *rz : ResizeArgs{}, rz ? 1 : 0,
-                           warp_tables ? 1 : 0);
+        e = launch_chained(k_update_tables, table_ctas, warps * kWarp, smem, side, a,
+                           rz ? *rz : ResizeArgs{}, rz ? 1 : 0, warp_tables ? 1 : 0);
         if (e != cudaSuccess) return e;
         if ((e = cudaEventRecord(join, side)) != cudaSuccess) return e;
     }
     ++*launches;
-    e = launch_chained(k_update_plan, (a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st, a);
+    if (a.B <= kPlanOneMaxB && (long long)a.L * a.n <= 32LL * kPlanOneWords)
+        e = launch_chained(k_update_plan_one, 1, kPlanOneThreads, 0, st, a);
+    else
+        e = launch_chained(k_update_plan, (a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st, a);
     if (e != cudaSuccess) return e;
     // Eq. 7: at most min(B, n) classes appear per layer; a CTA of 1024 threads per (layer, class) job, one per SM
     const int centre_ctas = std::min(std::min(a.B, a.n) * (a.warm_layer >= 0 ? 1 : a.L), sm_count);
@@ -718,7 +768,7 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
 }
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
-    static size_t opted = 48 * 1024;
+    static size_t opted = 40 * 1024;  // static + dynamic above 48 KB needs the opt-in
     const size_t smem = resize_cta_smem(a.n, a.k_max);
     const cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_resize), smem, &opted);
     if (e != cudaSuccess) return e;

@@ -286,6 +286,16 @@ def test_fused_lookup_every_cluster_size(B):
     assert rep.frames == 2 * B and rep.lookups >= 2 * B
 
 
+def test_update_of_a_batch_too_large_for_the_single_cta_plan():
+    # up to 4096 frames the update lists the (layer, class) pairs of Eq. 7 with one CTA and a bitmap in shared
+    # memory; beyond that many CTAs elect them through tags in global memory.  4200 small frames of one stream
+    # take the second way (every other test takes the first).
+    w = si.Workload("big_batch", si.F16, si.NCHW, B=4200, stages=((64, 4, 4), (128, 2, 2)), n=60, k_init=10, k_min=6,
+                    k_max=24, S=1, T=3, tau=0.8, window_W=4, sigma=0.5, zipf_s=1.0, repeat_p=0.3, seed=77)
+    rep = run_workload(w)
+    assert rep.frames == 3 * 4200 and sum(rep.exits) > 0
+
+
 def test_fused_lookup_exact_ties_go_to_the_lower_class():
     # two classes with the same centre at every layer: their similarities tie bit for bit, the lower class id
     # ranks first (top-1 / top-2 are selected through 64-bit keys in the fused kernel) and such a frame never exits
