@@ -46,6 +46,7 @@ __device__ __forceinline__ void table_step(int& ft, int& ts, bool appears, int f
 constexpr int kUpdThreads = 256;
 constexpr int kUpdWarps = kUpdThreads / kWarp;
 constexpr int kTblWarps = 16;  // warps (streams) to a CTA of k_update_tables in its warp-per-stream form
+constexpr int kTblGroups = 16;  // groups of 32 frames a warp looks up per trip to memory
 
 // The label a finished frame ends up with: the prediction if it exited, else the fallback label
 // (the full network's answer, -1 = none); a label outside the memory counts as no label.
@@ -292,6 +293,13 @@ __device__ __forceinline__ int compact_tile(int hit, int value, int* list, int* 
 // Sec. 6.1 for the stream whose first frame in the batch is g, by one warp with the stream's
 // tables in registers (class c lives in lane c % 32, register c / 32), then, if asked, that
 // stream's Eq. 5 / Eq. 6 refresh.  `smem` is this warp's resize_smem(n, k_max) bytes.
+// 16 bytes from global to shared memory without passing through registers (both addresses 16-byte
+// aligned); the thread goes on and collects all of its copies with copy_async_wait_all().
+__device__ __forceinline__ void copy_async_16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void copy_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 // The stream's tables are staged in shared memory (class c belongs to lane c % 32) and every pass
 // over the classes is a rolled loop: the kernel runs once per warp, so its time is the time to
 // fetch its instructions, and unrolled loops over registers were several times slower.
@@ -305,10 +313,21 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
     int32_t* tsp = a.ts + (size_t)s * a.n;
     int* s_ft = reinterpret_cast<int*>(smem + resize_smem(a.n, rz.k_max));  // [n]
     int* s_ts = s_ft + a.n + (a.n & 1);                                     // [n]
+    // Staged by 16-byte asynchronous copies where the rows allow it: every copy is in flight at once and
+    // lands while the stream's frames are being looked up below.
+    const bool staged_async = (a.n & 3) == 0 && ((reinterpret_cast<uintptr_t>(ftp) | reinterpret_cast<uintptr_t>(tsp) |
+                                                   smem_u32(s_ft) | smem_u32(s_ts)) & 15) == 0;
+    if (staged_async) {
+        for (int v = lane; v < a.n / 4; v += kWarp) {
+            copy_async_16(s_ft + 4 * v, ftp + 4 * v);
+            copy_async_16(s_ts + 4 * v, tsp + 4 * v);
+        }
+    } else {
 #pragma unroll 4
-    for (int c = lane; c < a.n; c += kWarp) {
-        s_ft[c] = ftp[c];
-        s_ts[c] = tsp[c];
+        for (int c = lane; c < a.n; c += kWarp) {
+            s_ft[c] = ftp[c];
+            s_ts[c] = tsp[c];
+        }
     }
     // Plain counts have a closed form (see the one-CTA-per-stream variant in k_update_tables): per class
     // the number of appearances and the position of the last one, gathered in the space the refresh
@@ -323,19 +342,21 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
         }
     __syncwarp();
     int m = 0;  // frames of the stream so far
-    // The stream's frames in ascending index (none precedes g), eight groups of 32 frames per trip
+    // The stream's frames in ascending index (none precedes g), kTblGroups groups of 32 frames per trip
     // to memory: their labels are listed in order (s_hits, this warp's), then applied.
-    for (int b0 = g - g % kWarp; b0 < a.B; b0 += 8 * kWarp) {
-        int sidv[8], labv[8];
+    for (int b0 = g - g % kWarp; b0 < a.B; b0 += kTblGroups * kWarp) {
+        int sidv[kTblGroups], labv[kTblGroups];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {  // unconditional loads (a clamped index), all in flight at once
+        for (int u = 0; u < kTblGroups; ++u) {  // unconditional loads (a clamped index), all in flight at once
             const int bb = min(b0 + u * kWarp + lane, a.B - 1);
             sidv[u] = a.stream_id ? a.stream_id[bb] : 0;
-            labv[u] = final_label_of(a, bb);
+            const int dn = a.done ? a.done[bb] : 0, pr = a.done ? a.pred[bb] : -1, fb = a.fallback ? a.fallback[bb] : -1;
+            const int lab = dn != 0 ? pr : fb;  // final_label_of with every load issued up front
+            labv[u] = lab >= a.n ? -1 : lab;
         }
         int n_hits = 0;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < kTblGroups; ++u) {
             const int b = b0 + u * kWarp + lane;
             const bool hit = b >= g && b < a.B && sidv[u] == s;
             const unsigned mask = __ballot_sync(kFull, hit);
@@ -343,6 +364,10 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
             n_hits += __popc(mask);
         }
         __syncwarp();
+        if (!plain && staged_async) {  // the replay works on the staged tables
+            copy_async_wait_all();
+            __syncwarp();
+        }
         if (plain) {
             for (int h = lane; h < n_hits; h += kWarp) {
                 const int l = s_hits[h];
@@ -360,6 +385,10 @@ __device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g,
             }
         }
         m += n_hits;
+        __syncwarp();
+    }
+    if (staged_async) {
+        copy_async_wait_all();
         __syncwarp();
     }
     if (plain)
@@ -476,7 +505,7 @@ __global__ void __launch_bounds__(kTblWarps * kWarp) k_update_tables(const Updat
     __shared__ int s_list[kUpdThreads];
     __shared__ int s_scan[33];
     __shared__ unsigned long long s_part[kUpdWarps];
-    __shared__ int s_hits[kTblWarps][8 * kWarp];  // labels of a stream's frames among 256 consecutive ones, per warp
+    __shared__ int s_hits[kTblWarps][kTblGroups * kWarp];  // labels of a stream's frames among 512 consecutive ones, per warp
     const int tid = threadIdx.x;
     chain_wait();
     chain_release();
@@ -488,10 +517,10 @@ __global__ void __launch_bounds__(kTblWarps * kWarp) k_update_tables(const Updat
             const int s = a.stream_id ? a.stream_id[g] : 0;
             // not the stream's first frame in the batch: the warp of that frame does the work
             bool earlier = !a.stream_id && g > 0;
-            for (int b0 = 0; a.stream_id && b0 < g && !earlier; b0 += 8 * kWarp) {
+            for (int b0 = 0; a.stream_id && b0 < g && !earlier; b0 += kTblGroups * kWarp) {
                 bool same = false;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {  // unconditional loads (a clamped index), all in flight at once
+                for (int u = 0; u < kTblGroups; ++u) {  // unconditional loads (a clamped index), all in flight at once
                     const int bb = b0 + u * kWarp + (tid & 31);
                     same |= a.stream_id[min(bb, g)] == s && bb < g;
                 }
@@ -726,8 +755,8 @@ cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm
 cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, cudaStream_t side,
                           cudaEvent_t fork, cudaEvent_t join, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
-    // static + dynamic shared memory above 48 KB needs the opt-in; the kernel's static arrays take 18 KB of that
-    static size_t opted = 24 * 1024;
+    // static + dynamic shared memory above 48 KB needs the opt-in; the kernel's static arrays take 34 KB of that
+    static size_t opted = 8 * 1024;
     // a warp per frame when eight streams' tables and refresh buffers fit a CTA's shared memory
     const size_t per_warp = tables_smem(a.n, rz ? rz->k_max : 0);
     const bool warp_tables = per_warp * kUpdWarps <= 100 * 1024;
