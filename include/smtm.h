@@ -268,7 +268,10 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * smtm_lookup_exit (a step = L consecutive calls) record a pair of CUDA events on
  * the caller's stream right around that kernel, up to max_lookups pairs; 0
  * switches it off and frees the events.  Inside a stream capture the events
- * become graph nodes that are re-recorded at every replay.
+ * become graph nodes that are re-recorded at every replay.  A negative `every`
+ * profiles every |every|-th step with the device-clock stamps alone (below): no
+ * event is recorded, so the step's launches follow one another as in an
+ * unprofiled step, but for the memset that clears the stamps at its start.
  * smtm_cache_get_profile adds up the elapsed times of the recorded lookups of
  * one layer.  smtm_cache_get_profile_device reports, for the same steps, how long
  * each kernel of the step ran by the device's own clock, from the moment its
@@ -278,12 +281,21 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * layer i (i < SMTM_MAX_LAYERS; lookups that took another route count zero)
  * and for the three update kernels (SMTM_PROF_PLAN, _CENTERS, _TABLES).  This
  * leaves out what the event nodes add around a kernel.  Only the most recent
- * run of each profiled step is kept.  All three synchronise the device. */
+ * run of each profiled step is kept.  smtm_cache_get_profile_timeline gives the
+ * two stamps themselves for the step-th profiled step (counted from 0;
+ * SMTM_ERR_INVALID_ARG beyond the steps recorded): h_begin_ns[i] and
+ * h_end_ns[i], i < SMTM_PROF_KERNELS, in nanoseconds of the device's global
+ * timer, both 0 for a kernel that did not run in that step, so that the gaps
+ * between the kernels of a step can be read off.  All four synchronise the
+ * device. */
 enum { SMTM_PROF_PLAN = SMTM_MAX_LAYERS, SMTM_PROF_CENTERS, SMTM_PROF_TABLES, SMTM_PROF_KERNELS };
 smtm_status_t smtm_cache_profile(smtm_cache_t* cache, int32_t max_lookups, int32_t every);
 smtm_status_t smtm_cache_get_profile(smtm_cache_t* cache, int32_t layer, double* h_total_ms, int64_t* h_count);
 smtm_status_t smtm_cache_get_profile_device(smtm_cache_t* cache, double* h_total_ms /*[SMTM_PROF_KERNELS]*/,
                                             int64_t* h_count /*[SMTM_PROF_KERNELS]*/);
+smtm_status_t smtm_cache_get_profile_timeline(smtm_cache_t* cache, int64_t step,
+                                              uint64_t* h_begin_ns /*[SMTM_PROF_KERNELS]*/,
+                                              uint64_t* h_end_ns /*[SMTM_PROF_KERNELS]*/);
 
 /* Number of kernels the library has launched on behalf of this cache so far. */
 smtm_status_t smtm_cache_get_launches(smtm_cache_t* cache, int64_t* h_out);

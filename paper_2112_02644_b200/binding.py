@@ -103,6 +103,7 @@ def load_library():
     lib.smtm_cache_profile.argtypes = [vp, i32, i32]
     lib.smtm_cache_get_profile.argtypes = [vp, i32, vp, vp]
     lib.smtm_cache_get_profile_device.argtypes = [vp, vp, vp]
+    lib.smtm_cache_get_profile_timeline.argtypes = [vp, ctypes.c_int64, vp, vp]
     lib.smtm_cache_status.argtypes = [vp]
     lib.smtm_status_string.argtypes = [i32]
     lib.smtm_status_string.restype = ctypes.c_char_p
@@ -344,6 +345,16 @@ def smtm_cache_get_profile_device(cache: Cache):
     _check(load_library().smtm_cache_get_profile_device(cache.handle, total.ctypes.data, count.ctypes.data),
            "smtm_cache_get_profile_device")
     return total, count
+
+
+def smtm_cache_get_profile_timeline(cache: Cache, step: int):
+    """(begin ns [PROF_KERNELS], end ns [PROF_KERNELS]) of the step-th profiled step by the device's global timer;
+    both 0 for a kernel that did not run in it."""
+    begin = np.zeros(PROF_KERNELS, np.uint64)
+    end = np.zeros(PROF_KERNELS, np.uint64)
+    _check(load_library().smtm_cache_get_profile_timeline(cache.handle, int(step), begin.ctypes.data, end.ctypes.data),
+           "smtm_cache_get_profile_timeline")
+    return begin, end
 
 
 def smtm_cache_status(cache: Cache) -> int:

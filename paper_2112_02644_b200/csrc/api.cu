@@ -657,7 +657,9 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* c, int64_t* h_out) {
 }
 
 smtm_status_t smtm_cache_profile(smtm_cache_t* c, int32_t max_lookups, int32_t every) {
-    if (!c || max_lookups < 0 || max_lookups > (1 << 20) || every < 1) return SMTM_ERR_INVALID_ARG;
+    if (!c || max_lookups < 0 || max_lookups > (1 << 20) || every == 0 || every == INT32_MIN) return SMTM_ERR_INVALID_ARG;
+    const bool stamps_only = every < 0;  // no events: the chain of launches stays that of an unprofiled step
+    if (stamps_only) every = -every;
     SMTM_CUDA(cudaDeviceSynchronize());
     drop_profile(c);
     c->prof_every = every;
@@ -674,7 +676,7 @@ smtm_status_t smtm_cache_profile(smtm_cache_t* c, int32_t max_lookups, int32_t e
         drop_profile(c);
         return SMTM_ERR_ALLOC;
     }
-    for (int i = 0; i < 2 * max_lookups; ++i) {
+    for (int i = 0; !stamps_only && i < 2 * max_lookups; ++i) {
         cudaEvent_t ev;
         if (cudaEventCreate(&ev) != cudaSuccess) {
             (void)cudaGetLastError();
@@ -720,6 +722,22 @@ smtm_status_t smtm_cache_get_profile_device(smtm_cache_t* c, double* h_total_ms,
             h_total_ms[k] += double(end - begin) * 1e-6;
             ++h_count[k];
         }
+    }
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_get_profile_timeline(smtm_cache_t* c, int64_t step, uint64_t* h_begin_ns, uint64_t* h_end_ns) {
+    if (!c || !h_begin_ns || !h_end_ns) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    if (!c->d_prof_clock || step < 0 || size_t(step) >= c->prof_steps_used) return SMTM_ERR_INVALID_ARG;
+    std::vector<unsigned long long> stamps(2 * SMTM_PROF_KERNELS);
+    SMTM_CUDA(cudaMemcpy(stamps.data(), c->d_prof_clock + size_t(step) * stamps.size(),
+                         stamps.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+    for (int k = 0; k < SMTM_PROF_KERNELS; ++k) {
+        const unsigned long long begin = ~stamps[2 * k], end = stamps[2 * k + 1];  // the begin is kept as its complement
+        const bool ran = end != 0 && end >= begin;
+        h_begin_ns[k] = ran ? begin : 0;
+        h_end_ns[k] = ran ? end : 0;
     }
     return SMTM_OK;
 }

@@ -346,6 +346,28 @@ def test_device_clock_profile_reports_every_kernel_of_a_step():
     assert count[2:smtm.MAX_LAYERS].sum() == 0
     ev_ms, ev_n = smtm.smtm_cache_get_profile(cache, 0)
     assert ev_n == 2 and ev_ms >= total[0] * 0.5
+    # the stamps themselves: the kernels of a step in the order of their dependencies, the durations the same ones
+    spans = np.zeros(smtm.PROF_KERNELS)
+    for step in range(2):
+        begin, end = smtm.smtm_cache_get_profile_timeline(cache, step)
+        ran = [0, 1, smtm.PROF_PLAN, smtm.PROF_CENTERS, smtm.PROF_TABLES]
+        assert (begin[ran] > 0).all() and (end[ran] >= begin[ran]).all()
+        assert not begin[2:smtm.MAX_LAYERS].any() and not end[2:smtm.MAX_LAYERS].any()
+        assert end[0] <= begin[1] and end[1] <= begin[smtm.PROF_PLAN] and end[1] <= begin[smtm.PROF_TABLES]
+        assert end[smtm.PROF_PLAN] <= begin[smtm.PROF_CENTERS]
+        spans += (end - begin).astype(np.float64) * 1e-6
+    assert np.allclose(spans, total)
+    with pytest.raises(smtm.SmtmError):
+        smtm.smtm_cache_get_profile_timeline(cache, 2)
+    # stamps alone (negative period): no events, the device clock still reports the step
+    smtm.smtm_cache_profile(cache, 8, -1)
+    for l in range(w.L):
+        x = si.frames(w, l, labs[0], 0, device="cuda")
+        (smtm.smtm_lookup_exit_begin if l == 0 else smtm.smtm_lookup_exit)(
+            cache, l, smtm.Fmap(x, w.dtype, w.layout, *si.shape4(w, l)), gb)
+    smtm.smtm_cache_update_resize(cache, gb, torch.from_numpy(si.fallback_labels(w, labs[0])).cuda())
+    assert smtm.smtm_cache_get_profile(cache, 0)[1] == 0
+    assert list(smtm.smtm_cache_get_profile_device(cache)[1][[0, 1, smtm.PROF_PLAN]]) == [1, 1, 1]
     smtm.smtm_cache_profile(cache, 0, 1)
     assert smtm.smtm_cache_get_profile_device(cache)[1].sum() == 0
     smtm.smtm_cache_destroy(cache)
