@@ -770,12 +770,12 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
     cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_tables), smem, &opted);
     if (e != cudaSuccess) return e;
     const bool tables = a.warm_layer < 0;  // a warm-up batch has no streams
+    const int table_ctas = warp_tables ? (a.B + warps - 1) / warps : a.B;
     if (tables) {
         // the tables need nothing of the plan: they run beside plan + centres on the side stream
         // (inside a stream capture the side stream joins the capture through the events)
         if ((e = cudaEventRecord(fork, st)) != cudaSuccess) return e;
         if ((e = cudaStreamWaitEvent(side, fork, 0)) != cudaSuccess) return e;
-        const int table_ctas = warp_tables ? (a.B + warps - 1) / warps : a.B;
         ++*launches;
         e = launch_chained(k_update_tables, table_ctas, warps * kWarp, smem, side, a,
                            rz ? *rz : ResizeArgs{}, rz ? 1 : 0, warp_tables ? 1 : 0);
@@ -789,7 +789,11 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
         e = launch_chained(k_update_plan, (a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st, a);
     if (e != cudaSuccess) return e;
     // Eq. 7: at most min(B, n) classes appear per layer; a CTA of 1024 threads per (layer, class) job, one per SM
-    const int centre_ctas = std::min(std::min(a.B, a.n) * (a.warm_layer >= 0 ? 1 : a.L), sm_count);
+    // A centres CTA fills an SM's registers, and plan + centres start before the side stream's tables do:
+    // with a centres CTA on every SM the tables wait until some have left.  Up to a quarter of the SMs are
+    // left to the tables' CTAs.
+    const int table_sms = tables && warp_tables ? std::min(table_ctas, sm_count / 4) : 0;
+    const int centre_ctas = std::min(std::min(a.B, a.n) * (a.warm_layer >= 0 ? 1 : a.L), sm_count - table_sms);
     ++*launches;
     e = launch_chained(k_update_centers, centre_ctas, kCenThreads, 0, st, a);
     if (e != cudaSuccess) return e;
