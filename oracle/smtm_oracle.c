@@ -146,10 +146,12 @@ static void top2(const double* v, const int32_t* ids, int k, int* hi, int* sh) {
 
 /* (top - second) / second with the sign cases spelled out:
  *   top <= 0 (or NaN)           -> 0
+ *   second NaN                  -> NaN (Eq. 2 / Eq. 4 as printed, on a NaN operand)
  *   second <= 0 < top           -> +inf
  *   otherwise                   -> Eq. 2 / Eq. 4 as printed. */
 static double ratio_margin(double top, double second) {
     if (!(top > 0.0)) return 0.0;
+    if (isnan(second)) return NAN;
     if (!(second > 0.0)) return INFINITY;
     return (top - second) / second;
 }

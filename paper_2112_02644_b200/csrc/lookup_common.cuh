@@ -45,9 +45,10 @@ __device__ __forceinline__ Top2 warp_top2(const float* v, const int32_t* ids, in
     return t;
 }
 
-// (top - second) / second with the sign cases: top <= 0 -> 0; second <= 0 < top -> +inf.
+// (top - second) / second with the sign cases: top <= 0 -> 0; second NaN -> NaN; second <= 0 < top -> +inf.
 __device__ __forceinline__ float ratio_margin(float top, float second) {
     if (!(top > 0.f)) return 0.f;
+    if (isnan(second)) return __int_as_float(0x7fc00000);
     if (!(second > 0.f)) return INFINITY;
     return __fdiv_rn(__fsub_rn(top, second), second);
 }

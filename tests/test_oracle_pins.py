@@ -427,3 +427,75 @@ def test_forgetting_tables_equal_eq5_score_until_a_class_reappears_and_forget_af
     assert ft[0, 0] == 1
     oracle.tables_update(np.zeros(W, np.int32), np.ones(W, np.int32), ft, ts, forgetting_W=W)
     assert ft[0, 0] == 0
+
+
+# --------------------------------------------------------------------------- branches the paper is silent on
+
+def test_nan_similarity_ranks_below_every_number_and_an_all_nan_frame_never_exits():
+    # Sec. 5, Eq. 4 says nothing about non-finite similarities.  Reading: a NaN ranks after every
+    # number in top-1 / top-2 (ties among NaN by class id) and a frame whose SA are all NaN
+    # reports AC = 0 and stays in.  A NaN component in the semantic vector makes every cosine NaN;
+    # a NaN in one centre makes only that class's similarity NaN.
+    e = np.eye(3)
+    cen = e.copy()
+    cen[0, 1] = np.nan                       # class 0's centre is broken: its similarity is NaN
+    sv = np.array([[0.9, 0.5, 0.2]])
+    st = run_lookup([sv], [cen], [0, 1, 2], tau=0.8)
+    assert math.isnan(st["sa"][0, 0]) and not math.isnan(st["sa"][0, 1])
+    # the numbers rank first, in their own order: class 1 (0.5/|sv|) then class 2; the NaN is last
+    assert list(st["top"][0][0]) == [1, 2]
+    want = (0.5 - 0.2) / 0.2                 # cosines share the denominator |sv|
+    assert st["ac"][0][0] == pytest.approx(want, rel=1e-12) and st["done"][0] == 1 and st["pred"][0] == 1
+    # one number among NaNs: the number is top-1, a NaN (lowest class id) second.  Eq. 4 with a NaN
+    # runner-up is NaN, and a NaN confidence exceeds no threshold: the frame stays in
+    cen2 = e.copy(); cen2[0, 0] = np.nan; cen2[2, 2] = np.nan
+    for tau in (0.8, 0.0, -1.0):
+        st = run_lookup([np.array([[0.1, 0.7, 0.1]])], [cen2], [0, 1, 2], tau=tau)
+        assert list(st["top"][0][0]) == [1, 0] and math.isnan(st["ac"][0][0])
+        assert st["done"][0] == 0 and st["pred"][0] == -1 and st["near"][0][0] == 0
+    # every similarity NaN (a NaN in the frame itself): top-1 is the lowest class id by the tie rule,
+    # AC = 0, no exit at any threshold, and nothing is predicted
+    svn = np.array([[np.nan, 1.0, 0.0]])
+    for tau in (0.8, 0.0, -1.0):
+        st = run_lookup([svn], [e], [2, 0, 1], tau=tau)
+        assert np.isnan(st["sa"]).all()
+        assert st["done"][0] == 0 and st["ac"][0][0] == 0.0 and st["pred"][0] == -1
+        assert list(st["top"][0][0]) == [0, 1]
+    # an infinite component: inf / inf in Eq. 1 is NaN as well, same outcome
+    st = run_lookup([np.array([[np.inf, 1.0, 0.0]])], [e], [0, 1, 2], tau=0.5)
+    assert np.isnan(st["sa"]).all() and st["done"][0] == 0 and st["ac"][0][0] == 0.0
+
+
+def test_replacement_score_exponent_is_clamped_at_twelve_windows():
+    # Eq. 5's 0.25^floor(TS / W) is held as the integer FT * 4^(12 - e): beyond e = 12 the factor
+    # would drop below one unit, so e stops there (a stated deviation: FT * 4^0 = FT from 12 W on).
+    W, unit = 16, 4 ** 12
+    assert oracle.score(7, 11 * W + W - 1, W) == 7 * 4          # e = 11: the last exact window
+    assert Fraction(oracle.score(7, 11 * W, W), unit) == Fraction(7) * Fraction(1, 4) ** 11
+    for ts in (12 * W, 12 * W + 5, 13 * W, 40 * W, 2 ** 31 - 1):
+        assert oracle.score(7, ts, W) == 7                       # e clamped: never below FT * 4^0
+        assert oracle.score(1 << 20, ts, W) == 1 << 20
+    assert oracle.score(0, 40 * W, W) == 0
+    # the clamp keeps the order of Eq. 5 among old classes (monotone in FT) and against fresh ones
+    assert oracle.score(3, 40 * W, W) < oracle.score(4, 40 * W, W) < oracle.score(2, 11 * W, W)
+
+
+def test_frequency_count_saturates_and_time_stamp_stops_at_its_ceiling():
+    # FT stops at 2^20 (so that Eq. 6's sums of FT * 4^12 over up to 8192 classes fit 64 bits) and TS at
+    # INT32_MAX; neither wraps.
+    sid = np.zeros(3, np.int32)
+    ft = np.array([[(1 << 20) - 1, 5]], np.int32)
+    ts = np.array([[9, 2 ** 31 - 2]], np.int32)
+    oracle.tables_update(sid, np.array([0, 0, 0], np.int32), ft, ts)
+    assert ft[0, 0] == 1 << 20 and ts[0, 0] == 0            # one more appearance reaches the cap, two more stay
+    assert ft[0, 1] == 5 and ts[0, 1] == 2 ** 31 - 1        # aged once to the ceiling, then held
+    oracle.tables_update(sid, np.array([1, -1, 0], np.int32), ft, ts)
+    assert ft[0, 0] == 1 << 20 and ft[0, 1] == 6 and ts[0, 1] == 2 and ts[0, 0] == 0
+    # the score of a saturated count is the cap times the window factor, still exact in 64 bits
+    assert oracle.score(1 << 20, 0, 16) == (1 << 20) * 4 ** 12
+    assert oracle.score((1 << 20) + 123, 0, 16) == (1 << 20) * 4 ** 12    # a larger stored value reads as the cap
+    # the forgetting table saturates at the same count in its fixed-point unit and ages to the same ceiling
+    ft = np.array([[((1 << 20) << oracle.FT_FRAC) - 1, 0]], np.int32)
+    ts = np.array([[0, 2 ** 31 - 2]], np.int32)
+    oracle.tables_update(np.zeros(2, np.int32), np.array([0, 0], np.int32), ft, ts, forgetting_W=1 << 30)
+    assert ft[0, 0] == (1 << 20) << oracle.FT_FRAC and ts[0, 1] == 2 ** 31 - 1
