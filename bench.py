@@ -6,13 +6,17 @@ one bf16 frame each, looked up at the ResNet-50 stage-3 exit (1024x14x14) and,
 for frames that did not exit, at the stage-4 exit (2048x7x7), followed by the
 table / centre update and the adaptive resize of every stream's fast memory.
 Inputs are synthetic, seeded, resident in HBM and distinct per step (308 MB per
-step, larger than L2).  Prints one JSON line.
+step, larger than L2).  The timed steps are steps W .. W+K-1 of the workload:
+the memory is put back into the state it had after the W warm-up steps right
+before the clock starts, and the exit histogram of the timed steps is checked
+against the CPU oracle run over the same steps.  Prints one JSON line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 """
 from __future__ import annotations
 
 import argparse
+import concurrent.futures
 import json
 import math
 import os
@@ -31,6 +35,7 @@ import smtm_inputs as si  # noqa: E402
 
 WORKLOAD = si.C5   # the default and the benchmark line of record; --workload picks another for profiling
 METRIC = "frames/sec through encode+lookup+exit per exit layer (whole path incl. update+resize)"
+L2_BYTES = 126e6
 
 
 # DRAM bytes (read + write) of one launch of the dominant kernel from an ncu capture, per workload,
@@ -39,17 +44,21 @@ NCU_TRAFFIC = {"c5_streaming_bf16": (211_305_728, "753063d277df5b74")}
 _KERNEL_SOURCES = ("encode.cu", "common.cuh", "lookup_common.cuh")
 
 
-def ncu_traffic(workload_name: str, frames: int, full_frames: int):
+def kernel_digest() -> str:
     import hashlib
 
-    if workload_name not in NCU_TRAFFIC or frames != full_frames:
-        return None
     h = hashlib.sha256()
     for f in _KERNEL_SOURCES:
         with open(os.path.join(ROOT, "paper_2112_02644_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload_name: str, frames: int, full_frames: int):
+    if workload_name not in NCU_TRAFFIC or frames != full_frames:
+        return None
     traffic, digest = NCU_TRAFFIC[workload_name]
-    return traffic if h.hexdigest()[:16] == digest else None
+    return traffic if kernel_digest() == digest else None
 
 
 # --------------------------------------------------------------------------- helpers
@@ -59,8 +68,8 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
-        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy read+write)"
-    return 6650.0, "fallback (earlier measurement on this pool)"
+        return float(p["hbm_gbs"]), float(p.get("bf16_tflops", 1590.0)), "measured (MEASURED_PEAKS.json, copy read+write)"
+    return 6650.0, 1590.0, "fallback (earlier measurement on this pool)"
 
 
 class ClockSampler:
@@ -134,12 +143,312 @@ def job_throughput(frames_per_rank: int, ms_local: float, world: int, device="cu
     return frames_per_rank * world / (ms * 1e-3), ms
 
 
+def launch_ranks(n: int, argv, port=None) -> int:
+    """Starts `n` ranks of this script on this node (one per GPU) under torch's launcher and returns its exit
+    code; used when --gpus N is given and no launcher has set WORLD_SIZE."""
+    port = port or 29500 + os.getpid() % 1000
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def rank_check(args):
+    """The multi-rank plumbing alone, on the host (gloo): rendezvous, one shard of streams per rank, the
+    job's time as the maximum over ranks.  No GPU work; rank 0 prints one JSON line."""
+    import torch.distributed as dist
+
+    rank, _, world = dist_env()
+    if world > 1:
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+    w = shard_for_rank(WORKLOAD.scaled(B=16, S=16), rank)
+    value, ms = job_throughput(1000, 10.0 * (rank + 1), world, device="cpu")
+    seeds = [None] * world
+    if world > 1:
+        dist.all_gather_object(seeds, w.seed)
+        dist.barrier()
+        dist.destroy_process_group()
+    else:
+        seeds = [w.seed]
+    return {"rank_check": True, "n_gpus": world, "value": value, "ms": ms, "seeds": seeds} if rank == 0 else None
+
+
+# --------------------------------------------------------------------------- the oracle on the host cores
+
+class OracleRun:
+    """The CPU oracle stepped over a workload from a fresh memory, either on one thread or with the frames of a
+    step split over a pool of threads (the C functions release the interpreter lock).  Lookups of a step are
+    independent per frame; tables and fast memories per stream; Eq. 7 per class."""
+
+    def __init__(self, w, threads: int = 1):
+        import oracle
+
+        self.o = oracle
+        self.w = w
+        cents, counts = si.initial_centers(w)
+        self.mem = oracle.OracleMemory(w.n, w.dims, [w.tau] * w.L, cents, counts, w.S, w.k_init, w.k_min, w.k_max,
+                                       w.window_W, forgetting=w.forgetting)
+        self.sid = si.stream_ids(w)
+        self.threads = threads
+        self.pool = concurrent.futures.ThreadPoolExecutor(threads) if threads > 1 else None
+        self.seconds = 0.0
+        self.frames = 0
+        self.exits_after = []   # cumulative exits per layer after each step
+
+    def close(self):
+        if self.pool:
+            self.pool.shutdown()
+
+    def step(self, maps_cpu, fallback):
+        t0 = time.perf_counter()
+        (self._step_threaded if self.pool else self._step_serial)(maps_cpu, fallback)
+        self.seconds += time.perf_counter() - t0
+        self.frames += self.w.B
+        self.exits_after.append(self.mem.exits_per_layer.copy())
+
+    def _step_serial(self, maps_cpu, fallback):
+        w, mem = self.w, self.mem
+        ob = mem.new_batch(w.B, self.sid)
+        for l in range(w.L):
+            mem.lookup_exit(l, maps_cpu[l], w.dtype, w.layout, si.shape4(w, l), ob)
+        mem.update(ob, fallback)
+        mem.resize()
+
+    def _step_threaded(self, maps_cpu, fallback):
+        # Frames are cut into one contiguous slice per thread.  Every slice is looked up against the memory as
+        # it stood when the step began; then tables and fast memories are updated per slice of streams (this
+        # split needs each stream's frames inside one slice: one frame per stream, or a single stream), and
+        # Eq. 7 per range of classes (each range sees every frame, in ascending order, with the labels outside
+        # the range blanked).  The arithmetic is the oracle's own functions, untouched.
+        o, w, mem = self.o, self.w, self.mem
+        B, n_thr = w.B, self.threads
+        cuts = [B * i // n_thr for i in range(n_thr + 1)]
+        slices = [(a, b) for a, b in zip(cuts[:-1], cuts[1:]) if b > a]
+        ob = mem.new_batch(B, self.sid)
+        exits = np.zeros(w.L, np.int64)
+        for l in range(w.L):
+            B_, C, H, W = si.shape4(w, l)
+            raw = o._raw(maps_cpu[l]).reshape(B, -1)
+
+            def look(ab, l=l, C=C, H=H, W=W, raw=raw):
+                a, b = ab
+                todo = ob["done"][a:b] == 0
+                o.gap(raw[a:b], w.dtype, w.layout, b - a, C, H, W, skip=ob["done"][a:b], out=ob["sv"][l][a:b])
+                ac, sep, top, near = o.lookup_layer(l + 1, ob["sv"][l][a:b], mem.centers[l], ob["stream_id"][a:b],
+                                                    mem.members, mem.k, mem.tau[l], ob["sa"][a:b], ob["done"][a:b],
+                                                    ob["exit_layer"][a:b], ob["pred"][a:b])
+                return int(np.count_nonzero(todo & (ob["done"][a:b] == 1))), int(near[todo].sum())
+
+            for ex, near in self.pool.map(look, slices):
+                exits[l] += ex
+                mem.near_count += near
+        mem.exits_per_layer += exits
+        fb = np.where(fallback >= mem.n, -1, fallback).astype(np.int32)
+        exited = ob["done"] == 1
+        final = np.ascontiguousarray(np.where(exited, ob["pred"], fb), np.int32)
+        stop = np.ascontiguousarray(np.where(exited, ob["exit_layer"], mem.L), np.int32)
+        per_stream = w.S > 1      # one frame per stream: slice b0..b1 of the frames is streams b0..b1
+
+        def tables(ab):
+            a, b = ab
+            if per_stream:
+                o.tables_update(np.ascontiguousarray(ob["stream_id"][a:b] - a), final[a:b], mem.ft[a:b], mem.ts[a:b],
+                                mem.W if mem.forgetting else 0)
+                o.resize(mem.ft[a:b], mem.ts[a:b], mem.W, mem.k_min, mem.k_max, mem.cl_num, mem.cl_den,
+                         mem.members[a:b], mem.k[a:b], forgetting=mem.forgetting)
+
+        def centres(job):
+            l0, lo, hi = job
+            mine = np.ascontiguousarray(np.where((final >= lo) & (final < hi), final, -1), np.int32)
+            o.centers_update(l0, ob["sv"][l0 - 1], mine, stop, mem.centers[l0 - 1], mem.m[l0 - 1])
+
+        ccuts = [mem.n * i // n_thr for i in range(n_thr + 1)]
+        jobs = [(l0, a, b) for l0 in range(1, mem.L + 1) for a, b in zip(ccuts[:-1], ccuts[1:]) if b > a]
+        if per_stream:
+            futs = [self.pool.submit(tables, ab) for ab in slices] + [self.pool.submit(centres, j) for j in jobs]
+        else:       # a single stream: its tables are one sequential replay
+            o.tables_update(ob["stream_id"], final, mem.ft, mem.ts, mem.W if mem.forgetting else 0)
+            futs = [self.pool.submit(centres, j) for j in jobs]
+        for f in futs:
+            f.result()
+        if not per_stream:
+            mem.resize()
+
+
 # --------------------------------------------------------------------------- the CUDA arm
 
 def make_cache(smtm, w, cents, counts):
     return smtm.smtm_cache_create(w.n, w.dims, [w.tau] * w.L, cents, counts, n_streams=w.S, k_init=w.k_init,
                                   k_min=w.k_min, k_max=w.k_max, window_W=w.window_W, max_batch=w.B,
                                   flags=(smtm.FLAG_FORGET_FT if w.forgetting else 0) | smtm.FLAG_MAPS_READY)
+
+
+PROFILE_EVERY = 16  # every 16th step carries timing events and device-clock stamps (they cost a few us and break the chain of launches)
+
+
+class Resident:
+    """A workload's inputs resident in HBM: distinct maps for enough steps that consecutive steps never find
+    their maps in L2 (and, for the streaming workload, every step of the timed region its own maps)."""
+
+    def __init__(self, smtm, w, steps_needed: int):
+        self.w = w
+        step_bytes = sum(w.B * w.frame_bytes(l) for l in range(w.L))
+        if w.T > 1:
+            self.R = min(w.T, steps_needed)
+        else:   # a single-batch workload: the same labels under fresh noise, enough copies to defeat L2
+            self.R = max(2, int(math.ceil(2.2 * L2_BYTES / step_bytes)))
+            self.R += self.R % 2
+        self.step_bytes = step_bytes
+        self.labs = si.labels(w)
+        self.maps, self.fmaps, self.fbs = [], [], []
+        for r in range(self.R):
+            lab = self.labs[r % w.T]
+            m = [si.frames(w, l, lab, r, device="cuda") for l in range(w.L)]
+            self.maps.append(m)
+            self.fmaps.append([smtm.Fmap(m[l], w.dtype, w.layout, *si.shape4(w, l)) for l in range(w.L)])
+            self.fbs.append(torch.from_numpy(si.fallback_labels(w, lab)).cuda())
+        torch.cuda.synchronize()
+
+    def fallback_host(self, t):
+        return si.fallback_labels(self.w, self.labs[(t % self.R) % self.w.T])
+
+
+def measure(smtm, w, K, W, local_rank, world, verify_steps=0, oracle_threads=1):
+    """Times steps W .. W+K-1 of workload `w` through CUDA graphs and returns the figures of the run.
+    verify_steps > 0: the CPU oracle is run over steps 0 .. W+verify_steps-1 of the same maps and the exits it
+    takes in steps W .. W+verify_steps-1 are compared with the library's."""
+    if world > 1:
+        import torch.distributed as dist
+    res = Resident(smtm, w, W + K)
+    R = res.R
+    G = math.gcd(K, 32)         # steps captured into one CUDA graph
+    cents, counts = si.initial_centers(w)
+    sid = si.stream_ids(w) if w.S > 1 else None
+    # All launches go to one side stream so that every step can be captured into a CUDA graph.
+    stream = torch.cuda.Stream()
+    sh = stream.cuda_stream
+
+    def step(cache, gbs, t):
+        gb = gbs[t % 2]   # two carries alternate: the cache was created with FLAG_MAPS_READY (maps are resident)
+        smtm.smtm_lookup_exit_begin(cache, 0, res.fmaps[t % R][0], gb, sh)     # starts the batch: no separate reset
+        for l in range(1, w.L):
+            smtm.smtm_lookup_exit(cache, l, res.fmaps[t % R][l], gb, sh)
+        smtm.smtm_cache_update_resize(cache, gb, res.fbs[t % R], sh)
+
+    cache = make_cache(smtm, w, cents, counts)
+    gb = [smtm.Batch(cache, w.B, stream_id=sid, with_diagnostics=False) for _ in range(2)]
+    with torch.cuda.stream(stream):
+        for t in range(W):          # eager warm-up: kernels, clocks; these are steps 0 .. W-1 of the workload
+            step(cache, gb, t)
+        stream.synchronize()
+        snapshot = smtm.smtm_cache_export(cache)   # the memory after the warm-up steps: where the timed region starts
+        # One graph per G consecutive steps (their feature maps are baked in); the cache state lives in
+        # device memory the graphs point to, so replaying them in order advances it as eager calls
+        # would.  Inside a graph the kernels of consecutive steps are chained like those of one step.
+        n_prof = (K // PROFILE_EVERY + 2) * w.L
+        smtm.smtm_cache_profile(cache, n_prof, PROFILE_EVERY)
+        launches0 = smtm.smtm_cache_get_launches(cache)
+        graphs, order = {}, []
+        for t0 in range(W, W + K, G):
+            key = (t0 % R, t0 % 2) if R % G == 0 else t0     # steps t0 and t0 + R read the same maps
+            if key not in graphs:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    for t in range(t0, t0 + G):
+                        step(cache, gb, t)
+                graphs[key] = g
+            order.append(graphs[key])
+        launches_per_graph = (smtm.smtm_cache_get_launches(cache) - launches0) // max(len(graphs), 1)
+        for g in graphs.values():   # every graph once, untimed: its first launch uploads it to the device
+            g.replay()
+        stream.synchronize()
+
+        def restart():
+            smtm.smtm_cache_import(cache, snapshot)      # back to the state after step W-1 (synchronises)
+
+        check = None
+        V = min(verify_steps, K) // G * G
+        if V > 0:
+            check = {"steps": [W, W + V]}
+            if V < K:   # the timed region is longer than what the oracle covers: a separate, untimed pass
+                restart()
+                for g in order[: V // G]:
+                    g.replay()
+                stream.synchronize()
+                ctr = smtm.smtm_cache_get_counters(cache)
+                check["gpu_exits"] = [int(v) for v in ctr[: w.L]]
+                check["near_threshold_lookups"] = int(ctr[smtm.CTR_NEAR])
+        restart()
+        ctr0 = smtm.smtm_cache_get_counters(cache)
+        if check is not None and "gpu_exits" in check:
+            check["gpu_exits"] = [a - int(b) for a, b in zip(check["gpu_exits"], ctr0[: w.L])]
+            check["near_threshold_lookups"] -= int(ctr0[smtm.CTR_NEAR])
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler = ClockSampler(local_rank)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        start.record(stream)
+        for g in order:
+            g.replay()
+        stop.record(stream)
+        torch.cuda.synchronize()
+        ctr = smtm.smtm_cache_get_counters(cache) - ctr0
+        # The timed region lasts milliseconds, less than one sampling period of nvidia-smi: the same graphs
+        # are replayed for a quarter of a second more (untimed) so that the clocks are read under this load.
+        t_end = time.perf_counter() + 0.25
+        while time.perf_counter() < t_end:
+            for g in order:
+                g.replay()
+            stream.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    clocks["sampled"] = "timed region plus 0.25 s more of the same graphs, untimed"
+    ms_local = start.elapsed_time(stop)
+    out = {
+        "w": w, "res": res, "cents": cents, "counts": counts, "sid": sid, "sh": sh, "G": G, "R": R,
+        "ms_local": ms_local, "clocks": clocks, "launches": int(launches_per_graph * len(order)),
+        "exits": [int(v) for v in ctr[: w.L]], "near": int(ctr[smtm.CTR_NEAR]),
+        "status": smtm.smtm_cache_status(cache), "routes": [int(v) for v in smtm.smtm_cache_get_routes(cache)],
+    }
+    if check is not None and "gpu_exits" not in check:
+        check["gpu_exits"], check["near_threshold_lookups"] = out["exits"], out["near"]
+    # per-kernel figures of the profiled steps
+    ev = [smtm.smtm_cache_get_profile(cache, l) for l in range(w.L)]
+    out["event_us"] = [tot / max(n, 1) * 1e3 for tot, n in ev]
+    out["event_n"] = [int(n) for _, n in ev]
+    dev_total, dev_cnt = smtm.smtm_cache_get_profile_device(cache)
+    names = ["lookup_layer%d" % l for l in range(w.L)] + ["update_plan", "update_centers", "update_tables", "score_tc"]
+    idx = list(range(w.L)) + [smtm.PROF_PLAN, smtm.PROF_CENTERS, smtm.PROF_TABLES, smtm.PROF_SCORE_TC]
+    out["device_us"] = {nm: (float(dev_total[i]) / int(dev_cnt[i]) * 1e3 if dev_cnt[i] else None) for nm, i in zip(names, idx)}
+    out["device_n"] = int(dev_cnt[0])
+    smtm.smtm_cache_destroy(cache)
+
+    if check is not None:   # the oracle over the same steps, from a fresh memory
+        run = OracleRun(w, threads=1)
+        for t in range(W + V):
+            run.step([m.cpu() for m in res.maps[t % R]], res.fallback_host(t))
+        before = run.exits_after[W - 1] if W > 0 else np.zeros(w.L, np.int64)
+        check["oracle_exits"] = [int(a - b) for a, b in zip(run.exits_after[-1], before)]
+        diff = sum(abs(a - b) for a, b in zip(check["gpu_exits"], check["oracle_exits"]))
+        # a decision within 1e-4 of the threshold may fall either way; anything beyond that is an error
+        check["match"] = diff <= 2 * (check["near_threshold_lookups"] + run.mem.near_count)
+        check["frames"] = V * w.B
+        out["oracle_check"] = check
+        out["oracle_run"] = run
+    return out
+
+
+def roofline_of(w, m, peak, layer=0):
+    """Roofline figures of the streaming kernel of `layer`: algorithmic bytes of one launch over its duration.
+    Layer 0 sees every frame of the batch (the batch starts there)."""
+    C = w.stages[layer][0]
+    nbytes = w.B * (w.frame_bytes(layer) + 4 * C)
+    us_ev, us_dev = m["event_us"][layer], m["device_us"]["lookup_layer%d" % layer]
+    ach = nbytes / (us_ev * 1e-6) / 1e9 if us_ev else None
+    ach_dev = nbytes / (us_dev * 1e-6) / 1e9 if us_dev else None
+    return nbytes, us_ev, ach, us_dev, ach_dev
 
 
 def run_ours(args):
@@ -153,99 +462,16 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     # every rank serves its own 512 streams (weak scaling by stream); no data-path collective
     base = si.WORKLOADS[[k for k in si.WORKLOADS if k.startswith(args.workload)][0]]
-    w = shard_for_rank(base, rank)
+    w = shard_for_rank(base, rank) if base.T > 1 else base
     K, W = args.steps, args.warmup
-    G = math.gcd(K, 32)         # steps captured into one CUDA graph
-    while G > 1 and G > w.T:    # not more than the workload has
-        G //= 2
-    m = G if G % 2 == 0 else 2 * G   # resident steps: a whole number of graphs, and even (two carries alternate)
-    T = min(w.T, max(K, W, m))
-    T = max(m, T - T % m)
-    labs = si.labels(w)
-    cents, counts = si.initial_centers(w)
-    sid = si.stream_ids(w)
-    maps, fmaps, fbs = [], [], []
-    for t in range(T):
-        m = [si.frames(w, l, labs[t], t, device="cuda") for l in range(w.L)]
-        maps.append(m)
-        fmaps.append([smtm.Fmap(m[l], w.dtype, w.layout, *si.shape4(w, l)) for l in range(w.L)])
-        fbs.append(torch.from_numpy(si.fallback_labels(w, labs[t])).cuda())
-    torch.cuda.synchronize()
-    # All launches go to one side stream so that every step can be captured into a CUDA graph.
-    stream = torch.cuda.Stream()
-    sh = stream.cuda_stream
-    PROFILE_EVERY = 16  # every 16th step carries timing events and device-clock stamps (they cost a few us and break the chain of launches)
+    peak, tc_peak, peak_src = measured_peaks()
+    with_oracle = rank == 0 and world == 1 and not args.no_cpu_baseline
+    verify = min(K, max(w.T - W, 0) if w.T > 1 else 4) if with_oracle else 0
+    m = measure(smtm, w, K, W, local_rank, world, verify_steps=verify)
+    value, ms = job_throughput(K * w.B, m["ms_local"], world)
+    dom_bytes, dom_us, achieved, dev_us, dev_ach = roofline_of(w, m, peak)
 
-    def step(cache, gbs, t):
-        gb = gbs[t % 2]   # two carries alternate: the cache was created with FLAG_MAPS_READY (maps are resident)
-        smtm.smtm_lookup_exit_begin(cache, 0, fmaps[t % T][0], gb, sh)     # starts the batch: no separate reset
-        for l in range(1, w.L):
-            smtm.smtm_lookup_exit(cache, l, fmaps[t % T][l], gb, sh)
-        smtm.smtm_cache_update_resize(cache, gb, fbs[t % T], sh)
-
-    cache = make_cache(smtm, w, cents, counts)
-    gb = [smtm.Batch(cache, w.B, stream_id=sid, with_diagnostics=False) for _ in range(2)]
-    with torch.cuda.stream(stream):
-        for t in range(W):          # eager warm-up: kernels, clocks, one-time function attributes
-            step(cache, gb, t)
-        stream.synchronize()
-        # One graph per G resident steps (their feature maps are baked in); the cache state lives in
-        # device memory the graphs point to, so replaying them in order advances it as eager calls
-        # would.  Inside a graph the kernels of consecutive steps are chained like those of one step.
-        smtm.smtm_cache_profile(cache, (T // PROFILE_EVERY + 1) * w.L, PROFILE_EVERY)
-        launches0 = smtm.smtm_cache_get_launches(cache)
-        graphs = []
-        for g0 in range(0, T, G):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                for t in range(g0, g0 + G):
-                    step(cache, gb, t)
-            graphs.append(g)
-        launches_per_cycle = smtm.smtm_cache_get_launches(cache) - launches0
-        for g in graphs:   # every graph once, untimed: its first launch uploads it to the device
-            g.replay()
-        stream.synchronize()
-        ctr0 = smtm.smtm_cache_get_counters(cache)
-        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        sampler = ClockSampler(local_rank)
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-        sampler.start()
-        start.record(stream)
-        for i in range(K // G):
-            graphs[i % len(graphs)].replay()
-        stop.record(stream)
-        torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    clocks = sampler.stop()
-    ms = start.elapsed_time(stop)
-    launches = launches_per_cycle * K // T
-    ctr = smtm.smtm_cache_get_counters(cache) - ctr0
-    status = smtm.smtm_cache_status(cache)
-    value, ms = job_throughput(K * w.B, ms, world)
-
-    # roofline of the dominant launch (stage-3 lookup: every frame active)
-    dom_total_ms, dom_n = smtm.smtm_cache_get_profile(cache, 0)
-    dom_ms = dom_total_ms / max(dom_n, 1)
-    dev_total, dev_cnt = smtm.smtm_cache_get_profile_device(cache)
-    dev_n = int(dev_cnt[0])
-    dev_ms = float(dev_total[0]) / dev_n if dev_n else None
-    dev_names = ["lookup_layer%d" % l for l in range(w.L)] + ["update_plan", "update_centers", "update_tables"]
-    dev_idx = list(range(w.L)) + [smtm.PROF_PLAN, smtm.PROF_CENTERS, smtm.PROF_TABLES]
-    dev_us = {nm: (float(dev_total[i]) / int(dev_cnt[i]) * 1e3 if dev_cnt[i] else None) for nm, i in zip(dev_names, dev_idx)}
-    l1_total_ms, l1_n = smtm.smtm_cache_get_profile(cache, 1) if w.L > 1 else (0.0, 0)
-    C0 = w.stages[0][0]
-    dom_bytes = w.B * (w.frame_bytes(0) + 4 * C0)
-    peak, peak_src = measured_peaks()
-    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
-    exits = [int(v) for v in ctr[: w.L]]
-    sid = sid if w.S > 1 else None
-
-    e2e = None
-    if rank == 0 or world > 1:
-        e2e = run_e2e(smtm, w, cents, counts, labs, maps, sid if w.S > 1 else None, min(K, 16), world, sh)
+    e2e = run_e2e(smtm, w, m, min(K, 16), world)
     out = None
     if rank == 0:
         out = {
@@ -257,47 +483,115 @@ def run_ours(args):
                        "map_dtype": {si.F32: "f32", si.F16: "f16", si.BF16: "bf16"}[w.dtype],
                        "layout": "NCHW" if w.layout == si.NCHW else "NHWC",
                        "classes": w.n, "fast_memory": [w.k_min, w.k_max], "tau": w.tau, "window_W": w.window_W,
-                       "distinct_steps_resident": T, "l2_policy": "distinct maps per step, %.0f MB per step (L2 is 126 MB)" % (sum(w.B * w.frame_bytes(l) for l in range(w.L)) / 1e6),
+                       "timed_steps": [W, W + K], "workload_steps": w.T, "distinct_steps_resident": m["R"],
+                       "l2_policy": "distinct maps per step, %.0f MB per step (L2 is 126 MB)" % (m["res"].step_bytes / 1e6),
+                       "state": "the memory is put back to its state after step W-1 (smtm_cache_import) right before the timed region",
                        "sharding": "streams across GPUs, no collective",
-                       "launch": "CUDA graphs of %d steps (per step: %d lookups, update+refresh), chained launches, SMTM_FLAG_MAPS_READY with two alternating carries" % (G, w.L)},
+                       "launch": "CUDA graphs of %d steps (per step: %d lookups, update+refresh), chained launches, SMTM_FLAG_MAPS_READY with two alternating carries" % (m["G"], w.L)},
             "e2e": e2e,
-            "gpu_launches": int(launches),
-            "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "streaming kernel of the first exit layer (fused encode + similarity scoring where the fast memory has <= 64 entries), %d frames per launch" % w.B, "achieved": achieved,
-                         "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                         "traffic": ncu_traffic(base.name, w.B, base.B), "bytes_per_launch": dom_bytes, "us_per_launch": dom_ms * 1e3,
-                         "frac_of_nominal_8TBs": achieved / 8000.0, "launches_timed": int(dom_n),
-                         "stage4_kernel_us_per_launch": l1_total_ms / max(l1_n, 1) * 1e3,
-                         "device_clock": None if dev_ms is None else {
-                             "us_per_launch": dev_ms * 1e3, "achieved": dom_bytes / (dev_ms * 1e-3) / 1e9,
-                             "frac": dom_bytes / (dev_ms * 1e-3) / 1e9 / peak, "launches_timed": int(dev_n),
-                             "note": "first CTA's start to last CTA's end by %globaltimer; the CUDA-event figure above also holds the two event nodes around the kernel"}},
-            "step_kernels_device_clock_us": dev_us,
-            "exit_histogram": {"per_layer": exits, "none": K * w.B - sum(exits)},
-            "near_threshold_lookups": int(ctr[smtm.CTR_NEAR]),
-            "device_status": status,
+            "gpu_launches": m["launches"],
+            "clocks": m["clocks"],
+            "roofline": {"bound": "hbm", "kernel": "streaming kernel of the first exit layer (fused encode + similarity scoring where the fast memory has <= 64 entries), %d frames per launch" % w.B,
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak if achieved else None,
+                         "peak_source": peak_src, "traffic": ncu_traffic(base.name, w.B, base.B),
+                         "bytes_per_launch": dom_bytes, "us_per_launch": dom_us,
+                         "frac_of_nominal_8TBs": achieved / 8000.0 if achieved else None, "launches_timed": m["event_n"][0],
+                         "later_layers_kernel_us_per_launch": m["event_us"][1:],
+                         "device_clock": None if dev_us is None else {
+                             "us_per_launch": dev_us, "achieved": dev_ach, "frac": dev_ach / peak, "launches_timed": m["device_n"],
+                             "note": "first CTA's start to last CTA's end by %globaltimer; the CUDA-event figure above also holds the two event nodes around the kernel"},
+                         "whole_step": {"bytes": None, "achieved": None, "frac": None}},
+            "step_kernels_device_clock_us": m["device_us"],
+            "exit_histogram": {"per_layer": m["exits"], "none": K * w.B - sum(m["exits"])},
+            "near_threshold_lookups": m["near"],
+            "routes": dict(zip(("fused", "dense", "plain"), m["routes"])),
+            "device_status": m["status"],
         }
-        if world == 1 and not args.no_cpu_baseline:
-            out["cpu_baseline"] = cpu_baseline(w, budget_s=12.0)
-    smtm.smtm_cache_destroy(cache)
+        # bytes the whole step had to move (maps of the frames still in at each layer + their SV rows) over the step time
+        step_bytes = w.B * (w.frame_bytes(0) + 4 * w.stages[0][0])
+        left = K * w.B
+        for l in range(1, w.L):
+            left -= m["exits"][l - 1]
+            step_bytes += left / K * (w.frame_bytes(l) + 4 * w.stages[l][0])
+        ws = step_bytes / (ms / K * 1e-3) / 1e9
+        out["roofline"]["whole_step"] = {"bytes": int(step_bytes), "achieved": ws, "frac": ws / peak}
+        if "oracle_check" in m:
+            out["oracle_check"] = m["oracle_check"]
+            run = m["oracle_run"]
+            out["cpu_baseline"] = {"value": run.frames / run.seconds, "unit": "frames/s", "cores": 1, "kind": "oracle",
+                                   "sample": f"steps 0..{len(run.exits_after) - 1} of {w.name} at full width ({w.B} frames per step), oracle time only",
+                                   "host_cores_available": os.cpu_count()}
+            out["cpu_baseline_all_cores"] = cpu_all_cores(w, m, run, budget_s=10.0)
+    del m["res"]
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_other_workloads and base.name == WORKLOAD.name:
+        out["other_workloads"] = [other_workload(smtm, si.WORKLOADS[k], peak, tc_peak, with_oracle)
+                                  for k in si.WORKLOADS if k[:2] in ("c1", "c2", "c3", "c4")]
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+    if out is not None and "oracle_check" in out and not out["oracle_check"]["match"]:
+        print(json.dumps(out))
+        sys.exit("exit histogram of the timed steps differs from the oracle's: %r" % (out["oracle_check"],))
     return out
 
 
-def run_e2e(smtm, w, cents, counts, labs, maps, sid, K, world, sh):
+def cpu_all_cores(w, m, serial_run, budget_s):
+    """The oracle with the frames of a step split over all host cores, from a fresh memory; its exits must be
+    the single-thread run's."""
+    cores = os.cpu_count() or 1
+    run = OracleRun(w, threads=cores)
+    res = m["res"]
+    t = 0
+    while t < len(serial_run.exits_after) and run.seconds < budget_s:
+        run.step([mm.cpu() for mm in res.maps[t % res.R]], res.fallback_host(t))
+        t += 1
+    run.close()
+    same = all(np.array_equal(a, b) for a, b in zip(run.exits_after, serial_run.exits_after))
+    return {"value": run.frames / run.seconds, "unit": "frames/s", "cores": cores, "kind": "oracle",
+            "sample": f"steps 0..{t - 1} of {w.name}, frames of a step split over {cores} threads, oracle time only",
+            "same_exits_as_one_thread": bool(same)}
+
+
+def other_workload(smtm, w, peak, tc_peak, with_oracle):
+    """A short pass of one of the single-batch workloads: the same machinery, fewer steps."""
+    K, W = 16, 3
+    m = measure(smtm, w, K, W, 0, 1, verify_steps=(1 if w.n >= 1000 else 4) if with_oracle else 0)
+    nbytes, us_ev, ach, us_dev, ach_dev = roofline_of(w, m, peak)
+    ms = m["ms_local"] / K
+    out = {"workload": w.name, "steps": K, "warmup": W, "ms_per_step": ms, "frames_per_s": w.B / (ms * 1e-3),
+           "dominant_kernel_us": us_dev if us_dev else us_ev, "dominant_kernel_us_cuda_events": us_ev,
+           "frac": (ach_dev if ach_dev else ach) / peak if (ach_dev or ach) else None,
+           "bytes_per_launch": nbytes, "routes": dict(zip(("fused", "dense", "plain"), m["routes"])),
+           "exit_histogram": {"per_layer": m["exits"], "none": K * w.B - sum(m["exits"])},
+           "near_threshold_lookups": m["near"], "step_kernels_device_clock_us": m["device_us"],
+           "distinct_steps_resident": m["R"], "device_status": m["status"]}
+    step_bytes = sum(w.B * w.frame_bytes(l) for l in range(w.L))
+    out["hbm_floor_us_all_frames_active"] = step_bytes / (peak * 1e9) * 1e6
+    if m["device_us"].get("score_tc"):   # Eq. 1 as a dense contraction: three bf16 products of B x n x D
+        flops = 3 * 2.0 * w.B * w.n * w.stages[0][0]
+        out["score_tc"] = {"us": m["device_us"]["score_tc"], "tflops_split_bf16": flops / (m["device_us"]["score_tc"] * 1e-6) / 1e12,
+                           "frac_of_bf16_peak": flops / (m["device_us"]["score_tc"] * 1e-6) / 1e12 / tc_peak}
+    if "oracle_check" in m:
+        out["oracle_check"] = m["oracle_check"]
+    del m["res"]
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_e2e(smtm, w, m, K, world):
     """Same metric through smtm_step_host: host buffers in, decisions out, copies inside the timed region."""
-    cache = make_cache(smtm, w, cents, counts)
-    hm = [[m.cpu().pin_memory() for m in maps[t]] for t in range(min(K, len(maps)))]
+    res, sid, sh = m["res"], m["sid"], m["sh"]
+    cache = make_cache(smtm, w, m["cents"], m["counts"])
+    hm = [[x.cpu().pin_memory() for x in res.maps[t]] for t in range(min(K, res.R))]
     fm = [smtm.Fmap(None, w.dtype, w.layout, *si.shape4(w, l)) for l in range(w.L)]
     done = torch.zeros(w.B, dtype=torch.uint8).pin_memory().numpy()
     el = torch.zeros(w.B, dtype=torch.int32).pin_memory().numpy()
     pred = torch.zeros(w.B, dtype=torch.int32).pin_memory().numpy()
-    fbs = [si.fallback_labels(w, labs[t]) for t in range(len(hm))]
+    fbs = [res.fallback_host(t) for t in range(len(hm))]
     smtm.smtm_step_host(cache, fm, hm[0], sid, fbs[0], True, done, el, pred, sh)   # allocates staging
     smtm.smtm_cache_destroy(cache)
-    cache = make_cache(smtm, w, cents, counts)
+    cache = make_cache(smtm, w, m["cents"], m["counts"])
     smtm.smtm_step_host(cache, fm, hm[0], sid, fbs[0], True, done, el, pred, sh)
     torch.cuda.synchronize()
     t0 = time.perf_counter()
@@ -323,36 +617,14 @@ def run_e2e(smtm, w, cents, counts, labs, maps, sid, K, world, sh):
 
 def oracle_steps(w, n_steps, budget_s=None, device="cpu"):
     """Runs the CPU oracle over the first steps of the workload; returns (frames, seconds in the oracle)."""
-    import oracle
-
+    run = OracleRun(w, threads=1)
     labs = si.labels(w)
-    cents, counts = si.initial_centers(w)
-    mem = oracle.OracleMemory(w.n, w.dims, [w.tau] * w.L, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W,
-                              forgetting=w.forgetting)
-    sid = si.stream_ids(w)
-    spent, frames = 0.0, 0
     for t in range(n_steps):
         maps = [si.frames(w, l, labs[t % w.T], t % w.T, device=device).cpu() for l in range(w.L)]
-        fb = si.fallback_labels(w, labs[t % w.T])
-        t0 = time.perf_counter()
-        ob = mem.new_batch(w.B, sid)
-        for l in range(w.L):
-            mem.lookup_exit(l, maps[l], w.dtype, w.layout, si.shape4(w, l), ob)
-        mem.update(ob, fb)
-        mem.resize()
-        spent += time.perf_counter() - t0
-        frames += w.B
-        if budget_s is not None and spent >= budget_s:
+        run.step(maps, si.fallback_labels(w, labs[t % w.T]))
+        if budget_s is not None and run.seconds >= budget_s:
             break
-    return frames, spent
-
-
-def cpu_baseline(w, budget_s):
-    dev = "cuda" if torch.cuda.is_available() else "cpu"
-    frames, spent = oracle_steps(w, 32, budget_s=budget_s, device=dev)
-    return {"value": frames / spent, "unit": "frames/s", "cores": 1, "kind": "oracle",
-            "sample": f"first {frames // w.B} steps of {w.name} at full width ({w.B} streams), oracle time only",
-            "host_cores_available": os.cpu_count()}
+    return run.frames, run.seconds
 
 
 def run_reference(args):
@@ -378,14 +650,21 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=640)
+    ap.add_argument("--steps", type=int, default=60, help="timed steps; warm-up + steps = 64 walks the streaming workload once")
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5", help="c1..c5 (prefix of a workload name); c5 is the benchmark of record")
-    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg (profiling runs)")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle legs (profiling runs)")
+    ap.add_argument("--no-other-workloads", action="store_true", help="skip the short passes of c1..c4")
+    ap.add_argument("--rank-check", action="store_true", help="multi-rank plumbing only, on the host (gloo)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:   # no launcher above us: start the ranks ourselves
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    out = run_reference(args) if args.impl == "reference" else run_ours(args)
+    if args.rank_check:
+        out = rank_check(args)
+    else:
+        out = run_reference(args) if args.impl == "reference" else run_ours(args)
     if out is not None:
         print(json.dumps(out))
 

@@ -67,8 +67,8 @@ enum {
 };
 
 /* Config flag.  SMTM_FLAG_FORGET_FT: the variant the paper uses for rapidly changing scenes
- * (Sec. 7.1, "decay the historical memory in the frequency table" by the forgetting mechanism
- * of Sec. 6.1): the 0.25-per-window decay of Eq. 5 is applied to the frequency table itself.
+ * (Sec. 7.1: the forgetting of Sec. 6.1 applied to the frequency table itself): the
+ * 0.25-per-window decay of Eq. 5 is applied to the stored counts.
  * FT is then fixed point with 10 fractional bits (smtm_cache_get_tables returns it raw): an
  * appearance adds 1024, each further W consecutive unseen frames multiply it by 0.25 rounding
  * down, and Eq. 5's score is FT itself. */
@@ -114,7 +114,10 @@ typedef struct {
  * A layer is looked up at most once per batch. */
 typedef struct {
     int32_t B;
-    const int32_t* d_stream_id; /* [B] fast memory each frame looks up; NULL = all stream 0 */
+    const int32_t* d_stream_id; /* [B] fast memory each frame looks up, in [0, S); NULL = all stream 0.  A frame
+                                   whose id lies outside that range is scored against nothing (AC = 0, it stays
+                                   in), takes no part in the update of tables or centres, and
+                                   SMTM_ERR_INVALID_ARG is recorded in the sticky status word */
     float* d_sa;                /* [B][k_max] cumulative similarity per fast-memory slot (Eq. 3) */
     uint8_t* d_done;            /* [B] 1 once a frame has exited; later lookups skip it, reading none of its map */
     int32_t* d_exit_layer;      /* [B] 0 = not exited, else the paper's l in 1..L */
@@ -193,7 +196,9 @@ smtm_status_t smtm_lookup_exit_begin(smtm_cache_t* cache, int32_t layer, const s
  * up the array's device address; make that first call outside any stream
  * capture.  All calls on a device share the one array, which keeps the previous
  * call's contents (the call clears what it accumulates into): two calls whose
- * GPU work overlaps, e.g. on different streams, race on it. */
+ * GPU work overlaps, e.g. on different streams, race on it.  Calls on one stream
+ * are ordered: the entry never uses the early start of SMTM_FLAG_MAPS_READY, so
+ * nothing of the array is touched before the stream's previous kernel is done. */
 enum { SMTM_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024 };
 smtm_status_t smtm_lookup_exit_static(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t* fmap,
                                       const int32_t* d_stream_id, uint8_t* d_exit, int32_t* d_pred,
@@ -223,8 +228,8 @@ smtm_status_t smtm_cache_update(smtm_cache_t* cache, const smtm_batch_t* batch,
 smtm_status_t smtm_cache_update_resize(smtm_cache_t* cache, const smtm_batch_t* batch,
                                        const int32_t* d_fallback_label, void* stream);
 
-/* Centre warm-up (Sec. 5: the centres are "initialized with a grouping center (the
- * average of semantic vectors) on the training dataset"; Sec. 6.3): encodes a batch
+/* Centre warm-up (Sec. 5 / Sec. 6.3: a centre starts as the mean semantic vector of
+ * its class over training frames): encodes a batch
  * of labelled frames at `layer` and folds each into the centre of its class
  * d_labels[b] (-1 = skip) by Eq. 7 in ascending frame order; a centre created with
  * count 0 thereby becomes the class mean.  Tables and fast memories are not touched.
@@ -277,9 +282,12 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * each kernel of the step ran by the device's own clock, from the moment its
  * first CTA began (after its wait for the previous kernel) to the moment its
  * last CTA ended: h_total_ms[i] and h_count[i], i < SMTM_PROF_KERNELS, are the
- * sum over the profiled steps and their number, for the fused lookup kernel of
- * layer i (i < SMTM_MAX_LAYERS; lookups that took another route count zero)
- * and for the three update kernels (SMTM_PROF_PLAN, _CENTERS, _TABLES).  This
+ * sum over the profiled steps and their number, for the streaming kernel of
+ * layer i (i < SMTM_MAX_LAYERS: the fused lookup kernel, or the pooling kernel
+ * of the other routes), for the three update kernels (SMTM_PROF_PLAN, _CENTERS,
+ * _TABLES) and for the tensor-core scorer of the dense route
+ * (SMTM_PROF_SCORE_TC; with several dense layers in a step, from the first
+ * one's begin to the last one's end).  This
  * leaves out what the event nodes add around a kernel.  Only the most recent
  * run of each profiled step is kept.  smtm_cache_get_profile_timeline gives the
  * two stamps themselves for the step-th profiled step (counted from 0;
@@ -288,7 +296,7 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * timer, both 0 for a kernel that did not run in that step, so that the gaps
  * between the kernels of a step can be read off.  All four synchronise the
  * device. */
-enum { SMTM_PROF_PLAN = SMTM_MAX_LAYERS, SMTM_PROF_CENTERS, SMTM_PROF_TABLES, SMTM_PROF_KERNELS };
+enum { SMTM_PROF_PLAN = SMTM_MAX_LAYERS, SMTM_PROF_CENTERS, SMTM_PROF_TABLES, SMTM_PROF_SCORE_TC, SMTM_PROF_KERNELS };
 smtm_status_t smtm_cache_profile(smtm_cache_t* cache, int32_t max_lookups, int32_t every);
 smtm_status_t smtm_cache_get_profile(smtm_cache_t* cache, int32_t layer, double* h_total_ms, int64_t* h_count);
 smtm_status_t smtm_cache_get_profile_device(smtm_cache_t* cache, double* h_total_ms /*[SMTM_PROF_KERNELS]*/,
@@ -299,6 +307,32 @@ smtm_status_t smtm_cache_get_profile_timeline(smtm_cache_t* cache, int64_t step,
 
 /* Number of kernels the library has launched on behalf of this cache so far. */
 smtm_status_t smtm_cache_get_launches(smtm_cache_t* cache, int64_t* h_out);
+
+/* How many lookups (smtm_lookup_exit, _begin, _static and the lookups inside smtm_step_host) each
+ * route has served so far.  Eq. 1 is evaluated on one of three routes, chosen from the shape:
+ *   SMTM_ROUTE_FUSED  pooling, Eq. 1, Eq. 3, Eq. 4 and the exit rule in one streaming kernel
+ *                     (fast memories of at most 64 entries; NCHW shapes and NHWC shapes whose
+ *                     pixel rows are multiples of 16 bytes);
+ *   SMTM_ROUTE_DENSE  fast memories above 64 entries: pooling, then Eq. 1's dot products against
+ *                     every class on the tensor cores, then a finishing kernel;
+ *   SMTM_ROUTE_PLAIN  everything else: pooling, then a CUDA-core scoring kernel. */
+enum { SMTM_ROUTE_FUSED = 0, SMTM_ROUTE_DENSE = 1, SMTM_ROUTE_PLAIN = 2, SMTM_ROUTE_COUNT = 3 };
+smtm_status_t smtm_cache_get_routes(smtm_cache_t* cache, int64_t* h_out /*[SMTM_ROUTE_COUNT]*/);
+
+/* Snapshot of the memory of Sec. 6 (the paper keeps it for the life of the application; a host copy
+ * lets a caller put a cache back into a known state, or carry it to another process): semantic centres
+ * (with their lengths) and their update counts m (Eq. 7) of every layer, frequency and time-stamp tables (Sec. 6.1), the
+ * fast memories and their sizes (Eq. 5, Eq. 6), and the counters.  smtm_cache_export_size gives the
+ * size of the blob; smtm_cache_export writes it to h_blob (`bytes` = the room there, SMTM_ERR_SHAPE if
+ * too small); smtm_cache_import reads one back into a cache of the same shape (n, L, C_l, S, k_max and
+ * the forgetting flag must match: SMTM_ERR_SHAPE otherwise; a blob that is not a snapshot, or whose
+ * fast memories name classes outside [0, n), SMTM_ERR_INVALID_ARG); the steps that follow give bit for
+ * bit what they gave after the export.  Nothing is changed when an error is returned.  The blob's layout is
+ * private to one build of the library.  All three synchronise the device; profiling records and the
+ * sticky status word are not part of the snapshot. */
+smtm_status_t smtm_cache_export_size(smtm_cache_t* cache, uint64_t* h_bytes);
+smtm_status_t smtm_cache_export(smtm_cache_t* cache, void* h_blob, uint64_t bytes);
+smtm_status_t smtm_cache_import(smtm_cache_t* cache, const void* h_blob, uint64_t bytes);
 
 /* Reads the sticky device status word (synchronises the device): SMTM_OK or
  * the first device-side error recorded since creation. */

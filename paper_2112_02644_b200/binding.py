@@ -100,6 +100,10 @@ def load_library():
     lib.smtm_cache_get_tables.argtypes = [vp, vp, vp]
     lib.smtm_cache_get_counters.argtypes = [vp, vp]
     lib.smtm_cache_get_launches.argtypes = [vp, vp]
+    lib.smtm_cache_get_routes.argtypes = [vp, vp]
+    lib.smtm_cache_export_size.argtypes = [vp, vp]
+    lib.smtm_cache_export.argtypes = [vp, vp, ctypes.c_uint64]
+    lib.smtm_cache_import.argtypes = [vp, vp, ctypes.c_uint64]
     lib.smtm_cache_profile.argtypes = [vp, i32, i32]
     lib.smtm_cache_get_profile.argtypes = [vp, i32, vp, vp]
     lib.smtm_cache_get_profile_device.argtypes = [vp, vp, vp]
@@ -321,6 +325,31 @@ def smtm_cache_get_launches(cache: Cache) -> int:
     return int(out[0])
 
 
+ROUTE_FUSED, ROUTE_DENSE, ROUTE_PLAIN, ROUTE_COUNT = 0, 1, 2, 3
+
+
+def smtm_cache_get_routes(cache: Cache) -> np.ndarray:
+    """Lookups served so far by the fused, the dense (tensor-core) and the plain route."""
+    out = np.zeros(ROUTE_COUNT, np.int64)
+    _check(load_library().smtm_cache_get_routes(cache.handle, out.ctypes.data), "smtm_cache_get_routes")
+    return out
+
+
+def smtm_cache_export(cache: Cache) -> np.ndarray:
+    """Snapshot of the memory (centres, counts, tables, fast memories, counters) as a host byte array."""
+    size = ctypes.c_uint64(0)
+    _check(load_library().smtm_cache_export_size(cache.handle, ctypes.byref(size)), "smtm_cache_export_size")
+    blob = np.zeros(size.value, np.uint8)
+    _check(load_library().smtm_cache_export(cache.handle, blob.ctypes.data, blob.nbytes), "smtm_cache_export")
+    return blob
+
+
+def smtm_cache_import(cache: Cache, blob: np.ndarray) -> None:
+    """Puts a cache of the same shape back into the state a snapshot holds."""
+    assert isinstance(blob, np.ndarray) and blob.dtype == np.uint8 and blob.flags.c_contiguous
+    _check(load_library().smtm_cache_import(cache.handle, blob.ctypes.data, blob.nbytes), "smtm_cache_import")
+
+
 def smtm_cache_profile(cache: Cache, max_lookups: int, every: int = 1) -> None:
     _check(load_library().smtm_cache_profile(cache.handle, int(max_lookups), int(every)), "smtm_cache_profile")
 
@@ -334,7 +363,8 @@ def smtm_cache_get_profile(cache: Cache, layer: int):
     return total.value, count.value
 
 
-PROF_PLAN, PROF_CENTERS, PROF_TABLES, PROF_KERNELS = MAX_LAYERS, MAX_LAYERS + 1, MAX_LAYERS + 2, MAX_LAYERS + 3
+PROF_PLAN, PROF_CENTERS, PROF_TABLES, PROF_SCORE_TC, PROF_KERNELS = (MAX_LAYERS, MAX_LAYERS + 1, MAX_LAYERS + 2, MAX_LAYERS + 3,
+                                                                    MAX_LAYERS + 4)
 
 
 def smtm_cache_get_profile_device(cache: Cache):

@@ -1,5 +1,7 @@
 // C ABI of the SMTM library: argument checking, state ownership and launch planning.
 // Every step of the path runs in the kernels of encode.cu, lookup.cu and memory.cu.
+#include <string.h>
+
 #include <new>
 #include <vector>
 
@@ -44,6 +46,8 @@ struct smtm_cache {
     long long prof_seq;                     // lookup calls since profiling was switched on
     int device, sm_count;
     int64_t launches;
+    int64_t routes[SMTM_ROUTE_COUNT];  // lookups served by each route (a host-side decision, counted on the host)
+    FusedCaps fused_caps;              // cluster capacities of the fused kernel on this cache's device
     // device-side carry and staging used only by smtm_step_host (allocated on first use)
     bool host_ready;
     smtm_batch_t hb;
@@ -186,6 +190,8 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     a.sep = b->d_sep;
     a.top = b->d_top;
     a.counters = c->d_counters;
+    a.S = c->S;
+    a.status = c->d_status;
     const EncodeArgs e = encode_args(c, f, b->d_done, b->d_sv[layer]);
     bool fused = false;
     const cudaEvent_t* timing = nullptr;
@@ -202,14 +208,19 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
         timing = c->prof_events->data() + 2 * c->prof_used;
         (*c->prof_layer)[c->prof_used++] = layer;
     }
-    SMTM_CUDA(launch_lookup_fused(e, a, c->sm_count, st, &c->launches, &fused, timing));
-    if (fused) return SMTM_OK;
+    SMTM_CUDA(launch_lookup_fused(e, a, c->sm_count, &c->fused_caps, st, &c->launches, &fused, timing));
+    if (fused) {
+        ++c->routes[SMTM_ROUTE_FUSED];
+        return SMTM_OK;
+    }
     const bool dense = c->d_dense && dense_scoring_supported(a.D, a.n);  // large fast memory: tensor cores
+    ++c->routes[dense ? SMTM_ROUTE_DENSE : SMTM_ROUTE_PLAIN];
     if (begin && !dense) {  // the plain route reads the carry: put it into its reset state with a kernel of its own
         SMTM_CUDA(launch_batch_reset(b->d_sa, b->d_done, b->d_exit_layer, b->d_pred, b->B, c->k_max, st, &c->launches));
         a.fresh = 0;
     }
     EncodeArgs e2 = e;
+    e2.clock = a.clock ? a.clock + 2 * layer : nullptr;  // the pooling kernel is this layer's streaming kernel
     if (a.fresh) e2.skip = nullptr;  // a batch that starts here: every frame is in, whatever the flags hold
     if (dense) dense_sv_split(c->d_dense, c->max_batch, c->d_max, &e2.sv_hi, &e2.sv_lo);
     bool sv_split = false;
@@ -220,7 +231,7 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
         float *dots = nullptr, *dots2 = nullptr;
         SMTM_CUDA(launch_dense_dots(a.sv, a.fresh ? nullptr : a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max,
                                     sv_split, c->d_cen_split[layer], c->d_split_current + layer, &dots, &dots2, c->d_status,
-                                    st, &c->launches));
+                                    a.clock ? a.clock + 2 * SMTM_PROF_SCORE_TC : nullptr, st, &c->launches));
         SMTM_CUDA(launch_finish_dense(a, dots, dots2, c->d_split_current + layer, st, &c->launches));
         return SMTM_OK;
     }
@@ -268,6 +279,7 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     a.fallback = d_fallback;
     a.clock = c->prof_events ? c->prof_step : nullptr;
     a.split_current = c->d_split_current;
+    a.status = c->d_status;
     a.ft = c->d_ft;
     a.ts = c->d_ts;
     for (int l = 0; l < c->L; ++l) {
@@ -287,6 +299,16 @@ smtm_status_t resize_impl(smtm_cache* c, cudaStream_t st) {
     return SMTM_OK;
 }
 
+smtm_status_t check_lookup(const smtm_cache* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b) {
+    smtm_status_t s = check_fmap(c, layer, f);
+    if (s != SMTM_OK) return s;
+    if ((s = check_batch(c, b)) != SMTM_OK) return s;
+    if (b->B != f->B) return SMTM_ERR_SHAPE;
+    if (!f->d_data || !b->d_sv[layer]) return SMTM_ERR_INVALID_ARG;
+    if (!aligned16(f->d_data) || !aligned16(b->d_sv[layer])) return SMTM_ERR_ALIGN;
+    return SMTM_OK;
+}
+
 smtm_status_t check_update(const smtm_cache* c, const smtm_batch_t* b) {
     if (!c) return SMTM_ERR_INVALID_ARG;
     const smtm_status_t s = check_batch(c, b);
@@ -297,6 +319,13 @@ smtm_status_t check_update(const smtm_cache* c, const smtm_batch_t* b) {
 }
 
 }  // namespace
+
+smtm_status_t smtm::lookup_begin_ordered(smtm_cache_t* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b,
+                                         void* stream) {
+    const smtm_status_t s = check_lookup(c, layer, f, b);
+    if (s != SMTM_OK) return s;
+    return lookup_impl(c, layer, f, b, static_cast<cudaStream_t>(stream), true, false);
+}
 
 extern "C" {
 
@@ -352,7 +381,8 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
         return SMTM_ERR_CUDA;
     }
 
-    bool ok = encode_setup() == cudaSuccess;
+    bool ok = encode_setup() == cudaSuccess && lookup_setup() == cudaSuccess && memory_setup() == cudaSuccess;
+    if (ok && c->k_max > kFusedMaxK) ok = dense_setup() == cudaSuccess;
     for (int l = 0; ok && l < c->L; ++l) {
         const size_t nd = size_t(n) * c->dims[l];
         ok = ok && dev_alloc(&c->d_centers[l], nd) == cudaSuccess;
@@ -454,23 +484,15 @@ smtm_status_t smtm_encode(smtm_cache_t* c, int32_t layer, const smtm_fmap_t* f, 
 
 smtm_status_t smtm_lookup_exit(smtm_cache_t* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b,
                                void* stream) {
-    smtm_status_t s = check_fmap(c, layer, f);
+    const smtm_status_t s = check_lookup(c, layer, f, b);
     if (s != SMTM_OK) return s;
-    if ((s = check_batch(c, b)) != SMTM_OK) return s;
-    if (b->B != f->B) return SMTM_ERR_SHAPE;
-    if (!f->d_data || !b->d_sv[layer]) return SMTM_ERR_INVALID_ARG;
-    if (!aligned16(f->d_data) || !aligned16(b->d_sv[layer])) return SMTM_ERR_ALIGN;
     return lookup_impl(c, layer, f, b, static_cast<cudaStream_t>(stream), false);
 }
 
 smtm_status_t smtm_lookup_exit_begin(smtm_cache_t* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b,
                                      void* stream) {
-    smtm_status_t s = check_fmap(c, layer, f);
+    const smtm_status_t s = check_lookup(c, layer, f, b);
     if (s != SMTM_OK) return s;
-    if ((s = check_batch(c, b)) != SMTM_OK) return s;
-    if (b->B != f->B) return SMTM_ERR_SHAPE;
-    if (!f->d_data || !b->d_sv[layer]) return SMTM_ERR_INVALID_ARG;
-    if (!aligned16(f->d_data) || !aligned16(b->d_sv[layer])) return SMTM_ERR_ALIGN;
     return lookup_impl(c, layer, f, b, static_cast<cudaStream_t>(stream), true);
 }
 
@@ -515,6 +537,7 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
     a.plan.epoch = c->d_epoch;
     a.fallback = d_labels;
     a.split_current = c->d_split_current;
+    a.status = c->d_status;
     a.ft = c->d_ft;
     a.ts = c->d_ts;
     for (int l = 0; l < c->L; ++l) {
@@ -739,6 +762,112 @@ smtm_status_t smtm_cache_get_profile_timeline(smtm_cache_t* c, int64_t step, uin
         h_begin_ns[k] = ran ? begin : 0;
         h_end_ns[k] = ran ? end : 0;
     }
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_get_routes(smtm_cache_t* c, int64_t* h_out) {
+    if (!c || !h_out) return SMTM_ERR_INVALID_ARG;
+    for (int r = 0; r < SMTM_ROUTE_COUNT; ++r) h_out[r] = c->routes[r];
+    return SMTM_OK;
+}
+
+// ---- snapshot of the memory (export / import) ----------------------------------------------------------------
+
+namespace {
+
+struct BlobHeader {
+    uint64_t magic;
+    uint32_t version, n, L, S, k_max, forgetting;
+    uint32_t dims[SMTM_MAX_LAYERS];
+    uint64_t bytes;  // of the whole blob
+};
+constexpr uint64_t kBlobMagic = 0x4d454d2d4d544d53ull;  // "SMTM-MEM"
+
+size_t blob_bytes(const smtm_cache* c) {
+    size_t b = sizeof(BlobHeader);
+    for (int l = 0; l < c->L; ++l)  // centres, their lengths, their counts
+        b += size_t(c->n) * c->dims[l] * sizeof(float) + size_t(c->n) * sizeof(float) + size_t(c->n) * sizeof(uint32_t);
+    b += 2 * size_t(c->S) * c->n * sizeof(int32_t);                        // FT, TS
+    b += size_t(c->S) * c->k_max * sizeof(int32_t) + size_t(c->S) * sizeof(int32_t);  // members, k
+    b += SMTM_CTR_COUNT * sizeof(uint64_t);
+    return b;
+}
+
+// Walks the sections of a blob in their fixed order, copying each to (to_host) or from the device.
+cudaError_t blob_copy(smtm_cache* c, unsigned char* p, bool to_host) {
+    cudaError_t e = cudaSuccess;
+    const auto section = [&](void* dev, size_t bytes) {
+        if (e == cudaSuccess)
+            e = to_host ? cudaMemcpy(p, dev, bytes, cudaMemcpyDeviceToHost) : cudaMemcpy(dev, p, bytes, cudaMemcpyHostToDevice);
+        p += bytes;
+    };
+    for (int l = 0; l < c->L; ++l) {
+        section(c->d_centers[l], size_t(c->n) * c->dims[l] * sizeof(float));
+        section(c->d_cnorm[l], size_t(c->n) * sizeof(float));  // as the kernels left them: recomputing would round differently
+        section(c->d_m[l], size_t(c->n) * sizeof(uint32_t));
+    }
+    section(c->d_ft, size_t(c->S) * c->n * sizeof(int32_t));
+    section(c->d_ts, size_t(c->S) * c->n * sizeof(int32_t));
+    section(c->d_members, size_t(c->S) * c->k_max * sizeof(int32_t));
+    section(c->d_k, size_t(c->S) * sizeof(int32_t));
+    section(c->d_counters, SMTM_CTR_COUNT * sizeof(uint64_t));
+    return e;
+}
+
+}  // namespace
+
+smtm_status_t smtm_cache_export_size(smtm_cache_t* c, uint64_t* h_bytes) {
+    if (!c || !h_bytes) return SMTM_ERR_INVALID_ARG;
+    *h_bytes = blob_bytes(c);
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_export(smtm_cache_t* c, void* h_blob, uint64_t bytes) {
+    if (!c || !h_blob) return SMTM_ERR_INVALID_ARG;
+    if (bytes < blob_bytes(c)) return SMTM_ERR_SHAPE;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    BlobHeader h{};
+    h.magic = kBlobMagic;
+    h.version = 1;
+    h.n = uint32_t(c->n);
+    h.L = uint32_t(c->L);
+    h.S = uint32_t(c->S);
+    h.k_max = uint32_t(c->k_max);
+    h.forgetting = c->forgetting ? 1u : 0u;
+    for (int l = 0; l < c->L; ++l) h.dims[l] = uint32_t(c->dims[l]);
+    h.bytes = blob_bytes(c);
+    unsigned char* p = static_cast<unsigned char*>(h_blob);
+    memcpy(p, &h, sizeof(h));
+    SMTM_CUDA(blob_copy(c, p + sizeof(h), true));
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_import(smtm_cache_t* c, const void* h_blob, uint64_t bytes) {
+    if (!c || !h_blob) return SMTM_ERR_INVALID_ARG;
+    if (bytes < sizeof(BlobHeader)) return SMTM_ERR_SHAPE;
+    BlobHeader h;
+    memcpy(&h, h_blob, sizeof(h));
+    if (h.magic != kBlobMagic || h.version != 1) return SMTM_ERR_INVALID_ARG;
+    bool same = h.n == uint32_t(c->n) && h.L == uint32_t(c->L) && h.S == uint32_t(c->S) && h.k_max == uint32_t(c->k_max) &&
+                h.forgetting == (c->forgetting ? 1u : 0u) && h.bytes == blob_bytes(c) && bytes >= h.bytes;
+    for (int l = 0; same && l < c->L; ++l) same = h.dims[l] == uint32_t(c->dims[l]);
+    if (!same) return SMTM_ERR_SHAPE;  // a snapshot of a memory of another shape
+    // the sections are checked before anything is overwritten: sizes in range, members inside the memory
+    const unsigned char* p = static_cast<const unsigned char*>(h_blob) + sizeof(h);
+    for (int l = 0; l < c->L; ++l)
+        p += size_t(c->n) * c->dims[l] * sizeof(float) + size_t(c->n) * sizeof(float) + size_t(c->n) * sizeof(uint32_t);
+    p += 2 * size_t(c->S) * c->n * sizeof(int32_t);
+    const int32_t* members = reinterpret_cast<const int32_t*>(p);
+    const int32_t* ks = members + size_t(c->S) * c->k_max;
+    for (size_t i = 0; i < size_t(c->S) * c->k_max; ++i)
+        if (members[i] < 0 || members[i] >= c->n) return SMTM_ERR_INVALID_ARG;
+    for (int s = 0; s < c->S; ++s)
+        if (ks[s] < 1 || ks[s] > c->k_max) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    SMTM_CUDA(blob_copy(c, const_cast<unsigned char*>(static_cast<const unsigned char*>(h_blob)) + sizeof(h), false));
+    // the tensor-core scorer's bf16 copy of the centres is derived from them: stale now
+    if (c->d_split_current) SMTM_CUDA(cudaMemset(c->d_split_current, 0, SMTM_MAX_LAYERS * sizeof(int)));
+    SMTM_CUDA(cudaDeviceSynchronize());
     return SMTM_OK;
 }
 

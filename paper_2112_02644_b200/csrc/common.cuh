@@ -12,6 +12,7 @@ constexpr int kWarp = 32;
 constexpr unsigned kFull = 0xffffffffu;
 
 // Error codes written to the sticky device status word (same values as smtm_status_t).
+constexpr int kDevInvalidArg = 1;
 constexpr int kDevTimeout = 8;
 
 __device__ __forceinline__ void set_status(int* status, int code) {

@@ -52,6 +52,7 @@ struct NchwParams {
     int team;                // team-per-channel: lanes per channel (power of two)
     int vec_per_channel;     // team-per-channel: 16-byte vectors per channel
     int max_in_flight;       // copies the producer keeps outstanding (<= kStages)
+    unsigned long long* clock;  // nullptr, or two words for the device-clock stamps of the pooling kernel
 };
 
 // Writes the bf16 head and tail of n consecutive values (n a multiple of 2, dst 4-byte aligned).
@@ -211,6 +212,7 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
     __syncthreads();
     chain_wait();  // the barriers are set up while the previous kernel finishes
     chain_release();
+    const ClockScope stamps(p.clock);
 
     const bool producer = warp == kConsumers;  // last warp; lane 0 issues the copies
     int it = 0;                                // chunks of this CTA that are not skipped, so far
@@ -497,9 +499,9 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         int nx_k = 0, nx_ids[2] = {0, 0};
         if (nu > 0) {
             const int b = my_units[0];
-            const int sid = a.stream_id ? a.stream_id[b] : 0;
-            nx_k = min(a.k[sid], kFusedMaxK);
-            const int32_t* mem = a.members + (size_t)sid * a.k_max;
+            const int sid = stream_of(a, b);
+            nx_k = sid < 0 ? 0 : min(a.k[sid], kFusedMaxK);  // a stream id outside the cache: nothing to score against
+            const int32_t* mem = a.members + (size_t)max(sid, 0) * a.k_max;
             nx_ids[0] = lane < nx_k ? mem[lane] : 0;
             nx_ids[1] = lane + kWarp < nx_k ? mem[lane + kWarp] : 0;
         }
@@ -584,8 +586,9 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
                 peer_arrive(peer_smem(&rx_full[x], fin));  // this warp's share of the part has been delivered
             }
             if (u + 1 < nu) {  // fast memory of the next frame (its stream id has arrived by now)
-                nx_k = min(a.k[nb_sid], kFusedMaxK);
-                const int32_t* mem = a.members + (size_t)nb_sid * a.k_max;
+                nb_sid = stream_checked(a, nb_sid);
+                nx_k = nb_sid < 0 ? 0 : min(a.k[nb_sid], kFusedMaxK);
+                const int32_t* mem = a.members + (size_t)max(nb_sid, 0) * a.k_max;
                 nx_ids[0] = lane < nx_k ? mem[lane] : 0;
                 nx_ids[1] = lane + kWarp < nx_k ? mem[lane + kWarp] : 0;
             }
@@ -668,10 +671,11 @@ template <class E>
 __global__ void __launch_bounds__(kThreadsNhwc) k_encode_nhwc(const uint8_t* __restrict__ x,
                                                               const uint8_t* __restrict__ skip,
                                                               float* __restrict__ sv, int B, int C, int HW,
-                                                              float inv_hw) {
+                                                              float inv_hw, unsigned long long* clock) {
     extern __shared__ float part[];  // [phases][min(C, 256 * kPerVec)]
     chain_wait();
     chain_release();
+    const ClockScope stamps(clock);
     constexpr int V = E::kPerVec;
     const int CG = C / V;            // 16-byte vectors per pixel
     for (int b = blockIdx.x; b < B; b += gridDim.x) {
@@ -725,9 +729,11 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_encode_nhwc(const uint8_t* __r
 
 template <class E>
 __global__ void k_encode_generic(const void* __restrict__ x, const uint8_t* __restrict__ skip,
-                                 float* __restrict__ sv, int B, int C, int HW, int nhwc, float inv_hw) {
+                                 float* __restrict__ sv, int B, int C, int HW, int nhwc, float inv_hw,
+                                 unsigned long long* clock) {
     chain_wait();
     chain_release();
+    const ClockScope stamps(clock);
     const long long total = (long long)B * C;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -774,7 +780,7 @@ cudaError_t launch_generic(const EncodeArgs& a, cudaStream_t st) {
     const long long total = (long long)a.B * a.C;
     const int grid = int(std::min<long long>((total + 255) / 256, 148 * 16));
     return launch_chained(k_encode_generic<E>, grid, 256, 0, st, a.x, a.skip, a.sv, a.B, a.C, a.H * a.W,
-                          int(a.layout == SMTM_NHWC), 1.0f / float(a.H * a.W));
+                          int(a.layout == SMTM_NHWC), 1.0f / float(a.H * a.W), a.clock);
 }
 
 template <class E>
@@ -783,7 +789,7 @@ cudaError_t launch_nhwc(const EncodeArgs& a, cudaStream_t st) {
     const int cgs = std::min(CG, kThreadsNhwc);
     const size_t smem = size_t(kThreadsNhwc / cgs) * cgs * E::kPerVec * sizeof(float);
     return launch_chained(k_encode_nhwc<E>, a.B, kThreadsNhwc, smem, st, static_cast<const uint8_t*>(a.x), a.skip, a.sv,
-                          a.B, a.C, a.H * a.W, 1.0f / float(a.H * a.W));
+                          a.B, a.C, a.H * a.W, 1.0f / float(a.H * a.W), a.clock);
 }
 
 int pow2_floor(int v) {
@@ -812,6 +818,7 @@ Reducer plan_nchw(const EncodeArgs& a, NchwParams* p) {
     p->sv_hi = static_cast<__nv_bfloat16*>(a.sv_hi);
     p->sv_lo = static_cast<__nv_bfloat16*>(a.sv_lo);
     p->status = a.status;
+    p->clock = a.clock;
     p->C = a.C;
     p->ch_bytes = HW * es;
     p->frame_bytes = (long long)a.C * p->ch_bytes;
@@ -919,7 +926,7 @@ cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, in
     return launch_generic<BF16>(a, st);
 }
 
-cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm_count, cudaStream_t st,
+cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm_count, FusedCaps* caps, cudaStream_t st,
                                 int64_t* launches, bool* handled, const cudaEvent_t* timing) {
     *handled = false;
     if (e.B <= 0 || e.layout != SMTM_NCHW || a.k_max > kFusedMaxK) return cudaSuccess;
@@ -927,20 +934,21 @@ cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm
     const Reducer r = plan_nchw(e, &f.e);
     if (r == kNone) return cudaSuccess;
     const int cpf = f.e.chunks_per_frame;
-    if ((e.C & 3) || (f.e.chunk_channels & 3)) return cudaSuccess;
+    if (e.C & 3) return cudaSuccess;
     // Parts per frame = CTAs per cluster.  A part must fit the scorers' registers (slice <= kMaxSlice
     // channels, a multiple of 4) and the CTA's shared memory; among 1, 2, 4, 8 take the smallest
     // that keeps the SMs 95 % busy over the rounds of frames (else the busiest).
-    static int cluster_cap[kTeamBf16 + 1][kMaxCluster + 1];  // clusters the device runs at once, 0 = not asked yet
+    static_assert(kTeamBf16 < 16 && kMaxCluster < 9, "FusedCaps holds an entry per (reducer, cluster size)");
     int best_P = 0, best_grid = 0;
     double best_eff = -1.0;
     for (int P = 1; P <= kMaxCluster; P *= 2) {
         if (cpf % P || (cpf / P) * f.e.chunk_channels > kMaxSlice) continue;
+        if (((cpf / P) * f.e.chunk_channels) & 3) continue;  // the scorers read a part's slice as 16-byte vectors
         const size_t smem = fused_smem((cpf / P) * f.e.chunk_channels, P);
         if (smem > kSmemLimit) continue;
         int clusters = sm_count;
         if (P > 1) {
-            int& cap = cluster_cap[r][P];
+            int& cap = caps->clusters[r][P];  // clusters the device runs at once, 0 = not asked yet
             if (cap == 0) {
                 cudaError_t err = cudaSuccess;
 #define SMTM_ASK(...) err = max_clusters<__VA_ARGS__>(P, smem, &cap)

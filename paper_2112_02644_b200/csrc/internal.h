@@ -48,6 +48,26 @@ cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, siz
 
 // Number of exit layers and the fast-memory capacity of a cache.
 void cache_shape(const smtm_cache_t* cache, int* n_layers, int* k_max);
+// smtm_lookup_exit_begin without the early start that SMTM_FLAG_MAPS_READY allows: nothing is read or
+// written before the stream's previous kernel is complete.  For callers whose carry is not private to
+// the batch (the entry point that works in the library's fixed array).
+smtm_status_t lookup_begin_ordered(smtm_cache_t* cache, int32_t layer, const smtm_fmap_t* fmap,
+                                   const smtm_batch_t* batch, void* stream);
+
+// Sets `kernel`'s limit on dynamic shared memory to everything the current device offers beside the
+// kernel's static arrays.  The attribute belongs to the (kernel, device) pair and setting it again is
+// harmless, so every cache sets it for its own device when it is created and no process-wide record of
+// what has been set is kept.
+template <class K>
+cudaError_t allow_max_dynamic_smem(K kernel) {
+    int dev = 0, optin = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    cudaFuncAttributes fa{};
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, kernel);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - int(fa.sharedSizeBytes));
+}
 
 // ---- encode (Sec. 4.1) ------------------------------------------------------------------
 struct EncodeArgs {
@@ -59,19 +79,26 @@ struct EncodeArgs {
     void* sv_hi;          // optional: bf16 head and tail of sv for the tensor-core scorer (same indexing)
     void* sv_lo;
     int* status;          // device sticky status word
+    unsigned long long* clock;  // nullptr, or two words for the kernel's device-clock stamps (see ClockScope)
 };
 // Enqueues the pooling of every non-skipped frame.  *launches is incremented per kernel launched.
 // *wrote_split (may be null) tells whether sv_hi / sv_lo were filled by the kernel that ran.
 cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches,
                           bool* wrote_split = nullptr);
-// Opt-in to large dynamic shared memory for the kernels that need it (once per device).
+// Opt-in to large dynamic shared memory for the kernels that need it, on the current device (every
+// cache does this for its own device at creation).
 cudaError_t encode_setup();
+cudaError_t lookup_setup();
+cudaError_t memory_setup();
+cudaError_t dense_setup();
 cudaError_t launch_row_norm2(const float* sv, const uint8_t* skip, int B, int D, float* out, cudaStream_t st,
                              int64_t* launches);
 
 // ---- lookup (Sec. 4.2, Sec. 5) -------------------------------------------------------------
 struct LookupArgs {
     int layer, L, B, D, n, k_max;
+    int S;                    // streams of the cache: a frame whose stream id lies outside [0, S) is not looked up
+    int* status;              // device sticky status word
     int early;                // (fused route, with fresh) the maps may be read and the SV stash written before the previous kernel is complete
     int fresh;                // the batch starts here: the carry is taken as SA = 0, nobody done, and is overwritten
     float tau;
@@ -96,8 +123,13 @@ cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* lau
 // memories of at most 64 entries).  *handled is false when the shape is not served, in which
 // case nothing was launched.
 constexpr int kFusedMaxK = 64;  // fast-memory capacity the fused path supports (two slots per lane)
+// What the device answered when asked how many clusters of 2, 4, 8 CTAs of each variant of the fused
+// kernel it runs at once (0 = not asked yet, -1 = refused); kept per cache, i.e. per device.
+struct FusedCaps {
+    int clusters[16][9];
+};
 // timing: nullptr, or two events recorded on `st` right before and after the kernel.
-cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm_count, cudaStream_t st,
+cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm_count, FusedCaps* caps, cudaStream_t st,
                                 int64_t* launches, bool* handled, const cudaEvent_t* timing);
 // ---- large fast memories: dot products against every class on the tensor cores ---------------
 bool dense_scoring_supported(int D, int n);
@@ -109,8 +141,8 @@ size_t dense_scratch_bytes(int max_batch, int n, int d_max);
 void dense_sv_split(void* scratch, int max_batch, int d_max, void** hi, void** lo);
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
                               void* scratch, int max_batch, int d_max, bool sv_split_done, void* centers_split,
-                              int* centers_split_current, float** dots_out, float** dots2_out, int* status, cudaStream_t st,
-                              int64_t* launches);
+                              int* centers_split_current, float** dots_out, float** dots2_out, int* status,
+                              unsigned long long* clock, cudaStream_t st, int64_t* launches);
 size_t dense_centers_split_bytes(int n, int D);
 // Eq. 1 from the dot products, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule; dots: [B][n], and dots2
 // (nullptr, or [B][n]: the second half of the vector length, added to the first).
@@ -150,6 +182,7 @@ struct UpdateArgs {
     const int32_t* fallback;   // [B] or nullptr
     int32_t* ft;               // [S][n]
     int32_t* ts;               // [S][n]
+    int* status;               // device sticky status word
     int dims[SMTM_MAX_LAYERS];
     const float* sv[SMTM_MAX_LAYERS];
     float* centers[SMTM_MAX_LAYERS];

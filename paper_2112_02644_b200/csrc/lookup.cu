@@ -30,9 +30,9 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
     const int b = blockIdx.x;
     if (a.done[b]) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int sid = a.stream_id ? a.stream_id[b] : 0;
-    const int k = a.k[sid];
-    const int32_t* mem = a.members + (size_t)sid * a.k_max;
+    const int sid = stream_of(a, b);
+    const int k = sid < 0 ? 0 : a.k[sid];  // a stream id outside the cache: nothing to score against
+    const int32_t* mem = a.members + (size_t)max(sid, 0) * a.k_max;
     const float* row = a.sv + (size_t)b * a.D;
 
     float nrm = 0.f;
@@ -118,9 +118,9 @@ __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, c
     if (b == 0 && threadIdx.x == 0 && split_current) *split_current = 1;  // the scorer before this kernel used (or made) a current split
     if (!a.fresh && a.done[b]) return;
     const int tid = threadIdx.x;
-    const int sid = a.stream_id ? a.stream_id[b] : 0;
-    const int k = a.k[sid];
-    const int32_t* mem = a.members + (size_t)sid * a.k_max;
+    const int sid = stream_of(a, b);
+    const int k = sid < 0 ? 0 : a.k[sid];  // a stream id outside the cache: nothing to score against
+    const int32_t* mem = a.members + (size_t)max(sid, 0) * a.k_max;
     const float* row = a.sv + (size_t)b * a.D;
     const float weight = float(1u << a.layer);
     const float* __restrict__ drow = dots + (size_t)b * a.n;
@@ -186,6 +186,8 @@ __global__ void k_batch_reset(float* __restrict__ sa, uint8_t* __restrict__ done
 
 }  // namespace
 
+cudaError_t lookup_setup() { return allow_max_dynamic_smem(k_score_exit); }
+
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,
                                cudaStream_t st, int64_t* launches) {
     if (B <= 0) return cudaSuccess;
@@ -205,12 +207,6 @@ cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const fl
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
     const size_t smem = (size_t(a.D) + 2 * size_t(a.k_max)) * sizeof(float);
-    static size_t opted = 48 * 1024;
-    if (smem > opted) {
-        cudaError_t e = cudaFuncSetAttribute(k_score_exit, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-        if (e != cudaSuccess) return e;
-        opted = smem;
-    }
     ++*launches;
     return launch_chained(k_score_exit, a.B, kThreads, smem, st, a);
 }

@@ -17,6 +17,18 @@ __device__ __forceinline__ bool ranks_before(float va, int ida, float vb, int id
     return ida < idb;
 }
 
+// The fast memory frame b looks up: its stream id, or -1 (and an invalid-argument code in the status word)
+// when the id lies outside [0, S).  Such a frame is scored against nothing, stays in, and is left out of
+// the update.
+__device__ __forceinline__ int stream_checked(const LookupArgs& a, int sid) {
+    if (sid >= 0 && sid < a.S) return sid;
+    set_status(a.status, kDevInvalidArg);
+    return -1;
+}
+__device__ __forceinline__ int stream_of(const LookupArgs& a, int b) {
+    return stream_checked(a, a.stream_id ? a.stream_id[b] : 0);
+}
+
 struct Top2 {
     float v1, v2;
     int id1, id2;  // class ids, -1 = absent

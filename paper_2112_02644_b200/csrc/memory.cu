@@ -70,9 +70,14 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a)
         // of labelled frames)
         const int dn = a.done ? a.done[b] : 0, pr = a.done ? a.pred[b] : -1, el = a.done ? a.exit_layer[b] : 0;
         const int fb = a.fallback ? a.fallback[b] : -1;
+        const int sid = a.stream_id ? a.stream_id[b] : 0;
         const bool ex = dn != 0;
         int lab = ex ? pr : fb;
         if (lab >= a.n) lab = -1;  // a label outside the memory counts as no label
+        if (sid < 0 || sid >= a.S) {  // a stream outside the cache: the frame takes no part in the update
+            lab = -1;
+            set_status(a.status, kDevInvalidArg);
+        }
         a.plan.final_label[b] = lab;
         a.plan.stop_layer[b] = ex ? el : a.L;
         if (lab >= 0) {
@@ -118,9 +123,14 @@ __global__ void __launch_bounds__(kPlanOneThreads) k_update_plan_one(const Updat
     for (int b = tid; b < a.B; b += kPlanOneThreads) {
         const int dn = a.done ? a.done[b] : 0, pr = a.done ? a.pred[b] : -1, el = a.done ? a.exit_layer[b] : 0;
         const int fb = a.fallback ? a.fallback[b] : -1;
+        const int sid = a.stream_id ? a.stream_id[b] : 0;
         const bool ex = dn != 0;
         int lab = ex ? pr : fb;
         if (lab >= a.n) lab = -1;
+        if (sid < 0 || sid >= a.S) {  // a stream outside the cache: the frame takes no part in the update
+            lab = -1;
+            set_status(a.status, kDevInvalidArg);
+        }
         a.plan.final_label[b] = lab;
         a.plan.stop_layer[b] = ex ? el : a.L;
         if (lab >= 0) {
@@ -515,6 +525,7 @@ __global__ void __launch_bounds__(kTblWarps * kWarp) k_update_tables(const Updat
             const int g = blockIdx.x * (blockDim.x >> 5) + (tid >> 5);  // the launch decides how many warps share a CTA
             if (g >= a.B) return;
             const int s = a.stream_id ? a.stream_id[g] : 0;
+            if (s < 0 || s >= a.S) return;  // no such stream: nothing to update (the plan kernel records the error)
             // not the stream's first frame in the batch: the warp of that frame does the work
             bool earlier = !a.stream_id && g > 0;
             for (int b0 = 0; a.stream_id && b0 < g && !earlier; b0 += kTblGroups * kWarp) {
@@ -535,6 +546,7 @@ __global__ void __launch_bounds__(kTblWarps * kWarp) k_update_tables(const Updat
         // ---- Sec. 6.1 by a whole CTA: the stream's frames, ascending, replayed per class -------
         const int g = blockIdx.x;
         const int s = a.stream_id ? a.stream_id[g] : 0;
+        if (s < 0 || s >= a.S) return;  // no such stream (the same for every thread of the CTA)
         int earlier = (!a.stream_id && g > 0) ? 1 : 0;  // an earlier frame of the same stream: its CTA does the work
         for (int b = tid; a.stream_id && b < g; b += kUpdThreads) earlier |= a.stream_id[b] == s ? 1 : 0;
         if (__syncthreads_or(earlier)) return;
@@ -657,9 +669,10 @@ __global__ void __launch_bounds__(kCenThreads, 1) k_update_centers(const UpdateA
         int q = 0;
         for (int d0 = 0; d0 < D; d0 += kCenCols) {  // a sweep of columns, four per thread
             const int d = d0 + cg * 4;
-            float old[4] = {0.f, 0.f, 0.f, 0.f}, m = 0.f;  // the centre and its count as they are, fetched along with the rows
+            float old[4] = {0.f, 0.f, 0.f, 0.f};  // the centre and its count as they are, fetched along with the rows
+            uint32_t m = 0;
             if (grp == 0) {
-                m = float(a.m[l0][cls]);
+                m = a.m[l0][cls];
                 for (int j = 0; j < 4; ++j)
                     if (d + j < D) old[j] = cen[d + j];
             }
@@ -707,7 +720,8 @@ __global__ void __launch_bounds__(kCenThreads, 1) k_update_centers(const UpdateA
                 }
                 for (int j = 0; j < 4; ++j)
                     if (d + j < D) {
-                        const float v = __fdiv_rn(__fmaf_rn(old[j], m, acc[j]), m + float(q));
+                        // Eq. 7 in double: the count is exact at any size and SC m + sum SV is rounded once
+                        const float v = float((double(old[j]) * double(m) + double(acc[j])) / (double(m) + double(q)));
                         cen[d + j] = v;
                         nrm = fmaf(v, v, nrm);
                     }
@@ -737,14 +751,12 @@ __global__ void k_center_norms(const float* __restrict__ centers, int n, int D, 
     if (threadIdx.x == 0) cnorm[c] = __fsqrt_rn(nrm);
 }
 
-cudaError_t opt_in_smem(const void* fn, size_t smem, size_t* opted) {
-    if (smem <= *opted) return cudaSuccess;
-    const cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e == cudaSuccess) *opted = smem;
-    return e;
-}
-
 }  // namespace
+
+cudaError_t memory_setup() {
+    const cudaError_t e = allow_max_dynamic_smem(k_update_tables);
+    return e != cudaSuccess ? e : allow_max_dynamic_smem(k_resize);
+}
 
 cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm, cudaStream_t st,
                                 int64_t* launches) {
@@ -755,8 +767,6 @@ cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm
 cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, cudaStream_t side,
                           cudaEvent_t fork, cudaEvent_t join, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
-    // static + dynamic shared memory above 48 KB needs the opt-in; the kernel's static arrays take 34 KB of that
-    static size_t opted = 8 * 1024;
     // a warp per frame when eight streams' tables and refresh buffers fit a CTA's shared memory
     const size_t per_warp = tables_smem(a.n, rz ? rz->k_max : 0);
     const bool warp_tables = per_warp * kUpdWarps <= 100 * 1024;
@@ -767,8 +777,7 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
     const int warps = !warp_tables ? kUpdWarps : (per_warp * kTblWarps <= 180 * 1024 ? kTblWarps : kUpdWarps);
     const size_t smem = warp_tables ? per_warp * warps
                                     : std::max<size_t>(rz ? resize_cta_smem(a.n, rz->k_max) : 0, size_t(a.n) * 2 * sizeof(int));
-    cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_update_tables), smem, &opted);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
     const bool tables = a.warm_layer < 0;  // a warm-up batch has no streams
     const int table_ctas = warp_tables ? (a.B + warps - 1) / warps : a.B;
     if (tables) {
@@ -801,10 +810,7 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
 }
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
-    static size_t opted = 40 * 1024;  // static + dynamic above 48 KB needs the opt-in
     const size_t smem = resize_cta_smem(a.n, a.k_max);
-    const cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_resize), smem, &opted);
-    if (e != cudaSuccess) return e;
     ++*launches;
     return launch_chained(k_resize, a.S, kUpdThreads, smem, st, a);
 }

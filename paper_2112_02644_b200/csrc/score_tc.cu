@@ -123,6 +123,7 @@ struct TcParams {
     float* out;        // [splits][M][ld_out] dot products over each part of the vector length
     size_t split_stride;  // floats between the result arrays of two parts
     int* status;
+    unsigned long long* clock;  // nullptr, or two words for the device-clock stamps
 };
 
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -163,6 +164,7 @@ k_score_tc(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__
     const uint32_t tmem_acc = *tmem_slot;
     chain_wait();  // barriers and tensor memory are set up while the previous kernel finishes
     chain_release();
+    const ClockScope stamps(p.clock);
 
     bool failed = false;
     int issued = 0;
@@ -304,6 +306,10 @@ bool make_map(CUtensorMap* map, const __nv_bfloat16* ptr, int rows, int D, int b
 
 }  // namespace
 
+cudaError_t dense_setup() {
+    return cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kTcSmem));
+}
+
 bool dense_scoring_supported(int D, int n) {
     return D % 8 == 0 && D >= 4 * kTileK && n % 4 == 0 && encode_tiled_fn() != nullptr;
 }
@@ -323,8 +329,8 @@ void dense_sv_split(void* scratch, int max_batch, int d_max, void** hi, void** l
 
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
                               void* scratch, int max_batch, int d_max, bool sv_split_done, void* centers_split,
-                              int* centers_split_current, float** dots_out, float** dots2_out, int* status, cudaStream_t st,
-                              int64_t* launches) {
+                              int* centers_split_current, float** dots_out, float** dots2_out, int* status,
+                              unsigned long long* clock, cudaStream_t st, int64_t* launches) {
     __nv_bfloat16* a_hi = reinterpret_cast<__nv_bfloat16*>(scratch);
     __nv_bfloat16* a_lo = a_hi + size_t(max_batch) * d_max;
     __nv_bfloat16* b_hi = reinterpret_cast<__nv_bfloat16*>(centers_split);
@@ -340,13 +346,6 @@ cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const
     if (!make_map(&ma_hi, a_hi, B, D, kTileM) || !make_map(&ma_lo, a_lo, B, D, kTileM) ||
         !make_map(&mb_hi, b_hi, n, D, kTileN) || !make_map(&mb_lo, b_lo, n, D, kTileN))
         return cudaErrorInvalidValue;
-    static bool opted = false;
-    if (!opted) {
-        const cudaError_t e =
-            cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kTcSmem));
-        if (e != cudaSuccess) return e;
-        opted = true;
-    }
     if (!sv_split_done) {
         ++*launches;
         const int grid_a = int(std::min<long long>(((long long)B * D / 4 + 255) / 256, 148 * 8));
@@ -371,6 +370,7 @@ cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const
     p.out = dots;
     p.split_stride = size_t(max_batch) * n;
     p.status = status;
+    p.clock = clock;
     const dim3 grid((n + kTileN - 1) / kTileN, (B + kTileM - 1) / kTileM, splits);
     return launch_chained(k_score_tc, grid, kTcThreads, kTcSmem, st, ma_hi, ma_lo, mb_hi, mb_lo, p);
 }

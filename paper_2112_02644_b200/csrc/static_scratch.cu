@@ -7,7 +7,7 @@
 // semantic vectors, the cumulative similarities, the exit layers), which such a caller has
 // nowhere to put.  Here it lives in a fixed array compiled into the library image, so the
 // call touches no allocator at all: not cudaMalloc / cudaFree, not torch, not the host heap.
-#include <mutex>
+#include <atomic>
 
 #include "internal.h"
 
@@ -20,8 +20,10 @@ __device__ __align__(256) static unsigned char g_static_scratch[SMTM_STATIC_SCRA
 namespace {
 
 constexpr int kMaxDevices = 64;
-std::mutex g_mu;
-unsigned char* g_scratch_addr[kMaxDevices];  // device address of g_static_scratch, per device
+// Device address of g_static_scratch, per device; null until the first call on that device.  Published
+// through an atomic so that the calls after the first one take no lock (two first calls that race both
+// ask the runtime and store the same address).
+std::atomic<unsigned char*> g_scratch_addr[kMaxDevices];
 
 // In host code the name g_static_scratch is only a handle for the runtime, not an address a
 // kernel can use; the device address is obtained, once per device and with that device
@@ -31,14 +33,13 @@ cudaError_t scratch_address(unsigned char** out) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    std::lock_guard<std::mutex> lock(g_mu);
-    if (!g_scratch_addr[dev]) {
-        unsigned char* p = nullptr;
+    unsigned char* p = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!p) {
         e = cudaGetSymbolAddress((void**)&p, g_static_scratch);
         if (e != cudaSuccess) return e;
-        g_scratch_addr[dev] = p;
+        g_scratch_addr[dev].store(p, std::memory_order_release);
     }
-    *out = g_scratch_addr[dev];
+    *out = p;
     return cudaSuccess;
 }
 
@@ -75,6 +76,8 @@ extern "C" smtm_status_t smtm_lookup_exit_static(smtm_cache_t* cache, int32_t la
     b.d_pred = d_pred;
     b.d_ac = d_ac;
     b.d_sv[layer] = reinterpret_cast<float*>(base);
-    // the array keeps whatever the previous call left: the lookup starts the carry afresh
-    return smtm_lookup_exit_begin(cache, layer, fmap, &b, stream);
+    // The array keeps whatever the previous call left: the lookup starts the carry afresh.  It never starts
+    // early (SMTM_FLAG_MAPS_READY is for carries that alternate; every call here shares the one array, which
+    // the stream's previous kernel may be a static call still reading).
+    return lookup_begin_ordered(cache, layer, fmap, &b, stream);
 }

@@ -32,6 +32,7 @@ class Report:
     max_sv_err: float = 0.0
     max_sa_err: float = 0.0
     max_center_err: float = 0.0
+    routes: list = field(default_factory=list)   # lookups served by the fused, dense and plain routes
 
 
 def make_pair(w: si.Workload, max_batch=None):
@@ -51,17 +52,29 @@ def abs_mean_scale(x: torch.Tensor, w: si.Workload, layer: int) -> np.ndarray:
     return x.float().abs().mean(dim=axes).cpu().numpy().astype(np.float64)
 
 
+def same_specials(g: np.ndarray, o: np.ndarray) -> np.ndarray:
+    """Asserts that NaN and +-inf sit in the same places on both sides; returns the mask of finite entries."""
+    assert np.array_equal(np.isnan(g), np.isnan(o)), "NaN in different places"
+    inf = np.isinf(o)
+    assert np.array_equal(np.isinf(g), inf) and np.array_equal(g[inf], o[inf]), "infinities differ"
+    return np.isfinite(o)
+
+
 def compare_layer(w, layer, x, gb, ob, todo, rep: Report):
-    """Element-wise comparison of everything one lookup produced for the frames in ``todo``."""
-    sv_g = gb.sv[layer].cpu().numpy().astype(np.float64)
-    sv_o = ob["sv"][layer]
-    scale = np.maximum(abs_mean_scale(x, w, layer), 1e-30)
-    err = np.abs(sv_g - sv_o)[todo] / scale[todo]
+    """Element-wise comparison of everything one lookup produced for the frames in ``todo``.
+    Non-finite values (a NaN or an infinite element in a map propagates) must sit in the same places."""
+    sv_g = gb.sv[layer].cpu().numpy().astype(np.float64)[todo]
+    sv_o = ob["sv"][layer][todo]
+    fin = same_specials(sv_g, sv_o)
+    scale = np.maximum(np.nan_to_num(abs_mean_scale(x, w, layer)[todo], nan=1.0, posinf=1.0), 1e-30)
+    err = np.where(fin, np.abs(sv_g - np.where(fin, sv_o, 0.0)), 0.0) / scale
     rep.max_sv_err = max(rep.max_sv_err, float(err.max(initial=0.0)))
     assert err.max(initial=0.0) <= SV_RTOL, f"semantic vectors off by {err.max():.3g} (relative) at layer {layer}"
     # cumulative similarity: weights add up to 2^(layer+1) - 1, each cosine within SCORE_ATOL
-    sa_g = gb.sa.cpu().numpy().astype(np.float64)
-    sa_err = np.abs(sa_g - ob["sa"])[todo]
+    sa_g = gb.sa.cpu().numpy().astype(np.float64)[todo]
+    sa_o = ob["sa"][todo]
+    fin = same_specials(sa_g, sa_o)
+    sa_err = np.where(fin, np.abs(sa_g - np.where(fin, sa_o, 0.0)), 0.0)
     rep.max_sa_err = max(rep.max_sa_err, float(sa_err.max(initial=0.0)))
     assert sa_err.max(initial=0.0) <= SCORE_ATOL * (2 ** (layer + 1) - 1), f"cumulative similarity off by {sa_err.max():.3g}"
     # accumulated confidence and separability where the ratio is well conditioned
@@ -70,6 +83,7 @@ def compare_layer(w, layer, x, gb, ob, todo, rep: Report):
     sep_g = gb.sep.cpu().numpy().astype(np.float64)[:, layer]
     sep_o = ob["sep"][:, layer]
     for g, o in ((ac_g, ac_o), (sep_g, sep_o)):
+        assert np.array_equal(np.isnan(g[todo]), np.isnan(o[todo])), "AC / separability: NaN in different places"
         fin = todo & np.isfinite(o) & np.isfinite(g) & (np.abs(o) < 5.0)
         assert np.all(np.abs(g[fin] - o[fin]) <= 2e-3 * (1 + np.abs(o[fin]))), "AC / separability mismatch"
     # top-1 class wherever the oracle's lead is clear of rounding
@@ -80,8 +94,9 @@ def compare_layer(w, layer, x, gb, ob, todo, rep: Report):
         assert np.array_equal(top_g[clear, 0], ob["top"][clear, 0]), "top-1 class differs"
 
 
-def step_pair(w, cache, mem, gb, lab, step, rep: Report, device="cuda", compare_values=True):
-    """One step on both sides, compared layer by layer.  Returns the oracle's batch."""
+def step_pair(w, cache, mem, gb, lab, step, rep: Report, device="cuda", compare_values=True, edit=None):
+    """One step on both sides, compared layer by layer.  Returns the oracle's batch.
+    edit(layer, x): optional, changes the maps of a layer in place before either side sees them."""
     sid = si.stream_ids(w) if w.S > 1 else None
     ob = mem.new_batch(w.B, sid)
     begin = step % 2 == 1      # odd steps start with smtm_lookup_exit_begin on a carry full of garbage
@@ -95,6 +110,8 @@ def step_pair(w, cache, mem, gb, lab, step, rep: Report, device="cuda", compare_
     fb = si.fallback_labels(w, lab)
     for l in range(w.L):
         x = si.frames(w, l, lab, step, device=device)
+        if edit is not None:
+            edit(l, x)
         B, C, H, W = si.shape4(w, l)
         todo = ob["done"] == 0
         (smtm.smtm_lookup_exit_begin if begin and l == 0 else smtm.smtm_lookup_exit)(
@@ -153,8 +170,10 @@ def compare_state(w, cache, mem, rep: Report):
     for l in range(w.L):
         cen, m = smtm.smtm_cache_get_centers(cache, l)
         assert np.array_equal(m, mem.m[l]), "update counts differ"
-        scale = np.maximum(np.abs(mem.centers[l]), np.abs(mem.centers[l]).mean(axis=1, keepdims=True))
-        err = np.abs(cen.astype(np.float64) - mem.centers[l]) / np.maximum(scale, 1e-30)
+        fin = same_specials(cen.astype(np.float64), mem.centers[l])   # a NaN folded into a centre by Eq. 7 stays there
+        ref = np.where(fin, mem.centers[l], 0.0)
+        scale = np.maximum(np.abs(ref), np.abs(ref).mean(axis=1, keepdims=True))
+        err = np.where(fin, np.abs(cen.astype(np.float64) - ref), 0.0) / np.maximum(scale, 1e-30)
         rep.max_center_err = max(rep.max_center_err, float(err.max()))
         assert err.max() <= CENTER_RTOL, f"centres off by {err.max():.3g} at layer {l}"
     assert smtm.smtm_cache_status(cache) == 0, "device status word set"
@@ -175,5 +194,6 @@ def run_workload(w: si.Workload, steps=None, device="cuda", compare_values=True,
     rep.exits = [int(v) for v in ctr[: w.L]]
     assert rep.exits == [int(v) for v in mem.exits_per_layer], (rep.exits, mem.exits_per_layer)
     assert int(ctr[smtm.CTR_LOOKUPS]) == rep.lookups
+    rep.routes = [int(v) for v in smtm.smtm_cache_get_routes(cache)]
     smtm.smtm_cache_destroy(cache)
     return rep

@@ -116,11 +116,13 @@ def test_argument_errors_launch_nothing():
 def test_c1_single_layer_fp32():
     rep = run_workload(si.C1)
     assert rep.exits == [8] and rep.band_mismatches == 0
+    assert rep.routes == [1, 0, 0]       # one fused launch: pooling, Eq. 1, Eq. 3, Eq. 4 and the decision
 
 
 def test_c2_resnet50_bf16_four_layers():
     rep = run_workload(si.C2)
     assert sum(rep.exits) > 30 and rep.frames == 64
+    assert rep.routes == [4, 0, 0]
 
 
 def test_c2_exits_disabled_streams_every_layer():
@@ -141,6 +143,7 @@ def test_c3_mobilenetv2_fp16_nhwc_novel_classes_do_not_exit():
 def test_c4_large_cache_straddles_threshold():
     rep = run_workload(si.C4)
     assert 100 < rep.exits[0] < 900
+    assert rep.routes == [0, 1, 0], "the 1000-entry fast memory must be scored on the tensor cores (Eq. 1 as a dense contraction)"
     print("c4 max |SA error|:", rep.max_sa_err, "max SV error:", rep.max_sv_err)
     print("c4 near-threshold lookups (oracle):", rep.near_oracle, "band mismatches:", rep.band_mismatches)
 
@@ -149,6 +152,7 @@ def test_c4_large_cache_straddles_threshold():
 def test_c5_streaming_full_width(T):
     rep = run_workload(si.C5, steps=T)
     assert rep.frames == 512 * T and rep.exits[0] > 0
+    assert rep.routes == [2 * T, 0, 0]
 
 
 def test_c5_full_length_64_steps_state_only():
@@ -178,10 +182,11 @@ def test_large_fast_memory_over_several_layers_uses_tensor_cores():
                     k_min=70, k_max=196, S=1, T=4, tau=0.8, window_W=2, sigma=0.6, zipf_s=0.9, repeat_p=0.3, seed=6)
     rep = run_workload(w)
     assert rep.frames == 70 * 4 and rep.lookups > 70
+    assert rep.routes == [0, 8, 0]       # both layers of all four steps on the tensor-core route
     w3 = si.Workload("dense_nhwc", si.F16, si.NHWC, B=33, stages=((320, 7, 7),), n=72, k_init=72, k_min=72, k_max=72,
                      S=1, T=2, tau=0.8, sigma=1.0, zipf_s=1.0, seed=8)
     rep3 = run_workload(w3)
-    assert rep3.frames == 66
+    assert rep3.frames == 66 and rep3.routes == [0, 2, 0]
 
 
 def test_forgetting_frequency_table_rapid_scene_change():
@@ -486,3 +491,179 @@ def test_bench_launch_configuration_matches_oracle(w):
     ctr = smtm.smtm_cache_get_counters(cache)
     assert [int(v) for v in ctr[: w.L]] == [int(v) for v in mem.exits_per_layer]
     smtm.smtm_cache_destroy(cache)
+
+
+# ---------------------------------------------------------------------------- degenerate inputs on every route
+
+EDGE_ROUTES = {
+    # route -> (workload, index into Report.routes that must serve every lookup)
+    "fused": (si.Workload("edge_fused", si.BF16, si.NCHW, B=40, stages=((256, 14, 14), (512, 7, 7)), n=24, k_init=6,
+                          k_min=2, k_max=9, S=1, T=3, tau=0.8, window_W=2, sigma=0.5, zipf_s=0.6, repeat_p=0.3, seed=41), 0),
+    "dense": (si.Workload("edge_dense", si.BF16, si.NCHW, B=40, stages=((256, 14, 14), (512, 7, 7)), n=80, k_init=72,
+                          k_min=66, k_max=80, S=1, T=3, tau=0.8, window_W=2, sigma=0.5, zipf_s=0.6, repeat_p=0.3, seed=42), 1),
+    "plain": (si.Workload("edge_plain", si.F32, si.NHWC, B=40, stages=((21, 9, 5), (38, 3, 3)), n=24, k_init=6,
+                          k_min=2, k_max=9, S=1, T=3, tau=0.8, window_W=2, sigma=0.5, zipf_s=0.6, repeat_p=0.3, seed=43), 2),
+}
+
+
+@pytest.mark.parametrize("one_entry", [False, True], ids=["k6", "k1"])
+@pytest.mark.parametrize("route", list(EDGE_ROUTES))
+def test_degenerate_frames_match_the_oracle_on_every_route(route, one_entry):
+    # Sec. 5 is silent on these inputs; the readings are pinned on the oracle (tests/test_oracle_pins.py) and the
+    # kernels must follow them element by element: an all-zero map (post-ReLU features make it a real input:
+    # zero-length SV, similarity 0 to everything, no exit), a map with one NaN element and one with one +Inf
+    # element (they propagate: NaN similarities rank last, the frame never exits, Eq. 7 carries the NaN into the
+    # centre of the frame's class, which then ranks last for every later frame), and a fast memory with a single
+    # entry (no runner-up: never exits).  Three steps, so that the poisoned centres are looked up as well.
+    from harness import Report, compare_state, make_pair, step_pair
+
+    w, served = EDGE_ROUTES[route]
+    if one_entry:
+        w = w.scaled(name=w.name + "_k1", k_init=1, k_min=1, k_max=max(w.k_max, 70) if route == "dense" else 3)
+    cache, mem = make_pair(w)
+    gb = smtm.Batch(cache, w.B)
+    labs = si.labels(w)
+
+    def poison(step):
+        def edit(layer, x):
+            flat = x.view(w.B, -1)
+            flat[0].zero_()                                  # every layer: nothing to pool
+            flat[21 + step, 5] = float("-inf")               # every layer
+            if layer == 0:                                   # first layer only: the NaN then rides on in SA
+                flat[1 + step, 17] = float("nan")
+                flat[11 + step, flat.shape[1] - 3] = float("inf")
+        return edit
+
+    rep = Report()
+    for t in range(w.T):
+        ob = step_pair(w, cache, mem, gb, labs[t], t, rep, edit=poison(t))
+        compare_state(w, cache, mem, rep)
+        done = gb.done.cpu().numpy()
+        assert not done[[0, 1 + t, 11 + t, 21 + t]].any()       # none of the degenerate frames exits
+        assert np.isnan(ob["sa"][[1 + t, 11 + t, 21 + t], 0]).all()
+        assert gb.ac.cpu().numpy()[0, w.L - 1] == 0.0
+        if one_entry and t == 0:
+            assert not done.any() and (gb.top.cpu().numpy()[:, 1] == -1).all()
+    routes = smtm.smtm_cache_get_routes(cache)
+    assert routes[served] == w.T * w.L and routes.sum() == w.T * w.L, routes
+    assert np.isnan(mem.centers[0]).any()                        # Eq. 7 did carry a NaN into a centre
+    smtm.smtm_cache_destroy(cache)
+
+
+def test_stream_id_outside_the_cache_skips_the_frame_and_sets_the_status_word():
+    # a frame that names a stream the cache does not have is scored against nothing, stays in, takes no part in
+    # the update, and the sticky status word reports an invalid argument; the other frames are served as usual
+    from harness import Report, compare_state
+
+    w = si.C5.scaled(name="bad_sid", B=24, S=24, T=2)
+    cents, counts = si.initial_centers(w)
+    tau = [w.tau] * w.L
+    good = si.stream_ids(w)
+    bad = good.copy()
+    bad[5], bad[17] = w.S, -3
+    for fused in (True, False):       # the second cache is fed maps in a shape only the plain route serves
+        ww = w if fused else w.scaled(name="bad_sid_plain", dtype=si.F32, layout=si.NHWC, stages=((21, 3, 3), (38, 2, 2)))
+        cents, counts = si.initial_centers(ww)
+        cache = smtm.smtm_cache_create(ww.n, ww.dims, tau, cents, counts, n_streams=ww.S, k_init=ww.k_init, k_min=ww.k_min,
+                                       k_max=ww.k_max, window_W=ww.window_W, max_batch=ww.B)
+        mem = oracle.OracleMemory(ww.n, ww.dims, tau, cents, counts, ww.S, ww.k_init, ww.k_min, ww.k_max, ww.window_W)
+        gb = smtm.Batch(cache, ww.B, stream_id=bad)
+        labs = si.labels(ww)
+        for t in range(ww.T):
+            fb = si.fallback_labels(ww, labs[t])
+            ob = mem.new_batch(ww.B, good)
+            for l in range(ww.L):
+                x = si.frames(ww, l, labs[t], t, device="cuda")
+                (smtm.smtm_lookup_exit_begin if l == 0 else smtm.smtm_lookup_exit)(
+                    cache, l, smtm.Fmap(x, ww.dtype, ww.layout, *si.shape4(ww, l)), gb)
+                mem.lookup_exit(l, x.cpu(), ww.dtype, ww.layout, si.shape4(ww, l), ob)
+            smtm.smtm_cache_update_resize(cache, gb, torch.from_numpy(fb).cuda())
+            # the oracle is told what the library is documented to do with such a frame: it does not exit and is
+            # left out of the update (no label); its stream's tables (which it does not name) see nothing
+            for b in (5, 17):
+                ob["done"][b], ob["exit_layer"][b], ob["pred"][b] = 0, 0, -1
+            fb2 = fb.copy(); fb2[[5, 17]] = -1
+            sid_o = good.copy()
+            keep = np.ones(ww.B, bool); keep[[5, 17]] = False
+            sub = {k: (v[keep] if isinstance(v, np.ndarray) and v.shape[:1] == (ww.B,) else v) for k, v in ob.items()}
+            sub["sv"] = [v[keep] for v in ob["sv"]]
+            sub["B"] = int(keep.sum()); sub["stream_id"] = np.ascontiguousarray(sid_o[keep])
+            mem.update(sub, fb2[keep])
+            mem.resize()
+            done = gb.done.cpu().numpy()
+            assert not done[[5, 17]].any() and np.array_equal(done[keep], ob["done"][keep])
+            assert np.array_equal(gb.pred.cpu().numpy()[keep & (done == 1)], ob["pred"][keep & (done == 1)])
+            assert (gb.ac.cpu().numpy()[[5, 17]] == 0.0).all()
+        assert smtm.smtm_cache_status(cache) == 1                 # SMTM_ERR_INVALID_ARG, sticky
+        ft, ts = smtm.smtm_cache_get_tables(cache)
+        assert np.array_equal(ft, mem.ft) and np.array_equal(ts, mem.ts)
+        assert not ft[[5, 17]].any() and not ts[[5, 17]].any()    # the streams those frames should have named saw nothing
+        members, k = smtm.smtm_cache_get_members(cache)
+        assert np.array_equal(k, mem.k)
+        for s_ in range(ww.S):      # (slots beyond k are unspecified in a fast memory that was never refreshed)
+            assert np.array_equal(members[s_, : k[s_]], mem.members[s_, : k[s_]]), s_
+        for l in range(ww.L):
+            cen, m = smtm.smtm_cache_get_centers(cache, l)
+            assert np.array_equal(m, mem.m[l])
+            np.testing.assert_allclose(cen, mem.centers[l], rtol=2e-5, atol=1e-7)
+        assert smtm.smtm_cache_get_routes(cache)[0 if fused else 2] == ww.T * ww.L
+        smtm.smtm_cache_destroy(cache)
+
+
+def test_export_then_import_puts_the_cache_back_bit_for_bit():
+    # snapshot after two steps, run three more, import the snapshot, run the same three again: identical decisions
+    # and an identical final state; the snapshot also moves to a second cache of the same shape, and is refused
+    # by a cache of another shape
+    w = si.C5.scaled(name="snapshot", B=64, S=64, T=5)
+    cents, counts = si.initial_centers(w)
+    tau = [w.tau] * w.L
+    mk = lambda ww=w: smtm.smtm_cache_create(ww.n, ww.dims, tau, cents, counts, n_streams=ww.S, k_init=ww.k_init,
+                                              k_min=ww.k_min, k_max=ww.k_max, window_W=ww.window_W, max_batch=ww.B)
+    labs = si.labels(w)
+    sid = si.stream_ids(w)
+    maps = [[si.frames(w, l, labs[t], t, device="cuda") for l in range(w.L)] for t in range(w.T)]
+
+    def run(cache, steps):
+        gb = smtm.Batch(cache, w.B, stream_id=sid)
+        out = []
+        for t in steps:
+            for l in range(w.L):
+                (smtm.smtm_lookup_exit_begin if l == 0 else smtm.smtm_lookup_exit)(
+                    cache, l, smtm.Fmap(maps[t][l], w.dtype, w.layout, *si.shape4(w, l)), gb)
+            smtm.smtm_cache_update_resize(cache, gb, torch.from_numpy(si.fallback_labels(w, labs[t])).cuda())
+            torch.cuda.synchronize()
+            out.append((gb.done.cpu().numpy().copy(), gb.pred.cpu().numpy().copy(), gb.sa.cpu().numpy().copy()))
+        return out
+
+    def state(cache):
+        return [smtm.smtm_cache_get_tables(cache), smtm.smtm_cache_get_members(cache),
+                [smtm.smtm_cache_get_centers(cache, l) for l in range(w.L)], smtm.smtm_cache_get_counters(cache)]
+
+    def same(a, b):
+        flat = lambda x: [x] if isinstance(x, np.ndarray) else [z for y in x for z in flat(y)]
+        return all(np.array_equal(p, q) for p, q in zip(flat(a), flat(b)))
+
+    a = mk()
+    run(a, [0, 1])
+    blob = smtm.smtm_cache_export(a)
+    at_snapshot = state(a)
+    first = run(a, [2, 3, 4])
+    after = state(a)
+    assert not same(at_snapshot, after)
+    smtm.smtm_cache_import(a, blob)
+    assert same(state(a), at_snapshot)
+    second = run(a, [2, 3, 4])
+    assert same(first, second) and same(state(a), after)
+    b = mk()                                     # a fresh cache of the same shape takes the snapshot too
+    smtm.smtm_cache_import(b, blob)
+    assert same(run(b, [2, 3, 4]), first) and same(state(b), after)
+    other = mk(w.scaled(S=32, B=32))
+    with pytest.raises(smtm.SmtmError) as e:
+        smtm.smtm_cache_import(other, blob)
+    assert e.value.status == 2
+    bad = blob.copy(); bad[:8] = 0
+    with pytest.raises(smtm.SmtmError) as e:
+        smtm.smtm_cache_import(b, bad)
+    assert e.value.status == 1 and same(state(b), after)          # nothing was changed
+    for c in (a, b, other):
+        smtm.smtm_cache_destroy(c)

@@ -59,3 +59,39 @@ def test_reference_arm_runs_the_oracle_on_rank_0_only():
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["value"] > 0 and line["unit"] == "frames/s"
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_gpus_flag_starts_that_many_ranks_itself():
+    # without a launcher above it, `bench.py --gpus 2` starts two ranks on this node; --rank-check runs only the
+    # multi-rank plumbing (gloo rendezvous, one shard of streams per rank, time = max over ranks) on the host
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rank-check"], env=env,
+                         capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads([l for l in out.stdout.splitlines() if l.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["ms"] == 20.0 and line["value"] == 2 * 1000 / 20e-3
+    assert len(set(line["seeds"])) == 2                      # every rank serves its own streams
+
+
+def test_oracle_split_over_threads_equals_the_oracle_on_one_thread():
+    # the all-cores leg of the CPU baseline splits the frames of a step over threads; it must leave exactly the
+    # state the plain frame-by-frame run leaves (one frame per stream, a single stream, the forgetting tables)
+    sys.path.insert(0, ROOT)
+    import bench
+    import smtm_inputs as si
+
+    for w in (si.C5.scaled(B=24, S=24, T=5), si.C2.scaled(B=16), si.C6.scaled(B=16, S=16, T=3)):
+        a, b = bench.OracleRun(w, 1), bench.OracleRun(w, 3)
+        labs = si.labels(w)
+        for t in range(4):
+            lab = labs[t % w.T]
+            maps = [si.frames(w, l, lab, t) for l in range(w.L)]
+            fb = si.fallback_labels(w, lab)
+            a.step(maps, fb)
+            b.step(maps, fb)
+        b.close()
+        assert all(np.array_equal(x, y) for x, y in zip(a.exits_after, b.exits_after))
+        for name in ("ft", "ts", "members", "k"):
+            assert np.array_equal(getattr(a.mem, name), getattr(b.mem, name)), (w.name, name)
+        for x, y in zip(a.mem.centers + a.mem.m, b.mem.centers + b.mem.m):
+            assert np.array_equal(x, y)
