@@ -312,7 +312,7 @@ class Resident:
         return si.fallback_labels(self.w, self.labs[(t % self.R) % self.w.T])
 
 
-def measure(smtm, w, K, W, local_rank, world, verify_steps=0, oracle_threads=1):
+def measure(smtm, w, K, W, local_rank, world, verify_steps=0, graph_steps=32):
     """Times steps W .. W+K-1 of workload `w` through CUDA graphs and returns the figures of the run.
     verify_steps > 0: the CPU oracle is run over steps 0 .. W+verify_steps-1 of the same maps and the exits it
     takes in steps W .. W+verify_steps-1 are compared with the library's."""
@@ -320,7 +320,7 @@ def measure(smtm, w, K, W, local_rank, world, verify_steps=0, oracle_threads=1):
         import torch.distributed as dist
     res = Resident(smtm, w, W + K)
     R = res.R
-    G = math.gcd(K, 32)         # steps captured into one CUDA graph
+    G = math.gcd(K, graph_steps)   # steps captured into one CUDA graph
     cents, counts = si.initial_centers(w)
     sid = si.stream_ids(w) if w.S > 1 else None
     # All launches go to one side stream so that every step can be captured into a CUDA graph.
@@ -556,7 +556,7 @@ def cpu_all_cores(w, m, serial_run, budget_s):
 def other_workload(smtm, w, peak, tc_peak, with_oracle):
     """A short pass of one of the single-batch workloads: the same machinery, fewer steps."""
     K, W = 16, 3
-    m = measure(smtm, w, K, W, 0, 1, verify_steps=(1 if w.n >= 1000 else 4) if with_oracle else 0)
+    m = measure(smtm, w, K, W, 0, 1, verify_steps=4 if with_oracle else 0, graph_steps=4)
     nbytes, us_ev, ach, us_dev, ach_dev = roofline_of(w, m, peak)
     ms = m["ms_local"] / K
     out = {"workload": w.name, "steps": K, "warmup": W, "ms_per_step": ms, "frames_per_s": w.B / (ms * 1e-3),

@@ -29,11 +29,12 @@ struct smtm_cache {
     void* d_cen_split[SMTM_MAX_LAYERS];   // bf16 heads and tails of the centres, per layer (same condition)
     int* d_split_current;  // [L] device flags: the centres' split of a layer is current (same condition as d_dense)
     int d_max;          // largest C_l
-    int32_t* d_plan;    // scratch of the update: final label and stop layer, 2 x [max_batch]
+    int32_t* d_plan;    // scratch of the update: final label and stop layer of every frame, [max_batch]
     unsigned long long* d_tags;  // scratch of the update: stamps of (layer, class), [L][n]
     cudaStream_t side_stream;    // the update's tables run here, beside plan + centres on the caller's stream
     cudaEvent_t ev_fork, ev_join;
-    int32_t* d_jobs;             // scratch of the update: [2] counters, [L][n] (layer, class) pairs to fold
+    int32_t* d_jobs;             // scratch of the update: [4] counters, [L][n] (layer, class) pairs to fold, [16][L][n] work items
+    uint32_t* d_m_next;          // scratch of the update: [L][n] counts after the update
     unsigned long long* d_epoch; // [2] device: update calls so far, and the plan kernel's ticket
     // optional timing of the streaming kernel of every lookup (smtm_cache_profile)
     std::vector<cudaEvent_t>* prof_events;  // pairs, in launch order
@@ -121,6 +122,7 @@ void free_all(smtm_cache* c) {
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     cudaFree(c->d_jobs);
+    cudaFree(c->d_m_next);
     cudaFree(c->hb.d_sa);
     cudaFree(c->hb.d_done);
     cudaFree(c->hb.d_exit_layer);
@@ -265,12 +267,12 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     a.L = c->L;
     a.forget_W = c->forgetting ? c->W : 0;
     a.warm_layer = -1;
-    const size_t mb = size_t(c->max_batch);
-    a.plan.final_label = c->d_plan;
-    a.plan.stop_layer = c->d_plan + mb;
+    a.plan.frame_code = c->d_plan;
     a.plan.class_tag = c->d_tags;
     a.plan.job_count = c->d_jobs;
     a.plan.jobs = c->d_jobs + 4;
+    a.plan.items = c->d_jobs + 4 + size_t(c->L) * c->n;
+    a.m_next = c->d_m_next;
     a.plan.epoch = c->d_epoch;
     a.stream_id = b->d_stream_id;
     a.done = b->d_done;
@@ -290,7 +292,7 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
         a.m[l] = c->d_m[l];
     }
     const ResizeArgs rz = resize_args(c);
-    SMTM_CUDA(launch_update(a, with_resize ? &rz : nullptr, c->sm_count, st, c->side_stream, c->ev_fork, c->ev_join, &c->launches));
+    SMTM_CUDA(launch_update(a, with_resize ? &rz : nullptr, c->sm_count, st, &c->launches));
     return SMTM_OK;
 }
 
@@ -395,7 +397,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     ok = ok && dev_alloc(&c->d_k, S) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_counters, SMTM_CTR_COUNT) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_status, 1) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_plan, 2 * size_t(c->max_batch)) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_plan, size_t(c->max_batch)) == cudaSuccess;
     for (int l = 0; l < c->L; ++l) c->d_max = c->dims[l] > c->d_max ? c->dims[l] : c->d_max;
     c->d_max = (c->d_max + 7) / 8 * 8;  // keeps the bf16 operand arrays of the tensor-core scorer 16-byte aligned
     if (ok && c->k_max > kFusedMaxK) {
@@ -406,7 +408,8 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
             ok = cudaMalloc(&c->d_cen_split[l], dense_centers_split_bytes(n, c->dims[l])) == cudaSuccess;
     }
     ok = ok && dev_alloc(&c->d_tags, size_t(c->L) * n) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_jobs, 4 + size_t(c->L) * n) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_jobs, 4 + 17 * size_t(c->L) * n) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_m_next, size_t(c->L) * n) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_epoch, 2) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
@@ -439,7 +442,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     if (e == cudaSuccess) e = cudaMemset(c->d_counters, 0, SMTM_CTR_COUNT * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->d_tags, 0, size_t(c->L) * n * sizeof(unsigned long long));
-    if (e == cudaSuccess) e = cudaMemset(c->d_jobs, 0, (4 + size_t(c->L) * n) * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(c->d_jobs, 0, (4 + 17 * size_t(c->L) * n) * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(c->d_epoch, 0, 2 * sizeof(unsigned long long));
     if (e == cudaSuccess)
         e = cudaMemcpy(c->d_members, members.data(), members.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
@@ -528,12 +531,12 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
     a.n = c->n;
     a.L = c->L;
     a.warm_layer = layer;
-    const size_t mb = size_t(c->max_batch);
-    a.plan.final_label = c->d_plan;
-    a.plan.stop_layer = c->d_plan + mb;
+    a.plan.frame_code = c->d_plan;
     a.plan.class_tag = c->d_tags;
     a.plan.job_count = c->d_jobs;
     a.plan.jobs = c->d_jobs + 4;
+    a.plan.items = c->d_jobs + 4 + size_t(c->L) * c->n;
+    a.m_next = c->d_m_next;
     a.plan.epoch = c->d_epoch;
     a.fallback = d_labels;
     a.split_current = c->d_split_current;
@@ -547,7 +550,7 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
         a.cnorm[l] = c->d_cnorm[l];
         a.m[l] = c->d_m[l];
     }
-    SMTM_CUDA(launch_update(a, nullptr, c->sm_count, st, c->side_stream, c->ev_fork, c->ev_join, &c->launches));
+    SMTM_CUDA(launch_update(a, nullptr, c->sm_count, st, &c->launches));
     return SMTM_OK;
 }
 

@@ -157,12 +157,12 @@ cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm
 
 // Scratch of an update (all device).
 struct UpdatePlan {
-    int32_t* final_label;            // [max_batch] label each frame ends up with (-1 = none)
-    int32_t* stop_layer;             // [max_batch] the paper's l at which its inference stopped
+    int32_t* frame_code;             // [max_batch] per frame: final label | stop layer (the paper's l) << 16, or -1 without a label
     unsigned long long* class_tag;   // [L][n] number of the last update call that touched (layer, class)
     int32_t* job_count;              // [0], [1]: (layer, class) pairs listed by this call ([number & 1]) and, zeroed, for the
-                                     // next; [2]: this call's count, published by the plan kernel's last CTA
+                                     // next; [2]: this call's count, published by the plan kernel's last CTA; [3]: its items
     int32_t* jobs;                   // [L][n] the (layer << 16 | class) pairs Eq. 7 touches in this call, in no particular order
+    int32_t* items;                  // [16][L][n] work items of the apply kernel: a pair, or one of the column blocks a heavy pair is cut into
     unsigned long long* epoch;       // [2] device: [0] number of update calls completed so far, [1] CTAs of the plan
                                      // kernel that are through (zero between calls).  The number lives on the
                                      // device so that a replayed CUDA graph counts on like eager calls do.
@@ -188,6 +188,7 @@ struct UpdateArgs {
     float* centers[SMTM_MAX_LAYERS];
     float* cnorm[SMTM_MAX_LAYERS];
     uint32_t* m[SMTM_MAX_LAYERS];
+    uint32_t* m_next;          // [L][n] scratch: the counts after this update, written by Eq. 7's CTAs, adopted by the norms kernel
 };
 
 
@@ -201,10 +202,7 @@ struct ResizeArgs {
 };
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches);
 // Tables and centres; with rz != nullptr also the Eq. 5 / Eq. 6 refresh of every stream that
-// had a frame in the batch.
-// side, fork, join: a second stream and two events (no timing) of the caller's, used to run the tables beside
-// the plan and the centres.
-cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, cudaStream_t side,
-                          cudaEvent_t fork, cudaEvent_t join, int64_t* launches);
+// had a frame in the batch.  Two launches on `st`.
+cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, int64_t* launches);
 
 }  // namespace smtm

@@ -5,18 +5,21 @@
 // ascending frame index, so the result is the one a frame-by-frame replay would give and does
 // not depend on scheduling.
 //
-// An update is three launches on two streams.  The plan kernel writes every frame's final label
-// and stop layer and lists the (layer, class) pairs Eq. 7 has to touch: up to 4096 frames and
+// An update is two launches on the caller's stream.  The plan kernel writes every frame's final
+// label and stop layer and lists the (layer, class) pairs Eq. 7 has to touch: up to 4096 frames and
 // 65 536 pairs a single CTA elects the pairs in a shared-memory bitmap (k_update_plan_one); past
 // that k_update_plan does it with many CTAs (the first frame to stamp a pair with the call's
 // sequence number appends it; the number is kept on the device and moved on by the kernel
-// itself, so that a replayed CUDA graph counts on exactly like eager calls).  The CTAs of
-// k_update_centers then walk that list.  k_update_tables depends on neither:
-// a warp per frame checks whether an earlier frame of the batch belongs to the same stream and
-// leaves if so, else it applies the stream's frames to the stream's tables (staged in shared memory)
-// and, when asked, refreshes the stream's fast memory (Eq. 5 / Eq. 6).  It runs on a side
-// stream, forked before the plan and joined after the centres, so the two halves of the update
-// overlap.  Classes and streams the batch does not touch cost nothing.
+// itself, so that a replayed CUDA graph counts on exactly like eager calls).  The apply kernel is
+// a grid of small CTAs (128 threads, a few KB of shared memory) with two kinds of work: the
+// first B CTAs look after the tables, one per frame (the CTA of a stream's first frame in the
+// batch applies all of the stream's frames to its tables and, when asked, refreshes its fast
+// memory by Eq. 5 / Eq. 6; the others leave at once); the remaining CTAs take the listed pairs,
+// one each, and fold the pair's frames into the centre (Eq. 7).  Small CTAs on purpose: there
+// are hundreds of independent pieces of work, each a short chain of dependent trips to L2, so
+// the kernel is as fast as the number of pieces in flight, and its CTAs fit beside the CTAs of a
+// streaming kernel that holds most of an SM's shared memory.  Classes and streams the batch does
+// not touch cost nothing.
 #include <algorithm>
 
 #include "common.cuh"
@@ -43,10 +46,8 @@ __device__ __forceinline__ void table_step(int& ft, int& ts, bool appears, int f
     }
 }
 
-constexpr int kUpdThreads = 256;
-constexpr int kUpdWarps = kUpdThreads / kWarp;
-constexpr int kTblWarps = 16;  // warps (streams) to a CTA of k_update_tables in its warp-per-stream form
-constexpr int kTblGroups = 16;  // groups of 32 frames a warp looks up per trip to memory
+constexpr int kUpdThreads = 256;   // plan kernel (many-CTA form) and the stand-alone refresh
+constexpr int kApplyThreads = 128; // CTAs of the apply kernel
 
 // The label a finished frame ends up with: the prediction if it exited, else the fallback label
 // (the full network's answer, -1 = none); a label outside the memory counts as no label.
@@ -56,6 +57,28 @@ __device__ __forceinline__ int final_label_of(const UpdateArgs& a, int b) {
 }
 
 // ---- plan -----------------------------------------------------------------------------------
+//
+// What the plan leaves for the kernels that follow: per frame its final label and stop layer packed into one
+// word (label | stop layer << 16, or -1 for a frame without a label); the list of
+// pairs (layer, class) Eq. 7 touches (`jobs`, job_count[2] of them); and the list of work items of the apply
+// kernel (`items`, job_count[3] of them): a pair whose frames are many is cut into several items, each a
+// block of the vector's columns, so that no CTA folds more than a few rows per thread.
+//   item = layer << 16 | class | block << 20 | log2(blocks) << 24      (class < 2^13, layer < 2^4, blocks <= 16)
+
+constexpr int kItemBlocksMax = 16;
+
+// Column blocks for a pair with `rows` frames at a layer whose vector has D entries: a CTA of the apply kernel
+// should not load more than about eight 16-byte pieces per thread.  A power of two, at most 16, and no block
+// narrower than 32 columns; vectors that are not a whole number of 16-byte pieces are never cut.
+__device__ __forceinline__ int item_blocks(int rows, int D) {
+    if (D & 3) return 1;
+    const int D4 = D >> 2;
+    const long long want = ((long long)rows * D4 + 8 * kApplyThreads - 1) / (8 * kApplyThreads);
+    int nb = 1;
+    while (nb < want && nb < kItemBlocksMax && (D4 / (2 * nb)) >= 8) nb *= 2;
+    return nb;
+}
+__device__ __forceinline__ int ilog2_pow2(int v) { return 31 - __clz(v); }
 
 // Label and stop layer of a finished frame: the prediction and exit layer if it exited,
 // else the fallback label (the full network's answer, -1 = none) and L.
@@ -78,16 +101,19 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a)
             lab = -1;
             set_status(a.status, kDevInvalidArg);
         }
-        a.plan.final_label[b] = lab;
-        a.plan.stop_layer[b] = ex ? el : a.L;
+        a.plan.frame_code[b] = lab < 0 ? -1 : (lab | ((ex ? el : a.L) << 16));
         if (lab >= 0) {
             // Eq. 7 touches the layers up to the stop layer: the first frame to stamp (layer, class)
-            // with the call's number lists the pair as a job
+            // with the call's number lists the pair as a job, and as a single item (this form of the plan
+            // does not count the frames of a pair)
             const int l_lo = a.warm_layer >= 0 ? a.warm_layer : 0;
             const int l_hi = a.warm_layer >= 0 ? a.warm_layer + 1 : (ex ? el : a.L);
             for (int l = l_lo; l < l_hi; ++l)
-                if (atomicExch(a.plan.class_tag + (size_t)l * a.n + lab, epoch) != epoch)
-                    a.plan.jobs[atomicAdd(a.plan.job_count + (epoch & 1), 1)] = (l << 16) | lab;
+                if (atomicExch(a.plan.class_tag + (size_t)l * a.n + lab, epoch) != epoch) {
+                    const int at = atomicAdd(a.plan.job_count + (epoch & 1), 1);
+                    a.plan.jobs[at] = (l << 16) | lab;
+                    a.plan.items[at] = (l << 16) | lab;
+                }
         }
     }
     if (b == 0) a.plan.job_count[(epoch + 1) & 1] = 0;  // the next call's counter (the call before this one is over)
@@ -97,25 +123,32 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a)
     __syncthreads();
     if (threadIdx.x == 0 && atomicAdd(a.plan.epoch + 1, 1ull) == gridDim.x - 1) {
         __threadfence();
-        a.plan.job_count[2] = *reinterpret_cast<volatile int32_t*>(a.plan.job_count + (epoch & 1));
+        const int jobs = *reinterpret_cast<volatile int32_t*>(a.plan.job_count + (epoch & 1));
+        a.plan.job_count[2] = jobs;
+        a.plan.job_count[3] = jobs;
         a.plan.epoch[1] = 0;
         a.plan.epoch[0] = epoch;
     }
 }
 
 // The same plan by a single CTA, for batches and memories small enough that one CTA's trip to
-// memory is all it takes: the pairs are elected in a bitmap in shared memory and counted there, so
-// nothing waits on a ticket or a fence.
+// memory is all it takes.  Up to kPlanCountMax pairs the frames of every pair are counted in shared memory
+// (integer atomics: a sum), and a pair is listed with as many items as its count asks for; beyond, the pairs
+// are only elected, in a bitmap, and listed with one item each.  Nothing waits on a ticket or a fence.
 constexpr int kPlanOneThreads = 1024;
 constexpr int kPlanOneMaxB = 4 * kPlanOneThreads;
-constexpr int kPlanOneWords = 2048;  // 65 536 (layer, class) pairs
+constexpr int kPlanOneWords = 2048;   // 65 536 (layer, class) pairs as a bitmap
+constexpr int kPlanCountMax = 8192;   // pairs that get a counter each
 
 __global__ void __launch_bounds__(kPlanOneThreads) k_update_plan_one(const UpdateArgs a) {
-    __shared__ unsigned int s_seen[kPlanOneWords];
-    __shared__ int s_jobs;
+    extern __shared__ int s_plan[];  // counters [pairs] or bitmap words
+    __shared__ int s_jobs, s_items;
     const int tid = threadIdx.x;
-    for (int i = tid; i < (a.L * a.n + 31) / 32; i += kPlanOneThreads) s_seen[i] = 0u;
-    if (tid == 0) s_jobs = 0;
+    const int pairs = a.L * a.n;
+    const bool counted = pairs <= kPlanCountMax;
+    const int words = counted ? pairs : (pairs + 31) / 32;
+    for (int i = tid; i < words; i += kPlanOneThreads) s_plan[i] = 0;
+    if (tid == 0) s_jobs = s_items = 0;
     chain_wait();
     chain_release();
     const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_PLAN : nullptr);
@@ -131,20 +164,42 @@ __global__ void __launch_bounds__(kPlanOneThreads) k_update_plan_one(const Updat
             lab = -1;
             set_status(a.status, kDevInvalidArg);
         }
-        a.plan.final_label[b] = lab;
-        a.plan.stop_layer[b] = ex ? el : a.L;
+        a.plan.frame_code[b] = lab < 0 ? -1 : (lab | ((ex ? el : a.L) << 16));
         if (lab >= 0) {
             const int l_lo = a.warm_layer >= 0 ? a.warm_layer : 0;
             const int l_hi = a.warm_layer >= 0 ? a.warm_layer + 1 : (ex ? el : a.L);
             for (int l = l_lo; l < l_hi; ++l) {
                 const int pair = l * a.n + lab;
-                const unsigned int bit = 1u << (pair & 31);
-                if (!(atomicOr(&s_seen[pair >> 5], bit) & bit)) a.plan.jobs[atomicAdd(&s_jobs, 1)] = (l << 16) | lab;
+                if (counted) {
+                    atomicAdd(&s_plan[pair], 1);
+                } else {
+                    const unsigned int bit = 1u << (pair & 31);
+                    if (!(atomicOr(reinterpret_cast<unsigned int*>(&s_plan[pair >> 5]), bit) & bit)) {
+                        const int at = atomicAdd(&s_jobs, 1);
+                        a.plan.jobs[at] = (l << 16) | lab;
+                        a.plan.items[at] = (l << 16) | lab;
+                    }
+                }
             }
         }
     }
     __syncthreads();
-    if (tid == 0) a.plan.job_count[2] = s_jobs;
+    if (counted) {
+        for (int pair = tid; pair < pairs; pair += kPlanOneThreads) {
+            const int rows = s_plan[pair];
+            if (rows == 0) continue;
+            const int l = pair / a.n, code = (l << 16) | (pair - l * a.n);
+            a.plan.jobs[atomicAdd(&s_jobs, 1)] = code;
+            const int nb = item_blocks(rows, a.dims[l]), lg = ilog2_pow2(nb);
+            const int at = atomicAdd(&s_items, nb);
+            for (int k = 0; k < nb; ++k) a.plan.items[at + k] = code | (k << 20) | (lg << 24);
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        a.plan.job_count[2] = s_jobs;
+        a.plan.job_count[3] = counted ? s_items : s_jobs;
+    }
 }
 
 // ---- Eq. 5 / Eq. 6 ------------------------------------------------------------------------
@@ -157,137 +212,249 @@ __device__ __forceinline__ unsigned long long score_of(int ft, int ts, int W, in
     return f << (2 * (kEMax - e));  // FT * 4^(12 - e) = 4^12 * FT * 0.25^e
 }
 
-__host__ __device__ constexpr size_t resize_smem(int n, int k_max) { return size_t(n) * 8 + size_t(n + (n & 1)) * 4 + size_t(k_max) * 8; }
-// The one-CTA-per-stream refresh sorts: its score and id arrays are padded to a power of two.
 __host__ __device__ constexpr int pow2_at_least(int v) {
     int p = 2;
     while (p < v) p *= 2;
     return p;
 }
-__host__ __device__ constexpr size_t resize_cta_smem(int n, int k_max) {
-    return size_t(pow2_at_least(n)) * 12 + size_t(k_max) * 8;
+// Ranking key of a class with a non-zero score: the score above the complement of the class id, so that a
+// larger key means (score descending, id ascending).  Scores stay below 2^44 (FT <= 2^20 times 4^12, or a
+// fixed-point FT below 2^31) and ids below 2^13.
+static_assert(SMTM_MAX_CLASSES <= (1 << 13), "the ranking key keeps 13 bits for the class id");
+__device__ __forceinline__ unsigned long long refresh_key(unsigned long long score, int id) {
+    return (score << 13) | (unsigned long long)(8191 - id);
+}
+__device__ __forceinline__ int key_class(unsigned long long key) { return 8191 - int(key & 8191ull); }
+__device__ __forceinline__ unsigned long long key_score(unsigned long long key) { return key >> 13; }
+
+// Shared memory of a refresh: the keys of the non-zero scores (padded to a power of two for the sort) and the
+// k_max best scores.
+__host__ __device__ constexpr size_t refresh_smem(int n, int k_max) { return size_t(pow2_at_least(n)) * 8 + size_t(k_max) * 8; }
+
+constexpr int kCountRankMax = 256;  // up to this many non-zero scores are ranked by counting, more by sorting
+
+// Sum over the block of a 64-bit value; every thread gets the total.  s_part holds >= 32 words.
+__device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v, unsigned long long* s_part) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = v;
+    __syncthreads();
+    unsigned long long t = 0;
+    for (int w = 0; w < int(blockDim.x + 31) >> 5; ++w) t += s_part[w];
+    return t;
 }
 
-// Refresh of one stream's fast memory by a CTA of kUpdThreads threads.  Classes with a
-// non-zero score are compacted in ascending id and ranked among themselves by counting;
-// zero-score classes follow in ascending id.  `smem` holds resize_cta_smem(n, k_max) bytes.
-__device__ void resize_stream(const ResizeArgs& a, int s, unsigned char* smem, int* s_scan,
-                              unsigned long long* s_part) {
-    unsigned long long* s_score = reinterpret_cast<unsigned long long*>(smem);  // [n] compacted non-zero scores
-    const int cap = pow2_at_least(a.n);                                         // both arrays hold `cap` entries
-    int* s_id = reinterpret_cast<int*>(s_score + cap);                          // their class ids
-    unsigned long long* s_top = reinterpret_cast<unsigned long long*>(s_id + cap);  // [k_max]
-    const int tid = threadIdx.x;
-    const int32_t* ft = a.ft + (size_t)s * a.n;
-    const int32_t* ts = a.ts + (size_t)s * a.n;
-    int32_t* mem = a.members + (size_t)s * a.k_max;
-
-    // pass 1: compact the non-zero scores (ascending id) and add everything up
-    int nz = 0;
-    unsigned long long local = 0;
-    for (int c0 = 0; c0 < a.n; c0 += kUpdThreads) {
-        const int c = c0 + tid;
-        const unsigned long long sc = c < a.n ? score_of(ft[c], ts[c], a.W, a.forgetting) : 0ull;
-        int cnt;
-        const int pos = block_exclusive_scan(sc != 0 ? 1 : 0, s_scan, &cnt);
-        if (sc != 0) {
-            s_score[nz + pos] = sc;
-            s_id[nz + pos] = c;
-        }
-        nz += cnt;
-        local += sc;
-    }
+// Eq. 6 by one warp: the smallest k in [k_min, k_max] with cl_den * (sum of the k best scores) > cl_num * total,
+// by a scan of 32 entries per step; s_top holds the k_max best scores in rank order.
+__device__ __forceinline__ void adaptive_size(const ResizeArgs& a, int s, const unsigned long long* s_top,
+                                              unsigned long long total, int lane) {
+    unsigned long long carry = 0;
+    int chosen = a.k_max;
+    for (int base = 0; base < a.k_max; base += kWarp) {
+        const int idx = base + lane;
+        unsigned long long v = idx < a.k_max ? s_top[idx] : 0ull;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(kFull, local, o);
-    __syncthreads();
-    if ((tid & 31) == 0) s_part[tid >> 5] = local;
-    __syncthreads();
-    unsigned long long total = 0;
-    for (int w = 0; w < kUpdThreads / 32; ++w) total += s_part[w];
-    if (total == 0) return;  // nothing seen yet: keep size and members
-
-    // pass 2: order the non-zero classes by (score descending, id ascending): a bitonic sort of the
-    // pairs, padded to a power of two with entries that rank last; rank r < k_max goes to slot r
-    const int P = pow2_at_least(nz);
-    for (int i = nz + tid; i < P; i += kUpdThreads) {
-        s_score[i] = 0ull;
-        s_id[i] = INT32_MAX;
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long t = __shfl_up_sync(kFull, v, o);
+            if (lane >= o) v += t;
+        }
+        const unsigned long long prefix = carry + v;
+        const bool ok = idx < a.k_max && idx + 1 >= a.k_min &&
+                        (unsigned long long)a.cl_den * prefix > (unsigned long long)a.cl_num * total;
+        const unsigned m = __ballot_sync(kFull, ok);
+        if (m) {
+            chosen = base + __ffs(m);
+            break;
+        }
+        carry += __shfl_sync(kFull, v, 31);
     }
+    if (lane == 0) a.k[s] = chosen;
+}
+
+// Descending bitonic sort of nz keys in s_key by the whole CTA (padded to a power of two with zeros: no key is zero).
+__device__ void sort_keys(unsigned long long* s_key, int nz) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int P = pow2_at_least(nz);
+    for (int i = nz + tid; i < P; i += nt) s_key[i] = 0ull;
     __syncthreads();
     for (int k = 2; k <= P; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int t = tid; t < P / 2; t += kUpdThreads) {
+            for (int t = tid; t < P / 2; t += nt) {
                 const int i = 2 * j * (t / j) + (t % j), l = i + j;
-                const unsigned long long si = s_score[i], sl = s_score[l];
-                const int ii = s_id[i], il = s_id[l];
-                const bool l_first = sl > si || (sl == si && il < ii);  // the entry at l ranks before the one at i
-                if (((i & k) == 0) ? l_first : !l_first) {             // (ids are distinct: never equal)
-                    s_score[i] = sl; s_score[l] = si;
-                    s_id[i] = il; s_id[l] = ii;
+                const unsigned long long ki = s_key[i], kl = s_key[l];
+                if (((i & k) == 0) ? kl > ki : kl < ki) {
+                    s_key[i] = kl;
+                    s_key[l] = ki;
                 }
             }
             __syncthreads();
         }
     }
-    for (int r = tid; r < nz && r < a.k_max; r += kUpdThreads) {
-        mem[r] = s_id[r];
-        s_top[r] = s_score[r];
-    }
-    // pass 3: zero-score classes fill the remaining slots in ascending id
-    if (nz < a.k_max) {
-        int filled = nz;
-        for (int c0 = 0; c0 < a.n && filled < a.k_max; c0 += kUpdThreads) {
-            const int c = c0 + tid;
-            const int z = (c < a.n && score_of(ft[c], ts[c], a.W, a.forgetting) == 0) ? 1 : 0;
-            int cnt;
-            const int pos = block_exclusive_scan(z, s_scan, &cnt);
-            if (z && filled + pos < a.k_max) {
-                mem[filled + pos] = c;
-                s_top[filled + pos] = 0;
+}
+
+// Eq. 5 / Eq. 6 for stream s when every thread of the CTA holds the scores of its PER consecutive classes
+// (c_lo ...) in registers.  The keys of the non-zero scores are appended to a list in shared memory in whatever
+// order the threads come (a key carries its class, and ranking by key does not care about the list's order);
+// the rest is one warp's work: ranks by counting (a sort by the whole CTA when the keys are many), zero-score
+// classes in ascending id for the slots that remain (they are among the first k_max ids), Eq. 6.
+// `dyn`: keys [pow2 >= n] | best scores [k_max] | zero flags [k_max] bytes.  *s_nz and *s_total are zero on entry.
+template <int PER>
+__device__ void refresh_from_registers(const ResizeArgs& a, int s, const unsigned long long (&sc)[PER], int c_lo,
+                                       unsigned char* dyn, int* s_nz, unsigned long long* s_total) {
+    const int cap = pow2_at_least(a.n);
+    unsigned long long* s_key = reinterpret_cast<unsigned long long*>(dyn);  // [cap]
+    unsigned long long* s_top = s_key + cap;                                 // [k_max]
+    unsigned char* s_zero = reinterpret_cast<unsigned char*>(s_top + a.k_max);  // [k_max]
+    const int tid = threadIdx.x, lane = tid & 31;
+    unsigned long long local = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int c = c_lo + i;
+        if (c < a.n) {
+            if (sc[i] != 0) {
+                s_key[atomicAdd(s_nz, 1)] = refresh_key(sc[i], c);
+                local += sc[i];
             }
-            filled += cnt;
+            if (c < a.k_max) s_zero[c] = sc[i] == 0 ? 1 : 0;
         }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(kFull, local, o);
+    if (lane == 0 && local != 0) atomicAdd(s_total, local);
+    __syncthreads();
+    const int nz = *s_nz;
+    const unsigned long long total = *s_total;
+    if (total == 0) return;  // nothing seen yet: keep size and members (the same for every thread)
+    const bool sorted = nz > kCountRankMax;
+    if (sorted) sort_keys(s_key, nz);
+    if (tid >= kWarp) return;
+    int32_t* mem = a.members + (size_t)s * a.k_max;
+    if (sorted) {
+        for (int r = lane; r < nz && r < a.k_max; r += kWarp) {
+            mem[r] = key_class(s_key[r]);
+            s_top[r] = key_score(s_key[r]);
+        }
+    } else {
+        for (int i = lane; i < nz; i += kWarp) {  // rank = keys larger than this one (keys are distinct)
+            const unsigned long long key = s_key[i];
+            int r0 = 0, r1 = 0;
+            int j = 0;
+            for (; j + 1 < nz; j += 2) {
+                r0 += s_key[j] > key ? 1 : 0;
+                r1 += s_key[j + 1] > key ? 1 : 0;
+            }
+            if (j < nz) r0 += s_key[j] > key ? 1 : 0;
+            const int r = r0 + r1;
+            if (r < a.k_max) {
+                mem[r] = key_class(key);
+                s_top[r] = key_score(key);
+            }
+        }
+    }
+    const unsigned lt = (1u << lane) - 1u;
+    int filled = nz;
+    for (int c0 = 0; c0 < a.k_max && filled < a.k_max; c0 += kWarp) {
+        const int c = c0 + lane;
+        const bool z = c < a.k_max && s_zero[c] != 0;
+        const unsigned m = __ballot_sync(kFull, z);
+        const int pos = filled + __popc(m & lt);
+        if (z && pos < a.k_max) {
+            mem[pos] = c;
+            s_top[pos] = 0;
+        }
+        filled += __popc(m);
+    }
+    __syncwarp();
+    adaptive_size(a, s, s_top, total, lane);
+}
+
+// Eq. 5 / Eq. 6 for stream s by the whole CTA (any number of threads), from the stream's tables in global memory
+// as this CTA left them.  Every thread looks after a run of consecutive classes; the keys of the
+// non-zero scores are compacted by one scan over the threads and ranked, largest first: by counting when they
+// are few, by a bitonic sort otherwise; zero-score classes follow in ascending id.  Then the smallest k in
+// [k_min, k_max] whose k best scores exceed cl_num / cl_den of all.  `dyn` holds refresh_smem(n, k_max) bytes.
+__device__ void refresh_stream(const ResizeArgs& a, int s, unsigned char* dyn, int* s_scan, unsigned long long* s_part) {
+    const int cap = pow2_at_least(a.n);
+    unsigned long long* s_key = reinterpret_cast<unsigned long long*>(dyn);  // [cap]
+    unsigned long long* s_top = s_key + cap;                                 // [k_max]
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int32_t* ft = a.ft + (size_t)s * a.n;
+    const int32_t* ts = a.ts + (size_t)s * a.n;
+    int32_t* mem = a.members + (size_t)s * a.k_max;
+    const int per = (a.n + nt - 1) / nt;
+    const int c_lo = min(a.n, tid * per), c_hi = min(a.n, c_lo + per);
+    const auto score_at = [&](int c) { return score_of(ft[c], ts[c], a.W, a.forgetting); };
+
+    int nzl = 0;
+    unsigned long long local = 0;
+    for (int c = c_lo; c < c_hi; ++c) {
+        const unsigned long long sc = score_at(c);
+        nzl += sc != 0 ? 1 : 0;
+        local += sc;
+    }
+    int nz;
+    int pos = block_exclusive_scan(nzl, s_scan, &nz);
+    const unsigned long long total = block_sum_u64(local, s_part);
+    if (total == 0) return;  // nothing seen yet: keep size and members (the same for every thread)
+    for (int c = c_lo; c < c_hi && nzl; ++c) {
+        const unsigned long long sc = score_at(c);
+        if (sc != 0) s_key[pos++] = refresh_key(sc, c);
     }
     __syncthreads();
-    // pass 4: smallest k in [k_min, k_max] with cl_den * prefix(k) > cl_num * total
-    if (tid < kWarp) {  // warp 0: a scan of 32 entries per step
-        const int lane = tid;
-        unsigned long long carry = 0;
-        int chosen = a.k_max;
-        for (int base = 0; base < a.k_max; base += kWarp) {
-            const int idx = base + lane;
-            unsigned long long v = idx < a.k_max ? s_top[idx] : 0ull;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const unsigned long long t = __shfl_up_sync(kFull, v, o);
-                if (lane >= o) v += t;
+    if (nz <= kCountRankMax) {
+        // rank = keys larger than this one (keys are distinct); rank r < k_max goes to slot r
+        for (int i = tid; i < nz; i += nt) {
+            const unsigned long long key = s_key[i];
+            int r0 = 0, r1 = 0;
+            int j = 0;
+            for (; j + 1 < nz; j += 2) {
+                r0 += s_key[j] > key ? 1 : 0;
+                r1 += s_key[j + 1] > key ? 1 : 0;
             }
-            const unsigned long long prefix = carry + v;
-            const bool ok = idx < a.k_max && idx + 1 >= a.k_min &&
-                            (unsigned long long)a.cl_den * prefix > (unsigned long long)a.cl_num * total;
-            const unsigned m = __ballot_sync(kFull, ok);
-            if (m) {
-                chosen = base + __ffs(m);
-                break;
+            if (j < nz) r0 += s_key[j] > key ? 1 : 0;
+            const int r = r0 + r1;
+            if (r < a.k_max) {
+                mem[r] = key_class(key);
+                s_top[r] = key_score(key);
             }
-            carry += __shfl_sync(kFull, v, 31);
         }
-        if (lane == 0) a.k[s] = chosen;
+    } else {
+        sort_keys(s_key, nz);
+        for (int r = tid; r < nz && r < a.k_max; r += nt) {
+            mem[r] = key_class(s_key[r]);
+            s_top[r] = key_score(s_key[r]);
+        }
     }
+    // zero-score classes fill the remaining slots in ascending id
+    if (nz < a.k_max) {
+        int zl = 0;
+        for (int c = c_lo; c < c_hi; ++c) zl += score_at(c) == 0 ? 1 : 0;
+        int zt;
+        int zp = nz + block_exclusive_scan(zl, s_scan, &zt);
+        for (int c = c_lo; c < c_hi && zl && zp < a.k_max; ++c)
+            if (score_at(c) == 0) {
+                mem[zp] = c;
+                s_top[zp] = 0;
+                ++zp;
+            }
+    }
+    __syncthreads();
+    if (tid < kWarp) adaptive_size(a, s, s_top, total, tid);
 }
 
 __global__ void __launch_bounds__(kUpdThreads) k_resize(const ResizeArgs a) {
     extern __shared__ unsigned long long s_dyn[];
     __shared__ int s_scan[33];
-    __shared__ unsigned long long s_part[kUpdThreads / 32];
+    __shared__ unsigned long long s_part[32];
     chain_wait();
     chain_release();
-    resize_stream(a, blockIdx.x, reinterpret_cast<unsigned char*>(s_dyn), s_scan, s_part);
+    refresh_stream(a, blockIdx.x, reinterpret_cast<unsigned char*>(s_dyn), s_scan, s_part);
 }
 
-// ---- apply ------------------------------------------------------------------------------------
+// ---- apply: tables ----------------------------------------------------------------------------
 
-// Compacts, in ascending frame index, the frames of a tile of kUpdThreads for which `hit`
+// Compacts, in ascending frame index, the frames of a tile of blockDim.x for which `hit`
 // is set into list[0..cnt); returns cnt (the same in every thread).
 __device__ __forceinline__ int compact_tile(int hit, int value, int* list, int* s_scan) {
     int cnt;
@@ -300,438 +467,343 @@ __device__ __forceinline__ int compact_tile(int hit, int value, int* list, int* 
     return cnt;
 }
 
-// Sec. 6.1 for the stream whose first frame in the batch is g, by one warp with the stream's
-// tables in registers (class c lives in lane c % 32, register c / 32), then, if asked, that
-// stream's Eq. 5 / Eq. 6 refresh.  `smem` is this warp's resize_smem(n, k_max) bytes.
-// 16 bytes from global to shared memory without passing through registers (both addresses 16-byte
-// aligned); the thread goes on and collects all of its copies with copy_async_wait_all().
-__device__ __forceinline__ void copy_async_16(void* smem_dst, const void* gmem_src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+// Shared memory of a tables CTA: the refresh buffers, which also serve as the two integer arrays [n] of the
+// closed form before the refresh begins.
+__host__ __device__ constexpr size_t tables_smem(int n, int k_max, bool with_refresh) {
+    const size_t closed = size_t(n) * 2 * sizeof(int);
+    const size_t refresh = with_refresh ? refresh_smem(n, k_max) + size_t(k_max) : 0;  // ... and a flag per slot
+    return closed > refresh ? closed : refresh;
 }
-__device__ __forceinline__ void copy_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
-// The stream's tables are staged in shared memory (class c belongs to lane c % 32) and every pass
-// over the classes is a rolled loop: the kernel runs once per warp, so its time is the time to
-// fetch its instructions, and unrolled loops over registers were several times slower.
-__host__ __device__ constexpr size_t tables_smem(int n, int k_max) { return resize_smem(n, k_max) + size_t(n + (n & 1)) * 8; }
-
-__device__ void tables_by_warp(const UpdateArgs& a, const ResizeArgs& rz, int g, int s, int do_resize,
-                               unsigned char* smem, int* s_hits) {
-    const int lane = threadIdx.x & 31;
-    const unsigned lt = (1u << lane) - 1u;
-    int32_t* ftp = a.ft + (size_t)s * a.n;
-    int32_t* tsp = a.ts + (size_t)s * a.n;
-    int* s_ft = reinterpret_cast<int*>(smem + resize_smem(a.n, rz.k_max));  // [n]
-    int* s_ts = s_ft + a.n + (a.n & 1);                                     // [n]
-    // Staged by 16-byte asynchronous copies where the rows allow it: every copy is in flight at once and
-    // lands while the stream's frames are being looked up below.
-    const bool staged_async = (a.n & 3) == 0 && ((reinterpret_cast<uintptr_t>(ftp) | reinterpret_cast<uintptr_t>(tsp) |
-                                                   smem_u32(s_ft) | smem_u32(s_ts)) & 15) == 0;
-    if (staged_async) {
-        for (int v = lane; v < a.n / 4; v += kWarp) {
-            copy_async_16(s_ft + 4 * v, ftp + 4 * v);
-            copy_async_16(s_ts + 4 * v, tsp + 4 * v);
-        }
-    } else {
-#pragma unroll 4
-        for (int c = lane; c < a.n; c += kWarp) {
-            s_ft[c] = ftp[c];
-            s_ts[c] = tsp[c];
+// Sec. 6.1 for the stream of frame g by one CTA, if g is the stream's first frame in the batch (else the
+// CTA of that frame does it): all of the stream's frames, in ascending index, applied to its tables; then,
+// if asked, the stream's Eq. 5 / Eq. 6 refresh.  Every thread looks after a run of PER consecutive classes
+// and keeps their entries in registers from the one trip to memory that fetches them to the refresh
+// (PER == 0: any number of classes, the entries stay in global memory).
+template <int PER>
+__device__ void tables_of_frame(const UpdateArgs& a, const ResizeArgs& rz, int g, int do_resize, unsigned char* dyn,
+                                int* s_list, int* s_scan, unsigned long long* s_part) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    if (tid == 0) {  // the refresh's counters (read after the barriers below)
+        s_scan[32] = 0;
+        s_part[31] = 0ull;
+    }
+    const int s = a.stream_id ? a.stream_id[g] : 0;
+    if (s < 0 || s >= a.S) return;  // no such stream (the same for every thread; the plan kernel records the error)
+    const int per = PER ? PER : (a.n + nt - 1) / nt;
+    const int c_lo = min(a.n, tid * per), c_hi = min(a.n, c_lo + per);
+    int32_t* ft = a.ft + (size_t)s * a.n;
+    int32_t* ts = a.ts + (size_t)s * a.n;
+    // the label frame g ends up with, every load issued at once (final_label_of would wait for the exit flag first)
+    const int dn_g = a.done ? a.done[g] : 0, pr_g = a.done ? a.pred[g] : -1, fb_g = a.fallback ? a.fallback[g] : -1;
+    int f[PER ? PER : 1], t[PER ? PER : 1];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {  // in flight with the stream ids below
+        f[i] = c_lo + i < a.n ? ft[c_lo + i] : 0;
+        t[i] = c_lo + i < a.n ? ts[c_lo + i] : 0;
+    }
+    // an earlier frame of the same stream: its CTA does the work.  Also: is g the stream's only frame?
+    int earlier = (!a.stream_id && g > 0) ? 1 : 0, later = (!a.stream_id && g + 1 < a.B) ? 1 : 0;
+    for (int b0 = 0; a.stream_id && b0 < a.B; b0 += 4 * nt) {
+        int sidv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) sidv[u] = a.stream_id[min(b0 + u * nt + tid, a.B - 1)];  // one trip to memory
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int b = b0 + u * nt + tid;
+            const int same = (b < a.B && sidv[u] == s) ? 1 : 0;
+            earlier |= (b < g) ? same : 0;
+            later |= (b > g) ? same : 0;
         }
     }
-    // Plain counts have a closed form (see the one-CTA-per-stream variant in k_update_tables): per class
-    // the number of appearances and the position of the last one, gathered in the space the refresh
-    // uses afterwards.  The forgetting table is replayed frame by frame.
-    const bool plain = a.forget_W == 0;
-    int* s_cnt = reinterpret_cast<int*>(smem);  // [n]
-    int* s_last = s_cnt + a.n;                  // [n]
-    if (plain)
-        for (int c = lane; c < a.n; c += kWarp) {
+    if (__syncthreads_or(earlier)) return;
+    const bool single = !__syncthreads_or(later);
+    int label_g = dn_g != 0 ? pr_g : fb_g;
+    if (label_g >= a.n) label_g = -1;
+    if (single) {
+        // one frame (a video stream that delivers a frame per step): Sec. 6.1 as printed, one pass over the classes
+        if (PER) {
+#pragma unroll
+            for (int i = 0; i < PER; ++i) table_step(f[i], t[i], c_lo + i == label_g, a.forget_W);
+        } else {
+            for (int c = c_lo; c < c_hi; ++c) {
+                int fc = ft[c], tc = ts[c];
+                table_step(fc, tc, c == label_g, a.forget_W);
+                ft[c] = fc;
+                ts[c] = tc;
+            }
+        }
+    } else if (a.forget_W == 0) {
+        // Plain counts: what a frame-by-frame replay leaves behind has a closed form per class.  With
+        // m frames of the stream in the batch, a class that appears q times, last at position p, ends
+        // with FT + q and TS = m - 1 - p; one that does not appear ends with TS + m.  q and p are
+        // gathered by shared-memory atomics on integers (a sum and a maximum: order does not matter).
+        int* s_cnt = reinterpret_cast<int*>(dyn);  // [n]; the refresh below reuses the space
+        int* s_last = s_cnt + a.n;                 // [n]
+        for (int c = tid; c < a.n; c += nt) {
             s_cnt[c] = 0;
             s_last[c] = -1;
         }
-    __syncwarp();
-    int m = 0;  // frames of the stream so far
-    // The stream's frames in ascending index (none precedes g), kTblGroups groups of 32 frames per trip
-    // to memory: their labels are listed in order (s_hits, this warp's), then applied.
-    for (int b0 = g - g % kWarp; b0 < a.B; b0 += kTblGroups * kWarp) {
-        int sidv[kTblGroups], labv[kTblGroups];
-#pragma unroll
-        for (int u = 0; u < kTblGroups; ++u) {  // unconditional loads (a clamped index), all in flight at once
-            const int bb = min(b0 + u * kWarp + lane, a.B - 1);
-            sidv[u] = a.stream_id ? a.stream_id[bb] : 0;
-            const int dn = a.done ? a.done[bb] : 0, pr = a.done ? a.pred[bb] : -1, fb = a.fallback ? a.fallback[bb] : -1;
-            const int lab = dn != 0 ? pr : fb;  // final_label_of with every load issued up front
-            labv[u] = lab >= a.n ? -1 : lab;
-        }
-        int n_hits = 0;
-#pragma unroll
-        for (int u = 0; u < kTblGroups; ++u) {
-            const int b = b0 + u * kWarp + lane;
-            const bool hit = b >= g && b < a.B && sidv[u] == s;
-            const unsigned mask = __ballot_sync(kFull, hit);
-            if (hit) s_hits[n_hits + __popc(mask & lt)] = labv[u];
-            n_hits += __popc(mask);
-        }
-        __syncwarp();
-        if (!plain && staged_async) {  // the replay works on the staged tables
-            copy_async_wait_all();
-            __syncwarp();
-        }
-        if (plain) {
-            for (int h = lane; h < n_hits; h += kWarp) {
-                const int l = s_hits[h];
-                if (l >= 0) {
-                    atomicAdd(&s_cnt[l], 1);
-                    atomicMax(&s_last[l], m + h);
-                }
+        __syncthreads();
+        int m = 0;
+        for (int t0 = g - g % nt; t0 < a.B; t0 += nt) {
+            const int b = t0 + tid;
+            const int hit = (b >= g && b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
+            const int cnt = compact_tile(hit, hit ? final_label_of(a, b) : -1, s_list, s_scan);
+            if (tid < cnt && s_list[tid] >= 0) {
+                atomicAdd(&s_cnt[s_list[tid]], 1);
+                atomicMax(&s_last[s_list[tid]], m + tid);
             }
-        } else {
-#pragma unroll 1
-            for (int h = 0; h < n_hits; ++h) {
-                const int l = s_hits[h];
-#pragma unroll 2
-                for (int c = lane; c < a.n; c += kWarp) table_step(s_ft[c], s_ts[c], c == l, a.forget_W);
-            }
+            m += cnt;
         }
-        m += n_hits;
-        __syncwarp();
-    }
-    if (staged_async) {
-        copy_async_wait_all();
-        __syncwarp();
-    }
-    if (plain)
-        for (int c = lane; c < a.n; c += kWarp) {
+        __syncthreads();
+        const auto closed = [&](int c, int& fc, int& tc) {
             const int q = s_cnt[c];
             if (q > 0) {
-                s_ft[c] = int(min((long long)s_ft[c] + q, (long long)kFtMax));
-                s_ts[c] = m - 1 - s_last[c];
+                fc = int(min((long long)fc + q, (long long)kFtMax));
+                tc = m - 1 - s_last[c];
             } else {
-                s_ts[c] = int(min((long long)s_ts[c] + m, (long long)INT32_MAX));
+                tc = int(min((long long)tc + m, (long long)INT32_MAX));
             }
-        }
-    __syncwarp();
-#pragma unroll 4
-    for (int c = lane; c < a.n; c += kWarp) {
-        ftp[c] = s_ft[c];
-        tsp[c] = s_ts[c];
-    }
-    if (!do_resize) return;
-
-    // Eq. 5 scores; non-zero ones compacted in ascending class id
-    unsigned long long* s_score = reinterpret_cast<unsigned long long*>(smem);  // [n]
-    int* s_id = reinterpret_cast<int*>(s_score + a.n);                          // [n]
-    unsigned long long* s_top = reinterpret_cast<unsigned long long*>(s_id + a.n + (a.n & 1));  // [k_max]
-    int32_t* mem = rz.members + (size_t)s * rz.k_max;
-    unsigned long long total = 0;
-    int nz = 0;
-#pragma unroll 1
-    for (int c0 = 0; c0 < a.n; c0 += kWarp) {
-        const int c = c0 + lane;
-        const unsigned long long sc = c < a.n ? score_of(s_ft[c], s_ts[c], rz.W, rz.forgetting) : 0ull;
-        const unsigned m = __ballot_sync(kFull, sc != 0);
-        if (sc != 0) {
-            const int pos = nz + __popc(m & lt);
-            s_score[pos] = sc;
-            s_id[pos] = c;
-        }
-        nz += __popc(m);
-        total += sc;
-    }
+        };
+        if (PER) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(kFull, total, o);
-    if (total == 0) return;  // nothing seen yet: keep size and members
-    __syncwarp();
-    // rank the non-zero classes by counting; rank r < k_max goes to slot r
-    for (int i = lane; i < nz; i += kWarp) {
-        const unsigned long long sc = s_score[i];
-        int r0 = 0, r1 = 0, r2 = 0, r3 = 0;  // four counters: the loop is a chain of additions otherwise
-        int j = 0;
-        for (; j + 3 < nz; j += 4) {
-            const unsigned long long o0 = s_score[j], o1 = s_score[j + 1], o2 = s_score[j + 2], o3 = s_score[j + 3];
-            r0 += (o0 > sc || (o0 == sc && j < i)) ? 1 : 0;  // compacted order is ascending id
-            r1 += (o1 > sc || (o1 == sc && j + 1 < i)) ? 1 : 0;
-            r2 += (o2 > sc || (o2 == sc && j + 2 < i)) ? 1 : 0;
-            r3 += (o3 > sc || (o3 == sc && j + 3 < i)) ? 1 : 0;
-        }
-        for (; j < nz; ++j) {
-            const unsigned long long o = s_score[j];
-            r0 += (o > sc || (o == sc && j < i)) ? 1 : 0;
-        }
-        const int r = (r0 + r1) + (r2 + r3);
-        if (r < rz.k_max) {
-            mem[r] = s_id[i];
-            s_top[r] = sc;
-        }
-    }
-    // zero-score classes fill the remaining slots in ascending id
-    int filled = nz;
-#pragma unroll 1
-    for (int c0 = 0; c0 < a.n && filled < rz.k_max; c0 += kWarp) {
-        const int c = c0 + lane;
-        const bool z = c < a.n && score_of(s_ft[c], s_ts[c], rz.W, rz.forgetting) == 0;
-        const unsigned m = __ballot_sync(kFull, z);
-        if (z) {
-            const int pos = filled + __popc(m & lt);
-            if (pos < rz.k_max) {
-                mem[pos] = c;
-                s_top[pos] = 0;
-            }
-        }
-        filled += __popc(m);
-    }
-    __syncwarp();
-    // Eq. 6: smallest k in [k_min, k_max] with cl_den * prefix(k) > cl_num * total
-    unsigned long long carry = 0;
-    int chosen = rz.k_max;
-    for (int base = 0; base < rz.k_max; base += kWarp) {
-        const int idx = base + lane;
-        unsigned long long v = idx < rz.k_max ? s_top[idx] : 0ull;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned long long t = __shfl_up_sync(kFull, v, o);
-            if (lane >= o) v += t;
-        }
-        const unsigned long long prefix = carry + v;
-        const bool ok = idx < rz.k_max && idx + 1 >= rz.k_min &&
-                        (unsigned long long)rz.cl_den * prefix > (unsigned long long)rz.cl_num * total;
-        const unsigned m = __ballot_sync(kFull, ok);
-        if (m) {
-            chosen = base + __ffs(m);
-            break;
-        }
-        carry += __shfl_sync(kFull, v, 31);
-    }
-    if (lane == 0) rz.k[s] = chosen;
-}
-
-// Tables (and, if asked, the refresh) of the streams whose first frames are among this CTA's
-// frames: a warp per frame, or, when the classes do not fit a warp's registers, the whole CTA
-// for one frame.
-__global__ void __launch_bounds__(kTblWarps * kWarp) k_update_tables(const UpdateArgs a, const ResizeArgs rz, int do_resize,
-                                                               int warp_tables) {
-    extern __shared__ unsigned long long s_dyn[];
-    __shared__ int s_list[kUpdThreads];
-    __shared__ int s_scan[33];
-    __shared__ unsigned long long s_part[kUpdWarps];
-    __shared__ int s_hits[kTblWarps][kTblGroups * kWarp];  // labels of a stream's frames among 512 consecutive ones, per warp
-    const int tid = threadIdx.x;
-    chain_wait();
-    chain_release();
-    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_TABLES : nullptr, true);
-    {
-        if (warp_tables) {
-            const int g = blockIdx.x * (blockDim.x >> 5) + (tid >> 5);  // the launch decides how many warps share a CTA
-            if (g >= a.B) return;
-            const int s = a.stream_id ? a.stream_id[g] : 0;
-            if (s < 0 || s >= a.S) return;  // no such stream: nothing to update (the plan kernel records the error)
-            // not the stream's first frame in the batch: the warp of that frame does the work
-            bool earlier = !a.stream_id && g > 0;
-            for (int b0 = 0; a.stream_id && b0 < g && !earlier; b0 += kTblGroups * kWarp) {
-                bool same = false;
-#pragma unroll
-                for (int u = 0; u < kTblGroups; ++u) {  // unconditional loads (a clamped index), all in flight at once
-                    const int bb = b0 + u * kWarp + (tid & 31);
-                    same |= a.stream_id[min(bb, g)] == s && bb < g;
-                }
-                earlier = __any_sync(kFull, same);
-            }
-            if (earlier) return;
-            tables_by_warp(a, rz, g, s, do_resize,
-                           reinterpret_cast<unsigned char*>(s_dyn) + size_t(tid >> 5) * tables_smem(a.n, rz.k_max),
-                           s_hits[tid >> 5]);
-            return;
-        }
-        // ---- Sec. 6.1 by a whole CTA: the stream's frames, ascending, replayed per class -------
-        const int g = blockIdx.x;
-        const int s = a.stream_id ? a.stream_id[g] : 0;
-        if (s < 0 || s >= a.S) return;  // no such stream (the same for every thread of the CTA)
-        int earlier = (!a.stream_id && g > 0) ? 1 : 0;  // an earlier frame of the same stream: its CTA does the work
-        for (int b = tid; a.stream_id && b < g; b += kUpdThreads) earlier |= a.stream_id[b] == s ? 1 : 0;
-        if (__syncthreads_or(earlier)) return;
-        if (a.forget_W == 0) {
-            // Plain counts: what a frame-by-frame replay leaves behind has a closed form per class.  With
-            // m frames of the stream in the batch, a class that appears q times, last at position p, ends
-            // with FT + q and TS = m - 1 - p; one that does not appear ends with TS + m.  q and p are
-            // gathered by shared-memory atomics on integers (a sum and a maximum: order does not matter).
-            int* s_cnt = reinterpret_cast<int*>(s_dyn);  // [n]; the refresh below reuses the space
-            int* s_last = s_cnt + a.n;                   // [n]
-            for (int c = tid; c < a.n; c += kUpdThreads) {
-                s_cnt[c] = 0;
-                s_last[c] = -1;
-            }
-            __syncthreads();
-            int m = 0;
-            for (int t0 = g - g % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
-                const int b = t0 + tid;
-                const int hit = (b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
-                const int cnt = compact_tile(hit, hit ? final_label_of(a, b) : -1, s_list, s_scan);
-                if (tid < cnt && s_list[tid] >= 0) {
-                    atomicAdd(&s_cnt[s_list[tid]], 1);
-                    atomicMax(&s_last[s_list[tid]], m + tid);
-                }
-                m += cnt;
-            }
-            __syncthreads();
-            for (int c = tid; c < a.n; c += kUpdThreads) {
-                const size_t at = (size_t)s * a.n + c;
-                const int q = s_cnt[c];
-                if (q > 0) {
-                    a.ft[at] = int(min((long long)a.ft[at] + q, (long long)kFtMax));
-                    a.ts[at] = m - 1 - s_last[c];
-                } else {
-                    a.ts[at] = int(min((long long)a.ts[at] + m, (long long)INT32_MAX));
-                }
-            }
+            for (int i = 0; i < PER; ++i)
+                if (c_lo + i < a.n) closed(c_lo + i, f[i], t[i]);
         } else {
-            for (int t0 = g - g % kUpdThreads; t0 < a.B; t0 += kUpdThreads) {
-                const int b = t0 + tid;
-                const int hit = (b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
-                const int cnt = compact_tile(hit, hit ? final_label_of(a, b) : -1, s_list, s_scan);
-                if (cnt == 0) continue;
-                for (int c = tid; c < a.n; c += kUpdThreads) {
-                    int f = a.ft[(size_t)s * a.n + c], t = a.ts[(size_t)s * a.n + c];
-                    for (int i = 0; i < cnt; ++i) table_step(f, t, s_list[i] == c, a.forget_W);
-                    a.ft[(size_t)s * a.n + c] = f;
-                    a.ts[(size_t)s * a.n + c] = t;
+            for (int c = c_lo; c < c_hi; ++c) {
+                int fc = ft[c], tc = ts[c];
+                closed(c, fc, tc);
+                ft[c] = fc;
+                ts[c] = tc;
+            }
+        }
+    } else {
+        // the forgetting table has no closed form: the stream's frames, a tile at a time, replayed per class
+        for (int t0 = g - g % nt; t0 < a.B; t0 += nt) {
+            const int b = t0 + tid;
+            const int hit = (b >= g && b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
+            const int cnt = compact_tile(hit, hit ? final_label_of(a, b) : -1, s_list, s_scan);
+            if (cnt == 0) continue;
+            if (PER) {
+#pragma unroll
+                for (int i = 0; i < PER; ++i)
+                    for (int j = 0; j < cnt; ++j) table_step(f[i], t[i], s_list[j] == c_lo + i, a.forget_W);
+            } else {
+                for (int c = c_lo; c < c_hi; ++c) {
+                    int fc = ft[c], tc = ts[c];
+                    for (int j = 0; j < cnt; ++j) table_step(fc, tc, s_list[j] == c, a.forget_W);
+                    ft[c] = fc;
+                    ts[c] = tc;
                 }
             }
         }
-        if (do_resize) {
-            __syncthreads();  // this CTA's table writes are visible to all of its threads
-            resize_stream(rz, s, reinterpret_cast<unsigned char*>(s_dyn), s_scan, s_part);
+    }
+    unsigned long long sc[PER ? PER : 1];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        if (c_lo + i < a.n) {
+            ft[c_lo + i] = f[i];
+            ts[c_lo + i] = t[i];
         }
+        sc[i] = c_lo + i < a.n ? score_of(f[i], t[i], rz.W, rz.forgetting) : 0ull;
+    }
+    if (do_resize) {
+        __syncthreads();  // every thread is done with the closed form's arrays (and sees its own table entries)
+        if (PER)
+            refresh_from_registers<(PER ? PER : 1)>(rz, s, sc, c_lo, dyn, &s_scan[32], &s_part[31]);
+        else
+            refresh_stream(rz, s, dyn, s_scan, s_part);
     }
 }
 
-// Eq. 7 over the jobs (layer, class) listed by the plan kernel, taken round-robin by CTAs of
-// 1024 threads.  The frames' labels and stop layers are staged in shared memory once; per job the
-// matching frames are listed in ascending index (every thread looks at a run of consecutive
-// frames, one block scan), then thread = (four columns, group): group r folds the listed frames
-// r, r + 4, ... with eight rows in flight, the four groups are added in a fixed order, and the
-// centre, its length and its count are rewritten.  Nothing here waits on another CTA.
-constexpr int kCenThreads = 1024;
-constexpr int kCenCols = kCenThreads;        // columns per sweep: 256 threads x 4 columns, four groups
-constexpr int kCenTile = 2 * kCenThreads;    // frames staged and listed at a time
+// ---- apply: Eq. 7 -----------------------------------------------------------------------------
 
-// Lists, in ascending index, the frames of the staged tile whose label is cls and that stopped at
-// layer l0 + 1 or deeper; returns how many.  s_code[i] = label | stop layer << 16, or -1.
-__device__ __forceinline__ int list_frames(const int* s_code, int tile_frames, int cls, int l0, int* s_list, int* s_scan) {
-    const int per = (tile_frames + kCenThreads - 1) / kCenThreads;  // consecutive frames per thread (1 or 2)
-    const int f0 = threadIdx.x * per;
+constexpr int kCenPer = 4;                         // consecutive frames a thread looks at
+constexpr int kCenTile = kCenPer * kApplyThreads;  // frames listed at a time
+constexpr int kRowGroupsMax = 8;
+
+// Lists, in ascending index, the frames base .. base + kCenTile - 1 whose label is cls and that stopped at
+// layer l0 + 1 or deeper; returns how many (the same in every thread).  Every thread fetches the codes of its
+// run of consecutive frames in one trip to memory; one scan over the threads places them.
+__device__ __forceinline__ int list_pair_frames(const UpdateArgs& a, int base, int cls, int l0, int* s_list, int* s_scan) {
+    const int f0 = base + threadIdx.x * kCenPer;
+    int code[kCenPer];
+#pragma unroll
+    for (int i = 0; i < kCenPer; ++i) code[i] = a.plan.frame_code[min(f0 + i, a.B - 1)];
     int mine = 0;
-    for (int i = 0; i < per; ++i) {
-        const int code = f0 + i < tile_frames ? s_code[f0 + i] : -1;
-        mine += (code >= 0 && (code & 0xffff) == cls && (code >> 16) >= l0 + 1) ? 1 : 0;
+#pragma unroll
+    for (int i = 0; i < kCenPer; ++i) {
+        const bool hit = f0 + i < a.B && code[i] >= 0 && (code[i] & 0xffff) == cls && (code[i] >> 16) >= l0 + 1;
+        code[i] = hit ? 1 : 0;
+        mine += code[i];
     }
     int cnt;
     int pos = block_exclusive_scan(mine, s_scan, &cnt);
-    for (int i = 0; i < per && mine; ++i) {
-        const int code = f0 + i < tile_frames ? s_code[f0 + i] : -1;
-        if (code >= 0 && (code & 0xffff) == cls && (code >> 16) >= l0 + 1) s_list[pos++] = f0 + i;
-    }
+    if (cnt == 0) return 0;
+    __syncthreads();  // the previous tile's readers are done with the list
+#pragma unroll
+    for (int i = 0; i < kCenPer; ++i)
+        if (code[i]) s_list[pos++] = f0 + i;
     __syncthreads();
     return cnt;
 }
 
-__global__ void __launch_bounds__(kCenThreads, 1) k_update_centers(const UpdateArgs a) {
-    __shared__ int s_code[kCenTile];
-    __shared__ int s_list[kCenTile];
-    __shared__ float4 s_acc[3][kCenCols / 4];
-    __shared__ int s_scan[33];
-    __shared__ float s_red[32];
-    const int tid = threadIdx.x;
-    chain_wait();
-    chain_release();
-    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_CENTERS : nullptr);
-    const bool single = a.B <= kCenTile;  // the whole batch fits one tile: staged once, listed once per job
-    const auto stage = [&](int base) {
-        for (int i = tid; i < kCenTile && base + i < a.B; i += kCenThreads) {
-            const int lab = a.plan.final_label[base + i], stop = a.plan.stop_layer[base + i];
-            s_code[i] = lab < 0 ? -1 : (lab | (stop << 16));
-        }
-        __syncthreads();
-    };
-    const int n_jobs = a.plan.job_count[2];
-    int next_code = a.plan.jobs[blockIdx.x];  // (the list has room for every pair) in flight with the count and the labels
-    if (single) stage(0);
-    const int cg = tid & (kCenCols / 4 - 1), grp = tid / (kCenCols / 4);
-    for (int job = blockIdx.x; job < n_jobs; job += gridDim.x) {
-        const int cls = next_code & 0xffff, l0 = next_code >> 16;  // l0 is 0-based; the paper's is l0 + 1
-        if (job + int(gridDim.x) < n_jobs) next_code = a.plan.jobs[job + gridDim.x];
-        const int D = a.dims[l0];
-        const bool vec = (D & 3) == 0;  // rows are 16-byte aligned
-        const float* sv = a.sv[l0];
-        float* cen = a.centers[l0] + (size_t)cls * D;
-        int cnt = single ? list_frames(s_code, a.B, cls, l0, s_list, s_scan) : 0;
-        float nrm = 0.f;
-        int q = 0;
-        for (int d0 = 0; d0 < D; d0 += kCenCols) {  // a sweep of columns, four per thread
-            const int d = d0 + cg * 4;
-            float old[4] = {0.f, 0.f, 0.f, 0.f};  // the centre and its count as they are, fetched along with the rows
-            uint32_t m = 0;
-            if (grp == 0) {
-                m = a.m[l0][cls];
-                for (int j = 0; j < 4; ++j)
-                    if (d + j < D) old[j] = cen[d + j];
-            }
+// Eq. 7 for one item: the columns [block's share] of the centre of (layer l0, class cls).  The frames whose
+// label is cls and that stopped at layer l0 + 1 or deeper are listed in ascending index, a tile of frames at a
+// time (every thread looks at a run of consecutive frames, one scan over the threads).  A thread is (a 16-byte
+// group of columns, a row group): row group r adds the listed rows r, r + R, ... in that order (eight rows in
+// flight), the groups' sums are added in a fixed order, then SC = (SC m + sum SV) / (m + q).  The centre's
+// length and its count are left to k_update_norms (the items of a pair share them); the item of block 0
+// leaves the new count in m_next.
+__device__ void centre_item(const UpdateArgs& a, int item, int* s_list, int* s_scan, float4* s_acc) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int cls = item & 0x1fff, l0 = (item >> 16) & 15, blk = (item >> 20) & 15, nblk = 1 << ((item >> 24) & 7);
+    const int D = a.dims[l0];
+    const float* sv = a.sv[l0];
+    float* cen = a.centers[l0] + (size_t)cls * D;
+    const uint32_t m = a.m[l0][cls];
+    if ((D & 3) == 0) {
+        const int D4 = D >> 2, per_blk = (D4 + nblk - 1) / nblk;
+        const int lo4 = min(D4, blk * per_blk), hi4 = min(D4, lo4 + per_blk);  // this item's 16-byte column groups
+        int R = 1;                                                             // row groups
+        while (R < kRowGroupsMax && 2 * R * (hi4 - lo4) <= nt) R *= 2;
+        const int cpp = nt / R;                                                // column groups per sweep
+        const int rg = tid / cpp, c = tid - rg * cpp;
+        for (int s4 = lo4; s4 < hi4; s4 += cpp) {  // (one sweep unless the item is wider than the CTA)
+            const int c4 = s4 + c;
+            const bool mine_col = c4 < hi4;
+            float4 old = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (mine_col && rg == 0) old = *reinterpret_cast<const float4*>(cen + 4 * c4);  // in flight with the listing
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            q = 0;
+            int q = 0;
             for (int base = 0; base < a.B; base += kCenTile) {
-                if (!single) {
-                    __syncthreads();  // the previous tile's readers are done with the staged codes and the list
-                    stage(base);
-                    cnt = list_frames(s_code, min(kCenTile, a.B - base), cls, l0, s_list, s_scan);
-                }
+                const int cnt = list_pair_frames(a, base, cls, l0, s_list, s_scan);
+                if (cnt == 0) continue;  // (the same for every thread)
                 q += cnt;
-                if (d >= D) continue;
-                if (vec) {
-                    // eight rows in flight per thread; each group adds its rows in ascending frame order
-                    for (int i0 = grp; i0 < cnt; i0 += 32) {
-                        float4 r[8];
+                if (!mine_col) continue;
+                for (int i0 = rg; i0 < cnt; i0 += 8 * R) {
+                    float4 r[8];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u)  // unconditional loads (past the end: the last row again, unused)
-                            r[u] = __ldg(reinterpret_cast<const float4*>(
-                                sv + (size_t)(base + s_list[min(i0 + 4 * u, cnt - 1)]) * D + d));
+                    for (int u = 0; u < 8; ++u)  // unconditional loads (past the end: the last row again, unused)
+                        r[u] = __ldg(reinterpret_cast<const float4*>(sv + (size_t)s_list[min(i0 + u * R, cnt - 1)] * D) + c4);
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            if (i0 + 4 * u < cnt) {
-                                acc[0] += r[u].x; acc[1] += r[u].y; acc[2] += r[u].z; acc[3] += r[u].w;
-                            }
+                    for (int u = 0; u < 8; ++u)
+                        if (i0 + u * R < cnt) {
+                            acc[0] += r[u].x; acc[1] += r[u].y; acc[2] += r[u].z; acc[3] += r[u].w;
                         }
-                    }
-                } else {
-                    for (int i = grp; i < cnt; i += 4)
-                        for (int j = 0; j < 4; ++j)
-                            if (d + j < D) acc[j] += sv[(size_t)(base + s_list[i]) * D + d + j];
                 }
             }
-            if (q == 0) break;  // cannot happen for a listed job; kept so that nothing divides by the old count alone
-            // the groups' sums in a fixed order: ((g0 + g1) + g2) + g3
+            // the row groups' sums in a fixed order: ((g0 + g1) + g2) + ...
             __syncthreads();
-            if (grp > 0) s_acc[grp - 1][cg] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            if (rg > 0 && mine_col) s_acc[(rg - 1) * cpp + c] = make_float4(acc[0], acc[1], acc[2], acc[3]);
             __syncthreads();
-            if (grp == 0 && d < D) {
-#pragma unroll
-                for (int g = 0; g < 3; ++g) {
-                    const float4 o = s_acc[g][cg];
+            if (rg == 0 && mine_col && q > 0) {
+                for (int g2 = 1; g2 < R; ++g2) {
+                    const float4 o = s_acc[(g2 - 1) * cpp + c];
                     acc[0] += o.x; acc[1] += o.y; acc[2] += o.z; acc[3] += o.w;
                 }
-                for (int j = 0; j < 4; ++j)
-                    if (d + j < D) {
-                        // Eq. 7 in double: the count is exact at any size and SC m + sum SV is rounded once
-                        const float v = float((double(old[j]) * double(m) + double(acc[j])) / (double(m) + double(q)));
-                        cen[d + j] = v;
-                        nrm = fmaf(v, v, nrm);
+                // Eq. 7 in double: the count is exact at any size and SC m + sum SV is rounded once
+                const double dm = double(m), inv = 1.0 / (dm + double(q));
+                float4 v;
+                v.x = float((double(old.x) * dm + double(acc[0])) * inv);
+                v.y = float((double(old.y) * dm + double(acc[1])) * inv);
+                v.z = float((double(old.z) * dm + double(acc[2])) * inv);
+                v.w = float((double(old.w) * dm + double(acc[3])) * inv);
+                *reinterpret_cast<float4*>(cen + 4 * c4) = v;
+            }
+            if (tid == 0 && blk == 0 && s4 == lo4) a.m_next[(size_t)l0 * a.n + cls] = m + uint32_t(q);
+        }
+    } else {
+        // a vector that is not a whole number of 16-byte pieces (never cut into blocks): a column per thread
+        int q = 0;
+        for (int d = tid; d < D || d - tid < D; d += nt) {  // every thread makes every trip (the listing is the CTA's)
+            float acc = 0.f;
+            q = 0;
+            for (int base = 0; base < a.B; base += kCenTile) {
+                const int cnt = list_pair_frames(a, base, cls, l0, s_list, s_scan);
+                if (cnt == 0) continue;
+                q += cnt;
+                if (d < D)
+                    for (int i = 0; i < cnt; ++i) acc += sv[(size_t)s_list[i] * D + d];
+            }
+            if (d < D && q > 0) cen[d] = float((double(cen[d]) * double(m) + double(acc)) / (double(m) + double(q)));
+        }
+        if (tid == 0) a.m_next[(size_t)l0 * a.n + cls] = m + uint32_t(q);
+    }
+}
+
+// The apply kernel: CTAs [0, table_ctas) are tables CTAs, one per frame; the others take the listed items.
+__global__ void __launch_bounds__(kApplyThreads, 8) k_update_apply(const UpdateArgs a, const ResizeArgs rz, int do_resize,
+                                                                    int table_ctas) {
+    extern __shared__ unsigned long long s_dyn[];
+    __shared__ int s_list[kCenTile];
+    __shared__ int s_scan[33];
+    __shared__ unsigned long long s_part[32];
+    __shared__ float4 s_acc[kApplyThreads];  // (row groups - 1) x column groups of a sweep
+    chain_wait();
+    chain_release();
+    if (int(blockIdx.x) < table_ctas) {
+        const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_TABLES : nullptr);
+        unsigned char* dyn = reinterpret_cast<unsigned char*>(s_dyn);
+        if (a.n <= 4 * kApplyThreads)
+            tables_of_frame<4>(a, rz, blockIdx.x, do_resize, dyn, s_list, s_scan, s_part);
+        else if (a.n <= 8 * kApplyThreads)
+            tables_of_frame<8>(a, rz, blockIdx.x, do_resize, dyn, s_list, s_scan, s_part);
+        else
+            tables_of_frame<0>(a, rz, blockIdx.x, do_resize, dyn, s_list, s_scan, s_part);
+        return;
+    }
+    const int first = int(blockIdx.x) - table_ctas, stride = int(gridDim.x) - table_ctas;
+    int item = a.plan.items[first];  // (the list has room for every CTA) in flight with the count
+    const int n_items = a.plan.job_count[3];
+    if (first >= n_items) return;
+    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_CENTERS : nullptr);
+    for (int it = first; it < n_items; it += stride) {
+        if (it != first) {
+            __syncthreads();  // the previous item's readers are done with the list
+            item = a.plan.items[it];
+        }
+        centre_item(a, item, s_list, s_scan, s_acc);
+    }
+}
+
+// Length and count of every centre the apply kernel moved: a warp per listed pair.
+__global__ void __launch_bounds__(kUpdThreads) k_update_norms(const UpdateArgs a) {
+    chain_wait();
+    chain_release();
+    const int lane = threadIdx.x & 31;
+    const int first = blockIdx.x * (kUpdThreads / kWarp) + (threadIdx.x >> 5);
+    int code = a.plan.jobs[first];  // (the list has room for every warp) in flight with the count
+    const int n_jobs = a.plan.job_count[2];
+    for (int job = first; job < n_jobs; job += gridDim.x * (kUpdThreads / kWarp)) {
+        if (job != first) code = a.plan.jobs[job];
+        const int cls = code & 0xffff, l0 = code >> 16;
+        const int D = a.dims[l0];
+        const float* cen = a.centers[l0] + (size_t)cls * D;
+        float nrm = 0.f;
+        if ((D & 3) == 0) {
+            const float4* c4 = reinterpret_cast<const float4*>(cen);
+            const int D4 = D >> 2;
+            for (int i0 = 0; i0 < D4; i0 += 8 * kWarp) {  // eight pieces per lane in flight
+                float4 v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = c4[min(i0 + u * kWarp + lane, D4 - 1)];
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (i0 + u * kWarp + lane < D4) {
+                        nrm = fmaf(v[u].x, v[u].x, nrm); nrm = fmaf(v[u].y, v[u].y, nrm);
+                        nrm = fmaf(v[u].z, v[u].z, nrm); nrm = fmaf(v[u].w, v[u].w, nrm);
                     }
             }
+        } else {
+            for (int i = lane; i < D; i += kWarp) nrm = fmaf(cen[i], cen[i], nrm);
         }
-        if (q == 0) continue;
-        nrm = block_sum(nrm, s_red);  // also separates the reads of the count above from its update below
-        if (tid == 0) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) nrm += __shfl_xor_sync(kFull, nrm, o);
+        if (lane == 0) {
             a.cnorm[l0][cls] = __fsqrt_rn(nrm);
-            a.m[l0][cls] += (uint32_t)q;
+            a.m[l0][cls] = a.m_next[(size_t)l0 * a.n + cls];
             if (a.split_current) a.split_current[l0] = 0;  // the tensor-core scorer's copy of this layer's centres is stale
         }
     }
@@ -754,8 +826,9 @@ __global__ void k_center_norms(const float* __restrict__ centers, int n, int D, 
 }  // namespace
 
 cudaError_t memory_setup() {
-    const cudaError_t e = allow_max_dynamic_smem(k_update_tables);
-    return e != cudaSuccess ? e : allow_max_dynamic_smem(k_resize);
+    cudaError_t e = allow_max_dynamic_smem(k_update_apply);
+    if (e == cudaSuccess) e = allow_max_dynamic_smem(k_resize);
+    return e;   // (the single-CTA plan needs at most 32 KB + its statics: below the default limit)
 }
 
 cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm, cudaStream_t st,
@@ -764,55 +837,37 @@ cudaError_t launch_center_norms(const float* centers, int n, int D, float* cnorm
     return launch_chained(k_center_norms, n, 256, 0, st, centers, n, D, cnorm);
 }
 
-cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, cudaStream_t side,
-                          cudaEvent_t fork, cudaEvent_t join, int64_t* launches) {
+cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_count, cudaStream_t st, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
-    // a warp per frame when eight streams' tables and refresh buffers fit a CTA's shared memory
-    const size_t per_warp = tables_smem(a.n, rz ? rz->k_max : 0);
-    const bool warp_tables = per_warp * kUpdWarps <= 100 * 1024;
-    // one CTA per stream: the refresh buffers, and at least the two integer arrays [n] of the closed-form tables
-    // Sixteen warps to a CTA when their buffers fit: the CTAs of k_update_centers fill an SM's registers, so
-    // every SM a tables CTA sits on is one that Eq. 7 cannot use until the tables are done (512 streams: 32
-    // SMs for the tables, 116 for the centres; with eight warps to a CTA it was 64 and 84)
-    const int warps = !warp_tables ? kUpdWarps : (per_warp * kTblWarps <= 180 * 1024 ? kTblWarps : kUpdWarps);
-    const size_t smem = warp_tables ? per_warp * warps
-                                    : std::max<size_t>(rz ? resize_cta_smem(a.n, rz->k_max) : 0, size_t(a.n) * 2 * sizeof(int));
     cudaError_t e = cudaSuccess;
-    const bool tables = a.warm_layer < 0;  // a warm-up batch has no streams
-    const int table_ctas = warp_tables ? (a.B + warps - 1) / warps : a.B;
-    if (tables) {
-        // the tables need nothing of the plan: they run beside plan + centres on the side stream
-        // (inside a stream capture the side stream joins the capture through the events)
-        if ((e = cudaEventRecord(fork, st)) != cudaSuccess) return e;
-        if ((e = cudaStreamWaitEvent(side, fork, 0)) != cudaSuccess) return e;
-        ++*launches;
-        e = launch_chained(k_update_tables, table_ctas, warps * kWarp, smem, side, a,
-                           rz ? *rz : ResizeArgs{}, rz ? 1 : 0, warp_tables ? 1 : 0);
-        if (e != cudaSuccess) return e;
-        if ((e = cudaEventRecord(join, side)) != cudaSuccess) return e;
-    }
     ++*launches;
-    if (a.B <= kPlanOneMaxB && (long long)a.L * a.n <= 32LL * kPlanOneWords)
-        e = launch_chained(k_update_plan_one, 1, kPlanOneThreads, 0, st, a);
-    else
+    const long long pairs = (long long)a.L * a.n;
+    if (a.B <= kPlanOneMaxB && pairs <= 32LL * kPlanOneWords) {
+        const size_t words = pairs <= kPlanCountMax ? size_t(pairs) : size_t((pairs + 31) / 32);
+        e = launch_chained(k_update_plan_one, 1, kPlanOneThreads, words * sizeof(int), st, a);
+    } else {
         e = launch_chained(k_update_plan, (a.B + kUpdThreads - 1) / kUpdThreads, kUpdThreads, 0, st, a);
+    }
     if (e != cudaSuccess) return e;
-    // Eq. 7: at most min(B, n) classes appear per layer; a CTA of 1024 threads per (layer, class) job, one per SM
-    // A centres CTA fills an SM's registers, and plan + centres start before the side stream's tables do:
-    // with a centres CTA on every SM the tables wait until some have left.  Up to a quarter of the SMs are
-    // left to the tables' CTAs.
-    const int table_sms = tables && warp_tables ? std::min(table_ctas, sm_count / 4) : 0;
-    const int centre_ctas = std::min(std::min(a.B, a.n) * (a.warm_layer >= 0 ? 1 : a.L), sm_count - table_sms);
+    const bool tables = a.warm_layer < 0;  // a warm-up batch has no streams
+    const int table_ctas = tables ? a.B : 0;
+    // Eq. 7: at most min(B, n) classes appear per layer; a CTA per item, and a heavy pair is several items (never
+    // more than twice the rows' worth); beyond a few waves of CTAs they stride
+    const int pairs_max = std::min(a.B, a.n) * (a.warm_layer >= 0 ? 1 : a.L);
+    const int centre_ctas = std::min(pairs_max + pairs_max / 2 + kItemBlocksMax, 16 * sm_count);
+    const size_t smem = tables ? tables_smem(a.n, rz ? rz->k_max : 0, rz != nullptr) : 0;
     ++*launches;
-    e = launch_chained(k_update_centers, centre_ctas, kCenThreads, 0, st, a);
+    e = launch_chained(k_update_apply, table_ctas + centre_ctas, kApplyThreads, smem, st, a, rz ? *rz : ResizeArgs{},
+                       rz ? 1 : 0, table_ctas);
     if (e != cudaSuccess) return e;
-    return tables ? cudaStreamWaitEvent(st, join, 0) : cudaSuccess;
+    ++*launches;
+    const int norm_ctas = std::max(1, std::min((pairs_max + kUpdThreads / kWarp - 1) / (kUpdThreads / kWarp), 4 * sm_count));
+    return launch_chained(k_update_norms, norm_ctas, kUpdThreads, 0, st, a);
 }
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
-    const size_t smem = resize_cta_smem(a.n, a.k_max);
     ++*launches;
-    return launch_chained(k_resize, a.S, kUpdThreads, smem, st, a);
+    return launch_chained(k_resize, a.S, kUpdThreads, refresh_smem(a.n, a.k_max), st, a);
 }
 
 }  // namespace smtm
