@@ -320,7 +320,7 @@ def measure(smtm, w, K, W, local_rank, world, verify_steps=0, graph_steps=32):
         import torch.distributed as dist
     res = Resident(smtm, w, W + K)
     R = res.R
-    G = math.gcd(K, graph_steps)   # steps captured into one CUDA graph
+    G = max(d for d in range(1, graph_steps + 1) if K % d == 0)   # steps captured into one CUDA graph
     cents, counts = si.initial_centers(w)
     sid = si.stream_ids(w) if w.S > 1 else None
     # All launches go to one side stream so that every step can be captured into a CUDA graph.
@@ -419,8 +419,10 @@ def measure(smtm, w, K, W, local_rank, world, verify_steps=0, graph_steps=32):
     out["event_us"] = [tot / max(n, 1) * 1e3 for tot, n in ev]
     out["event_n"] = [int(n) for _, n in ev]
     dev_total, dev_cnt = smtm.smtm_cache_get_profile_device(cache)
-    names = ["lookup_layer%d" % l for l in range(w.L)] + ["update_plan", "update_centers", "update_tables", "score_tc"]
-    idx = list(range(w.L)) + [smtm.PROF_PLAN, smtm.PROF_CENTERS, smtm.PROF_TABLES, smtm.PROF_SCORE_TC]
+    names = ["lookup_layer%d" % l for l in range(w.L)] + ["score_layer%d" % l for l in range(w.L)] + \
+        ["update_plan", "update_centers", "update_tables", "update_norms", "score_tc"]
+    idx = list(range(w.L)) + [smtm.PROF_SCORE + l for l in range(w.L)] + \
+        [smtm.PROF_PLAN, smtm.PROF_CENTERS, smtm.PROF_TABLES, smtm.PROF_NORMS, smtm.PROF_SCORE_TC]
     out["device_us"] = {nm: (float(dev_total[i]) / int(dev_cnt[i]) * 1e3 if dev_cnt[i] else None) for nm, i in zip(names, idx)}
     out["device_n"] = int(dev_cnt[0])
     smtm.smtm_cache_destroy(cache)
@@ -504,7 +506,7 @@ def run_ours(args):
             "step_kernels_device_clock_us": m["device_us"],
             "exit_histogram": {"per_layer": m["exits"], "none": K * w.B - sum(m["exits"])},
             "near_threshold_lookups": m["near"],
-            "routes": dict(zip(("fused", "dense", "plain"), m["routes"])),
+            "routes": dict(zip(("fused", "dense", "plain", "pipelined"), m["routes"])),
             "device_status": m["status"],
         }
         # bytes the whole step had to move (maps of the frames still in at each layer + their SV rows) over the step time
@@ -562,7 +564,7 @@ def other_workload(smtm, w, peak, tc_peak, with_oracle):
     out = {"workload": w.name, "steps": K, "warmup": W, "ms_per_step": ms, "frames_per_s": w.B / (ms * 1e-3),
            "dominant_kernel_us": us_dev if us_dev else us_ev, "dominant_kernel_us_cuda_events": us_ev,
            "frac": (ach_dev if ach_dev else ach) / peak if (ach_dev or ach) else None,
-           "bytes_per_launch": nbytes, "routes": dict(zip(("fused", "dense", "plain"), m["routes"])),
+           "bytes_per_launch": nbytes, "routes": dict(zip(("fused", "dense", "plain", "pipelined"), m["routes"])),
            "exit_histogram": {"per_layer": m["exits"], "none": K * w.B - sum(m["exits"])},
            "near_threshold_lookups": m["near"], "step_kernels_device_clock_us": m["device_us"],
            "distinct_steps_resident": m["R"], "device_status": m["status"]}

@@ -73,15 +73,18 @@ enum {
  * appearance adds 1024, each further W consecutive unseen frames multiply it by 0.25 rounding
  * down, and Eq. 5's score is FT itself. */
 enum { SMTM_FLAG_FORGET_FT = 1, SMTM_FLAG_MAPS_READY = 2 };
-/* SMTM_FLAG_MAPS_READY is a promise of the caller that lets smtm_lookup_exit_begin start reading
- * feature maps while the library's previous kernel on the stream (the end of the previous
- * step's update) is still running: (1) the maps given to smtm_lookup_exit_begin are complete in
- * memory when the call is enqueued, i.e. they are not written by earlier work on the same
- * stream; (2) consecutive batches use different smtm_batch_t carries (two that alternate are
- * enough), because the call writes its batch's d_sv[layer] while the previous batch's update
- * may still read its own.  Everything that depends on the memory (members, centres) and every
- * other output still waits for the previous kernel.  Without the flag nothing is touched
- * before the previous kernel is complete. */
+/* SMTM_FLAG_MAPS_READY is a promise of the caller that lets the library pipeline consecutive steps:
+ * (1) the maps given to smtm_lookup_exit_begin are complete in memory when the call is enqueued, i.e.
+ * they are not written by earlier work on the same stream; (2) consecutive batches use different
+ * smtm_batch_t carries (two that alternate are enough).  Pooling (Sec. 4.1) reads only the maps and
+ * does not depend on the memory, so the library then runs the pooling of a step's first layer on a
+ * stream of its own, beside the later layers and the update of the step before (which are bound by
+ * latency, not by bandwidth), and everything that depends on the memory (Eq. 1 onwards) after them on
+ * the caller's stream.  The first lookup writes its batch's d_sv[layer] while the previous batch's
+ * update may still read its own; it is ordered after all work the caller's stream held when the first
+ * lookup before it was enqueued.  To the caller every result is ordered on its stream as usual, and
+ * inside a stream capture the library's stream joins the capture (fork and join become part of the
+ * graph).  Without the flag nothing is touched before the stream's previous work is complete. */
 
 typedef struct {
     int32_t n_classes;      /* n: classes in global memory (Sec. 6), 1..SMTM_MAX_CLASSES */
@@ -284,8 +287,11 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * last CTA ended: h_total_ms[i] and h_count[i], i < SMTM_PROF_KERNELS, are the
  * sum over the profiled steps and their number, for the streaming kernel of
  * layer i (i < SMTM_MAX_LAYERS: the fused lookup kernel, or the pooling kernel
- * of the other routes), for the three update kernels (SMTM_PROF_PLAN, _CENTERS,
- * _TABLES) and for the tensor-core scorer of the dense route
+ * of the other routes), for the scoring kernel of layer i where pooling and
+ * scoring are separate kernels (SMTM_PROF_SCORE + i), for the update (the plan
+ * kernel SMTM_PROF_PLAN; the CTAs of the apply kernel that fold centres,
+ * _CENTERS, and those that keep the tables, _TABLES; the kernel that renews the
+ * centres' lengths, _NORMS) and for the tensor-core scorer of the dense route
  * (SMTM_PROF_SCORE_TC; with several dense layers in a step, from the first
  * one's begin to the last one's end).  This
  * leaves out what the event nodes add around a kernel.  Only the most recent
@@ -296,7 +302,11 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * timer, both 0 for a kernel that did not run in that step, so that the gaps
  * between the kernels of a step can be read off.  All four synchronise the
  * device. */
-enum { SMTM_PROF_PLAN = SMTM_MAX_LAYERS, SMTM_PROF_CENTERS, SMTM_PROF_TABLES, SMTM_PROF_SCORE_TC, SMTM_PROF_KERNELS };
+enum {
+    SMTM_PROF_SCORE = SMTM_MAX_LAYERS,  /* + layer: the scoring kernel of a layer whose pooling is a kernel of its own */
+    SMTM_PROF_PLAN = 2 * SMTM_MAX_LAYERS, SMTM_PROF_CENTERS, SMTM_PROF_TABLES, SMTM_PROF_SCORE_TC, SMTM_PROF_NORMS,
+    SMTM_PROF_KERNELS
+};
 smtm_status_t smtm_cache_profile(smtm_cache_t* cache, int32_t max_lookups, int32_t every);
 smtm_status_t smtm_cache_get_profile(smtm_cache_t* cache, int32_t layer, double* h_total_ms, int64_t* h_count);
 smtm_status_t smtm_cache_get_profile_device(smtm_cache_t* cache, double* h_total_ms /*[SMTM_PROF_KERNELS]*/,
@@ -315,8 +325,12 @@ smtm_status_t smtm_cache_get_launches(smtm_cache_t* cache, int64_t* h_out);
  *                     pixel rows are multiples of 16 bytes);
  *   SMTM_ROUTE_DENSE  fast memories above 64 entries: pooling, then Eq. 1's dot products against
  *                     every class on the tensor cores, then a finishing kernel;
- *   SMTM_ROUTE_PLAIN  everything else: pooling, then a CUDA-core scoring kernel. */
-enum { SMTM_ROUTE_FUSED = 0, SMTM_ROUTE_DENSE = 1, SMTM_ROUTE_PLAIN = 2, SMTM_ROUTE_COUNT = 3 };
+ *   SMTM_ROUTE_PLAIN  everything else: pooling, then a CUDA-core scoring kernel;
+ *   SMTM_ROUTE_PIPELINED  on a cache created with SMTM_FLAG_MAPS_READY (small fast memories, NCHW shapes
+ *                     the streaming kernels serve): the pooling of a step's first layer runs on a stream of
+ *                     the cache's own, under the previous step's later layers and update; scoring follows
+ *                     on the caller's stream; later layers are pooled and scored by small CTAs. */
+enum { SMTM_ROUTE_FUSED = 0, SMTM_ROUTE_DENSE = 1, SMTM_ROUTE_PLAIN = 2, SMTM_ROUTE_PIPELINED = 3, SMTM_ROUTE_COUNT = 4 };
 smtm_status_t smtm_cache_get_routes(smtm_cache_t* cache, int64_t* h_out /*[SMTM_ROUTE_COUNT]*/);
 
 /* Snapshot of the memory of Sec. 6 (the paper keeps it for the life of the application; a host copy

@@ -325,11 +325,11 @@ def smtm_cache_get_launches(cache: Cache) -> int:
     return int(out[0])
 
 
-ROUTE_FUSED, ROUTE_DENSE, ROUTE_PLAIN, ROUTE_COUNT = 0, 1, 2, 3
+ROUTE_FUSED, ROUTE_DENSE, ROUTE_PLAIN, ROUTE_PIPELINED, ROUTE_COUNT = 0, 1, 2, 3, 4
 
 
 def smtm_cache_get_routes(cache: Cache) -> np.ndarray:
-    """Lookups served so far by the fused, the dense (tensor-core) and the plain route."""
+    """Lookups served so far by the fused, the dense (tensor-core), the plain and the pipelined route."""
     out = np.zeros(ROUTE_COUNT, np.int64)
     _check(load_library().smtm_cache_get_routes(cache.handle, out.ctypes.data), "smtm_cache_get_routes")
     return out
@@ -363,8 +363,9 @@ def smtm_cache_get_profile(cache: Cache, layer: int):
     return total.value, count.value
 
 
-PROF_PLAN, PROF_CENTERS, PROF_TABLES, PROF_SCORE_TC, PROF_KERNELS = (MAX_LAYERS, MAX_LAYERS + 1, MAX_LAYERS + 2, MAX_LAYERS + 3,
-                                                                    MAX_LAYERS + 4)
+PROF_SCORE = MAX_LAYERS   # + layer: the scoring kernel of a layer whose pooling is a kernel of its own
+PROF_PLAN, PROF_CENTERS, PROF_TABLES, PROF_SCORE_TC, PROF_NORMS, PROF_KERNELS = (
+    2 * MAX_LAYERS, 2 * MAX_LAYERS + 1, 2 * MAX_LAYERS + 2, 2 * MAX_LAYERS + 3, 2 * MAX_LAYERS + 4, 2 * MAX_LAYERS + 5)
 
 
 def smtm_cache_get_profile_device(cache: Cache):

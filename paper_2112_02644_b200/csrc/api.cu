@@ -31,8 +31,13 @@ struct smtm_cache {
     int d_max;          // largest C_l
     int32_t* d_plan;    // scratch of the update: final label and stop layer of every frame, [max_batch]
     unsigned long long* d_tags;  // scratch of the update: stamps of (layer, class), [L][n]
-    cudaStream_t side_stream;    // the update's tables run here, beside plan + centres on the caller's stream
-    cudaEvent_t ev_fork, ev_join;
+    // pipelined route (SMTM_FLAG_MAPS_READY): the pooling of a step's first layer runs on a stream of the cache's own
+    cudaStream_t pool_stream;
+    cudaEvent_t ev_fork, ev_pool;       // the caller's stream -> pool stream, and back
+    cudaEvent_t ev_mark[2];             // where the caller's stream stood at the last two first lookups (they alternate)
+    unsigned long long mark_capture[2]; // the stream capture each was recorded in (0 = none)
+    bool mark_valid[2];
+    int mark_next;                      // which of the two the next first lookup records
     int32_t* d_jobs;             // scratch of the update: [4] counters, [L][n] (layer, class) pairs to fold, [16][L][n] work items
     uint32_t* d_m_next;          // scratch of the update: [L][n] counts after the update
     unsigned long long* d_epoch; // [2] device: update calls so far, and the plan kernel's ticket
@@ -118,9 +123,11 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_split_current);
     cudaFree(c->d_tags);
     cudaFree(c->d_epoch);
-    if (c->side_stream) cudaStreamDestroy(c->side_stream);
+    if (c->pool_stream) cudaStreamDestroy(c->pool_stream);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
-    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->ev_pool) cudaEventDestroy(c->ev_pool);
+    for (cudaEvent_t e : c->ev_mark)
+        if (e) cudaEventDestroy(e);
     cudaFree(c->d_jobs);
     cudaFree(c->d_m_next);
     cudaFree(c->hb.d_sa);
@@ -166,11 +173,70 @@ EncodeArgs encode_args(const smtm_cache* c, const smtm_fmap_t* f, const uint8_t*
     return e;
 }
 
+// CTA size of the scoring kernel and ring depth of the pooling kernel on the pipelined route: small enough that
+// the CTAs of the latency-bound kernels of a step (scoring, sparse pooling, update) fit on an SM beside a CTA of
+// the next step's pooling kernel.
+constexpr int kPipelinedScoreThreads = 128;
+constexpr int kPipelinedRingStages = 6;
+constexpr int kPipelinedRingConsumers = 3;  // (each looks after two stages)
+// Copies the pooling kernel keeps outstanding per SM on this route.  Every access the latency-bound kernels make
+// to memory queues behind them, so no more than the bandwidth needs (148 x 2 x 25 KB = 7.4 MB in flight).
+constexpr int kPipelinedInFlight = 2;
+
+// The capture the stream is in (0 = none).
+cudaError_t capture_of(cudaStream_t st, unsigned long long* id) {
+    cudaStreamCaptureStatus status = cudaStreamCaptureStatusNone;
+    unsigned long long cid = 0;
+    const cudaError_t e = cudaStreamGetCaptureInfo(st, &status, &cid);
+    *id = (e == cudaSuccess && status == cudaStreamCaptureStatusActive) ? cid : 0ull;
+    return e;
+}
+
+// First lookup of a batch on the pipelined route.  Pooling reads only the maps (complete, by the caller's promise)
+// and writes only this batch's SV stash, so it does not have to wait for the step before: it runs on the cache's
+// pool stream, ordered after the previous pooling (stream order) and after everything the caller's stream held at
+// the first lookup before this one (by then the batch before last, whose stash this batch may share, is done
+// with: batches alternate).  Scoring waits for it and for the caller's stream.  Inside a stream capture the pool
+// stream joins the capture through these events; a mark recorded outside the capture under way is not waited for
+// (the launch of the graph orders the graph after it), and a pool stream that is not part of the capture yet
+// is forked from the caller's stream where it stands.
+smtm_status_t pooled_first_lookup(smtm_cache* c, const EncodeArgs& e, const LookupArgs& a, cudaStream_t st,
+                                  const cudaEvent_t* timing, bool profiled_step) {
+    unsigned long long cap = 0, pool_cap = 0;
+    SMTM_CUDA(capture_of(st, &cap));
+    SMTM_CUDA(capture_of(c->pool_stream, &pool_cap));
+    const int cur = c->mark_next, prev = cur ^ 1;
+    const bool wait_prev = c->mark_valid[prev] && c->mark_capture[prev] == cap;
+    if (wait_prev) SMTM_CUDA(cudaStreamWaitEvent(c->pool_stream, c->ev_mark[prev], 0));
+    if (!wait_prev || (cap != 0 && pool_cap != cap)) {
+        // no usable mark (the first call, a capture that has just begun): the pooling follows all of the caller's stream
+        SMTM_CUDA(cudaEventRecord(c->ev_fork, st));
+        SMTM_CUDA(cudaStreamWaitEvent(c->pool_stream, c->ev_fork, 0));
+    }
+    SMTM_CUDA(cudaEventRecord(c->ev_mark[cur], st));
+    c->mark_capture[cur] = cap;
+    c->mark_valid[cur] = true;
+    c->mark_next = prev;
+    EncodeArgs ep = e;
+    ep.skip = nullptr;  // the batch starts here: every frame is in
+    ep.ring_stages = kPipelinedRingStages;
+    ep.ring_consumers = kPipelinedRingConsumers;
+    ep.ring_in_flight = kPipelinedInFlight;
+    if (profiled_step && a.layer == 0 && ep.clock)  // the caller's stream clears the step's other stamps at a time of its own
+        SMTM_CUDA(cudaMemsetAsync(ep.clock, 0, 2 * sizeof(unsigned long long), c->pool_stream));
+    if (timing) SMTM_CUDA(record_timing(timing[0], c->pool_stream));
+    SMTM_CUDA(launch_encode(ep, c->sm_count, c->pool_stream, &c->launches));
+    if (timing) SMTM_CUDA(record_timing(timing[1], c->pool_stream));
+    SMTM_CUDA(cudaEventRecord(c->ev_pool, c->pool_stream));
+    SMTM_CUDA(cudaStreamWaitEvent(st, c->ev_pool, 0));
+    SMTM_CUDA(launch_score_exit(a, st, &c->launches, kPipelinedScoreThreads));
+    return SMTM_OK;
+}
+
 smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, const smtm_batch_t* b,
                           cudaStream_t st, bool begin, bool allow_early = true) {
     LookupArgs a{};
     a.fresh = begin ? 1 : 0;
-    a.early = (begin && c->maps_ready && allow_early) ? 1 : 0;
     a.layer = layer;
     a.L = c->L;
     a.B = f->B;
@@ -194,14 +260,22 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     a.counters = c->d_counters;
     a.S = c->S;
     a.status = c->d_status;
-    const EncodeArgs e = encode_args(c, f, b->d_done, b->d_sv[layer]);
+    EncodeArgs e = encode_args(c, f, b->d_done, b->d_sv[layer]);
     bool fused = false;
     const cudaEvent_t* timing = nullptr;
+    bool profiled_step_begins = false;
+    // The pipelined route: a cache whose caller keeps the maps resident and alternates its carries
+    // (SMTM_FLAG_MAPS_READY), small fast memories, shapes the streaming kernels serve.
+    const bool pipelined = c->maps_ready && allow_early && c->k_max <= kFusedMaxK && launch_pool_sparse_supported(e);
     if (c->prof_events && c->prof_seq % c->L == 0) {  // a step begins: does it get a slot for the device-clock stamps?
         c->prof_step = nullptr;
         if ((c->prof_seq / c->L) % c->prof_every == 0 && c->prof_steps_used < c->prof_steps_cap) {
             c->prof_step = c->d_prof_clock + c->prof_steps_used++ * size_t(2 * SMTM_PROF_KERNELS);
-            SMTM_CUDA(cudaMemsetAsync(c->prof_step, 0, 2 * SMTM_PROF_KERNELS * sizeof(unsigned long long), st));
+            // (the first two words are the stamps of the first layer's streaming kernel: on the pipelined route that
+            // kernel runs on the pool stream, which clears them itself)
+            const size_t skip = (pipelined && begin && layer == 0) ? 2 : 0;
+            SMTM_CUDA(cudaMemsetAsync(c->prof_step + skip, 0, (2 * SMTM_PROF_KERNELS - skip) * sizeof(unsigned long long), st));
+            profiled_step_begins = true;
         }
     }
     a.clock = c->prof_events ? c->prof_step : nullptr;
@@ -210,6 +284,17 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
         timing = c->prof_events->data() + 2 * c->prof_used;
         (*c->prof_layer)[c->prof_used++] = layer;
     }
+    if (pipelined) {
+        ++c->routes[SMTM_ROUTE_PIPELINED];
+        e.clock = a.clock ? a.clock + 2 * layer : nullptr;  // the pooling kernel is this layer's streaming kernel
+        if (begin) return pooled_first_lookup(c, e, a, st, timing, profiled_step_begins);
+        // a later layer: the frames still in are few; small CTAs pool them, small CTAs score them
+        if (timing) SMTM_CUDA(record_timing(timing[0], st));
+        SMTM_CUDA(launch_pool_sparse(e, c->sm_count, st, &c->launches));
+        if (timing) SMTM_CUDA(record_timing(timing[1], st));
+        SMTM_CUDA(launch_score_exit(a, st, &c->launches, kPipelinedScoreThreads));
+        return SMTM_OK;
+    }
     SMTM_CUDA(launch_lookup_fused(e, a, c->sm_count, &c->fused_caps, st, &c->launches, &fused, timing));
     if (fused) {
         ++c->routes[SMTM_ROUTE_FUSED];
@@ -217,10 +302,6 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     }
     const bool dense = c->d_dense && dense_scoring_supported(a.D, a.n);  // large fast memory: tensor cores
     ++c->routes[dense ? SMTM_ROUTE_DENSE : SMTM_ROUTE_PLAIN];
-    if (begin && !dense) {  // the plain route reads the carry: put it into its reset state with a kernel of its own
-        SMTM_CUDA(launch_batch_reset(b->d_sa, b->d_done, b->d_exit_layer, b->d_pred, b->B, c->k_max, st, &c->launches));
-        a.fresh = 0;
-    }
     EncodeArgs e2 = e;
     e2.clock = a.clock ? a.clock + 2 * layer : nullptr;  // the pooling kernel is this layer's streaming kernel
     if (a.fresh) e2.skip = nullptr;  // a batch that starts here: every frame is in, whatever the flags hold
@@ -411,9 +492,10 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     ok = ok && dev_alloc(&c->d_jobs, 4 + 17 * size_t(c->L) * n) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_m_next, size_t(c->L) * n) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_epoch, 2) == cudaSuccess;
-    ok = ok && cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->pool_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
-    ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_pool, cudaEventDisableTiming) == cudaSuccess;
+    for (cudaEvent_t& e : c->ev_mark) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();
         free_all(c);

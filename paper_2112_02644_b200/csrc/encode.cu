@@ -51,7 +51,9 @@ struct NchwParams {
     float inv_hw;
     int team;                // team-per-channel: lanes per channel (power of two)
     int vec_per_channel;     // team-per-channel: 16-byte vectors per channel
-    int max_in_flight;       // copies the producer keeps outstanding (<= kStages)
+    int max_in_flight;       // copies the producer keeps outstanding (<= stages)
+    int stages;              // k_encode_nchw: ring depth, 2 .. kStages (the fused kernel always uses kStages)
+    int consumers;           // k_encode_nchw: consumer warps, 1 .. kConsumers; the CTA has one more warp, the producer's
     unsigned long long* clock;  // nullptr, or two words for the device-clock stamps of the pooling kernel
 };
 
@@ -198,12 +200,13 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     uint8_t* stages = base;
-    uint64_t* full = reinterpret_cast<uint64_t*>(base + size_t(kStages) * kStageCap);
-    uint64_t* empty = full + kStages;
+    const int n_stages = p.stages;
+    uint64_t* full = reinterpret_cast<uint64_t*>(base + size_t(n_stages) * kStageCap);
+    uint64_t* empty = full + n_stages;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
@@ -214,7 +217,9 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
     chain_release();
     const ClockScope stamps(p.clock);
 
-    const bool producer = warp == kConsumers;  // last warp; lane 0 issues the copies
+    const int n_consumers = p.consumers;
+    const bool producer = warp == n_consumers;  // last warp; lane 0 issues the copies
+    const uint64_t stream_once = l2_evict_first_policy();
     int it = 0;                                // chunks of this CTA that are not skipped, so far
     bool failed = false;
     if (!producer || lane == 0) {
@@ -222,8 +227,8 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
             const int b = int(g / p.chunks_per_frame);
             if (p.skip && p.skip[b]) continue;
             const int ci = int(g - (long long)b * p.chunks_per_frame);
-            const int stage = it % kStages;
-            const uint32_t use = uint32_t(it / kStages);
+            const int stage = it % n_stages;
+            const uint32_t use = uint32_t(it / n_stages);
             const int c0 = ci * p.chunk_channels;
             const int nch = min(p.chunk_channels, p.C - c0);
             if (producer) {
@@ -233,16 +238,16 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
                 }
                 if (it >= p.max_in_flight) {  // bound the bytes in flight: wait for an older copy to land
                     const int old = it - p.max_in_flight;
-                    if (!mbar_wait_bounded(&full[old % kStages], (old / kStages) & 1, p.status)) {
+                    if (!mbar_wait_bounded(&full[old % n_stages], (old / n_stages) & 1, p.status)) {
                         failed = true;
                         break;
                     }
                 }
                 const uint32_t bytes = uint32_t(nch) * uint32_t(p.ch_bytes);
                 mbar_expect_tx(&full[stage], bytes);
-                bulk_load(stages + size_t(stage) * kStageCap,
-                          p.x + (long long)b * p.frame_bytes + (long long)c0 * p.ch_bytes, bytes, &full[stage]);
-            } else if (stage % kConsumers == warp) {
+                bulk_load_hint(stages + size_t(stage) * kStageCap,
+                               p.x + (long long)b * p.frame_bytes + (long long)c0 * p.ch_bytes, bytes, &full[stage], stream_once);
+            } else if (stage % n_consumers == warp) {
                 if (!mbar_wait_bounded(&full[stage], use & 1, p.status)) {
                     failed = true;
                     break;
@@ -258,8 +263,8 @@ __global__ void __launch_bounds__(kThreadsTma, 1) k_encode_nchw(const NchwParams
     // stay allocated until the copy engine is done with it.
     const int any_failed = __syncthreads_or(failed ? 1 : 0);
     if (any_failed && producer && lane == 0) {
-        for (int s = 0; s < kStages && s < it; ++s) {
-            const uint32_t last_use = uint32_t((it - 1 - s) / kStages);
+        for (int s = 0; s < n_stages && s < it; ++s) {
+            const uint32_t last_use = uint32_t((it - 1 - s) / n_stages);
             mbar_wait_bounded(&full[s], last_use & 1, p.status);
         }
     }
@@ -408,15 +413,9 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         const long long u = (long long)cluster + (long long)idx * n_clusters;
         if (u < a.B) my_units[idx] = int(u);
     }
-    // Everything above touched shared memory only and overlaps the previous kernel's tail.  With
-    // a.early the producer and the reducers go on without waiting (they read the caller's maps and
-    // write this batch's SV stash, which the previous kernel does not touch); the dot warps and
-    // the finisher, which read the memory and write the carry, wait on their own.
-    const bool early = a.fresh && a.early;
-    if (!early) {
-        chain_wait();
-        chain_release();
-    }
+    // Everything above touched shared memory only and overlaps the previous kernel's tail.
+    chain_wait();
+    chain_release();
     const ClockScope stamps(a.clock ? a.clock + 2 * a.layer : nullptr);  // profiling
     for (int t0 = 0; !a.fresh && t0 < a.B; t0 += kThreadsFused) {
         const int b = t0 + threadIdx.x;
@@ -466,6 +465,7 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
     } else if (warp == kReducersF) {
         // ---- producer -------------------------------------------------------------------------
         if (lane == 0) {
+            const uint64_t stream_once = l2_evict_first_policy();
             for (int it = 0; it < n_chunks; ++it) {
                 const int i = it / cpu, c = it - i * cpu;
                 const int b = my_units[i];
@@ -480,18 +480,14 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
                 }
                 const uint32_t bytes = uint32_t(nch) * uint32_t(p.ch_bytes);
                 mbar_expect_tx(&full[stage], bytes);
-                bulk_load(stages + size_t(stage) * kStageCap,
-                          p.x + (long long)b * p.frame_bytes + (long long)c0 * p.ch_bytes, bytes, &full[stage]);
+                bulk_load_hint(stages + size_t(stage) * kStageCap,
+                               p.x + (long long)b * p.frame_bytes + (long long)c0 * p.ch_bytes, bytes, &full[stage], stream_once);
                 issued = it + 1;
             }
         }
     } else if (warp <= kReducersF + kDotWarps) {
         // ---- dot warps: all of them work on frame u together, slot j on warp j % kDotWarps -------
         const int dw = warp - kReducersF - 1;
-        if (early) {
-            chain_wait();
-            if (dw == 0 && lane == 0) chain_release();
-        }
         const int sb = rank * f.slice_cap;          // first channel of this CTA's slice
         const int Dp = max(0, min(f.slice_cap, p.C - sb));  // channels in it (a multiple of 4)
         const int n4 = Dp >> 2;
@@ -595,7 +591,6 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
         }
     } else {
         // ---- finisher warp: every P-th frame of the cluster; lane l looks after slots l and l + 32 ----
-        if (early) chain_wait();
         const float weight = float(1u << a.layer);  // 2^(l-1) with l = layer + 1
         const int reuse = max(P, kRx);              // frames between two uses of a receive buffer in this CTA
         for (int u = rank; u < nu; u += P) {
@@ -663,6 +658,90 @@ __global__ void __launch_bounds__(kThreadsFused, 1) k_lookup_nchw(const FusedPar
     if (P > 1) cluster_sync_all();
 }
 
+// ---- pooling of the few frames still in at a later layer, by small CTAs ------------------------
+//
+// When most frames have left at an earlier layer, the streaming kernel above is the wrong tool: it
+// wants a whole SM per CTA, and on a device whose SMs are held by another streaming kernel (the
+// pooling of the next step's first layer, see the pipelined route in api.cu) it would wait for one.
+// This kernel pools the active frames with CTAs of 128 threads and a single 12.5 KB stage, so that
+// several fit beside such a kernel.  The grid is cpf x G CTAs: CTA c looks after chunk c % cpf of the
+// active frames number c / cpf, c / cpf + G, ... (every CTA compacts the list of active frames for
+// itself, as the fused kernel does).  A chunk is fetched with plain coalesced 16-byte loads, all in
+// flight at once, and reduced by the reducers of the streaming kernel, the warps sharing its
+// channels: every channel is summed in the same order as there, so both kernels give the same bits.
+constexpr int kLightThreads = 128;
+constexpr int kLightStageCap = 12800;   // bytes of a chunk here (half a stage of the streaming kernel)
+constexpr int kLightFrames = 256;       // frames a CTA can be given
+
+struct LightParams {
+    NchwParams e;   // chunking as for the streaming kernel, with chunks of at most kLightStageCap bytes
+    int groups;     // G
+    int gran;       // channels that must stay in one warp's share (the reducer's unit)
+};
+
+template <class R>
+__global__ void __launch_bounds__(kLightThreads) k_pool_sparse(const LightParams f) {
+    __shared__ __align__(16) uint8_t stage[kLightStageCap];
+    __shared__ int my_frames[kLightFrames];
+    __shared__ int s_scan[33];
+    const NchwParams& p = f.e;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int B = int(p.total_chunks / p.chunks_per_frame);
+    const int ci = int(blockIdx.x) % p.chunks_per_frame, group = int(blockIdx.x) / p.chunks_per_frame;
+    chain_wait();  // the exit flags are the previous kernel's
+    chain_release();
+    const ClockScope stamps(p.clock);
+    uint8_t flags[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int n_active = 0;
+    for (int t0 = 0; t0 < B; t0 += kLightThreads) {
+        const int b = t0 + tid;
+        int act = b < B ? 1 : 0;
+        if (p.skip) {  // the flags of eight tiles in one trip to memory
+            if ((t0 / kLightThreads) % 8 == 0) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) flags[u] = p.skip[min(b + u * kLightThreads, B - 1)];
+            }
+            uint8_t mine = 0;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) mine = ((t0 / kLightThreads) % 8 == u) ? flags[u] : mine;
+            act = (b < B && !mine) ? 1 : 0;
+        }
+        int cnt;
+        const int pos = block_exclusive_scan(act, s_scan, &cnt);
+        if (act) {
+            const int u = n_active + pos;
+            if (u % f.groups == group && u / f.groups < kLightFrames) my_frames[u / f.groups] = b;
+        }
+        n_active += cnt;
+    }
+    const int nu = n_active > group ? min((n_active - group + f.groups - 1) / f.groups, kLightFrames) : 0;
+    __syncthreads();
+    const int c0 = ci * p.chunk_channels;
+    const int nch = min(p.chunk_channels, p.C - c0);
+    const int vectors = nch * p.ch_bytes / 16;
+    // this warp's share of the chunk's channels (whole reducer units)
+    const int units = (nch + f.gran - 1) / f.gran;
+    const int u_lo = min(units, warp * ((units + 3) / 4)), u_hi = min(units, u_lo + (units + 3) / 4);
+    const int w_c0 = u_lo * f.gran, w_nch = min(nch, u_hi * f.gran) - w_c0;
+    for (int k = 0; k < nu; ++k) {
+        const int b = my_frames[k];
+        const uint4* src = reinterpret_cast<const uint4*>(p.x + (long long)b * p.frame_bytes + (long long)c0 * p.ch_bytes);
+        uint4* dst = reinterpret_cast<uint4*>(stage);
+        for (int v0 = 0; v0 < vectors; v0 += 8 * kLightThreads) {  // eight loads per thread in flight
+            uint4 r[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) r[u] = __ldg(src + min(v0 + u * kLightThreads + tid, vectors - 1));
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (v0 + u * kLightThreads + tid < vectors) dst[v0 + u * kLightThreads + tid] = r[u];
+        }
+        __syncthreads();
+        if (w_nch > 0)
+            R::run(stage + size_t(w_c0) * p.ch_bytes, w_nch, lane, p.sv + (long long)b * p.C + c0 + w_c0, nullptr, p.inv_hw, p);
+        __syncthreads();  // the stage is free for the next frame
+    }
+}
+
 // ---- NHWC: direct coalesced loads ----------------------------------------------------------
 
 constexpr int kThreadsNhwc = 256;
@@ -725,6 +804,72 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_encode_nhwc(const uint8_t* __r
     }
 }
 
+// ---- NHWC, small fast memory: pooling, scoring and the decision by one CTA per frame ---------------
+//
+// A frame of an NHWC map is H*W rows of C channels: pooling is a column sum, and one CTA holds all of a
+// frame's column sums at the end, so the same CTA goes on to Eq. 1, Eq. 3, Eq. 4 and the exit rule (one
+// launch per layer).  Thread = (16-byte column group, pixel phase); every thread keeps eight loads in
+// flight (a frame is a few dozen KB: the CTA's time is the number of trips to memory it makes); the
+// phases are added in ascending order through shared memory.  Frames that have exited cost a CTA that
+// leaves at once.
+template <class E>
+__global__ void __launch_bounds__(kThreadsNhwc) k_lookup_nhwc(const uint8_t* __restrict__ x, int C, int HW, float inv_hw,
+                                                              float* __restrict__ sv_out, const LookupArgs a) {
+    extern __shared__ float nhwc_smem[];  // sv [C] | s_cur [k_max] | s_acc [k_max] | part [phases][cgs * V]
+    __shared__ float scratch[32];
+    float* sv_s = nhwc_smem;
+    float* s_cur = sv_s + C;
+    float* s_acc = s_cur + a.k_max;
+    float* part = s_acc + a.k_max;
+    chain_wait();
+    chain_release();
+    const ClockScope stamps(a.clock ? a.clock + 2 * a.layer : nullptr);
+    const int b = blockIdx.x;
+    const int sid_raw = a.stream_id ? a.stream_id[b] : 0;  // in flight with the exit flag
+    if (!a.fresh && a.done[b]) return;
+    constexpr int V = E::kPerVec;
+    const int CG = C / V;  // 16-byte vectors per pixel
+    const uint4* f = reinterpret_cast<const uint4*>(x + (long long)b * HW * C * E::kSize);
+    float nrm = 0.f;
+    for (int cg0 = 0; cg0 < CG; cg0 += kThreadsNhwc) {
+        const int cgs = min(CG - cg0, kThreadsNhwc);  // column groups handled in this sweep
+        const int phases = kThreadsNhwc / cgs;
+        const int ph = threadIdx.x / cgs, cg = threadIdx.x - ph * cgs;
+        float acc[V];
+#pragma unroll
+        for (int j = 0; j < V; ++j) acc[j] = 0.f;
+        if (ph < phases) {
+            const uint4* col = f + cg0 + cg;
+            for (int px = ph; px < HW; px += 8 * phases) {
+                uint4 v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = __ldg(col + (long long)min(px + u * phases, HW - 1) * CG);
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (px + u * phases < HW) {
+#pragma unroll
+                        for (int j = 0; j < V; ++j) acc[j] += E::at(v[u], j);
+                    }
+            }
+            float* dst = part + (size_t(ph) * cgs + cg) * V;
+#pragma unroll
+            for (int j = 0; j < V; ++j) dst[j] = acc[j];
+        }
+        __syncthreads();
+        for (int c = threadIdx.x; c < cgs * V; c += kThreadsNhwc) {
+            float s = 0.f;
+            for (int q = 0; q < phases; ++q) s += part[size_t(q) * cgs * V + c];
+            s *= inv_hw;
+            sv_s[cg0 * V + c] = s;
+            sv_out[(long long)b * C + cg0 * V + c] = s;
+            nrm = fmaf(s, s, nrm);
+        }
+        __syncthreads();
+    }
+    nrm = block_sum(nrm, scratch);  // also orders the shared writes above
+    score_frame(a, b, sid_raw, sv_s, nrm, s_cur, s_acc);
+}
+
 // ---- any shape: one thread per (frame, channel) ---------------------------------------------
 
 template <class E>
@@ -765,9 +910,11 @@ __global__ void k_row_norm2(const float* __restrict__ sv, const uint8_t* __restr
     if (threadIdx.x == 0) out[b] = s;
 }
 
+constexpr size_t nchw_smem(int stages) { return size_t(stages) * kStageCap + 2 * size_t(stages) * sizeof(uint64_t) + 128; }
+
 template <class R>
 cudaError_t launch_nchw(const NchwParams& p, int grid, cudaStream_t st) {
-    return launch_chained(k_encode_nchw<R>, grid, kThreadsTma, kSmemTma, st, p);
+    return launch_chained(k_encode_nchw<R>, grid, (p.consumers + 1) * kWarp, nchw_smem(p.stages), st, p);
 }
 
 template <class R>
@@ -823,7 +970,10 @@ Reducer plan_nchw(const EncodeArgs& a, NchwParams* p) {
     p->ch_bytes = HW * es;
     p->frame_bytes = (long long)a.C * p->ch_bytes;
     p->inv_hw = 1.0f / float(HW);
-    p->max_in_flight = kMaxInFlight;
+    p->max_in_flight = a.ring_in_flight > 0 ? std::min(a.ring_in_flight, kMaxInFlight) : kMaxInFlight;
+    p->stages = (a.ring_stages >= 2 && a.ring_stages <= kStages) ? a.ring_stages : kStages;
+    if (p->max_in_flight > p->stages - 1) p->max_in_flight = p->stages - 1;
+    p->consumers = (a.ring_consumers >= 1 && a.ring_consumers <= kConsumers) ? a.ring_consumers : kConsumers;
     // unit-per-lane shapes (compile-time H*W)
     int G = 0;
     if ((HW == 49 || HW == 196) && es == 2) G = HW == 49 ? 8 : 2;
@@ -888,10 +1038,19 @@ cudaError_t max_clusters(int parts, size_t smem, int* out) {
 
 }  // namespace
 
+template <class R>
+cudaError_t carveout_pipelined() {
+    cudaError_t e = prefer_max_smem_carveout(k_encode_nchw<R>);
+    return e != cudaSuccess ? e : prefer_max_smem_carveout(k_pool_sparse<R>);
+}
+
 cudaError_t encode_setup() {
-    cudaError_t e = cudaSuccess;
+    cudaError_t e = allow_max_dynamic_smem(k_lookup_nhwc<F32>);
+    if (e == cudaSuccess) e = allow_max_dynamic_smem(k_lookup_nhwc<F16>);
+    if (e == cudaSuccess) e = allow_max_dynamic_smem(k_lookup_nhwc<BF16>);
 #define SMTM_OPT_IN(...)                                        \
     if (e == cudaSuccess) e = opt_in<__VA_ARGS__>();            \
+    if (e == cudaSuccess) e = carveout_pipelined<__VA_ARGS__>();  \
     if (e == cudaSuccess) e = opt_in_fused<__VA_ARGS__>();
     for (int r = kUnitBf16x49; r <= kTeamBf16; ++r) SMTM_FOR_REDUCER(r, SMTM_OPT_IN)
 #undef SMTM_OPT_IN
@@ -926,10 +1085,63 @@ cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, in
     return launch_generic<BF16>(a, st);
 }
 
+bool launch_pool_sparse_supported(const EncodeArgs& a) {
+    if (a.layout != SMTM_NCHW || a.B <= 0) return false;
+    NchwParams p;
+    const Reducer r = plan_nchw(a, &p);
+    return r != kNone && p.ch_bytes <= kLightStageCap;
+}
+
+cudaError_t launch_pool_sparse(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches) {
+    LightParams f{};
+    const Reducer r = plan_nchw(a, &f.e);
+    if (r == kNone || f.e.ch_bytes > kLightStageCap) return cudaErrorInvalidValue;
+    // chunks of at most kLightStageCap bytes: half the units of a unit-per-lane chunk, or as many whole channels as fit
+    const bool unit = r <= kUnitF32x49;
+    f.gran = unit ? f.e.chunk_channels / 32 : std::max(1, 32 / std::max(1, f.e.team));
+    if (unit) {
+        f.e.chunk_channels /= 2;
+    } else {
+        int cc = kLightStageCap / f.e.ch_bytes;
+        if (cc > f.gran) cc -= cc % f.gran;
+        f.e.chunk_channels = std::min(cc, a.C);
+    }
+    f.e.chunks_per_frame = (a.C + f.e.chunk_channels - 1) / f.e.chunk_channels;
+    f.e.total_chunks = (long long)a.B * f.e.chunks_per_frame;
+    // about four CTAs to an SM; enough groups that no CTA is given more frames than it can list
+    const int cpf = f.e.chunks_per_frame;
+    int groups = std::max(1, std::min(a.B, 8 * sm_count / cpf));
+    groups = std::max(groups, (a.B + kLightFrames - 1) / kLightFrames);
+    f.groups = groups;
+    cudaError_t e = cudaSuccess;
+    ++*launches;
+#define SMTM_LAUNCH(...) e = launch_chained(k_pool_sparse<__VA_ARGS__>, cpf * groups, kLightThreads, 0, st, f)
+    SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
+#undef SMTM_LAUNCH
+    return e;
+}
+
 cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm_count, FusedCaps* caps, cudaStream_t st,
                                 int64_t* launches, bool* handled, const cudaEvent_t* timing) {
     *handled = false;
-    if (e.B <= 0 || e.layout != SMTM_NCHW || a.k_max > kFusedMaxK) return cudaSuccess;
+    if (e.B <= 0 || a.k_max > kFusedMaxK) return cudaSuccess;
+    if (e.layout == SMTM_NHWC) {
+        const int V = e.dtype == SMTM_F32 ? 4 : 8;
+        if (e.C % V || e.C > 8192) return cudaSuccess;
+        const int cgs = std::min(e.C / V, kThreadsNhwc);
+        const size_t smem = (size_t(e.C) + 2 * size_t(a.k_max) + size_t(kThreadsNhwc / cgs) * cgs * V) * sizeof(float);
+        const float inv_hw = 1.0f / float(e.H * e.W);
+        const uint8_t* x = static_cast<const uint8_t*>(e.x);
+        cudaError_t err = cudaSuccess;
+        if (timing) record_timing(timing[0], st);
+        if (e.dtype == SMTM_F32) err = launch_chained(k_lookup_nhwc<F32>, e.B, kThreadsNhwc, smem, st, x, e.C, e.H * e.W, inv_hw, e.sv, a);
+        else if (e.dtype == SMTM_F16) err = launch_chained(k_lookup_nhwc<F16>, e.B, kThreadsNhwc, smem, st, x, e.C, e.H * e.W, inv_hw, e.sv, a);
+        else err = launch_chained(k_lookup_nhwc<BF16>, e.B, kThreadsNhwc, smem, st, x, e.C, e.H * e.W, inv_hw, e.sv, a);
+        if (timing) record_timing(timing[1], st);
+        ++*launches;
+        *handled = true;
+        return err;
+    }
     FusedParams f{};
     const Reducer r = plan_nchw(e, &f.e);
     if (r == kNone) return cudaSuccess;

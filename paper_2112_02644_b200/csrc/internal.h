@@ -80,14 +80,30 @@ struct EncodeArgs {
     void* sv_lo;
     int* status;          // device sticky status word
     unsigned long long* clock;  // nullptr, or two words for the kernel's device-clock stamps (see ClockScope)
+    int ring_stages;      // 0 = the default depth of the streaming kernel's ring; fewer stages leave shared memory to
+                          // the kernels that run beside it
+    int ring_consumers;   // 0 = the default number of reducer warps; fewer leave registers to those kernels
+    int ring_in_flight;   // 0 = the default number of copies kept outstanding per CTA
 };
 // Enqueues the pooling of every non-skipped frame.  *launches is incremented per kernel launched.
 // *wrote_split (may be null) tells whether sv_hi / sv_lo were filled by the kernel that ran.
 cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches,
                           bool* wrote_split = nullptr);
+// Asks that SMs running `kernel` be configured with as much shared memory as they can have.  Kernels that
+// are meant to share an SM with a streaming kernel (whose CTAs need most of it) must not leave the SM in a
+// configuration with less: a CTA of the streaming kernel would wait until the SM has drained.
+template <class K>
+cudaError_t prefer_max_smem_carveout(K kernel) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, int(cudaSharedmemCarveoutMaxShared));
+}
+
 // Opt-in to large dynamic shared memory for the kernels that need it, on the current device (every
 // cache does this for its own device at creation).
 cudaError_t encode_setup();
+// Pooling of the frames that are still in (skip[b] == 0) by small CTAs that fit beside a streaming kernel; NCHW
+// shapes the streaming pipeline serves whose channels are at most 12.5 KB.  Same bits as launch_encode.
+bool launch_pool_sparse_supported(const EncodeArgs& a);
+cudaError_t launch_pool_sparse(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches);
 cudaError_t lookup_setup();
 cudaError_t memory_setup();
 cudaError_t dense_setup();
@@ -99,7 +115,6 @@ struct LookupArgs {
     int layer, L, B, D, n, k_max;
     int S;                    // streams of the cache: a frame whose stream id lies outside [0, S) is not looked up
     int* status;              // device sticky status word
-    int early;                // (fused route, with fresh) the maps may be read and the SV stash written before the previous kernel is complete
     int fresh;                // the batch starts here: the carry is taken as SA = 0, nobody done, and is overwritten
     float tau;
     const float* sv;          // [B][D]
@@ -118,7 +133,8 @@ struct LookupArgs {
     unsigned long long* counters;
     unsigned long long* clock;  // nullptr, or the profiled step's stamps [SMTM_PROF_KERNELS][2] (see ClockScope)
 };
-cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches);
+// threads: CTA size (a multiple of 32, at most 256; 0 = 256).  Smaller CTAs fit beside a streaming kernel.
+cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches, int threads = 0);
 // Encode + score + exit in one kernel (NCHW shapes the streaming pipeline serves, fast
 // memories of at most 64 entries).  *handled is false when the shape is not served, in which
 // case nothing was launched.

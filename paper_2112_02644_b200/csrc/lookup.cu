@@ -18,6 +18,7 @@ namespace {
 
 constexpr int kThreads = 256;
 
+// Any whole number of warps up to kThreads per CTA.
 __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
     extern __shared__ float smem[];
     float* sv = smem;                 // [D]
@@ -27,51 +28,20 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
 
     chain_wait();
     chain_release();
+    const ClockScope stamps(a.clock ? a.clock + 2 * (SMTM_PROF_SCORE + a.layer) : nullptr);
     const int b = blockIdx.x;
-    if (a.done[b]) return;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int sid = stream_of(a, b);
-    const int k = sid < 0 ? 0 : a.k[sid];  // a stream id outside the cache: nothing to score against
-    const int32_t* mem = a.members + (size_t)max(sid, 0) * a.k_max;
+    const int sid_raw = a.stream_id ? a.stream_id[b] : 0;  // in flight with the exit flag
+    if (!a.fresh && a.done[b]) return;  // (a batch that starts here: every frame is in, whatever the flags hold)
+    const int tid = threadIdx.x, nthreads = blockDim.x;
     const float* row = a.sv + (size_t)b * a.D;
-
     float nrm = 0.f;
-    for (int d = tid; d < a.D; d += kThreads) {
+    for (int d = tid; d < a.D; d += nthreads) {
         const float v = row[d];
         sv[d] = v;
         nrm = fmaf(v, v, nrm);
     }
     nrm = block_sum(nrm, scratch);  // also orders the shared writes above
-
-    const float weight = float(1u << a.layer);  // 2^(l-1) with l = layer + 1
-    const int D4 = (a.D & 3) ? 0 : a.D >> 2;  // 128-bit loads need rows that are multiples of 16 bytes
-    for (int j = warp; j < k; j += kThreads / kWarp) {
-        const int cls = mem[j];
-        const float4* c4 = reinterpret_cast<const float4*>(a.centers + (size_t)cls * a.D);
-        const float4* v4 = reinterpret_cast<const float4*>(sv);
-        float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
-        for (int i = lane; i < D4; i += kWarp) {
-            const float4 c = __ldg(c4 + i);
-            const float4 v = v4[i];
-            d0 = fmaf(c.x, v.x, d0); d1 = fmaf(c.y, v.y, d1); d2 = fmaf(c.z, v.z, d2); d3 = fmaf(c.w, v.w, d3);
-        }
-        for (int i = (D4 << 2) + lane; i < a.D; i += kWarp) d0 = fmaf(a.centers[(size_t)cls * a.D + i], sv[i], d0);
-        float dot = (d0 + d1) + (d2 + d3);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(kFull, dot, o);
-        if (lane == 0) {
-            const float cl = a.cnorm[cls];
-            const float s = cosine_from(dot, nrm, cl);                                                 // Eq. 1
-            const float acc = __fmaf_rn(s, weight, a.sa[(size_t)b * a.k_max + j]);                     // Eq. 3
-            a.sa[(size_t)b * a.k_max + j] = acc;
-            s_cur[j] = s;
-            s_acc[j] = acc;
-        }
-    }
-    __syncthreads();
-    if (warp != 0) return;
-
-    decide_frame(a, b, s_cur, s_acc, mem, k, lane);
+    score_frame(a, b, sid_raw, sv, nrm, s_cur, s_acc);
 }
 
 // Finishing kernel of the tensor-core path: one CTA per frame turns the frame's row of dot
@@ -186,7 +156,11 @@ __global__ void k_batch_reset(float* __restrict__ sa, uint8_t* __restrict__ done
 
 }  // namespace
 
-cudaError_t lookup_setup() { return allow_max_dynamic_smem(k_score_exit); }
+cudaError_t lookup_setup() {
+    cudaError_t e = allow_max_dynamic_smem(k_score_exit);
+    if (e == cudaSuccess) e = prefer_max_smem_carveout(k_score_exit);
+    return e;
+}
 
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,
                                cudaStream_t st, int64_t* launches) {
@@ -204,11 +178,11 @@ cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const fl
     return launch_chained(k_finish_dense, a.B, kThreads, 0, st, a, dots, dots2, split_current);
 }
 
-cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches) {
+cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches, int threads) {
     if (a.B <= 0) return cudaSuccess;
     const size_t smem = (size_t(a.D) + 2 * size_t(a.k_max)) * sizeof(float);
     ++*launches;
-    return launch_chained(k_score_exit, a.B, kThreads, smem, st, a);
+    return launch_chained(k_score_exit, a.B, threads > 0 ? threads : kThreads, smem, st, a);
 }
 
 }  // namespace smtm

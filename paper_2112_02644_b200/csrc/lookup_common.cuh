@@ -167,6 +167,66 @@ __device__ __forceinline__ void decide_from_top2(const LookupArgs& a, int b, con
     if (r & 1) atomicAdd(&a.counters[SMTM_CTR_EXITS + a.layer], 1ull);
 }
 
+// Scores frame b against the members of its fast memory and decides, by a whole CTA (any whole number of
+// warps): sid_raw is the frame's stream id as read from memory (the caller fetches it along with its own first
+// loads), sv the frame's semantic vector in shared memory (already visible to every thread), nrm its squared
+// length; s_cur / s_acc hold k_max floats each.  Each warp takes fast-memory slots round-robin and reads the
+// member's centre (L2-resident) with 128-bit loads; lanes keep four independent fp32 accumulators and combine
+// with xor-shuffles, so every dot product has a fixed evaluation order.  Warp 0 then selects the two best.
+// The kernel's time is the number of dependent trips to memory: the size of the fast memory and the warp's
+// first class come in one trip, and a slot's centre, its length, its carry and the next slot's class in one more.
+__device__ __forceinline__ void score_frame(const LookupArgs& a, int b, int sid_raw, const float* sv, float nrm,
+                                            float* s_cur, float* s_acc) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x, nw = nthreads / kWarp;
+    const int sid = stream_checked(a, sid_raw);
+    const int32_t* mem = a.members + (size_t)max(sid, 0) * a.k_max;
+    int cls_next = mem[min(warp, a.k_max - 1)];  // unconditional: in flight with the size
+    const int k = sid < 0 ? 0 : a.k[sid];        // a stream id outside the cache: nothing to score against
+    const float weight = float(1u << a.layer);   // 2^(l-1) with l = layer + 1
+    const int D4 = (a.D & 3) ? 0 : a.D >> 2;     // 128-bit loads need rows that are multiples of 16 bytes
+    const float4* v4 = reinterpret_cast<const float4*>(sv);
+    for (int j = warp; j < k; j += nw) {
+        const int cls = cls_next;
+        const float4* c4 = reinterpret_cast<const float4*>(a.centers + (size_t)cls * a.D);
+        float cl = 0.f, old = 0.f;
+        if (lane == 0) {  // issued with the centre's loads
+            cl = a.cnorm[cls];
+            old = a.fresh ? 0.f : a.sa[(size_t)b * a.k_max + j];
+        }
+        if (j + nw < k) cls_next = mem[j + nw];
+        float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+        for (int i0 = 0; i0 < D4; i0 += 8 * kWarp) {  // eight pieces per lane in flight
+            float4 c[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) c[u] = __ldg(c4 + min(i0 + u * kWarp + lane, D4 - 1));
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * kWarp + lane;
+                if (i < D4) {
+                    const float4 v = v4[i];
+                    d0 = fmaf(c[u].x, v.x, d0); d1 = fmaf(c[u].y, v.y, d1); d2 = fmaf(c[u].z, v.z, d2); d3 = fmaf(c[u].w, v.w, d3);
+                }
+            }
+        }
+        for (int i = (D4 << 2) + lane; i < a.D; i += kWarp) d0 = fmaf(a.centers[(size_t)cls * a.D + i], sv[i], d0);
+        float dot = (d0 + d1) + (d2 + d3);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(kFull, dot, o);
+        if (lane == 0) {
+            const float s = cosine_from(dot, nrm, cl);    // Eq. 1
+            const float acc = __fmaf_rn(s, weight, old);  // Eq. 3
+            a.sa[(size_t)b * a.k_max + j] = acc;
+            s_cur[j] = s;
+            s_acc[j] = acc;
+        }
+    }
+    if (a.fresh)
+        for (int j = k + tid; j < a.k_max; j += nthreads) a.sa[(size_t)b * a.k_max + j] = 0.f;  // unused slots start from zero too
+    __syncthreads();
+    if (warp != 0) return;
+    decide_frame(a, b, s_cur, s_acc, mem, k, lane);
+}
+
 // Eq. 1 from a dot product and the two lengths; a zero-length vector is similar to nothing.
 __device__ __forceinline__ float cosine_from(float dot, float sv_norm2, float center_len) {
     return (sv_norm2 == 0.f || center_len == 0.f) ? 0.f

@@ -135,8 +135,8 @@ __global__ void __launch_bounds__(kUpdThreads) k_update_plan(const UpdateArgs a)
 // memory is all it takes.  Up to kPlanCountMax pairs the frames of every pair are counted in shared memory
 // (integer atomics: a sum), and a pair is listed with as many items as its count asks for; beyond, the pairs
 // are only elected, in a bitmap, and listed with one item each.  Nothing waits on a ticket or a fence.
-constexpr int kPlanOneThreads = 1024;
-constexpr int kPlanOneMaxB = 4 * kPlanOneThreads;
+constexpr int kPlanOneThreads = 512;   // (a CTA that fits on an SM beside a streaming kernel's)
+constexpr int kPlanOneMaxB = 8 * kPlanOneThreads;
 constexpr int kPlanOneWords = 2048;   // 65 536 (layer, class) pairs as a bitmap
 constexpr int kPlanCountMax = 8192;   // pairs that get a counter each
 
@@ -772,6 +772,7 @@ __global__ void __launch_bounds__(kApplyThreads, 8) k_update_apply(const UpdateA
 __global__ void __launch_bounds__(kUpdThreads) k_update_norms(const UpdateArgs a) {
     chain_wait();
     chain_release();
+    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_NORMS : nullptr);
     const int lane = threadIdx.x & 31;
     const int first = blockIdx.x * (kUpdThreads / kWarp) + (threadIdx.x >> 5);
     int code = a.plan.jobs[first];  // (the list has room for every warp) in flight with the count
@@ -828,6 +829,11 @@ __global__ void k_center_norms(const float* __restrict__ centers, int n, int D, 
 cudaError_t memory_setup() {
     cudaError_t e = allow_max_dynamic_smem(k_update_apply);
     if (e == cudaSuccess) e = allow_max_dynamic_smem(k_resize);
+    // the update's kernels share SMs with the next step's pooling kernel on the pipelined route
+    if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_apply);
+    if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_plan_one);
+    if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_plan);
+    if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_norms);
     return e;   // (the single-CTA plan needs at most 32 KB + its statics: below the default limit)
 }
 

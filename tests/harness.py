@@ -112,6 +112,7 @@ def step_pair(w, cache, mem, gb, lab, step, rep: Report, device="cuda", compare_
         x = si.frames(w, l, lab, step, device=device)
         if edit is not None:
             edit(l, x)
+        torch.cuda.synchronize()   # the maps are complete before the lookup is enqueued (SMTM_FLAG_MAPS_READY asks for it)
         B, C, H, W = si.shape4(w, l)
         todo = ob["done"] == 0
         (smtm.smtm_lookup_exit_begin if begin and l == 0 else smtm.smtm_lookup_exit)(

@@ -116,13 +116,13 @@ def test_argument_errors_launch_nothing():
 def test_c1_single_layer_fp32():
     rep = run_workload(si.C1)
     assert rep.exits == [8] and rep.band_mismatches == 0
-    assert rep.routes == [1, 0, 0]       # one fused launch: pooling, Eq. 1, Eq. 3, Eq. 4 and the decision
+    assert rep.routes == [1, 0, 0, 0]       # one fused launch: pooling, Eq. 1, Eq. 3, Eq. 4 and the decision
 
 
 def test_c2_resnet50_bf16_four_layers():
     rep = run_workload(si.C2)
     assert sum(rep.exits) > 30 and rep.frames == 64
-    assert rep.routes == [4, 0, 0]
+    assert rep.routes == [4, 0, 0, 0]
 
 
 def test_c2_exits_disabled_streams_every_layer():
@@ -143,7 +143,7 @@ def test_c3_mobilenetv2_fp16_nhwc_novel_classes_do_not_exit():
 def test_c4_large_cache_straddles_threshold():
     rep = run_workload(si.C4)
     assert 100 < rep.exits[0] < 900
-    assert rep.routes == [0, 1, 0], "the 1000-entry fast memory must be scored on the tensor cores (Eq. 1 as a dense contraction)"
+    assert rep.routes == [0, 1, 0, 0], "the 1000-entry fast memory must be scored on the tensor cores (Eq. 1 as a dense contraction)"
     print("c4 max |SA error|:", rep.max_sa_err, "max SV error:", rep.max_sv_err)
     print("c4 near-threshold lookups (oracle):", rep.near_oracle, "band mismatches:", rep.band_mismatches)
 
@@ -152,7 +152,7 @@ def test_c4_large_cache_straddles_threshold():
 def test_c5_streaming_full_width(T):
     rep = run_workload(si.C5, steps=T)
     assert rep.frames == 512 * T and rep.exits[0] > 0
-    assert rep.routes == [2 * T, 0, 0]
+    assert rep.routes == [2 * T, 0, 0, 0]
 
 
 def test_c5_full_length_64_steps_state_only():
@@ -182,11 +182,11 @@ def test_large_fast_memory_over_several_layers_uses_tensor_cores():
                     k_min=70, k_max=196, S=1, T=4, tau=0.8, window_W=2, sigma=0.6, zipf_s=0.9, repeat_p=0.3, seed=6)
     rep = run_workload(w)
     assert rep.frames == 70 * 4 and rep.lookups > 70
-    assert rep.routes == [0, 8, 0]       # both layers of all four steps on the tensor-core route
+    assert rep.routes == [0, 8, 0, 0]       # both layers of all four steps on the tensor-core route
     w3 = si.Workload("dense_nhwc", si.F16, si.NHWC, B=33, stages=((320, 7, 7),), n=72, k_init=72, k_min=72, k_max=72,
                      S=1, T=2, tau=0.8, sigma=1.0, zipf_s=1.0, seed=8)
     rep3 = run_workload(w3)
-    assert rep3.frames == 66 and rep3.routes == [0, 2, 0]
+    assert rep3.frames == 66 and rep3.routes == [0, 2, 0, 0]
 
 
 def test_forgetting_frequency_table_rapid_scene_change():
@@ -414,6 +414,8 @@ def test_maps_ready_flag_with_alternating_batches():
     assert np.array_equal(gbs[(w.T - 1) % 2].done.cpu().numpy(), ob["done"])
     assert np.array_equal(gbs[(w.T - 1) % 2].pred.cpu().numpy(), ob["pred"])
     compare_state(w, cache, mem, rep)
+    routes = smtm.smtm_cache_get_routes(cache)
+    assert routes[smtm.ROUTE_PIPELINED] == 2 * 2 * w.T and routes.sum() == routes[smtm.ROUTE_PIPELINED]
     smtm.smtm_cache_destroy(cache)
 
 

@@ -108,6 +108,10 @@ def test_static_lookups_back_to_back_on_a_cache_that_may_start_early():
         we, wp, wac = want[r]
         assert np.array_equal(e.cpu().numpy(), we), r
         assert np.array_equal(p.cpu().numpy(), np.where(we == 1, wp, -1)), r
-        assert np.array_equal(ac.cpu().numpy()[:, r % 2], wac[:, r % 2]), r
+        # (the regular lookup of such a cache may take another route than the static one: same decisions, and
+        # confidences equal up to the rounding of the dot products)
+        got_ac, want_ac = ac.cpu().numpy()[:, r % 2].astype(np.float64), wac[:, r % 2].astype(np.float64)
+        fin = np.isfinite(want_ac)
+        assert np.array_equal(np.isfinite(got_ac), fin) and np.all(np.abs(got_ac[fin] - want_ac[fin]) <= 2e-3 * (1 + np.abs(want_ac[fin]))), r
     assert smtm.smtm_cache_status(cache) == 0
     smtm.smtm_cache_destroy(cache)
