@@ -290,8 +290,7 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * of the other routes), for the scoring kernel of layer i where pooling and
  * scoring are separate kernels (SMTM_PROF_SCORE + i), for the update (the plan
  * kernel SMTM_PROF_PLAN; the CTAs of the apply kernel that fold centres,
- * _CENTERS, and those that keep the tables, _TABLES; the kernel that renews the
- * centres' lengths, _NORMS) and for the tensor-core scorer of the dense route
+ * _CENTERS, and those that keep the tables, _TABLES) and for the tensor-core scorer of the dense route
  * (SMTM_PROF_SCORE_TC; with several dense layers in a step, from the first
  * one's begin to the last one's end).  This
  * leaves out what the event nodes add around a kernel.  Only the most recent
@@ -304,7 +303,7 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * device. */
 enum {
     SMTM_PROF_SCORE = SMTM_MAX_LAYERS,  /* + layer: the scoring kernel of a layer whose pooling is a kernel of its own */
-    SMTM_PROF_PLAN = 2 * SMTM_MAX_LAYERS, SMTM_PROF_CENTERS, SMTM_PROF_TABLES, SMTM_PROF_SCORE_TC, SMTM_PROF_NORMS,
+    SMTM_PROF_PLAN = 2 * SMTM_MAX_LAYERS, SMTM_PROF_CENTERS, SMTM_PROF_TABLES, SMTM_PROF_SCORE_TC,
     SMTM_PROF_KERNELS
 };
 smtm_status_t smtm_cache_profile(smtm_cache_t* cache, int32_t max_lookups, int32_t every);

@@ -364,8 +364,8 @@ def smtm_cache_get_profile(cache: Cache, layer: int):
 
 
 PROF_SCORE = MAX_LAYERS   # + layer: the scoring kernel of a layer whose pooling is a kernel of its own
-PROF_PLAN, PROF_CENTERS, PROF_TABLES, PROF_SCORE_TC, PROF_NORMS, PROF_KERNELS = (
-    2 * MAX_LAYERS, 2 * MAX_LAYERS + 1, 2 * MAX_LAYERS + 2, 2 * MAX_LAYERS + 3, 2 * MAX_LAYERS + 4, 2 * MAX_LAYERS + 5)
+PROF_PLAN, PROF_CENTERS, PROF_TABLES, PROF_SCORE_TC, PROF_KERNELS = (
+    2 * MAX_LAYERS, 2 * MAX_LAYERS + 1, 2 * MAX_LAYERS + 2, 2 * MAX_LAYERS + 3, 2 * MAX_LAYERS + 4)
 
 
 def smtm_cache_get_profile_device(cache: Cache):

@@ -39,7 +39,8 @@ struct smtm_cache {
     bool mark_valid[2];
     int mark_next;                      // which of the two the next first lookup records
     int32_t* d_jobs;             // scratch of the update: [4] counters, [L][n] (layer, class) pairs to fold, [16][L][n] work items
-    uint32_t* d_m_next;          // scratch of the update: [L][n] counts after the update
+    float* d_norm_part;          // scratch of the update: [L][n][16] squared lengths of the blocks of a centre folded by several CTAs
+    int32_t* d_ticket;           // scratch of the update: [L][n] tickets of those CTAs (zero between updates)
     unsigned long long* d_epoch; // [2] device: update calls so far, and the plan kernel's ticket
     // optional timing of the streaming kernel of every lookup (smtm_cache_profile)
     std::vector<cudaEvent_t>* prof_events;  // pairs, in launch order
@@ -129,7 +130,8 @@ void free_all(smtm_cache* c) {
     for (cudaEvent_t e : c->ev_mark)
         if (e) cudaEventDestroy(e);
     cudaFree(c->d_jobs);
-    cudaFree(c->d_m_next);
+    cudaFree(c->d_norm_part);
+    cudaFree(c->d_ticket);
     cudaFree(c->hb.d_sa);
     cudaFree(c->hb.d_done);
     cudaFree(c->hb.d_exit_layer);
@@ -177,10 +179,10 @@ EncodeArgs encode_args(const smtm_cache* c, const smtm_fmap_t* f, const uint8_t*
 // the CTAs of the latency-bound kernels of a step (scoring, sparse pooling, update) fit on an SM beside a CTA of
 // the next step's pooling kernel.
 constexpr int kPipelinedScoreThreads = 128;
-constexpr int kPipelinedRingStages = 6;
-constexpr int kPipelinedRingConsumers = 3;  // (each looks after two stages)
-// Copies the pooling kernel keeps outstanding per SM on this route.  Every access the latency-bound kernels make
-// to memory queues behind them, so no more than the bandwidth needs (148 x 2 x 25 KB = 7.4 MB in flight).
+constexpr int kPipelinedRingStages = 5;
+constexpr int kPipelinedRingConsumers = 3;
+// Copies the pooling kernel keeps outstanding per SM on this route (148 x 2 x 25 KB = 7.4 MB in flight; more did not
+// make it faster beside the latency-bound kernels, and every access those make to memory queues behind them).
 constexpr int kPipelinedInFlight = 2;
 
 // The capture the stream is in (0 = none).
@@ -288,11 +290,16 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
         ++c->routes[SMTM_ROUTE_PIPELINED];
         e.clock = a.clock ? a.clock + 2 * layer : nullptr;  // the pooling kernel is this layer's streaming kernel
         if (begin) return pooled_first_lookup(c, e, a, st, timing, profiled_step_begins);
-        // a later layer: the frames still in are few; small CTAs pool them, small CTAs score them
+        // a later layer: the frames still in are few; clusters of small CTAs look them up whole, or, for shapes
+        // those do not serve, small CTAs pool them and small CTAs score them
         if (timing) SMTM_CUDA(record_timing(timing[0], st));
-        SMTM_CUDA(launch_pool_sparse(e, c->sm_count, st, &c->launches));
+        const bool whole = launch_lookup_sparse_supported(e, a);
+        if (whole)
+            SMTM_CUDA(launch_lookup_sparse(e, a, c->sm_count, st, &c->launches));
+        else
+            SMTM_CUDA(launch_pool_sparse(e, c->sm_count, st, &c->launches));
         if (timing) SMTM_CUDA(record_timing(timing[1], st));
-        SMTM_CUDA(launch_score_exit(a, st, &c->launches, kPipelinedScoreThreads));
+        if (!whole) SMTM_CUDA(launch_score_exit(a, st, &c->launches, kPipelinedScoreThreads));
         return SMTM_OK;
     }
     SMTM_CUDA(launch_lookup_fused(e, a, c->sm_count, &c->fused_caps, st, &c->launches, &fused, timing));
@@ -353,7 +360,8 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     a.plan.job_count = c->d_jobs;
     a.plan.jobs = c->d_jobs + 4;
     a.plan.items = c->d_jobs + 4 + size_t(c->L) * c->n;
-    a.m_next = c->d_m_next;
+    a.norm_part = c->d_norm_part;
+    a.ticket = c->d_ticket;
     a.plan.epoch = c->d_epoch;
     a.stream_id = b->d_stream_id;
     a.done = b->d_done;
@@ -490,7 +498,8 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     }
     ok = ok && dev_alloc(&c->d_tags, size_t(c->L) * n) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_jobs, 4 + 17 * size_t(c->L) * n) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_m_next, size_t(c->L) * n) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_norm_part, 16 * size_t(c->L) * n) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_ticket, size_t(c->L) * n) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_epoch, 2) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->pool_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
@@ -526,6 +535,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     if (e == cudaSuccess) e = cudaMemset(c->d_tags, 0, size_t(c->L) * n * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMemset(c->d_jobs, 0, (4 + 17 * size_t(c->L) * n) * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(c->d_epoch, 0, 2 * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(c->d_ticket, 0, size_t(c->L) * n * sizeof(int32_t));
     if (e == cudaSuccess)
         e = cudaMemcpy(c->d_members, members.data(), members.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(c->d_k, ks.data(), ks.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
@@ -618,7 +628,8 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
     a.plan.job_count = c->d_jobs;
     a.plan.jobs = c->d_jobs + 4;
     a.plan.items = c->d_jobs + 4 + size_t(c->L) * c->n;
-    a.m_next = c->d_m_next;
+    a.norm_part = c->d_norm_part;
+    a.ticket = c->d_ticket;
     a.plan.epoch = c->d_epoch;
     a.fallback = d_labels;
     a.split_current = c->d_split_current;

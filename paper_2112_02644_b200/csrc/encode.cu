@@ -742,6 +742,206 @@ __global__ void __launch_bounds__(kLightThreads) k_pool_sparse(const LightParams
     }
 }
 
+// ---- the same frames looked up whole: pooling, scoring and the decision by a cluster of small CTAs ----
+//
+// A thread-block cluster of P CTAs takes active frames one at a time; CTA `rank` fetches chunk `rank` of the
+// frame (one trip to memory for the whole frame), pools it, and scores its slice of the semantic vector
+// against the frame's fast-memory centres; the partial dot products and the partial squared length go
+// through distributed shared memory to the cluster's first CTA, whose first warp adds the parts in rank
+// order and decides (Eq. 1, Eq. 3, top-2, Eq. 4, the exit rule), as the fused streaming kernel does.  One
+// cluster-wide barrier per frame; two receive buffers take turns.  P = chunks per frame <= 8, and a chunk
+// here is a chunk of the streaming kernel (<= 25 KB): a whole frame is in flight at once.
+constexpr int kSparseStageCap = kStageCap;
+constexpr int kSparseFrames = 64;    // frames a cluster can be given
+constexpr int kSparseSlice = 1024;   // channels of a chunk at most (as the fused kernel's slices)
+
+struct SparseParams {
+    NchwParams e;
+    LookupArgs a;
+    int groups;  // clusters
+    int gran;    // channels that must stay in one warp's share (the reducer's unit)
+};
+
+constexpr size_t sparse_smem(int slice) {
+    return size_t(kSparseStageCap) + size_t(slice) * 4 + 2 * size_t(kMaxCluster) * kRxRow * 4 + 2 * kSparseFrames * 4 + 64 * 4 + 64;
+}
+
+template <class R>
+__global__ void __launch_bounds__(kLightThreads) k_lookup_sparse(const SparseParams f) {
+    extern __shared__ uint8_t smem_raw[];
+    const NchwParams& p = f.e;
+    const LookupArgs& a = f.a;
+    uint8_t* stage = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 15) & ~uintptr_t(15));
+    float* sv_s = reinterpret_cast<float*>(stage + kSparseStageCap);       // [chunk_channels] this CTA's slice
+    float* rx = sv_s + p.chunk_channels;                                   // [2][P][kRxRow] (used in the first CTA)
+    int* my_frames = reinterpret_cast<int*>(rx + 2 * kMaxCluster * kRxRow);  // [kSparseFrames]
+    int* my_sids = my_frames + kSparseFrames;                              // [kSparseFrames] their stream ids
+    int* s_scan = my_sids + kSparseFrames;                                 // [33]
+    const int P = p.chunks_per_frame;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int B = a.B;
+    const int rank = int(blockIdx.x) % P, group = int(blockIdx.x) / P;
+    chain_wait();  // the exit flags are the previous kernel's
+    chain_release();
+    const ClockScope stamps(a.clock ? a.clock + 2 * a.layer : nullptr);
+    // The active frames of this cluster and their streams.  Exit flags and stream ids of eight tiles of frames
+    // come in one trip to memory.
+    uint8_t flags[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int sids[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int n_active = 0;
+    for (int t0 = 0; t0 < B; t0 += kLightThreads) {
+        const int b = t0 + tid;
+        if ((t0 / kLightThreads) % 8 == 0) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                flags[u] = a.done[min(b + u * kLightThreads, B - 1)];
+                sids[u] = a.stream_id ? a.stream_id[min(b + u * kLightThreads, B - 1)] : 0;
+            }
+        }
+        uint8_t mine = 0;
+        int sid_b = 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            mine = ((t0 / kLightThreads) % 8 == u) ? flags[u] : mine;
+            sid_b = ((t0 / kLightThreads) % 8 == u) ? sids[u] : sid_b;
+        }
+        const int act = (b < B && !mine) ? 1 : 0;
+        int cnt;
+        const int pos = block_exclusive_scan(act, s_scan, &cnt);
+        if (act) {
+            const int u = n_active + pos;
+            if (u % f.groups == group && u / f.groups < kSparseFrames) {
+                my_frames[u / f.groups] = b;
+                my_sids[u / f.groups] = sid_b;
+            }
+        }
+        n_active += cnt;
+    }
+    const int nu = n_active > group ? min((n_active - group + f.groups - 1) / f.groups, kSparseFrames) : 0;
+    __syncthreads();
+    const int c0 = rank * p.chunk_channels;
+    const int nch = min(p.chunk_channels, p.C - c0);   // channels of this CTA's slice (a multiple of 4)
+    const int vectors = nch * p.ch_bytes / 16;
+    const int units = (nch + f.gran - 1) / f.gran;
+    const int u_lo = min(units, warp * ((units + 3) / 4)), u_hi = min(units, u_lo + (units + 3) / 4);
+    const int w_c0 = u_lo * f.gran, w_nch = min(nch, u_hi * f.gran) - w_c0;
+    const int n4 = nch >> 2;
+    const int pp = (n4 + kWarp - 1) / kWarp;       // 16-byte pieces of a centre's slice per lane (at most 8)
+    const int spr = max(1, 8 / max(pp, 1));        // slots a warp scores per trip to memory
+    const float weight = float(1u << a.layer);     // 2^(l-1) with l = layer + 1
+    constexpr int kLoads = (kSparseStageCap / 16 + kLightThreads - 1) / kLightThreads;  // 13: a whole chunk in flight
+    for (int k_it = 0; k_it < nu; ++k_it) {
+        const int b = my_frames[k_it];
+        const int sid = stream_checked(a, my_sids[k_it]);
+        const uint4* src = reinterpret_cast<const uint4*>(p.x + (long long)b * p.frame_bytes + (long long)c0 * p.ch_bytes);
+        uint4* dst = reinterpret_cast<uint4*>(stage);
+        uint4 r[kLoads];
+#pragma unroll
+        for (int u = 0; u < kLoads; ++u) r[u] = __ldg(src + min(u * kLightThreads + tid, vectors - 1));
+        // the frame's fast memory: its size and this warp's classes (slot j = warp + 4 i), in flight with the chunk
+        const int32_t* mem = a.members + (size_t)max(sid, 0) * a.k_max;
+        const int k = sid < 0 ? 0 : min(a.k[sid], kFusedMaxK);
+        int cls_w = 0;  // lane i < 16 holds the class of slot warp + 4 i
+        if (lane < kFusedMaxK / 4 && warp + 4 * lane < a.k_max) cls_w = mem[warp + 4 * lane];
+        // the finisher's own loads: the slots' classes (lane l: slots l and l + 32)
+        int ids[2] = {0, 0};
+        if (rank == 0 && warp == 0) {
+            ids[0] = lane < a.k_max ? mem[lane] : 0;
+            ids[1] = lane + kWarp < a.k_max ? mem[lane + kWarp] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < kLoads; ++u)
+            if (u * kLightThreads + tid < vectors) dst[u * kLightThreads + tid] = r[u];
+        __syncthreads();
+        if (w_nch > 0)
+            R::run(stage + size_t(w_c0) * p.ch_bytes, w_nch, lane, p.sv + (long long)b * p.C + c0 + w_c0, sv_s + w_c0, p.inv_hw, p);
+        __syncthreads();  // the slice is complete; the stage is free
+        const uint32_t out = peer_smem(rx + ((k_it & 1) * kMaxCluster + rank) * kRxRow, 0);
+        const float4* v4 = reinterpret_cast<const float4*>(sv_s);
+        // the centres' lengths and the carry, for the finisher: in flight with the centre slices below
+        float clen[2] = {0.f, 0.f}, sa_old[2] = {0.f, 0.f};
+        if (rank == 0 && warp == 0) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = lane + h * kWarp;
+                if (j < k) {
+                    clen[h] = a.cnorm[ids[h]];
+                    sa_old[h] = a.fresh ? 0.f : a.sa[(size_t)b * a.k_max + j];
+                }
+            }
+        }
+        if (warp == 3) {  // partial squared length of the semantic vector
+            float nn = 0.f;
+            for (int q = lane; q < n4; q += kWarp) {
+                const float4 xv = v4[q];
+                nn = fmaf(xv.x, xv.x, nn); nn = fmaf(xv.y, xv.y, nn); nn = fmaf(xv.z, xv.z, nn); nn = fmaf(xv.w, xv.w, nn);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(kFull, nn, o);
+            if (lane == 0) peer_store(out + kFusedMaxK * 4, nn);
+        }
+        // this warp's slots, `spr` of them per trip to memory: eight pieces of centre slices per lane in flight
+        for (int i0 = 0; warp + 4 * i0 < k; i0 += spr) {
+            float4 c[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int si = e / pp, piece = e - si * pp;       // slot within the round, piece of its slice
+                const int j = warp + 4 * (i0 + si), q = lane + piece * kWarp;
+                const int cls = __shfl_sync(kFull, cls_w, min(i0 + si, kFusedMaxK / 4 - 1));
+                c[e] = (si < spr && j < k && q < n4)
+                           ? __ldg(reinterpret_cast<const float4*>(a.centers + (size_t)cls * p.C + c0) + q)
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            for (int si = 0; si < spr; ++si) {
+                const int j = warp + 4 * (i0 + si);
+                if (j >= k) break;
+                float d = 0.f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int q = lane + (e - si * pp) * kWarp;
+                    if (e / pp == si && q < n4) {
+                        const float4 xv = v4[q];
+                        d = fmaf(c[e].x, xv.x, d); d = fmaf(c[e].y, xv.y, d); d = fmaf(c[e].z, xv.z, d); d = fmaf(c[e].w, xv.w, d);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(kFull, d, o);
+                if (lane == 0) peer_store(out + j * 4, d);
+            }
+        }
+        // every part of this frame has been delivered (and the previous frame's decision is made)
+        if (P > 1) cluster_sync_all(); else __syncthreads();
+        if (rank == 0 && warp == 0) {
+            const float* rxb = rx + (k_it & 1) * kMaxCluster * kRxRow;
+            float nn = 0.f, dots[2] = {0.f, 0.f};
+            for (int rr = 0; rr < P; ++rr) {  // the parts in rank order
+                const float* row = rxb + rr * kRxRow;
+                nn += row[kFusedMaxK];
+                if (lane < k) dots[0] += row[lane];
+                if (lane + kWarp < k) dots[1] += row[lane + kWarp];
+            }
+            float s_cur[2] = {0.f, 0.f}, s_acc[2] = {0.f, 0.f};
+            const float sv_len = __fsqrt_rn(nn);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = lane + h * kWarp;
+                if (j < k) {
+                    s_cur[h] = (nn == 0.f || clen[h] == 0.f) ? 0.f : __fdiv_rn(dots[h], __fmul_rn(sv_len, clen[h]));  // Eq. 1
+                    s_acc[h] = __fmaf_rn(s_cur[h], weight, sa_old[h]);   // Eq. 3
+                    a.sa[(size_t)b * a.k_max + j] = s_acc[h];
+                } else if (a.fresh && j < a.k_max) {
+                    a.sa[(size_t)b * a.k_max + j] = 0.f;                 // unused slots start from zero too
+                }
+            }
+            const Top2 ta = warp_top2_keys(s_acc, ids, k, lane);
+            Top2 ts{0.f, 0.f, -1, -1};
+            if (a.sep) ts = warp_top2_keys(s_cur, ids, k, lane);  // only Eq. 2 (a diagnostic) needs it
+            if (lane == 0) decide_from_top2(a, b, ta, ts);
+        }
+    }
+    if (P > 1) cluster_sync_all();  // no CTA leaves while a peer may still write to its shared memory
+}
+
 // ---- NHWC: direct coalesced loads ----------------------------------------------------------
 
 constexpr int kThreadsNhwc = 256;
@@ -1041,7 +1241,10 @@ cudaError_t max_clusters(int parts, size_t smem, int* out) {
 template <class R>
 cudaError_t carveout_pipelined() {
     cudaError_t e = prefer_max_smem_carveout(k_encode_nchw<R>);
-    return e != cudaSuccess ? e : prefer_max_smem_carveout(k_pool_sparse<R>);
+    if (e == cudaSuccess) e = prefer_max_smem_carveout(k_pool_sparse<R>);
+    if (e == cudaSuccess) e = prefer_max_smem_carveout(k_lookup_sparse<R>);
+    if (e == cudaSuccess) e = allow_max_dynamic_smem(k_lookup_sparse<R>);
+    return e;
 }
 
 cudaError_t encode_setup() {
@@ -1119,6 +1322,42 @@ cudaError_t launch_pool_sparse(const EncodeArgs& a, int sm_count, cudaStream_t s
     SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
 #undef SMTM_LAUNCH
     return e;
+}
+
+// The layout of a sparse lookup, or kNone when the shape is not served: chunks as the streaming kernel cuts
+// them, at most 8 to a frame, slices that are whole 16-byte pieces and fit the scorers' registers.
+Reducer plan_sparse(const EncodeArgs& e, const LookupArgs& a, SparseParams* f) {
+    if (e.layout != SMTM_NCHW || e.B <= 0 || a.k_max > kFusedMaxK || (e.C & 3)) return kNone;
+    const Reducer r = plan_nchw(e, &f->e);
+    if (r == kNone) return kNone;
+    if (f->e.chunks_per_frame > kMaxCluster || (f->e.chunk_channels & 3) || f->e.chunk_channels > kSparseSlice) return kNone;
+    f->gran = r <= kUnitF32x49 ? f->e.chunk_channels / 32 : std::max(1, 32 / std::max(1, f->e.team));
+    return r;
+}
+
+bool launch_lookup_sparse_supported(const EncodeArgs& e, const LookupArgs& a) {
+    SparseParams f{};
+    return plan_sparse(e, a, &f) != kNone;
+}
+
+cudaError_t launch_lookup_sparse(const EncodeArgs& e, const LookupArgs& a, int sm_count, cudaStream_t st, int64_t* launches) {
+    SparseParams f{};
+    const Reducer r = plan_sparse(e, a, &f);
+    if (r == kNone) return cudaErrorInvalidValue;
+    f.a = a;
+    const int P = f.e.chunks_per_frame;
+    // about three CTAs to an SM (they sit beside a streaming kernel); enough clusters that none is given more
+    // frames than it can list
+    int groups = std::max(1, std::min(e.B, 3 * sm_count / P));
+    groups = std::max(groups, (e.B + kSparseFrames - 1) / kSparseFrames);
+    f.groups = groups;
+    const size_t smem = sparse_smem(f.e.chunk_channels);
+    cudaError_t err = cudaSuccess;
+    ++*launches;
+#define SMTM_LAUNCH(...) err = launch_chained_cluster(k_lookup_sparse<__VA_ARGS__>, P * groups, kLightThreads, smem, P, st, f)
+    SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
+#undef SMTM_LAUNCH
+    return err;
 }
 
 cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm_count, FusedCaps* caps, cudaStream_t st,

@@ -139,6 +139,10 @@ cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* lau
 // memories of at most 64 entries).  *handled is false when the shape is not served, in which
 // case nothing was launched.
 constexpr int kFusedMaxK = 64;  // fast-memory capacity the fused path supports (two slots per lane)
+// Lookup (pooling, scoring, decision) of the frames still in at a later layer by clusters of small CTAs that fit
+// beside a streaming kernel: NCHW shapes the streaming pipeline cuts into at most 8 chunks per frame.
+bool launch_lookup_sparse_supported(const EncodeArgs& e, const LookupArgs& a);
+cudaError_t launch_lookup_sparse(const EncodeArgs& e, const LookupArgs& a, int sm_count, cudaStream_t st, int64_t* launches);
 // What the device answered when asked how many clusters of 2, 4, 8 CTAs of each variant of the fused
 // kernel it runs at once (0 = not asked yet, -1 = refused); kept per cache, i.e. per device.
 struct FusedCaps {
@@ -204,7 +208,8 @@ struct UpdateArgs {
     float* centers[SMTM_MAX_LAYERS];
     float* cnorm[SMTM_MAX_LAYERS];
     uint32_t* m[SMTM_MAX_LAYERS];
-    uint32_t* m_next;          // [L][n] scratch: the counts after this update, written by Eq. 7's CTAs, adopted by the norms kernel
+    float* norm_part;          // [L][n][16] scratch: squared lengths of the column blocks of a centre that several CTAs fold
+    int32_t* ticket;           // [L][n] scratch, zero between updates: how many of those CTAs are through
 };
 
 

@@ -15,7 +15,8 @@
 // first B CTAs look after the tables, one per frame (the CTA of a stream's first frame in the
 // batch applies all of the stream's frames to its tables and, when asked, refreshes its fast
 // memory by Eq. 5 / Eq. 6; the others leave at once); the remaining CTAs take the listed pairs,
-// one each, and fold the pair's frames into the centre (Eq. 7).  Small CTAs on purpose: there
+// one each, and fold the pair's frames into the centre (Eq. 7; a pair with many frames is several items, each
+// a block of the vector's columns).  Small CTAs on purpose: there
 // are hundreds of independent pieces of work, each a short chain of dependent trips to L2, so
 // the kernel is as fast as the number of pieces in flight, and its CTAs fit beside the CTAs of a
 // streaming kernel that holds most of an SM's shared memory.  Classes and streams the batch does
@@ -625,12 +626,15 @@ constexpr int kRowGroupsMax = 8;
 
 // Lists, in ascending index, the frames base .. base + kCenTile - 1 whose label is cls and that stopped at
 // layer l0 + 1 or deeper; returns how many (the same in every thread).  Every thread fetches the codes of its
-// run of consecutive frames in one trip to memory; one scan over the threads places them.
-__device__ __forceinline__ int list_pair_frames(const UpdateArgs& a, int base, int cls, int l0, int* s_list, int* s_scan) {
+// run of consecutive frames in one trip to memory (first_tile: those of frames 0 .. kCenTile - 1, which do not
+// depend on the pair and are fetched before the pair is known); one scan over the threads places them.
+__device__ __forceinline__ int list_pair_frames(const UpdateArgs& a, int base, int cls, int l0, int* s_list, int* s_scan,
+                                                const int (&first_tile)[kCenPer]) {
     const int f0 = base + threadIdx.x * kCenPer;
     int code[kCenPer];
 #pragma unroll
-    for (int i = 0; i < kCenPer; ++i) code[i] = a.plan.frame_code[min(f0 + i, a.B - 1)];
+    for (int i = 0; i < kCenPer; ++i)  // (the first tile's codes were fetched when the CTA began)
+        code[i] = base == 0 ? first_tile[i] : a.plan.frame_code[min(f0 + i, a.B - 1)];
     int mine = 0;
 #pragma unroll
     for (int i = 0; i < kCenPer; ++i) {
@@ -653,16 +657,20 @@ __device__ __forceinline__ int list_pair_frames(const UpdateArgs& a, int base, i
 // label is cls and that stopped at layer l0 + 1 or deeper are listed in ascending index, a tile of frames at a
 // time (every thread looks at a run of consecutive frames, one scan over the threads).  A thread is (a 16-byte
 // group of columns, a row group): row group r adds the listed rows r, r + R, ... in that order (eight rows in
-// flight), the groups' sums are added in a fixed order, then SC = (SC m + sum SV) / (m + q).  The centre's
-// length and its count are left to k_update_norms (the items of a pair share them); the item of block 0
-// leaves the new count in m_next.
-__device__ void centre_item(const UpdateArgs& a, int item, int* s_list, int* s_scan, float4* s_acc) {
+// flight), the groups' sums are added in a fixed order, then SC = (SC m + sum SV) / (m + q).  A pair that is a
+// single item then renews the centre's length and count itself.  The items of a cut pair leave the squared
+// length of their blocks in norm_part and take a ticket; the last one through adds the blocks in order and
+// renews length and count (every item has read the count by then), and puts the ticket back to zero.
+__device__ void centre_item(const UpdateArgs& a, int item, const int (&first_tile)[kCenPer], int* s_list, int* s_scan,
+                            float4* s_acc) {
     const int tid = threadIdx.x, nt = blockDim.x;
     const int cls = item & 0x1fff, l0 = (item >> 16) & 15, blk = (item >> 20) & 15, nblk = 1 << ((item >> 24) & 7);
     const int D = a.dims[l0];
     const float* sv = a.sv[l0];
     float* cen = a.centers[l0] + (size_t)cls * D;
     const uint32_t m = a.m[l0][cls];
+    float nrm = 0.f;
+    int q = 0;
     if ((D & 3) == 0) {
         const int D4 = D >> 2, per_blk = (D4 + nblk - 1) / nblk;
         const int lo4 = min(D4, blk * per_blk), hi4 = min(D4, lo4 + per_blk);  // this item's 16-byte column groups
@@ -676,9 +684,9 @@ __device__ void centre_item(const UpdateArgs& a, int item, int* s_list, int* s_s
             float4 old = make_float4(0.f, 0.f, 0.f, 0.f);
             if (mine_col && rg == 0) old = *reinterpret_cast<const float4*>(cen + 4 * c4);  // in flight with the listing
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            int q = 0;
+            q = 0;
             for (int base = 0; base < a.B; base += kCenTile) {
-                const int cnt = list_pair_frames(a, base, cls, l0, s_list, s_scan);
+                const int cnt = list_pair_frames(a, base, cls, l0, s_list, s_scan, first_tile);
                 if (cnt == 0) continue;  // (the same for every thread)
                 q += cnt;
                 if (!mine_col) continue;
@@ -711,26 +719,45 @@ __device__ void centre_item(const UpdateArgs& a, int item, int* s_list, int* s_s
                 v.z = float((double(old.z) * dm + double(acc[2])) * inv);
                 v.w = float((double(old.w) * dm + double(acc[3])) * inv);
                 *reinterpret_cast<float4*>(cen + 4 * c4) = v;
+                nrm = fmaf(v.x, v.x, nrm); nrm = fmaf(v.y, v.y, nrm); nrm = fmaf(v.z, v.z, nrm); nrm = fmaf(v.w, v.w, nrm);
             }
-            if (tid == 0 && blk == 0 && s4 == lo4) a.m_next[(size_t)l0 * a.n + cls] = m + uint32_t(q);
         }
     } else {
         // a vector that is not a whole number of 16-byte pieces (never cut into blocks): a column per thread
-        int q = 0;
         for (int d = tid; d < D || d - tid < D; d += nt) {  // every thread makes every trip (the listing is the CTA's)
             float acc = 0.f;
             q = 0;
             for (int base = 0; base < a.B; base += kCenTile) {
-                const int cnt = list_pair_frames(a, base, cls, l0, s_list, s_scan);
+                const int cnt = list_pair_frames(a, base, cls, l0, s_list, s_scan, first_tile);
                 if (cnt == 0) continue;
                 q += cnt;
                 if (d < D)
                     for (int i = 0; i < cnt; ++i) acc += sv[(size_t)s_list[i] * D + d];
             }
-            if (d < D && q > 0) cen[d] = float((double(cen[d]) * double(m) + double(acc)) / (double(m) + double(q)));
+            if (d < D && q > 0) {
+                const float v = float((double(cen[d]) * double(m) + double(acc)) / (double(m) + double(q)));
+                cen[d] = v;
+                nrm = fmaf(v, v, nrm);
+            }
         }
-        if (tid == 0) a.m_next[(size_t)l0 * a.n + cls] = m + uint32_t(q);
     }
+    if (q == 0) return;  // cannot happen for a listed pair (the same for every thread)
+    __syncthreads();     // s_acc is free: it serves the sum below
+    nrm = block_sum(nrm, reinterpret_cast<float*>(s_acc));
+    if (tid != 0) return;
+    if (nblk > 1) {
+        const size_t pair = (size_t)l0 * a.n + cls;
+        a.norm_part[pair * kItemBlocksMax + blk] = nrm;
+        __threadfence();  // this item's part of the centre and of its length, before the ticket
+        if (atomicAdd(a.ticket + pair, 1) != nblk - 1) return;
+        __threadfence();
+        nrm = 0.f;
+        for (int k = 0; k < nblk; ++k) nrm += *reinterpret_cast<volatile float*>(a.norm_part + pair * kItemBlocksMax + k);
+        a.ticket[pair] = 0;
+    }
+    a.cnorm[l0][cls] = __fsqrt_rn(nrm);
+    a.m[l0][cls] = m + uint32_t(q);
+    if (a.split_current) a.split_current[l0] = 0;  // the tensor-core scorer's copy of this layer's centres is stale
 }
 
 // The apply kernel: CTAs [0, table_ctas) are tables CTAs, one per frame; the others take the listed items.
@@ -755,7 +782,10 @@ __global__ void __launch_bounds__(kApplyThreads, 8) k_update_apply(const UpdateA
         return;
     }
     const int first = int(blockIdx.x) - table_ctas, stride = int(gridDim.x) - table_ctas;
-    int item = a.plan.items[first];  // (the list has room for every CTA) in flight with the count
+    int first_tile[kCenPer];  // the codes of the first frames, the item and the count: one trip to memory
+#pragma unroll
+    for (int i = 0; i < kCenPer; ++i) first_tile[i] = a.plan.frame_code[min(int(threadIdx.x) * kCenPer + i, a.B - 1)];
+    int item = a.plan.items[first];  // (the list has room for every CTA)
     const int n_items = a.plan.job_count[3];
     if (first >= n_items) return;
     const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_CENTERS : nullptr);
@@ -764,49 +794,7 @@ __global__ void __launch_bounds__(kApplyThreads, 8) k_update_apply(const UpdateA
             __syncthreads();  // the previous item's readers are done with the list
             item = a.plan.items[it];
         }
-        centre_item(a, item, s_list, s_scan, s_acc);
-    }
-}
-
-// Length and count of every centre the apply kernel moved: a warp per listed pair.
-__global__ void __launch_bounds__(kUpdThreads) k_update_norms(const UpdateArgs a) {
-    chain_wait();
-    chain_release();
-    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_NORMS : nullptr);
-    const int lane = threadIdx.x & 31;
-    const int first = blockIdx.x * (kUpdThreads / kWarp) + (threadIdx.x >> 5);
-    int code = a.plan.jobs[first];  // (the list has room for every warp) in flight with the count
-    const int n_jobs = a.plan.job_count[2];
-    for (int job = first; job < n_jobs; job += gridDim.x * (kUpdThreads / kWarp)) {
-        if (job != first) code = a.plan.jobs[job];
-        const int cls = code & 0xffff, l0 = code >> 16;
-        const int D = a.dims[l0];
-        const float* cen = a.centers[l0] + (size_t)cls * D;
-        float nrm = 0.f;
-        if ((D & 3) == 0) {
-            const float4* c4 = reinterpret_cast<const float4*>(cen);
-            const int D4 = D >> 2;
-            for (int i0 = 0; i0 < D4; i0 += 8 * kWarp) {  // eight pieces per lane in flight
-                float4 v[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = c4[min(i0 + u * kWarp + lane, D4 - 1)];
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    if (i0 + u * kWarp + lane < D4) {
-                        nrm = fmaf(v[u].x, v[u].x, nrm); nrm = fmaf(v[u].y, v[u].y, nrm);
-                        nrm = fmaf(v[u].z, v[u].z, nrm); nrm = fmaf(v[u].w, v[u].w, nrm);
-                    }
-            }
-        } else {
-            for (int i = lane; i < D; i += kWarp) nrm = fmaf(cen[i], cen[i], nrm);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) nrm += __shfl_xor_sync(kFull, nrm, o);
-        if (lane == 0) {
-            a.cnorm[l0][cls] = __fsqrt_rn(nrm);
-            a.m[l0][cls] = a.m_next[(size_t)l0 * a.n + cls];
-            if (a.split_current) a.split_current[l0] = 0;  // the tensor-core scorer's copy of this layer's centres is stale
-        }
+        centre_item(a, item, first_tile, s_list, s_scan, s_acc);
     }
 }
 
@@ -833,7 +821,7 @@ cudaError_t memory_setup() {
     if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_apply);
     if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_plan_one);
     if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_plan);
-    if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_norms);
+
     return e;   // (the single-CTA plan needs at most 32 KB + its statics: below the default limit)
 }
 
@@ -863,12 +851,8 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
     const int centre_ctas = std::min(pairs_max + pairs_max / 2 + kItemBlocksMax, 16 * sm_count);
     const size_t smem = tables ? tables_smem(a.n, rz ? rz->k_max : 0, rz != nullptr) : 0;
     ++*launches;
-    e = launch_chained(k_update_apply, table_ctas + centre_ctas, kApplyThreads, smem, st, a, rz ? *rz : ResizeArgs{},
-                       rz ? 1 : 0, table_ctas);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-    const int norm_ctas = std::max(1, std::min((pairs_max + kUpdThreads / kWarp - 1) / (kUpdThreads / kWarp), 4 * sm_count));
-    return launch_chained(k_update_norms, norm_ctas, kUpdThreads, 0, st, a);
+    return launch_chained(k_update_apply, table_ctas + centre_ctas, kApplyThreads, smem, st, a, rz ? *rz : ResizeArgs{},
+                          rz ? 1 : 0, table_ctas);
 }
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
