@@ -233,6 +233,7 @@ __device__ __forceinline__ unsigned long long key_score(unsigned long long key) 
 __host__ __device__ constexpr size_t refresh_smem(int n, int k_max) { return size_t(pow2_at_least(n)) * 8 + size_t(k_max) * 8; }
 
 constexpr int kCountRankMax = 256;  // up to this many non-zero scores are ranked by counting, more by sorting
+constexpr int kResizeThreadsMax = 1024;  // CTA of the stand-alone refresh when the memory has many classes
 
 // Sum over the block of a 64-bit value; every thread gets the total.  s_part holds >= 32 words.
 __device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v, unsigned long long* s_part) {
@@ -403,7 +404,7 @@ __device__ void refresh_stream(const ResizeArgs& a, int s, unsigned char* dyn, i
         if (sc != 0) s_key[pos++] = refresh_key(sc, c);
     }
     __syncthreads();
-    if (nz <= kCountRankMax) {
+    if (nz <= max(kCountRankMax, 4 * nt)) {  // (a few keys per thread at most: every thread reads all of them)
         // rank = keys larger than this one (keys are distinct); rank r < k_max goes to slot r
         for (int i = tid; i < nz; i += nt) {
             const unsigned long long key = s_key[i];
@@ -444,7 +445,7 @@ __device__ void refresh_stream(const ResizeArgs& a, int s, unsigned char* dyn, i
     if (tid < kWarp) adaptive_size(a, s, s_top, total, tid);
 }
 
-__global__ void __launch_bounds__(kUpdThreads) k_resize(const ResizeArgs a) {
+__global__ void __launch_bounds__(kResizeThreadsMax) k_resize(const ResizeArgs a) {
     extern __shared__ unsigned long long s_dyn[];
     __shared__ int s_scan[33];
     __shared__ unsigned long long s_part[32];
@@ -849,15 +850,23 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
     // more than twice the rows' worth); beyond a few waves of CTAs they stride
     const int pairs_max = std::min(a.B, a.n) * (a.warm_layer >= 0 ? 1 : a.L);
     const int centre_ctas = std::min(pairs_max + pairs_max / 2 + kItemBlocksMax, 16 * sm_count);
-    const size_t smem = tables ? tables_smem(a.n, rz ? rz->k_max : 0, rz != nullptr) : 0;
+    // A memory of many classes is refreshed by a kernel of its own with CTAs of 1024 threads (ranking a thousand
+    // scores is a million comparisons: too much for the 128 threads of a tables CTA); it refreshes every stream,
+    // which gives the streams without a frame in the batch the fast memory they already have.
+    const bool refresh_apart = tables && rz && a.n > 4 * kApplyThreads;
+    const bool refresh_here = tables && rz && !refresh_apart;
+    const size_t smem = tables ? tables_smem(a.n, rz ? rz->k_max : 0, refresh_here) : 0;
     ++*launches;
-    return launch_chained(k_update_apply, table_ctas + centre_ctas, kApplyThreads, smem, st, a, rz ? *rz : ResizeArgs{},
-                          rz ? 1 : 0, table_ctas);
+    e = launch_chained(k_update_apply, table_ctas + centre_ctas, kApplyThreads, smem, st, a, rz ? *rz : ResizeArgs{},
+                       refresh_here ? 1 : 0, table_ctas);
+    if (e != cudaSuccess || !refresh_apart) return e;
+    return launch_resize(*rz, st, launches);
 }
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
     ++*launches;
-    return launch_chained(k_resize, a.S, kUpdThreads, refresh_smem(a.n, a.k_max), st, a);
+    const int threads = a.n > 4 * kApplyThreads ? kResizeThreadsMax : kUpdThreads;
+    return launch_chained(k_resize, a.S, threads, refresh_smem(a.n, a.k_max), st, a);
 }
 
 }  // namespace smtm
