@@ -348,8 +348,18 @@ smtm_status_t smtm_cache_export(smtm_cache_t* cache, void* h_blob, uint64_t byte
 smtm_status_t smtm_cache_import(smtm_cache_t* cache, const void* h_blob, uint64_t bytes);
 
 /* Reads the sticky device status word (synchronises the device): SMTM_OK or
- * the first device-side error recorded since creation. */
+ * the first device-side error recorded since creation (or since it was cleared). */
 smtm_status_t smtm_cache_status(smtm_cache_t* cache);
+
+/* Puts the status word back to SMTM_OK (synchronises the device). */
+smtm_status_t smtm_cache_clear_status(smtm_cache_t* cache);
+
+/* Self-test of the bounded waits: enqueues one small kernel that waits on a shared-memory barrier
+ * nobody will ever arrive on, exactly as the streaming kernels wait for their copies.  The wait
+ * gives up after its limit (about 2^31 clock cycles: a second or so), records SMTM_ERR_TIMEOUT in
+ * the status word and the kernel returns normally: nothing traps, the context stays usable, and
+ * smtm_cache_status reports the timeout.  Costs a second of device time; meant for tests. */
+smtm_status_t smtm_cache_selftest_wait(smtm_cache_t* cache, void* stream);
 
 const char* smtm_status_string(smtm_status_t status);
 

@@ -109,6 +109,8 @@ def load_library():
     lib.smtm_cache_get_profile_device.argtypes = [vp, vp, vp]
     lib.smtm_cache_get_profile_timeline.argtypes = [vp, ctypes.c_int64, vp, vp]
     lib.smtm_cache_status.argtypes = [vp]
+    lib.smtm_cache_clear_status.argtypes = [vp]
+    lib.smtm_cache_selftest_wait.argtypes = [vp, vp]
     lib.smtm_status_string.argtypes = [i32]
     lib.smtm_status_string.restype = ctypes.c_char_p
     for name in declared_symbols():
@@ -390,3 +392,12 @@ def smtm_cache_get_profile_timeline(cache: Cache, step: int):
 
 def smtm_cache_status(cache: Cache) -> int:
     return int(load_library().smtm_cache_status(cache.handle))
+
+
+def smtm_cache_clear_status(cache: Cache) -> None:
+    _check(load_library().smtm_cache_clear_status(cache.handle), "smtm_cache_clear_status")
+
+
+def smtm_cache_selftest_wait(cache: Cache, stream=None) -> None:
+    """Enqueues a kernel whose bounded wait runs out (about a second); the status word then reads SMTM_ERR_TIMEOUT."""
+    _check(load_library().smtm_cache_selftest_wait(cache.handle, _stream(stream)), "smtm_cache_selftest_wait")

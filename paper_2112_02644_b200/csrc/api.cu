@@ -981,6 +981,19 @@ smtm_status_t smtm_cache_status(smtm_cache_t* c) {
     return static_cast<smtm_status_t>(v);
 }
 
+smtm_status_t smtm_cache_clear_status(smtm_cache_t* c) {
+    if (!c) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(cudaDeviceSynchronize());
+    SMTM_CUDA(cudaMemset(c->d_status, 0, sizeof(int)));
+    return SMTM_OK;
+}
+
+smtm_status_t smtm_cache_selftest_wait(smtm_cache_t* c, void* stream) {
+    if (!c) return SMTM_ERR_INVALID_ARG;
+    SMTM_CUDA(launch_wait_selftest(c->d_status, static_cast<cudaStream_t>(stream), &c->launches));
+    return SMTM_OK;
+}
+
 const char* smtm_status_string(smtm_status_t s) {
     switch (s) {
         case SMTM_OK: return "ok";

@@ -139,6 +139,10 @@ __device__ __forceinline__ void bulk_load_hint(void* dst_smem, const void* src_g
         : "memory");
 }
 
+// 16 bytes of a feature map by a plain load: read once, so marked for early eviction from L2 (the data the
+// kernels keep coming back to should stay there).
+__device__ __forceinline__ uint4 load_once(const uint4* p) { return __ldcs(p); }
+
 // ---- element widening -----------------------------------------------------------------
 
 struct F32 {

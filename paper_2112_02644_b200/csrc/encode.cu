@@ -730,7 +730,7 @@ __global__ void __launch_bounds__(kLightThreads) k_pool_sparse(const LightParams
         for (int v0 = 0; v0 < vectors; v0 += 8 * kLightThreads) {  // eight loads per thread in flight
             uint4 r[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) r[u] = __ldg(src + min(v0 + u * kLightThreads + tid, vectors - 1));
+            for (int u = 0; u < 8; ++u) r[u] = load_once(src + min(v0 + u * kLightThreads + tid, vectors - 1));
 #pragma unroll
             for (int u = 0; u < 8; ++u)
                 if (v0 + u * kLightThreads + tid < vectors) dst[v0 + u * kLightThreads + tid] = r[u];
@@ -837,7 +837,7 @@ __global__ void __launch_bounds__(kLightThreads) k_lookup_sparse(const SparsePar
         uint4* dst = reinterpret_cast<uint4*>(stage);
         uint4 r[kLoads];
 #pragma unroll
-        for (int u = 0; u < kLoads; ++u) r[u] = __ldg(src + min(u * kLightThreads + tid, vectors - 1));
+        for (int u = 0; u < kLoads; ++u) r[u] = load_once(src + min(u * kLightThreads + tid, vectors - 1));
         // the frame's fast memory: its size and this warp's classes (slot j = warp + 4 i), in flight with the chunk
         const int32_t* mem = a.members + (size_t)max(sid, 0) * a.k_max;
         const int k = sid < 0 ? 0 : min(a.k[sid], kFusedMaxK);
@@ -971,10 +971,10 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_encode_nhwc(const uint8_t* __r
                 const uint4* col = f + cg0 + cg;
                 int px = ph;
                 for (; px + 3 * phases < HW; px += 4 * phases) {
-                    const uint4 v0 = __ldg(col + (long long)px * CG);
-                    const uint4 v1 = __ldg(col + (long long)(px + phases) * CG);
-                    const uint4 v2 = __ldg(col + (long long)(px + 2 * phases) * CG);
-                    const uint4 v3 = __ldg(col + (long long)(px + 3 * phases) * CG);
+                    const uint4 v0 = load_once(col + (long long)px * CG);
+                    const uint4 v1 = load_once(col + (long long)(px + phases) * CG);
+                    const uint4 v2 = load_once(col + (long long)(px + 2 * phases) * CG);
+                    const uint4 v3 = load_once(col + (long long)(px + 3 * phases) * CG);
 #pragma unroll
                     for (int j = 0; j < V; ++j) acc[j] += E::at(v0, j);
 #pragma unroll
@@ -985,7 +985,7 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_encode_nhwc(const uint8_t* __r
                     for (int j = 0; j < V; ++j) acc[j] += E::at(v3, j);
                 }
                 for (; px < HW; px += phases) {
-                    const uint4 v = __ldg(col + (long long)px * CG);
+                    const uint4 v = load_once(col + (long long)px * CG);
 #pragma unroll
                     for (int j = 0; j < V; ++j) acc[j] += E::at(v, j);
                 }
@@ -1012,9 +1012,11 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_encode_nhwc(const uint8_t* __r
 // flight (a frame is a few dozen KB: the CTA's time is the number of trips to memory it makes); the
 // phases are added in ascending order through shared memory.  Frames that have exited cost a CTA that
 // leaves at once.
+constexpr int kThreadsNhwcLookup = 512;  // more threads, fewer trips to memory per thread: a frame is one CTA's
+
 template <class E>
-__global__ void __launch_bounds__(kThreadsNhwc) k_lookup_nhwc(const uint8_t* __restrict__ x, int C, int HW, float inv_hw,
-                                                              float* __restrict__ sv_out, const LookupArgs a) {
+__global__ void __launch_bounds__(kThreadsNhwcLookup) k_lookup_nhwc(const uint8_t* __restrict__ x, int C, int HW, float inv_hw,
+                                                                    float* __restrict__ sv_out, const LookupArgs a) {
     extern __shared__ float nhwc_smem[];  // sv [C] | s_cur [k_max] | s_acc [k_max] | part [phases][cgs * V]
     __shared__ float scratch[32];
     float* sv_s = nhwc_smem;
@@ -1027,13 +1029,15 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_lookup_nhwc(const uint8_t* __r
     const int b = blockIdx.x;
     const int sid_raw = a.stream_id ? a.stream_id[b] : 0;  // in flight with the exit flag
     if (!a.fresh && a.done[b]) return;
+    const SlotPrefetch pf = prefetch_slots(a, sid_raw);    // in flight with the map
     constexpr int V = E::kPerVec;
+    constexpr int T = kThreadsNhwcLookup;
     const int CG = C / V;  // 16-byte vectors per pixel
     const uint4* f = reinterpret_cast<const uint4*>(x + (long long)b * HW * C * E::kSize);
     float nrm = 0.f;
-    for (int cg0 = 0; cg0 < CG; cg0 += kThreadsNhwc) {
-        const int cgs = min(CG - cg0, kThreadsNhwc);  // column groups handled in this sweep
-        const int phases = kThreadsNhwc / cgs;
+    for (int cg0 = 0; cg0 < CG; cg0 += T) {
+        const int cgs = min(CG - cg0, T);  // column groups handled in this sweep
+        const int phases = T / cgs;
         const int ph = threadIdx.x / cgs, cg = threadIdx.x - ph * cgs;
         float acc[V];
 #pragma unroll
@@ -1043,7 +1047,7 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_lookup_nhwc(const uint8_t* __r
             for (int px = ph; px < HW; px += 8 * phases) {
                 uint4 v[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = __ldg(col + (long long)min(px + u * phases, HW - 1) * CG);
+                for (int u = 0; u < 8; ++u) v[u] = load_once(col + (long long)min(px + u * phases, HW - 1) * CG);
 #pragma unroll
                 for (int u = 0; u < 8; ++u)
                     if (px + u * phases < HW) {
@@ -1056,7 +1060,7 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_lookup_nhwc(const uint8_t* __r
             for (int j = 0; j < V; ++j) dst[j] = acc[j];
         }
         __syncthreads();
-        for (int c = threadIdx.x; c < cgs * V; c += kThreadsNhwc) {
+        for (int c = threadIdx.x; c < cgs * V; c += T) {
             float s = 0.f;
             for (int q = 0; q < phases; ++q) s += part[size_t(q) * cgs * V + c];
             s *= inv_hw;
@@ -1067,7 +1071,7 @@ __global__ void __launch_bounds__(kThreadsNhwc) k_lookup_nhwc(const uint8_t* __r
         __syncthreads();
     }
     nrm = block_sum(nrm, scratch);  // also orders the shared writes above
-    score_frame(a, b, sid_raw, sv_s, nrm, s_cur, s_acc);
+    score_frame(a, b, pf, sv_s, nrm, s_cur, s_acc);
 }
 
 // ---- any shape: one thread per (frame, channel) ---------------------------------------------
@@ -1367,15 +1371,15 @@ cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm
     if (e.layout == SMTM_NHWC) {
         const int V = e.dtype == SMTM_F32 ? 4 : 8;
         if (e.C % V || e.C > 8192) return cudaSuccess;
-        const int cgs = std::min(e.C / V, kThreadsNhwc);
-        const size_t smem = (size_t(e.C) + 2 * size_t(a.k_max) + size_t(kThreadsNhwc / cgs) * cgs * V) * sizeof(float);
+        const int cgs = std::min(e.C / V, kThreadsNhwcLookup);
+        const size_t smem = (size_t(e.C) + 2 * size_t(a.k_max) + size_t(kThreadsNhwcLookup / cgs) * cgs * V) * sizeof(float);
         const float inv_hw = 1.0f / float(e.H * e.W);
         const uint8_t* x = static_cast<const uint8_t*>(e.x);
         cudaError_t err = cudaSuccess;
         if (timing) record_timing(timing[0], st);
-        if (e.dtype == SMTM_F32) err = launch_chained(k_lookup_nhwc<F32>, e.B, kThreadsNhwc, smem, st, x, e.C, e.H * e.W, inv_hw, e.sv, a);
-        else if (e.dtype == SMTM_F16) err = launch_chained(k_lookup_nhwc<F16>, e.B, kThreadsNhwc, smem, st, x, e.C, e.H * e.W, inv_hw, e.sv, a);
-        else err = launch_chained(k_lookup_nhwc<BF16>, e.B, kThreadsNhwc, smem, st, x, e.C, e.H * e.W, inv_hw, e.sv, a);
+        if (e.dtype == SMTM_F32) err = launch_chained(k_lookup_nhwc<F32>, e.B, kThreadsNhwcLookup, smem, st, x, e.C, e.H * e.W, inv_hw, e.sv, a);
+        else if (e.dtype == SMTM_F16) err = launch_chained(k_lookup_nhwc<F16>, e.B, kThreadsNhwcLookup, smem, st, x, e.C, e.H * e.W, inv_hw, e.sv, a);
+        else err = launch_chained(k_lookup_nhwc<BF16>, e.B, kThreadsNhwcLookup, smem, st, x, e.C, e.H * e.W, inv_hw, e.sv, a);
         if (timing) record_timing(timing[1], st);
         ++*launches;
         *handled = true;

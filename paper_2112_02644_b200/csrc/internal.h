@@ -168,6 +168,8 @@ size_t dense_centers_split_bytes(int n, int D);
 // (nullptr, or [B][n]: the second half of the vector length, added to the first).
 cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, int* split_current,
                                 cudaStream_t st, int64_t* launches);
+// One warp that waits, bounded, on a barrier nobody arrives on (the self-test of the time-out path).
+cudaError_t launch_wait_selftest(int* status, cudaStream_t st, int64_t* launches);
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,
                                cudaStream_t st, int64_t* launches);
 

@@ -33,6 +33,7 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
     const int sid_raw = a.stream_id ? a.stream_id[b] : 0;  // in flight with the exit flag
     if (!a.fresh && a.done[b]) return;  // (a batch that starts here: every frame is in, whatever the flags hold)
     const int tid = threadIdx.x, nthreads = blockDim.x;
+    const SlotPrefetch pf = prefetch_slots(a, sid_raw);  // in flight with the semantic vector
     const float* row = a.sv + (size_t)b * a.D;
     float nrm = 0.f;
     for (int d = tid; d < a.D; d += nthreads) {
@@ -41,7 +42,7 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
         nrm = fmaf(v, v, nrm);
     }
     nrm = block_sum(nrm, scratch);  // also orders the shared writes above
-    score_frame(a, b, sid_raw, sv, nrm, s_cur, s_acc);
+    score_frame(a, b, pf, sv, nrm, s_cur, s_acc);
 }
 
 // Finishing kernel of the tensor-core path: one CTA per frame turns the frame's row of dot
@@ -154,7 +155,24 @@ __global__ void k_batch_reset(float* __restrict__ sa, uint8_t* __restrict__ done
     }
 }
 
+// The wait of the streaming kernels (mbar_wait_bounded), on a barrier that never completes its phase.
+__global__ void k_wait_selftest(int* status) {
+    __shared__ uint64_t bar;
+    chain_wait();
+    chain_release();
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_init_fence();
+        mbar_wait_bounded(&bar, 0, status);  // gives up after its limit and records the time-out
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_wait_selftest(int* status, cudaStream_t st, int64_t* launches) {
+    ++*launches;
+    return launch_chained(k_wait_selftest, 1, kWarp, 0, st, status);
+}
 
 cudaError_t lookup_setup() {
     cudaError_t e = allow_max_dynamic_smem(k_score_exit);

@@ -168,20 +168,33 @@ __device__ __forceinline__ void decide_from_top2(const LookupArgs& a, int b, con
 }
 
 // Scores frame b against the members of its fast memory and decides, by a whole CTA (any whole number of
-// warps): sid_raw is the frame's stream id as read from memory (the caller fetches it along with its own first
-// loads), sv the frame's semantic vector in shared memory (already visible to every thread), nrm its squared
+// warps): pf is what prefetch_slots returned for the frame's stream id, sv the frame's semantic vector in shared memory (already visible to every thread), nrm its squared
 // length; s_cur / s_acc hold k_max floats each.  Each warp takes fast-memory slots round-robin and reads the
 // member's centre (L2-resident) with 128-bit loads; lanes keep four independent fp32 accumulators and combine
 // with xor-shuffles, so every dot product has a fixed evaluation order.  Warp 0 then selects the two best.
 // The kernel's time is the number of dependent trips to memory: the size of the fast memory and the warp's
 // first class come in one trip, and a slot's centre, its length, its carry and the next slot's class in one more.
-__device__ __forceinline__ void score_frame(const LookupArgs& a, int b, int sid_raw, const float* sv, float nrm,
+// What score_frame needs of the frame's fast memory before it can fetch a centre: its size and this warp's
+// first class.  Fetched early (the loads only need the stream id), so that they are in flight with the
+// caller's own loads (the semantic vector, or the map that is being pooled).
+struct SlotPrefetch {
+    int sid, k, cls;
+};
+__device__ __forceinline__ SlotPrefetch prefetch_slots(const LookupArgs& a, int sid_raw) {
+    SlotPrefetch pf;
+    pf.sid = stream_checked(a, sid_raw);
+    const int32_t* mem = a.members + (size_t)max(pf.sid, 0) * a.k_max;
+    pf.cls = mem[min(int(threadIdx.x >> 5), a.k_max - 1)];  // unconditional: in flight with the size
+    pf.k = pf.sid < 0 ? 0 : a.k[pf.sid];                     // a stream id outside the cache: nothing to score against
+    return pf;
+}
+
+__device__ __forceinline__ void score_frame(const LookupArgs& a, int b, const SlotPrefetch& pf, const float* sv, float nrm,
                                             float* s_cur, float* s_acc) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x, nw = nthreads / kWarp;
-    const int sid = stream_checked(a, sid_raw);
-    const int32_t* mem = a.members + (size_t)max(sid, 0) * a.k_max;
-    int cls_next = mem[min(warp, a.k_max - 1)];  // unconditional: in flight with the size
-    const int k = sid < 0 ? 0 : a.k[sid];        // a stream id outside the cache: nothing to score against
+    const int32_t* mem = a.members + (size_t)max(pf.sid, 0) * a.k_max;
+    int cls_next = pf.cls;
+    const int k = pf.k;
     const float weight = float(1u << a.layer);   // 2^(l-1) with l = layer + 1
     const int D4 = (a.D & 3) ? 0 : a.D >> 2;     // 128-bit loads need rows that are multiples of 16 bytes
     const float4* v4 = reinterpret_cast<const float4*>(sv);

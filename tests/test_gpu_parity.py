@@ -669,3 +669,28 @@ def test_export_then_import_puts_the_cache_back_bit_for_bit():
     assert e.value.status == 1 and same(state(b), after)          # nothing was changed
     for c in (a, b, other):
         smtm.smtm_cache_destroy(c)
+
+
+def test_a_wait_that_runs_out_sets_the_status_word_and_leaves_the_context_usable():
+    # The streaming kernels wait for their copies with a limit (about a second); a wait that runs out records
+    # SMTM_ERR_TIMEOUT in the sticky status word and the kernel returns.  The self-test waits on a barrier that
+    # nobody arrives on: nothing traps or hangs, the status reads 8, and after clearing it the same cache
+    # serves a step that matches the oracle.
+    from harness import Report, compare_state, make_pair, step_pair
+
+    w = si.C5.scaled(name="after_timeout", B=24, S=24, T=2)
+    cache, mem = make_pair(w)
+    assert smtm.smtm_cache_status(cache) == 0
+    smtm.smtm_cache_selftest_wait(cache)
+    assert smtm.smtm_cache_status(cache) == 8            # SMTM_ERR_TIMEOUT
+    assert smtm.smtm_status_string(8) == "device-side wait timed out"
+    assert smtm.smtm_cache_status(cache) == 8            # sticky
+    smtm.smtm_cache_clear_status(cache)
+    assert smtm.smtm_cache_status(cache) == 0
+    gb = smtm.Batch(cache, w.B, stream_id=si.stream_ids(w))
+    rep = Report()
+    labs = si.labels(w)
+    for t in range(w.T):
+        step_pair(w, cache, mem, gb, labs[t], t, rep)
+    compare_state(w, cache, mem, rep)                    # also asserts that the status word is clear
+    smtm.smtm_cache_destroy(cache)
