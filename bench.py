@@ -276,9 +276,15 @@ class OracleRun:
 
 # --------------------------------------------------------------------------- the CUDA arm
 
+def maps_ready(w) -> bool:
+    return w.T > 1 or w.k_max > 64
+
+
 def make_cache(smtm, w, cents, counts):
     # the streaming workload keeps its maps resident and alternates two carries: the library may pipeline its steps
-    flags = (smtm.FLAG_FORGET_FT if w.forgetting else 0) | (smtm.FLAG_MAPS_READY if w.T > 1 else 0)
+    # (so does the workload with the large fast memory; the others are served by the fused kernels, which the flag
+    # would take them off)
+    flags = (smtm.FLAG_FORGET_FT if w.forgetting else 0) | (smtm.FLAG_MAPS_READY if maps_ready(w) else 0)
     return smtm.smtm_cache_create(w.n, w.dims, [w.tau] * w.L, cents, counts, n_streams=w.S, k_init=w.k_init,
                                   k_min=w.k_min, k_max=w.k_max, window_W=w.window_W, max_batch=w.B, flags=flags)
 
@@ -421,9 +427,10 @@ def measure(smtm, w, K, W, local_rank, world, verify_steps=0, graph_steps=32):
     out["event_n"] = [int(n) for _, n in ev]
     dev_total, dev_cnt = smtm.smtm_cache_get_profile_device(cache)
     names = ["lookup_layer%d" % l for l in range(w.L)] + ["score_layer%d" % l for l in range(w.L)] + \
-        ["update_plan", "update_centers", "update_tables", "score_tc"]
+        ["update_plan", "update_centers", "update_tables", "score_tc", "finish_dense", "refresh"]
     idx = list(range(w.L)) + [smtm.PROF_SCORE + l for l in range(w.L)] + \
-        [smtm.PROF_PLAN, smtm.PROF_CENTERS, smtm.PROF_TABLES, smtm.PROF_SCORE_TC]
+        [smtm.PROF_PLAN, smtm.PROF_CENTERS, smtm.PROF_TABLES, smtm.PROF_SCORE_TC, smtm.PROF_FINISH_DENSE,
+         smtm.PROF_REFRESH]
     out["device_us"] = {nm: (float(dev_total[i]) / int(dev_cnt[i]) * 1e3 if dev_cnt[i] else None) for nm, i in zip(names, idx)}
     out["device_n"] = int(dev_cnt[0])
     # the first layer's pooling kernel alone on the device (smtm_encode over the resident maps, back to back):
@@ -504,7 +511,7 @@ def run_ours(args):
                        "l2_policy": "distinct maps per step, %.0f MB per step (L2 is 126 MB)" % (m["res"].step_bytes / 1e6),
                        "state": "the memory is put back to its state after step W-1 (smtm_cache_import) right before the timed region",
                        "sharding": "streams across GPUs, no collective",
-                       "launch": "CUDA graphs of %d steps (per step: %d lookups, update+refresh), chained launches, SMTM_FLAG_MAPS_READY with two alternating carries" % (m["G"], w.L)},
+                       "launch": "CUDA graphs of %d steps (per step: %d lookups, update+refresh), chained launches%s" % (m["G"], w.L, ", SMTM_FLAG_MAPS_READY with two alternating carries" if maps_ready(w) else "")},
             "e2e": e2e,
             "gpu_launches": m["launches"],
             "clocks": m["clocks"],
@@ -524,7 +531,7 @@ def run_ours(args):
             "step_kernels_device_clock_us": m["device_us"],
             "exit_histogram": {"per_layer": m["exits"], "none": K * w.B - sum(m["exits"])},
             "near_threshold_lookups": m["near"],
-            "routes": dict(zip(("fused", "dense", "plain", "pipelined"), m["routes"])),
+            "routes": dict(zip(("fused", "dense", "plain", "pipelined", "pipelined_dense"), m["routes"])),
             "device_status": m["status"],
         }
         # bytes the whole step had to move (maps of the frames still in at each layer + their SV rows) over the step time
@@ -582,7 +589,7 @@ def other_workload(smtm, w, peak, tc_peak, with_oracle):
     out = {"workload": w.name, "steps": K, "warmup": W, "ms_per_step": ms, "frames_per_s": w.B / (ms * 1e-3),
            "dominant_kernel_us": us_dev if us_dev else us_ev, "dominant_kernel_us_cuda_events": us_ev,
            "frac": (ach_dev if ach_dev else ach) / peak if (ach_dev or ach) else None,
-           "bytes_per_launch": nbytes, "routes": dict(zip(("fused", "dense", "plain", "pipelined"), m["routes"])),
+           "bytes_per_launch": nbytes, "routes": dict(zip(("fused", "dense", "plain", "pipelined", "pipelined_dense"), m["routes"])),
            "exit_histogram": {"per_layer": m["exits"], "none": K * w.B - sum(m["exits"])},
            "near_threshold_lookups": m["near"], "step_kernels_device_clock_us": m["device_us"],
            "distinct_steps_resident": m["R"], "device_status": m["status"]}

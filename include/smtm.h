@@ -215,12 +215,10 @@ smtm_status_t smtm_lookup_exit_static(smtm_cache_t* cache, int32_t layer, const 
  * class j and layer l0 the frames with label j and stop layer >= l0 are folded
  * into the centre in ascending b:  SC = (SC m + sum SV) / (m + q), m += q
  * (summed as four interleaved partial sums added in a fixed order).
- * The tables are updated on a stream of the cache's own that is forked from
- * `stream` and joined back to it before the call returns control of the stream,
- * so that they run beside the centres; to the caller everything is ordered on
- * `stream` as usual, and inside a stream capture the fork and join become part
- * of the captured graph.  The call's bookkeeping lives on the device: a captured
- * update may be replayed any number of times. */
+ * Tables and centres are kept by different CTAs of one kernel, after a small
+ * kernel that plans the work; everything is enqueued on `stream`.  The call's
+ * bookkeeping lives on the device: a captured update may be replayed any number
+ * of times. */
 smtm_status_t smtm_cache_update(smtm_cache_t* cache, const smtm_batch_t* batch,
                                 const int32_t* d_fallback_label, void* stream);
 
@@ -290,9 +288,11 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
  * of the other routes), for the scoring kernel of layer i where pooling and
  * scoring are separate kernels (SMTM_PROF_SCORE + i), for the update (the plan
  * kernel SMTM_PROF_PLAN; the CTAs of the apply kernel that fold centres,
- * _CENTERS, and those that keep the tables, _TABLES) and for the tensor-core scorer of the dense route
- * (SMTM_PROF_SCORE_TC; with several dense layers in a step, from the first
- * one's begin to the last one's end).  This
+ * _CENTERS, and those that keep the tables, _TABLES; the refresh of the fast
+ * memories where it is a kernel of its own, _REFRESH) and for the dense route
+ * (the tensor-core scorer SMTM_PROF_SCORE_TC and the decision kernel after it,
+ * _FINISH_DENSE; with several dense layers in a step, from the first one's
+ * begin to the last one's end).  This
  * leaves out what the event nodes add around a kernel.  Only the most recent
  * run of each profiled step is kept.  smtm_cache_get_profile_timeline gives the
  * two stamps themselves for the step-th profiled step (counted from 0;
@@ -304,6 +304,7 @@ smtm_status_t smtm_cache_get_counters(smtm_cache_t* cache, int64_t* h_out /*[SMT
 enum {
     SMTM_PROF_SCORE = SMTM_MAX_LAYERS,  /* + layer: the scoring kernel of a layer whose pooling is a kernel of its own */
     SMTM_PROF_PLAN = 2 * SMTM_MAX_LAYERS, SMTM_PROF_CENTERS, SMTM_PROF_TABLES, SMTM_PROF_SCORE_TC,
+    SMTM_PROF_FINISH_DENSE, SMTM_PROF_REFRESH,
     SMTM_PROF_KERNELS
 };
 smtm_status_t smtm_cache_profile(smtm_cache_t* cache, int32_t max_lookups, int32_t every);
@@ -318,7 +319,7 @@ smtm_status_t smtm_cache_get_profile_timeline(smtm_cache_t* cache, int64_t step,
 smtm_status_t smtm_cache_get_launches(smtm_cache_t* cache, int64_t* h_out);
 
 /* How many lookups (smtm_lookup_exit, _begin, _static and the lookups inside smtm_step_host) each
- * route has served so far.  Eq. 1 is evaluated on one of three routes, chosen from the shape:
+ * route has served so far.  The route is chosen from the shape and the cache's flags:
  *   SMTM_ROUTE_FUSED  pooling, Eq. 1, Eq. 3, Eq. 4 and the exit rule in one streaming kernel
  *                     (fast memories of at most 64 entries; NCHW shapes and NHWC shapes whose
  *                     pixel rows are multiples of 16 bytes);
@@ -328,8 +329,14 @@ smtm_status_t smtm_cache_get_launches(smtm_cache_t* cache, int64_t* h_out);
  *   SMTM_ROUTE_PIPELINED  on a cache created with SMTM_FLAG_MAPS_READY (small fast memories, NCHW shapes
  *                     the streaming kernels serve): the pooling of a step's first layer runs on a stream of
  *                     the cache's own, under the previous step's later layers and update; scoring follows
- *                     on the caller's stream; later layers are pooled and scored by small CTAs. */
-enum { SMTM_ROUTE_FUSED = 0, SMTM_ROUTE_DENSE = 1, SMTM_ROUTE_PLAIN = 2, SMTM_ROUTE_PIPELINED = 3, SMTM_ROUTE_COUNT = 4 };
+ *                     on the caller's stream; later layers are pooled and scored by small CTAs;
+ *   SMTM_ROUTE_PIPELINED_DENSE  the same for fast memories above 64 entries, first lookup of a batch only:
+ *                     the pooling runs on the cache's stream beside the previous step's decision kernel and
+ *                     update, the tensor-core kernel and the decision kernel follow on the caller's stream. */
+enum {
+    SMTM_ROUTE_FUSED = 0, SMTM_ROUTE_DENSE = 1, SMTM_ROUTE_PLAIN = 2, SMTM_ROUTE_PIPELINED = 3,
+    SMTM_ROUTE_PIPELINED_DENSE = 4, SMTM_ROUTE_COUNT = 5
+};
 smtm_status_t smtm_cache_get_routes(smtm_cache_t* cache, int64_t* h_out /*[SMTM_ROUTE_COUNT]*/);
 
 /* Snapshot of the memory of Sec. 6 (the paper keeps it for the life of the application; a host copy

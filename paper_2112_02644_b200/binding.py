@@ -327,7 +327,7 @@ def smtm_cache_get_launches(cache: Cache) -> int:
     return int(out[0])
 
 
-ROUTE_FUSED, ROUTE_DENSE, ROUTE_PLAIN, ROUTE_PIPELINED, ROUTE_COUNT = 0, 1, 2, 3, 4
+ROUTE_FUSED, ROUTE_DENSE, ROUTE_PLAIN, ROUTE_PIPELINED, ROUTE_PIPELINED_DENSE, ROUTE_COUNT = 0, 1, 2, 3, 4, 5
 
 
 def smtm_cache_get_routes(cache: Cache) -> np.ndarray:
@@ -366,8 +366,8 @@ def smtm_cache_get_profile(cache: Cache, layer: int):
 
 
 PROF_SCORE = MAX_LAYERS   # + layer: the scoring kernel of a layer whose pooling is a kernel of its own
-PROF_PLAN, PROF_CENTERS, PROF_TABLES, PROF_SCORE_TC, PROF_KERNELS = (
-    2 * MAX_LAYERS, 2 * MAX_LAYERS + 1, 2 * MAX_LAYERS + 2, 2 * MAX_LAYERS + 3, 2 * MAX_LAYERS + 4)
+PROF_PLAN, PROF_CENTERS, PROF_TABLES, PROF_SCORE_TC, PROF_FINISH_DENSE, PROF_REFRESH, PROF_KERNELS = (
+    2 * MAX_LAYERS + i for i in range(7))
 
 
 def smtm_cache_get_profile_device(cache: Cache):

@@ -27,7 +27,6 @@ struct smtm_cache {
     float* d_warm_sv;   // scratch of smtm_cache_warmup: [max_batch][C_max] semantic vectors (allocated on first use)
     void* d_dense;      // scratch of the tensor-core scorer (fast memories above 64 entries), else NULL
     void* d_cen_split[SMTM_MAX_LAYERS];   // bf16 heads and tails of the centres, per layer (same condition)
-    int* d_split_current;  // [L] device flags: the centres' split of a layer is current (same condition as d_dense)
     int d_max;          // largest C_l
     int32_t* d_plan;    // scratch of the update: final label and stop layer of every frame, [max_batch]
     unsigned long long* d_tags;  // scratch of the update: stamps of (layer, class), [L][n]
@@ -35,6 +34,10 @@ struct smtm_cache {
     cudaStream_t pool_stream;
     cudaEvent_t ev_fork, ev_pool;       // the caller's stream -> pool stream, and back
     cudaEvent_t ev_mark[2];             // where the caller's stream stood at the last two first lookups (they alternate)
+    cudaEvent_t ev_scored;              // dense scoring of the pipelined route: the tensor-core kernel of the last first lookup is done
+    unsigned long long scored_capture;  // the capture ev_scored was recorded in (0 = none)
+    bool scored_valid;
+    int split_which;                    // which of the two split buffers the batch under way uses (0 unless pipelined)
     unsigned long long mark_capture[2]; // the stream capture each was recorded in (0 = none)
     bool mark_valid[2];
     int mark_next;                      // which of the two the next first lookup records
@@ -121,12 +124,12 @@ void free_all(smtm_cache* c) {
     cudaFree(c->d_plan);
     cudaFree(c->d_warm_sv);
     cudaFree(c->d_dense);
-    cudaFree(c->d_split_current);
     cudaFree(c->d_tags);
     cudaFree(c->d_epoch);
     if (c->pool_stream) cudaStreamDestroy(c->pool_stream);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_pool) cudaEventDestroy(c->ev_pool);
+    if (c->ev_scored) cudaEventDestroy(c->ev_scored);
     for (cudaEvent_t e : c->ev_mark)
         if (e) cudaEventDestroy(e);
     cudaFree(c->d_jobs);
@@ -158,6 +161,16 @@ smtm_status_t check_batch(const smtm_cache* c, const smtm_batch_t* b) {
     if (b->B < 1 || b->B > c->max_batch) return SMTM_ERR_SHAPE;
     if (!b->d_sa || !b->d_done || !b->d_exit_layer || !b->d_pred) return SMTM_ERR_INVALID_ARG;
     return SMTM_OK;
+}
+
+// The tensor-core scorer reads the centres as bf16 heads and tails.  That copy is made here whenever the centres of
+// a layer are set as a whole (creation, import); Eq. 7's kernel keeps it in step with every centre it moves.
+// Layers the scorer does not serve (vectors that are not a multiple of eight long) have none.
+bool has_centre_split(const smtm_cache* c, int l) { return c->d_cen_split[l] != nullptr && c->dims[l] % 8 == 0; }
+
+cudaError_t split_centres(smtm_cache* c, int l, cudaStream_t st) {
+    if (!has_centre_split(c, l)) return cudaSuccess;
+    return launch_centers_split(c->d_centers[l], c->n, c->dims[l], c->d_cen_split[l], st, &c->launches);
 }
 
 EncodeArgs encode_args(const smtm_cache* c, const smtm_fmap_t* f, const uint8_t* skip, float* sv) {
@@ -202,8 +215,14 @@ cudaError_t capture_of(cudaStream_t st, unsigned long long* id) {
 // stream joins the capture through these events; a mark recorded outside the capture under way is not waited for
 // (the launch of the graph orders the graph after it), and a pool stream that is not part of the capture yet
 // is forked from the caller's stream where it stands.
+//
+// With a large fast memory (dense) the scoring is the tensor-core kernel and the decision kernel after it.  The
+// CTAs of the tensor-core kernel need most of an SM's shared memory and cannot sit beside a pooling CTA, so the
+// next batch's pooling is also ordered after that kernel (else whichever of the two came second would wait for
+// the other to leave the SMs, and the step's latency-bound kernels with it); it runs beside the decision kernel
+// and the update.  The vectors' bf16 split alternates between two buffers like the batches do.
 smtm_status_t pooled_first_lookup(smtm_cache* c, const EncodeArgs& e, const LookupArgs& a, cudaStream_t st,
-                                  const cudaEvent_t* timing, bool profiled_step) {
+                                  const cudaEvent_t* timing, bool profiled_step, bool dense) {
     unsigned long long cap = 0, pool_cap = 0;
     SMTM_CUDA(capture_of(st, &cap));
     SMTM_CUDA(capture_of(c->pool_stream, &pool_cap));
@@ -215,6 +234,8 @@ smtm_status_t pooled_first_lookup(smtm_cache* c, const EncodeArgs& e, const Look
         SMTM_CUDA(cudaEventRecord(c->ev_fork, st));
         SMTM_CUDA(cudaStreamWaitEvent(c->pool_stream, c->ev_fork, 0));
     }
+    if (dense && c->scored_valid && c->scored_capture == cap && wait_prev)
+        SMTM_CUDA(cudaStreamWaitEvent(c->pool_stream, c->ev_scored, 0));
     SMTM_CUDA(cudaEventRecord(c->ev_mark[cur], st));
     c->mark_capture[cur] = cap;
     c->mark_valid[cur] = true;
@@ -226,12 +247,29 @@ smtm_status_t pooled_first_lookup(smtm_cache* c, const EncodeArgs& e, const Look
     ep.ring_in_flight = kPipelinedInFlight;
     if (profiled_step && a.layer == 0 && ep.clock)  // the caller's stream clears the step's other stamps at a time of its own
         SMTM_CUDA(cudaMemsetAsync(ep.clock, 0, 2 * sizeof(unsigned long long), c->pool_stream));
+    bool sv_split = false;
+    if (dense) {
+        // this batch's buffer, for its later layers too (the next batch's pooling writes the other one meanwhile)
+        c->split_which = cur;
+        dense_sv_split(c->d_dense, c->max_batch, c->d_max, cur, &ep.sv_hi, &ep.sv_lo);
+    }
     if (timing) SMTM_CUDA(record_timing(timing[0], c->pool_stream));
-    SMTM_CUDA(launch_encode(ep, c->sm_count, c->pool_stream, &c->launches));
+    SMTM_CUDA(launch_encode(ep, c->sm_count, c->pool_stream, &c->launches, dense ? &sv_split : nullptr));
     if (timing) SMTM_CUDA(record_timing(timing[1], c->pool_stream));
     SMTM_CUDA(cudaEventRecord(c->ev_pool, c->pool_stream));
-    SMTM_CUDA(cudaStreamWaitEvent(st, c->ev_pool, 0));
-    SMTM_CUDA(launch_score_exit(a, st, &c->launches, kPipelinedScoreThreads));
+    if (!dense) {
+        SMTM_CUDA(cudaStreamWaitEvent(st, c->ev_pool, 0));
+        SMTM_CUDA(launch_score_exit(a, st, &c->launches, kPipelinedScoreThreads));
+        return SMTM_OK;
+    }
+    float *dots = nullptr, *dots2 = nullptr;
+    SMTM_CUDA(launch_dense_dots(a.sv, nullptr, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max, cur, sv_split,
+                                c->ev_pool, c->d_cen_split[a.layer], &dots, &dots2, c->d_status,
+                                a.clock ? a.clock + 2 * SMTM_PROF_SCORE_TC : nullptr, st, &c->launches));
+    SMTM_CUDA(cudaEventRecord(c->ev_scored, st));
+    c->scored_capture = cap;
+    c->scored_valid = true;
+    SMTM_CUDA(launch_finish_dense(a, dots, dots2, st, &c->launches));
     return SMTM_OK;
 }
 
@@ -269,13 +307,16 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     // The pipelined route: a cache whose caller keeps the maps resident and alternates its carries
     // (SMTM_FLAG_MAPS_READY), small fast memories, shapes the streaming kernels serve.
     const bool pipelined = c->maps_ready && allow_early && c->k_max <= kFusedMaxK && launch_pool_sparse_supported(e);
+    // ... or, for a large fast memory scored on the tensor cores, the first lookup of a batch alone
+    const bool dense = c->d_dense && dense_scoring_supported(a.D, a.n);
+    const bool pipelined_dense = c->maps_ready && allow_early && begin && dense && launch_encode_ring_supported(e);
     if (c->prof_events && c->prof_seq % c->L == 0) {  // a step begins: does it get a slot for the device-clock stamps?
         c->prof_step = nullptr;
         if ((c->prof_seq / c->L) % c->prof_every == 0 && c->prof_steps_used < c->prof_steps_cap) {
             c->prof_step = c->d_prof_clock + c->prof_steps_used++ * size_t(2 * SMTM_PROF_KERNELS);
             // (the first two words are the stamps of the first layer's streaming kernel: on the pipelined route that
             // kernel runs on the pool stream, which clears them itself)
-            const size_t skip = (pipelined && begin && layer == 0) ? 2 : 0;
+            const size_t skip = ((pipelined || pipelined_dense) && begin && layer == 0) ? 2 : 0;
             SMTM_CUDA(cudaMemsetAsync(c->prof_step + skip, 0, (2 * SMTM_PROF_KERNELS - skip) * sizeof(unsigned long long), st));
             profiled_step_begins = true;
         }
@@ -289,7 +330,7 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     if (pipelined) {
         ++c->routes[SMTM_ROUTE_PIPELINED];
         e.clock = a.clock ? a.clock + 2 * layer : nullptr;  // the pooling kernel is this layer's streaming kernel
-        if (begin) return pooled_first_lookup(c, e, a, st, timing, profiled_step_begins);
+        if (begin) return pooled_first_lookup(c, e, a, st, timing, profiled_step_begins, false);
         // a later layer: the frames still in are few; clusters of small CTAs look them up whole, or, for shapes
         // those do not serve, small CTAs pool them and small CTAs score them
         if (timing) SMTM_CUDA(record_timing(timing[0], st));
@@ -302,17 +343,21 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
         if (!whole) SMTM_CUDA(launch_score_exit(a, st, &c->launches, kPipelinedScoreThreads));
         return SMTM_OK;
     }
+    if (pipelined_dense) {
+        ++c->routes[SMTM_ROUTE_PIPELINED_DENSE];
+        e.clock = a.clock ? a.clock + 2 * layer : nullptr;
+        return pooled_first_lookup(c, e, a, st, timing, profiled_step_begins, true);
+    }
     SMTM_CUDA(launch_lookup_fused(e, a, c->sm_count, &c->fused_caps, st, &c->launches, &fused, timing));
     if (fused) {
         ++c->routes[SMTM_ROUTE_FUSED];
         return SMTM_OK;
     }
-    const bool dense = c->d_dense && dense_scoring_supported(a.D, a.n);  // large fast memory: tensor cores
     ++c->routes[dense ? SMTM_ROUTE_DENSE : SMTM_ROUTE_PLAIN];
     EncodeArgs e2 = e;
     e2.clock = a.clock ? a.clock + 2 * layer : nullptr;  // the pooling kernel is this layer's streaming kernel
     if (a.fresh) e2.skip = nullptr;  // a batch that starts here: every frame is in, whatever the flags hold
-    if (dense) dense_sv_split(c->d_dense, c->max_batch, c->d_max, &e2.sv_hi, &e2.sv_lo);
+    if (dense) dense_sv_split(c->d_dense, c->max_batch, c->d_max, c->split_which, &e2.sv_hi, &e2.sv_lo);
     bool sv_split = false;
     if (timing) SMTM_CUDA(record_timing(timing[0], st));
     SMTM_CUDA(launch_encode(e2, c->sm_count, st, &c->launches, &sv_split));
@@ -320,9 +365,9 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     if (dense) {
         float *dots = nullptr, *dots2 = nullptr;
         SMTM_CUDA(launch_dense_dots(a.sv, a.fresh ? nullptr : a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max,
-                                    sv_split, c->d_cen_split[layer], c->d_split_current + layer, &dots, &dots2, c->d_status,
+                                    c->split_which, sv_split, nullptr, c->d_cen_split[layer], &dots, &dots2, c->d_status,
                                     a.clock ? a.clock + 2 * SMTM_PROF_SCORE_TC : nullptr, st, &c->launches));
-        SMTM_CUDA(launch_finish_dense(a, dots, dots2, c->d_split_current + layer, st, &c->launches));
+        SMTM_CUDA(launch_finish_dense(a, dots, dots2, st, &c->launches));
         return SMTM_OK;
     }
     SMTM_CUDA(launch_score_exit(a, st, &c->launches));
@@ -343,6 +388,7 @@ ResizeArgs resize_args(const smtm_cache* c) {
     a.ts = c->d_ts;
     a.members = c->d_members;
     a.k = c->d_k;
+    a.clock = c->prof_events ? c->prof_step : nullptr;
     return a;
 }
 
@@ -369,7 +415,6 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
     a.pred = b->d_pred;
     a.fallback = d_fallback;
     a.clock = c->prof_events ? c->prof_step : nullptr;
-    a.split_current = c->d_split_current;
     a.status = c->d_status;
     a.ft = c->d_ft;
     a.ts = c->d_ts;
@@ -379,6 +424,7 @@ smtm_status_t update_impl(smtm_cache* c, const smtm_batch_t* b, const int32_t* d
         a.centers[l] = c->d_centers[l];
         a.cnorm[l] = c->d_cnorm[l];
         a.m[l] = c->d_m[l];
+        a.cen_split[l] = has_centre_split(c, l) ? static_cast<__nv_bfloat16*>(c->d_cen_split[l]) : nullptr;
     }
     const ResizeArgs rz = resize_args(c);
     SMTM_CUDA(launch_update(a, with_resize ? &rz : nullptr, c->sm_count, st, &c->launches));
@@ -491,8 +537,6 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     c->d_max = (c->d_max + 7) / 8 * 8;  // keeps the bf16 operand arrays of the tensor-core scorer 16-byte aligned
     if (ok && c->k_max > kFusedMaxK) {
         ok = cudaMalloc(&c->d_dense, dense_scratch_bytes(c->max_batch, n, c->d_max)) == cudaSuccess;
-        ok = ok && dev_alloc(&c->d_split_current, SMTM_MAX_LAYERS) == cudaSuccess &&
-             cudaMemset(c->d_split_current, 0, SMTM_MAX_LAYERS * sizeof(int)) == cudaSuccess;
         for (int l = 0; ok && l < c->L; ++l)
             ok = cudaMalloc(&c->d_cen_split[l], dense_centers_split_bytes(n, c->dims[l])) == cudaSuccess;
     }
@@ -504,6 +548,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     ok = ok && cudaStreamCreateWithFlags(&c->pool_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_pool, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_scored, cudaEventDisableTiming) == cudaSuccess;
     for (cudaEvent_t& e : c->ev_mark) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();
@@ -527,6 +572,7 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
             e = cudaMemcpy(c->d_m[l], (h_counts && h_counts[l]) ? h_counts[l] : ones.data(), n * sizeof(uint32_t),
                            cudaMemcpyHostToDevice);
         if (e == cudaSuccess) e = launch_center_norms(c->d_centers[l], n, c->dims[l], c->d_cnorm[l], 0, &c->launches);
+        if (e == cudaSuccess) e = split_centres(c, l, 0);
     }
     if (e == cudaSuccess) e = cudaMemset(c->d_ft, 0, size_t(S) * n * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(c->d_ts, 0, size_t(S) * n * sizeof(int32_t));
@@ -632,7 +678,6 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
     a.ticket = c->d_ticket;
     a.plan.epoch = c->d_epoch;
     a.fallback = d_labels;
-    a.split_current = c->d_split_current;
     a.status = c->d_status;
     a.ft = c->d_ft;
     a.ts = c->d_ts;
@@ -642,6 +687,7 @@ smtm_status_t smtm_cache_warmup(smtm_cache_t* c, int32_t layer, const smtm_fmap_
         a.centers[l] = c->d_centers[l];
         a.cnorm[l] = c->d_cnorm[l];
         a.m[l] = c->d_m[l];
+        a.cen_split[l] = has_centre_split(c, l) ? static_cast<__nv_bfloat16*>(c->d_cen_split[l]) : nullptr;
     }
     SMTM_CUDA(launch_update(a, nullptr, c->sm_count, st, &c->launches));
     return SMTM_OK;
@@ -961,8 +1007,7 @@ smtm_status_t smtm_cache_import(smtm_cache_t* c, const void* h_blob, uint64_t by
         if (ks[s] < 1 || ks[s] > c->k_max) return SMTM_ERR_INVALID_ARG;
     SMTM_CUDA(cudaDeviceSynchronize());
     SMTM_CUDA(blob_copy(c, const_cast<unsigned char*>(static_cast<const unsigned char*>(h_blob)) + sizeof(h), false));
-    // the tensor-core scorer's bf16 copy of the centres is derived from them: stale now
-    if (c->d_split_current) SMTM_CUDA(cudaMemset(c->d_split_current, 0, SMTM_MAX_LAYERS * sizeof(int)));
+    for (int l = 0; l < c->L; ++l) SMTM_CUDA(split_centres(c, l, 0));  // the tensor-core scorer's bf16 copy of the centres
     SMTM_CUDA(cudaDeviceSynchronize());
     return SMTM_OK;
 }

@@ -1017,12 +1017,12 @@ constexpr int kThreadsNhwcLookup = 512;  // more threads, fewer trips to memory 
 template <class E>
 __global__ void __launch_bounds__(kThreadsNhwcLookup) k_lookup_nhwc(const uint8_t* __restrict__ x, int C, int HW, float inv_hw,
                                                                     float* __restrict__ sv_out, const LookupArgs a) {
-    extern __shared__ float nhwc_smem[];  // sv [C] | s_cur [k_max] | s_acc [k_max] | part [phases][cgs * V]
+    extern __shared__ float nhwc_smem[];  // sv [C] | s_cur [k_max] | s_acc [k_max] | classes [k_max] | part [phases][cgs * V]
     __shared__ float scratch[32];
     float* sv_s = nhwc_smem;
     float* s_cur = sv_s + C;
     float* s_acc = s_cur + a.k_max;
-    float* part = s_acc + a.k_max;
+    float* part = s_acc + 2 * a.k_max;
     chain_wait();
     chain_release();
     const ClockScope stamps(a.clock ? a.clock + 2 * a.layer : nullptr);
@@ -1292,6 +1292,12 @@ cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, in
     return launch_generic<BF16>(a, st);
 }
 
+bool launch_encode_ring_supported(const EncodeArgs& a) {
+    if (a.layout != SMTM_NCHW || a.B <= 0) return false;
+    NchwParams p;
+    return plan_nchw(a, &p) != kNone;
+}
+
 bool launch_pool_sparse_supported(const EncodeArgs& a) {
     if (a.layout != SMTM_NCHW || a.B <= 0) return false;
     NchwParams p;
@@ -1372,7 +1378,7 @@ cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm
         const int V = e.dtype == SMTM_F32 ? 4 : 8;
         if (e.C % V || e.C > 8192) return cudaSuccess;
         const int cgs = std::min(e.C / V, kThreadsNhwcLookup);
-        const size_t smem = (size_t(e.C) + 2 * size_t(a.k_max) + size_t(kThreadsNhwcLookup / cgs) * cgs * V) * sizeof(float);
+        const size_t smem = (size_t(e.C) + 3 * size_t(a.k_max) + size_t(kThreadsNhwcLookup / cgs) * cgs * V) * sizeof(float);
         const float inv_hw = 1.0f / float(e.H * e.W);
         const uint8_t* x = static_cast<const uint8_t*>(e.x);
         cudaError_t err = cudaSuccess;

@@ -1,6 +1,7 @@
 // Host-side declarations shared by the translation units of the SMTM library.
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -89,6 +90,8 @@ struct EncodeArgs {
 // *wrote_split (may be null) tells whether sv_hi / sv_lo were filled by the kernel that ran.
 cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches,
                           bool* wrote_split = nullptr);
+// Whether launch_encode serves the shape with the streaming ring, whose depth the ring_* fields set.
+bool launch_encode_ring_supported(const EncodeArgs& a);
 // Asks that SMs running `kernel` be configured with as much shared memory as they can have.  Kernels that
 // are meant to share an SM with a streaming kernel (whose CTAs need most of it) must not leave the SM in a
 // configuration with less: a CTA of the streaming kernel would wait until the SM has drained.
@@ -155,19 +158,23 @@ cudaError_t launch_lookup_fused(const EncodeArgs& e, const LookupArgs& a, int sm
 bool dense_scoring_supported(int D, int n);
 size_t dense_scratch_bytes(int max_batch, int n, int d_max);
 // DOT[b][c] = <sv[b], centers[c]> for b < B, c < n into scratch; *dots_out = the [B][n] result.
-// The bf16 heads and tails of the semantic vectors sit at the start of scratch (see
-// dense_sv_split); sv_split_done says whether they are already current; centers_split_current is a device flag
-// that says the same of the centres' split (set by the finishing kernel, cleared by every update of the layer).
-void dense_sv_split(void* scratch, int max_batch, int d_max, void** hi, void** lo);
+// The bf16 heads and tails of the semantic vectors sit at the start of scratch, in two sets (see
+// dense_sv_split; `which` picks one); sv_split_done says whether they are already current; sv_ready: nullptr, or
+// an event `st` has to wait for before it reads the vectors or their split (the pooling of the pipelined route).
+// centers_split holds the same split of the centres ([n][D] heads, then [n][D] tails, D a multiple of 4): made by
+// launch_centers_split whenever the centres are set as a whole, and kept in step by Eq. 7's kernel afterwards.
+void dense_sv_split(void* scratch, int max_batch, int d_max, int which, void** hi, void** lo);
+cudaError_t launch_centers_split(const float* centers, int n, int D, void* centers_split, cudaStream_t st,
+                                 int64_t* launches);
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
-                              void* scratch, int max_batch, int d_max, bool sv_split_done, void* centers_split,
-                              int* centers_split_current, float** dots_out, float** dots2_out, int* status,
-                              unsigned long long* clock, cudaStream_t st, int64_t* launches);
+                              void* scratch, int max_batch, int d_max, int which, bool sv_split_done,
+                              cudaEvent_t sv_ready, void* centers_split, float** dots_out, float** dots2_out,
+                              int* status, unsigned long long* clock, cudaStream_t st, int64_t* launches);
 size_t dense_centers_split_bytes(int n, int D);
 // Eq. 1 from the dot products, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule; dots: [B][n], and dots2
 // (nullptr, or [B][n]: the second half of the vector length, added to the first).
-cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, int* split_current,
-                                cudaStream_t st, int64_t* launches);
+cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, cudaStream_t st,
+                                int64_t* launches);
 // One warp that waits, bounded, on a barrier nobody arrives on (the self-test of the time-out path).
 cudaError_t launch_wait_selftest(int* status, cudaStream_t st, int64_t* launches);
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,
@@ -193,7 +200,7 @@ struct UpdatePlan {
 struct UpdateArgs {
     int B, S, n, L;
     unsigned long long* clock;  // nullptr, or the profiled step's stamps [SMTM_PROF_KERNELS][2] (see ClockScope)
-    int* split_current;         // nullptr, or [L]: the centres' bf16 split of a layer is current (cleared when Eq. 7 moves a centre)
+    __nv_bfloat16* cen_split[SMTM_MAX_LAYERS];  // nullptr, or that split ([n][D] heads, then [n][D] tails): Eq. 7 keeps it in step with the centre it moves
     int forget_W;              // 0, or W when the frequency table itself forgets (SMTM_FLAG_FORGET_FT)
     int warm_layer;            // -1, or the one layer a warm-up batch folds into (no tables; done == nullptr)
     UpdatePlan plan;
@@ -222,6 +229,7 @@ struct ResizeArgs {
     const int32_t* ts;
     int32_t* members;  // [S][k_max]
     int32_t* k;        // [S]
+    unsigned long long* clock;  // nullptr, or the profiled step's stamps [SMTM_PROF_KERNELS][2] (see ClockScope)
 };
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches);
 // Tables and centres; with rz != nullptr also the Eq. 5 / Eq. 6 refresh of every stream that

@@ -17,13 +17,14 @@ namespace smtm {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kFinishThreads = 128;  // decision kernel of the dense route: eight CTAs fit an SM, a frame each
 
 // Any whole number of warps up to kThreads per CTA.
 __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
     extern __shared__ float smem[];
     float* sv = smem;                 // [D]
     float* s_cur = sv + a.D;          // [k_max] similarities of this layer
-    float* s_acc = s_cur + a.k_max;   // [k_max] cumulative similarities
+    float* s_acc = s_cur + a.k_max;   // [k_max] cumulative similarities, then [k_max] the slots' classes
     __shared__ float scratch[32];
 
     chain_wait();
@@ -49,15 +50,6 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
 // products into similarities of its fast-memory slots and decides.  Every thread keeps the
 // two best of its own slots as 64-bit ranking keys; warps merge by two warp-wide maxima, the
 // CTA through shared memory.  With a.fresh the carry is taken as SA = 0, nobody done.
-__device__ __forceinline__ void keep_two(unsigned long long e, unsigned long long& b1, unsigned long long& b2) {
-    if (e > b1) {
-        b2 = b1;
-        b1 = e;
-    } else if (e > b2) {
-        b2 = e;
-    }
-}
-
 // The best two keys of the CTA, valid in thread 0.  (b1, b2): this thread's best two; s_keys: [2 * warps].
 __device__ __forceinline__ Top2 block_top2_keys(unsigned long long b1, unsigned long long b2, unsigned long long* s_keys) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -71,7 +63,7 @@ __device__ __forceinline__ Top2 block_top2_keys(unsigned long long b1, unsigned 
     Top2 t{0.f, 0.f, -1, -1};
     if (threadIdx.x == 0) {
         unsigned long long c1 = 0ull, c2 = 0ull;
-        for (int i = 0; i < 2 * (kThreads / kWarp); ++i) keep_two(s_keys[i], c1, c2);
+        for (int i = 0; i < 2 * int(blockDim.x >> 5); ++i) keep_two(s_keys[i], c1, c2);
         rank_key_decode(c1, &t.v1, &t.id1);
         rank_key_decode(c2, &t.v2, &t.id2);
     }
@@ -79,14 +71,14 @@ __device__ __forceinline__ Top2 block_top2_keys(unsigned long long b1, unsigned 
     return t;
 }
 
-__global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, const float* __restrict__ dots,
-                                                           const float* __restrict__ dots2, int* split_current) {
+__global__ void __launch_bounds__(kFinishThreads, 8) k_finish_dense(const LookupArgs a, const float* __restrict__ dots,
+                                                           const float* __restrict__ dots2) {
     __shared__ float scratch[32];
-    __shared__ unsigned long long s_keys[2 * (kThreads / kWarp)];
+    __shared__ unsigned long long s_keys[2 * (kFinishThreads / kWarp)];
     chain_wait();
     chain_release();
+    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_FINISH_DENSE : nullptr);
     const int b = blockIdx.x;
-    if (b == 0 && threadIdx.x == 0 && split_current) *split_current = 1;  // the scorer before this kernel used (or made) a current split
     if (!a.fresh && a.done[b]) return;
     const int tid = threadIdx.x;
     const int sid = stream_of(a, b);
@@ -100,30 +92,39 @@ __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, c
     float* sa_row = a.sa + (size_t)b * a.k_max;
     unsigned long long a1 = 0ull, a2 = 0ull, c1 = 0ull, c2 = 0ull;  // best two cumulative / single-layer keys
     float nrm = 0.f, sv_len = 0.f;
-    for (int j0 = 0; j0 < k; j0 += 4 * kThreads) {  // four slots per thread, every load issued before any store
+    for (int j0 = 0; j0 < k; j0 += 4 * kFinishThreads) {  // four slots per thread, every load issued before any store
         int cls[4];
         float dot[4], cl[4], old[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int j = j0 + u * kThreads + tid;
+            const int j = j0 + u * kFinishThreads + tid;
             cls[u] = mem[min(j, k - 1)];
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int j = j0 + u * kThreads + tid;
+            const int j = j0 + u * kFinishThreads + tid;
             dot[u] = drow[cls[u]];
             if (drow2) dot[u] += drow2[cls[u]];
             cl[u] = clen[cls[u]];
             old[u] = (j < k && !a.fresh) ? sa_row[j] : 0.f;
         }
         if (j0 == 0) {  // the squared length of the semantic vector, while the loads above are in flight
-            for (int d = tid; d < a.D; d += kThreads) nrm = fmaf(row[d], row[d], nrm);
+            const float4* row4 = reinterpret_cast<const float4*>(row);  // (D is a multiple of 8 on this route)
+            float q[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int d = tid; d < a.D / 4; d += kFinishThreads) {
+                const float4 v = row4[d];
+                q[0] = fmaf(v.x, v.x, q[0]);
+                q[1] = fmaf(v.y, v.y, q[1]);
+                q[2] = fmaf(v.z, v.z, q[2]);
+                q[3] = fmaf(v.w, v.w, q[3]);
+            }
+            nrm = (q[0] + q[1]) + (q[2] + q[3]);
             nrm = block_sum(nrm, scratch);
             sv_len = __fsqrt_rn(nrm);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int j = j0 + u * kThreads + tid;
+            const int j = j0 + u * kFinishThreads + tid;
             if (j < k) {
                 const float s = (nrm == 0.f || cl[u] == 0.f) ? 0.f : __fdiv_rn(dot[u], __fmul_rn(sv_len, cl[u]));  // Eq. 1
                 const float acc = __fmaf_rn(s, weight, old[u]);    // Eq. 3
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(kThreads) k_finish_dense(const LookupArgs a, c
         }
     }
     if (a.fresh)
-        for (int j = k + tid; j < a.k_max; j += kThreads) sa_row[j] = 0.f;  // unused slots start from zero too
+        for (int j = k + tid; j < a.k_max; j += kFinishThreads) sa_row[j] = 0.f;  // unused slots start from zero too
     const Top2 ta = block_top2_keys(a1, a2, s_keys);
     Top2 ts{0.f, 0.f, -1, -1};
     if (a.sep) ts = block_top2_keys(c1, c2, s_keys);
@@ -177,6 +178,7 @@ cudaError_t launch_wait_selftest(int* status, cudaStream_t st, int64_t* launches
 cudaError_t lookup_setup() {
     cudaError_t e = allow_max_dynamic_smem(k_score_exit);
     if (e == cudaSuccess) e = prefer_max_smem_carveout(k_score_exit);
+    if (e == cudaSuccess) e = prefer_max_smem_carveout(k_finish_dense);
     return e;
 }
 
@@ -189,16 +191,16 @@ cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, in
     return launch_chained(k_batch_reset, grid, 256, 0, st, sa, done, exit_layer, pred, B, n_sa);
 }
 
-cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, int* split_current,
+cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2,
                                 cudaStream_t st, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
     ++*launches;
-    return launch_chained(k_finish_dense, a.B, kThreads, 0, st, a, dots, dots2, split_current);
+    return launch_chained(k_finish_dense, a.B, kFinishThreads, 0, st, a, dots, dots2);
 }
 
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches, int threads) {
     if (a.B <= 0) return cudaSuccess;
-    const size_t smem = (size_t(a.D) + 2 * size_t(a.k_max)) * sizeof(float);
+    const size_t smem = (size_t(a.D) + 3 * size_t(a.k_max)) * sizeof(float);
     ++*launches;
     return launch_chained(k_score_exit, a.B, threads > 0 ? threads : kThreads, smem, st, a);
 }

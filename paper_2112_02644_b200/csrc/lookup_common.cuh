@@ -34,29 +34,6 @@ struct Top2 {
     int id1, id2;  // class ids, -1 = absent
 };
 
-__device__ __forceinline__ void top2_push(Top2& t, float v, int id) {
-    if (t.id1 < 0 || ranks_before(v, id, t.v1, t.id1)) {
-        t.v2 = t.v1; t.id2 = t.id1;
-        t.v1 = v; t.id1 = id;
-    } else if (t.id2 < 0 || ranks_before(v, id, t.v2, t.id2)) {
-        t.v2 = v; t.id2 = id;
-    }
-}
-
-// Best two of the values v[0..k) with class ids ids[0..k); executed by one full warp.
-__device__ __forceinline__ Top2 warp_top2(const float* v, const int32_t* ids, int k, int lane) {
-    Top2 t{0.f, 0.f, -1, -1};
-    for (int j = lane; j < k; j += kWarp) top2_push(t, v[j], ids[j]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float ov1 = __shfl_xor_sync(kFull, t.v1, o), ov2 = __shfl_xor_sync(kFull, t.v2, o);
-        const int oi1 = __shfl_xor_sync(kFull, t.id1, o), oi2 = __shfl_xor_sync(kFull, t.id2, o);
-        if (oi1 >= 0) top2_push(t, ov1, oi1);
-        if (oi2 >= 0) top2_push(t, ov2, oi2);
-    }
-    return t;
-}
-
 // (top - second) / second with the sign cases: top <= 0 -> 0; second NaN -> NaN; second <= 0 < top -> +inf.
 __device__ __forceinline__ float ratio_margin(float top, float second) {
     if (!(top > 0.f)) return 0.f;
@@ -102,6 +79,30 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
     return v;
 }
 
+// Keeps the two largest keys seen so far.
+__device__ __forceinline__ void keep_two(unsigned long long e, unsigned long long& b1, unsigned long long& b2) {
+    if (e > b1) {
+        b2 = b1;
+        b1 = e;
+    } else if (e > b2) {
+        b2 = e;
+    }
+}
+
+// Best two of v[0..k) with classes ids[0..k) (any k), executed by one full warp: every lane keeps the best two keys of
+// its own slots, then two warp-wide maxima (keys are distinct: the runner-up sits below the winner in the
+// winner's lane or is some lane's best).
+__device__ __forceinline__ Top2 warp_top2_by_keys(const float* v, const int32_t* ids, int k, int lane) {
+    unsigned long long b1 = 0ull, b2 = 0ull;
+    for (int j = lane; j < k; j += kWarp) keep_two(rank_key(v[j], ids[j]), b1, b2);
+    const unsigned long long k1 = warp_max_u64(b1);
+    const unsigned long long k2 = warp_max_u64(b1 == k1 ? b2 : b1);
+    Top2 t;
+    rank_key_decode(k1, &t.v1, &t.id1);
+    rank_key_decode(k2, &t.v2, &t.id2);
+    return t;
+}
+
 // Best two of values held in registers (lane l holds slots l and l + 32 of k), by two warp-wide
 // maxima over the keys: the same result as pushing every entry through top2_push and merging by
 // shuffles, in a fraction of the instructions.
@@ -123,8 +124,9 @@ __device__ __forceinline__ Top2 warp_top2_keys(const float (&v)[2], const int (&
 // writes the frame's outputs and the counters.
 __device__ __forceinline__ void decide_frame(const LookupArgs& a, int b, const float* s_cur, const float* s_acc,
                                              const int32_t* mem, int k, int lane) {
-    const Top2 ta = warp_top2(s_acc, mem, k, lane);
-    const Top2 ts = warp_top2(s_cur, mem, k, lane);
+    const Top2 ta = warp_top2_by_keys(s_acc, mem, k, lane);
+    Top2 ts{0.f, 0.f, -1, -1};
+    if (a.sep) ts = warp_top2_by_keys(s_cur, mem, k, lane);  // only Eq. 2 (a diagnostic) needs it
     if (lane != 0) return;
     decide_from_top2(a, b, ta, ts);
 }
@@ -169,7 +171,7 @@ __device__ __forceinline__ void decide_from_top2(const LookupArgs& a, int b, con
 
 // Scores frame b against the members of its fast memory and decides, by a whole CTA (any whole number of
 // warps): pf is what prefetch_slots returned for the frame's stream id, sv the frame's semantic vector in shared memory (already visible to every thread), nrm its squared
-// length; s_cur / s_acc hold k_max floats each.  Each warp takes fast-memory slots round-robin and reads the
+// length; s_cur and s_acc hold k_max floats each and s_acc is followed by k_max more words (the slots' classes).  Each warp takes fast-memory slots round-robin and reads the
 // member's centre (L2-resident) with 128-bit loads; lanes keep four independent fp32 accumulators and combine
 // with xor-shuffles, so every dot product has a fixed evaluation order.  Warp 0 then selects the two best.
 // The kernel's time is the number of dependent trips to memory: the size of the fast memory and the warp's
@@ -192,6 +194,7 @@ __device__ __forceinline__ SlotPrefetch prefetch_slots(const LookupArgs& a, int 
 __device__ __forceinline__ void score_frame(const LookupArgs& a, int b, const SlotPrefetch& pf, const float* sv, float nrm,
                                             float* s_cur, float* s_acc) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x, nw = nthreads / kWarp;
+    int32_t* s_ids = reinterpret_cast<int32_t*>(s_acc + a.k_max);  // the slots' classes, for the decision
     const int32_t* mem = a.members + (size_t)max(pf.sid, 0) * a.k_max;
     int cls_next = pf.cls;
     const int k = pf.k;
@@ -231,13 +234,14 @@ __device__ __forceinline__ void score_frame(const LookupArgs& a, int b, const Sl
             a.sa[(size_t)b * a.k_max + j] = acc;
             s_cur[j] = s;
             s_acc[j] = acc;
+            s_ids[j] = cls;
         }
     }
     if (a.fresh)
         for (int j = k + tid; j < a.k_max; j += nthreads) a.sa[(size_t)b * a.k_max + j] = 0.f;  // unused slots start from zero too
     __syncthreads();
     if (warp != 0) return;
-    decide_frame(a, b, s_cur, s_acc, mem, k, lane);
+    decide_frame(a, b, s_cur, s_acc, s_ids, k, lane);
 }
 
 // Eq. 1 from a dot product and the two lengths; a zero-length vector is similar to nothing.

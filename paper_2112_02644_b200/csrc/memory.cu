@@ -24,6 +24,8 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include <cuda_bf16.h>
+
 #include "internal.h"
 
 namespace smtm {
@@ -49,6 +51,7 @@ __device__ __forceinline__ void table_step(int& ft, int& ts, bool appears, int f
 
 constexpr int kUpdThreads = 256;   // plan kernel (many-CTA form) and the stand-alone refresh
 constexpr int kApplyThreads = 128; // CTAs of the apply kernel
+constexpr int kTabPer = 8;         // consecutive frames a thread of a tables CTA looks at per trip to memory
 
 // The label a finished frame ends up with: the prediction if it exited, else the fallback label
 // (the full network's answer, -1 = none); a label outside the memory counts as no label.
@@ -247,29 +250,34 @@ __device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v
     return t;
 }
 
-// Eq. 6 by one warp: the smallest k in [k_min, k_max] with cl_den * (sum of the k best scores) > cl_num * total,
-// by a scan of 32 entries per step; s_top holds the k_max best scores in rank order.
+// Eq. 6 by one warp: the smallest k in [k_min, k_max] with cl_den * (sum of the k best scores) > cl_num * total;
+// s_top holds the k_max best scores in rank order.  Every lane looks after a run of consecutive ranks (of odd
+// length, which spreads the lanes over the banks): it adds its run up, a scan over the lanes gives the sum of
+// the ranks before it, and a second walk finds the first rank of the run that satisfies the test.
 __device__ __forceinline__ void adaptive_size(const ResizeArgs& a, int s, const unsigned long long* s_top,
                                               unsigned long long total, int lane) {
-    unsigned long long carry = 0;
     int chosen = a.k_max;
-    for (int base = 0; base < a.k_max; base += kWarp) {
-        const int idx = base + lane;
-        unsigned long long v = idx < a.k_max ? s_top[idx] : 0ull;
+    if (a.k_min < a.k_max) {  // (otherwise there is nothing to choose)
+        const int per = ((a.k_max + kWarp - 1) / kWarp) | 1;
+        const int lo = min(lane * per, a.k_max), hi = min(lo + per, a.k_max);
+        unsigned long long run = 0;
+        for (int r = lo; r < hi; ++r) run += s_top[r];
+        unsigned long long inc = run;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned long long t = __shfl_up_sync(kFull, v, o);
-            if (lane >= o) v += t;
+        for (int o = 1; o < kWarp; o <<= 1) {
+            const unsigned long long t = __shfl_up_sync(kFull, inc, o);
+            if (lane >= o) inc += t;
         }
-        const unsigned long long prefix = carry + v;
-        const bool ok = idx < a.k_max && idx + 1 >= a.k_min &&
-                        (unsigned long long)a.cl_den * prefix > (unsigned long long)a.cl_num * total;
-        const unsigned m = __ballot_sync(kFull, ok);
-        if (m) {
-            chosen = base + __ffs(m);
-            break;
+        unsigned long long prefix = inc - run;
+        const unsigned long long need = (unsigned long long)a.cl_num * total;
+        for (int r = lo; r < hi; ++r) {
+            prefix += s_top[r];
+            if (r + 1 >= a.k_min && (unsigned long long)a.cl_den * prefix > need) {
+                chosen = r + 1;
+                break;
+            }
         }
-        carry += __shfl_sync(kFull, v, 31);
+        chosen = __reduce_min_sync(kFull, chosen);
     }
     if (lane == 0) a.k[s] = chosen;
 }
@@ -277,22 +285,55 @@ __device__ __forceinline__ void adaptive_size(const ResizeArgs& a, int s, const 
 // Descending bitonic sort of nz keys in s_key by the whole CTA (padded to a power of two with zeros: no key is zero).
 __device__ void sort_keys(unsigned long long* s_key, int nz) {
     const int tid = threadIdx.x, nt = blockDim.x;
-    const int P = pow2_at_least(nz);
+    const int P = pow2_at_least(nz), half = P >> 1;
     for (int i = nz + tid; i < P; i += nt) s_key[i] = 0ull;
     __syncthreads();
+    // Pair t of a round with stride j is (i, i + j), i = t with a zero bit put in at j's position.  Thread t keeps
+    // pair t in every round, so with strides up to 32 the pairs of a warp stay inside the 64 keys that warp alone
+    // touches: such a round needs the whole CTA only when the round before or after it has a longer stride.
     for (int k = 2; k <= P; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int t = tid; t < P / 2; t += nt) {
-                const int i = 2 * j * (t / j) + (t % j), l = i + j;
+            for (int t = tid; t < half; t += nt) {
+                const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1)), l = i + j;
                 const unsigned long long ki = s_key[i], kl = s_key[l];
                 if (((i & k) == 0) ? kl > ki : kl < ki) {
                     s_key[i] = kl;
                     s_key[l] = ki;
                 }
             }
-            __syncthreads();
+            const int next = j > 1 ? j >> 1 : k;  // (the next phase opens with stride k)
+            if (j > kWarp || next > kWarp) __syncthreads();
+            else __syncwarp();
         }
     }
+    __syncthreads();
+}
+
+// Descending bitonic sort with one key per thread (thread i holds element i; a CTA of P threads, P a power of two
+// and a multiple of 32; every thread of the CTA calls): partners up to 16 apart trade keys by warp shuffle, those
+// further apart through shared memory, one barrier per round over two alternating buffers of P words each.
+__device__ __forceinline__ unsigned long long sort_one_key_per_thread(unsigned long long key, int P,
+                                                                      unsigned long long* s_x) {
+    const int i = threadIdx.x;
+    int flip = 0;
+    for (int k = 2; k <= P; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            unsigned long long other;
+            if (j < kWarp) {
+                other = __shfl_xor_sync(kFull, key, j);
+            } else {
+                unsigned long long* buf = s_x + (flip ? P : 0);
+                flip ^= 1;
+                buf[i] = key;
+                __syncthreads();
+                other = buf[i ^ j];
+            }
+            // the lower index of a pair keeps the larger key where the run is descending, the smaller one elsewhere
+            const bool larger = ((i & j) == 0) == ((i & k) == 0);
+            key = larger ? max(key, other) : min(key, other);
+        }
+    }
+    return key;
 }
 
 // Eq. 5 / Eq. 6 for stream s when every thread of the CTA holds the scores of its PER consecutive classes
@@ -384,6 +425,24 @@ __device__ void refresh_stream(const ResizeArgs& a, int s, unsigned char* dyn, i
     const int32_t* ft = a.ft + (size_t)s * a.n;
     const int32_t* ts = a.ts + (size_t)s * a.n;
     int32_t* mem = a.members + (size_t)s * a.k_max;
+    if (nt == cap) {
+        // A thread per class: the key of class tid (one more than the ranking key, so that the classes with a zero
+        // score sort behind the others in ascending id, as the refresh wants them, and before the padding),
+        // sorted in registers; thread r ends up with the class of rank r.
+        const bool real = tid < a.n;
+        const unsigned long long sc = real ? score_of(ft[tid], ts[tid], a.W, a.forgetting) : 0ull;
+        const unsigned long long total = block_sum_u64(sc, s_part);
+        if (total == 0) return;  // nothing seen yet: keep size and members (the same for every thread)
+        const unsigned long long key = sort_one_key_per_thread(real ? refresh_key(sc, tid) + 1ull : 0ull, cap, s_key);
+        unsigned long long* s_best = s_key + 2 * cap;
+        if (tid < a.k_max && tid < a.n) {
+            mem[tid] = key_class(key - 1ull);
+            s_best[tid] = key_score(key - 1ull);
+        }
+        __syncthreads();
+        if (tid < kWarp) adaptive_size(a, s, s_best, total, tid);
+        return;
+    }
     const int per = (a.n + nt - 1) / nt;
     const int c_lo = min(a.n, tid * per), c_hi = min(a.n, c_lo + per);
     const auto score_at = [&](int c) { return score_of(ft[c], ts[c], a.W, a.forgetting); };
@@ -404,7 +463,7 @@ __device__ void refresh_stream(const ResizeArgs& a, int s, unsigned char* dyn, i
         if (sc != 0) s_key[pos++] = refresh_key(sc, c);
     }
     __syncthreads();
-    if (nz <= max(kCountRankMax, 4 * nt)) {  // (a few keys per thread at most: every thread reads all of them)
+    if (nz <= kCountRankMax) {
         // rank = keys larger than this one (keys are distinct); rank r < k_max goes to slot r
         for (int i = tid; i < nz; i += nt) {
             const unsigned long long key = s_key[i];
@@ -451,6 +510,7 @@ __global__ void __launch_bounds__(kResizeThreadsMax) k_resize(const ResizeArgs a
     __shared__ unsigned long long s_part[32];
     chain_wait();
     chain_release();
+    const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_REFRESH : nullptr);
     refresh_stream(a, blockIdx.x, reinterpret_cast<unsigned char*>(s_dyn), s_scan, s_part);
 }
 
@@ -478,7 +538,8 @@ __host__ __device__ constexpr size_t tables_smem(int n, int k_max, bool with_ref
 }
 
 // Sec. 6.1 for the stream of frame g by one CTA, if g is the stream's first frame in the batch (else the
-// CTA of that frame does it): all of the stream's frames, in ascending index, applied to its tables; then,
+// CTA of that frame does it; g < 0: the only stream of a cache that has one, whichever frame of it comes
+// first): all of the stream's frames, in ascending index, applied to its tables; then,
 // if asked, the stream's Eq. 5 / Eq. 6 refresh.  Every thread looks after a run of PER consecutive classes
 // and keeps their entries in registers from the one trip to memory that fetches them to the refresh
 // (PER == 0: any number of classes, the entries stay in global memory).
@@ -490,7 +551,9 @@ __device__ void tables_of_frame(const UpdateArgs& a, const ResizeArgs& rz, int g
         s_scan[32] = 0;
         s_part[31] = 0ull;
     }
-    const int s = a.stream_id ? a.stream_id[g] : 0;
+    const bool lone = g < 0;
+    if (lone) g = 0;
+    const int s = (a.stream_id && !lone) ? a.stream_id[g] : 0;
     if (s < 0 || s >= a.S) return;  // no such stream (the same for every thread; the plan kernel records the error)
     const int per = PER ? PER : (a.n + nt - 1) / nt;
     const int c_lo = min(a.n, tid * per), c_hi = min(a.n, c_lo + per);
@@ -505,8 +568,8 @@ __device__ void tables_of_frame(const UpdateArgs& a, const ResizeArgs& rz, int g
         t[i] = c_lo + i < a.n ? ts[c_lo + i] : 0;
     }
     // an earlier frame of the same stream: its CTA does the work.  Also: is g the stream's only frame?
-    int earlier = (!a.stream_id && g > 0) ? 1 : 0, later = (!a.stream_id && g + 1 < a.B) ? 1 : 0;
-    for (int b0 = 0; a.stream_id && b0 < a.B; b0 += 4 * nt) {
+    int earlier = (!a.stream_id && g > 0) ? 1 : 0, later = ((!a.stream_id && g + 1 < a.B) || lone) ? 1 : 0;
+    for (int b0 = 0; a.stream_id && !lone && b0 < a.B; b0 += 4 * nt) {
         int sidv[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) sidv[u] = a.stream_id[min(b0 + u * nt + tid, a.B - 1)];  // one trip to memory
@@ -547,15 +610,35 @@ __device__ void tables_of_frame(const UpdateArgs& a, const ResizeArgs& rz, int g
             s_last[c] = -1;
         }
         __syncthreads();
+        // Every thread looks at a run of eight consecutive frames (their stream ids and the plan's codes in one
+        // trip to memory); a scan over the threads gives each of the stream's frames its position in the stream.
         int m = 0;
-        for (int t0 = g - g % nt; t0 < a.B; t0 += nt) {
-            const int b = t0 + tid;
-            const int hit = (b >= g && b < a.B && (a.stream_id ? a.stream_id[b] : 0) == s) ? 1 : 0;
-            const int cnt = compact_tile(hit, hit ? final_label_of(a, b) : -1, s_list, s_scan);
-            if (tid < cnt && s_list[tid] >= 0) {
-                atomicAdd(&s_cnt[s_list[tid]], 1);
-                atomicMax(&s_last[s_list[tid]], m + tid);
+        for (int p0 = g; p0 < a.B; p0 += kTabPer * nt) {
+            const int b0 = p0 + tid * kTabPer;
+            int sidv[kTabPer], code[kTabPer];
+#pragma unroll
+            for (int i = 0; i < kTabPer; ++i) {
+                const int b = min(b0 + i, a.B - 1);
+                sidv[i] = a.stream_id ? a.stream_id[b] : s;
+                code[i] = a.plan.frame_code[b];
             }
+            int hits = 0;
+#pragma unroll
+            for (int i = 0; i < kTabPer; ++i) {
+                sidv[i] = (b0 + i < a.B && sidv[i] == s) ? 1 : 0;
+                hits += sidv[i];
+            }
+            int cnt;
+            int pos = m + block_exclusive_scan(hits, s_scan, &cnt);
+#pragma unroll
+            for (int i = 0; i < kTabPer; ++i)
+                if (sidv[i]) {
+                    if (code[i] >= 0) {  // (a frame without a label only ages the classes)
+                        atomicAdd(&s_cnt[code[i] & 0xffff], 1);
+                        atomicMax(&s_last[code[i] & 0xffff], pos);
+                    }
+                    ++pos;
+                }
             m += cnt;
         }
         __syncthreads();
@@ -621,7 +704,7 @@ __device__ void tables_of_frame(const UpdateArgs& a, const ResizeArgs& rz, int g
 
 // ---- apply: Eq. 7 -----------------------------------------------------------------------------
 
-constexpr int kCenPer = 4;                         // consecutive frames a thread looks at
+constexpr int kCenPer = 8;                         // consecutive frames a thread looks at
 constexpr int kCenTile = kCenPer * kApplyThreads;  // frames listed at a time
 constexpr int kRowGroupsMax = 8;
 
@@ -720,6 +803,19 @@ __device__ void centre_item(const UpdateArgs& a, int item, const int (&first_til
                 v.z = float((double(old.z) * dm + double(acc[2])) * inv);
                 v.w = float((double(old.w) * dm + double(acc[3])) * inv);
                 *reinterpret_cast<float4*>(cen + 4 * c4) = v;
+                if (a.cen_split[l0]) {  // the tensor-core scorer's copy of the centre follows it (x = hi + lo in bf16)
+                    __nv_bfloat16* hi = a.cen_split[l0] + (size_t)cls * D + 4 * c4;
+                    __nv_bfloat16* lo = hi + (size_t)a.n * D;
+                    const float x[4] = {v.x, v.y, v.z, v.w};
+                    __nv_bfloat16 h[4], t[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        h[j] = __float2bfloat16_rn(x[j]);
+                        t[j] = __float2bfloat16_rn(x[j] - __bfloat162float(h[j]));
+                    }
+                    *reinterpret_cast<uint2*>(hi) = *reinterpret_cast<const uint2*>(h);
+                    *reinterpret_cast<uint2*>(lo) = *reinterpret_cast<const uint2*>(t);
+                }
                 nrm = fmaf(v.x, v.x, nrm); nrm = fmaf(v.y, v.y, nrm); nrm = fmaf(v.z, v.z, nrm); nrm = fmaf(v.w, v.w, nrm);
             }
         }
@@ -758,10 +854,10 @@ __device__ void centre_item(const UpdateArgs& a, int item, const int (&first_til
     }
     a.cnorm[l0][cls] = __fsqrt_rn(nrm);
     a.m[l0][cls] = m + uint32_t(q);
-    if (a.split_current) a.split_current[l0] = 0;  // the tensor-core scorer's copy of this layer's centres is stale
 }
 
-// The apply kernel: CTAs [0, table_ctas) are tables CTAs, one per frame; the others take the listed items.
+// The apply kernel: CTAs [0, table_ctas) are tables CTAs, one per frame (a single one for a cache with one stream);
+// the others take the listed items.
 __global__ void __launch_bounds__(kApplyThreads, 8) k_update_apply(const UpdateArgs a, const ResizeArgs rz, int do_resize,
                                                                     int table_ctas) {
     extern __shared__ unsigned long long s_dyn[];
@@ -775,11 +871,11 @@ __global__ void __launch_bounds__(kApplyThreads, 8) k_update_apply(const UpdateA
         const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_TABLES : nullptr);
         unsigned char* dyn = reinterpret_cast<unsigned char*>(s_dyn);
         if (a.n <= 4 * kApplyThreads)
-            tables_of_frame<4>(a, rz, blockIdx.x, do_resize, dyn, s_list, s_scan, s_part);
+            tables_of_frame<4>(a, rz, a.S == 1 ? -1 : int(blockIdx.x), do_resize, dyn, s_list, s_scan, s_part);
         else if (a.n <= 8 * kApplyThreads)
-            tables_of_frame<8>(a, rz, blockIdx.x, do_resize, dyn, s_list, s_scan, s_part);
+            tables_of_frame<8>(a, rz, a.S == 1 ? -1 : int(blockIdx.x), do_resize, dyn, s_list, s_scan, s_part);
         else
-            tables_of_frame<0>(a, rz, blockIdx.x, do_resize, dyn, s_list, s_scan, s_part);
+            tables_of_frame<0>(a, rz, a.S == 1 ? -1 : int(blockIdx.x), do_resize, dyn, s_list, s_scan, s_part);
         return;
     }
     const int first = int(blockIdx.x) - table_ctas, stride = int(gridDim.x) - table_ctas;
@@ -822,6 +918,7 @@ cudaError_t memory_setup() {
     if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_apply);
     if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_plan_one);
     if (e == cudaSuccess) e = prefer_max_smem_carveout(k_update_plan);
+    if (e == cudaSuccess) e = prefer_max_smem_carveout(k_resize);
 
     return e;   // (the single-CTA plan needs at most 32 KB + its statics: below the default limit)
 }
@@ -845,14 +942,15 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
     }
     if (e != cudaSuccess) return e;
     const bool tables = a.warm_layer < 0;  // a warm-up batch has no streams
-    const int table_ctas = tables ? a.B : 0;
+    const int table_ctas = tables ? (a.S == 1 ? 1 : a.B) : 0;  // a CTA per frame finds out whether its frame is its stream's first
     // Eq. 7: at most min(B, n) classes appear per layer; a CTA per item, and a heavy pair is several items (never
     // more than twice the rows' worth); beyond a few waves of CTAs they stride
     const int pairs_max = std::min(a.B, a.n) * (a.warm_layer >= 0 ? 1 : a.L);
     const int centre_ctas = std::min(pairs_max + pairs_max / 2 + kItemBlocksMax, 16 * sm_count);
-    // A memory of many classes is refreshed by a kernel of its own with CTAs of 1024 threads (ranking a thousand
-    // scores is a million comparisons: too much for the 128 threads of a tables CTA); it refreshes every stream,
-    // which gives the streams without a frame in the batch the fast memory they already have.
+    // A memory of many classes is refreshed by a kernel of its own with CTAs of 1024 threads (sorting a thousand
+    // keys is 55 rounds of compare-exchange: a round per barrier with 1024 threads, eight times that with the 128
+    // threads of a tables CTA); it refreshes every stream, which gives the streams without a frame in the batch
+    // the fast memory they already have.
     const bool refresh_apart = tables && rz && a.n > 4 * kApplyThreads;
     const bool refresh_here = tables && rz && !refresh_apart;
     const size_t smem = tables ? tables_smem(a.n, rz ? rz->k_max : 0, refresh_here) : 0;
@@ -865,8 +963,12 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
 
 cudaError_t launch_resize(const ResizeArgs& a, cudaStream_t st, int64_t* launches) {
     ++*launches;
-    const int threads = a.n > 4 * kApplyThreads ? kResizeThreadsMax : kUpdThreads;
-    return launch_chained(k_resize, a.S, threads, refresh_smem(a.n, a.k_max), st, a);
+    // a memory of more than 512 and up to 1024 classes gets a thread per class (padded to a power of two): the
+    // sort then runs in registers and needs two buffers for the trades; larger ones 1024 threads
+    const int cap = pow2_at_least(a.n);
+    const int threads = a.n > 4 * kApplyThreads ? std::min(cap, kResizeThreadsMax) : kUpdThreads;
+    const size_t smem = refresh_smem(a.n, a.k_max) + (threads == cap ? size_t(cap) * 8 : 0);
+    return launch_chained(k_resize, a.S, threads, smem, st, a);
 }
 
 }  // namespace smtm

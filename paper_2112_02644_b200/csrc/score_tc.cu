@@ -50,11 +50,9 @@ constexpr size_t kTcSmem = size_t(kTcStages) * kStageBytes + 1024 + 256;
 
 // x = hi + lo with hi = bf16(x) and lo = bf16(x - hi); rows of skipped frames are left alone.
 __global__ void k_split_bf16(const float* __restrict__ src, const uint8_t* __restrict__ skip, int rows, int D,
-                             __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
-                             const int* __restrict__ current) {
+                             __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
     chain_wait();
     chain_release();
-    if (current && *current) return;  // the split on file is that of the source as it stands
     const long long total = (long long)rows * D;
     for (long long i = (blockIdx.x * (long long)blockDim.x + threadIdx.x) * 4; i < total;
          i += (long long)gridDim.x * blockDim.x * 4) {
@@ -315,28 +313,41 @@ bool dense_scoring_supported(int D, int n) {
 }
 
 size_t dense_scratch_bytes(int max_batch, int n, int d_max) {
-    // bf16 heads and tails of the semantic vectors, then the dot products
-    return size_t(max_batch) * d_max * 2 * 2 + size_t(kSplitK) * max_batch * n * sizeof(float) + 1024;
+    // bf16 heads and tails of the semantic vectors (two sets: the pipelined route pools a batch while the one
+    // before it is still being scored), then the dot products
+    return 2 * size_t(max_batch) * d_max * 2 * 2 + size_t(kSplitK) * max_batch * n * sizeof(float) + 1024;
 }
 
 size_t dense_centers_split_bytes(int n, int D) { return size_t(n) * D * 2 * 2; }
 
-void dense_sv_split(void* scratch, int max_batch, int d_max, void** hi, void** lo) {
-    __nv_bfloat16* a_hi = reinterpret_cast<__nv_bfloat16*>(scratch);
+void dense_sv_split(void* scratch, int max_batch, int d_max, int which, void** hi, void** lo) {
+    __nv_bfloat16* a_hi = reinterpret_cast<__nv_bfloat16*>(scratch) + size_t(which & 1) * 2 * size_t(max_batch) * d_max;
     *hi = a_hi;
     *lo = a_hi + size_t(max_batch) * d_max;
 }
 
+cudaError_t launch_centers_split(const float* centers, int n, int D, void* centers_split, cudaStream_t st,
+                                 int64_t* launches) {
+    __nv_bfloat16* b_hi = reinterpret_cast<__nv_bfloat16*>(centers_split);
+    ++*launches;
+    const int grid = int(std::min<long long>(((long long)n * D / 4 + 255) / 256, 148 * 8));
+    return launch_chained(k_split_bf16, grid, 256, 0, st, centers, static_cast<const uint8_t*>(nullptr), n, D, b_hi,
+                          b_hi + size_t(n) * D);
+}
+
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
-                              void* scratch, int max_batch, int d_max, bool sv_split_done, void* centers_split,
-                              int* centers_split_current, float** dots_out, float** dots2_out, int* status,
-                              unsigned long long* clock, cudaStream_t st, int64_t* launches) {
-    __nv_bfloat16* a_hi = reinterpret_cast<__nv_bfloat16*>(scratch);
-    __nv_bfloat16* a_lo = a_hi + size_t(max_batch) * d_max;
+                              void* scratch, int max_batch, int d_max, int which, bool sv_split_done,
+                              cudaEvent_t sv_ready, void* centers_split, float** dots_out, float** dots2_out,
+                              int* status, unsigned long long* clock, cudaStream_t st, int64_t* launches) {
+    void *hi = nullptr, *lo = nullptr;
+    dense_sv_split(scratch, max_batch, d_max, which, &hi, &lo);
+    __nv_bfloat16* a_hi = static_cast<__nv_bfloat16*>(hi);
+    __nv_bfloat16* a_lo = static_cast<__nv_bfloat16*>(lo);
     __nv_bfloat16* b_hi = reinterpret_cast<__nv_bfloat16*>(centers_split);
     __nv_bfloat16* b_lo = b_hi + size_t(n) * D;
     float* dots = reinterpret_cast<float*>(
-        (reinterpret_cast<uintptr_t>(a_lo + size_t(max_batch) * d_max) + 255) & ~uintptr_t(255));
+        (reinterpret_cast<uintptr_t>(reinterpret_cast<__nv_bfloat16*>(scratch) + 4 * size_t(max_batch) * d_max) + 255) &
+        ~uintptr_t(255));
     // the vector length is cut in two when each part still has a k-block for every accumulator
     const int splits = (D + kTileK - 1) / kTileK >= kSplitK * kHeadRuns ? kSplitK : 1;
     *dots_out = dots;
@@ -346,19 +357,14 @@ cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const
     if (!make_map(&ma_hi, a_hi, B, D, kTileM) || !make_map(&ma_lo, a_lo, B, D, kTileM) ||
         !make_map(&mb_hi, b_hi, n, D, kTileN) || !make_map(&mb_lo, b_lo, n, D, kTileN))
         return cudaErrorInvalidValue;
+    if (sv_ready) {
+        const cudaError_t e = cudaStreamWaitEvent(st, sv_ready, 0);
+        if (e != cudaSuccess) return e;
+    }
     if (!sv_split_done) {
         ++*launches;
         const int grid_a = int(std::min<long long>(((long long)B * D / 4 + 255) / 256, 148 * 8));
-        const cudaError_t e = launch_chained(k_split_bf16, grid_a, 256, 0, st, sv, skip, B, D, a_hi, a_lo,
-                                             static_cast<const int*>(nullptr));
-        if (e != cudaSuccess) return e;
-    }
-    {  // always launched: whether the centres' split is current is a flag on the device (a replayed graph must not
-       // rely on what the host knew at capture); the kernel leaves at once when it is
-        ++*launches;
-        const int grid_b = int(std::min<long long>(((long long)n * D / 4 + 255) / 256, 148 * 8));
-        const cudaError_t e = launch_chained(k_split_bf16, grid_b, 256, 0, st, centers, static_cast<const uint8_t*>(nullptr), n, D, b_hi, b_lo,
-                                             static_cast<const int*>(centers_split_current));
+        const cudaError_t e = launch_chained(k_split_bf16, grid_a, 256, 0, st, sv, skip, B, D, a_hi, a_lo);
         if (e != cudaSuccess) return e;
     }
     ++*launches;

@@ -116,13 +116,13 @@ def test_argument_errors_launch_nothing():
 def test_c1_single_layer_fp32():
     rep = run_workload(si.C1)
     assert rep.exits == [8] and rep.band_mismatches == 0
-    assert rep.routes == [1, 0, 0, 0]       # one fused launch: pooling, Eq. 1, Eq. 3, Eq. 4 and the decision
+    assert rep.routes == [1, 0, 0, 0, 0]       # one fused launch: pooling, Eq. 1, Eq. 3, Eq. 4 and the decision
 
 
 def test_c2_resnet50_bf16_four_layers():
     rep = run_workload(si.C2)
     assert sum(rep.exits) > 30 and rep.frames == 64
-    assert rep.routes == [4, 0, 0, 0]
+    assert rep.routes == [4, 0, 0, 0, 0]
 
 
 def test_c2_exits_disabled_streams_every_layer():
@@ -143,7 +143,7 @@ def test_c3_mobilenetv2_fp16_nhwc_novel_classes_do_not_exit():
 def test_c4_large_cache_straddles_threshold():
     rep = run_workload(si.C4)
     assert 100 < rep.exits[0] < 900
-    assert rep.routes == [0, 1, 0, 0], "the 1000-entry fast memory must be scored on the tensor cores (Eq. 1 as a dense contraction)"
+    assert rep.routes == [0, 1, 0, 0, 0], "the 1000-entry fast memory must be scored on the tensor cores (Eq. 1 as a dense contraction)"
     print("c4 max |SA error|:", rep.max_sa_err, "max SV error:", rep.max_sv_err)
     print("c4 near-threshold lookups (oracle):", rep.near_oracle, "band mismatches:", rep.band_mismatches)
 
@@ -152,7 +152,7 @@ def test_c4_large_cache_straddles_threshold():
 def test_c5_streaming_full_width(T):
     rep = run_workload(si.C5, steps=T)
     assert rep.frames == 512 * T and rep.exits[0] > 0
-    assert rep.routes == [2 * T, 0, 0, 0]
+    assert rep.routes == [2 * T, 0, 0, 0, 0]
 
 
 def test_c5_full_length_64_steps_state_only():
@@ -182,11 +182,11 @@ def test_large_fast_memory_over_several_layers_uses_tensor_cores():
                     k_min=70, k_max=196, S=1, T=4, tau=0.8, window_W=2, sigma=0.6, zipf_s=0.9, repeat_p=0.3, seed=6)
     rep = run_workload(w)
     assert rep.frames == 70 * 4 and rep.lookups > 70
-    assert rep.routes == [0, 8, 0, 0]       # both layers of all four steps on the tensor-core route
+    assert rep.routes == [0, 8, 0, 0, 0]       # both layers of all four steps on the tensor-core route
     w3 = si.Workload("dense_nhwc", si.F16, si.NHWC, B=33, stages=((320, 7, 7),), n=72, k_init=72, k_min=72, k_max=72,
                      S=1, T=2, tau=0.8, sigma=1.0, zipf_s=1.0, seed=8)
     rep3 = run_workload(w3)
-    assert rep3.frames == 66 and rep3.routes == [0, 2, 0, 0]
+    assert rep3.frames == 66 and rep3.routes == [0, 2, 0, 0, 0]
 
 
 def test_forgetting_frequency_table_rapid_scene_change():
@@ -421,6 +421,68 @@ def test_maps_ready_flag_with_alternating_batches():
 
 DENSE_GRAPH = si.Workload("dense_graph", si.BF16, si.NCHW, B=70, stages=((256, 14, 14), (512, 7, 7)), n=196, k_init=100,
                            k_min=70, k_max=196, S=1, T=8, tau=0.8, window_W=2, sigma=0.6, zipf_s=0.9, repeat_p=0.3, seed=6)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("graph", [False, True], ids=["eager", "graph"])
+def test_maps_ready_flag_with_a_large_fast_memory(graph):
+    # SMTM_FLAG_MAPS_READY on a cache whose fast memory is scored on the tensor cores: the first layer's pooling
+    # of a step runs on the library's stream beside the previous step's decision kernel and update, into the
+    # other of two split buffers.  Steps run back to back (eagerly, or captured in one graph and replayed from
+    # a restored memory); results are those of the oracle.
+    from harness import Report, compare_state
+
+    w = DENSE_GRAPH
+    cents, counts = si.initial_centers(w)
+    tau = [w.tau] * w.L
+    mem = oracle.OracleMemory(w.n, w.dims, tau, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W)
+    cache = smtm.smtm_cache_create(w.n, w.dims, tau, cents, counts, n_streams=w.S, k_init=w.k_init, k_min=w.k_min,
+                                   k_max=w.k_max, window_W=w.window_W, max_batch=w.B, flags=smtm.FLAG_MAPS_READY)
+    sid = si.stream_ids(w)
+    gbs = [smtm.Batch(cache, w.B, stream_id=sid), smtm.Batch(cache, w.B, stream_id=sid)]
+    labs = si.labels(w)
+    maps = [[si.frames(w, l, labs[t], t, device="cuda") for l in range(w.L)] for t in range(w.T)]
+    fbs = [torch.from_numpy(si.fallback_labels(w, labs[t])).cuda() for t in range(w.T)]
+    torch.cuda.synchronize()
+
+    def steps(stream=None):
+        for t in range(w.T):
+            gb = gbs[t % 2]
+            smtm.smtm_lookup_exit_begin(cache, 0, smtm.Fmap(maps[t][0], w.dtype, w.layout, *si.shape4(w, 0)), gb, stream)
+            smtm.smtm_lookup_exit(cache, 1, smtm.Fmap(maps[t][1], w.dtype, w.layout, *si.shape4(w, 1)), gb, stream)
+            smtm.smtm_cache_update_resize(cache, gb, fbs[t], stream)
+
+    if graph:
+        blob = smtm.smtm_cache_export(cache)
+        st = torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=st):
+                steps(st.cuda_stream)
+            g.replay()
+            st.synchronize()                      # (the import below is not ordered on this stream)
+            smtm.smtm_cache_import(cache, blob)   # the replay that counts starts from the initial memory
+            g.replay()
+        st.synchronize()
+    else:
+        steps()
+    torch.cuda.synchronize()
+    for t in range(w.T):
+        ob = mem.new_batch(w.B, sid)
+        for l in range(w.L):
+            mem.lookup_exit(l, maps[t][l].cpu(), w.dtype, w.layout, si.shape4(w, l), ob)
+        mem.update(ob, si.fallback_labels(w, labs[t]))
+        mem.resize()
+    last = gbs[(w.T - 1) % 2]
+    assert np.array_equal(last.done.cpu().numpy(), ob["done"])
+    assert np.array_equal(last.pred.cpu().numpy(), ob["pred"])
+    assert np.array_equal(last.exit_layer.cpu().numpy(), ob["exit_layer"])
+    compare_state(w, cache, mem, Report())
+    routes = smtm.smtm_cache_get_routes(cache)
+    assert routes[smtm.ROUTE_PIPELINED_DENSE] == w.T and routes[smtm.ROUTE_DENSE] == w.T, routes
+    assert smtm.smtm_cache_status(cache) == 0
+    smtm.smtm_cache_destroy(cache)
+
 
 
 @pytest.mark.parametrize("w", [si.C5.scaled(T=8), DENSE_GRAPH], ids=["c5_full_width", "tensor_core_route"])
