@@ -276,20 +276,15 @@ class OracleRun:
 
 # --------------------------------------------------------------------------- the CUDA arm
 
-def maps_ready(w) -> bool:
-    return w.T > 1 or w.k_max > 64
-
-
 def make_cache(smtm, w, cents, counts):
-    # the streaming workload keeps its maps resident and alternates two carries: the library may pipeline its steps
-    # (so does the workload with the large fast memory; the others are served by the fused kernels, which the flag
-    # would take them off)
-    flags = (smtm.FLAG_FORGET_FT if w.forgetting else 0) | (smtm.FLAG_MAPS_READY if maps_ready(w) else 0)
+    # every workload here keeps its maps resident and alternates two carries: the library may pipeline its steps
+    # (it does where the shapes allow: NCHW maps; the NHWC workload stays on the one-kernel-per-layer route)
+    flags = (smtm.FLAG_FORGET_FT if w.forgetting else 0) | smtm.FLAG_MAPS_READY
     return smtm.smtm_cache_create(w.n, w.dims, [w.tau] * w.L, cents, counts, n_streams=w.S, k_init=w.k_init,
                                   k_min=w.k_min, k_max=w.k_max, window_W=w.window_W, max_batch=w.B, flags=flags)
 
 
-PROFILE_EVERY = 16  # every 16th step carries timing events and device-clock stamps (they cost a few us and break the chain of launches)
+PROFILE_EVERY = 20  # every 20th step carries timing events and device-clock stamps (they cost a few us and break the chain of launches)
 
 
 class Resident:
@@ -511,7 +506,7 @@ def run_ours(args):
                        "l2_policy": "distinct maps per step, %.0f MB per step (L2 is 126 MB)" % (m["res"].step_bytes / 1e6),
                        "state": "the memory is put back to its state after step W-1 (smtm_cache_import) right before the timed region",
                        "sharding": "streams across GPUs, no collective",
-                       "launch": "CUDA graphs of %d steps (per step: %d lookups, update+refresh), chained launches%s" % (m["G"], w.L, ", SMTM_FLAG_MAPS_READY with two alternating carries" if maps_ready(w) else "")},
+                       "launch": "CUDA graphs of %d steps (per step: %d lookups, update+refresh), chained launches, SMTM_FLAG_MAPS_READY with two alternating carries" % (m["G"], w.L)},
             "e2e": e2e,
             "gpu_launches": m["launches"],
             "clocks": m["clocks"],
@@ -675,6 +670,7 @@ def run_reference(args):
 
 
 def main():
+    global PROFILE_EVERY
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=60, help="timed steps; warm-up + steps = 64 walks the streaming workload once")
@@ -683,8 +679,11 @@ def main():
     ap.add_argument("--workload", default="c5", help="c1..c5 (prefix of a workload name); c5 is the benchmark of record")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle legs (profiling runs)")
     ap.add_argument("--no-other-workloads", action="store_true", help="skip the short passes of c1..c4")
+    ap.add_argument("--profile-every", type=int, default=PROFILE_EVERY,
+                    help="every N-th step of the timed region carries timing events and device-clock stamps")
     ap.add_argument("--rank-check", action="store_true", help="multi-rank plumbing only, on the host (gloo)")
     args = ap.parse_args()
+    PROFILE_EVERY = max(1, args.profile_every)
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:   # no launcher above us: start the ranks ourselves
         sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -34,9 +34,6 @@ struct smtm_cache {
     cudaStream_t pool_stream;
     cudaEvent_t ev_fork, ev_pool;       // the caller's stream -> pool stream, and back
     cudaEvent_t ev_mark[2];             // where the caller's stream stood at the last two first lookups (they alternate)
-    cudaEvent_t ev_scored;              // dense scoring of the pipelined route: the tensor-core kernel of the last first lookup is done
-    unsigned long long scored_capture;  // the capture ev_scored was recorded in (0 = none)
-    bool scored_valid;
     int split_which;                    // which of the two split buffers the batch under way uses (0 unless pipelined)
     unsigned long long mark_capture[2]; // the stream capture each was recorded in (0 = none)
     bool mark_valid[2];
@@ -129,7 +126,6 @@ void free_all(smtm_cache* c) {
     if (c->pool_stream) cudaStreamDestroy(c->pool_stream);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_pool) cudaEventDestroy(c->ev_pool);
-    if (c->ev_scored) cudaEventDestroy(c->ev_scored);
     for (cudaEvent_t e : c->ev_mark)
         if (e) cudaEventDestroy(e);
     cudaFree(c->d_jobs);
@@ -197,6 +193,10 @@ constexpr int kPipelinedRingConsumers = 3;
 // Copies the pooling kernel keeps outstanding per SM on this route (148 x 2 x 25 KB = 7.4 MB in flight; more did not
 // make it faster beside the latency-bound kernels, and every access those make to memory queues behind them).
 constexpr int kPipelinedInFlight = 2;
+// The same route with the tensor-core scorer: its ring of two stages (129 KB) and a pooling ring of three (77 KB)
+// share an SM.
+constexpr int kPipelinedDenseRingStages = 3;
+constexpr int kPipelinedDenseTcStages = 2;
 
 // The capture the stream is in (0 = none).
 cudaError_t capture_of(cudaStream_t st, unsigned long long* id) {
@@ -217,10 +217,10 @@ cudaError_t capture_of(cudaStream_t st, unsigned long long* id) {
 // is forked from the caller's stream where it stands.
 //
 // With a large fast memory (dense) the scoring is the tensor-core kernel and the decision kernel after it.  The
-// CTAs of the tensor-core kernel need most of an SM's shared memory and cannot sit beside a pooling CTA, so the
-// next batch's pooling is also ordered after that kernel (else whichever of the two came second would wait for
-// the other to leave the SMs, and the step's latency-bound kernels with it); it runs beside the decision kernel
-// and the update.  The vectors' bf16 split alternates between two buffers like the batches do.
+// tensor-core kernel gets a ring of two stages and the pooling kernel one of three, so that a CTA of each fits on
+// an SM: the next batch's pooling starts as soon as this batch's is done and runs beside all of this batch's
+// kernels.  The decision kernel is launched in stream order (see launch_ordered).  The vectors' bf16 split
+// alternates between two buffers like the batches do.
 smtm_status_t pooled_first_lookup(smtm_cache* c, const EncodeArgs& e, const LookupArgs& a, cudaStream_t st,
                                   const cudaEvent_t* timing, bool profiled_step, bool dense) {
     unsigned long long cap = 0, pool_cap = 0;
@@ -234,15 +234,13 @@ smtm_status_t pooled_first_lookup(smtm_cache* c, const EncodeArgs& e, const Look
         SMTM_CUDA(cudaEventRecord(c->ev_fork, st));
         SMTM_CUDA(cudaStreamWaitEvent(c->pool_stream, c->ev_fork, 0));
     }
-    if (dense && c->scored_valid && c->scored_capture == cap && wait_prev)
-        SMTM_CUDA(cudaStreamWaitEvent(c->pool_stream, c->ev_scored, 0));
     SMTM_CUDA(cudaEventRecord(c->ev_mark[cur], st));
     c->mark_capture[cur] = cap;
     c->mark_valid[cur] = true;
     c->mark_next = prev;
     EncodeArgs ep = e;
     ep.skip = nullptr;  // the batch starts here: every frame is in
-    ep.ring_stages = kPipelinedRingStages;
+    ep.ring_stages = dense ? kPipelinedDenseRingStages : kPipelinedRingStages;
     ep.ring_consumers = kPipelinedRingConsumers;
     ep.ring_in_flight = kPipelinedInFlight;
     if (profiled_step && a.layer == 0 && ep.clock)  // the caller's stream clears the step's other stamps at a time of its own
@@ -265,11 +263,8 @@ smtm_status_t pooled_first_lookup(smtm_cache* c, const EncodeArgs& e, const Look
     float *dots = nullptr, *dots2 = nullptr;
     SMTM_CUDA(launch_dense_dots(a.sv, nullptr, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max, cur, sv_split,
                                 c->ev_pool, c->d_cen_split[a.layer], &dots, &dots2, c->d_status,
-                                a.clock ? a.clock + 2 * SMTM_PROF_SCORE_TC : nullptr, st, &c->launches));
-    SMTM_CUDA(cudaEventRecord(c->ev_scored, st));
-    c->scored_capture = cap;
-    c->scored_valid = true;
-    SMTM_CUDA(launch_finish_dense(a, dots, dots2, st, &c->launches));
+                                a.clock ? a.clock + 2 * SMTM_PROF_SCORE_TC : nullptr, kPipelinedDenseTcStages, st, &c->launches));
+    SMTM_CUDA(launch_finish_dense(a, dots, dots2, true, st, &c->launches));
     return SMTM_OK;
 }
 
@@ -366,8 +361,8 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
         float *dots = nullptr, *dots2 = nullptr;
         SMTM_CUDA(launch_dense_dots(a.sv, a.fresh ? nullptr : a.done, a.B, a.centers, a.n, a.D, c->d_dense, c->max_batch, c->d_max,
                                     c->split_which, sv_split, nullptr, c->d_cen_split[layer], &dots, &dots2, c->d_status,
-                                    a.clock ? a.clock + 2 * SMTM_PROF_SCORE_TC : nullptr, st, &c->launches));
-        SMTM_CUDA(launch_finish_dense(a, dots, dots2, st, &c->launches));
+                                    a.clock ? a.clock + 2 * SMTM_PROF_SCORE_TC : nullptr, 0, st, &c->launches));
+        SMTM_CUDA(launch_finish_dense(a, dots, dots2, false, st, &c->launches));
         return SMTM_OK;
     }
     SMTM_CUDA(launch_score_exit(a, st, &c->launches));
@@ -548,7 +543,6 @@ smtm_status_t smtm_cache_create(const smtm_config_t* cfg, const float* const* h_
     ok = ok && cudaStreamCreateWithFlags(&c->pool_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_pool, cudaEventDisableTiming) == cudaSuccess;
-    ok = ok && cudaEventCreateWithFlags(&c->ev_scored, cudaEventDisableTiming) == cudaSuccess;
     for (cudaEvent_t& e : c->ev_mark) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) {
         (void)cudaGetLastError();

@@ -1364,7 +1364,9 @@ cudaError_t launch_lookup_sparse(const EncodeArgs& e, const LookupArgs& a, int s
     const size_t smem = sparse_smem(f.e.chunk_channels);
     cudaError_t err = cudaSuccess;
     ++*launches;
-#define SMTM_LAUNCH(...) err = launch_chained_cluster(k_lookup_sparse<__VA_ARGS__>, P * groups, kLightThreads, smem, P, st, f)
+    // (in stream order, without the early start: the clusters would wait on the SMs for the scoring kernel before
+    // them and keep the next step's pooling CTAs out meanwhile)
+#define SMTM_LAUNCH(...) err = launch_ordered_cluster(k_lookup_sparse<__VA_ARGS__>, P * groups, kLightThreads, smem, P, st, f)
     SMTM_FOR_REDUCER(r, SMTM_LAUNCH)
 #undef SMTM_LAUNCH
     return err;

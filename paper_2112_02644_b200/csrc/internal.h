@@ -21,7 +21,7 @@ inline cudaError_t record_timing(cudaEvent_t ev, cudaStream_t st) {
 // Launches `kernel` so that it may start while the previous kernel of the stream is finishing
 // (programmatic stream serialisation); the kernel itself waits with chain_wait() before it
 // touches global memory.
-template <class... Params, class... Args>
+template <bool kEarly = true, class... Params, class... Args>
 cudaError_t launch_chained_cluster(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, int cluster_x,
                                    cudaStream_t st, Args&&... args) {
     cudaLaunchConfig_t cfg{};
@@ -31,7 +31,7 @@ cudaError_t launch_chained_cluster(void (*kernel)(Params...), dim3 grid, dim3 bl
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = kEarly ? 1 : 0;
     attr[1].id = cudaLaunchAttributeClusterDimension;  // thread-block clusters of cluster_x consecutive CTAs
     attr[1].val.clusterDim.x = unsigned(cluster_x);
     attr[1].val.clusterDim.y = 1;
@@ -45,6 +45,24 @@ template <class... Params, class... Args>
 cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
                            Args&&... args) {
     return launch_chained_cluster(kernel, grid, block, smem, 1, st, static_cast<Args&&>(args)...);
+}
+
+// The same launch without the early start.  A kernel launched with launch_chained becomes resident as soon as
+// every CTA of the kernel before it has called chain_release(), and its CTAs then sit in chain_wait() holding
+// their registers and shared memory.  On the pipelined route that is harmful for a kernel of many CTAs that
+// follows a long one: while they wait they keep the CTAs of the next step's pooling kernel, which comes from the
+// other stream at about the same time, off the SMs.  Such a kernel is launched in stream order instead; it costs
+// it a microsecond.
+template <class... Params, class... Args>
+cudaError_t launch_ordered_cluster(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, int cluster_x,
+                                   cudaStream_t st, Args&&... args) {
+    return launch_chained_cluster<false>(kernel, grid, block, smem, cluster_x, st, static_cast<Args&&>(args)...);
+}
+
+template <class... Params, class... Args>
+cudaError_t launch_ordered(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                           Args&&... args) {
+    return launch_chained_cluster<false>(kernel, grid, block, smem, 1, st, static_cast<Args&&>(args)...);
 }
 
 // Number of exit layers and the fast-memory capacity of a cache.
@@ -163,18 +181,21 @@ size_t dense_scratch_bytes(int max_batch, int n, int d_max);
 // an event `st` has to wait for before it reads the vectors or their split (the pooling of the pipelined route).
 // centers_split holds the same split of the centres ([n][D] heads, then [n][D] tails, D a multiple of 4): made by
 // launch_centers_split whenever the centres are set as a whole, and kept in step by Eq. 7's kernel afterwards.
+// ring_stages: 0 = the default depth of the operand ring; fewer stages leave shared memory to a kernel beside it.
 void dense_sv_split(void* scratch, int max_batch, int d_max, int which, void** hi, void** lo);
 cudaError_t launch_centers_split(const float* centers, int n, int D, void* centers_split, cudaStream_t st,
                                  int64_t* launches);
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
                               void* scratch, int max_batch, int d_max, int which, bool sv_split_done,
                               cudaEvent_t sv_ready, void* centers_split, float** dots_out, float** dots2_out,
-                              int* status, unsigned long long* clock, cudaStream_t st, int64_t* launches);
+                              int* status, unsigned long long* clock, int ring_stages, cudaStream_t st,
+                              int64_t* launches);
 size_t dense_centers_split_bytes(int n, int D);
 // Eq. 1 from the dot products, Eq. 3, top-2, Eq. 4 / Eq. 2 and the exit rule; dots: [B][n], and dots2
 // (nullptr, or [B][n]: the second half of the vector length, added to the first).
-cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, cudaStream_t st,
-                                int64_t* launches);
+// beside_pooling: the next batch's pooling kernel runs meanwhile (launched in stream order, see launch_ordered).
+cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, bool beside_pooling,
+                                cudaStream_t st, int64_t* launches);
 // One warp that waits, bounded, on a barrier nobody arrives on (the self-test of the time-out path).
 cudaError_t launch_wait_selftest(int* status, cudaStream_t st, int64_t* launches);
 cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, int32_t* pred, int B, int k_max,

@@ -46,10 +46,6 @@ __global__ void __launch_bounds__(kThreads) k_score_exit(const LookupArgs a) {
     score_frame(a, b, pf, sv, nrm, s_cur, s_acc);
 }
 
-// Finishing kernel of the tensor-core path: one CTA per frame turns the frame's row of dot
-// products into similarities of its fast-memory slots and decides.  Every thread keeps the
-// two best of its own slots as 64-bit ranking keys; warps merge by two warp-wide maxima, the
-// CTA through shared memory.  With a.fresh the carry is taken as SA = 0, nobody done.
 // The best two keys of the CTA, valid in thread 0.  (b1, b2): this thread's best two; s_keys: [2 * warps].
 __device__ __forceinline__ Top2 block_top2_keys(unsigned long long b1, unsigned long long b2, unsigned long long* s_keys) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -71,66 +67,87 @@ __device__ __forceinline__ Top2 block_top2_keys(unsigned long long b1, unsigned 
     return t;
 }
 
+// Finishing kernel of the tensor-core path: one CTA per frame turns the frame's row of dot products into
+// similarities of its fast-memory slots and decides.  The row (both halves of the vector length added) and the
+// centres' lengths come in with coalesced 16-byte loads and are parked in shared memory, from where the slots
+// pick their class's entry: a gather straight from global memory costs a sector per slot, and a thousand slots
+// for each of a thousand frames are then bound by that.  Everything a frame needs after its stream id is fetched
+// in one trip: the size and the members of its fast memory, the carries, the row, the lengths and the semantic
+// vector (for its length).  Every thread keeps the two best of its own slots as 64-bit ranking keys; warps merge
+// by two warp-wide maxima, the CTA through shared memory.  With a.fresh the carry is taken as SA = 0, nobody done.
+constexpr int kFinishSlots = 8;  // slots a thread fetches per trip
+
 __global__ void __launch_bounds__(kFinishThreads, 8) k_finish_dense(const LookupArgs a, const float* __restrict__ dots,
-                                                           const float* __restrict__ dots2) {
+                                                                    const float* __restrict__ dots2) {
+    extern __shared__ float s_row[];  // [n] dot products, then [n] lengths of the centres
     __shared__ float scratch[32];
     __shared__ unsigned long long s_keys[2 * (kFinishThreads / kWarp)];
     chain_wait();
     chain_release();
     const ClockScope stamps(a.clock ? a.clock + 2 * SMTM_PROF_FINISH_DENSE : nullptr);
-    const int b = blockIdx.x;
-    if (!a.fresh && a.done[b]) return;
-    const int tid = threadIdx.x;
-    const int sid = stream_of(a, b);
-    const int k = sid < 0 ? 0 : a.k[sid];  // a stream id outside the cache: nothing to score against
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int gone = a.fresh ? 0 : a.done[b];
+    const int sid = stream_of(a, b);  // (in flight with the flag)
+    if (gone) return;
+    float* s_len = s_row + a.n;
     const int32_t* mem = a.members + (size_t)max(sid, 0) * a.k_max;
-    const float* row = a.sv + (size_t)b * a.D;
-    const float weight = float(1u << a.layer);
-    const float* __restrict__ drow = dots + (size_t)b * a.n;
-    const float* __restrict__ drow2 = dots2 ? dots2 + (size_t)b * a.n : nullptr;  // second half of the vector length
-    const float* __restrict__ clen = a.cnorm;
     float* sa_row = a.sa + (size_t)b * a.k_max;
+    const float weight = float(1u << a.layer);
+    // this trip: the fast memory's size, the first slots' classes and carries (unconditional: up to k_max) ...
+    const int k = sid < 0 ? 0 : a.k[sid];  // a stream id outside the cache: nothing to score against
+    int cls[kFinishSlots];
+    float old[kFinishSlots];
+#pragma unroll
+    for (int u = 0; u < kFinishSlots; ++u) {
+        const int j = min(u * kFinishThreads + tid, a.k_max - 1);
+        cls[u] = mem[j];
+        old[u] = a.fresh ? 0.f : sa_row[j];
+    }
+    // ... the row of dot products and the lengths (n is a multiple of 4 on this route) ...
+    const float4* drow = reinterpret_cast<const float4*>(dots + (size_t)b * a.n);
+    const float4* drow2 = dots2 ? reinterpret_cast<const float4*>(dots2 + (size_t)b * a.n) : nullptr;
+    const float4* clen = reinterpret_cast<const float4*>(a.cnorm);
+    for (int c4 = tid; c4 < a.n / 4; c4 += kFinishThreads) {
+        float4 d = drow[c4];
+        if (drow2) {  // second half of the vector length
+            const float4 e = drow2[c4];
+            d.x += e.x; d.y += e.y; d.z += e.z; d.w += e.w;
+        }
+        reinterpret_cast<float4*>(s_row)[c4] = d;
+        reinterpret_cast<float4*>(s_len)[c4] = clen[c4];
+    }
+    // ... and the squared length of the semantic vector (D is a multiple of 8 on this route)
+    const float4* row4 = reinterpret_cast<const float4*>(a.sv + (size_t)b * a.D);
+    float q[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int d = tid; d < a.D / 4; d += kFinishThreads) {
+        const float4 v = row4[d];
+        q[0] = fmaf(v.x, v.x, q[0]);
+        q[1] = fmaf(v.y, v.y, q[1]);
+        q[2] = fmaf(v.z, v.z, q[2]);
+        q[3] = fmaf(v.w, v.w, q[3]);
+    }
+    const float nrm = block_sum((q[0] + q[1]) + (q[2] + q[3]), scratch);  // (also orders the shared writes above)
+    const float sv_len = __fsqrt_rn(nrm);
     unsigned long long a1 = 0ull, a2 = 0ull, c1 = 0ull, c2 = 0ull;  // best two cumulative / single-layer keys
-    float nrm = 0.f, sv_len = 0.f;
-    for (int j0 = 0; j0 < k; j0 += 4 * kFinishThreads) {  // four slots per thread, every load issued before any store
-        int cls[4];
-        float dot[4], cl[4], old[4];
+    for (int j0 = 0; j0 < k; j0 += kFinishSlots * kFinishThreads) {
+        if (j0 > 0) {  // a fast memory of more than 1024 slots: one more trip per 1024
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int j = j0 + u * kFinishThreads + tid;
-            cls[u] = mem[min(j, k - 1)];
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int j = j0 + u * kFinishThreads + tid;
-            dot[u] = drow[cls[u]];
-            if (drow2) dot[u] += drow2[cls[u]];
-            cl[u] = clen[cls[u]];
-            old[u] = (j < k && !a.fresh) ? sa_row[j] : 0.f;
-        }
-        if (j0 == 0) {  // the squared length of the semantic vector, while the loads above are in flight
-            const float4* row4 = reinterpret_cast<const float4*>(row);  // (D is a multiple of 8 on this route)
-            float q[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int d = tid; d < a.D / 4; d += kFinishThreads) {
-                const float4 v = row4[d];
-                q[0] = fmaf(v.x, v.x, q[0]);
-                q[1] = fmaf(v.y, v.y, q[1]);
-                q[2] = fmaf(v.z, v.z, q[2]);
-                q[3] = fmaf(v.w, v.w, q[3]);
+            for (int u = 0; u < kFinishSlots; ++u) {
+                const int j = min(j0 + u * kFinishThreads + tid, a.k_max - 1);
+                cls[u] = mem[j];
+                old[u] = a.fresh ? 0.f : sa_row[j];
             }
-            nrm = (q[0] + q[1]) + (q[2] + q[3]);
-            nrm = block_sum(nrm, scratch);
-            sv_len = __fsqrt_rn(nrm);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kFinishSlots; ++u) {
             const int j = j0 + u * kFinishThreads + tid;
             if (j < k) {
-                const float s = (nrm == 0.f || cl[u] == 0.f) ? 0.f : __fdiv_rn(dot[u], __fmul_rn(sv_len, cl[u]));  // Eq. 1
-                const float acc = __fmaf_rn(s, weight, old[u]);    // Eq. 3
+                const float dot = s_row[cls[u]], cl = s_len[cls[u]];
+                const float sim = (nrm == 0.f || cl == 0.f) ? 0.f : __fdiv_rn(dot, __fmul_rn(sv_len, cl));  // Eq. 1
+                const float acc = __fmaf_rn(sim, weight, old[u]);                                              // Eq. 3
                 sa_row[j] = acc;
                 keep_two(rank_key(acc, cls[u]), a1, a2);
-                if (a.sep) keep_two(rank_key(s, cls[u]), c1, c2);  // only Eq. 2 (a diagnostic) needs it
+                if (a.sep) keep_two(rank_key(sim, cls[u]), c1, c2);  // only Eq. 2 (a diagnostic) needs it
             }
         }
     }
@@ -179,6 +196,7 @@ cudaError_t lookup_setup() {
     cudaError_t e = allow_max_dynamic_smem(k_score_exit);
     if (e == cudaSuccess) e = prefer_max_smem_carveout(k_score_exit);
     if (e == cudaSuccess) e = prefer_max_smem_carveout(k_finish_dense);
+    if (e == cudaSuccess) e = allow_max_dynamic_smem(k_finish_dense);  // (two words per class: 64 KB at 8192 classes)
     return e;
 }
 
@@ -191,11 +209,13 @@ cudaError_t launch_batch_reset(float* sa, uint8_t* done, int32_t* exit_layer, in
     return launch_chained(k_batch_reset, grid, 256, 0, st, sa, done, exit_layer, pred, B, n_sa);
 }
 
-cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2,
+cudaError_t launch_finish_dense(const LookupArgs& a, const float* dots, const float* dots2, bool beside_pooling,
                                 cudaStream_t st, int64_t* launches) {
     if (a.B <= 0) return cudaSuccess;
     ++*launches;
-    return launch_chained(k_finish_dense, a.B, kFinishThreads, 0, st, a, dots, dots2);
+    const size_t smem = 2 * size_t(a.n) * sizeof(float);
+    if (beside_pooling) return launch_ordered(k_finish_dense, a.B, kFinishThreads, smem, st, a, dots, dots2);
+    return launch_chained(k_finish_dense, a.B, kFinishThreads, smem, st, a, dots, dots2);
 }
 
 cudaError_t launch_score_exit(const LookupArgs& a, cudaStream_t st, int64_t* launches, int threads) {

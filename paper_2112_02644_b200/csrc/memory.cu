@@ -336,6 +336,86 @@ __device__ __forceinline__ unsigned long long sort_one_key_per_thread(unsigned l
     return key;
 }
 
+// Descending bitonic sort of PER keys per thread (thread t holds elements t * PER ... in key[]; blockDim.x * PER a
+// power of two; every thread of the CTA calls).  A compare-exchange whose partner sits in the same thread is done
+// in registers, one up to 31 threads away by warp shuffle, the few beyond through shared memory (s_x: a word per
+// element, laid out [register][thread]).
+template <int PER>
+__device__ __forceinline__ void sort_keys_in_registers(unsigned long long (&key)[PER], unsigned long long* s_x) {
+    const int tid = threadIdx.x, nt = blockDim.x, P = nt * PER;
+    for (int k = 2; k <= P; k <<= 1) {
+        for (int j = k >> 1; j >= PER; j >>= 1) {
+            const int tj = j / PER;
+            // the lower element of a pair keeps the larger key where the run is descending, the smaller one elsewhere
+            const bool larger = ((tid & tj) == 0) == (((tid * PER) & k) == 0);
+            if (tj < kWarp) {
+#pragma unroll
+                for (int i = 0; i < PER; ++i) {
+                    const unsigned long long other = __shfl_xor_sync(kFull, key[i], tj);
+                    key[i] = larger ? max(key[i], other) : min(key[i], other);
+                }
+            } else {
+                __syncthreads();  // the previous round's readers are done
+#pragma unroll
+                for (int i = 0; i < PER; ++i) s_x[i * nt + tid] = key[i];
+                __syncthreads();
+#pragma unroll
+                for (int i = 0; i < PER; ++i) {
+                    const unsigned long long other = s_x[i * nt + (tid ^ tj)];
+                    key[i] = larger ? max(key[i], other) : min(key[i], other);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = PER >> 1; j > 0; j >>= 1) {
+            if (j < k) {
+#pragma unroll
+                for (int i = 0; i < PER; ++i)
+                    if ((i & j) == 0) {
+                        const bool desc = ((tid * PER + i) & k) == 0;
+                        const unsigned long long hi = max(key[i], key[i | j]), lo = min(key[i], key[i | j]);
+                        key[i] = desc ? hi : lo;
+                        key[i | j] = desc ? lo : hi;
+                    }
+            }
+        }
+    }
+}
+
+// Eq. 5 / Eq. 6 for stream s from the scores of PER consecutive classes per thread (c_lo ...), by a sort in
+// registers: for memories of so many classes that most scores are non-zero and ranking by counting would cost
+// a pass over all keys per key.  The key of a class is one more than its ranking key, so that classes with a zero
+// score sort behind the others in ascending id (as the refresh wants them) and before the padding.
+// `dyn`: blockDim.x * PER words for the sort, then the k_max best scores.
+template <int PER>
+__device__ void refresh_sorted_in_registers(const ResizeArgs& a, int s, const unsigned long long (&sc)[PER], int c_lo,
+                                            unsigned char* dyn, unsigned long long* s_part) {
+    const int tid = threadIdx.x, P = blockDim.x * PER;
+    unsigned long long* s_x = reinterpret_cast<unsigned long long*>(dyn);  // [P]
+    unsigned long long* s_top = s_x + P;                                    // [k_max]
+    unsigned long long key[PER], local = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int c = c_lo + i;
+        key[i] = c < a.n ? refresh_key(sc[i], c) + 1ull : 0ull;
+        local += c < a.n ? sc[i] : 0ull;
+    }
+    const unsigned long long total = block_sum_u64(local, s_part);
+    if (total == 0) return;  // nothing seen yet: keep size and members (the same for every thread)
+    sort_keys_in_registers<PER>(key, s_x);
+    int32_t* mem = a.members + (size_t)s * a.k_max;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int r = tid * PER + i;
+        if (r < a.k_max && r < a.n) {
+            mem[r] = key_class(key[i] - 1ull);
+            s_top[r] = key_score(key[i] - 1ull);
+        }
+    }
+    __syncthreads();
+    if (tid < kWarp) adaptive_size(a, s, s_top, total, tid);
+}
+
 // Eq. 5 / Eq. 6 for stream s when every thread of the CTA holds the scores of its PER consecutive classes
 // (c_lo ...) in registers.  The keys of the non-zero scores are appended to a list in shared memory in whatever
 // order the threads come (a key carries its class, and ranking by key does not care about the list's order);
@@ -695,7 +775,9 @@ __device__ void tables_of_frame(const UpdateArgs& a, const ResizeArgs& rz, int g
     }
     if (do_resize) {
         __syncthreads();  // every thread is done with the closed form's arrays (and sees its own table entries)
-        if (PER)
+        if (PER == 8)
+            refresh_sorted_in_registers<(PER ? PER : 1)>(rz, s, sc, c_lo, dyn, s_part);
+        else if (PER)
             refresh_from_registers<(PER ? PER : 1)>(rz, s, sc, c_lo, dyn, &s_scan[32], &s_part[31]);
         else
             refresh_stream(rz, s, dyn, s_scan, s_part);
@@ -707,6 +789,7 @@ __device__ void tables_of_frame(const UpdateArgs& a, const ResizeArgs& rz, int g
 constexpr int kCenPer = 8;                         // consecutive frames a thread looks at
 constexpr int kCenTile = kCenPer * kApplyThreads;  // frames listed at a time
 constexpr int kRowGroupsMax = 8;
+constexpr int kWideSweeps = 4;                     // an item up to this many times as wide as the CTA is folded in one go
 
 // Lists, in ascending index, the frames base .. base + kCenTile - 1 whose label is cls and that stopped at
 // layer l0 + 1 or deeper; returns how many (the same in every thread).  Every thread fetches the codes of its
@@ -737,6 +820,35 @@ __device__ __forceinline__ int list_pair_frames(const UpdateArgs& a, int base, i
     return cnt;
 }
 
+// Eq. 7 for one 16-byte group of columns of a centre: SC = (SC m + sum SV) / (m + q), in double (the count is
+// exact at any size and SC m + sum SV is rounded once; inv = 1 / (m + q)); the tensor-core scorer's bf16 copy of
+// the centre, where there is one, follows it (x = hi + lo).  Returns the group's part of the squared length.
+__device__ __forceinline__ float fold_centre(const UpdateArgs& a, int l0, int cls, int D, int c4, const float4& old,
+                                             const float (&acc)[4], double dm, double inv, float* cen) {
+    float4 v;
+    v.x = float((double(old.x) * dm + double(acc[0])) * inv);
+    v.y = float((double(old.y) * dm + double(acc[1])) * inv);
+    v.z = float((double(old.z) * dm + double(acc[2])) * inv);
+    v.w = float((double(old.w) * dm + double(acc[3])) * inv);
+    *reinterpret_cast<float4*>(cen + 4 * c4) = v;
+    if (a.cen_split[l0]) {
+        __nv_bfloat16* hi = a.cen_split[l0] + (size_t)cls * D + 4 * c4;
+        __nv_bfloat16* lo = hi + (size_t)a.n * D;
+        const float x[4] = {v.x, v.y, v.z, v.w};
+        __nv_bfloat16 h[4], t[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            h[j] = __float2bfloat16_rn(x[j]);
+            t[j] = __float2bfloat16_rn(x[j] - __bfloat162float(h[j]));
+        }
+        *reinterpret_cast<uint2*>(hi) = *reinterpret_cast<const uint2*>(h);
+        *reinterpret_cast<uint2*>(lo) = *reinterpret_cast<const uint2*>(t);
+    }
+    float nrm = 0.f;
+    nrm = fmaf(v.x, v.x, nrm); nrm = fmaf(v.y, v.y, nrm); nrm = fmaf(v.z, v.z, nrm); nrm = fmaf(v.w, v.w, nrm);
+    return nrm;
+}
+
 // Eq. 7 for one item: the columns [block's share] of the centre of (layer l0, class cls).  The frames whose
 // label is cls and that stopped at layer l0 + 1 or deeper are listed in ascending index, a tile of frames at a
 // time (every thread looks at a run of consecutive frames, one scan over the threads).  A thread is (a 16-byte
@@ -762,7 +874,33 @@ __device__ void centre_item(const UpdateArgs& a, int item, const int (&first_til
         while (R < kRowGroupsMax && 2 * R * (hi4 - lo4) <= nt) R *= 2;
         const int cpp = nt / R;                                                // column groups per sweep
         const int rg = tid / cpp, c = tid - rg * cpp;
-        for (int s4 = lo4; s4 < hi4; s4 += cpp) {  // (one sweep unless the item is wider than the CTA)
+        const int sweeps = (hi4 - lo4 + cpp - 1) / cpp;
+        const bool wide = sweeps > 1 && sweeps <= kWideSweeps && a.B <= kCenTile;  // (more than one sweep: R == 1)
+        if (wide) {
+            // An item a few times as wide as the CTA whose frames fit one listing (the usual pair: a row or two of
+            // a long vector): the frames are listed once, and a thread has its column groups of two sweeps in
+            // flight together, a row at a time.  Same order of additions as below.
+            const int cnt = list_pair_frames(a, 0, cls, l0, s_list, s_scan, first_tile);
+            q = cnt;
+            const double dm = double(m), inv = 1.0 / (dm + double(q));
+            for (int w0 = 0; w0 < sweeps && q > 0; w0 += 2) {
+                const int ca = lo4 + w0 * nt + tid, cb = ca + nt;
+                const int la = min(ca, hi4 - 1), lb = min(cb, hi4 - 1);  // unconditional loads (past the item's end: its last group)
+                float acc_a[4] = {0.f, 0.f, 0.f, 0.f}, acc_b[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+                for (int i = 0; i < cnt; ++i) {
+                    const float4* rp = reinterpret_cast<const float4*>(sv + (size_t)s_list[i] * D);
+                    const float4 ra = __ldg(rp + la), rb = __ldg(rp + lb);
+                    acc_a[0] += ra.x; acc_a[1] += ra.y; acc_a[2] += ra.z; acc_a[3] += ra.w;
+                    acc_b[0] += rb.x; acc_b[1] += rb.y; acc_b[2] += rb.z; acc_b[3] += rb.w;
+                }
+                const float4 old_a = *reinterpret_cast<const float4*>(cen + 4 * la);
+                const float4 old_b = *reinterpret_cast<const float4*>(cen + 4 * lb);
+                if (ca < hi4) nrm += fold_centre(a, l0, cls, D, ca, old_a, acc_a, dm, inv, cen);
+                if (cb < hi4) nrm += fold_centre(a, l0, cls, D, cb, old_b, acc_b, dm, inv, cen);
+            }
+        }
+        for (int s4 = lo4; s4 < hi4 && !wide; s4 += cpp) {  // (one sweep unless the item is wider than the CTA)
             const int c4 = s4 + c;
             const bool mine_col = c4 < hi4;
             float4 old = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -795,28 +933,8 @@ __device__ void centre_item(const UpdateArgs& a, int item, const int (&first_til
                     const float4 o = s_acc[(g2 - 1) * cpp + c];
                     acc[0] += o.x; acc[1] += o.y; acc[2] += o.z; acc[3] += o.w;
                 }
-                // Eq. 7 in double: the count is exact at any size and SC m + sum SV is rounded once
                 const double dm = double(m), inv = 1.0 / (dm + double(q));
-                float4 v;
-                v.x = float((double(old.x) * dm + double(acc[0])) * inv);
-                v.y = float((double(old.y) * dm + double(acc[1])) * inv);
-                v.z = float((double(old.z) * dm + double(acc[2])) * inv);
-                v.w = float((double(old.w) * dm + double(acc[3])) * inv);
-                *reinterpret_cast<float4*>(cen + 4 * c4) = v;
-                if (a.cen_split[l0]) {  // the tensor-core scorer's copy of the centre follows it (x = hi + lo in bf16)
-                    __nv_bfloat16* hi = a.cen_split[l0] + (size_t)cls * D + 4 * c4;
-                    __nv_bfloat16* lo = hi + (size_t)a.n * D;
-                    const float x[4] = {v.x, v.y, v.z, v.w};
-                    __nv_bfloat16 h[4], t[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        h[j] = __float2bfloat16_rn(x[j]);
-                        t[j] = __float2bfloat16_rn(x[j] - __bfloat162float(h[j]));
-                    }
-                    *reinterpret_cast<uint2*>(hi) = *reinterpret_cast<const uint2*>(h);
-                    *reinterpret_cast<uint2*>(lo) = *reinterpret_cast<const uint2*>(t);
-                }
-                nrm = fmaf(v.x, v.x, nrm); nrm = fmaf(v.y, v.y, nrm); nrm = fmaf(v.z, v.z, nrm); nrm = fmaf(v.w, v.w, nrm);
+                nrm += fold_centre(a, l0, cls, D, c4, old, acc, dm, inv, cen);
             }
         }
     } else {
@@ -951,7 +1069,7 @@ cudaError_t launch_update(const UpdateArgs& a, const ResizeArgs* rz, int sm_coun
     // keys is 55 rounds of compare-exchange: a round per barrier with 1024 threads, eight times that with the 128
     // threads of a tables CTA); it refreshes every stream, which gives the streams without a frame in the batch
     // the fast memory they already have.
-    const bool refresh_apart = tables && rz && a.n > 4 * kApplyThreads;
+    const bool refresh_apart = tables && rz && a.n > 8 * kApplyThreads;
     const bool refresh_here = tables && rz && !refresh_apart;
     const size_t smem = tables ? tables_smem(a.n, rz ? rz->k_max : 0, refresh_here) : 0;
     ++*launches;

@@ -122,6 +122,7 @@ struct TcParams {
     size_t split_stride;  // floats between the result arrays of two parts
     int* status;
     unsigned long long* clock;  // nullptr, or two words for the device-clock stamps
+    int stages;                 // depth of the operand ring, 2 .. kTcStages
 };
 
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -130,9 +131,10 @@ k_score_tc(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__
            const TcParams p) {
     extern __shared__ uint8_t tc_smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* full = reinterpret_cast<uint64_t*>(base + size_t(kTcStages) * kStageBytes);  // [kTcStages]
-    uint64_t* empty = full + kTcStages;                                                    // [kTcStages]
-    uint64_t* acc_full = empty + kTcStages;                                                // [1]
+    const int stages = p.stages;
+    uint64_t* full = reinterpret_cast<uint64_t*>(base + size_t(stages) * kStageBytes);  // [stages]
+    uint64_t* empty = full + stages;                                                    // [stages]
+    uint64_t* acc_full = empty + stages;                                                // [1]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -143,7 +145,7 @@ k_score_tc(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__
     const int n_kb = (int(blockIdx.z) + 1) * n_kb_all / int(gridDim.z) - kb0;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kTcStages; ++s) {
+        for (int s = 0; s < stages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
@@ -170,8 +172,8 @@ k_score_tc(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__
         // ---- producer: four tiles per k-block ---------------------------------------------------
         if (lane == 0) {
             for (int kb = 0; kb < n_kb; ++kb) {
-                const int s = kb % kTcStages;
-                const uint32_t use = uint32_t(kb / kTcStages);
+                const int s = kb % stages;
+                const uint32_t use = uint32_t(kb / stages);
                 if (use > 0 && !mbar_wait_bounded(&empty[s], (use - 1) & 1, p.status)) { failed = true; break; }
                 uint8_t* st = base + size_t(s) * kStageBytes;
                 mbar_expect_tx(&full[s], kStageBytes);
@@ -189,8 +191,8 @@ k_score_tc(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__
             const uint32_t idesc = idesc_bf16_f32(kTileM, kTileN);
             uint32_t started = 0;  // bit i: accumulator i holds something
             for (int kb = 0; kb < n_kb; ++kb) {
-                const int s = kb % kTcStages;
-                if (!mbar_wait_bounded(&full[s], (kb / kTcStages) & 1, p.status)) { failed = true; break; }
+                const int s = kb % stages;
+                if (!mbar_wait_bounded(&full[s], (kb / stages) & 1, p.status)) { failed = true; break; }
                 tc_fence_after();
                 const uint32_t a_hi = smem_u32(base + size_t(s) * kStageBytes);
                 const uint32_t a_lo = a_hi + kBytesA, b_hi = a_hi + 2 * kBytesA, b_lo = b_hi + kBytesB;
@@ -262,8 +264,8 @@ k_score_tc(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__
     tc_fence_before();
     const int any_failed = __syncthreads_or(failed ? 1 : 0);
     if (any_failed && warp == 0 && lane == 0) {  // let every copy that was issued land before leaving
-        for (int s = 0; s < kTcStages && s < issued; ++s)
-            mbar_wait_bounded(&full[s], uint32_t((issued - 1 - s) / kTcStages) & 1, p.status);
+        for (int s = 0; s < stages && s < issued; ++s)
+            mbar_wait_bounded(&full[s], uint32_t((issued - 1 - s) / stages) & 1, p.status);
     }
     if (warp == 1) {
         tc_fence_after();
@@ -305,7 +307,9 @@ bool make_map(CUtensorMap* map, const __nv_bfloat16* ptr, int rows, int D, int b
 }  // namespace
 
 cudaError_t dense_setup() {
-    return cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kTcSmem));
+    const cudaError_t e = cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kTcSmem));
+    // (with a short ring the kernel shares SMs with the pooling kernel of the pipelined route)
+    return e != cudaSuccess ? e : prefer_max_smem_carveout(k_score_tc);
 }
 
 bool dense_scoring_supported(int D, int n) {
@@ -338,7 +342,8 @@ cudaError_t launch_centers_split(const float* centers, int n, int D, void* cente
 cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const float* centers, int n, int D,
                               void* scratch, int max_batch, int d_max, int which, bool sv_split_done,
                               cudaEvent_t sv_ready, void* centers_split, float** dots_out, float** dots2_out,
-                              int* status, unsigned long long* clock, cudaStream_t st, int64_t* launches) {
+                              int* status, unsigned long long* clock, int ring_stages, cudaStream_t st,
+                              int64_t* launches) {
     void *hi = nullptr, *lo = nullptr;
     dense_sv_split(scratch, max_batch, d_max, which, &hi, &lo);
     __nv_bfloat16* a_hi = static_cast<__nv_bfloat16*>(hi);
@@ -377,8 +382,10 @@ cudaError_t launch_dense_dots(const float* sv, const uint8_t* skip, int B, const
     p.split_stride = size_t(max_batch) * n;
     p.status = status;
     p.clock = clock;
+    p.stages = ring_stages >= 2 && ring_stages <= kTcStages ? ring_stages : kTcStages;
     const dim3 grid((n + kTileN - 1) / kTileN, (B + kTileM - 1) / kTileM, splits);
-    return launch_chained(k_score_tc, grid, kTcThreads, kTcSmem, st, ma_hi, ma_lo, mb_hi, mb_lo, p);
+    const size_t smem = size_t(p.stages) * kStageBytes + 1024 + 256;
+    return launch_chained(k_score_tc, grid, kTcThreads, smem, st, ma_hi, ma_lo, mb_hi, mb_lo, p);
 }
 
 }  // namespace smtm
