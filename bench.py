@@ -278,7 +278,7 @@ class OracleRun:
 
 def make_cache(smtm, w, cents, counts):
     # every workload here keeps its maps resident and alternates two carries: the library may pipeline its steps
-    # (it does where the shapes allow: NCHW maps; the NHWC workload stays on the one-kernel-per-layer route)
+    # (for NHWC maps only the first layer of a step; its later layers keep their one kernel per layer)
     flags = (smtm.FLAG_FORGET_FT if w.forgetting else 0) | smtm.FLAG_MAPS_READY
     return smtm.smtm_cache_create(w.n, w.dims, [w.tau] * w.L, cents, counts, n_streams=w.S, k_init=w.k_init,
                                   k_min=w.k_min, k_max=w.k_max, window_W=w.window_W, max_batch=w.B, flags=flags)

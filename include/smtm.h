@@ -329,7 +329,9 @@ smtm_status_t smtm_cache_get_launches(smtm_cache_t* cache, int64_t* h_out);
  *   SMTM_ROUTE_PIPELINED  on a cache created with SMTM_FLAG_MAPS_READY (small fast memories, NCHW shapes
  *                     the streaming kernels serve): the pooling of a step's first layer runs on a stream of
  *                     the cache's own, under the previous step's later layers and update; scoring follows
- *                     on the caller's stream; later layers are pooled and scored by small CTAs;
+ *                     on the caller's stream; later layers are pooled and scored by small CTAs.  With
+ *                     NHWC maps whose pixel rows are multiples of 16 bytes only the first lookup of a
+ *                     batch takes this route (later layers: SMTM_ROUTE_FUSED);
  *   SMTM_ROUTE_PIPELINED_DENSE  the same for fast memories above 64 entries, first lookup of a batch only:
  *                     the pooling runs on the cache's stream beside the previous step's decision kernel and
  *                     update, the tensor-core kernel and the decision kernel follow on the caller's stream. */

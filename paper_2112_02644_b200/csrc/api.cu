@@ -302,6 +302,9 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
     // The pipelined route: a cache whose caller keeps the maps resident and alternates its carries
     // (SMTM_FLAG_MAPS_READY), small fast memories, shapes the streaming kernels serve.
     const bool pipelined = c->maps_ready && allow_early && c->k_max <= kFusedMaxK && launch_pool_sparse_supported(e);
+    // ... or, for NHWC maps, the first lookup of a batch alone (later layers keep their one kernel per layer)
+    const bool pipelined_nhwc = c->maps_ready && allow_early && begin && c->k_max <= kFusedMaxK &&
+                                launch_encode_nhwc_vector_supported(e);
     // ... or, for a large fast memory scored on the tensor cores, the first lookup of a batch alone
     const bool dense = c->d_dense && dense_scoring_supported(a.D, a.n);
     const bool pipelined_dense = c->maps_ready && allow_early && begin && dense && launch_encode_ring_supported(e);
@@ -311,7 +314,7 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
             c->prof_step = c->d_prof_clock + c->prof_steps_used++ * size_t(2 * SMTM_PROF_KERNELS);
             // (the first two words are the stamps of the first layer's streaming kernel: on the pipelined route that
             // kernel runs on the pool stream, which clears them itself)
-            const size_t skip = ((pipelined || pipelined_dense) && begin && layer == 0) ? 2 : 0;
+            const size_t skip = ((pipelined || pipelined_dense || pipelined_nhwc) && begin && layer == 0) ? 2 : 0;
             SMTM_CUDA(cudaMemsetAsync(c->prof_step + skip, 0, (2 * SMTM_PROF_KERNELS - skip) * sizeof(unsigned long long), st));
             profiled_step_begins = true;
         }
@@ -337,6 +340,11 @@ smtm_status_t lookup_impl(smtm_cache* c, int32_t layer, const smtm_fmap_t* f, co
         if (timing) SMTM_CUDA(record_timing(timing[1], st));
         if (!whole) SMTM_CUDA(launch_score_exit(a, st, &c->launches, kPipelinedScoreThreads));
         return SMTM_OK;
+    }
+    if (pipelined_nhwc) {
+        ++c->routes[SMTM_ROUTE_PIPELINED];
+        e.clock = a.clock ? a.clock + 2 * layer : nullptr;
+        return pooled_first_lookup(c, e, a, st, timing, profiled_step_begins, false);
     }
     if (pipelined_dense) {
         ++c->routes[SMTM_ROUTE_PIPELINED_DENSE];

@@ -1292,6 +1292,11 @@ cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, in
     return launch_generic<BF16>(a, st);
 }
 
+bool launch_encode_nhwc_vector_supported(const EncodeArgs& a) {
+    if (a.layout != SMTM_NHWC || a.B <= 0) return false;
+    return a.C % (a.dtype == SMTM_F32 ? 4 : 8) == 0;
+}
+
 bool launch_encode_ring_supported(const EncodeArgs& a) {
     if (a.layout != SMTM_NCHW || a.B <= 0) return false;
     NchwParams p;

@@ -108,6 +108,8 @@ struct EncodeArgs {
 // *wrote_split (may be null) tells whether sv_hi / sv_lo were filled by the kernel that ran.
 cudaError_t launch_encode(const EncodeArgs& a, int sm_count, cudaStream_t st, int64_t* launches,
                           bool* wrote_split = nullptr);
+// Whether launch_encode serves the NHWC shape with the kernel that reads whole 16-byte pieces of a pixel's row.
+bool launch_encode_nhwc_vector_supported(const EncodeArgs& a);
 // Whether launch_encode serves the shape with the streaming ring, whose depth the ring_* fields set.
 bool launch_encode_ring_supported(const EncodeArgs& a);
 // Asks that SMs running `kernel` be configured with as much shared memory as they can have.  Kernels that

@@ -419,6 +419,48 @@ def test_maps_ready_flag_with_alternating_batches():
     smtm.smtm_cache_destroy(cache)
 
 
+def test_maps_ready_flag_with_nhwc_maps():
+    # SMTM_FLAG_MAPS_READY with NHWC maps: the first layer of a step is pooled on the library's stream beside the
+    # previous step's other kernels and scored on the caller's stream; the later layers keep their one kernel
+    # per layer.  Steps run back to back with two alternating carries; results are those of the oracle.
+    from harness import Report, compare_state
+
+    w = si.C3.scaled(B=40, S=40, T=5, k_min=4, k_max=16, k_init=8)
+    cents, counts = si.initial_centers(w)
+    tau = [w.tau] * w.L
+    mem = oracle.OracleMemory(w.n, w.dims, tau, cents, counts, w.S, w.k_init, w.k_min, w.k_max, w.window_W)
+    cache = smtm.smtm_cache_create(w.n, w.dims, tau, cents, counts, n_streams=w.S, k_init=w.k_init, k_min=w.k_min,
+                                   k_max=w.k_max, window_W=w.window_W, max_batch=w.B, flags=smtm.FLAG_MAPS_READY)
+    sid = si.stream_ids(w)
+    gbs = [smtm.Batch(cache, w.B, stream_id=sid), smtm.Batch(cache, w.B, stream_id=sid)]
+    labs = si.labels(w)
+    maps = [[si.frames(w, l, labs[t], t, device="cuda") for l in range(w.L)] for t in range(w.T)]
+    fbs = [torch.from_numpy(si.fallback_labels(w, labs[t])).cuda() for t in range(w.T)]
+    torch.cuda.synchronize()
+    for t in range(w.T):
+        gb = gbs[t % 2]
+        for l in range(w.L):
+            (smtm.smtm_lookup_exit_begin if l == 0 else smtm.smtm_lookup_exit)(
+                cache, l, smtm.Fmap(maps[t][l], w.dtype, w.layout, *si.shape4(w, l)), gb)
+        smtm.smtm_cache_update_resize(cache, gb, fbs[t])
+    torch.cuda.synchronize()
+    for t in range(w.T):
+        ob = mem.new_batch(w.B, sid)
+        for l in range(w.L):
+            mem.lookup_exit(l, maps[t][l].cpu(), w.dtype, w.layout, si.shape4(w, l), ob)
+        mem.update(ob, si.fallback_labels(w, labs[t]))
+        mem.resize()
+    last = gbs[(w.T - 1) % 2]
+    assert np.array_equal(last.done.cpu().numpy(), ob["done"])
+    assert np.array_equal(last.pred.cpu().numpy(), ob["pred"])
+    assert np.array_equal(last.exit_layer.cpu().numpy(), ob["exit_layer"])
+    compare_state(w, cache, mem, Report())
+    routes = smtm.smtm_cache_get_routes(cache)
+    assert routes[smtm.ROUTE_PIPELINED] == w.T and routes[smtm.ROUTE_FUSED] == w.T * (w.L - 1), routes
+    assert smtm.smtm_cache_status(cache) == 0
+    smtm.smtm_cache_destroy(cache)
+
+
 DENSE_GRAPH = si.Workload("dense_graph", si.BF16, si.NCHW, B=70, stages=((256, 14, 14), (512, 7, 7)), n=196, k_init=100,
                            k_min=70, k_max=196, S=1, T=8, tau=0.8, window_W=2, sigma=0.6, zipf_s=0.9, repeat_p=0.3, seed=6)
 
