@@ -75,9 +75,9 @@ __device__ __forceinline__ Top2 block_top2_keys(unsigned long long b1, unsigned 
 // in one trip: the size and the members of its fast memory, the carries, the row, the lengths and the semantic
 // vector (for its length).  Every thread keeps the two best of its own slots as 64-bit ranking keys; warps merge
 // by two warp-wide maxima, the CTA through shared memory.  With a.fresh the carry is taken as SA = 0, nobody done.
-constexpr int kFinishSlots = 8;  // slots a thread fetches per trip
+constexpr int kFinishSlots = 4;  // slots a thread fetches per trip
 
-__global__ void __launch_bounds__(kFinishThreads, 8) k_finish_dense(const LookupArgs a, const float* __restrict__ dots,
+__global__ void __launch_bounds__(kFinishThreads, 10) k_finish_dense(const LookupArgs a, const float* __restrict__ dots,
                                                                     const float* __restrict__ dots2) {
     extern __shared__ float s_row[];  // [n] dot products, then [n] lengths of the centres
     __shared__ float scratch[32];
@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(kFinishThreads, 8) k_finish_dense(const Lookup
     const float sv_len = __fsqrt_rn(nrm);
     unsigned long long a1 = 0ull, a2 = 0ull, c1 = 0ull, c2 = 0ull;  // best two cumulative / single-layer keys
     for (int j0 = 0; j0 < k; j0 += kFinishSlots * kFinishThreads) {
-        if (j0 > 0) {  // a fast memory of more than 1024 slots: one more trip per 1024
+        if (j0 > 0) {  // a fast memory of more than 512 slots: one more trip per 512
 #pragma unroll
             for (int u = 0; u < kFinishSlots; ++u) {
                 const int j = min(j0 + u * kFinishThreads + tid, a.k_max - 1);
