@@ -419,6 +419,70 @@ def test_maps_ready_flag_with_alternating_batches():
     smtm.smtm_cache_destroy(cache)
 
 
+def _run_steps_against_oracle(w, S, sid, forgetting=False, split_refresh=False):
+    """Steps of workload w on a cache of S streams with the given stream ids, library and oracle side by side;
+    decisions of every step and the state after the last one must agree."""
+    from harness import Report, compare_state
+
+    cents, counts = si.initial_centers(w)
+    tau = [w.tau] * w.L
+    mem = oracle.OracleMemory(w.n, w.dims, tau, cents, counts, S, w.k_init, w.k_min, w.k_max, w.window_W,
+                              forgetting=forgetting)
+    cache = smtm.smtm_cache_create(w.n, w.dims, tau, cents, counts, n_streams=S, k_init=w.k_init, k_min=w.k_min,
+                                   k_max=w.k_max, window_W=w.window_W, max_batch=w.B,
+                                   flags=smtm.FLAG_FORGET_FT if forgetting else 0)
+    gb = smtm.Batch(cache, w.B, stream_id=sid)
+    labs = si.labels(w)
+    for t in range(w.T):
+        maps = [si.frames(w, l, labs[t], t, device="cuda") for l in range(w.L)]
+        fb = si.fallback_labels(w, labs[t])
+        for l in range(w.L):
+            (smtm.smtm_lookup_exit_begin if l == 0 else smtm.smtm_lookup_exit)(
+                cache, l, smtm.Fmap(maps[l], w.dtype, w.layout, *si.shape4(w, l)), gb)
+        if split_refresh:
+            smtm.smtm_cache_update(cache, gb, torch.from_numpy(fb).cuda())
+            smtm.smtm_cache_resize(cache)
+        else:
+            smtm.smtm_cache_update_resize(cache, gb, torch.from_numpy(fb).cuda())
+        ob = mem.new_batch(w.B, sid)
+        for l in range(w.L):
+            mem.lookup_exit(l, maps[l].cpu(), w.dtype, w.layout, si.shape4(w, l), ob)
+        mem.update(ob, fb)
+        mem.resize()
+        torch.cuda.synchronize()
+        assert np.array_equal(gb.done.cpu().numpy(), ob["done"]), "step %d" % t
+        assert np.array_equal(gb.pred.cpu().numpy(), ob["pred"]), "step %d" % t
+        assert np.array_equal(gb.exit_layer.cpu().numpy(), ob["exit_layer"]), "step %d" % t
+    compare_state(w, cache, mem, Report())
+    members, k = smtm.smtm_cache_get_members(cache)
+    assert smtm.smtm_cache_status(cache) == 0
+    smtm.smtm_cache_destroy(cache)
+    return k
+
+
+@pytest.mark.parametrize("forgetting", [False, True], ids=["counts", "forgetting"])
+def test_several_frames_per_stream_interleaved(forgetting):
+    # Six streams whose frames are interleaved in the batch, several frames each (two streams have a single
+    # frame): Sec. 6.1 applies a stream's frames in ascending index, so each frame's position counts among
+    # its own stream's frames only.
+    w = si.C5.scaled(B=37, S=37, T=5, n=40, k_init=6, k_min=3, k_max=12)
+    S = 6
+    sid = np.array([(b * 7 + 3) % 4 for b in range(w.B)], np.int32)   # streams 0..3, interleaved
+    sid[11], sid[20] = 4, 5                                             # streams 4 and 5: one frame each
+    _run_steps_against_oracle(w, S, sid, forgetting=forgetting)
+
+
+@pytest.mark.parametrize("split_refresh", [False, True], ids=["in-update", "stand-alone"])
+def test_memory_of_six_hundred_classes_with_adaptive_size(split_refresh):
+    # A memory of 513 .. 1024 classes: the refresh ranks by a sort in registers (inside the update's tables CTA,
+    # or a thread per class in the stand-alone refresh); most classes have a zero score and follow the others in
+    # ascending id; the fast memory's size moves between its bounds (Eq. 6).
+    w = si.Workload("six_hundred", si.BF16, si.NCHW, B=48, stages=((256, 14, 14),), n=600, k_init=20, k_min=8,
+                    k_max=100, S=1, T=5, tau=0.8, window_W=2, sigma=0.6, zipf_s=1.1, repeat_p=0.3, seed=11)
+    k = _run_steps_against_oracle(w, 1, None, split_refresh=split_refresh)
+    assert w.k_min <= int(k[0]) <= w.k_max
+
+
 def test_maps_ready_flag_with_nhwc_maps():
     # SMTM_FLAG_MAPS_READY with NHWC maps: the first layer of a step is pooled on the library's stream beside the
     # previous step's other kernels and scored on the caller's stream; the later layers keep their one kernel
