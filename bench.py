@@ -652,6 +652,63 @@ def oracle_steps(w, n_steps, budget_s=None, device="cpu"):
     return run.frames, run.seconds
 
 
+def run_timeline(args):
+    """Where the kernels of consecutive steps sit in time: one CUDA graph of N steps in which every kernel stamps
+    the device clock (no events; a memset per step and stream clears the stamps, which costs each step about a
+    microsecond), replayed three times from the same memory; the last replay is printed, in microseconds from the
+    begin of the first step's first kernel."""
+    import paper_2112_02644_b200 as smtm
+
+    torch.cuda.set_device(0)
+    w = si.WORKLOADS[[k for k in si.WORKLOADS if k.startswith(args.workload)][0]]
+    N, W = args.timeline, max(args.warmup, 3)
+    res = Resident(smtm, w, W + N)
+    cents, counts = si.initial_centers(w)
+    cache = make_cache(smtm, w, cents, counts)
+    gbs = [smtm.Batch(cache, w.B, stream_id=si.stream_ids(w) if w.S > 1 else None, with_diagnostics=False) for _ in range(2)]
+    stream = torch.cuda.Stream()
+    sh = stream.cuda_stream
+    R = len(res.fmaps)
+
+    def step(t):
+        gb = gbs[t % 2]
+        smtm.smtm_lookup_exit_begin(cache, 0, res.fmaps[t % R][0], gb, sh)
+        for l in range(1, w.L):
+            smtm.smtm_lookup_exit(cache, l, res.fmaps[t % R][l], gb, sh)
+        smtm.smtm_cache_update_resize(cache, gb, res.fbs[t % R], sh)
+
+    with torch.cuda.stream(stream):
+        for t in range(W):
+            step(t)
+        stream.synchronize()
+        blob = smtm.smtm_cache_export(cache)
+        smtm.smtm_cache_profile(cache, (N + 1) * w.L, -1)   # every step, device-clock stamps alone
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for t in range(W, W + N):
+                step(t)
+        for _ in range(3):
+            smtm.smtm_cache_import(cache, blob)
+            g.replay()
+            stream.synchronize()
+    names = {}
+    for l in range(w.L):
+        names[l] = "stream_layer%d" % l
+        names[smtm.PROF_SCORE + l] = "score_layer%d" % l
+    names.update({smtm.PROF_SCORE_TC: "score_tc", smtm.PROF_FINISH_DENSE: "finish_dense", smtm.PROF_PLAN: "update_plan",
+                  smtm.PROF_CENTERS: "update_centers", smtm.PROF_TABLES: "update_tables", smtm.PROF_REFRESH: "refresh"})
+    t0, steps = None, []
+    for i in range(N):
+        b, e = smtm.smtm_cache_get_profile_timeline(cache, i)
+        if t0 is None:
+            t0 = min(int(b[k]) for k in names if int(b[k]))
+        steps.append({nm: [round((int(b[k]) - t0) / 1e3, 2), round((int(e[k]) - t0) / 1e3, 2)] for k, nm in names.items() if int(b[k])})
+    out = {"timeline_us": steps, "workload": w.name, "steps": N, "warmup": W,
+           "routes": [int(v) for v in smtm.smtm_cache_get_routes(cache)], "device_status": smtm.smtm_cache_status(cache)}
+    smtm.smtm_cache_destroy(cache)
+    return out
+
+
 def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
@@ -684,6 +741,8 @@ def main():
     ap.add_argument("--no-other-workloads", action="store_true", help="skip the short passes of c1..c4")
     ap.add_argument("--profile-every", type=int, default=PROFILE_EVERY,
                     help="every N-th step of the timed region carries timing events and device-clock stamps")
+    ap.add_argument("--timeline", type=int, default=0, metavar="N",
+                    help="print where the kernels of N consecutive steps sit in time (device clock) instead of the benchmark line")
     ap.add_argument("--rank-check", action="store_true", help="multi-rank plumbing only, on the host (gloo)")
     args = ap.parse_args()
     PROFILE_EVERY = max(1, args.profile_every)
@@ -692,6 +751,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.rank_check:
         out = rank_check(args)
+    elif args.timeline > 0:
+        out = run_timeline(args)
     else:
         out = run_reference(args) if args.impl == "reference" else run_ours(args)
     if out is not None:
