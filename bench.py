@@ -317,7 +317,7 @@ class Resident:
         return si.fallback_labels(self.w, self.labs[(t % self.R) % self.w.T])
 
 
-def measure(smtm, w, K, W, local_rank, world, verify_steps=0, graph_steps=32):
+def measure(smtm, w, K, W, local_rank, world, verify_steps=0, graph_steps=64):
     """Times steps W .. W+K-1 of workload `w` through CUDA graphs and returns the figures of the run.
     verify_steps > 0: the CPU oracle is run over steps 0 .. W+verify_steps-1 of the same maps and the exits it
     takes in steps W .. W+verify_steps-1 are compared with the library's."""
